@@ -1,0 +1,75 @@
+"""Seeded synthetic inputs shared by the oracle-side and CUDA-side tests and by bench.py.
+
+This module holds none of the method's arithmetic: it only draws numbers.  Values come from a
+counter-based generator (Philox4x32-10: value = f(seed, tensor id, element index), independent of
+how the work is split -- the property Sec. 2.1 "Random number generation" asks of every random
+draw), turned into normals by Box-Muller in float64 and rounded to the requested storage type.
+
+bf16 tensors are returned as numpy ``uint16`` bit patterns.
+"""
+import numpy as np
+
+_M0 = np.uint64(0xD2511F53)
+_M1 = np.uint64(0xCD9E8D57)
+_W0 = 0x9E3779B9
+_W1 = 0xBB67AE85
+_MASK = np.uint64(0xFFFFFFFF)
+
+
+def philox4x32_10(ctr, key):
+    """ctr: uint32 array [..., 4]; key: (k0, k1).  Returns uint32 array [..., 4]."""
+    c = [np.asarray(ctr[..., i], np.uint64) for i in range(4)]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = _M0 * c[0]
+        p1 = _M1 * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & _MASK
+        hi1, lo1 = p1 >> np.uint64(32), p1 & _MASK
+        c = [hi1 ^ c[1] ^ np.uint64(k0), lo1, hi0 ^ c[3] ^ np.uint64(k1), lo0]
+        k0 = (k0 + _W0) & 0xFFFFFFFF
+        k1 = (k1 + _W1) & 0xFFFFFFFF
+    return np.stack([x.astype(np.uint32) for x in c], axis=-1)
+
+
+def _raw(n, seed, tid):
+    """n uint32 draws for (seed, tensor id); element i comes from counter i // 4, lane i % 4."""
+    nblk = (n + 3) // 4
+    ctr = np.zeros((nblk, 4), np.uint32)
+    idx = np.arange(nblk, dtype=np.uint64)
+    ctr[:, 0] = (idx & _MASK).astype(np.uint32)
+    ctr[:, 1] = (idx >> np.uint64(32)).astype(np.uint32)
+    return philox4x32_10(ctr, (seed, tid)).reshape(-1)[:n]
+
+
+def uniform01(n, seed, tid):
+    """float64 in (0, 1)."""
+    return (_raw(n, seed, tid).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+
+
+def normal_f32(shape, std=1.0, mean=0.0, seed=0, tid=0):
+    n = int(np.prod(shape))
+    h = (n + 1) // 2
+    u = uniform01(2 * h, seed, tid)
+    r = np.sqrt(-2.0 * np.log(u[:h]))
+    z = np.concatenate([r * np.cos(2 * np.pi * u[h:]), r * np.sin(2 * np.pi * u[h:])])[:n]
+    return (mean + std * z).astype(np.float32).reshape(shape)
+
+
+def to_bf16(x):
+    """float32 -> bf16 bit patterns (uint16), round-to-nearest-even; storage conversion of inputs only."""
+    u = np.ascontiguousarray(x, np.float32).view(np.uint32).astype(np.uint64)
+    u = u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))
+    return (u >> np.uint64(16)).astype(np.uint16).reshape(np.shape(x))
+
+
+def from_bf16(h):
+    return (np.asarray(h, np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def normal_bf16(shape, std=1.0, mean=0.0, seed=0, tid=0):
+    return to_bf16(normal_f32(shape, std, mean, seed, tid))
+
+
+def randint(shape, high, seed=0, tid=0):
+    n = int(np.prod(shape))
+    return (_raw(n, seed, tid).astype(np.uint64) % np.uint64(high)).astype(np.int32).reshape(shape)

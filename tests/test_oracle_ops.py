@@ -1,0 +1,410 @@
+"""Pins for the oracle's operations against independent references: brute-force integer GEMMs,
+float64 numpy evaluations, closed forms, hand-worked elements and invariants."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+
+F = np.float32
+bf = synth.from_bf16
+
+
+def rel_err(a, b):
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+
+
+def hadamard(n):
+    i = np.arange(n)
+    pc = np.array([[bin(a & b).count("1") for b in i] for a in i])
+    return np.where(pc % 2 == 0, 1, -1).astype(np.int64)
+
+
+# ---------------------------------------------------------------- LSQ linear
+def test_weight_step_closed_form():
+    # rows of constant magnitude c give exactly 2c * c127 (two roundings); Sec. 3.1 / Sec. 4.4 formula
+    c127 = F(1 / math.sqrt(127))
+    W = np.empty((3, 256), F)
+    for r, c in enumerate((0.5, 0.015625, 2.0)):
+        W[r] = c * np.where(np.arange(256) % 3 == 0, -1, 1)
+    s = oracle.lsq_weight_scale(synth.to_bf16(W))
+    exp = np.array([F(F(2 * c) * c127) for c in (0.5, 0.015625, 2.0)], F)
+    assert np.array_equal(s, exp)
+    Wn = synth.normal_bf16((64, 2048), 0.02, seed=0, tid=1)
+    s = oracle.lsq_weight_scale(Wn)
+    ref = 2 * np.abs(bf(Wn).astype(np.float64)).mean(axis=1) / math.sqrt(127)
+    assert np.allclose(s, ref, rtol=1e-5) and abs(s.mean() - 0.002832) < 1e-4
+    st = oracle.lsq_weight_scale(Wn, per_tensor=True)
+    assert np.all(st == st[0]) and abs(st[0] - ref.mean()) < 1e-6
+    sx = oracle.lsq_act_scale_init(Wn)
+    assert sx[0] == st[0]
+
+
+def test_quantiser_hand_cases():
+    # t = 0.5, 1.5, 2.5, -0.5, 127.5, -128.5, 300 -> 0, 2, 2, 0, 127, -128, 127 (ties to even, clip)
+    t = np.array([[0.5, 1.5, 2.5, -0.5, 127.5, -128.5, 300.0, -1.5]], F)
+    q = oracle.lsq_quantize(synth.to_bf16(t), np.array([1.0], F), per_row=False)
+    assert q.tolist() == [[0, 2, 2, 0, 127, -128, 127, -2]]
+
+
+def test_int_gemm_bruteforce_and_forward():
+    M, N, K = 37, 29, 384
+    X = synth.normal_bf16((M, K), 1.0, seed=0, tid=10)
+    W = synth.normal_bf16((N, K), 0.02, seed=0, tid=11)
+    s_w = oracle.lsq_weight_scale(W)
+    s_x = oracle.lsq_act_scale_init(X)
+    Y, qX, qW = oracle.linear_fwd(X, W, s_x, s_w)
+    acc = qX.astype(np.int64) @ qW.astype(np.int64).T
+    assert np.array_equal(oracle.igemm_tn(qX, qW).astype(np.int64), acc)
+    # independent quantiser in float64: products x*(1/s) are exact in double, rint ties to even
+    inv = F(1) / s_x[0]
+    t = (bf(X).astype(np.float64) * np.float64(inv)).astype(F)
+    assert np.array_equal(qX, np.clip(np.rint(t), -128, 127).astype(np.int8))
+    # dequantise: one f32 product of the scales, one f32 product with the accumulator, one bf16 rounding
+    sc = (np.float64(s_x[0]) * s_w.astype(np.float64)).astype(F)
+    ref = synth.to_bf16((acc.astype(F).astype(np.float64) * sc[None, :].astype(np.float64)).astype(F))
+    assert np.array_equal(Y, ref)
+    # and it approximates the unquantised product
+    assert rel_err(bf(Y), bf(X).astype(np.float64) @ bf(W).astype(np.float64).T) < 0.1
+
+
+def test_hadamard_butterflies():
+    H = hadamard(128)
+    v = np.random.default_rng(0).integers(-128, 128, 128).astype(np.int32)
+    assert np.array_equal(oracle.wht128_i(v).astype(np.int64), H @ v.astype(np.int64))
+    assert np.array_equal(oracle.wht128_i(oracle.wht128_i(v)), 128 * v)       # H*H = 128 I
+    x = np.random.default_rng(1).integers(-1000, 1000, 128).astype(F)          # small integers: exact in f32
+    assert np.array_equal(oracle.wht128_f(x).astype(np.int64), H @ x.astype(np.int64))
+    assert np.array_equal(oracle.wht128_f(oracle.wht128_f(x)), 128 * x)
+
+
+def _ref_linear_bwd(dY, X, W, s_x, s_w):
+    """float64 straight-through reference with exact (unquantised-gradient) contractions."""
+    inv = F(1) / s_x[0]
+    tx = (bf(X).astype(np.float64) * np.float64(inv)).astype(F)
+    qX = np.clip(np.rint(tx), -128, 127)
+    inv_w = (F(1) / s_w).astype(F)
+    tw = (bf(W).astype(np.float64) * inv_w[:, None].astype(np.float64)).astype(F)
+    qW = np.clip(np.rint(tw), -128, 127)
+    g = bf(dY).astype(np.float64)
+    gx = g @ (qW * s_w[:, None].astype(np.float64))
+    dX = np.where((tx >= -128) & (tx <= 127), gx, 0)
+    dW = np.where((tw >= -128) & (tw <= 127), g.T @ (qX * np.float64(s_x[0])), 0)
+    phi = np.where(tx < -128, -128, np.where(tx > 127, 127, qX - tx.astype(np.float64)))
+    ds = (gx * phi).sum() / math.sqrt(X.size * 127)
+    return dX, dW, ds
+
+
+@pytest.mark.parametrize("hb", [0, 128])
+def test_linear_bwd_against_float64(hb):
+    M, N, K = 256, 256, 384
+    X = synth.normal_bf16((M, K), 1.0, seed=0, tid=20)
+    X.reshape(-1)[:5] = synth.to_bf16(np.array([40, -40, 30, -35, 50], F))   # out-of-range activations (mask)
+    W = synth.normal_bf16((N, K), 0.02, seed=0, tid=21)
+    dY = synth.normal_bf16((M, N), 0.01, seed=0, tid=22)
+    s_w = oracle.lsq_weight_scale(W)
+    s_x = oracle.lsq_act_scale_init(X)
+    dX, dW, ds = oracle.linear_bwd(dY, X, W, s_x, s_w, hb=hb)
+    rX, rW, rs = _ref_linear_bwd(dY, X, W, s_x, s_w)
+    assert rel_err(bf(dX), rX) < 0.03
+    assert rel_err(dW, rW) < 0.03
+    assert abs(ds[0] - rs) < 0.05 * abs(rs) + 1e-6
+    assert np.all(bf(dX).reshape(-1)[:5] == 0)                               # STE range mask
+
+
+def test_hadamard_modes_agree_when_quantisation_is_exact():
+    # one non-zero per 128-block, power-of-two magnitudes: rotated and unrotated operands both quantise exactly
+    M = N = K = 128
+    X = np.zeros((M, K), F); W = np.zeros((N, K), F); dY = np.zeros((M, N), F)
+    X[5, 9] = 2.0
+    W[17, 9] = 0.5
+    dY[5, 17] = 0.25
+    s_x = np.array([2.0 / 64], F); s_w = np.full(N, 0.5 / 64, F)
+    a0 = oracle.linear_bwd(synth.to_bf16(dY), synth.to_bf16(X), synth.to_bf16(W), s_x, s_w, hb=0)
+    a1 = oracle.linear_bwd(synth.to_bf16(dY), synth.to_bf16(X), synth.to_bf16(W), s_x, s_w, hb=128)
+    for u, v in zip(a0, a1):
+        assert np.array_equal(u, v)
+    assert bf(a0[0])[5, 9] == F(0.25 * 0.5) and a0[1][17, 9] == F(0.25 * 2.0)
+
+
+def test_hadamard_reduces_weight_gradient_error_on_heavy_tails():
+    # Sec. 3.2: rotation flattens gradient outliers (paper: ~5% -> ~1% at its shapes; a sanity check)
+    M, N, K = 1024, 128, 128
+    X = synth.normal_bf16((M, K), 1.0, seed=0, tid=30)
+    W = synth.normal_bf16((N, K), 0.02, seed=0, tid=31)
+    g = synth.normal_f32((M, N), 0.01, seed=0, tid=32)
+    g[::97, ::13] *= 60.0                                                      # sparse outliers
+    dY = synth.to_bf16(g)
+    s_w = oracle.lsq_weight_scale(W); s_x = oracle.lsq_act_scale_init(X)
+    _, rW, _ = _ref_linear_bwd(dY, X, W, s_x, s_w)
+    e0 = rel_err(oracle.linear_bwd(dY, X, W, s_x, s_w, hb=0)[1], rW)
+    e1 = rel_err(oracle.linear_bwd(dY, X, W, s_x, s_w, hb=128)[1], rW)
+    assert e1 < 0.5 * e0 and e1 < 0.03
+
+
+# ---------------------------------------------------------------- RMSNorm
+def test_rmsnorm_hand_row_and_float64():
+    x = np.array([[1.0, 2.0, 2.0, 4.0]], F)        # mean square = 25/4 = 6.25, eps = 0 -> rstd = 0.4 (rounded)
+    g = np.array([1.0, 0.5, 2.0, 1.0], F)
+    y, rstd = oracle.rmsnorm_fwd(x, g, eps=0.0)
+    r = F(1) / F(2.5)
+    assert rstd[0] == r
+    assert np.array_equal(y[0], np.array([F(F(1 * r) * 1), F(F(2 * r) * F(0.5)), F(F(2 * r) * 2), F(F(4 * r) * 1)], F))
+    rows, D = 33, 2048
+    x = synth.normal_f32((rows, D), seed=0, tid=40)
+    g = 1 + synth.normal_f32(D, 0.02, seed=0, tid=41)
+    dy = synth.normal_f32((rows, D), seed=0, tid=42)
+    y, rstd = oracle.rmsnorm_fwd(x, g, eps=1e-6)
+    x64, g64, dy64 = x.astype(np.float64), g.astype(np.float64), dy.astype(np.float64)
+    rs64 = 1 / np.sqrt((x64 ** 2).mean(1) + 1e-6)
+    assert np.allclose(rstd, rs64, rtol=3e-7) and np.allclose(y, x64 * rs64[:, None] * g64, rtol=1e-6, atol=1e-7)
+    dx, dg = oracle.rmsnorm_bwd(dy, x, g, rstd)
+    w = dy64 * g64; xh = x64 * rs64[:, None]
+    dx64 = rs64[:, None] * (w - xh * (w * xh).mean(1, keepdims=True))
+    assert np.allclose(dx, dx64, rtol=1e-4, atol=1e-6) and np.allclose(dg, (dy64 * xh).sum(0), rtol=1e-4, atol=1e-5)
+    # constant row c: y = gamma * sign(c) (up to rounding), gain-free variant
+    yc, _ = oracle.rmsnorm_fwd(np.full((1, 256), 3.0, F), None, eps=0.0)
+    assert np.allclose(yc, 1.0, atol=2e-7)
+    # bf16 I/O variant rounds once at the output
+    xb = synth.to_bf16(x); gb = synth.to_bf16(g)
+    yb, rb = oracle.rmsnorm_fwd(xb, gb, bf=True)
+    yf, rf = oracle.rmsnorm_fwd(bf(xb), bf(gb))
+    assert np.array_equal(yb, synth.to_bf16(yf)) and np.array_equal(rb, rf)
+
+
+# ---------------------------------------------------------------- cross-entropy
+def test_xent_closed_forms():
+    V = 50304
+    z = np.full((2, V), 3.25, F)
+    loss, lse, lm, zm, bad = oracle.xent_fwd(z, np.array([7, V - 1], np.int32))
+    logV = oracle.prim("log", [float(V)])[0]                 # S = V exactly, so loss = det_log(V) ~ log V
+    assert bad == 0 and np.all(loss == F(F(3.25) + logV) - F(3.25)) and abs(loss[0] - math.log(V)) < 2e-6
+    z = np.zeros((1, 1000), F); z[0, 5] = 100.0                # gap >= 88: every other term flushes to +0
+    loss, lse, lm, _, _ = oracle.xent_fwd(z, np.array([5], np.int32))
+    assert loss[0] == 0 and lse[0] == 100 and lm[0] == 0
+    z = np.array([[0.0, 1.0]], F)                               # V = 2 by hand: log(1 + e^-1) for target 1
+    loss, lse, _, _, _ = oracle.xent_fwd(z, np.array([1], np.int32))
+    assert abs(loss[0] - math.log1p(math.exp(-1))) < 1e-6
+    # out-of-range target: counted, row contributes zero
+    loss, _, lm, _, bad = oracle.xent_fwd(z, np.array([2], np.int32))
+    assert bad == 1 and loss[0] == 0
+
+
+def test_xent_against_float64():
+    rows, V = 16, 50304
+    z = synth.normal_f32((rows, V), 2.0, seed=0, tid=50)
+    t = synth.randint(rows, V, seed=0, tid=51)
+    loss, lse, lm, zm, _ = oracle.xent_fwd(z, t, z_weight=1e-4)
+    z64 = z.astype(np.float64)
+    lse64 = np.log(np.exp(z64 - z64.max(1, keepdims=True)).sum(1)) + z64.max(1)
+    assert np.allclose(lse, lse64, rtol=3e-7)
+    assert np.allclose(loss, lse64 - z64[np.arange(rows), t], rtol=1e-5)
+    assert abs(lm[0] - ((lse64 - z64[np.arange(rows), t]).mean() + 1e-4 * (lse64 ** 2).mean())) < 1e-5
+    dz = oracle.xent_bwd(z, t, lse, scale=1.0 / rows)
+    p = np.exp(z64 - lse64[:, None]); p[np.arange(rows), t] -= 1
+    assert np.allclose(dz, p / rows, rtol=1e-4, atol=1e-9)
+    assert np.abs(dz.astype(np.float64).sum(1)).max() < 1e-6   # softmax gradient sums to ~0 without z-loss
+    dzz = oracle.xent_bwd(z, t, lse, z_weight=1e-4, scale=1.0)
+    pz = np.exp(z64 - lse64[:, None])
+    ref = pz * (1 + 2e-4 * lse64[:, None]); ref[np.arange(rows), t] -= 1
+    assert np.allclose(dzz, ref, rtol=1e-4, atol=1e-9)
+
+
+# ---------------------------------------------------------------- attention
+def _attn_ref(qkv, B, H, S):
+    x = bf(qkv).astype(np.float64).reshape(B, S, 3, H, 128)
+    q, k, v = (x[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+    s = q @ k.transpose(0, 1, 3, 2) / math.sqrt(128)
+    s = np.where(np.tril(np.ones((S, S), bool)), s, -np.inf)
+    lse = np.log(np.exp(s - s.max(-1, keepdims=True)).sum(-1)) + s.max(-1)
+    p = np.exp(s - lse[..., None])
+    return q, k, v, p, p @ v, lse
+
+
+def test_attention_forward_pins():
+    B, H, S = 1, 2, 257                       # 257 exercises a full tile, a second full tile and a 1-key tile
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=60)
+    out, lse = oracle.attn_fwd(qkv, B, H, S)
+    q, k, v, p, o, l = _attn_ref(qkv, B, H, S)
+    o = o.transpose(0, 2, 1, 3).reshape(B * S, H * 128)
+    assert np.abs(bf(out) - o).max() < 0.02 and np.allclose(lse, l, rtol=1e-5, atol=1e-5)
+    assert np.array_equal(out[0], qkv[0, 2 * H * 128:])                       # i = 0 -> out = v_0 exactly
+    # causality: changing keys/values after position i leaves rows <= i bit-identical
+    qkv2 = qkv.copy(); qkv2[200:, H * 128:] = synth.normal_bf16((S - 200, 2 * H * 128), 1.0, seed=1, tid=61)
+    out2, lse2 = oracle.attn_fwd(qkv2, B, H, S)
+    assert np.array_equal(out2[:200], out[:200]) and np.array_equal(lse2[:, :, :200], lse[:, :, :200])
+    # q = 0 -> uniform weights, out_i ~ mean(v_0..v_i)
+    qkv3 = qkv.copy(); qkv3[:, :H * 128] = 0
+    out3, lse3 = oracle.attn_fwd(qkv3, B, H, S)
+    vm = np.cumsum(bf(qkv3[:, 2 * H * 128:]).astype(np.float64), 0) / np.arange(1, S + 1)[:, None]
+    assert np.abs(bf(out3) - vm).max() < 0.02
+    assert np.allclose(lse3[0, 0], np.log(np.arange(1, S + 1)), atol=1e-5)
+
+
+def test_attention_backward_against_float64():
+    B, H, S = 2, 1, 160
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=62)
+    dout = synth.normal_bf16((B * S, H * 128), 0.1, seed=0, tid=63)
+    out, lse = oracle.attn_fwd(qkv, B, H, S)
+    dqkv = oracle.attn_bwd(dout, qkv, out, lse, B, H, S)
+    q, k, v, p, o, _ = _attn_ref(qkv, B, H, S)
+    do = bf(dout).astype(np.float64).reshape(B, S, H, 128).transpose(0, 2, 1, 3)
+    dv = p.transpose(0, 1, 3, 2) @ do
+    dp = do @ v.transpose(0, 1, 3, 2)
+    ds = p * (dp - (do * o).sum(-1, keepdims=True)) / math.sqrt(128)
+    dq = ds @ k; dk = ds.transpose(0, 1, 3, 2) @ q
+    ref = np.stack([dq, dk, dv], 2).transpose(0, 3, 2, 1, 4).reshape(B * S, 3 * H * 128)
+    got = bf(dqkv).astype(np.float64)
+    for c in range(3):
+        sl = slice(c * H * 128, (c + 1) * H * 128)
+        assert rel_err(got[:, sl], ref[:, sl]) < 0.01
+    # causal invariance of the backward: dq rows < 100 ignore later positions' inputs
+    qkv2 = qkv.copy(); qkv2[B * S - 30:, :] = synth.normal_bf16((30, 3 * H * 128), 1.0, seed=2, tid=64)
+    out2, lse2 = oracle.attn_fwd(qkv2, B, H, S)
+    d2 = oracle.attn_bwd(dout, qkv2, out2, lse2, B, H, S)
+    assert np.array_equal(d2[:S, :], dqkv[:S, :]) and np.array_equal(d2[S:S + 130 - 0, :H * 128], dqkv[S:S + 130, :H * 128])
+
+
+# ---------------------------------------------------------------- glue
+def test_glue_ops():
+    gu = synth.normal_bf16((9, 512), 2.0, seed=0, tid=70)
+    h = oracle.swiglu_fwd(gu)
+    g, u = bf(gu[:, :256]).astype(np.float64), bf(gu[:, 256:]).astype(np.float64)
+    sg = 1 / (1 + np.exp(-g))
+    assert np.allclose(bf(h), g * sg * u, rtol=1e-2, atol=1e-3)
+    dh = synth.normal_bf16((9, 256), 1.0, seed=0, tid=71)
+    dgu = oracle.swiglu_bwd(dh, gu)
+    d = bf(dh).astype(np.float64)
+    assert np.allclose(bf(dgu[:, 256:]), d * g * sg, rtol=1e-2, atol=1e-3)
+    assert np.allclose(bf(dgu[:, :256]), d * u * sg * (1 + g * (1 - sg)), rtol=1e-2, atol=1e-3)
+    big = synth.to_bf16(np.array([[-200.0, 200.0, 1.0, 1.0]], F))             # exp overflow path: silu(-200) = -0
+    hb = bf(oracle.swiglu_fwd(big))
+    assert hb[0, 0] == 0 and hb[0, 1] == 200
+    a = synth.normal_bf16(1000, seed=0, tid=72); b = synth.normal_bf16(1000, seed=0, tid=73)
+    assert np.array_equal(oracle.residual_add(a, b), synth.to_bf16(bf(a) + bf(b)))
+    # embedding: gather, and ordered scatter-add with duplicate tokens
+    E = synth.normal_bf16((11, 8), seed=0, tid=74)
+    tok = np.array([3, 5, 3, 3, 10, 5], np.int32)
+    assert np.array_equal(oracle.embed_fwd(tok, E), E[tok])
+    dy = synth.to_bf16(np.array([[2.0 ** 24] * 8, [1.0] * 8, [1.0] * 8, [1.0] * 8, [4.0] * 8, [2.0] * 8], F))
+    dE = oracle.embed_bwd(tok, dy, 11)
+    assert np.all(dE[3] == 2.0 ** 24)            # sequential: (2^24 + 1) + 1 stays 2^24; a tree would give 2^24 + 2
+    assert np.all(dE[5] == 3) and np.all(dE[10] == 4) and np.all(dE[0] == 0)
+
+
+def test_lmhead_against_float64_and_order():
+    M, V, K = 24, 40, 256
+    Hh = synth.normal_bf16((M, K), 1.0, seed=0, tid=80)
+    W = synth.normal_bf16((V, K), 0.02, seed=0, tid=81)
+    lg = oracle.lmhead_fwd(Hh, W)
+    assert np.allclose(lg, bf(Hh).astype(np.float64) @ bf(W).astype(np.float64).T, rtol=1e-4, atol=1e-5)
+    # sequential order: python restatement of one output
+    acc = F(0)
+    for kk in range(K):
+        acc = F(acc + F(bf(Hh)[3, kk] * bf(W)[7, kk]))
+    assert lg[3, 7] == acc
+    dl = synth.normal_f32((M, V), 1e-3, seed=0, tid=82)
+    dH, dW = oracle.lmhead_bwd(dl, Hh, W)
+    g = bf(synth.to_bf16(dl)).astype(np.float64)
+    assert rel_err(bf(dH), g @ bf(W).astype(np.float64)) < 0.01
+    assert rel_err(dW, g.T @ bf(Hh).astype(np.float64)) < 1e-5
+    # chunked accumulation over tokens continues the same ordered sum
+    _, dWa = oracle.lmhead_bwd(dl[:10], Hh[:10], W)
+    _, dWb = oracle.lmhead_bwd(dl[10:], Hh[10:], W, dW=dWa)
+    assert np.array_equal(dWb, dW)
+
+
+# ---------------------------------------------------------------- reduction replay, clip, AdamW
+def test_treefold_paper_facts():
+    n = 16
+    for R in range(1, 17):
+        acc = oracle.Accum(1, 1, R, n)
+        for r in range(R):
+            acc.push(np.full(n, float(r + 1), F))
+        assert acc.stack_size == bin(R).count("1")                 # one residual entry per set bit (App. A.1)
+        out = acc.result()
+        assert np.all(out == F(F(R * (R + 1) // 2) * F(1.0 / R)))
+        if R == 8:
+            assert acc.max_resident == 4                           # App. A.1: "the fold needs at most 4"
+    # pairing order: R = 4 gives (g0+g1)+(g2+g3); R = 7 gives A + (B + C) with A = 4 replicas, B = 2, C = 1
+    acc = oracle.Accum(1, 1, 4, 1)
+    for v in (2.0 ** 24, 1.0, 1.0, 1.0):
+        acc.push(np.array([v], F))
+    assert acc.result()[0] == F(F(16777218) * F(0.25))
+    acc = oracle.Accum(1, 1, 7, 1)
+    for v in (2.0 ** 24, 0, 0, 0, 1.0, 0, 1.0):
+        acc.push(np.array([v], F))
+    assert acc.result()[0] == F(F(16777218) * F(1.0 / 7))
+    with pytest.raises(ValueError):
+        a = oracle.Accum(2, 2, 2, 1); a.push(np.zeros(1, F)); a.result()
+
+
+def test_mesh_order_and_exact_means():
+    # integer-valued gradients: every mesh gives the exact mean; the three levels use reciprocal multiplies
+    n = 1000
+    gs = [np.round(synth.normal_f32(n, 50.0, seed=0, tid=90 + i)) * 8 for i in range(8)]
+    mean = np.sum(np.array(gs, np.float64), 0) / 8
+    for mesh in ((8, 1, 1), (2, 2, 2), (1, 8, 1), (1, 1, 8), (4, 2, 1), (2, 1, 4)):
+        acc = oracle.Accum(*mesh, n)
+        for g in gs:
+            acc.push(g)
+        assert np.array_equal(acc.result().astype(np.float64), mean)
+    # non-integer data: different meshes are different summation orders (Appendix A: ~1e-11.. not bitwise)
+    gs = [synth.normal_f32(n, 1e-3, seed=0, tid=100 + i) for i in range(8)]
+    outs = []
+    for mesh in ((8, 1, 1), (2, 2, 2), (1, 1, 8)):
+        acc = oracle.Accum(*mesh, n)
+        for g in gs:
+            acc.push(g)
+        outs.append(acc.result())
+    assert not np.array_equal(outs[0], outs[2]) and np.allclose(outs[0], outs[2], rtol=1e-5, atol=1e-9)
+    # python restatement of mesh (2,2,2): ranks r = rep*2 + shard own micro-batches 2r, 2r+1
+    half = F(0.5)
+    gr = [F(F(F(0) + gs[2 * r] * half) + gs[2 * r + 1] * half) for r in range(4)]
+    inner = [F(F(gr[0] + gr[1]) * half), F(F(gr[2] + gr[3]) * half)]
+    assert np.array_equal(outs[1], F(F(inner[0] + inner[1]) * half))
+
+
+def test_grad_norm_and_clip():
+    for k in range(1, 9):
+        norm, coef = oracle.grad_norm([np.ones(4 ** k, F)], max_norm=1.0)
+        assert norm == F(2 ** k)
+        assert coef == F(1) / F(F(2 ** k) + F(1e-6))
+    g = synth.normal_f32(1 << 20, 1e-3, seed=0, tid=110)
+    norm, coef = oracle.grad_norm([g[:1000], g[1000:]], max_norm=1.0)
+    assert abs(norm - np.linalg.norm(g.astype(np.float64))) < 1e-5 and coef == F(1) / F(norm + F(1e-6)) or coef == 1
+    norm2, coef2 = oracle.grad_norm([g], max_norm=0.0)
+    assert coef2 == 1
+    assert np.array_equal(oracle.scale(g, F(0.5)), g * F(0.5))
+
+
+def test_adamw_hand_element_and_float64():
+    lr, b1, b2, eps, wd = 3e-4, 0.9, 0.95, 1e-8, 0.1
+    p = synth.to_bf16(np.array([1.0, -2.0, 0.5], F)); g = np.array([0.25, -1e-3, 0.0], F)
+    p1, m1, v1 = oracle.adamw(p, g, np.zeros(3, F), np.zeros(3, F), lr, b1, b2, eps, wd, 1)
+    # t = 1 by hand: m = (1-b1) g, v = (1-b2) g^2, bias-corrected ratio = g/|g| -> |dp| ~ lr (+ decay lr*wd*p)
+    omb1 = F(1) - F(b1); omb2 = F(1) - F(b2)
+    assert np.array_equal(m1, (omb1 * g).astype(F)) and np.array_equal(v1, (omb2 * (g * g).astype(F)).astype(F))
+    exp_p = np.array([1.0 * (1 - lr * wd) - lr, -2.0 * (1 - lr * wd) + lr, 0.5 * (1 - lr * wd)])
+    assert np.allclose(bf(p1), exp_p, rtol=2 ** -8)
+    assert bf(p1)[2] == bf(synth.to_bf16(np.array([F(0.5) * F(1 - lr * wd)], F)))[0]   # zero gradient: pure decay
+    # f32 parameters (LSQ activation steps): no rounding to bf16, no weight decay
+    pf = np.array([0.03], F)
+    p2, _, _ = oracle.adamw(pf, np.array([1e-4], F), np.zeros(1, F), np.zeros(1, F), lr, b1, b2, eps, 0.0, 1)
+    assert abs(float(p2[0]) - (0.03 - lr)) < 1e-7
+    # two steps against float64 AdamW
+    n = 4096
+    pw = synth.normal_f32(n, 0.02, seed=0, tid=120); gw = synth.normal_f32(n, 1e-3, seed=0, tid=121)
+    pb = synth.to_bf16(pw); m = np.zeros(n, F); v = np.zeros(n, F)
+    P = bf(pb).astype(np.float64); M = np.zeros(n); Vv = np.zeros(n)
+    for t in (1, 2):
+        pb, m, v = oracle.adamw(pb, gw, m, v, lr, b1, b2, eps, wd, t)
+        M = b1 * M + (1 - b1) * gw; Vv = b2 * Vv + (1 - b2) * gw.astype(np.float64) ** 2
+        P = P * (1 - lr * wd) - lr * (M / (1 - b1 ** t)) / (np.sqrt(Vv / (1 - b2 ** t)) + eps)
+        P = bf(synth.to_bf16(P.astype(F))).astype(np.float64)
+    assert np.mean(bf(pb) == P) > 0.98 and np.allclose(bf(pb), P, rtol=2 ** -7)
+    assert np.allclose(m, M, rtol=1e-5, atol=1e-12) and np.allclose(v, Vv, rtol=1e-5, atol=1e-14)
