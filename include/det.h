@@ -1,0 +1,206 @@
+/* det.h -- C-ABI of libdet: the replayed, bit-exact training-step arithmetic on B200 (sm_100a).
+ *
+ * The sequence of calls below is the normative statement of one training step of the paper's auditable
+ * regime (Sec. 2.2 "forward pass, gradient calculation, weight updates"; Sec. 6, Algorithm 1 for the
+ * gradient reduction).  Every tensor that crosses a call boundary is rounded to its declared type.
+ *
+ * Conventions for every call
+ *  - returns DET_OK (0) or a negative det_status; errors that the host can see (bad shape, misaligned
+ *    pointer, workspace too small) return before anything is launched;
+ *  - every tensor pointer is a DEVICE pointer owned by the caller, row-major and contiguous unless a
+ *    leading dimension is given; the library allocates nothing, frees nothing and keeps no pointer after
+ *    it returns.  Scratch comes from the caller's `ws` buffer of `ws_bytes` bytes (256-byte aligned),
+ *    sized by the matching det_*_ws_bytes() query;
+ *  - work is asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream), except
+ *    det_tensor_hash which synchronises that stream;
+ *  - data-dependent scalars (LSQ steps, norms, losses) are device scalars so that no call forces a sync;
+ *  - device-detected conditions (bad target index, a bounded wait that expired, a non-finite norm) are
+ *    OR-ed into *status_dev (device int, may be NULL) as DET_DEV_* bits; kernels never trap;
+ *  - floating point: IEEE binary32, round-to-nearest-even, multiply and add never fused, subnormal
+ *    inputs and results flushed to zero (Sec. 2.1).  Sums run in the fixed pairwise tree "det_sum":
+ *    level by level, adjacent elements paired, an odd last element carried up unchanged, so the tree
+ *    shape depends only on the length, never on the launch configuration.
+ *  - bf16 tensors are passed as uint16_t bit patterns.
+ */
+#ifndef DET_H
+#define DET_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t det_bf16;
+
+typedef enum {
+  DET_OK = 0,
+  DET_ERR_ARG = -1,       /* NULL pointer, negative size, inconsistent arguments */
+  DET_ERR_SHAPE = -2,     /* dimension not supported by the kernels (see each call) */
+  DET_ERR_ALIGN = -3,     /* pointer or leading dimension not 16-byte aligned */
+  DET_ERR_WORKSPACE = -4, /* ws_bytes too small */
+  DET_ERR_RANGE = -5,     /* contraction length >= 2^17 could overflow the int32 accumulator */
+  DET_ERR_CUDA = -6       /* launch or runtime error (no synchronisation beyond the stream query) */
+} det_status;
+
+/* bits OR-ed into *status_dev by kernels */
+#define DET_DEV_TARGET 1    /* cross-entropy target outside [0, V) */
+#define DET_DEV_TIMEOUT 2   /* a bounded in-kernel wait expired; outputs of that launch are undefined */
+#define DET_DEV_NONFINITE 4 /* non-finite gradient norm */
+
+typedef enum { DET_F32 = 0, DET_BF16 = 1 } det_dtype;
+
+/* library / device information: returns the number of SMs of the current device (or a negative status) */
+int det_device_sm_count(void);
+
+/* ---- primitives (test hook) ---------------------------------------------------------------------
+ * Elementwise evaluation of one primitive of Sec. 2.1 on device arrays: op 0 add, 1 sub, 2 mul, 3 div,
+ * 4 sqrt(a), 5 det_exp(a), 6 det_log(a), 7 max, 8 bf16 round trip of a, 9 unfused a*b+b.  b may be NULL
+ * for unary ops.  Lets a test compare the device arithmetic with the CPU statement of the same rule. */
+int det_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream);
+
+/* ---- order-fixed sums (Sec. 2.1 "Reduction order") ----------------------------------------------- */
+/* out[0] = det_sum_i x[i]^2 (squares == 1) or det_sum_i x[i] (squares == 0).  n >= 0. */
+size_t det_sum_ws_bytes(size_t n);
+int det_sum(const float* x, size_t n, int squares, float* out, void* ws, size_t ws_bytes, void* stream);
+
+/* Global gradient norm and clip coefficient (Sec. 3.2 "Optimizer": clip to global l2 norm 1.0).
+ * g_ptrs / n_elems are HOST arrays of ntensors device pointers / lengths in canonical parameter order.
+ * per-tensor det_sum(g^2), then det_sum over the per-tensor sums, norm = sqrt(total),
+ * coef = min(1, max_norm / (norm + 1e-6)); max_norm <= 0 gives coef = 1.  norm_out, coef_out: device. */
+size_t det_grad_norm_ws_bytes(const size_t* n_elems, int ntensors);
+int det_grad_norm(const float* const* g_ptrs, const size_t* n_elems, int ntensors, float max_norm, float* norm_out,
+                  float* coef_out, void* ws, size_t ws_bytes, void* stream, int* status_dev);
+/* g[i] *= *coef_dev, in place */
+int det_scale_inplace(float* g, size_t n, const float* coef_dev, void* stream);
+
+/* ---- LSQ int8 linear (Sec. 3.1 "int8 quantization-aware training"; Sec. 3.2 "int8 computation";
+ *      Sec. 4.4 "Quantizer Step-Size Drift": weight steps re-pinned every optimizer step) ------------- */
+/* s_w[n] = max(2 * mean_k|W[n,k]| / sqrt(127), 2^-40); per_tensor != 0 fills all N entries with the
+ * whole-tensor value.  W bf16 [N,K]; K % 8 == 0. */
+size_t det_lsq_weight_scale_ws_bytes(int N, int K);
+int det_lsq_weight_scale(const det_bf16* W, int N, int K, int per_tensor, float* s_w, void* ws, size_t ws_bytes,
+                         void* stream);
+/* s_x[0] = max(2 * mean|x| / sqrt(127), 2^-40) over n elements (LSQ initialisation of the activation step) */
+size_t det_lsq_act_scale_init_ws_bytes(size_t n);
+int det_lsq_act_scale_init(const det_bf16* X, size_t n, float* s_x, void* ws, size_t ws_bytes, void* stream);
+/* Once per optimizer step per linear: qW[n,k] = rne(clamp(W[n,k] * (1/s_w[n]), -128, 127)) (int8 [N,K]) and,
+ * for the backward, qWt_bwd int8 [K,N] = quantised (hadamard_block == 128: block-128 Walsh-Hadamard rotated
+ * along n, per-tensor absmax step s_u[0]; hadamard_block == 0: plain transpose, s_u[0] = 1) copy.
+ * N % 128 == 0, K % 128 == 0.  qWt_bwd / s_u may be NULL to skip the backward copy. */
+size_t det_lsq_quantize_weight_ws_bytes(int N, int K);
+int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int N, int K, int hadamard_block, int8_t* qW,
+                            int8_t* qWt_bwd, float* s_u, void* ws, size_t ws_bytes, void* stream);
+
+/* Forward: qX = rne(clamp(X * (1/s_x), -128, 127)) (saved to qX_save, int8 [M,K], required),
+ * acc = qX . qW^T in int32 on the tensor cores (exact), Y[m,n] = bf16(float(acc) * (s_x * s_w[n])).
+ * X bf16 [M,K], qW int8 [N,K], Y bf16 [M,N].  M % 128 == 0, N % 128 == 0, K % 128 == 0, K < 2^17. */
+int det_linear_fwd(const det_bf16* X, const int8_t* qW, const float* s_x, const float* s_w, int M, int N, int K,
+                   det_bf16* Y, int8_t* qX_save, void* stream, int* status_dev);
+/* Backward (straight-through estimator; both gradient GEMMs in int8 after a block-`hadamard_block`
+ * Walsh-Hadamard rotation along the contraction dimension, 0 = no rotation):
+ *   dX bf16 [M,K]  = mask_x ? 2^-7 s_a s_u (A_q . U_q) : 0,   A = rotate_n(dY * s_w[n]) quantised per tensor
+ *   dW f32  [N,K]  = mask_w ? 2^-7 s_g s_z s_x (G_q^T . Z_q) : 0 (overwritten), G = rotate_m(dY), Z = rotate_m(qX)
+ *   ds_x f32 [1]   = LSQ step gradient: det_sum over (m,k) of dXhat * phi, times 1/sqrt(M K 127)
+ * mask_x: -128 <= X/s_x <= 127; mask_w likewise per channel.  Same shape limits as the forward, M < 2^17. */
+size_t det_linear_bwd_ws_bytes(int M, int N, int K);
+int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, const det_bf16* W, const int8_t* qWt_bwd,
+                   const float* s_x, const float* s_w, const float* s_u, int M, int N, int K, int hadamard_block,
+                   det_bf16* dX, float* dW, float* ds_x, void* ws, size_t ws_bytes, void* stream, int* status_dev);
+/* exact int8 x int8 -> int32 contraction C[i,j] = sum_k A[i,k] B[j,k] (tcgen05); test hook for the GEMM core.
+ * I % 128 == 0, J % 128 == 0, K % 128 == 0. */
+int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream, int* status_dev);
+
+/* ---- RMSNorm (Sec. 3.1 "RMSNorm", FP32 internals) -------------------------------------------------
+ * y = (x * rstd) * gamma, rstd = 1 / sqrt(det_sum(x^2) * (1/D) + eps); gamma NULL = gain-free.
+ * io: dtype of x, y, gamma, dy, dx (DET_F32 or DET_BF16); rstd f32 [rows]; D % 8 == 0, D <= 8192. */
+int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int rows, int D, float eps, void* y, float* rstd,
+                    void* stream);
+/* dx = rstd * (w - xhat * c), w = dy*gamma, xhat = x*rstd, c = det_sum(w*xhat) * (1/D);
+ * dgamma[j] = det_sum over rows of dy[r,j] * xhat[r,j] (f32 [D], may be NULL). */
+size_t det_rmsnorm_bwd_ws_bytes(int rows, int D);
+int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void* gamma, const float* rstd, int rows, int D,
+                    void* dx, float* dgamma, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- cross-entropy with optional z-loss (Sec. 3.1 "Z-loss"; loss in FP32) ---------------------------
+ * per row: m = max z, S = det_sum exp(z - m), lse = m + log S, loss_row = lse - z[target];
+ * loss_mean[0] = det_sum(loss_row)/rows (+ z_weight * z_mean), z_mean[0] = det_sum(lse^2)/rows.
+ * A target outside [0,V) sets DET_DEV_TARGET and its row contributes zero.  V % 4 == 0. */
+size_t det_xent_ws_bytes(int rows, int V);
+int det_xent_fwd(const float* logits, const int32_t* target, int rows, int V, float z_weight, float* loss_row,
+                 float* lse, float* loss_mean, float* z_mean, void* ws, size_t ws_bytes, void* stream, int* status_dev);
+/* in place: logits[r,j] <- (p - [j == target] (+ 2 z_weight lse p)) * scale, p = exp(z - lse) */
+int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, int rows, int V, float z_weight,
+                 float scale, void* stream);
+
+/* ---- causal attention, head_dim 128 (Sec. 3.2: QK^T and softmax in higher precision; BF16 flash
+ *      backward that recomputes the weights) ----------------------------------------------------------
+ * q, k, v: bf16, row (b*S + i) of head h starts at element ld*(b*S+i) + h*128.  Online softmax over KV
+ * tiles of 128 keys in ascending order; dot products are sequential over the 128 dimensions; tile row sums
+ * are adjacent trees over the 128 slots; P is rounded to bf16 before P.V.  lse f32 [B,H,S]. */
+int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S,
+                 det_bf16* out, int ld_out, float* lse, void* stream);
+/* dq, dk, dv with leading dimension ld_d; every contraction is a sequential ascending sum from +0.
+ * ws holds the bf16 dS matrix: B*H*S*S*2 bytes + B*H*S*4 bytes. */
+size_t det_attn_bwd_ws_bytes(int B, int H, int S);
+int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,
+                 const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq, det_bf16* dk,
+                 det_bf16* dv, int ld_d, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- elementwise glue (Sec. 3.1: SwiGLU with fused gate/up projection, pre-norm residuals, embedding) */
+/* gu bf16 [rows, 2F] (gate | up), h bf16 [rows, F] = silu(gate) * up;  F % 8 == 0 */
+int det_swiglu_fwd(const det_bf16* gu, int rows, int F, det_bf16* h, void* stream);
+int det_swiglu_bwd(const det_bf16* dh, const det_bf16* gu, int rows, int F, det_bf16* dgu, void* stream);
+/* y = bf16(a + b); y may alias a or b; n % 8 == 0 */
+int det_residual_add(const det_bf16* a, const det_bf16* b, size_t n, det_bf16* y, void* stream);
+int det_embed_fwd(const int32_t* tok, int T, const det_bf16* E, int V, int D, det_bf16* y, void* stream);
+/* dE f32 [V,D] is overwritten: rows of unused tokens are zero; a row used several times is the sequential
+ * sum of its positions' gradients in ascending position, from +0.  D % 4 == 0. */
+int det_embed_bwd(const int32_t* tok, int T, const det_bf16* dy, int V, int D, float* dE, void* stream);
+
+/* ---- LM head in full precision (Sec. 3.2: excluded from quantisation) -------------------------------
+ * logits[m,n] = sequential-k f32 sum from +0 of the exact products H[m,k] W[n,k].  K % 16 == 0. */
+int det_lmhead_fwd(const det_bf16* H, const det_bf16* W, int M, int V, int K, float* logits, void* stream);
+/* dlogits is rounded to bf16 first.  dH bf16 [M,K]: sum over the vocabulary ascending.  dW f32 [V,K]: sum over
+ * tokens ascending, continuing from the value already in dW unless first_chunk != 0. */
+int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH,
+                   float* dW, int first_chunk, void* stream);
+
+/* ---- gradient accumulation = single-device replay of the data-parallel reduction
+ *      (Sec. 6, Algorithm 1; Appendix A, Algorithm 2 "TreeFold"; A.3 reciprocal-multiply averages) -------
+ * The state is a caller-owned POD; bufs holds det_grad_accum_nbufs(dp_replicate) * n floats on the device. */
+typedef struct {
+  int accum, dp_shard, dp_replicate, pushes, nstack;
+  int level[34];
+  int slot[34];
+  unsigned long long free_mask;
+  size_t n;
+  float* bufs;
+  int inner_slot, gr_slot;
+} det_accum;
+int det_grad_accum_nbufs(int dp_replicate);
+int det_grad_accum_init(det_accum* st, int accum, int dp_shard, int dp_replicate, size_t n, float* bufs);
+/* micro-batch gradients in mesh order: rank r = replica * dp_shard + shard, then k = 0..accum-1 */
+int det_grad_accum_push(det_accum* st, const float* g_microbatch, void* stream);
+/* DET_ERR_ARG unless exactly accum * dp_shard * dp_replicate pushes were made */
+int det_grad_accum_result(det_accum* st, float* g_out, void* stream);
+
+/* ---- AdamW (Sec. 3.2 "Optimizer", "Optimizer-state precision": FP32 moments, one BF16 rounding) ------- */
+typedef struct {
+  double lr, beta1, beta2, eps, weight_decay; /* weight_decay = 0 for embedding, norms and LSQ steps */
+  int step;                                   /* t >= 1 */
+} det_adamw_desc;
+/* p: bf16 (pdtype DET_BF16) or f32 (DET_F32) parameters, updated in place; g, m, v f32 */
+int det_adamw_step(const det_adamw_desc* h, int pdtype, void* p, const float* g, float* m, float* v, size_t n,
+                   void* stream);
+
+/* ---- tensor hash (Appendix B: per-step state hash, here on the device) --------------------------------
+ * SHA-256 of every 64 KiB chunk of the raw bytes on the device; root = SHA-256(chunk digests || u64le(nbytes))
+ * finished on the host.  out32_host receives 32 bytes.  Synchronises `stream`. */
+size_t det_tensor_hash_ws_bytes(size_t nbytes);
+int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -38,8 +38,21 @@ static inline float ftz(float x) {
  * has no fused instruction to pick. */
 static inline float fadd(float a, float b) { return ftz(ftz(a) + ftz(b)); }
 static inline float fsub(float a, float b) { return ftz(ftz(a) - ftz(b)); }
-static inline float fmul(float a, float b) { return ftz(ftz(a) * ftz(b)); }
-static inline float fdiv(float a, float b) { return ftz(ftz(a) / ftz(b)); }
+/* Products and quotients are flushed when their EXACT value is below 2^-126 in magnitude (tininess
+ * judged before rounding): an exact value just under the smallest normal that IEEE rounding would
+ * lift onto it is still flushed.  This is the "least permissive backend" of Sec. 2.1 "Subnormals";
+ * sums and differences that small are exact, so the two ways of judging never differ for them. */
+static inline float fmul(float a, float b) {
+  double p = (double)ftz(a) * (double)ftz(b); /* exact: 48 significant bits */
+  if (fabs(p) < 0x1p-126) return u2f((f2u(a) ^ f2u(b)) & 0x80000000u);
+  return (float)p; /* one rounding of the exact product */
+}
+static inline float fdiv(float a, float b) {
+  a = ftz(a); b = ftz(b);
+  if (b != 0.0f && a != 0.0f && !isinf(b) && !isinf(a) && fabs((double)a) < ldexp(fabs((double)b), -126))
+    return u2f((f2u(a) ^ f2u(b)) & 0x80000000u);
+  return ftz(a / b);
+}
 static inline float fsqrt(float a) { return ftz(sqrtf(ftz(a))); }
 static inline float fabs1(float a) { return u2f(f2u(ftz(a)) & 0x7fffffffu); }
 static inline float fneg(float a) { return u2f(f2u(ftz(a)) ^ 0x80000000u); }

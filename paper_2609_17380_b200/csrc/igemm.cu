@@ -1,0 +1,406 @@
+// int8 x int8 -> int32 contraction on the 5th-generation tensor cores (tcgen05), used by the three GEMMs
+// of every LSQ linear layer (Sec. 3.2 "int8 computation": forward, grad-x and grad-W all run in int8 and
+// accumulate in int32, which is exact and therefore order-free).
+//
+//   C[i,j] = sum_k A[i,k] * B[j,k]        A: int8 [I,K] row-major, B: int8 [J,K] row-major (both K-major)
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0    TMA producer: 128-byte-swizzled tiles of A (128 x 128 B) and B (BN x 128 B) into a 4-stage ring
+//   warp 1    allocates TMEM (512 columns = two BN=256 accumulators) and issues tcgen05.mma.kind::i8
+//             (M=128, N=BN, K=32 per instruction, 4 per stage); tcgen05.commit releases ring slots
+//   warps 2-5 epilogue: tcgen05.ld of the int32 accumulator (lane = row), dequantise / mask in registers,
+//             stores; overlaps with the next tile's MMAs through the second accumulator
+// Every mbarrier wait is bounded: on expiry the kernel raises DET_DEV_TIMEOUT in *status, stops issuing
+// work, lets in-flight copies land, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace det {
+
+constexpr int BM = 128;
+constexpr int BK = 128;  // bytes (= int8 elements) per stage along K
+constexpr int STAGES = 4;
+constexpr int GEMM_THREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;  // ~1 s
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait; returns false when the limit expired or another role already gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  int polls = 0;
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if ((++polls & 63) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        *abort_flag = 1;
+        or_status(status, DET_DEV_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset: 8 rows * 128 B
+  d |= (uint64_t)1 << 46;                    // descriptor version (sm_100)
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+    k_igemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, EpiParams ep, int I, int J,
+            int K, int* status) {
+  constexpr int STAGE_A = BM * BK, STAGE_B = BN * BK, STAGE_BYTES = STAGE_A + STAGE_B;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_tfull[2], bar_tempty[2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&bar_tfull[a], 1); mbar_init(&bar_tempty[a], 4); }
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  const int tiles_i = I / BM, tiles_j = J / BN;
+  const int num_tiles = tiles_i * tiles_j;
+  const int kblocks = K / BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int i0 = (tile % tiles_i) * BM, j0 = (tile / tiles_i) * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
+          uint8_t* sa = smem + stage * STAGE_BYTES;
+          tma_load_2d(sa, &tmA, kb * BK, i0, &bar_full[stage]);
+          tma_load_2d(sa + STAGE_A, &tmB, kb * BK, j0, &bar_full[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: D = S32, A = B = signed 8-bit, both K-major, N = BN, M = 128
+      constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(&bar_tempty[acc], acc_phase ^ 1u, abort_flag, status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_full[stage], phase, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + STAGE_A);
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 32; ++k4)
+            umma_i8(tmem_d, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+          umma_commit(&bar_empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(&bar_tfull[acc]);
+      }
+    }
+  } else {
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int it = 0;
+    bool ok = true;
+    float cscale = 1.0f, inv_s = 1.0f, sx = 1.0f;
+    if (EPI == EPI_FWD) sx = ep.s_x[0];
+    if (EPI == EPI_DX) {
+      const float am = __uint_as_float(ep.amax1[0]);
+      const float s_a = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
+      cscale = fmul(fmul(s_a, ep.s_u[0]), ep.rot);
+      inv_s = fdiv(1.0f, ep.s_x[0]);
+    }
+    if (EPI == EPI_DW) {
+      const float am = __uint_as_float(ep.amax1[0]);
+      const float s_g = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
+      float s_z = 1.0f;
+      if (ep.amax2) {
+        const int az = (int)ep.amax2[0];
+        s_z = (az > 0) ? fdiv(__int2float_rn(az), 127.0f) : 0.0f;
+      }
+      cscale = fmul(fmul(fmul(s_g, s_z), ep.s_x[0]), ep.rot);
+    }
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      const int i0 = (tile % tiles_i) * BM, j0 = (tile / tiles_i) * BN;
+      if (!mbar_wait(&bar_tfull[acc], acc_phase, abort_flag, status)) { ok = false; break; }
+      tc_fence_after();
+      const int row = i0 + q * 32 + lane;
+      const size_t rbase = (size_t)row * J + j0;
+      if (EPI == EPI_DW) inv_s = fdiv(1.0f, ep.s_w[row]);
+#pragma unroll 1
+      for (int h = 0; h < BN / 128; ++h) {
+      float grp[4];
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c0 = h * 128 + cc * 32;
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+        if (EPI == EPI_RAW) {
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<int32_t*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 8; ++v) o[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+        } else if (EPI == EPI_FWD) {
+          const float4* sw = reinterpret_cast<const float4*>(ep.s_w + j0 + c0);
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float4 w0 = __ldg(sw + 2 * v), w1 = __ldg(sw + 2 * v + 1);
+            float f[8];
+            f[0] = fmul(__int2float_rn((int)r[8 * v + 0]), fmul(sx, w0.x));
+            f[1] = fmul(__int2float_rn((int)r[8 * v + 1]), fmul(sx, w0.y));
+            f[2] = fmul(__int2float_rn((int)r[8 * v + 2]), fmul(sx, w0.z));
+            f[3] = fmul(__int2float_rn((int)r[8 * v + 3]), fmul(sx, w0.w));
+            f[4] = fmul(__int2float_rn((int)r[8 * v + 4]), fmul(sx, w1.x));
+            f[5] = fmul(__int2float_rn((int)r[8 * v + 5]), fmul(sx, w1.y));
+            f[6] = fmul(__int2float_rn((int)r[8 * v + 6]), fmul(sx, w1.z));
+            f[7] = fmul(__int2float_rn((int)r[8 * v + 7]), fmul(sx, w1.w));
+            o[v] = make_uint4(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]), pack_bf2(f[4], f[5]), pack_bf2(f[6], f[7]));
+          }
+        } else if (EPI == EPI_DX) {
+          const uint4* xr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+          float term[32];
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 xu = __ldg(xr + v);
+            const uint32_t xs[4] = {xu.x, xu.y, xu.z, xu.w};
+            float g[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float xv = (e & 1) ? bfhi(xs[e >> 1]) : bflo(xs[e >> 1]);
+              const float gx = fmul(__int2float_rn((int)r[8 * v + e]), cscale);
+              const float t = fmul(xv, inv_s);
+              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
+              const float phi = t < -128.0f ? -128.0f : (t > 127.0f ? 127.0f : fsub(rintf(t), t));
+              g[e] = in_range ? gx : 0.0f;
+              term[8 * v + e] = fmul(gx, phi);
+            }
+            o[v] = make_uint4(pack_bf2(g[0], g[1]), pack_bf2(g[2], g[3]), pack_bf2(g[4], g[5]), pack_bf2(g[6], g[7]));
+          }
+          // adjacent tree over this lane's 32 columns
+#pragma unroll
+          for (int w = 1; w < 32; w <<= 1)
+#pragma unroll
+            for (int e = 0; e < 32; e += 2 * w) term[e] = fadd(term[e], term[e + w]);
+          grp[cc] = term[0];
+        } else {  // EPI_DW
+          const uint4* wr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
+          float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 wu = __ldg(wr + v);
+            const uint32_t wsr[4] = {wu.x, wu.y, wu.z, wu.w};
+            float g[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float wv = (e & 1) ? bfhi(wsr[e >> 1]) : bflo(wsr[e >> 1]);
+              const float t = fmul(wv, inv_s);
+              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
+              g[e] = in_range ? fmul(__int2float_rn((int)r[8 * v + e]), cscale) : 0.0f;
+            }
+            o[2 * v] = make_float4(g[0], g[1], g[2], g[3]);
+            o[2 * v + 1] = make_float4(g[4], g[5], g[6], g[7]);
+          }
+        }
+      }
+      if (EPI == EPI_DX)
+        ep.ds_partial[(size_t)row * (J / 128) + (j0 / 128) + h] = fadd(fadd(grp[0], grp[1]), fadd(grp[2], grp[3]));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_tempty[acc]);
+    }
+  }
+
+  // teardown: everyone meets here; after a timeout give in-flight copies time to land first
+  __syncthreads();
+  if (abort_s) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+static bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t gstr[1] = {(cuuint64_t)K};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)base, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+static int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const EpiParams& ep, int I, int J, int K, int* status,
+                      cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(k_igemm<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return DET_ERR_CUDA;
+    configured = true;
+  }
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const int tiles = (I / BM) * (J / BN);
+  const int grid = tiles < sms ? tiles : sms;
+  k_igemm<BN, EPI><<<grid, GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
+  if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
+  return DET_OK;
+}
+
+int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
+                 cudaStream_t st) {
+  if (!A || !B || I <= 0 || J <= 0 || K <= 0) return DET_ERR_ARG;
+  if (I % BM || J % 128 || K % BK) return DET_ERR_SHAPE;
+  if (K >= (1 << 17)) return DET_ERR_RANGE;
+  if (!aligned16(A) || !aligned16(B)) return DET_ERR_ALIGN;
+  const int bn = (J % 256 == 0) ? 256 : 128;
+  CUtensorMap ta, tb;
+  if (!make_map(&ta, A, I, K, BM) || !make_map(&tb, B, J, K, bn)) return DET_ERR_CUDA;
+#define DET_GEMM_CASE(E)                                                     \
+  case E:                                                                    \
+    return bn == 256 ? launch_one<256, E>(ta, tb, ep, I, J, K, status, st)   \
+                     : launch_one<128, E>(ta, tb, ep, I, J, K, status, st);
+  switch (epi) {
+    DET_GEMM_CASE(EPI_RAW)
+    DET_GEMM_CASE(EPI_FWD)
+    DET_GEMM_CASE(EPI_DX)
+    DET_GEMM_CASE(EPI_DW)
+  }
+#undef DET_GEMM_CASE
+  return DET_ERR_ARG;
+}
+
+}  // namespace det
+
+using namespace det;
+
+extern "C" int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream,
+                            int* status_dev) {
+  if (!C) return DET_ERR_ARG;
+  if (!aligned16(C)) return DET_ERR_ALIGN;
+  EpiParams ep = {};
+  ep.out = C;
+  return igemm_launch(EPI_RAW, A, B, I, J, K, ep, status_dev, (cudaStream_t)stream);
+}

@@ -1,0 +1,30 @@
+// Host-side helpers shared between the translation units of libdet.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace det {
+// floats of scratch the multi-level tree sum needs for n elements
+size_t sum_ws_floats(size_t n);
+// out[0] = det_sum(x[0..n)) (squares: of x^2); launches on st, scratch in ws (sum_ws_floats(n) floats)
+int sum_launch(const float* x, size_t n, int squares, float* out, float* ws, cudaStream_t st);
+
+// Epilogue descriptions.  All data-dependent scalars are read from device memory.
+enum { EPI_RAW = 0, EPI_FWD = 1, EPI_DX = 2, EPI_DW = 3 };
+struct EpiParams {
+  void* out;              // RAW: int32 [I,J]; FWD: bf16 [I,J]; DX: bf16 [I,J]; DW: f32 [I,J]
+  const float* s_x;       // FWD, DX, DW: activation step (device scalar)
+  const float* s_w;       // FWD: per column j; DW: per row i
+  const uint32_t* amax1;  // DX: float bits of absmax(A); DW: float bits of absmax(G)
+  const uint32_t* amax2;  // DW: int absmax(Z) (NULL: scale 1)
+  const float* s_u;       // DX: step of the rotated weights
+  const uint16_t* ref;    // DX: X bf16 [I,J]; DW: W bf16 [I,J] (range masks)
+  float rot;              // 2^-7 with rotation, 1 without
+  float* ds_partial;      // DX: [I, J/128] partial sums of dXhat * phi
+};
+
+// C[i,j] = sum_k A[i,k] B[j,k] on the tensor cores with the chosen epilogue; host-side checks included
+int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
+                 cudaStream_t st);
+}  // namespace det

@@ -1,0 +1,393 @@
+// LSQ int8 linear layer around the tensor-core GEMM: step sizes, quantisers, Walsh-Hadamard operand
+// preparation for the two gradient GEMMs, and the det_linear_fwd / det_linear_bwd entry points
+// (Sec. 3.1 "int8 quantization-aware training", Sec. 3.2 "int8 computation", Sec. 4.4 step re-pin).
+#include "common.cuh"
+#include "internal.h"
+
+namespace det {
+
+#define C127 0x1.6b7612p-4f
+
+__device__ __forceinline__ int8_t quant1(float v, float inv_s) {
+  float t = fminf(fmaxf(fmul(v, inv_s), -128.0f), 127.0f);
+  return (int8_t)__float2int_rn(t);
+}
+__device__ __forceinline__ void unpack8u(const uint4& u, float v[8]) {
+  v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
+  v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
+}
+
+// ---- step sizes -------------------------------------------------------------------------------
+// per output channel: one warp per row of W, K <= 8192
+__global__ void __launch_bounds__(256) k_wscale_rows(const uint16_t* __restrict__ W, int N, int K, float invK,
+                                                     float* __restrict__ s_w) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= N) return;
+  const int nl = (K + 255) >> 8;
+  float mine = 0.0f;
+  for (int j = 0; j < nl; ++j) {
+    const int e0 = j * 256 + lane * 8;
+    float v[8];
+    if (e0 < K) {
+      unpack8u(*reinterpret_cast<const uint4*>(W + (size_t)row * K + e0), v);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[t] = fabsf(v[t]);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[t] = 0.0f;
+    }
+    float leaf = warp_tree(tree8_full(v), (long long)j * 256, 8, K);
+    if (lane == j) mine = leaf;
+  }
+  float s = warp_tree(mine, 0, 256, K);
+  s = fmaxf(fmul(fmul(2.0f, fmul(s, invK)), C127), 0x1p-40f);
+  if (lane == 0) s_w[row] = s;
+}
+
+// chunk sums of |x| over a flat bf16 tensor (chunk = 16384 elements), same tree as det_sum
+__global__ void __launch_bounds__(256) k_abs_chunk(const uint16_t* __restrict__ x, long long n, float* __restrict__ partial) {
+  __shared__ float wsum[8];
+  const long long base = (long long)blockIdx.x * 16384;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float s[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const long long lf = base + (warp * 8 + j) * 256;
+    const long long e0 = lf + lane * 8;
+    float v[8];
+    if (e0 + 8 <= n) {
+      unpack8u(*reinterpret_cast<const uint4*>(x + e0), v);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[t] = (e0 + t < n) ? bf2f(x[e0 + t]) : 0.0f;
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) v[t] = fabsf(v[t]);
+    s[j] = warp_tree(tree8(v, e0, n), lf, 8, n);
+  }
+  float r = reg_tree<8>(s, base + (long long)warp * 2048, 256, n);
+  if (lane == 0) wsum[warp] = r;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = wsum[j];
+    partial[blockIdx.x] = reg_tree<8>(w, base, 2048, n);
+  }
+}
+__global__ void k_scale_finish(const float* sum, float inv_n, float* out, int count) {
+  const float s = fmaxf(fmul(fmul(2.0f, fmul(sum[0], inv_n)), C127), 0x1p-40f);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x) out[i] = s;
+}
+
+// ---- quantisers ---------------------------------------------------------------------------------
+// rows x cols bf16 -> int8, step per row (per_row) or one step for the tensor; cols % 16 == 0
+__global__ void __launch_bounds__(256) k_quantize(const uint16_t* __restrict__ X, size_t n16, int cols16,
+                                                  const float* __restrict__ s, int per_row, int8_t* __restrict__ q) {
+  size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n16) return;
+  const float inv = fdiv(1.0f, s[per_row ? (i / cols16) : 0]);
+  const uint4* p = reinterpret_cast<const uint4*>(X) + 2 * i;
+  float a[8], b[8];
+  unpack8u(__ldg(p), a);
+  unpack8u(__ldg(p + 1), b);
+  uint32_t o[4];
+#pragma unroll
+  for (int w = 0; w < 2; ++w) {
+    o[w] = ((uint32_t)(uint8_t)quant1(a[4 * w], inv)) | ((uint32_t)(uint8_t)quant1(a[4 * w + 1], inv) << 8) |
+           ((uint32_t)(uint8_t)quant1(a[4 * w + 2], inv) << 16) | ((uint32_t)(uint8_t)quant1(a[4 * w + 3], inv) << 24);
+    o[2 + w] = ((uint32_t)(uint8_t)quant1(b[4 * w], inv)) | ((uint32_t)(uint8_t)quant1(b[4 * w + 1], inv) << 8) |
+               ((uint32_t)(uint8_t)quant1(b[4 * w + 2], inv) << 16) | ((uint32_t)(uint8_t)quant1(b[4 * w + 3], inv) << 24);
+  }
+  reinterpret_cast<uint4*>(q)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// ---- Walsh-Hadamard operand preparation -----------------------------------------------------------
+// Unnormalised butterflies, stages h = 1..64, (a, b) -> (a + b, a - b) for index pairs (i, i + h).
+
+// (1) rotation along the row (contiguous) direction: A = rotate_n(dY[m,n] * s_w[n]).
+//     A warp owns one 128-element block: a lane holds 4 adjacent elements (stages 1, 2 in registers,
+//     stages 4..64 by shuffles).  PASS 0 records the absmax, PASS 1 quantises.
+template <int PASS, bool ROT>
+__global__ void __launch_bounds__(256) k_rot_rows(const uint16_t* __restrict__ dY, const float* __restrict__ s_w, int M,
+                                                  int N, uint32_t* __restrict__ amax, int8_t* __restrict__ Aq) {
+  const int lane = threadIdx.x & 31;
+  const size_t blk = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const size_t nblk = (size_t)M * (N / 128);
+  float local = 0.0f;
+  if (blk < nblk) {
+    const size_t m = blk / (N / 128);
+    const int n0 = (int)(blk % (N / 128)) * 128 + lane * 4;
+    uint2 u = __ldg(reinterpret_cast<const uint2*>(dY + m * N + n0));
+    float4 w = __ldg(reinterpret_cast<const float4*>(s_w + n0));
+    float v[4] = {fmul(bflo(u.x), w.x), fmul(bfhi(u.x), w.y), fmul(bflo(u.y), w.z), fmul(bfhi(u.y), w.w)};
+    if (ROT) {
+      float a0 = fadd(v[0], v[1]), a1 = fsub(v[0], v[1]), a2 = fadd(v[2], v[3]), a3 = fsub(v[2], v[3]);
+      v[0] = fadd(a0, a2); v[2] = fsub(a0, a2); v[1] = fadd(a1, a3); v[3] = fsub(a1, a3);
+#pragma unroll
+      for (int hl = 1; hl < 32; hl <<= 1) {
+        const bool upper = lane & hl;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float o = __shfl_xor_sync(0xffffffffu, v[e], hl);
+          v[e] = upper ? fsub(o, v[e]) : fadd(v[e], o);
+        }
+      }
+    }
+    if (PASS == 0) {
+      local = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+    } else {
+      const float am = __uint_as_float(amax[0]);
+      const float inv = (am > 0.0f) ? fdiv(127.0f, am) : 0.0f;
+      uint32_t o = ((uint32_t)(uint8_t)quant1(v[0], inv)) | ((uint32_t)(uint8_t)quant1(v[1], inv) << 8) |
+                   ((uint32_t)(uint8_t)quant1(v[2], inv) << 16) | ((uint32_t)(uint8_t)quant1(v[3], inv) << 24);
+      *reinterpret_cast<uint32_t*>(Aq + m * N + n0) = o;
+    }
+  }
+  if (PASS == 0) {
+#pragma unroll
+    for (int w = 16; w; w >>= 1) local = fmaxf(local, __shfl_xor_sync(0xffffffffu, local, w));
+    if (lane == 0 && local > 0.0f) atomicMax(amax, __float_as_uint(local));  // non-negative floats order as uints
+  }
+}
+
+// (2) rotation along the row-index (strided) direction with a transposed int8 result:
+//     in [R, C] (bf16 for G = dY, int8 for Z = qX and U = qW)  ->  out int8 [C, R],
+//     out[c, r] = quantise(rotate_r(in[:, c]))[r].  A CTA owns a tile of 128 rows x 64 columns in shared
+//     memory; each butterfly stage touches disjoint pairs, so the per-element rounding order is fixed.
+template <typename TIN, int PASS, bool ROT>
+__global__ void __launch_bounds__(256) k_rot_cols(const TIN* __restrict__ in, int R, int C, uint32_t* __restrict__ amax,
+                                                  int8_t* __restrict__ outT) {
+  constexpr bool ISF = (sizeof(TIN) == 2);
+  constexpr int TC = 64;
+  __shared__ float tile[128][TC + 1];  // int path stores the int32 bit pattern
+  int* itile = reinterpret_cast<int*>(&tile[0][0]);
+  const int r0 = blockIdx.y * 128, c0 = blockIdx.x * TC;
+  // load: 128 rows x 64 cols; thread t reads 4 adjacent columns of 8 rows
+  for (int i = threadIdx.x; i < 128 * (TC / 4); i += 256) {
+    const int r = i / (TC / 4), c = (i % (TC / 4)) * 4;
+    if (ISF) {
+      uint2 u = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(in) + (size_t)(r0 + r) * C + c0 + c));
+      tile[r][c] = bflo(u.x); tile[r][c + 1] = bfhi(u.x); tile[r][c + 2] = bflo(u.y); tile[r][c + 3] = bfhi(u.y);
+    } else {
+      uint32_t u = __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(in) + (size_t)(r0 + r) * C + c0 + c));
+#pragma unroll
+      for (int e = 0; e < 4; ++e) itile[r * (TC + 1) + c + e] = (int)(int8_t)(u >> (8 * e));
+    }
+  }
+  __syncthreads();
+  if (ROT) {
+    for (int h = 1; h < 128; h <<= 1) {
+      for (int i = threadIdx.x; i < 64 * TC; i += 256) {
+        const int c = i % TC, p = i / TC;                 // p-th pair of this stage
+        const int lo = ((p & ~(h - 1)) << 1) | (p & (h - 1));
+        if (ISF) {
+          float a = tile[lo][c], b = tile[lo + h][c];
+          tile[lo][c] = fadd(a, b); tile[lo + h][c] = fsub(a, b);
+        } else {
+          int a = itile[lo * (TC + 1) + c], b = itile[(lo + h) * (TC + 1) + c];
+          itile[lo * (TC + 1) + c] = a + b; itile[(lo + h) * (TC + 1) + c] = a - b;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (PASS == 0) {
+    uint32_t local = 0;
+    for (int i = threadIdx.x; i < 128 * TC; i += 256) {
+      const int r = i / TC, c = i % TC;
+      if (ISF) local = max(local, __float_as_uint(fabsf(tile[r][c])));
+      else local = max(local, (uint32_t)abs(itile[r * (TC + 1) + c]));
+    }
+#pragma unroll
+    for (int w = 16; w; w >>= 1) local = max(local, __shfl_xor_sync(0xffffffffu, local, w));
+    if ((threadIdx.x & 31) == 0 && local) atomicMax(amax, local);
+  } else {
+    float inv;
+    if (ISF) {
+      const float am = __uint_as_float(amax[0]);
+      inv = (am > 0.0f) ? fdiv(127.0f, am) : 0.0f;
+    } else {
+      const int am = (int)amax[0];
+      inv = (am > 0) ? fdiv(127.0f, __int2float_rn(am)) : 0.0f;
+    }
+    // out[c0 + c, r0 .. r0+127]: thread writes 4 adjacent r (one 32-bit store); 32 threads cover a column
+    for (int i = threadIdx.x; i < TC * 32; i += 256) {
+      const int c = i / 32, r = (i % 32) * 4;
+      uint32_t o = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        int8_t qv;
+        if (ISF) qv = quant1(tile[r + e][c], inv);
+        else if (ROT) qv = quant1(__int2float_rn(itile[(r + e) * (TC + 1) + c]), inv);
+        else qv = (int8_t)itile[(r + e) * (TC + 1) + c];
+        o |= ((uint32_t)(uint8_t)qv) << (8 * e);
+      }
+      *reinterpret_cast<uint32_t*>(outT + (size_t)(c0 + c) * R + r0 + r) = o;
+    }
+  }
+}
+
+__global__ void k_su_finish(const uint32_t* amax, int rotated, float* s_u) {
+  if (!rotated) { s_u[0] = 1.0f; return; }
+  const int am = (int)amax[0];
+  s_u[0] = (am > 0) ? fdiv(__int2float_rn(am), 127.0f) : 0.0f;
+}
+__global__ void k_dsx_finish(const float* sum, float gs, float* ds_x) { ds_x[0] = fmul(gs, sum[0]); }
+
+}  // namespace det
+
+using namespace det;
+
+extern "C" size_t det_lsq_weight_scale_ws_bytes(int N, int K) {
+  size_t n = (size_t)N * K;
+  size_t c = (n + 16383) / 16384;
+  return (align_up(c, 64) + 64 + sum_ws_floats(c)) * sizeof(float);
+}
+static int abs_mean_scale(const det_bf16* X, size_t n, float* out, int count, float* ws, cudaStream_t st) {
+  const size_t c = (n + 16383) / 16384;
+  float* partial = ws;
+  float* total = partial + align_up(c, 64);
+  float* scratch = total + 64;
+  k_abs_chunk<<<(unsigned)c, 256, 0, st>>>(X, (long long)n, partial);
+  sum_launch(partial, c, 0, total, scratch, st);
+  k_scale_finish<<<(count + 255) / 256 < 64 ? (count + 255) / 256 : 64, 256, 0, st>>>(total, (float)(1.0 / (double)n), out, count);
+  return DET_OK;
+}
+extern "C" int det_lsq_weight_scale(const det_bf16* W, int N, int K, int per_tensor, float* s_w, void* ws,
+                                    size_t ws_bytes, void* stream) {
+  if (!W || !s_w || N <= 0 || K <= 0) return DET_ERR_ARG;
+  if (K % 8 || (!per_tensor && K > 8192)) return DET_ERR_SHAPE;
+  if (!aligned16(W)) return DET_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (per_tensor) {
+    if (!ws || ws_bytes < det_lsq_weight_scale_ws_bytes(N, K)) return DET_ERR_WORKSPACE;
+    abs_mean_scale(W, (size_t)N * K, s_w, N, (float*)ws, st);
+  } else {
+    k_wscale_rows<<<(N + 7) / 8, 256, 0, st>>>(W, N, K, (float)(1.0 / (double)K), s_w);
+  }
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+extern "C" size_t det_lsq_act_scale_init_ws_bytes(size_t n) { return det_lsq_weight_scale_ws_bytes(1, (int)1) + ((n + 16383) / 16384 + 128) * 2 * sizeof(float); }
+extern "C" int det_lsq_act_scale_init(const det_bf16* X, size_t n, float* s_x, void* ws, size_t ws_bytes, void* stream) {
+  if (!X || !s_x || n == 0) return DET_ERR_ARG;
+  if (!aligned16(X)) return DET_ERR_ALIGN;
+  if (!ws || ws_bytes < det_lsq_act_scale_init_ws_bytes(n)) return DET_ERR_WORKSPACE;
+  abs_mean_scale(X, n, s_x, 1, (float*)ws, (cudaStream_t)stream);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" size_t det_lsq_quantize_weight_ws_bytes(int N, int K) { (void)N; (void)K; return 256; }
+extern "C" int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int N, int K, int hadamard_block, int8_t* qW,
+                                       int8_t* qWt_bwd, float* s_u, void* ws, size_t ws_bytes, void* stream) {
+  if (!W || !s_w || !qW || N <= 0 || K <= 0 || (qWt_bwd && !s_u)) return DET_ERR_ARG;
+  if (N % 128 || K % 128 || (hadamard_block != 0 && hadamard_block != 128)) return DET_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(qW) || (qWt_bwd && !aligned16(qWt_bwd))) return DET_ERR_ALIGN;
+  if (qWt_bwd && (!ws || ws_bytes < 256)) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t n16 = (size_t)N * K / 16;
+  k_quantize<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(W, n16, K / 16, s_w, 1, qW);
+  if (qWt_bwd) {
+    uint32_t* amax = (uint32_t*)ws;
+    cudaMemsetAsync(amax, 0, 256, st);
+    dim3 grid(K / 64, N / 128);
+    if (hadamard_block) {
+      k_rot_cols<int8_t, 0, true><<<grid, 256, 0, st>>>(qW, N, K, amax, nullptr);
+      k_rot_cols<int8_t, 1, true><<<grid, 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+    } else {
+      k_rot_cols<int8_t, 1, false><<<grid, 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+    }
+    k_su_finish<<<1, 1, 0, st>>>(amax, hadamard_block != 0, s_u);
+  }
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" int det_linear_fwd(const det_bf16* X, const int8_t* qW, const float* s_x, const float* s_w, int M, int N, int K,
+                              det_bf16* Y, int8_t* qX_save, void* stream, int* status_dev) {
+  if (!X || !qW || !s_x || !s_w || !Y || !qX_save || M <= 0 || N <= 0 || K <= 0) return DET_ERR_ARG;
+  if (M % 128 || N % 128 || K % 128) return DET_ERR_SHAPE;
+  if (K >= (1 << 17)) return DET_ERR_RANGE;
+  if (!aligned16(X) || !aligned16(qW) || !aligned16(Y) || !aligned16(qX_save) || !aligned16(s_w)) return DET_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t n16 = (size_t)M * K / 16;
+  k_quantize<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(X, n16, K / 16, s_x, 0, qX_save);
+  DET_CHECK_LAUNCH();
+  EpiParams ep = {};
+  ep.out = Y; ep.s_x = s_x; ep.s_w = s_w;
+  return igemm_launch(EPI_FWD, qX_save, qW, M, N, K, ep, status_dev, st);
+}
+
+static size_t bwd_ws_layout(int M, int N, int K, size_t* oA, size_t* oG, size_t* oZ, size_t* oP, size_t* oS) {
+  size_t off = 256;
+  *oA = off; off += align_up((size_t)M * N, 256);
+  *oG = off; off += align_up((size_t)M * N, 256);
+  *oZ = off; off += align_up((size_t)M * K, 256);
+  const size_t np = (size_t)M * (K / 128);
+  *oP = off; off += align_up(np * sizeof(float), 256);
+  *oS = off; off += align_up((sum_ws_floats(np) + 64) * sizeof(float), 256);
+  return off;
+}
+extern "C" size_t det_linear_bwd_ws_bytes(int M, int N, int K) {
+  size_t a, g, z, p, s;
+  return bwd_ws_layout(M, N, K, &a, &g, &z, &p, &s);
+}
+extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, const det_bf16* W,
+                              const int8_t* qWt_bwd, const float* s_x, const float* s_w, const float* s_u, int M, int N,
+                              int K, int hadamard_block, det_bf16* dX, float* dW, float* ds_x, void* ws, size_t ws_bytes,
+                              void* stream, int* status_dev) {
+  if (!dY || !X || !qX || !W || !qWt_bwd || !s_x || !s_w || !s_u || !dX || !dW || !ds_x || M <= 0 || N <= 0 || K <= 0)
+    return DET_ERR_ARG;
+  if (M % 128 || N % 128 || K % 128 || (hadamard_block != 0 && hadamard_block != 128)) return DET_ERR_SHAPE;
+  if (K >= (1 << 17) || N >= (1 << 17) || M >= (1 << 17)) return DET_ERR_RANGE;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(qX) || !aligned16(W) || !aligned16(qWt_bwd) || !aligned16(dX) ||
+      !aligned16(dW) || !aligned16(s_w) || !aligned16(ws))
+    return DET_ERR_ALIGN;
+  size_t oA, oG, oZ, oP, oS;
+  if (!ws || ws_bytes < bwd_ws_layout(M, N, K, &oA, &oG, &oZ, &oP, &oS)) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* base = (uint8_t*)ws;
+  uint32_t* amax = (uint32_t*)base;  // [0] A (float bits), [1] G (float bits), [2] Z (int)
+  int8_t* Aq = (int8_t*)(base + oA);
+  int8_t* GqT = (int8_t*)(base + oG);
+  int8_t* ZqT = (int8_t*)(base + oZ);
+  float* partial = (float*)(base + oP);
+  float* sscr = (float*)(base + oS);
+  const bool rot = hadamard_block != 0;
+  cudaMemsetAsync(amax, 0, 256, st);
+  const size_t nblk = (size_t)M * (N / 128);
+  const unsigned g1 = (unsigned)((nblk + 7) / 8);
+  dim3 gG(N / 64, M / 128), gZ(K / 64, M / 128);
+  if (rot) {
+    k_rot_rows<0, true><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
+    k_rot_cols<uint16_t, 0, true><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rot_cols<int8_t, 0, true><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, nullptr);
+    k_rot_rows<1, true><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
+    k_rot_cols<uint16_t, 1, true><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rot_cols<int8_t, 1, true><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+  } else {
+    k_rot_rows<0, false><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
+    k_rot_cols<uint16_t, 0, false><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rot_rows<1, false><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
+    k_rot_cols<uint16_t, 1, false><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rot_cols<int8_t, 1, false><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+  }
+  DET_CHECK_LAUNCH();
+  const float rotf = rot ? 0x1p-7f : 1.0f;
+  // grad wrt x: [M,K] = A_q [M,N] . (U_q^T [K,N])^T
+  EpiParams ex = {};
+  ex.out = dX; ex.s_x = s_x; ex.amax1 = amax + 0; ex.s_u = s_u; ex.ref = X; ex.rot = rotf; ex.ds_partial = partial;
+  int rc = igemm_launch(EPI_DX, Aq, qWt_bwd, M, K, N, ex, status_dev, st);
+  if (rc != DET_OK) return rc;
+  const size_t np = (size_t)M * (K / 128);
+  sum_launch(partial, np, 0, sscr, sscr + 64, st);
+  k_dsx_finish<<<1, 1, 0, st>>>(sscr, (float)(1.0 / sqrt((double)M * (double)K * 127.0)), ds_x);
+  DET_CHECK_LAUNCH();
+  // grad wrt W: [N,K] = G_q^T [N,M] . (Z_q^T [K,M])^T
+  EpiParams ew = {};
+  ew.out = dW; ew.s_x = s_x; ew.s_w = s_w; ew.amax1 = amax + 1; ew.amax2 = rot ? amax + 2 : nullptr; ew.ref = W; ew.rot = rotf;
+  return igemm_launch(EPI_DW, GqT, ZqT, N, K, M, ew, status_dev, st);
+}

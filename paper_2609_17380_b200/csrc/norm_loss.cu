@@ -1,0 +1,396 @@
+// RMSNorm forward/backward and cross-entropy (+ z-loss) forward/backward: HBM-bound kernels whose
+// reductions are the fixed pairwise tree with 256-element leaves (a lane owns 8 adjacent elements,
+// a warp owns a leaf).
+#include "common.cuh"
+#include "internal.h"
+
+namespace det {
+
+template <bool BF>
+__device__ __forceinline__ void load8(const void* p, size_t idx, float v[8]) {
+  if (BF) {
+    uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(p) + idx);
+    v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
+    v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
+  } else {
+    const float4* q = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + idx);
+    float4 a = q[0], b = q[1];
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+}
+template <bool BF>
+__device__ __forceinline__ void store8(void* p, size_t idx, const float v[8]) {
+  if (BF) {
+    uint4 u;
+    u.x = pack_bf2(v[0], v[1]); u.y = pack_bf2(v[2], v[3]); u.z = pack_bf2(v[4], v[5]); u.w = pack_bf2(v[6], v[7]);
+    *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p) + idx) = u;
+  } else {
+    float4* q = reinterpret_cast<float4*>(reinterpret_cast<float*>(p) + idx);
+    q[0] = make_float4(v[0], v[1], v[2], v[3]);
+    q[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// RMSNorm.  One warp per row; the row (up to 32 leaves) is held in registers between the reduction
+// and the normalisation when it has at most 8 leaves (D <= 2048), else it is read again.
+// ------------------------------------------------------------------------------------------------
+template <bool BF, int NL>  // NL = leaves held in registers (0: re-read)
+__global__ void __launch_bounds__(256) k_rmsnorm_fwd(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
+                                                     int D, float eps, float invD, void* __restrict__ y,
+                                                     float* __restrict__ rstd) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= rows) return;
+  const size_t rb = (size_t)row * D;
+  const int nl = (D + 255) >> 8;
+  float keep[NL > 0 ? NL : 1][8];
+  float mine = 0.0f;
+#pragma unroll
+  for (int j = 0; j < (NL > 0 ? NL : 32); ++j) {
+    if (j >= nl) break;
+    const int e0 = j * 256 + lane * 8;
+    float v[8], sq[8];
+    if (e0 < D) load8<BF>(x, rb + e0, v);
+    else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[t] = 0.0f;
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) sq[t] = fmul(v[t], v[t]);
+    if (NL > 0) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) keep[j][t] = v[t];
+    }
+    float leaf = warp_tree(tree8_full(sq), (long long)j * 256, 8, D);
+    if (lane == j) mine = leaf;
+  }
+  float ss = warp_tree(mine, 0, 256, D);
+  float rs = fdiv(1.0f, fsqrt(fadd(fmul(ss, invD), eps)));
+  if (lane == 0) rstd[row] = rs;
+#pragma unroll
+  for (int j = 0; j < (NL > 0 ? NL : 32); ++j) {
+    if (j >= nl) break;
+    const int e0 = j * 256 + lane * 8;
+    if (e0 >= D) continue;
+    float v[8], o[8];
+    if (NL > 0) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) v[t] = keep[j][t];
+    } else {
+      load8<BF>(x, rb + e0, v);
+    }
+    if (gamma) {
+      float g[8];
+      load8<BF>(gamma, e0, g);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = fmul(fmul(v[t], rs), g[t]);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = fmul(v[t], rs);
+    }
+    store8<BF>(y, rb + e0, o);
+  }
+}
+
+template <bool BF, int NL>
+__global__ void __launch_bounds__(256) k_rmsnorm_bwd(const void* __restrict__ dy, const void* __restrict__ x,
+                                                     const void* __restrict__ gamma, const float* __restrict__ rstd,
+                                                     int rows, int D, float invD, void* __restrict__ dx) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= rows) return;
+  const size_t rb = (size_t)row * D;
+  const int nl = (D + 255) >> 8;
+  const float rs = rstd[row];
+  float kw[NL > 0 ? NL : 1][8], kx[NL > 0 ? NL : 1][8];
+  float mine = 0.0f;
+#pragma unroll
+  for (int j = 0; j < (NL > 0 ? NL : 32); ++j) {
+    if (j >= nl) break;
+    const int e0 = j * 256 + lane * 8;
+    float w[8], xh[8], pr[8];
+    if (e0 < D) {
+      load8<BF>(dy, rb + e0, w);
+      load8<BF>(x, rb + e0, xh);
+      if (gamma) {
+        float g[8];
+        load8<BF>(gamma, e0, g);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) w[t] = fmul(w[t], g[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xh[t] = fmul(xh[t], rs);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { w[t] = 0.0f; xh[t] = 0.0f; }
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) pr[t] = fmul(w[t], xh[t]);
+    if (NL > 0) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { kw[j][t] = w[t]; kx[j][t] = xh[t]; }
+    }
+    float leaf = warp_tree(tree8_full(pr), (long long)j * 256, 8, D);
+    if (lane == j) mine = leaf;
+  }
+  const float c = fmul(warp_tree(mine, 0, 256, D), invD);
+#pragma unroll
+  for (int j = 0; j < (NL > 0 ? NL : 32); ++j) {
+    if (j >= nl) break;
+    const int e0 = j * 256 + lane * 8;
+    if (e0 >= D) continue;
+    float w[8], xh[8], o[8];
+    if (NL > 0) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { w[t] = kw[j][t]; xh[t] = kx[j][t]; }
+    } else {
+      load8<BF>(dy, rb + e0, w);
+      load8<BF>(x, rb + e0, xh);
+      if (gamma) {
+        float g[8];
+        load8<BF>(gamma, e0, g);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) w[t] = fmul(w[t], g[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xh[t] = fmul(xh[t], rs);
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[t], fmul(xh[t], c)));
+    store8<BF>(dx, rb + e0, o);
+  }
+}
+
+// dgamma partials: CTA = 256 rows (one leaf of the row-direction tree) x 32 columns.
+template <bool BF>
+__global__ void __launch_bounds__(256) k_dgamma_partial(const void* __restrict__ dy, const void* __restrict__ x,
+                                                        const float* __restrict__ rstd, int rows, int D,
+                                                        float* __restrict__ partial) {
+  __shared__ float sm[8][33];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col = blockIdx.x * 32 + lane;
+  const long long r0 = (long long)blockIdx.y * 256 + warp * 32;
+  float s[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    long long r = r0 + i;
+    float v = 0.0f;
+    if (r < rows && col < D) {
+      size_t idx = (size_t)r * D + col;
+      float a, b;
+      if (BF) { a = bf2f(reinterpret_cast<const uint16_t*>(dy)[idx]); b = bf2f(reinterpret_cast<const uint16_t*>(x)[idx]); }
+      else { a = reinterpret_cast<const float*>(dy)[idx]; b = reinterpret_cast<const float*>(x)[idx]; }
+      v = fmul(a, fmul(b, rstd[r]));
+    }
+    s[i] = v;
+  }
+  sm[warp][lane] = reg_tree<32>(s, r0, 1, rows);
+  __syncthreads();
+  if (warp == 0 && col < D) {
+    float w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = sm[j][lane];
+    partial[(size_t)blockIdx.y * D + col] = reg_tree<8>(w, (long long)blockIdx.y * 256, 32, rows);
+  }
+}
+// level-by-level tree over the nb row-block partials of each column, in place; result in row 0
+__global__ void k_col_tree(float* __restrict__ partial, int nb, int D, float* __restrict__ out) {
+  const int col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= D) return;
+  int n = nb;
+  while (n > 1) {
+    int m = (n + 1) >> 1;
+    for (int i = 0; i < (n >> 1); ++i)
+      partial[(size_t)i * D + col] = fadd(partial[(size_t)(2 * i) * D + col], partial[(size_t)(2 * i + 1) * D + col]);
+    if (n & 1) partial[(size_t)(m - 1) * D + col] = partial[(size_t)(n - 1) * D + col];
+    n = m;
+  }
+  out[col] = partial[col];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Cross-entropy.  One CTA (512 threads) per row: max, then exp and the leaf sums, then the tree over
+// leaf sums in shared memory.
+// ------------------------------------------------------------------------------------------------
+constexpr int XT = 512;
+__global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logits, const int32_t* __restrict__ target,
+                                                 int V, float* __restrict__ loss_row, float* __restrict__ lse_out,
+                                                 float* __restrict__ zsq_row, int* status) {
+  extern __shared__ float leafs[];  // ceil(V/256) floats, >= 32
+  __shared__ float red[XT / 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* z = logits + (size_t)blockIdx.x * V;
+  float m = __int_as_float(0xff800000);
+  for (int i = threadIdx.x * 4; i < V; i += XT * 4) {
+    float4 a = *reinterpret_cast<const float4*>(z + i);
+    m = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
+  }
+#pragma unroll
+  for (int w = 16; w; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = red[0];
+#pragma unroll
+  for (int w = 1; w < XT / 32; ++w) m = fmaxf(m, red[w]);
+  const int nl = (V + 255) >> 8;
+  for (int leaf = warp; leaf < nl; leaf += XT / 32) {
+    const int e0 = leaf * 256 + lane * 8;
+    float e[8];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (e0 + 4 * h < V) {
+        float4 a = *reinterpret_cast<const float4*>(z + e0 + 4 * h);
+        e[4 * h] = det_exp(fsub(a.x, m)); e[4 * h + 1] = det_exp(fsub(a.y, m));
+        e[4 * h + 2] = det_exp(fsub(a.z, m)); e[4 * h + 3] = det_exp(fsub(a.w, m));
+      } else {
+        e[4 * h] = e[4 * h + 1] = e[4 * h + 2] = e[4 * h + 3] = 0.0f;
+      }
+    }
+    float s = warp_tree(tree8(e, e0, V), (long long)leaf * 256, 8, V);
+    if (lane == 0) leafs[leaf] = s;
+  }
+  __syncthreads();
+  smem_tree(leafs, nl);
+  if (threadIdx.x == 0) {
+    float l = fadd(m, det_log(leafs[0]));
+    lse_out[blockIdx.x] = l;
+    int t = target[blockIdx.x];
+    if (t < 0 || t >= V) {
+      loss_row[blockIdx.x] = 0.0f;
+      zsq_row[blockIdx.x] = 0.0f;
+      or_status(status, DET_DEV_TARGET);
+    } else {
+      loss_row[blockIdx.x] = fsub(l, z[t]);
+      zsq_row[blockIdx.x] = fmul(l, l);
+    }
+  }
+}
+
+__global__ void k_xent_finish(const float* ce_sum, const float* z_sum, float inv_rows, float z_weight,
+                              float* loss_mean, float* z_mean) {
+  float ce = fmul(ce_sum[0], inv_rows), zm = fmul(z_sum[0], inv_rows);
+  z_mean[0] = zm;
+  loss_mean[0] = (z_weight != 0.0f) ? fadd(ce, fmul(z_weight, zm)) : ce;
+}
+
+__global__ void __launch_bounds__(256) k_xent_bwd(float* __restrict__ logits, const int32_t* __restrict__ target,
+                                                  const float* __restrict__ lse, int rows, int V, float z_weight, float scale) {
+  const int i = (blockIdx.x * 256 + threadIdx.x) * 4;
+  if (i >= V) return;
+  for (int row = blockIdx.y; row < rows; row += gridDim.y) {
+  float* z = logits + (size_t)row * V;
+  const int t = target[row];
+  const bool ok = t >= 0 && t < V;
+  const float l = lse[row];
+  const float zc = fmul(fmul(2.0f, z_weight), l);
+  float4 a = *reinterpret_cast<float4*>(z + i);
+  float v[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (!ok) { v[k] = 0.0f; continue; }
+    float p = det_exp(fsub(v[k], l));
+    float d = fsub(p, (i + k == t) ? 1.0f : 0.0f);
+    if (z_weight != 0.0f) d = fadd(d, fmul(zc, p));
+    v[k] = fmul(d, scale);
+  }
+  *reinterpret_cast<float4*>(z + i) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+}  // namespace det
+
+using namespace det;
+
+extern "C" int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int rows, int D, float eps, void* y,
+                               float* rstd, void* stream) {
+  if (!x || !y || !rstd || rows < 0 || D <= 0 || (io != DET_F32 && io != DET_BF16)) return DET_ERR_ARG;
+  if (D % 8 || D > 8192) return DET_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y) || (gamma && !aligned16(gamma))) return DET_ERR_ALIGN;
+  if (rows == 0) return DET_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  const float invD = (float)(1.0 / (double)D);
+  dim3 grid((rows + 7) / 8);
+  if (io == DET_BF16) {
+    if (D <= 2048) k_rmsnorm_fwd<true, 8><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    else k_rmsnorm_fwd<true, 0><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+  } else {
+    if (D <= 2048) k_rmsnorm_fwd<false, 8><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    else k_rmsnorm_fwd<false, 0><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+  }
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" size_t det_rmsnorm_bwd_ws_bytes(int rows, int D) {
+  return align_up((size_t)((rows + 255) / 256) * (size_t)D * sizeof(float), 256) + 256;
+}
+
+extern "C" int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void* gamma, const float* rstd, int rows,
+                               int D, void* dx, float* dgamma, void* ws, size_t ws_bytes, void* stream) {
+  if (!dy || !x || !rstd || !dx || rows < 0 || D <= 0 || (io != DET_F32 && io != DET_BF16)) return DET_ERR_ARG;
+  if (D % 8 || D > 8192) return DET_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || (gamma && !aligned16(gamma))) return DET_ERR_ALIGN;
+  if (dgamma && (!ws || ws_bytes < det_rmsnorm_bwd_ws_bytes(rows, D))) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (rows == 0) {
+    if (dgamma) cudaMemsetAsync(dgamma, 0, (size_t)D * sizeof(float), st);
+    return DET_OK;
+  }
+  const float invD = (float)(1.0 / (double)D);
+  dim3 grid((rows + 7) / 8);
+  if (io == DET_BF16) {
+    if (D <= 2048) k_rmsnorm_bwd<true, 8><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    else k_rmsnorm_bwd<true, 0><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+  } else {
+    if (D <= 2048) k_rmsnorm_bwd<false, 8><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    else k_rmsnorm_bwd<false, 0><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+  }
+  if (dgamma) {
+    const int nb = (rows + 255) / 256;
+    dim3 g2((D + 31) / 32, nb);
+    if (io == DET_BF16) k_dgamma_partial<true><<<g2, 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
+    else k_dgamma_partial<false><<<g2, 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
+    k_col_tree<<<(D + 127) / 128, 128, 0, st>>>((float*)ws, nb, D, dgamma);
+  }
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" size_t det_xent_ws_bytes(int rows, int V) {
+  (void)V;
+  size_t r = align_up((size_t)(rows > 0 ? rows : 1), 64);
+  return (r + 128 + sum_ws_floats((size_t)rows)) * sizeof(float);
+}
+
+extern "C" int det_xent_fwd(const float* logits, const int32_t* target, int rows, int V, float z_weight,
+                            float* loss_row, float* lse, float* loss_mean, float* z_mean, void* ws, size_t ws_bytes,
+                            void* stream, int* status_dev) {
+  if (!logits || !target || !loss_row || !lse || !loss_mean || !z_mean || rows <= 0 || V <= 0 || !ws) return DET_ERR_ARG;
+  if (V % 4 || V > 2 * XT * 256) return DET_ERR_SHAPE;
+  if (!aligned16(logits)) return DET_ERR_ALIGN;
+  if (ws_bytes < det_xent_ws_bytes(rows, V)) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* zsq = (float*)ws;
+  float* sums = zsq + align_up((size_t)rows, 64);
+  float* scratch = sums + 128;
+  const int nl = (V + 255) / 256;
+  size_t sh = (size_t)(nl < 32 ? 32 : nl) * sizeof(float);
+  k_xent_fwd<<<rows, XT, sh, st>>>(logits, target, V, loss_row, lse, zsq, status_dev);
+  sum_launch(loss_row, (size_t)rows, 0, sums, scratch, st);
+  sum_launch(zsq, (size_t)rows, 0, sums + 64, scratch, st);
+  k_xent_finish<<<1, 1, 0, st>>>(sums, sums + 64, (float)(1.0 / (double)rows), z_weight, loss_mean, z_mean);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, int rows, int V,
+                            float z_weight, float scale, void* stream) {
+  if (!logits_inout || !target || !lse || rows <= 0 || V <= 0) return DET_ERR_ARG;
+  if (V % 4) return DET_ERR_SHAPE;
+  if (!aligned16(logits_inout)) return DET_ERR_ALIGN;
+  dim3 grid((V / 4 + 255) / 256, rows < 65535 ? rows : 65535);
+  k_xent_bwd<<<grid, 256, 0, (cudaStream_t)stream>>>(logits_inout, target, lse, rows, V, z_weight, scale);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}

@@ -1,0 +1,412 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle, bit for bit (0 ULP), on seeded inputs that
+span several tiles and ragged tails."""
+import ctypes
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from gpu_util import assert_same_bits, dev, empty, host, ws
+
+pytestmark = pytest.mark.gpu
+F = np.float32
+
+
+@pytest.fixture(scope="module")
+def det():
+    import torch
+    import paper_2609_17380_b200 as d
+    d.load()
+    assert torch.cuda.is_available()
+    return d
+
+
+def _sync():
+    import torch
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ primitives
+def test_primitives_bitwise(det):
+    rng = np.random.default_rng(0)
+    a = np.concatenate([synth.normal_f32(200000, 10.0, seed=1, tid=1), rng.uniform(-90, 90, 200000).astype(F),
+                        np.array([0.0, -0.0, 1.0, -1.0, 2.0 ** -126, 2.0 ** -127, -2.0 ** -140, 2.0 ** -149, 88.7, 88.73, -87.3,
+                                  -87.34, -100.0, 3.4e38, -np.inf, np.inf], F)])
+    b = np.concatenate([synth.normal_f32(200000, 1e-20, seed=1, tid=2), rng.uniform(0.1, 4, 200000).astype(F),
+                        np.array([1.0, 1.0, 2.0 ** -126, 0.5, 0.5, 2.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 10.0, 1.0, 1.0], F)])
+    da, db, out = dev(a), dev(b), empty(a.shape, F)
+    for name, op in oracle.OPS.items():
+        x, y = a, b
+        if name in ("sqrt", "log"):
+            x = np.abs(a) + F(2.0 ** -100)
+            x[~np.isfinite(x)] = 1.0
+            da = dev(x)
+        else:
+            da = dev(a)
+        det.det_prim(op, da, db, out)
+        _sync()
+        assert_same_bits(host(out), oracle.prim(name, x, y), "prim " + name)
+
+
+def test_max_of_signed_zeros(det):
+    a = np.array([0.0, -0.0, -0.0, 0.0], F)
+    b = np.array([-0.0, 0.0, -0.0, 0.0], F)
+    out = empty(a.shape, F)
+    det.det_prim(oracle.OPS["max"], dev(a), dev(b), out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("max", a, b), "max of zeros")
+
+
+def test_flush_boundary_probe(det):
+    # products whose exact value lies just below 2^-126: rounding to the minimum normal must be kept on both sides
+    fh = float.fromhex
+    a = np.array([fh('0x1.fffffep-1'), fh('0x1.fffffcp-1'), fh('0x1.000002p+0'), fh('0x1.8p-1')], F)
+    b = np.array([2.0 ** -126, 2.0 ** -126, fh('0x1.fffffep-1') * 2.0 ** -126, 2.0 ** -126], F)
+    out = empty(a.shape, F)
+    det.det_prim(oracle.OPS["mul"], dev(a), dev(b), out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("mul", a, b), "ftz boundary")
+    # quotients: exact value (1 - 2^-24) * 2^-126 is a tie that IEEE would round up to the minimum normal
+    a = np.array([fh('0x1.fffffep-1'), fh('0x1.fffffep-1'), 1.0, fh('0x1.fffffep-100'), 3.0], F)
+    b = np.array([2.0 ** 126, 2.0 ** 125, 2.0 ** 126, 2.0 ** 27, fh('0x1.8p+127')], F)
+    out = empty(a.shape, F)
+    det.det_prim(oracle.OPS["div"], dev(a), dev(b), out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("div", a, b), "ftz boundary (div)")
+
+
+def test_exp_all_bf16_arguments(det):
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    x = oracle.bf2f(h)
+    x = x[np.isfinite(x)]
+    out = empty(x.shape, F)
+    det.det_prim(oracle.OPS["exp"], dev(x), None, out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("exp", x), "exp")
+
+
+# ------------------------------------------------------------------ sums
+@pytest.mark.parametrize("n", [0, 1, 2, 7, 255, 256, 257, 16383, 16384, 16385, 50304, 1000003, 16384 * 300 + 17])
+def test_det_sum_lengths(det, n):
+    x = synth.normal_f32(max(n, 1), 1.0, seed=2, tid=n % 97)[:n]
+    dx = dev(x) if n else empty((4,), F)
+    out = empty((1,), F)
+    w = ws(det.det_sum_ws_bytes(n))
+    for sq in (0, 1):
+        det.det_sum(dx, n, sq, out, w)
+        _sync()
+        want = oracle.sumsq(x) if sq else oracle.det_sum(x)
+        assert_same_bits(host(out), np.array([want], F), "det_sum n=%d sq=%d" % (n, sq))
+
+
+def test_det_sum_order_pins_on_device(det):
+    out = empty((1,), F)
+    w = ws(256)
+    for v, want in (([2.0 ** 24, 1, 1, 1], 16777218.0), ([2.0 ** 24, 0, 0, 0, 1, 0, 1], 16777218.0),
+                    ([1, 2.0 ** 24, 0, 0, 0, 0, 1], 16777216.0)):
+        x = np.array(v, F)
+        det.det_sum(dev(np.concatenate([x, np.zeros(8, F)])), x.size, 0, out, w)
+        _sync()
+        assert host(out)[0] == F(want)
+    x = np.full(5, -0.0, F)
+    det.det_sum(dev(np.concatenate([x, np.zeros(3, F)])), 5, 0, out, w)
+    _sync()
+    assert host(out).view(np.uint32)[0] == 0x80000000
+
+
+def test_grad_norm_and_scale(det):
+    sizes = [4, 1000, 16384, 70001 * 4, 3 * 16384 + 12]
+    gs = [synth.normal_f32(s, 1e-3, seed=3, tid=i) for i, s in enumerate(sizes)]
+    dg = [dev(g) for g in gs]
+    norm, coef = empty((1,), F), empty((1,), F)
+    w = ws(det.det_grad_norm_ws_bytes(dg))
+    for mx in (1.0, 1e-3, 0.0):
+        det.det_grad_norm(dg, mx, norm, coef, w)
+        _sync()
+        on, oc = oracle.grad_norm(gs, mx)
+        assert_same_bits(host(norm), np.array([on], F), "norm")
+        assert_same_bits(host(coef), np.array([oc], F), "coef")
+    det.det_grad_norm(dg, 1e-3, norm, coef, w)
+    det.det_scale_inplace(dg[3], sizes[3], coef)
+    _sync()
+    assert_same_bits(host(dg[3]), oracle.scale(gs[3], oracle.grad_norm(gs, 1e-3)[1]), "scale")
+    # all-ones of length 4^k has norm 2^k exactly
+    ones = dev(np.ones(4 ** 9, F))
+    det.det_grad_norm([ones], 1.0, norm, coef, ws(det.det_grad_norm_ws_bytes([ones])))
+    _sync()
+    assert host(norm)[0] == 512.0
+
+
+# ------------------------------------------------------------------ RMSNorm
+@pytest.mark.parametrize("bf,rows,D,gain", [(False, 300, 2048, True), (True, 300, 2048, True), (False, 33, 1000, False),
+                                            (True, 17, 4096, True), (False, 9, 8, True), (True, 513, 256, False)])
+def test_rmsnorm(det, bf, rows, D, gain):
+    x = synth.normal_f32((rows, D), 1.0, seed=4, tid=1)
+    g = (1 + synth.normal_f32(D, 0.02, seed=4, tid=2)) if gain else None
+    dy = synth.normal_f32((rows, D), 1.0, seed=4, tid=3)
+    if bf:
+        x, dy = synth.to_bf16(x), synth.to_bf16(dy)
+        g = synth.to_bf16(g) if gain else None
+    dt = np.uint16 if bf else F
+    y, rstd = empty((rows, D), dt), empty((rows,), F)
+    dg_ = dev(g) if gain else None
+    det.det_rmsnorm_fwd(int(bf), dev(x), dg_, rows, D, 1e-6, y, rstd)
+    _sync()
+    oy, orstd = oracle.rmsnorm_fwd(x, g, 1e-6, bf=bf)
+    assert_same_bits(host(rstd), orstd, "rstd")
+    assert_same_bits(host(y, dt), oy, "y")
+    dx, dgam = empty((rows, D), dt), empty((D,), F)
+    det.det_rmsnorm_bwd(int(bf), dev(dy), dev(x), dg_, rstd, rows, D, dx, dgam, ws(det.det_rmsnorm_bwd_ws_bytes(rows, D)))
+    _sync()
+    odx, odg = oracle.rmsnorm_bwd(dy, x, g, orstd, bf=bf)
+    assert_same_bits(host(dx, dt), odx, "dx")
+    assert_same_bits(host(dgam), odg, "dgamma")
+
+
+# ------------------------------------------------------------------ cross-entropy
+@pytest.mark.parametrize("rows,V,zw", [(24, 50304, 0.0), (8, 50304, 1e-4), (5, 1000, 0.0), (3, 4, 0.0), (2, 128256, 1e-4)])
+def test_xent(det, rows, V, zw):
+    z = synth.normal_f32((rows, V), 2.0, seed=5, tid=1)
+    t = synth.randint(rows, V, seed=5, tid=2)
+    dz = dev(z)
+    dt_ = dev(t)
+    loss_row, lse, lm, zm = empty((rows,), F), empty((rows,), F), empty((1,), F), empty((1,), F)
+    import torch
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_xent_fwd(dz, dt_, rows, V, zw, loss_row, lse, lm, zm, ws(det.det_xent_ws_bytes(rows, V)), status)
+    _sync()
+    ol, olse, olm, ozm, bad = oracle.xent_fwd(z, t, zw)
+    assert bad == 0 and int(status.item()) == 0
+    assert_same_bits(host(lse), olse, "lse")
+    assert_same_bits(host(loss_row), ol, "loss_row")
+    assert_same_bits(host(lm), olm, "loss_mean")
+    assert_same_bits(host(zm), ozm, "z_mean")
+    det.det_xent_bwd(dz, dt_, lse, rows, V, zw, 1.0 / 64)
+    _sync()
+    assert_same_bits(host(dz), oracle.xent_bwd(z, t, olse, zw, 1.0 / 64), "dlogits")
+
+
+def test_xent_closed_forms_and_bad_target(det):
+    import torch
+    V = 50304
+    z = np.full((2, V), 3.25, F)
+    t = np.array([7, V], np.int32)                 # second target is out of range
+    loss_row, lse, lm, zm = empty((2,), F), empty((2,), F), empty((1,), F), empty((1,), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_xent_fwd(dev(z), dev(t), 2, V, 0.0, loss_row, lse, lm, zm, ws(det.det_xent_ws_bytes(2, V)), status)
+    _sync()
+    assert int(status.item()) & det.DEV_TARGET
+    ol, olse, olm, _, bad = oracle.xent_fwd(z, t)
+    assert bad == 1
+    assert_same_bits(host(loss_row), ol, "loss")
+    assert abs(float(host(loss_row)[0]) - np.log(V)) < 2e-6 and host(loss_row)[1] == 0
+
+
+# ------------------------------------------------------------------ glue
+def test_glue(det):
+    rows, Fd = 37, 1024
+    gu = synth.normal_bf16((rows, 2 * Fd), 2.0, seed=6, tid=1)
+    gu[0, :4] = synth.to_bf16(np.array([-200.0, 200.0, 90.0, -90.0], F))
+    dh = synth.normal_bf16((rows, Fd), 1.0, seed=6, tid=2)
+    h = empty((rows, Fd), np.uint16)
+    det.det_swiglu_fwd(dev(gu), rows, Fd, h)
+    dgu = empty((rows, 2 * Fd), np.uint16)
+    det.det_swiglu_bwd(dev(dh), dev(gu), rows, Fd, dgu)
+    _sync()
+    assert_same_bits(host(h, np.uint16), oracle.swiglu_fwd(gu), "swiglu")
+    assert_same_bits(host(dgu, np.uint16), oracle.swiglu_bwd(dh, gu), "swiglu bwd")
+    a = synth.normal_bf16(40000, 1.0, seed=6, tid=3)
+    b = synth.normal_bf16(40000, 1.0, seed=6, tid=4)
+    y = empty((40000,), np.uint16)
+    det.det_residual_add(dev(a), dev(b), 40000, y)
+    _sync()
+    assert_same_bits(host(y, np.uint16), oracle.residual_add(a, b), "residual")
+
+
+def test_embedding(det):
+    V, D, T = 1000, 512, 700
+    E = synth.normal_bf16((V, D), 0.02, seed=7, tid=1)
+    tok = synth.randint(T, 50, seed=7, tid=2)          # many duplicates
+    tok[::7] = synth.randint((T + 6) // 7, V, seed=7, tid=3)
+    y = empty((T, D), np.uint16)
+    det.det_embed_fwd(dev(tok), T, dev(E), V, D, y)
+    dy = synth.normal_bf16((T, D), 1.0, seed=7, tid=4)
+    dE = empty((V, D), F)
+    det.det_embed_bwd(dev(tok), T, dev(dy), V, D, dE)
+    _sync()
+    assert_same_bits(host(y, np.uint16), oracle.embed_fwd(tok, E), "embed")
+    assert_same_bits(host(dE), oracle.embed_bwd(tok, dy, V), "embed bwd")
+
+
+# ------------------------------------------------------------------ gradient accumulation, AdamW, hash
+@pytest.mark.parametrize("mesh", [(8, 1, 1), (2, 2, 2), (1, 8, 1), (1, 1, 8), (1, 1, 7), (2, 1, 3), (1, 3, 2)])
+def test_grad_accum(det, mesh):
+    n = 40000
+    accum, shard, rep = mesh
+    total = accum * shard * rep
+    gs = [synth.normal_f32(n, 1e-3, seed=8, tid=i) for i in range(total)]
+    nb = det.det_grad_accum_nbufs(rep)
+    bufs = empty((nb * n,), F)
+    st = det.det_accum()
+    det.det_grad_accum_init(st, accum, shard, rep, n, bufs)
+    oa = oracle.Accum(accum, shard, rep, n)
+    out = empty((n,), F)
+    with pytest.raises(det.DetError):
+        det.det_grad_accum_result(st, out)             # too few pushes
+    for g in gs:
+        det.det_grad_accum_push(st, dev(g))
+        oa.push(g)
+    det.det_grad_accum_result(st, out)
+    _sync()
+    assert_same_bits(host(out), oa.result(), "accum %s" % (mesh,))
+    with pytest.raises(det.DetError):
+        det.det_grad_accum_push(st, dev(gs[0]))        # too many pushes
+
+
+@pytest.mark.parametrize("bf,n", [(True, 100003), (False, 96), (True, 4096)])
+def test_adamw(det, bf, n):
+    p = synth.normal_f32(n, 0.02, seed=9, tid=1)
+    if bf:
+        p = synth.to_bf16(p)
+    m = np.zeros(n, F)
+    v = np.zeros(n, F)
+    dp, dm, dv = dev(p), dev(m), dev(v)
+    for t in (1, 2, 3):
+        g = synth.normal_f32(n, 1e-3, seed=9, tid=10 + t)
+        wd = 0.1 if bf else 0.0
+        desc = det.det_adamw_desc(3e-4, 0.9, 0.95, 1e-8, wd, t)
+        det.det_adamw_step(desc, int(bf), dp, dev(g), dm, dv, n)
+        _sync()
+        p, m, v = oracle.adamw(p, g, m, v, 3e-4, 0.9, 0.95, 1e-8, wd, t)
+        assert_same_bits(host(dp, p.dtype), p, "p t=%d" % t)
+        assert_same_bits(host(dm), m, "m")
+        assert_same_bits(host(dv), v, "v")
+
+
+@pytest.mark.parametrize("n", [16, 65536, 65536 + 16, 3 * 65536 + 1000, 5000000])
+def test_tensor_hash(det, n):
+    b = np.random.default_rng(n).integers(0, 256, n).astype(np.uint8)
+    got = det.det_tensor_hash(dev(b), n, ws(det.det_tensor_hash_ws_bytes(n)))
+    assert got == oracle.tensor_hash(b)
+
+
+# ------------------------------------------------------------------ int8 GEMM and the LSQ linear layer
+@pytest.mark.parametrize("I,J,K", [(128, 128, 128), (256, 512, 512), (384, 256, 1024), (128, 384, 2048), (512, 768, 640)])
+def test_igemm_exact(det, I, J, K):
+    import torch
+    rng = np.random.default_rng(I + J + K)
+    A = rng.integers(-128, 128, (I, K)).astype(np.int8)
+    B = rng.integers(-128, 128, (J, K)).astype(np.int8)
+    Cd = empty((I, J), np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_igemm_tn(dev(A), dev(B), I, J, K, Cd, status)
+    _sync()
+    assert int(status.item()) == 0
+    want = A.astype(np.int32) @ B.astype(np.int32).T       # brute force, exact
+    assert_same_bits(host(Cd), want, "igemm")
+
+
+def _linear_case(M, N, K, seed):
+    X = synth.normal_bf16((M, K), 1.0, seed=seed, tid=1)
+    X.reshape(-1)[:7] = synth.to_bf16(np.array([40, -40, 30, -35, 50, 11.3, -11.3], F))
+    W = synth.normal_bf16((N, K), 0.02, seed=seed, tid=2)
+    dY = synth.normal_bf16((M, N), 0.01, seed=seed, tid=3)
+    return X, W, dY
+
+
+@pytest.mark.parametrize("M,N,K,per_tensor", [(256, 512, 512, False), (256, 512, 512, True), (384, 128, 1024, False),
+                                              (128, 640, 256, False)])
+def test_lsq_scales_quant_forward(det, M, N, K, per_tensor):
+    import torch
+    X, W, _ = _linear_case(M, N, K, 11)
+    dX_, dW_ = dev(X), dev(W)
+    s_w, s_x = empty((N,), F), empty((1,), F)
+    det.det_lsq_weight_scale(dW_, N, K, int(per_tensor), s_w, ws(det.det_lsq_weight_scale_ws_bytes(N, K)))
+    det.det_lsq_act_scale_init(dX_, M * K, s_x, ws(det.det_lsq_act_scale_init_ws_bytes(M * K)))
+    _sync()
+    osw = oracle.lsq_weight_scale(W, per_tensor)
+    osx = oracle.lsq_act_scale_init(X)
+    assert_same_bits(host(s_w), osw, "s_w")
+    assert_same_bits(host(s_x), osx, "s_x")
+    qW, qWt, s_u = empty((N, K), np.int8), empty((K, N), np.int8), empty((1,), F)
+    det.det_lsq_quantize_weight(dW_, s_w, N, K, 128, qW, qWt, s_u, ws(det.det_lsq_quantize_weight_ws_bytes(N, K)))
+    Y, qX = empty((M, N), np.uint16), empty((M, K), np.int8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_linear_fwd(dX_, qW, s_x, s_w, M, N, K, Y, qX, status)
+    _sync()
+    assert int(status.item()) == 0
+    oY, oqX, oqW = oracle.linear_fwd(X, W, osx, osw)
+    assert_same_bits(host(qW), oqW, "qW")
+    assert_same_bits(host(qX), oqX, "qX")
+    assert_same_bits(host(Y, np.uint16), oY, "Y")
+
+
+@pytest.mark.parametrize("M,N,K,hb", [(256, 512, 512, 128), (256, 512, 512, 0), (384, 128, 256, 128), (128, 256, 640, 128)])
+def test_linear_backward(det, M, N, K, hb):
+    import torch
+    X, W, dY = _linear_case(M, N, K, 12)
+    osw = oracle.lsq_weight_scale(W)
+    osx = oracle.lsq_act_scale_init(X)
+    odX, odW, ods, dbg = oracle.linear_bwd(dY, X, W, osx, osw, hb=hb, debug=True)
+    dX_, dW_, dY_ = dev(X), dev(W), dev(dY)
+    s_w, s_x = dev(osw), dev(osx)
+    qW, qWt, s_u = empty((N, K), np.int8), empty((K, N), np.int8), empty((1,), F)
+    det.det_lsq_quantize_weight(dW_, s_w, N, K, hb, qW, qWt, s_u, ws(det.det_lsq_quantize_weight_ws_bytes(N, K)))
+    Y, qX = empty((M, N), np.uint16), empty((M, K), np.int8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_linear_fwd(dX_, qW, s_x, s_w, M, N, K, Y, qX, status)
+    gX, gW, gs = empty((M, K), np.uint16), empty((N, K), F), empty((1,), F)
+    w = ws(det.det_linear_bwd_ws_bytes(M, N, K))
+    det.det_linear_bwd(dY_, dX_, qX, dW_, qWt, s_x, s_w, s_u, M, N, K, hb, gX, gW, gs, w, status)
+    _sync()
+    assert int(status.item()) == 0
+    assert_same_bits(host(qWt), dbg["UqT"], "UqT")
+    assert_same_bits(host(s_u), dbg["scales"][1:2], "s_u")
+    assert_same_bits(host(gX, np.uint16), odX, "dX")
+    assert_same_bits(host(gW), odW, "dW")
+    assert_same_bits(host(gs), ods, "ds_x")
+
+
+# ------------------------------------------------------------------ LM head and attention (ordered FP32)
+@pytest.mark.parametrize("M,V,K", [(128, 256, 256), (72, 1000, 64), (256, 50304 // 8, 128)])
+def test_lmhead(det, M, V, K):
+    Hh = synth.normal_bf16((M, K), 1.0, seed=13, tid=1)
+    W = synth.normal_bf16((V, K), 0.02, seed=13, tid=2)
+    lg = empty((M, V), F)
+    det.det_lmhead_fwd(dev(Hh), dev(W), M, V, K, lg)
+    _sync()
+    assert_same_bits(host(lg), oracle.lmhead_fwd(Hh, W), "logits")
+    dl = synth.normal_f32((M, V), 1e-3, seed=13, tid=3)
+    dH, dW = empty((M, K), np.uint16), empty((V, K), F)
+    h1 = M // 2 // 8 * 8
+    det.det_lmhead_bwd(dev(dl[:h1]), dev(Hh[:h1]), dev(W), h1, V, K, dH[:h1], dW, 1)
+    det.det_lmhead_bwd(dev(dl[h1:]), dev(Hh[h1:]), dev(W), M - h1, V, K, dH[h1:], dW, 0)
+    _sync()
+    oH, oW = oracle.lmhead_bwd(dl, Hh, W)
+    assert_same_bits(host(dH, np.uint16), oH, "dH")
+    assert_same_bits(host(dW), oW, "dW")
+
+
+@pytest.mark.parametrize("B,H,S", [(1, 2, 64), (2, 2, 192), (1, 1, 320)])
+def test_attention(det, B, H, S):
+    HD = H * 128
+    qkv = synth.normal_bf16((B * S, 3 * HD), 1.0, seed=14, tid=1)
+    dout = synth.normal_bf16((B * S, HD), 0.1, seed=14, tid=2)
+    dqkv_in = dev(qkv)
+    base = dqkv_in.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    det.det_attn_fwd(base, base + 2 * HD, base + 4 * HD, 3 * HD, B, H, S, out, HD, lse)
+    _sync()
+    oout, olse = oracle.attn_fwd(qkv, B, H, S)
+    assert_same_bits(host(lse), olse, "lse")
+    assert_same_bits(host(out, np.uint16), oout, "out")
+    dqkv = empty((B * S, 3 * HD), np.uint16)
+    db = dqkv.data_ptr()
+    det.det_attn_bwd(dev(dout), base, base + 2 * HD, base + 4 * HD, out, lse, 3 * HD, HD, B, H, S, db, db + 2 * HD,
+                     db + 4 * HD, 3 * HD, ws(det.det_attn_bwd_ws_bytes(B, H, S)))
+    _sync()
+    want = oracle.attn_bwd(dout, qkv, oout, olse, B, H, S)
+    got = host(dqkv, np.uint16)
+    for name, c in (("dq", 0), ("dk", 1), ("dv", 2)):
+        assert_same_bits(got[:, c * HD:(c + 1) * HD], want[:, c * HD:(c + 1) * HD], name)

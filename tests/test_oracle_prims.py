@@ -42,6 +42,11 @@ def test_flush_to_zero():
     assert r[0] == 0 and np.signbit(r[0])                    # sign-preserving zero
     assert oracle.prim("add", [tiny], [tiny])[0] == F(2.0 ** -125)
     assert oracle.prim("sub", [F(1.5) * tiny], [tiny])[0] == 0  # exact result 2^-127 is subnormal
+    # tininess is judged on the exact value: (1 - 2^-24) * 2^-126 would round up to 2^-126 but is flushed
+    almost_one = F(1 - 2.0 ** -24)
+    assert oracle.prim("mul", [almost_one], [tiny])[0] == 0
+    assert oracle.prim("div", [almost_one], [F(2.0 ** 126)])[0] == 0
+    assert oracle.prim("mul", [F(1 + 2.0 ** -23)], [tiny])[0] == F((1 + 2.0 ** -23) * 2.0 ** -126)
     assert oracle.prim("max", [-0.0], [0.0]).view(np.uint32)[0] == 0
     assert oracle.prim("max", [0.0], [-0.0]).view(np.uint32)[0] == 0
 
