@@ -73,3 +73,38 @@ def normal_bf16(shape, std=1.0, mean=0.0, seed=0, tid=0):
 def randint(shape, high, seed=0, tid=0):
     n = int(np.prod(shape))
     return (_raw(n, seed, tid).astype(np.uint64) % np.uint64(high)).astype(np.int32).reshape(shape)
+
+
+# ---- model-shaped inputs --------------------------------------------------------------------------------
+def model_param_specs(cfg):
+    """Canonical parameter order: embedding; per layer attn-norm gain, W_qkv, W_o, ffn-norm gain, W_gate/up,
+    W_down, the four activation steps; final-norm gain; LM head.  cfg: dict with n_layers, d_model, ffn, vocab.
+    Returns a list of (name, shape, kind) with kind in {"embed", "gain", "linear", "step", "head"}."""
+    D, Fh, V, L = cfg["d_model"], cfg["ffn"], cfg["vocab"], cfg["n_layers"]
+    specs = [("embed", (V, D), "embed")]
+    for l in range(L):
+        specs += [("l%d.attn_norm" % l, (D,), "gain"), ("l%d.w_qkv" % l, (3 * D, D), "linear"),
+                  ("l%d.w_o" % l, (D, D), "linear"), ("l%d.ffn_norm" % l, (D,), "gain"),
+                  ("l%d.w_gu" % l, (2 * Fh, D), "linear"), ("l%d.w_down" % l, (D, Fh), "linear"),
+                  ("l%d.s_x" % l, (4,), "step")]
+    specs += [("final_norm", (D,), "gain"), ("lm_head", (V, D), "head")]
+    return specs
+
+
+def model_params(cfg, seed=0):
+    """Random-init parameters: weights ~ N(0, 0.02) as bf16 bit patterns, gains = 1 (bf16), activation steps
+    filled later by a calibration forward (zeros here, float32)."""
+    out = {}
+    for tid, (name, shape, kind) in enumerate(model_param_specs(cfg)):
+        if kind == "gain":
+            out[name] = np.full(shape, 0x3F80, np.uint16)
+        elif kind == "step":
+            out[name] = np.zeros(shape, np.float32)
+        else:
+            out[name] = normal_bf16(shape, 0.02, seed=seed, tid=1000 + tid)
+    return out
+
+
+def model_tokens(cfg, n_microbatches, seed=0):
+    """Uniform random token ids, [n_microbatches, micro_batch, seq + 1] (inputs and shifted labels)."""
+    return randint((n_microbatches, cfg["micro_batch"], cfg["seq"] + 1), cfg["vocab"], seed=seed, tid=777)
