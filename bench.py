@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the replayed, bit-exact training step on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+A "step" is one full optimizer step of the 1B-shaped decoder (24 layers, d_model 2048, 16 heads, FFN 8192,
+vocab 50304, seq 2048, 32 sequences as 8 micro-batches of 4 in mesh (accum, dp_shard, dp_replicate) = (2,2,2)):
+weight-step re-pin and quantisation, 8 x (forward, backward), the fixed-order gradient reduction, global-norm
+clip, AdamW, and the SHA-256 state hash.  Inputs are seeded synthetic token ids and random-init weights.
+Prints ONE JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "replayed step tokens/s (bit-exact)"
+UNIT = "tokens/s"
+WORKLOAD = "config5: full 1B-shaped step, 24 layers, d_model 2048, 16 heads, FFN 8192, vocab 50304, seq 2048, " \
+           "8 micro-batches of 4 sequences, mesh (accum,dp_shard,dp_replicate)=(2,2,2), AdamW, SHA-256 of post-step state"
+
+
+def full_config_kwargs(layers=None):
+    kw = dict(n_layers=24, d_model=2048, n_heads=16, ffn=8192, vocab=50304, seq=2048, micro_batch=4, mesh=(2, 2, 2),
+              hadamard_block=128, lr=3e-4, betas=(0.9, 0.95), eps=1e-8, wd=0.1, clip=1.0)
+    if layers is not None:
+        kw["n_layers"] = layers
+    return kw
+
+
+# ---------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown," \
+        "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except Exception:
+                continue
+            for name, col in (("hw_slowdown", 4), ("hw_thermal_slowdown", 5), ("sw_thermal_slowdown", 6), ("sw_power_cap", 7)):
+                if len(r) > col and r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d["bf16_tflops_sustained"],
+                "sm_max_mhz": d.get("sm_max_mhz", 1965.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------------------
+def cpu_baseline(kw):
+    """The oracle, as it stands, on the host cores: a bounded sample of the same workload, scaled to tokens/s.
+
+    Sample: (a) 8 tokens through embedding + final norm + LM head + loss, forward and backward; (b) one full-width
+    decoder layer (norms, four LSQ int8 linears, 16-head attention at seq 128, SwiGLU, residuals) on 128 tokens,
+    forward and backward; (c) accumulate + clip + AdamW + hash on 4M parameters.  Scaled linearly in tokens, layers
+    and parameters to the full step.  Attention is sampled at seq 128 instead of 2048, so its quadratic part is
+    under-counted: the figure flatters the CPU."""
+    import numpy as np
+    import oracle as O
+    import synth
+    from oracle import step as ostep
+    cores = os.cpu_count() or 1
+    D, Fh, V, L, H = kw["d_model"], kw["ffn"], kw["vocab"], kw["n_layers"], kw["n_heads"]
+    # (a) head: 8 tokens (weights drawn with numpy's seeded generator: only the timing is used here)
+    th = 8
+    c = dict(kw)
+    c.update(seq=th, micro_batch=1, mesh=(1, 1, 1), n_layers=0)
+    rng = np.random.default_rng(0)
+    P = {"embed": synth.to_bf16((rng.standard_normal((V, D), dtype=np.float32) * 0.02)),
+         "lm_head": synth.to_bf16((rng.standard_normal((V, D), dtype=np.float32) * 0.02)),
+         "final_norm": np.full(D, 0x3F80, np.uint16)}
+    toks = rng.integers(0, V, (1, th + 1)).astype(np.int32)
+    t0 = time.time()
+    ostep.microbatch_grad(c, P, {}, toks)
+    t_head = time.time() - t0
+    # (b) one layer on 128 tokens
+    T = 128
+    x = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32))
+    dy = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32) * 0.01)
+    gain = np.full(D, 0x3F80, np.uint16)
+    Ws = [synth.to_bf16(rng.standard_normal(sh, dtype=np.float32) * 0.02) for sh in ((3 * D, D), (D, D), (2 * Fh, D), (D, Fh))]
+    sws = [O.lsq_weight_scale(W) for W in Ws]
+    t0 = time.time()
+    n1, r1 = O.rmsnorm_fwd(x, gain, 1e-6, bf=True)
+    s0 = O.lsq_act_scale_init(n1)
+    qkv, _, _ = O.linear_fwd(n1, Ws[0], s0, sws[0])
+    att, lse = O.attn_fwd(qkv, 1, H, T)
+    s1 = O.lsq_act_scale_init(att)
+    o, _, _ = O.linear_fwd(att, Ws[1], s1, sws[1])
+    h = O.residual_add(x, o)
+    n2, r2 = O.rmsnorm_fwd(h, gain, 1e-6, bf=True)
+    s2 = O.lsq_act_scale_init(n2)
+    gu, _, _ = O.linear_fwd(n2, Ws[2], s2, sws[2])
+    act = O.swiglu_fwd(gu)
+    s3 = O.lsq_act_scale_init(act)
+    dn, _, _ = O.linear_fwd(act, Ws[3], s3, sws[3])
+    O.residual_add(h, dn)
+    d_act, _, _ = O.linear_bwd(dy, act, Ws[3], s3, sws[3], 128)
+    d_gu = O.swiglu_bwd(d_act, gu)
+    d_n2, _, _ = O.linear_bwd(d_gu, n2, Ws[2], s2, sws[2], 128)
+    d_h2, _ = O.rmsnorm_bwd(d_n2, h, gain, r2, bf=True)
+    d_h = O.residual_add(dy, d_h2)
+    d_att, _, _ = O.linear_bwd(d_h, att, Ws[1], s1, sws[1], 128)
+    d_qkv = O.attn_bwd(d_att, qkv, att, lse, 1, H, T)
+    d_n1, _, _ = O.linear_bwd(d_qkv, n1, Ws[0], s0, sws[0], 128)
+    d_x1, _ = O.rmsnorm_bwd(d_n1, x, gain, r1, bf=True)
+    O.residual_add(d_h, d_x1)
+    t_layer = time.time() - t0
+    # (c) reduction + optimizer + hash on 4M parameters
+    n_opt = 1 << 22
+    g = rng.standard_normal(n_opt, dtype=np.float32) * np.float32(1e-3)
+    p = synth.to_bf16(rng.standard_normal(n_opt, dtype=np.float32) * 0.02)
+    t0 = time.time()
+    acc = O.Accum(1, 1, 1, n_opt)
+    acc.push(g)
+    t_push = time.time() - t0
+    gr = acc.result()
+    nrm, coef = O.grad_norm([gr], 1.0)
+    gr = O.scale(gr, coef)
+    O.adamw(p, gr, np.zeros(n_opt, np.float32), np.zeros(n_opt, np.float32), 3e-4, 0.9, 0.95, 1e-8, 0.1, 1)
+    O.tensor_hash(p)
+    t_opt = time.time() - t0
+    n_params = 2 * V * D + L * (4 * D * D + 3 * D * Fh + 2 * D + 4) + D
+    tokens_step = 8 * kw["micro_batch"] * kw["seq"]
+    est = t_head * (tokens_step / th) + L * t_layer * (tokens_step / T) + (t_opt + 7 * t_push) * (n_params / n_opt)
+    return {"value": tokens_step / est, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "8 tokens through embed+norm+head+loss fwd/bwd (%.1fs); one full-width layer fwd/bwd on 128 tokens at "
+                      "seq 128 (%.1fs); accumulate+clip+AdamW+hash on 4M params (%.1fs); scaled linearly to %d layers, "
+                      "%d tokens, %.2fB params" % (t_head, t_layer, t_opt, L, tokens_step, n_params / 1e9),
+            "sample_seconds": t_head + t_layer + t_opt, "est_step_seconds": est}
+
+
+def run_reference(args):
+    """Reference arm = the CPU oracle as it stands, on the host cores, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    kw = full_config_kwargs(args.layers)
+    vals, ms = [], []
+    for i in range(args.warmup + args.steps):
+        t0 = time.time()
+        cb = cpu_baseline(kw)
+        dt = time.time() - t0
+        if i >= args.warmup:
+            vals.append(cb["value"])
+            ms.append(cb["est_step_seconds"] * 1e3)
+    v = statistics.mean(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": statistics.mean(ms), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8+f32", "data": "synthetic", "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cb["cores"], "kind": "oracle", "sample": cb["sample"]},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import paper_2609_17380_b200 as det
+    from paper_2609_17380_b200 import step as dstep
+    det.load()
+    kw = full_config_kwargs(args.layers)
+    cfg = dstep.ModelConfig(**kw)
+    r = dstep.Replay(cfg)
+    r.init_params_on_device(seed=rank)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + rank)
+    n_mb = cfg.n_microbatches
+    tok_dev = torch.randint(0, cfg.vocab, (n_mb, cfg.micro_batch, cfg.seq + 1), generator=gen, device="cuda", dtype=torch.int32)
+    tok_host = tok_dev.cpu().pin_memory()
+    r.calibrate(tok_dev[0])
+    torch.cuda.synchronize()
+    tokens_per_step = n_mb * cfg.micro_batch * cfg.seq
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def do_steps(n, host_inputs):
+        outs = []
+        for _ in range(n):
+            if host_inputs:
+                tok = tok_host.to("cuda", non_blocking=True)
+            else:
+                tok = tok_dev
+            out = r.step(tok, per_tensor_hashes=False, want_losses=host_inputs)
+            r.cfg.step += 1
+            outs.append(out)
+        return outs
+
+    do_steps(args.warmup, False)
+    # ---- device-resident timing ----
+    r.prof = {}
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    l0 = det.det_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    outs = do_steps(args.steps, False)
+    e1.record()
+    barrier()
+    wall = time.time() - t0
+    launches = det.det_launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = e0.elapsed_time(e1)
+    prof = r.prof_summary()
+    r.prof = None
+    # ---- end to end: tokens from pinned host memory, losses + hashes back on the host every step ----
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    outs2 = do_steps(args.steps, True)
+    e3.record()
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+    t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    status = max(o["status"] for o in outs + outs2)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    per_step = ms / args.steps
+    value = world * tokens_per_step * args.steps / (ms / 1e3)
+    e2e_val = world * tokens_per_step * args.steps / (ms_e2e / 1e3)
+    # ---- roofline of the dominant kernel group (by device time inside the timed region) ----
+    total_prof = sum(v[1] for v in prof.values()) or 1.0
+    shares = {k: round(v[1] / total_prof, 4) for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}
+    B, H, S, D, Fh, V, L, T = cfg.micro_batch, cfg.n_heads, cfg.seq, cfg.d_model, cfg.ffn, cfg.vocab, cfg.n_layers, cfg.tokens_per_microbatch
+    unit = B * H * (S * S // 2) * 128                   # causal-half MACs of one attention contraction
+    alg = {  # name -> (bound, algorithmic work per launch group, unit of peak)
+        "attn_fwd": ("alu", 2 * unit * 2.0, "flop"),
+        "attn_bwd": ("alu", 5 * unit * 2.0, "flop"),
+        "lmhead_fwd": ("alu", T * V * D * 2.0, "flop"),
+        "lmhead_bwd": ("alu", 2 * T * V * D * 2.0, "flop"),
+    }
+    alu_peak = 148 * 128 * peaks["sm_max_mhz"] * 1e6 / 1e12       # unfused FP32 instructions: TFLOP/s
+    dom = next(iter(shares))
+    roof = {"kernel": dom, "share_of_step": shares[dom]}
+    if dom in alg:
+        n, tot_ms = prof[dom]
+        ach = alg[dom][1] / (tot_ms / n / 1e3) / 1e12
+        roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
+                     "traffic": None, "peak_source": "148 SMs x 128 FP32 lanes x %.0f MHz, one unfused op per lane per clock"
+                     % peaks["sm_max_mhz"]})
+    # the two fractions the benchmark spec asks for: int8 tensor pipe (linear GEMMs) and HBM (order-fixed reductions)
+    lin_macs_fwd = T * (3 * D * D + D * D + 2 * Fh * D + D * Fh)
+    extra = {}
+    if "linear_fwd" in prof:
+        n, tot_ms = prof["linear_fwd"]
+        extra["linear_fwd_int8_tops"] = 2.0 * lin_macs_fwd / 4 * n / (tot_ms / 1e3) / 1e12
+        extra["linear_fwd_frac_of_4.5POPs"] = extra["linear_fwd_int8_tops"] / 4500.0
+    if "linear_bwd" in prof:
+        n, tot_ms = prof["linear_bwd"]
+        extra["linear_bwd_int8_tops"] = 2.0 * 2 * lin_macs_fwd / 4 * n / (tot_ms / 1e3) / 1e12
+    if "grad_accum" in prof:
+        n, tot_ms = prof["grad_accum"]
+        extra["grad_accum_gbs"] = 3.0 * r.n_grad * 4 * n / (tot_ms / 1e3) / 1e9
+        extra["grad_accum_frac_of_hbm"] = extra["grad_accum_gbs"] / peaks["hbm_gbs"]
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8 tensor-core GEMMs + f32 ordered arithmetic (bf16 storage)", "data": "synthetic",
+            "config": {"workload": WORKLOAD if args.layers is None else WORKLOAD + " [REDUCED to %d layers]" % args.layers,
+                       "l2": "inputs_exceed_l2", "multi_gpu": "replicas only" if world > 1 else "single"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(tok_host.numel() * 4),
+                    "d2h_bytes_per_step": int(n_mb * 4 + 8 + 5 * 32)},
+            "roofline": roof, "kernel_time_shares": shares, "component_rates": extra, "peaks": peaks,
+            "wall_s_timed": wall, "device_status": status,
+            "state_hash": outs[-1]["hashes"].get("params_bf16")}
+    if world == 1 and not args.no_cpu_baseline:
+        try:
+            import oracle
+            oracle.build()
+            line["cpu_baseline"] = cpu_baseline(kw)
+        except Exception as ex:  # the oracle is a reported baseline, not part of the product path
+            line["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": "failed: %r" % ex}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=None, help="debug only: fewer layers (the line says REDUCED)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

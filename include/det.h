@@ -52,6 +52,8 @@ typedef enum { DET_F32 = 0, DET_BF16 = 1 } det_dtype;
 
 /* library / device information: returns the number of SMs of the current device (or a negative status) */
 int det_device_sm_count(void);
+/* number of kernels this library has launched in this process so far (host-side counter, not thread-safe) */
+unsigned long long det_launch_count(void);
 
 /* ---- primitives (test hook) ---------------------------------------------------------------------
  * Elementwise evaluation of one primitive of Sec. 2.1 on device arrays: op 0 add, 1 sub, 2 mul, 3 div,

@@ -137,6 +137,8 @@ def linear_bwd(dY, X, W, s_x, s_w, hb=128, debug=False):
     s_w = _c(s_w, np.float32)
     M, K = X.shape
     N = W.shape[0]
+    if hb:
+        assert hb == 128 and M % 128 == 0 and N % 128 == 0, "rotation blocks of 128 along both contraction dimensions"
     dX = np.empty((M, K), np.uint16)
     dW = np.empty((N, K), np.float32)
     ds = np.empty(1, np.float32)

@@ -53,6 +53,7 @@ def load():
                      "det_lsq_act_scale_init_ws_bytes", "det_lsq_quantize_weight_ws_bytes", "det_linear_bwd_ws_bytes",
                      "det_rmsnorm_bwd_ws_bytes", "det_xent_ws_bytes", "det_attn_bwd_ws_bytes", "det_tensor_hash_ws_bytes"):
             getattr(_lib, name).restype = C.c_size_t
+        _lib.det_launch_count.restype = C.c_ulonglong
     return _lib
 
 
@@ -81,6 +82,10 @@ def _ws(ws):
 # ---- information / primitives ------------------------------------------------------------------------
 def det_device_sm_count():
     return load().det_device_sm_count()
+
+
+def det_launch_count():
+    return load().det_launch_count()
 
 
 def det_prim(op, a, b, out):

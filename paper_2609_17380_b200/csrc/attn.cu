@@ -444,7 +444,7 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   static bool cfg = false;
   if (!cfg) { if (set_smem((const void*)k_attn_fwd, FWD_SMEM)) return DET_ERR_CUDA; cfg = true; }
   dim3 grid(S / FQ, H, B);
-  k_attn_fwd<<<grid, 256, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
+  k_attn_fwd<<<DET_L(grid), 256, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -471,10 +471,10 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   uint16_t* dS = (uint16_t*)ws;
   float* delta = (float*)((uint8_t*)ws + align_up((size_t)B * H * S * S * 2, 256));
   const size_t nrows = (size_t)B * H * S;
-  k_attn_delta<<<(unsigned)((nrows + 7) / 8), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
+  k_attn_delta<<<DET_L((unsigned)((nrows + 7) / 8)), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
   dim3 grid(S / BT, H, B);
-  k_attn_dkdv<<<grid, 256, DKDV_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, S, dk, dv, ld_d, dS);
-  k_attn_dq<<<grid, 256, DQ_SMEM, st>>>(k, dS, ld, H, S, dq, ld_d);
+  k_attn_dkdv<<<DET_L(grid), 256, DKDV_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, S, dk, dv, ld_d, dS);
+  k_attn_dq<<<DET_L(grid), 256, DQ_SMEM, st>>>(k, dS, ld, H, S, dq, ld_d);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

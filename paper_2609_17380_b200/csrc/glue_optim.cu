@@ -375,7 +375,7 @@ extern "C" int det_swiglu_fwd(const det_bf16* gu, int rows, int F, det_bf16* h, 
   if (!aligned16(gu) || !aligned16(h)) return DET_ERR_ALIGN;
   size_t n = (size_t)rows * (F / 8);
   if (!n) return DET_OK;
-  k_swiglu_fwd<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(gu, rows, F, h);
+  k_swiglu_fwd<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(gu, rows, F, h);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -385,7 +385,7 @@ extern "C" int det_swiglu_bwd(const det_bf16* dh, const det_bf16* gu, int rows, 
   if (!aligned16(gu) || !aligned16(dh) || !aligned16(dgu)) return DET_ERR_ALIGN;
   size_t n = (size_t)rows * (F / 8);
   if (!n) return DET_OK;
-  k_swiglu_bwd<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(dh, gu, rows, F, dgu);
+  k_swiglu_bwd<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(dh, gu, rows, F, dgu);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -394,7 +394,7 @@ extern "C" int det_residual_add(const det_bf16* a, const det_bf16* b, size_t n, 
   if (n % 8) return DET_ERR_SHAPE;
   if (!aligned16(a) || !aligned16(b) || !aligned16(y)) return DET_ERR_ALIGN;
   if (!n) return DET_OK;
-  k_residual<<<(unsigned)((n / 8 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(a, b, n / 8, y);
+  k_residual<<<DET_L((unsigned)((n / 8 + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(a, b, n / 8, y);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -403,7 +403,7 @@ extern "C" int det_embed_fwd(const int32_t* tok, int T, const det_bf16* E, int V
   if (D % 8) return DET_ERR_SHAPE;
   if (!aligned16(E) || !aligned16(y)) return DET_ERR_ALIGN;
   if (!T) return DET_OK;
-  k_embed_fwd<<<T, 256, 0, (cudaStream_t)stream>>>(tok, E, V, D, y);
+  k_embed_fwd<<<DET_L(T), 256, 0, (cudaStream_t)stream>>>(tok, E, V, D, y);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -413,7 +413,7 @@ extern "C" int det_embed_bwd(const int32_t* tok, int T, const det_bf16* dy, int 
   if (!aligned16(dy) || !aligned16(dE)) return DET_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
   cudaMemsetAsync(dE, 0, (size_t)V * D * sizeof(float), st);
-  if (T) k_embed_bwd<<<T, 256, 0, st>>>(tok, T, dy, V, D, dE);
+  if (T) k_embed_bwd<<<DET_L(T), 256, 0, st>>>(tok, T, dy, V, D, dE);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -493,7 +493,7 @@ extern "C" int det_grad_accum_push(det_accum* st, const float* g, void* stream) 
   }
   if (dst_slot < 0) return DET_ERR_ARG;
   op.dst = st->bufs + (size_t)dst_slot * n;
-  if (n) k_accum<<<(unsigned)((n / 4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(op, n);
+  if (n) k_accum<<<DET_L((unsigned)((n / 4 + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(op, n);
   for (int l = 0; l < npop; ++l) st->free_mask |= (1ull << popped[l]);
   st->pushes++;
   DET_CHECK_LAUNCH();
@@ -509,7 +509,7 @@ extern "C" int det_grad_accum_result(det_accum* st, float* g_out, void* stream) 
   for (int s = 0; s < st->nstack; ++s) op.part[s] = st->bufs + (size_t)st->slot[st->nstack - 1 - s] * st->n;
   op.inv_rep = (float)(1.0 / (double)st->dp_replicate);
   op.dst = g_out;
-  if (st->n) k_accum_result<<<(unsigned)((st->n / 4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(op, st->n);
+  if (st->n) k_accum_result<<<DET_L((unsigned)((st->n / 4 + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(op, st->n);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -529,8 +529,8 @@ extern "C" int det_adamw_step(const det_adamw_desc* d, int pdtype, void* p, cons
   h.isb2 = (float)(1.0 / sqrt(bc2));
   h.decay = (float)(1.0 - d->lr * d->weight_decay);
   unsigned grid = (unsigned)((n + 1023) / 1024);
-  if (pdtype == DET_BF16) k_adamw<true><<<grid, 256, 0, (cudaStream_t)stream>>>(h, p, g, m, v, n);
-  else k_adamw<false><<<grid, 256, 0, (cudaStream_t)stream>>>(h, p, g, m, v, n);
+  if (pdtype == DET_BF16) k_adamw<true><<<DET_L(grid), 256, 0, (cudaStream_t)stream>>>(h, p, g, m, v, n);
+  else k_adamw<false><<<DET_L(grid), 256, 0, (cudaStream_t)stream>>>(h, p, g, m, v, n);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -544,7 +544,7 @@ extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host
   if (ws_bytes < det_tensor_hash_ws_bytes(nbytes) || !ws) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t nc = (nbytes + 65535) / 65536;
-  if (nc) k_sha_chunks<<<(unsigned)((nc + 63) / 64), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, (uint8_t*)ws);
+  if (nc) k_sha_chunks<<<DET_L((unsigned)((nc + 63) / 64)), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, (uint8_t*)ws);
   DET_CHECK_LAUNCH();
   uint8_t* host = (uint8_t*)malloc(nc * 32 + 8);
   if (!host) return DET_ERR_ARG;

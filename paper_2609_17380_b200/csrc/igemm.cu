@@ -364,7 +364,7 @@ static int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const EpiPar
   }
   const int tiles = (I / BM) * (J / BN);
   const int grid = tiles < sms ? tiles : sms;
-  k_igemm<BN, EPI><<<grid, GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
+  k_igemm<BN, EPI><<<DET_L(grid), GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
   if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
   return DET_OK;
 }

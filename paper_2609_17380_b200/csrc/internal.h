@@ -5,6 +5,9 @@
 #include <stdint.h>
 
 namespace det {
+// every kernel launch of the library passes its grid through DET_L, which counts it
+int note_launch();
+#define DET_L(grid) (det::note_launch(), (grid))
 // floats of scratch the multi-level tree sum needs for n elements
 size_t sum_ws_floats(size_t n);
 // out[0] = det_sum(x[0..n)) (squares: of x^2); launches on st, scratch in ws (sum_ws_floats(n) floats)

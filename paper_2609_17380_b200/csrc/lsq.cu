@@ -250,9 +250,9 @@ static int abs_mean_scale(const det_bf16* X, size_t n, float* out, int count, fl
   float* partial = ws;
   float* total = partial + align_up(c, 64);
   float* scratch = total + 64;
-  k_abs_chunk<<<(unsigned)c, 256, 0, st>>>(X, (long long)n, partial);
+  k_abs_chunk<<<DET_L((unsigned)c), 256, 0, st>>>(X, (long long)n, partial);
   sum_launch(partial, c, 0, total, scratch, st);
-  k_scale_finish<<<(count + 255) / 256 < 64 ? (count + 255) / 256 : 64, 256, 0, st>>>(total, (float)(1.0 / (double)n), out, count);
+  k_scale_finish<<<DET_L((count + 255) / 256 < 64 ? (count + 255) / 256 : 64), 256, 0, st>>>(total, (float)(1.0 / (double)n), out, count);
   return DET_OK;
 }
 extern "C" int det_lsq_weight_scale(const det_bf16* W, int N, int K, int per_tensor, float* s_w, void* ws,
@@ -265,7 +265,7 @@ extern "C" int det_lsq_weight_scale(const det_bf16* W, int N, int K, int per_ten
     if (!ws || ws_bytes < det_lsq_weight_scale_ws_bytes(N, K)) return DET_ERR_WORKSPACE;
     abs_mean_scale(W, (size_t)N * K, s_w, N, (float*)ws, st);
   } else {
-    k_wscale_rows<<<(N + 7) / 8, 256, 0, st>>>(W, N, K, (float)(1.0 / (double)K), s_w);
+    k_wscale_rows<<<DET_L((N + 7) / 8), 256, 0, st>>>(W, N, K, (float)(1.0 / (double)K), s_w);
   }
   DET_CHECK_LAUNCH();
   return DET_OK;
@@ -289,18 +289,18 @@ extern "C" int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int 
   if (qWt_bwd && (!ws || ws_bytes < 256)) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t n16 = (size_t)N * K / 16;
-  k_quantize<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(W, n16, K / 16, s_w, 1, qW);
+  k_quantize<<<DET_L((unsigned)((n16 + 255) / 256)), 256, 0, st>>>(W, n16, K / 16, s_w, 1, qW);
   if (qWt_bwd) {
     uint32_t* amax = (uint32_t*)ws;
     cudaMemsetAsync(amax, 0, 256, st);
     dim3 grid(K / 64, N / 128);
     if (hadamard_block) {
-      k_rot_cols<int8_t, 0, true><<<grid, 256, 0, st>>>(qW, N, K, amax, nullptr);
-      k_rot_cols<int8_t, 1, true><<<grid, 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rot_cols<int8_t, 0, true><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, nullptr);
+      k_rot_cols<int8_t, 1, true><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
     } else {
-      k_rot_cols<int8_t, 1, false><<<grid, 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rot_cols<int8_t, 1, false><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
     }
-    k_su_finish<<<1, 1, 0, st>>>(amax, hadamard_block != 0, s_u);
+    k_su_finish<<<DET_L(1), 1, 0, st>>>(amax, hadamard_block != 0, s_u);
   }
   DET_CHECK_LAUNCH();
   return DET_OK;
@@ -314,7 +314,7 @@ extern "C" int det_linear_fwd(const det_bf16* X, const int8_t* qW, const float* 
   if (!aligned16(X) || !aligned16(qW) || !aligned16(Y) || !aligned16(qX_save) || !aligned16(s_w)) return DET_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t n16 = (size_t)M * K / 16;
-  k_quantize<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(X, n16, K / 16, s_x, 0, qX_save);
+  k_quantize<<<DET_L((unsigned)((n16 + 255) / 256)), 256, 0, st>>>(X, n16, K / 16, s_x, 0, qX_save);
   DET_CHECK_LAUNCH();
   EpiParams ep = {};
   ep.out = Y; ep.s_x = s_x; ep.s_w = s_w;
@@ -362,18 +362,18 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   const unsigned g1 = (unsigned)((nblk + 7) / 8);
   dim3 gG(N / 64, M / 128), gZ(K / 64, M / 128);
   if (rot) {
-    k_rot_rows<0, true><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
-    k_rot_cols<uint16_t, 0, true><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
-    k_rot_cols<int8_t, 0, true><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, nullptr);
-    k_rot_rows<1, true><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
-    k_rot_cols<uint16_t, 1, true><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, GqT);
-    k_rot_cols<int8_t, 1, true><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+    k_rot_rows<0, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
+    k_rot_cols<uint16_t, 0, true><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rot_cols<int8_t, 0, true><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, nullptr);
+    k_rot_rows<1, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
+    k_rot_cols<uint16_t, 1, true><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rot_cols<int8_t, 1, true><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
   } else {
-    k_rot_rows<0, false><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
-    k_rot_cols<uint16_t, 0, false><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
-    k_rot_rows<1, false><<<g1, 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
-    k_rot_cols<uint16_t, 1, false><<<gG, 256, 0, st>>>(dY, M, N, amax + 1, GqT);
-    k_rot_cols<int8_t, 1, false><<<gZ, 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+    k_rot_rows<0, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
+    k_rot_cols<uint16_t, 0, false><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rot_rows<1, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
+    k_rot_cols<uint16_t, 1, false><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rot_cols<int8_t, 1, false><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
   }
   DET_CHECK_LAUNCH();
   const float rotf = rot ? 0x1p-7f : 1.0f;
@@ -384,7 +384,7 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   if (rc != DET_OK) return rc;
   const size_t np = (size_t)M * (K / 128);
   sum_launch(partial, np, 0, sscr, sscr + 64, st);
-  k_dsx_finish<<<1, 1, 0, st>>>(sscr, (float)(1.0 / sqrt((double)M * (double)K * 127.0)), ds_x);
+  k_dsx_finish<<<DET_L(1), 1, 0, st>>>(sscr, (float)(1.0 / sqrt((double)M * (double)K * 127.0)), ds_x);
   DET_CHECK_LAUNCH();
   // grad wrt W: [N,K] = G_q^T [N,M] . (Z_q^T [K,M])^T
   EpiParams ew = {};

@@ -312,11 +312,11 @@ extern "C" int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int row
   const float invD = (float)(1.0 / (double)D);
   dim3 grid((rows + 7) / 8);
   if (io == DET_BF16) {
-    if (D <= 2048) k_rmsnorm_fwd<true, 8><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
-    else k_rmsnorm_fwd<true, 0><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    if (D <= 2048) k_rmsnorm_fwd<true, 8><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    else k_rmsnorm_fwd<true, 0><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
   } else {
-    if (D <= 2048) k_rmsnorm_fwd<false, 8><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
-    else k_rmsnorm_fwd<false, 0><<<grid, 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    if (D <= 2048) k_rmsnorm_fwd<false, 8><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    else k_rmsnorm_fwd<false, 0><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
   }
   DET_CHECK_LAUNCH();
   return DET_OK;
@@ -340,18 +340,18 @@ extern "C" int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void
   const float invD = (float)(1.0 / (double)D);
   dim3 grid((rows + 7) / 8);
   if (io == DET_BF16) {
-    if (D <= 2048) k_rmsnorm_bwd<true, 8><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
-    else k_rmsnorm_bwd<true, 0><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    if (D <= 2048) k_rmsnorm_bwd<true, 8><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    else k_rmsnorm_bwd<true, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
   } else {
-    if (D <= 2048) k_rmsnorm_bwd<false, 8><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
-    else k_rmsnorm_bwd<false, 0><<<grid, 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    if (D <= 2048) k_rmsnorm_bwd<false, 8><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+    else k_rmsnorm_bwd<false, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
   }
   if (dgamma) {
     const int nb = (rows + 255) / 256;
     dim3 g2((D + 31) / 32, nb);
-    if (io == DET_BF16) k_dgamma_partial<true><<<g2, 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
-    else k_dgamma_partial<false><<<g2, 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
-    k_col_tree<<<(D + 127) / 128, 128, 0, st>>>((float*)ws, nb, D, dgamma);
+    if (io == DET_BF16) k_dgamma_partial<true><<<DET_L(g2), 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
+    else k_dgamma_partial<false><<<DET_L(g2), 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
+    k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>((float*)ws, nb, D, dgamma);
   }
   DET_CHECK_LAUNCH();
   return DET_OK;
@@ -376,10 +376,10 @@ extern "C" int det_xent_fwd(const float* logits, const int32_t* target, int rows
   float* scratch = sums + 128;
   const int nl = (V + 255) / 256;
   size_t sh = (size_t)(nl < 32 ? 32 : nl) * sizeof(float);
-  k_xent_fwd<<<rows, XT, sh, st>>>(logits, target, V, loss_row, lse, zsq, status_dev);
+  k_xent_fwd<<<DET_L(rows), XT, sh, st>>>(logits, target, V, loss_row, lse, zsq, status_dev);
   sum_launch(loss_row, (size_t)rows, 0, sums, scratch, st);
   sum_launch(zsq, (size_t)rows, 0, sums + 64, scratch, st);
-  k_xent_finish<<<1, 1, 0, st>>>(sums, sums + 64, (float)(1.0 / (double)rows), z_weight, loss_mean, z_mean);
+  k_xent_finish<<<DET_L(1), 1, 0, st>>>(sums, sums + 64, (float)(1.0 / (double)rows), z_weight, loss_mean, z_mean);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -390,7 +390,7 @@ extern "C" int det_xent_bwd(float* logits_inout, const int32_t* target, const fl
   if (V % 4) return DET_ERR_SHAPE;
   if (!aligned16(logits_inout)) return DET_ERR_ALIGN;
   dim3 grid((V / 4 + 255) / 256, rows < 65535 ? rows : 65535);
-  k_xent_bwd<<<grid, 256, 0, (cudaStream_t)stream>>>(logits_inout, target, lse, rows, V, z_weight, scale);
+  k_xent_bwd<<<DET_L(grid), 256, 0, (cudaStream_t)stream>>>(logits_inout, target, lse, rows, V, z_weight, scale);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

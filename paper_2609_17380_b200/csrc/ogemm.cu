@@ -154,7 +154,7 @@ extern "C" int det_lmhead_fwd(const det_bf16* H, const det_bf16* W, int M, int V
   if (K % 16 || V % 4) return DET_ERR_SHAPE;
   if (!aligned16(H) || !aligned16(W) || !aligned16(logits)) return DET_ERR_ALIGN;
   dim3 grid((V + OT - 1) / OT, (M + OT - 1) / OT);
-  k_ogemm<CONTIG, CONTIG, false, false><<<grid, 256, 0, (cudaStream_t)stream>>>(H, W, M, V, K, K, K, logits, V, 0);
+  k_ogemm<CONTIG, CONTIG, false, false><<<DET_L(grid), 256, 0, (cudaStream_t)stream>>>(H, W, M, V, K, K, K, logits, V, 0);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -167,10 +167,10 @@ extern "C" int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det
   cudaStream_t st = (cudaStream_t)stream;
   // dH[m,k] = sum over v ascending of bf16(dlogits[m,v]) * W[v,k]
   dim3 g1((K + OT - 1) / OT, (M + OT - 1) / OT);
-  k_ogemm<CONTIG, STRIDED, true, true><<<g1, 256, 0, st>>>(dlogits, W, M, K, V, V, K, dH, K, 0);
+  k_ogemm<CONTIG, STRIDED, true, true><<<DET_L(g1), 256, 0, st>>>(dlogits, W, M, K, V, V, K, dH, K, 0);
   // dW[v,k] (+)= sum over m ascending of bf16(dlogits[m,v]) * H[m,k]
   dim3 g2((K + OT - 1) / OT, (V + OT - 1) / OT);
-  k_ogemm<STRIDED, STRIDED, true, false><<<g2, 256, 0, st>>>(dlogits, H, V, K, M, V, K, dW, K, first_chunk ? 0 : 1);
+  k_ogemm<STRIDED, STRIDED, true, false><<<DET_L(g2), 256, 0, st>>>(dlogits, H, V, K, M, V, K, dW, K, first_chunk ? 0 : 1);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

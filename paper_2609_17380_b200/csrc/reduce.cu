@@ -10,6 +10,10 @@
 
 namespace det {
 
+static unsigned long long g_launches = 0;
+int note_launch() { ++g_launches; return 0; }
+unsigned long long launches() { return g_launches; }
+
 constexpr int SUM_CHUNK = 16384;
 
 template <bool SQ>
@@ -88,7 +92,7 @@ size_t sum_ws_floats(size_t n) {
 
 int sum_launch(const float* x, size_t n, int squares, float* out, float* ws, cudaStream_t st) {
   if (n == 0) { cudaMemsetAsync(out, 0, sizeof(float), st); return DET_OK; }
-  if (n == 1) { k_flush1<<<1, 1, 0, st>>>(x, out, squares); return DET_OK; }
+  if (n == 1) { k_flush1<<<DET_L(1), 1, 0, st>>>(x, out, squares); return DET_OK; }
   const float* src = x;
   long long cur = (long long)n;
   bool sq = squares != 0;
@@ -96,8 +100,8 @@ int sum_launch(const float* x, size_t n, int squares, float* out, float* ws, cud
   while (true) {
     long long c = nchunks(cur);
     float* dst = (c == 1) ? out : w;
-    if (sq) k_sum_chunk<true><<<(unsigned)c, 256, 0, st>>>(src, cur, dst);
-    else k_sum_chunk<false><<<(unsigned)c, 256, 0, st>>>(src, cur, dst);
+    if (sq) k_sum_chunk<true><<<DET_L((unsigned)c), 256, 0, st>>>(src, cur, dst);
+    else k_sum_chunk<false><<<DET_L((unsigned)c), 256, 0, st>>>(src, cur, dst);
     if (c == 1) break;
     w += align_up((size_t)c, 64);
     src = dst;
@@ -157,6 +161,8 @@ __global__ void k_prim(int op, const float* a, const float* b, float* out, size_
 
 using namespace det;
 
+extern "C" unsigned long long det_launch_count(void) { return det::launches(); }
+
 extern "C" int det_device_sm_count(void) {
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return DET_ERR_CUDA;
@@ -167,7 +173,7 @@ extern "C" int det_device_sm_count(void) {
 extern "C" int det_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream) {
   if (!a || !out || op < 0 || op > 9) return DET_ERR_ARG;
   if (n == 0) return DET_OK;
-  k_prim<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(op, a, b, out, n);
+  k_prim<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(op, a, b, out, n);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -203,7 +209,7 @@ extern "C" int det_grad_norm(const float* const* g_ptrs, const size_t* n_elems, 
   float* scratch = total + 64;
   for (int t = 0; t < ntensors; ++t) sum_launch(g_ptrs[t], n_elems[t], 1, per + t, scratch, st);
   sum_launch(per, (size_t)ntensors, 0, total, scratch, st);
-  k_norm_finish<<<1, 1, 0, st>>>(total, max_norm, norm_out, coef_out, status_dev);
+  k_norm_finish<<<DET_L(1), 1, 0, st>>>(total, max_norm, norm_out, coef_out, status_dev);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
@@ -212,7 +218,7 @@ extern "C" int det_scale_inplace(float* g, size_t n, const float* coef_dev, void
   if ((n && !g) || !coef_dev) return DET_ERR_ARG;
   if (n && !aligned16(g)) return DET_ERR_ALIGN;
   if (n == 0) return DET_OK;
-  k_scale<<<(unsigned)((n + 1023) / 1024), 256, 0, (cudaStream_t)stream>>>(g, n, coef_dev);
+  k_scale<<<DET_L((unsigned)((n + 1023) / 1024)), 256, 0, (cudaStream_t)stream>>>(g, n, coef_dev);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

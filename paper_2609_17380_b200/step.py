@@ -116,6 +116,30 @@ class Replay:
                   *[det.det_linear_bwd_ws_bytes(T, N, K) for (N, K) in ((3 * D, D), (D, D), (2 * Fh, D), (D, Fh))])
         self.ws = e(wsb + 4096, torch.uint8)
         self.losses = []
+        self.prof = None
+
+    # ---- optional per-call-site device timing (CUDA events on the launching stream) --------------------
+    class _Span:
+        def __init__(self, owner, name):
+            self.o, self.name = owner, name
+
+        def __enter__(self):
+            if self.o.prof is not None:
+                self.e0 = torch.cuda.Event(enable_timing=True)
+                self.e0.record()
+
+        def __exit__(self, *a):
+            if self.o.prof is not None:
+                e1 = torch.cuda.Event(enable_timing=True)
+                e1.record()
+                self.o.prof.setdefault(self.name, []).append((self.e0, e1))
+
+    def span(self, name):
+        return Replay._Span(self, name)
+
+    def prof_summary(self):
+        """name -> (launch groups, total ms); call after a synchronize."""
+        return {k: (len(v), sum(a.elapsed_time(b) for a, b in v)) for k, v in (self.prof or {}).items()}
 
     # ---- parameter access ------------------------------------------------------------------------------
     def p(self, name):
@@ -173,7 +197,8 @@ class Replay:
         sx = self.sx[4 * l + idx:4 * l + idx + 1]
         if calibrate:
             det.det_lsq_act_scale_init(X, M * d["K"], sx, self.ws)
-        det.det_linear_fwd(X, d["qW"], sx, d["s_w"], M, d["N"], d["K"], Y, qx, self.status)
+        with self.span("linear_fwd"):
+            det.det_linear_fwd(X, d["qW"], sx, d["s_w"], M, d["N"], d["K"], Y, qx, self.status)
 
     def forward(self, tokens_mb, calibrate=False):
         cfg = self.cfg
@@ -189,7 +214,8 @@ class Replay:
             det.det_rmsnorm_fwd(det.DET_BF16, a["x"], self.p("l%d.attn_norm" % l), T, D, 1e-6, a["n1"], a["rstd1"])
             self._linear(l, "w_qkv", 0, a["n1"], T, a["qkv"], a["qx_qkv"], calibrate)
             qp = a["qkv"].data_ptr()
-            det.det_attn_fwd(qp, qp + 2 * D, qp + 4 * D, 3 * D, B, H, S, a["att"], D, a["lse"])
+            with self.span("attn_fwd"):
+                det.det_attn_fwd(qp, qp + 2 * D, qp + 4 * D, 3 * D, B, H, S, a["att"], D, a["lse"])
             o = self.tmp[1][:T * D]
             self._linear(l, "w_o", 1, a["att"], T, o, a["qx_o"], calibrate)
             det.det_residual_add(a["x"], o, T * D, a["h"])
@@ -201,26 +227,31 @@ class Replay:
             det.det_residual_add(a["h"], dn, T * D, x)
         self.xf.copy_(x)
         det.det_rmsnorm_fwd(det.DET_BF16, self.xf, self.p("final_norm"), T, D, 1e-6, self.nf, self.rstdf)
-        det.det_lmhead_fwd(self.nf, self.p("lm_head"), T, V, D, self.logits)
-        det.det_xent_fwd(self.logits, self.lab, T, V, cfg.z_weight, self.loss_row, self.lse_x, self.loss_mean, self.z_mean,
-                         self.ws, self.status)
+        with self.span("lmhead_fwd"):
+            det.det_lmhead_fwd(self.nf, self.p("lm_head"), T, V, D, self.logits)
+        with self.span("xent_fwd"):
+            det.det_xent_fwd(self.logits, self.lab, T, V, cfg.z_weight, self.loss_row, self.lse_x, self.loss_mean,
+                             self.z_mean, self.ws, self.status)
 
     def _linear_bwd(self, l, w, idx, dY, X, qx, M, dX):
         d = self.lin[(l, w)]
         name = "l%d.%s" % (l, w)
         sx = self.sx[4 * l + idx:4 * l + idx + 1]
         ds = self.g(self.gmb, "l%d.s_x" % l)[idx:idx + 1]
-        det.det_linear_bwd(dY, X, qx, self.p(name), d["qWt"], sx, d["s_w"], d["s_u"], M, d["N"], d["K"],
-                           self.cfg.hadamard_block, dX, self.g(self.gmb, name), ds, self.ws, self.status)
+        with self.span("linear_bwd"):
+            det.det_linear_bwd(dY, X, qx, self.p(name), d["qWt"], sx, d["s_w"], d["s_u"], M, d["N"], d["K"],
+                               self.cfg.hadamard_block, dX, self.g(self.gmb, name), ds, self.ws, self.status)
 
     def backward(self):
         cfg = self.cfg
         D, Fh, V, L, T = cfg.d_model, cfg.ffn, cfg.vocab, cfg.n_layers, cfg.tokens_per_microbatch
         B, H, S = cfg.micro_batch, cfg.n_heads, cfg.seq
-        det.det_xent_bwd(self.logits, self.lab, self.lse_x, T, V, cfg.z_weight, 1.0 / T)
+        with self.span("xent_bwd"):
+            det.det_xent_bwd(self.logits, self.lab, self.lse_x, T, V, cfg.z_weight, 1.0 / T)
         t0, t1, t2 = self.tmp
         d_nf = t0[:T * D]
-        det.det_lmhead_bwd(self.logits, self.nf, self.p("lm_head"), T, V, D, d_nf, self.g(self.gmb, "lm_head"), 1)
+        with self.span("lmhead_bwd"):
+            det.det_lmhead_bwd(self.logits, self.nf, self.p("lm_head"), T, V, D, d_nf, self.g(self.gmb, "lm_head"), 1)
         dx = t1[:T * D]
         det.det_rmsnorm_bwd(det.DET_BF16, d_nf, self.xf, self.p("final_norm"), self.rstdf, T, D, dx,
                             self.g(self.gmb, "final_norm"), self.ws)
@@ -241,8 +272,9 @@ class Replay:
             self._linear_bwd(l, "w_o", 1, d_h, a["att"], a["qx_o"], T, d_att)
             d_qkv = t2[:T * 3 * D]
             qp, dp = a["qkv"].data_ptr(), d_qkv.data_ptr()
-            det.det_attn_bwd(d_att, qp, qp + 2 * D, qp + 4 * D, a["att"], a["lse"], 3 * D, D, B, H, S, dp, dp + 2 * D,
-                             dp + 4 * D, 3 * D, self.ws)
+            with self.span("attn_bwd"):
+                det.det_attn_bwd(d_att, qp, qp + 2 * D, qp + 4 * D, a["att"], a["lse"], 3 * D, D, B, H, S, dp, dp + 2 * D,
+                                 dp + 4 * D, 3 * D, self.ws)
             d_n1 = t0[:T * D]
             self._linear_bwd(l, "w_qkv", 0, d_qkv, a["n1"], a["qx_qkv"], T, d_n1)
             d_x1 = t2[:T * D]
@@ -284,7 +316,8 @@ class Replay:
     def step(self, tokens, per_tensor_hashes=True, want_losses=True):
         """tokens: device int32 [n_microbatches, micro_batch, seq+1] in mesh order.  One optimizer step."""
         cfg = self.cfg
-        self.prepare_weights()
+        with self.span("prepare_weights"):
+            self.prepare_weights()
         st = det.det_accum()
         det.det_grad_accum_init(st, cfg.mesh[0], cfg.mesh[1], cfg.mesh[2], self.n_grad, self.abufs)
         losses = torch.empty(tokens.shape[0], dtype=F32, device=self.dev)
@@ -292,10 +325,13 @@ class Replay:
             self.forward(tokens[mb])
             losses[mb:mb + 1].copy_(self.loss_mean)
             self.backward()
-            det.det_grad_accum_push(st, self.gmb)
+            with self.span("grad_accum"):
+                det.det_grad_accum_push(st, self.gmb)
         det.det_grad_accum_result(st, self.gout)
-        self.optimizer()
-        h = self.hashes(per_tensor_hashes)
+        with self.span("optimizer"):
+            self.optimizer()
+        with self.span("hash"):
+            h = self.hashes(per_tensor_hashes)
         res = {"hashes": h, "status": int(self.status.item())}
         if want_losses:
             ls = losses.cpu().numpy()
