@@ -66,6 +66,22 @@ int det_prim(int op, const float* a, const float* b, float* out, size_t n, void*
 size_t det_sum_ws_bytes(size_t n);
 int det_sum(const float* x, size_t n, int squares, float* out, void* ws, size_t ws_bytes, void* stream);
 
+/* det_sum for callers that cannot allocate.  The paper has no counterpart for this entry point; it exists for users
+ * of this library who may not call cudaMalloc: code running inside a host application that owns all device memory
+ * and passes in only input and output buffers, or a loop that must not block on the allocator's device-wide
+ * synchronisation.  Same result as det_sum, bit for bit, but the scratch is a fixed 256 KiB array inside the library
+ * image (held by every GPU that loads the library until the process exits), so the call allocates and frees nothing.
+ *  - n may be at most DET_SUM_STATIC_MAX_N (also returned by det_sum_static_max_n()); larger n returns DET_ERR_SHAPE
+ *    and launches nothing.
+ *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress with that device
+ *    current); make that first call before starting any stream capture.
+ *  - All calls on a device share the one array and it keeps what the last call left there.  Nothing in it needs to
+ *    start at zero.  Two calls that overlap on the GPU (different streams, no ordering between them) race on it and
+ *    give undefined results: order them. */
+#define DET_SUM_STATIC_MAX_N (1u << 29)
+size_t det_sum_static_max_n(void);
+int det_sum_static(const float* x, size_t n, int squares, float* out, void* stream);
+
 /* Global gradient norm and clip coefficient (Sec. 3.2 "Optimizer": clip to global l2 norm 1.0).
  * g_ptrs / n_elems are HOST arrays of ntensors device pointers / lengths in canonical parameter order.
  * per-tensor det_sum(g^2), then det_sum over the per-tensor sums, norm = sqrt(total),

@@ -101,6 +101,17 @@ def det_sum(x, n, squares, out, ws):
     _check("det_sum", load().det_sum(_ptr(x), C.c_size_t(n), C.c_int(squares), _ptr(out), *_ws(ws), _stream()))
 
 
+def det_sum_static_max_n():
+    lib = load()
+    lib.det_sum_static_max_n.restype = C.c_size_t
+    return lib.det_sum_static_max_n()
+
+
+def det_sum_static(x, n, squares, out):
+    """det_sum without a workspace argument: scratch lives in a fixed array inside the library (see det.h)."""
+    _check("det_sum_static", load().det_sum_static(_ptr(x), C.c_size_t(n), C.c_int(squares), _ptr(out), _stream()))
+
+
 def _tensor_table(tensors):
     ptrs = (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
     ns = (C.c_size_t * len(tensors))(*[t.numel() for t in tensors])
