@@ -166,9 +166,12 @@ __global__ void __launch_bounds__(256) k_accum(AccumOp op, size_t n) {
     if (op.last_shard) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) v[k] = fmul(v[k], op.inv_shard);
-      for (int l = 0; l < op.nlower; ++l) {
-        float4 t = *reinterpret_cast<const float4*>(op.lower[l] + i);
-        v[0] = fadd(t.x, v[0]); v[1] = fadd(t.y, v[1]); v[2] = fadd(t.z, v[2]); v[3] = fadd(t.w, v[3]);
+#pragma unroll
+      for (int l = 0; l < 8; ++l) {  // static indices: the parameter struct must stay in constant space
+        if (l < op.nlower) {
+          float4 t = *reinterpret_cast<const float4*>(op.lower[l] + i);
+          v[0] = fadd(t.x, v[0]); v[1] = fadd(t.y, v[1]); v[2] = fadd(t.z, v[2]); v[3] = fadd(t.w, v[3]);
+        }
       }
     }
   }
@@ -185,9 +188,12 @@ __global__ void __launch_bounds__(256) k_accum_result(ResultOp op, size_t n) {
   if (i >= n) return;
   float4 a = *reinterpret_cast<const float4*>(op.part[0] + i);
   float v[4] = {a.x, a.y, a.z, a.w};
-  for (int s = 1; s < op.n; ++s) {
-    float4 t = *reinterpret_cast<const float4*>(op.part[s] + i);
-    v[0] = fadd(t.x, v[0]); v[1] = fadd(t.y, v[1]); v[2] = fadd(t.z, v[2]); v[3] = fadd(t.w, v[3]);
+#pragma unroll
+  for (int s = 1; s < 34; ++s) {
+    if (s < op.n) {
+      float4 t = *reinterpret_cast<const float4*>(op.part[s] + i);
+      v[0] = fadd(t.x, v[0]); v[1] = fadd(t.y, v[1]); v[2] = fadd(t.z, v[2]); v[3] = fadd(t.w, v[3]);
+    }
   }
   *reinterpret_cast<float4*>(op.dst + i) =
       make_float4(fmul(v[0], op.inv_rep), fmul(v[1], op.inv_rep), fmul(v[2], op.inv_rep), fmul(v[3], op.inv_rep));

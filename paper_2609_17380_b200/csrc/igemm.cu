@@ -109,6 +109,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Tile order: the dimension with fewer tiles runs fastest, so that the CTAs resident at one time share the smaller
+// operand's tiles and the larger operand streams through L2 once.
+__device__ __forceinline__ void tile_origin(int tile, int tiles_i, int tiles_j, int bn, int& i0, int& j0) {
+  if (tiles_j <= tiles_i) { j0 = (tile % tiles_j) * bn; i0 = (tile / tiles_j) * BM; }
+  else { i0 = (tile % tiles_i) * BM; j0 = (tile / tiles_i) * bn; }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
     k_igemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, EpiParams ep, int I, int J,
@@ -151,7 +158,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int i0 = (tile % tiles_i) * BM, j0 = (tile / tiles_i) * BN;
+        int i0, j0;
+        tile_origin(tile, tiles_i, tiles_j, BN, i0, j0);
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
           mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
@@ -215,7 +223,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-      const int i0 = (tile % tiles_i) * BM, j0 = (tile / tiles_i) * BN;
+      int i0, j0;
+        tile_origin(tile, tiles_i, tiles_j, BN, i0, j0);
       if (!mbar_wait(&bar_tfull[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const int row = i0 + q * 32 + lane;

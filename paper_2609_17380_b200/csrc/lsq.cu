@@ -148,83 +148,84 @@ __global__ void __launch_bounds__(256) k_rot_rows(const uint16_t* __restrict__ d
   if (PASS == 0) {
 #pragma unroll
     for (int w = 16; w; w >>= 1) local = fmaxf(local, __shfl_xor_sync(0xffffffffu, local, w));
-    if (lane == 0 && local > 0.0f) atomicMax(amax, __float_as_uint(local));  // non-negative floats order as uints
+    // non-negative floats order as uints; the plain read filters out almost every atomic (the maximum only grows)
+    if (lane == 0 && local > 0.0f && __float_as_uint(local) > *reinterpret_cast<volatile uint32_t*>(amax))
+      atomicMax(amax, __float_as_uint(local));
   }
 }
 
 // (2) rotation along the row-index (strided) direction with a transposed int8 result:
 //     in [R, C] (bf16 for G = dY, int8 for Z = qX and U = qW)  ->  out int8 [C, R],
-//     out[c, r] = quantise(rotate_r(in[:, c]))[r].  A CTA owns a tile of 128 rows x 64 columns in shared
-//     memory; each butterfly stage touches disjoint pairs, so the per-element rounding order is fixed.
-template <typename TIN, int PASS, bool ROT>
-__global__ void __launch_bounds__(256) k_rot_cols(const TIN* __restrict__ in, int R, int C, uint32_t* __restrict__ amax,
-                                                  int8_t* __restrict__ outT) {
-  constexpr bool ISF = (sizeof(TIN) == 2);
-  constexpr int TC = 64;
-  __shared__ float tile[128][TC + 1];  // int path stores the int32 bit pattern
-  int* itile = reinterpret_cast<int*>(&tile[0][0]);
-  const int r0 = blockIdx.y * 128, c0 = blockIdx.x * TC;
-  // load: 128 rows x 64 cols; thread t reads 4 adjacent columns of 8 rows
-  for (int i = threadIdx.x; i < 128 * (TC / 4); i += 256) {
-    const int r = i / (TC / 4), c = (i % (TC / 4)) * 4;
-    if (ISF) {
-      uint2 u = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(in) + (size_t)(r0 + r) * C + c0 + c));
-      tile[r][c] = bflo(u.x); tile[r][c + 1] = bfhi(u.x); tile[r][c + 2] = bflo(u.y); tile[r][c + 3] = bfhi(u.y);
-    } else {
-      uint32_t u = __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(in) + (size_t)(r0 + r) * C + c0 + c));
+//     out[c, r] = quantise(rotate_r(in[:, c]))[r].  A thread owns one column of a 128-row block: 128 values in
+//     registers (a warp reads 32 adjacent columns of each row, i.e. whole 32/64-byte sectors), the seven butterfly
+//     stages run in registers, and the thread writes its 128 quantised values as one contiguous 128-byte run of the
+//     transposed output.  Each stage touches disjoint pairs, so the rounding order per element is fixed.
+template <bool ISF, int PASS, bool ROT>
+__global__ void __launch_bounds__(128) k_rotc(const void* __restrict__ in, int R, int C, uint32_t* __restrict__ amax,
+                                              int8_t* __restrict__ outT) {
+  const int col = blockIdx.x * 128 + threadIdx.x;
+  const int r0 = blockIdx.y * 128;
+  float vf[ISF ? 128 : 1];
+  int vi[ISF ? 1 : 128];
+  if (ISF) {
+    const uint16_t* p = reinterpret_cast<const uint16_t*>(in) + (size_t)r0 * C + col;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) itile[r * (TC + 1) + c + e] = (int)(int8_t)(u >> (8 * e));
-    }
+    for (int i = 0; i < 128; ++i) vf[i] = bf2f(__ldg(p + (size_t)i * C));
+  } else {
+    const int8_t* p = reinterpret_cast<const int8_t*>(in) + (size_t)r0 * C + col;
+#pragma unroll
+    for (int i = 0; i < 128; ++i) vi[i] = (int)__ldg(p + (size_t)i * C);
   }
-  __syncthreads();
   if (ROT) {
+#pragma unroll
     for (int h = 1; h < 128; h <<= 1) {
-      for (int i = threadIdx.x; i < 64 * TC; i += 256) {
-        const int c = i % TC, p = i / TC;                 // p-th pair of this stage
-        const int lo = ((p & ~(h - 1)) << 1) | (p & (h - 1));
-        if (ISF) {
-          float a = tile[lo][c], b = tile[lo + h][c];
-          tile[lo][c] = fadd(a, b); tile[lo + h][c] = fsub(a, b);
-        } else {
-          int a = itile[lo * (TC + 1) + c], b = itile[(lo + h) * (TC + 1) + c];
-          itile[lo * (TC + 1) + c] = a + b; itile[(lo + h) * (TC + 1) + c] = a - b;
+#pragma unroll
+      for (int i = 0; i < 128; ++i) {
+        if (!(i & h)) {
+          if (ISF) { const float a = vf[i], b = vf[i + h]; vf[i] = fadd(a, b); vf[i + h] = fsub(a, b); }
+          else { const int a = vi[i], b = vi[i + h]; vi[i] = a + b; vi[i + h] = a - b; }
         }
       }
-      __syncthreads();
     }
   }
   if (PASS == 0) {
     uint32_t local = 0;
-    for (int i = threadIdx.x; i < 128 * TC; i += 256) {
-      const int r = i / TC, c = i % TC;
-      if (ISF) local = max(local, __float_as_uint(fabsf(tile[r][c])));
-      else local = max(local, (uint32_t)abs(itile[r * (TC + 1) + c]));
+#pragma unroll
+    for (int i = 0; i < 128; ++i) {
+      if (ISF) local = max(local, __float_as_uint(fabsf(vf[i])));
+      else local = max(local, (uint32_t)abs(vi[i]));
     }
 #pragma unroll
     for (int w = 16; w; w >>= 1) local = max(local, __shfl_xor_sync(0xffffffffu, local, w));
-    if ((threadIdx.x & 31) == 0 && local) atomicMax(amax, local);
+    if ((threadIdx.x & 31) == 0 && local > *reinterpret_cast<volatile uint32_t*>(amax)) atomicMax(amax, local);
   } else {
-    float inv;
+    float inv = 0.0f;
     if (ISF) {
       const float am = __uint_as_float(amax[0]);
       inv = (am > 0.0f) ? fdiv(127.0f, am) : 0.0f;
-    } else {
+    } else if (ROT) {
       const int am = (int)amax[0];
       inv = (am > 0) ? fdiv(127.0f, __int2float_rn(am)) : 0.0f;
     }
-    // out[c0 + c, r0 .. r0+127]: thread writes 4 adjacent r (one 32-bit store); 32 threads cover a column
-    for (int i = threadIdx.x; i < TC * 32; i += 256) {
-      const int c = i / 32, r = (i % 32) * 4;
-      uint32_t o = 0;
+    uint4* dst = reinterpret_cast<uint4*>(outT + (size_t)col * R + r0);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        int8_t qv;
-        if (ISF) qv = quant1(tile[r + e][c], inv);
-        else if (ROT) qv = quant1(__int2float_rn(itile[(r + e) * (TC + 1) + c]), inv);
-        else qv = (int8_t)itile[(r + e) * (TC + 1) + c];
-        o |= ((uint32_t)(uint8_t)qv) << (8 * e);
+    for (int g = 0; g < 8; ++g) {
+      uint32_t w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t o = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i = g * 16 + k * 4 + e;
+          int8_t qv;
+          if (ISF) qv = quant1(vf[i], inv);
+          else if (ROT) qv = quant1(__int2float_rn(vi[i]), inv);
+          else qv = (int8_t)vi[i];
+          o |= ((uint32_t)(uint8_t)qv) << (8 * e);
+        }
+        w[k] = o;
       }
-      *reinterpret_cast<uint32_t*>(outT + (size_t)(c0 + c) * R + r0 + r) = o;
+      dst[g] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 }
@@ -293,12 +294,12 @@ extern "C" int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int 
   if (qWt_bwd) {
     uint32_t* amax = (uint32_t*)ws;
     cudaMemsetAsync(amax, 0, 256, st);
-    dim3 grid(K / 64, N / 128);
+    dim3 grid(K / 128, N / 128);
     if (hadamard_block) {
-      k_rot_cols<int8_t, 0, true><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, nullptr);
-      k_rot_cols<int8_t, 1, true><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rotc<false, 0, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, nullptr);
+      k_rotc<false, 1, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
     } else {
-      k_rot_cols<int8_t, 1, false><<<DET_L(grid), 256, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rotc<false, 1, false><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
     }
     k_su_finish<<<DET_L(1), 1, 0, st>>>(amax, hadamard_block != 0, s_u);
   }
@@ -360,20 +361,20 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   cudaMemsetAsync(amax, 0, 256, st);
   const size_t nblk = (size_t)M * (N / 128);
   const unsigned g1 = (unsigned)((nblk + 7) / 8);
-  dim3 gG(N / 64, M / 128), gZ(K / 64, M / 128);
+  dim3 gG(N / 128, M / 128), gZ(K / 128, M / 128);
   if (rot) {
     k_rot_rows<0, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
-    k_rot_cols<uint16_t, 0, true><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
-    k_rot_cols<int8_t, 0, true><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, nullptr);
+    k_rotc<true, 0, true><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rotc<false, 0, true><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, nullptr);
     k_rot_rows<1, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
-    k_rot_cols<uint16_t, 1, true><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, GqT);
-    k_rot_cols<int8_t, 1, true><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+    k_rotc<true, 1, true><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rotc<false, 1, true><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, ZqT);
   } else {
     k_rot_rows<0, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
-    k_rot_cols<uint16_t, 0, false><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    k_rotc<true, 0, false><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, nullptr);
     k_rot_rows<1, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
-    k_rot_cols<uint16_t, 1, false><<<DET_L(gG), 256, 0, st>>>(dY, M, N, amax + 1, GqT);
-    k_rot_cols<int8_t, 1, false><<<DET_L(gZ), 256, 0, st>>>(qX, M, K, amax + 2, ZqT);
+    k_rotc<true, 1, false><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_rotc<false, 1, false><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, ZqT);
   }
   DET_CHECK_LAUNCH();
   const float rotf = rot ? 0x1p-7f : 1.0f;

@@ -32,9 +32,151 @@ __device__ __forceinline__ void store8(void* p, size_t idx, const float v[8]) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// RMSNorm.  One warp per row; the row (up to 32 leaves) is held in registers between the reduction
-// and the normalisation when it has at most 8 leaves (D <= 2048), else it is read again.
+// RMSNorm.  One warp per row.  Rows of at most 2048 elements (8 leaves) are loaded completely into
+// registers first (16 independent 128-bit loads per lane), reduced, normalised and stored; longer rows
+// use the two-pass variant that reads the row again.
 // ------------------------------------------------------------------------------------------------
+template <bool BF>
+__global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
+                                                      int D, float eps, float invD, void* __restrict__ y,
+                                                      float* __restrict__ rstd) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= rows) return;
+  const size_t rb = (size_t)row * D;
+  float xr[8][8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = j * 256 + lane * 8;
+    if (e0 < D) load8<BF>(x, rb + e0, xr[j]);
+    else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xr[j][t] = 0.0f;
+    }
+  }
+  float mine = 0.0f;
+  const bool full = (D & 255) == 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float sq[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) sq[t] = fmul(xr[j][t], xr[j][t]);
+    const float t8 = tree8_full(sq);
+    const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
+    if (lane == j) mine = leaf;
+  }
+  const float ss = warp_tree(mine, 0, 256, D);
+  const float rs = fdiv(1.0f, fsqrt(fadd(fmul(ss, invD), eps)));
+  if (lane == 0) rstd[row] = rs;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = j * 256 + lane * 8;
+    if (e0 >= D) continue;
+    float o[8];
+    if (gamma) {
+      float g[8];
+      load8<BF>(gamma, e0, g);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = fmul(fmul(xr[j][t], rs), g[t]);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = fmul(xr[j][t], rs);
+    }
+    store8<BF>(y, rb + e0, o);
+  }
+}
+
+// Backward for rows of at most 2048 elements.  With DG, the CTA (8 adjacent rows) also leaves the column-wise
+// tree over its 8 rows of dy*xhat in partial8[blockIdx.x][D] (the first three levels of the row-direction tree).
+template <bool BF, bool DG>
+__global__ void __launch_bounds__(256) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
+                                                      const void* __restrict__ gamma, const float* __restrict__ rstd,
+                                                      int rows, int D, float invD, void* __restrict__ dx,
+                                                      float* __restrict__ partial8) {
+  extern __shared__ __align__(16) float srow[];  // DG: [8][D]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  const bool live = row < rows;
+  const size_t rb = (size_t)row * D;
+  float w[8][8], xh[8][8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = j * 256 + lane * 8;
+    if (live && e0 < D) {
+      load8<BF>(dy, rb + e0, w[j]);
+      load8<BF>(x, rb + e0, xh[j]);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { w[j][t] = 0.0f; xh[j][t] = 0.0f; }
+    }
+  }
+  const float rs = live ? rstd[row] : 0.0f;
+  float mine = 0.0f;
+  const bool full = (D & 255) == 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = j * 256 + lane * 8;
+    float pr[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) xh[j][t] = fmul(xh[j][t], rs);
+    if (DG && e0 < D) {
+      float dgt[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[j][t], xh[j][t]);
+      *reinterpret_cast<float4*>(&srow[warp * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
+      *reinterpret_cast<float4*>(&srow[warp * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
+    }
+    if (gamma && e0 < D) {
+      float g[8];
+      load8<BF>(gamma, e0, g);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) w[j][t] = fmul(w[j][t], g[t]);
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) pr[t] = fmul(w[j][t], xh[j][t]);
+    const float t8 = tree8_full(pr);
+    const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
+    if (lane == j) mine = leaf;
+  }
+  const float c = fmul(warp_tree(mine, 0, 256, D), invD);
+  if (live) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int e0 = j * 256 + lane * 8;
+      if (e0 >= D) continue;
+      float o[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[j][t], fmul(xh[j][t], c)));
+      store8<BF>(dx, rb + e0, o);
+    }
+  }
+  if (DG) {
+    __syncthreads();
+    const long long r0 = (long long)blockIdx.x * 8;
+    for (int col = threadIdx.x; col < D; col += 256) {
+      float v[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) v[r] = srow[r * D + col];
+      partial8[(size_t)blockIdx.x * D + col] = reg_tree<8>(v, r0, 1, rows);
+    }
+  }
+}
+// partial8 [nb8][D] (node = 8 rows) -> partial256 [nb256][D]: tree over 32 adjacent 8-row nodes per column
+__global__ void __launch_bounds__(256) k_colsum32(const float* __restrict__ partial8, int nb8, int rows, int D,
+                                                  float* __restrict__ partial256) {
+  const int col = blockIdx.x * 256 + threadIdx.x;
+  if (col >= D) return;
+  const int g = blockIdx.y;
+  float s[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int b = g * 32 + i;
+    s[i] = (b < nb8) ? partial8[(size_t)b * D + col] : 0.0f;
+  }
+  partial256[(size_t)g * D + col] = reg_tree<32>(s, (long long)g * 256, 8, rows);
+}
+
+// generic two-pass variants (rows longer than 2048 elements)
 template <bool BF, int NL>  // NL = leaves held in registers (0: re-read)
 __global__ void __launch_bounds__(256) k_rmsnorm_fwd(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
                                                      int D, float eps, float invD, void* __restrict__ y,
@@ -194,17 +336,23 @@ __global__ void __launch_bounds__(256) k_dgamma_partial(const void* __restrict__
     partial[(size_t)blockIdx.y * D + col] = reg_tree<8>(w, (long long)blockIdx.y * 256, 32, rows);
   }
 }
-// level-by-level tree over the nb row-block partials of each column, in place; result in row 0
-__global__ void k_col_tree(float* __restrict__ partial, int nb, int D, float* __restrict__ out) {
+// tree over the nb row-block partials (each a node of 256 rows) of every column, 32 nodes at a time from independent
+// loads; the partial buffer is reused for the intermediate levels
+__global__ void k_col_tree(float* __restrict__ partial, int nb, int D, float* __restrict__ out, int rows) {
   const int col = blockIdx.x * blockDim.x + threadIdx.x;
   if (col >= D) return;
   int n = nb;
+  long long stride = 256;
   while (n > 1) {
-    int m = (n + 1) >> 1;
-    for (int i = 0; i < (n >> 1); ++i)
-      partial[(size_t)i * D + col] = fadd(partial[(size_t)(2 * i) * D + col], partial[(size_t)(2 * i + 1) * D + col]);
-    if (n & 1) partial[(size_t)(m - 1) * D + col] = partial[(size_t)(n - 1) * D + col];
-    n = m;
+    const int groups = (n + 31) / 32;
+    for (int g = 0; g < groups; ++g) {
+      float s[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) s[i] = (g * 32 + i < n) ? partial[(size_t)(g * 32 + i) * D + col] : 0.0f;
+      partial[(size_t)g * D + col] = reg_tree<32>(s, (long long)g * 32 * stride, stride, rows);
+    }
+    n = groups;
+    stride *= 32;
   }
   out[col] = partial[col];
 }
@@ -312,10 +460,10 @@ extern "C" int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int row
   const float invD = (float)(1.0 / (double)D);
   dim3 grid((rows + 7) / 8);
   if (io == DET_BF16) {
-    if (D <= 2048) k_rmsnorm_fwd<true, 8><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    if (D <= 2048) k_rmsnorm_fwd8<true><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
     else k_rmsnorm_fwd<true, 0><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
   } else {
-    if (D <= 2048) k_rmsnorm_fwd<false, 8><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
+    if (D <= 2048) k_rmsnorm_fwd8<false><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
     else k_rmsnorm_fwd<false, 0><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
   }
   DET_CHECK_LAUNCH();
@@ -323,7 +471,32 @@ extern "C" int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int row
 }
 
 extern "C" size_t det_rmsnorm_bwd_ws_bytes(int rows, int D) {
-  return align_up((size_t)((rows + 255) / 256) * (size_t)D * sizeof(float), 256) + 256;
+  const size_t nb8 = (size_t)((rows + 7) / 8), nb256 = (size_t)((rows + 255) / 256);
+  return align_up(nb8 * (size_t)D * sizeof(float), 256) + align_up(nb256 * (size_t)D * sizeof(float), 256) + 256;
+}
+
+template <bool BF>
+static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma, const float* rstd, int rows, int D,
+                               float invD, void* dx, float* dgamma, float* ws, cudaStream_t st) {
+  dim3 grid((rows + 7) / 8);
+  if (!dgamma) {
+    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
+    return DET_OK;
+  }
+  static bool cfg = false;
+  if (!cfg) {
+    if (cudaFuncSetAttribute(k_rmsnorm_bwd8<BF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 2048 * 4) != cudaSuccess)
+      return DET_ERR_CUDA;
+    cfg = true;
+  }
+  const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
+  float* partial8 = ws;
+  float* partial256 = ws + align_up((size_t)nb8 * D, 64);
+  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 256, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
+  dim3 g2((D + 255) / 256, nb256);
+  k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256);
+  k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>(partial256, nb256, D, dgamma, rows);
+  return DET_OK;
 }
 
 extern "C" int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void* gamma, const float* rstd, int rows,
@@ -331,27 +504,29 @@ extern "C" int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void
   if (!dy || !x || !rstd || !dx || rows < 0 || D <= 0 || (io != DET_F32 && io != DET_BF16)) return DET_ERR_ARG;
   if (D % 8 || D > 8192) return DET_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || (gamma && !aligned16(gamma))) return DET_ERR_ALIGN;
-  if (dgamma && (!ws || ws_bytes < det_rmsnorm_bwd_ws_bytes(rows, D))) return DET_ERR_WORKSPACE;
+  if (dgamma && (!ws || !aligned16(ws) || ws_bytes < det_rmsnorm_bwd_ws_bytes(rows, D))) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   if (rows == 0) {
     if (dgamma) cudaMemsetAsync(dgamma, 0, (size_t)D * sizeof(float), st);
     return DET_OK;
   }
   const float invD = (float)(1.0 / (double)D);
-  dim3 grid((rows + 7) / 8);
-  if (io == DET_BF16) {
-    if (D <= 2048) k_rmsnorm_bwd<true, 8><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
-    else k_rmsnorm_bwd<true, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
-  } else {
-    if (D <= 2048) k_rmsnorm_bwd<false, 8><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
-    else k_rmsnorm_bwd<false, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+  if (D <= 2048) {
+    int rc = (io == DET_BF16) ? rmsnorm_bwd8_launch<true>(dy, x, gamma, rstd, rows, D, invD, dx, dgamma, (float*)ws, st)
+                              : rmsnorm_bwd8_launch<false>(dy, x, gamma, rstd, rows, D, invD, dx, dgamma, (float*)ws, st);
+    if (rc != DET_OK) return rc;
+    DET_CHECK_LAUNCH();
+    return DET_OK;
   }
+  dim3 grid((rows + 7) / 8);
+  if (io == DET_BF16) k_rmsnorm_bwd<true, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
+  else k_rmsnorm_bwd<false, 0><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx);
   if (dgamma) {
     const int nb = (rows + 255) / 256;
     dim3 g2((D + 31) / 32, nb);
     if (io == DET_BF16) k_dgamma_partial<true><<<DET_L(g2), 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
     else k_dgamma_partial<false><<<DET_L(g2), 256, 0, st>>>(dy, x, rstd, rows, D, (float*)ws);
-    k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>((float*)ws, nb, D, dgamma);
+    k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>((float*)ws, nb, D, dgamma, rows);
   }
   DET_CHECK_LAUNCH();
   return DET_OK;
