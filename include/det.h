@@ -159,7 +159,7 @@ int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, i
 int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S,
                  det_bf16* out, int ld_out, float* lse, void* stream);
 /* dq, dk, dv with leading dimension ld_d; every contraction is a sequential ascending sum from +0.
- * ws holds the bf16 dS matrix: B*H*S*S*2 bytes + B*H*S*4 bytes. */
+ * ws holds bf16(P) and bf16(dS), [B*H, S, S] each, and Delta [B*H, S]: see det_attn_bwd_ws_bytes. */
 size_t det_attn_bwd_ws_bytes(int B, int H, int S);
 int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,
                  const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq, det_bf16* dk,
@@ -180,7 +180,7 @@ int det_embed_bwd(const int32_t* tok, int T, const det_bf16* dy, int V, int D, f
  * logits[m,n] = sequential-k f32 sum from +0 of the exact products H[m,k] W[n,k].  K % 16 == 0. */
 int det_lmhead_fwd(const det_bf16* H, const det_bf16* W, int M, int V, int K, float* logits, void* stream);
 /* dlogits is rounded to bf16 first.  dH bf16 [M,K]: sum over the vocabulary ascending.  dW f32 [V,K]: sum over
- * tokens ascending, continuing from the value already in dW unless first_chunk != 0. */
+ * tokens ascending, continuing from the value already in dW unless first_chunk != 0.  V % 16 == 0, M % 8 == 0. */
 int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH,
                    float* dW, int first_chunk, void* stream);
 

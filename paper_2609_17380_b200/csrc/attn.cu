@@ -8,8 +8,7 @@
 // Backward: P = exp(S - L) recomputed; dV, dK (per key) and dQ (per query) are single accumulators fed in
 // ascending order of the contraction index; bf16(dS) goes through global scratch from the dK/dV kernel to
 // the dQ kernel, so nothing is accumulated with atomics.
-#include "common.cuh"
-#include "internal.h"
+#include "ogemm_core.cuh"
 
 namespace det {
 
@@ -212,219 +211,90 @@ __global__ void __launch_bounds__(256) k_attn_delta(const uint16_t* __restrict__
   if (lane == 0) delta[w] = t;
 }
 
-constexpr int BT = 64;        // tile edge for the backward
-constexpr int LN = DH + 4;    // row pitch of [row][dim] tiles
-constexpr int LP = BT + 4;    // row pitch of [query][key] tiles
-constexpr size_t DKDV_SMEM = (size_t)(4 * BT * LN + 2 * BT * LP + 2 * BT) * sizeof(float);
-constexpr size_t DQ_SMEM = (size_t)(BT * LN + BT * LP) * sizeof(float);
-
-__device__ __forceinline__ void load_tile_nat(float (*dst)[LN], const uint16_t* base, int ld, int r0, int S) {
-  for (int idx = threadIdx.x; idx < BT * 16; idx += 256) {
-    const int r = idx >> 4, ch = idx & 15;
-    float t[8];
-    if (r0 + r < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(base + (size_t)(r0 + r) * ld + ch * 8)), t);
-    else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) t[e] = 0.0f;
-    }
-    *reinterpret_cast<float4*>(&dst[r][ch * 8]) = make_float4(t[0], t[1], t[2], t[3]);
-    *reinterpret_cast<float4*>(&dst[r][ch * 8 + 4]) = make_float4(t[4], t[5], t[6], t[7]);
-  }
-}
-
-// CTA = 64 keys of one (batch, head); loops over query tiles in ascending order
+// S = q.k^T and dP = dO.v^T for one 128 x 128 tile of one (batch, head), both sequential over the 128 head
+// dimensions; then P = exp(S*scale - L), dS = P (dP - Delta) scale, and bf16(P), bf16(dS) go to global scratch
+// [b*H+h][query][key] for the three gradient contractions.  Tiles above the diagonal are skipped and never read.
+constexpr size_t SDP_SMEM = (size_t)4 * 2 * OK * (OT + 4) * sizeof(float);
 __global__ void __launch_bounds__(256, 1)
-    k_attn_dkdv(const uint16_t* __restrict__ dout, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                const uint16_t* __restrict__ v, const float* __restrict__ lse, const float* __restrict__ delta, int ld,
-                int ld_out, int H, int S, uint16_t* __restrict__ dk, uint16_t* __restrict__ dv, int ld_d,
-                uint16_t* __restrict__ dS) {
-  extern __shared__ __align__(16) float sm[];
-  float(*Kn)[LN] = reinterpret_cast<float(*)[LN]>(sm);
-  float(*Vn)[LN] = reinterpret_cast<float(*)[LN]>(sm + BT * LN);
-  float(*Qn)[LN] = reinterpret_cast<float(*)[LN]>(sm + 2 * BT * LN);
-  float(*On)[LN] = reinterpret_cast<float(*)[LN]>(sm + 3 * BT * LN);
-  float(*Pt)[LP] = reinterpret_cast<float(*)[LP]>(sm + 4 * BT * LN);
-  float(*St)[LP] = reinterpret_cast<float(*)[LP]>(sm + 4 * BT * LN + BT * LP);
-  float* Ls = sm + 4 * BT * LN + 2 * BT * LP;
-  float* Ds = Ls + BT;
-  const int jb = blockIdx.x;  // small jb = most query tiles; blocks are issued in that order
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int j0 = jb * BT;
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    k_attn_sdp(const uint16_t* __restrict__ dout, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+               const uint16_t* __restrict__ v, const float* __restrict__ lse, const float* __restrict__ delta, int ld,
+               int ld_out, int H, int S, uint16_t* __restrict__ Pt, uint16_t* __restrict__ dSt) {
+  const int jt = blockIdx.x, it = blockIdx.y;
+  if (jt > it) return;
+  extern __shared__ __align__(16) unsigned char osm[];
+  typedef float(*Slab)[OK][OT + 4];
+  Slab Qs = reinterpret_cast<Slab>(osm);
+  Slab Os = reinterpret_cast<Slab>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
+  Slab Ks = reinterpret_cast<Slab>(osm + (size_t)4 * OK * (OT + 4) * sizeof(float));
+  Slab Vs = reinterpret_cast<Slab>(osm + (size_t)6 * OK * (OT + 4) * sizeof(float));
+  const int b = blockIdx.z / H, h = blockIdx.z % H;
+  const int i0 = it * OT, j0 = jt * OT;
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
   const size_t row0 = (size_t)b * S;
-  const size_t bh = (size_t)b * H + h;
-  load_tile_nat(Kn, k + row0 * ld + (size_t)h * DH, ld, j0, S);
-  load_tile_nat(Vn, v + row0 * ld + (size_t)h * DH, ld, j0, S);
-  float dvv[4][8], dkk[4][8];
+  const uint16_t* qp = q + row0 * ld + (size_t)h * DH;
+  const uint16_t* kp = k + row0 * ld + (size_t)h * DH;
+  const uint16_t* vp = v + row0 * ld + (size_t)h * DH;
+  const uint16_t* op = dout + row0 * ld_out + (size_t)h * DH;
+  float2 sa[8][4], da[8][4];
 #pragma unroll
-  for (int e = 0; e < 4; ++e)
+  for (int a = 0; a < 8; ++a)
 #pragma unroll
-    for (int c = 0; c < 8; ++c) { dvv[e][c] = 0.0f; dkk[e][c] = 0.0f; }
-  const int nt = S / BT;
-  for (int it = jb; it < nt; ++it) {
-    const int i0 = it * BT;
-    __syncthreads();
-    load_tile_nat(Qn, q + row0 * ld + (size_t)h * DH, ld, i0, S);
-    load_tile_nat(On, dout + row0 * ld_out + (size_t)h * DH, ld_out, i0, S);
-    if (tid < BT) { Ls[tid] = lse[bh * S + i0 + tid]; Ds[tid] = delta[bh * S + i0 + tid]; }
-    __syncthreads();
-    // S = q.k and dP = dO.v, thread = queries ty+16e x keys tx+16f, sequential over the 128 dims
-    float s[4][4], dp[4][4];
+    for (int c = 0; c < 4; ++c) { sa[a][c] = make_float2(0.f, 0.f); da[a][c] = make_float2(0.f, 0.f); }
+  float vq[8], vo[8], vk[8], vv[8];
+  slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, 0, vq);
+  slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, 0, vo);
+  slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, 0, vk);
+  slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, 0, vv);
+  slab_store<CONTIG, OT>(Qs[0], vq); slab_store<CONTIG, OT>(Os[0], vo);
+  slab_store<CONTIG, OT>(Ks[0], vk); slab_store<CONTIG, OT>(Vs[0], vv);
+  int tiny = __syncthreads_or(tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv));
+  constexpr int NS = DH / OK;
+  for (int s = 0; s < NS; ++s) {
+    const int cur = s & 1;
+    if (s + 1 < NS) {
+      slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, (s + 1) * OK, vq);
+      slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, (s + 1) * OK, vo);
+      slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, (s + 1) * OK, vk);
+      slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, (s + 1) * OK, vv);
+    }
+    if (tiny) { slab_mac<false, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<false, OT>(Os[cur], Vs[cur], ty, tx, da); }
+    else { slab_mac<true, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<true, OT>(Os[cur], Vs[cur], ty, tx, da); }
+    bool nt = false;
+    if (s + 1 < NS) {
+      slab_store<CONTIG, OT>(Qs[cur ^ 1], vq); slab_store<CONTIG, OT>(Os[cur ^ 1], vo);
+      slab_store<CONTIG, OT>(Ks[cur ^ 1], vk); slab_store<CONTIG, OT>(Vs[cur ^ 1], vv);
+      nt = tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv);
+    }
+    tiny = __syncthreads_or(nt);
+  }
+  const size_t bh = (size_t)blockIdx.z;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
+  for (int a = 0; a < 8; ++a) {
+    const int i = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+    if (i >= S) continue;
+    const float L = lse[bh * S + i], dl = delta[bh * S + i];
 #pragma unroll
-      for (int f = 0; f < 4; ++f) { s[e][f] = 0.0f; dp[e][f] = 0.0f; }
-#pragma unroll 2
-    for (int d = 0; d < DH; d += 4) {
-      float4 qa[4], ka[4];
+    for (int g = 0; g < 2; ++g) {
+      const int jb = j0 + g * 64 + tx * 4;
+      if (jb >= S) continue;
+      const float sv[4] = {sa[a][2 * g].x, sa[a][2 * g].y, sa[a][2 * g + 1].x, sa[a][2 * g + 1].y};
+      const float dv4[4] = {da[a][2 * g].x, da[a][2 * g].y, da[a][2 * g + 1].x, da[a][2 * g + 1].y};
+      float pv[4], dsv[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        qa[e] = *reinterpret_cast<const float4*>(&Qn[ty + 16 * e][d]);
-        ka[e] = *reinterpret_cast<const float4*>(&Kn[tx + 16 * e][d]);
+        pv[e] = 0.0f; dsv[e] = 0.0f;
+        if (jb + e <= i) {
+          pv[e] = det_exp(fsub(fmul(sv[e], ATT_SCALE), L));
+          dsv[e] = fmul(fmul(pv[e], fsub(dv4[e], dl)), ATT_SCALE);
+        }
       }
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-#pragma unroll
-        for (int f = 0; f < 4; ++f) {
-          s[e][f] = fadd(s[e][f], fmul(qa[e].x, ka[f].x));
-          s[e][f] = fadd(s[e][f], fmul(qa[e].y, ka[f].y));
-          s[e][f] = fadd(s[e][f], fmul(qa[e].z, ka[f].z));
-          s[e][f] = fadd(s[e][f], fmul(qa[e].w, ka[f].w));
-        }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        qa[e] = *reinterpret_cast<const float4*>(&On[ty + 16 * e][d]);
-        ka[e] = *reinterpret_cast<const float4*>(&Vn[tx + 16 * e][d]);
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-#pragma unroll
-        for (int f = 0; f < 4; ++f) {
-          dp[e][f] = fadd(dp[e][f], fmul(qa[e].x, ka[f].x));
-          dp[e][f] = fadd(dp[e][f], fmul(qa[e].y, ka[f].y));
-          dp[e][f] = fadd(dp[e][f], fmul(qa[e].z, ka[f].z));
-          dp[e][f] = fadd(dp[e][f], fmul(qa[e].w, ka[f].w));
-        }
+      const size_t off = (bh * S + i) * S + jb;
+      uint2 u;
+      u.x = pack_bf2(pv[0], pv[1]); u.y = pack_bf2(pv[2], pv[3]);
+      *reinterpret_cast<uint2*>(Pt + off) = u;
+      u.x = pack_bf2(dsv[0], dsv[1]); u.y = pack_bf2(dsv[2], dsv[3]);
+      *reinterpret_cast<uint2*>(dSt + off) = u;
     }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int il = ty + 16 * e;
-      const float L = Ls[il], dl = Ds[il];
-#pragma unroll
-      for (int f = 0; f < 4; ++f) {
-        const int jl = tx + 16 * f;
-        float p = 0.0f, ds = 0.0f;
-        if (j0 + jl <= i0 + il) {
-          p = det_exp(fsub(fmul(s[e][f], ATT_SCALE), L));
-          ds = fmul(fmul(p, fsub(dp[e][f], dl)), ATT_SCALE);
-        }
-        Pt[il][jl] = bf2f(f2bf(p));
-        St[il][jl] = bf2f(f2bf(ds));
-      }
-    }
-    __syncthreads();
-    // bf16(dS) tile to global scratch for the dQ kernel: row = tid/4, 16 columns
-    {
-      const int r = tid >> 2, c0 = (tid & 3) * 16;
-      uint32_t w[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) w[e] = pack_bf2(St[r][c0 + 2 * e], St[r][c0 + 2 * e + 1]);
-      uint4* dst = reinterpret_cast<uint4*>(dS + (bh * S + i0 + r) * S + j0 + c0);
-      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-    }
-    // dV += P~^T dO, dK += dS~^T q: thread = keys tx+16e x dims {4ty.., 64+4ty..}, queries ascending
-#pragma unroll 2
-    for (int i = 0; i < BT; ++i) {
-      float pa[4], sa[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) { pa[e] = Pt[i][tx + 16 * e]; sa[e] = St[i][tx + 16 * e]; }
-      const float4 o0 = *reinterpret_cast<const float4*>(&On[i][ty * 4]);
-      const float4 o1 = *reinterpret_cast<const float4*>(&On[i][64 + ty * 4]);
-      const float4 q0v = *reinterpret_cast<const float4*>(&Qn[i][ty * 4]);
-      const float4 q1v = *reinterpret_cast<const float4*>(&Qn[i][64 + ty * 4]);
-      const float ob[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
-      const float qbv[8] = {q0v.x, q0v.y, q0v.z, q0v.w, q1v.x, q1v.y, q1v.z, q1v.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          dvv[e][c] = fadd(dvv[e][c], fmul(pa[e], ob[c]));
-          dkk[e][c] = fadd(dkk[e][c], fmul(sa[e], qbv[c]));
-        }
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const size_t r = (row0 + j0 + tx + 16 * e) * ld_d + (size_t)h * DH;
-    uint2 a, c;
-    a.x = pack_bf2(dvv[e][0], dvv[e][1]); a.y = pack_bf2(dvv[e][2], dvv[e][3]);
-    c.x = pack_bf2(dvv[e][4], dvv[e][5]); c.y = pack_bf2(dvv[e][6], dvv[e][7]);
-    *reinterpret_cast<uint2*>(dv + r + ty * 4) = a;
-    *reinterpret_cast<uint2*>(dv + r + 64 + ty * 4) = c;
-    a.x = pack_bf2(dkk[e][0], dkk[e][1]); a.y = pack_bf2(dkk[e][2], dkk[e][3]);
-    c.x = pack_bf2(dkk[e][4], dkk[e][5]); c.y = pack_bf2(dkk[e][6], dkk[e][7]);
-    *reinterpret_cast<uint2*>(dk + r + ty * 4) = a;
-    *reinterpret_cast<uint2*>(dk + r + 64 + ty * 4) = c;
-  }
-}
-
-// CTA = 64 queries; dQ_ic = sum over keys ascending of dS~_ij k_jc
-__global__ void __launch_bounds__(256, 1)
-    k_attn_dq(const uint16_t* __restrict__ k, const uint16_t* __restrict__ dS, int ld, int H, int S,
-              uint16_t* __restrict__ dq, int ld_d) {
-  extern __shared__ __align__(16) float sm[];
-  float(*Kn)[LN] = reinterpret_cast<float(*)[LN]>(sm);
-  float(*St)[LP] = reinterpret_cast<float(*)[LP]>(sm + BT * LN);
-  const int ib = gridDim.x - 1 - blockIdx.x;
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int i0 = ib * BT;
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-  const size_t row0 = (size_t)b * S;
-  const size_t bh = (size_t)b * H + h;
-  float acc[4][8];
-#pragma unroll
-  for (int e = 0; e < 4; ++e)
-#pragma unroll
-    for (int c = 0; c < 8; ++c) acc[e][c] = 0.0f;
-  for (int jt = 0; jt <= ib; ++jt) {
-    const int j0 = jt * BT;
-    __syncthreads();
-    load_tile_nat(Kn, k + row0 * ld + (size_t)h * DH, ld, j0, S);
-    {
-      const int r = tid >> 2, c0 = (tid & 3) * 16;
-      const uint4* src = reinterpret_cast<const uint4*>(dS + (bh * S + i0 + r) * S + j0 + c0);
-      float t[8];
-      unpack8a(__ldg(src), t);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) St[r][c0 + e] = t[e];
-      unpack8a(__ldg(src + 1), t);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) St[r][c0 + 8 + e] = t[e];
-    }
-    __syncthreads();
-#pragma unroll 2
-    for (int j = 0; j < BT; ++j) {
-      float sa[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) sa[e] = St[ty + 16 * e][j];
-      const float4 k0 = *reinterpret_cast<const float4*>(&Kn[j][tx * 4]);
-      const float4 k1 = *reinterpret_cast<const float4*>(&Kn[j][64 + tx * 4]);
-      const float kb[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-#pragma unroll
-        for (int c = 0; c < 8; ++c) acc[e][c] = fadd(acc[e][c], fmul(sa[e], kb[c]));
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const size_t r = (row0 + i0 + ty + 16 * e) * ld_d + (size_t)h * DH;
-    uint2 a, c;
-    a.x = pack_bf2(acc[e][0], acc[e][1]); a.y = pack_bf2(acc[e][2], acc[e][3]);
-    c.x = pack_bf2(acc[e][4], acc[e][5]); c.y = pack_bf2(acc[e][6], acc[e][7]);
-    *reinterpret_cast<uint2*>(dq + r + tx * 4) = a;
-    *reinterpret_cast<uint2*>(dq + r + 64 + tx * 4) = c;
   }
 }
 
@@ -450,31 +320,49 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
 }
 
 extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int S) {
-  return align_up((size_t)B * H * S * S * 2, 256) + align_up((size_t)B * H * S * 4, 256);
+  return 2 * align_up((size_t)B * H * S * S * 2, 256) + align_up((size_t)B * H * S * 4, 256);
 }
 
 extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
                             const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq,
                             det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes, void* stream) {
   if (!dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv || B <= 0 || H <= 0 || S <= 0) return DET_ERR_ARG;
-  if (S % 64 || ld % 8 || ld_out % 8 || ld_d % 8 || H > 65535 || B > 65535) return DET_ERR_SHAPE;
+  if (S % 64 || ld % 8 || ld_out % 8 || ld_d % 8 || (long long)B * H > 65535) return DET_ERR_SHAPE;
   if (!aligned16(dout) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
     return DET_ERR_ALIGN;
   if (!ws || ws_bytes < det_attn_bwd_ws_bytes(B, H, S)) return DET_ERR_WORKSPACE;
   static bool cfg = false;
   if (!cfg) {
-    if (set_smem((const void*)k_attn_dkdv, DKDV_SMEM) || set_smem((const void*)k_attn_dq, DQ_SMEM)) return DET_ERR_CUDA;
+    if (set_smem((const void*)k_attn_sdp, SDP_SMEM)) return DET_ERR_CUDA;
     cfg = true;
   }
   cudaStream_t st = (cudaStream_t)stream;
-  uint16_t* dS = (uint16_t*)ws;
-  float* delta = (float*)((uint8_t*)ws + align_up((size_t)B * H * S * S * 2, 256));
+  const size_t mat = align_up((size_t)B * H * S * S * 2, 256);
+  uint16_t* Pt = (uint16_t*)ws;
+  uint16_t* dSt = (uint16_t*)((uint8_t*)ws + mat);
+  float* delta = (float*)((uint8_t*)ws + 2 * mat);
   const size_t nrows = (size_t)B * H * S;
   k_attn_delta<<<DET_L((unsigned)((nrows + 7) / 8)), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
-  dim3 grid(S / BT, H, B);
-  k_attn_dkdv<<<DET_L(grid), 256, DKDV_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, S, dk, dv, ld_d, dS);
-  k_attn_dq<<<DET_L(grid), 256, DQ_SMEM, st>>>(k, dS, ld, H, S, dq, ld_d);
+  const int nt = (S + OT - 1) / OT;
+  dim3 grid(nt, nt, B * H);
+  k_attn_sdp<<<DET_L(grid), 256, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, S, Pt, dSt);
+  DET_CHECK_LAUNCH();
+  // dV[j,c] = sum over queries i >= j ascending of P~[i,j] dO[i,c];  dK[j,c] likewise with dS~ and q
+  OgemmArgs p = {};
+  p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
+  p.range_mode = 1;
+  p.A = Pt; p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; p.b_h = DH;
+  p.out = dv; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
+  int rc = ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * H, st);
+  if (rc != DET_OK) return rc;
+  p.A = dSt; p.B = q; p.ldb = ld; p.b_b = (long long)S * ld; p.out = dk;
+  rc = ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * H, st);
+  if (rc != DET_OK) return rc;
+  // dQ[i,c] = sum over keys j <= i ascending of dS~[i,j] k[j,c]
+  p.B = k; p.out = dq; p.range_mode = 2;
+  rc = ogemm_launch<CONTIG, STRIDED, false, true, 128>(p, B * H, st);
+  if (rc != DET_OK) return rc;
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -1,0 +1,228 @@
+// Building blocks of the ordered FP32-ALU contractions (LM head, attention backward): operand slabs staged through
+// shared memory as f32, an 8 x (TN/16) register tile per thread, packed two-lane arithmetic, and the per-slab check
+// that decides between the fused and the two-instruction multiply-add (identical bits, see ogemm.cu).
+#pragma once
+#include "common.cuh"
+#include "internal.h"
+
+namespace det {
+
+constexpr int OT = 128;  // tile edge
+constexpr int OK = 16;   // slab depth
+
+// Operand access modes.  C[i,j] = sum_c A(i,c) * B(j,c).
+//   CONTIG : operand stored [rows, contraction] (contraction index contiguous)
+//   STRIDED: operand stored [contraction, rows] (row index contiguous)
+enum { CONTIG = 0, STRIDED = 1 };
+
+template <bool F32IN>
+__device__ __forceinline__ void load8_any(const void* base, size_t idx, bool ok, float v[8]) {
+  if (!ok) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) v[t] = 0.0f;
+    return;
+  }
+  if (F32IN) {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + idx);
+    float4 a = __ldg(p), b = __ldg(p + 1);
+    // operands of the gradient contractions are rounded to bf16 first
+    v[0] = bf2f(f2bf(a.x)); v[1] = bf2f(f2bf(a.y)); v[2] = bf2f(f2bf(a.z)); v[3] = bf2f(f2bf(a.w));
+    v[4] = bf2f(f2bf(b.x)); v[5] = bf2f(f2bf(b.y)); v[6] = bf2f(f2bf(b.z)); v[7] = bf2f(f2bf(b.w));
+  } else {
+    uint4 u = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + idx));
+    v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
+    v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
+  }
+}
+
+// fetch this thread's values of an operand slab of ROWS rows x 16 contraction steps:
+// ROWS == 128: 8 values per thread, ROWS == 256: 16 values per thread
+template <int MODE, bool F32IN, int ROWS>
+__device__ __forceinline__ void slab_fetch(const void* base, int rows, int C, int ld, int r0, int c0, float* v) {
+  const int tid = threadIdx.x;
+  constexpr int NV = ROWS / 16;  // values per thread
+  if (MODE == CONTIG) {
+    // thread -> (row, 8 or 16 consecutive contraction indices)
+    const int r = r0 + (ROWS == 128 ? (tid & 127) : tid), c = c0 + (ROWS == 128 ? (tid >> 7) * 8 : 0);
+#pragma unroll
+    for (int h = 0; h < NV / 8; ++h) load8_any<F32IN>(base, (size_t)r * ld + c + 8 * h, r < rows && c + 8 * h < C, v + 8 * h);
+  } else {
+    // thread -> (contraction index, NV consecutive rows)
+    const int c = c0 + (tid >> 4), r = r0 + (tid & 15) * NV;
+#pragma unroll
+    for (int h = 0; h < NV / 8; ++h) load8_any<F32IN>(base, (size_t)c * ld + r + 8 * h, c < C && r + 8 * h < rows, v + 8 * h);
+  }
+}
+template <int MODE, int ROWS>
+__device__ __forceinline__ void slab_store(float (*s)[ROWS + 4], const float* v) {
+  const int tid = threadIdx.x;
+  constexpr int NV = ROWS / 16;
+  if (MODE == CONTIG) {
+    const int r = (ROWS == 128 ? (tid & 127) : tid), k0 = (ROWS == 128 ? (tid >> 7) * 8 : 0);
+#pragma unroll
+    for (int t = 0; t < NV; ++t) s[k0 + t][r] = v[t];
+  } else {
+    const int k = tid >> 4, r = (tid & 15) * NV;
+#pragma unroll
+    for (int t = 0; t < NV; t += 4) *reinterpret_cast<float4*>(&s[k][r + t]) = make_float4(v[t], v[t + 1], v[t + 2], v[t + 3]);
+  }
+}
+
+// true if some value v has 0 < |v| < 2^-63 (biased exponent field in 1..63): a product with such a factor could
+// fall below 2^-126, where "multiply, flush, add" and a fused multiply-add differ
+template <int NV>
+__device__ __forceinline__ bool tiny_any(const float* v) {
+  bool t = false;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const uint32_t e = (__float_as_uint(v[i]) >> 23) & 0xffu;
+    t |= (e - 1u) < 63u;
+  }
+  return t;
+}
+
+
+template <int TN>
+constexpr size_t ogemm_smem() { return (size_t)2 * OK * ((OT + 4) + (TN + 4)) * sizeof(float); }
+
+// One 16-deep slab for this thread's 8 x (TN/16) outputs.  FUSED: a*b+acc in one instruction, used only for slabs in
+// which no product can be subnormal (every non-zero factor is at least 2^-63 in magnitude), where it gives exactly the
+// bits of the unfused sequence because a product of two bf16 values is exact in binary32.  Two accumulators are
+// processed per instruction (packed f32x2 arithmetic, each lane rounded on its own).
+template <bool FUSED, int TN>
+__device__ __forceinline__ void slab_mac(const float (*As)[OT + 4], const float (*Bs)[TN + 4], int ty, int tx,
+                                         float2 (&acc)[8][TN / 32]) {
+#pragma unroll
+  for (int k = 0; k < OK; ++k) {
+    const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+    const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
+    const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    float2 b[TN / 32];
+#pragma unroll
+    for (int g = 0; g < TN / 64; ++g) {
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[k][g * 64 + tx * 4]);
+      b[2 * g] = make_float2(bv.x, bv.y);
+      b[2 * g + 1] = make_float2(bv.z, bv.w);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float2 a = make_float2(av[i], av[i]);
+#pragma unroll
+      for (int j = 0; j < TN / 32; ++j) {
+        if (FUSED) acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
+        else acc[i][j] = __fadd2_rn(acc[i][j], __fmul2_rn(a, b[j]));
+      }
+    }
+  }
+}
+
+// C[i,j] = sum over c in [c_lo, c_hi) ascending of A(i,c) B(j,c), one accumulator per output.
+struct OgemmArgs {
+  const void* A;
+  const void* B;
+  void* out;
+  int I, J, C;          // rows of A, rows of B, contraction length
+  int lda, ldb, ldo;    // leading dimensions of the stored operands / output
+  int init;             // f32 output only: start from the values already in out
+  int H;                // batching: blockIdx.z = b * H + h
+  long long a_b, a_h, b_b, b_h, o_b, o_h;  // element offsets per batch index / head index
+  int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
+};
+
+// CTA tile 128 x TN; thread (ty, tx) owns rows {ty*4.., 64+ty*4..} and columns {g*64 + tx*4..}, g < TN/64.
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
+__global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
+  extern __shared__ __align__(16) unsigned char osm[];
+  float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
+  float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
+  const int i0 = blockIdx.y * OT, j0 = blockIdx.x * TN;
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  const long long zb = blockIdx.z / p.H, zh = blockIdx.z % p.H;
+  const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + zh * p.a_h)
+                       : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + zh * p.a_h);
+  const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + zh * p.b_h;
+  void* out = OUT_BF16 ? (void*)(reinterpret_cast<uint16_t*>(p.out) + zb * p.o_b + zh * p.o_h)
+                       : (void*)(reinterpret_cast<float*>(p.out) + zb * p.o_b + zh * p.o_h);
+  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
+  int c_lo = 0, C = p.C;
+  if (p.range_mode == 1) c_lo = i0;
+  if (p.range_mode == 2) C = min(p.C, i0 + OT);
+  float2 acc[8][TN / 32];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < TN / 32; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
+  if (p.init && !OUT_BF16) {
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+      for (int g = 0; g < TN / 64; ++g) {
+        const int c = j0 + g * 64 + tx * 4;
+        if (r < I && c < J) {
+          float4 t = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(out) + (size_t)r * ldo + c);
+          acc[a][2 * g] = make_float2(t.x, t.y);
+          acc[a][2 * g + 1] = make_float2(t.z, t.w);
+        }
+      }
+    }
+  }
+  float va[8], vb[TN / 16];
+  slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, va);
+  slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo, vb);
+  slab_store<AMODE, OT>(As[0], va);
+  slab_store<BMODE, TN>(Bs[0], vb);
+  int tiny = __syncthreads_or(tiny_any<8>(va) || tiny_any<TN / 16>(vb));
+  const int nslab = (C - c_lo + OK - 1) / OK;
+  for (int s = 0; s < nslab; ++s) {
+    const int cur = s & 1;
+    if (s + 1 < nslab) {
+      slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, va);
+      slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, vb);
+    }
+    if (tiny) slab_mac<false, TN>(As[cur], Bs[cur], ty, tx, acc);
+    else slab_mac<true, TN>(As[cur], Bs[cur], ty, tx, acc);
+    bool next_tiny = false;
+    if (s + 1 < nslab) {
+      slab_store<AMODE, OT>(As[cur ^ 1], va);
+      slab_store<BMODE, TN>(Bs[cur ^ 1], vb);
+      next_tiny = tiny_any<8>(va) || tiny_any<TN / 16>(vb);
+    }
+    tiny = __syncthreads_or(next_tiny);
+  }
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+    for (int g = 0; g < TN / 64; ++g) {
+      const int c = j0 + g * 64 + tx * 4;
+      if (r < I && c < J) {
+        const float2 lo = acc[a][2 * g], hi = acc[a][2 * g + 1];
+        if (OUT_BF16) {
+          uint2 u;
+          u.x = pack_bf2(lo.x, lo.y);
+          u.y = pack_bf2(hi.x, hi.y);
+          *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(out) + (size_t)r * ldo + c) = u;
+        } else {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ldo + c) = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+      }
+    }
+  }
+}
+
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
+static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
+  static bool cfg = false;
+  if (!cfg) {
+    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)ogemm_smem<TN>()) != cudaSuccess)
+      return DET_ERR_CUDA;
+    cfg = true;
+  }
+  dim3 grid((p.J + TN - 1) / TN, (p.I + OT - 1) / OT, batches);
+  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
+  return DET_OK;
+}
+
+}  // namespace det
