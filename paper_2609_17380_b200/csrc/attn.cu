@@ -21,20 +21,52 @@ __device__ __forceinline__ void unpack8a(const uint4& u, float v[8]) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// forward: CTA = 64 queries of one (batch, head); 256 threads, thread = 4 queries x 8 keys / 8 dims
+// forward: CTA = 128 queries of one (batch, head); 256 threads, thread = 8 queries x 8 keys / 8 dims.
+// Shared memory (f32): Q [dim][query], one buffer that holds K [dim][key] during the logits and V [key][dim]
+// during P.V, and P~ [key][query].  Multiply-adds use the fused instruction whenever no factor of the tile is
+// below 2^-63 in magnitude (then the exact bf16 x bf16 product cannot be subnormal and fused = unfused bit for bit).
 // ---------------------------------------------------------------------------------------------
-constexpr int FQ = 64, FK = 128;
-constexpr int LQ = FQ + 4, LK = FK + 4;
-constexpr size_t FWD_SMEM = (size_t)(DH * LQ + DH * LK + FK * LQ + FK * LK) * sizeof(float);
+constexpr int FQ = 128, FK = 128;
+constexpr int LQ = FQ + 4;
+constexpr size_t FWD_SMEM = (size_t)(3 * DH * LQ) * sizeof(float);
+
+__device__ __forceinline__ bool tiny8a(const float v[8]) {
+  bool t = false;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) t |= (((__float_as_uint(v[i]) >> 23) & 0xffu) - 1u) < 63u;
+  return t;
+}
+
+template <bool FUSED>
+__device__ __forceinline__ void mac_8x8(const float (*As)[LQ], const float (*Bs)[LQ], int n, int ty, int tx,
+                                        float2 (&acc)[8][4]) {
+#pragma unroll 4
+  for (int k = 0; k < n; ++k) {
+    const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+    const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
+    const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+    const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
+    const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float2 a = make_float2(av[i], av[i]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (FUSED) acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
+        else acc[i][j] = __fadd2_rn(acc[i][j], __fmul2_rn(a, b[j]));
+      }
+    }
+  }
+}
 
 __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                                                      const uint16_t* __restrict__ v, int ld, int H, int S,
                                                      uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse) {
   extern __shared__ __align__(16) float sm[];
-  float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                                   // [dim][query]
-  float(*Ks)[LK] = reinterpret_cast<float(*)[LK]>(sm + DH * LQ);                         // [dim][key]
-  float(*Ps)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + DH * LQ + DH * LK);               // [key][query]
-  float(*Vs)[LK] = reinterpret_cast<float(*)[LK]>(sm + DH * LQ + DH * LK + FK * LQ);     // [key][dim]
+  float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                 // [dim][query]
+  float(*KV)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + DH * LQ);       // K: [dim][key]; V: [key][dim]
+  float(*Ps)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + 2 * DH * LQ);   // [key][query]
   const int qb = gridDim.x - 1 - blockIdx.x;  // longest rows first
   const int h = blockIdx.y, b = blockIdx.z;
   const int q0 = qb * FQ;
@@ -44,26 +76,34 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
   const uint16_t* kp = k + row0 * ld + (size_t)h * DH;
   const uint16_t* vp = v + row0 * ld + (size_t)h * DH;
 
+  bool tq = false;
   for (int idx = tid; idx < FQ * 16; idx += 256) {
-    const int r = idx & 63, ch = idx >> 6;
+    const int r = idx & 127, ch = idx >> 7;
     float t[8];
-    unpack8a(__ldg(reinterpret_cast<const uint4*>(qp + (size_t)(q0 + r) * ld + ch * 8)), t);
+    if (q0 + r < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(qp + (size_t)(q0 + r) * ld + ch * 8)), t);
+    else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) t[e] = 0.0f;
+    }
+    tq |= tiny8a(t);
 #pragma unroll
     for (int e = 0; e < 8; ++e) Qs[ch * 8 + e][r] = t[e];
   }
-  float m[4], l[4], o[4][8];
+  const int tiny_q = __syncthreads_or(tq);
+  float m[8], l[8];
+  float2 o[8][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 8; ++i) {
     m[i] = __int_as_float(0xff800000);
     l[i] = 0.0f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) o[i][e] = 0.0f;
+    for (int e = 0; e < 4; ++e) o[i][e] = make_float2(0.0f, 0.0f);
   }
   const int ntiles = q0 / FK + 1;
   for (int jt = 0; jt < ntiles; ++jt) {
     const int j0 = jt * FK;
-    const int kmax = min(FK, q0 + FQ - j0);  // keys of this tile that some row of the block can see
-    __syncthreads();
+    // ---- K tile, transposed ----
+    bool tk = false;
     for (int idx = tid; idx < FK * 16; idx += 256) {
       const int key = idx & 127, ch = idx >> 7;
       float t[8];
@@ -72,77 +112,47 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
 #pragma unroll
         for (int e = 0; e < 8; ++e) t[e] = 0.0f;
       }
+      tk |= tiny8a(t);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) Ks[ch * 8 + e][key] = t[e];
+      for (int e = 0; e < 8; ++e) KV[ch * 8 + e][key] = t[e];
     }
-    for (int idx = tid; idx < FK * 16; idx += 256) {
-      const int key = idx >> 4, ch = idx & 15;
-      float t[8];
-      if (j0 + key < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(vp + (size_t)(j0 + key) * ld + ch * 8)), t);
-      else {
+    const int tiny_k = __syncthreads_or(tk);
+    float2 s[8][4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) t[e] = 0.0f;
-      }
-      *reinterpret_cast<float4*>(&Vs[key][ch * 8]) = make_float4(t[0], t[1], t[2], t[3]);
-      *reinterpret_cast<float4*>(&Vs[key][ch * 8 + 4]) = make_float4(t[4], t[5], t[6], t[7]);
-    }
-    __syncthreads();
-    // logits
-    float s[4][8];
+    for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+      for (int e = 0; e < 4; ++e) s[i][e] = make_float2(0.0f, 0.0f);
+    if (tiny_q || tiny_k) mac_8x8<false>(Qs, KV, DH, ty, tx, s);
+    else mac_8x8<true>(Qs, KV, DH, ty, tx, s);
+    // ---- online softmax statistics per row; P~ to shared memory ----
+    float alpha[8];
+    bool tp = false;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) s[i][e] = 0.0f;
-    if (kmax > 64) {
-#pragma unroll 4
-      for (int d = 0; d < DH; ++d) {
-        const float4 a = *reinterpret_cast<const float4*>(&Qs[d][ty * 4]);
-        const float4 b0 = *reinterpret_cast<const float4*>(&Ks[d][tx * 4]);
-        const float4 b1 = *reinterpret_cast<const float4*>(&Ks[d][64 + tx * 4]);
-        const float ar[4] = {a.x, a.y, a.z, a.w};
-        const float br[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) s[i][e] = fadd(s[i][e], fmul(ar[i], br[e]));
-      }
-    } else {
-#pragma unroll 4
-      for (int d = 0; d < DH; ++d) {
-        const float4 a = *reinterpret_cast<const float4*>(&Qs[d][ty * 4]);
-        const float4 b0 = *reinterpret_cast<const float4*>(&Ks[d][tx * 4]);
-        const float ar[4] = {a.x, a.y, a.z, a.w};
-        const float br[4] = {b0.x, b0.y, b0.z, b0.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) s[i][e] = fadd(s[i][e], fmul(ar[i], br[e]));
-      }
-    }
-    // online softmax statistics per row
-    float alpha[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int row = q0 + ty * 4 + i;
+    for (int i = 0; i < 8; ++i) {
+      const int rl = (i >> 2) * 64 + ty * 4 + (i & 3);
+      const int row = q0 + rl;
+      float sv[8] = {s[i][0].x, s[i][0].y, s[i][1].x, s[i][1].y, s[i][2].x, s[i][2].y, s[i][3].x, s[i][3].y};
       float mt = m[i];
       bool valid[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int key = j0 + ((e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4));
         valid[e] = key <= row;
-        s[i][e] = fmul(s[i][e], ATT_SCALE);
-        if (valid[e]) mt = fmaxf(mt, s[i][e]);
+        sv[e] = fmul(sv[e], ATT_SCALE);
+        if (valid[e]) mt = fmaxf(mt, sv[e]);
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
       alpha[i] = det_exp(fsub(m[i], mt));
       float p[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) p[e] = valid[e] ? det_exp(fsub(s[i][e], mt)) : 0.0f;
+      for (int e = 0; e < 8; ++e) p[e] = valid[e] ? det_exp(fsub(sv[e], mt)) : 0.0f;
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int kl = (e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4);
-        Ps[kl][ty * 4 + i] = bf2f(f2bf(p[e]));
+        const float pt = bf2f(f2bf(p[e]));
+        tp |= (((__float_as_uint(pt) >> 23) & 0xffu) - 1u) < 63u;
+        Ps[kl][rl] = pt;
       }
       float h0 = fadd(fadd(p[0], p[1]), fadd(p[2], p[3]));
       float h1 = fadd(fadd(p[4], p[5]), fadd(p[6], p[7]));
@@ -154,38 +164,48 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
       l[i] = fadd(fmul(l[i], alpha[i]), fadd(h0, h1));
       m[i] = mt;
     }
-    __syncthreads();
-    // u = P~ . V over the tile's keys in ascending order, then o = o*alpha + u
-    float u[4][8];
+    __syncthreads();  // every thread is done with K; P~ is complete
+    // ---- V tile, natural layout, into the same buffer ----
+    bool tv = false;
+    for (int idx = tid; idx < FK * 16; idx += 256) {
+      const int key = idx >> 4, ch = idx & 15;
+      float t[8];
+      if (j0 + key < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(vp + (size_t)(j0 + key) * ld + ch * 8)), t);
+      else {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) u[i][e] = 0.0f;
-#pragma unroll 4
-    for (int j = 0; j < kmax; ++j) {
-      const float4 a = *reinterpret_cast<const float4*>(&Ps[j][ty * 4]);
-      const float4 b0 = *reinterpret_cast<const float4*>(&Vs[j][tx * 4]);
-      const float4 b1 = *reinterpret_cast<const float4*>(&Vs[j][64 + tx * 4]);
-      const float ar[4] = {a.x, a.y, a.z, a.w};
-      const float br[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) u[i][e] = fadd(u[i][e], fmul(ar[i], br[e]));
+        for (int e = 0; e < 8; ++e) t[e] = 0.0f;
+      }
+      tv |= tiny8a(t);
+      *reinterpret_cast<float4*>(&KV[key][ch * 8]) = make_float4(t[0], t[1], t[2], t[3]);
+      *reinterpret_cast<float4*>(&KV[key][ch * 8 + 4]) = make_float4(t[4], t[5], t[6], t[7]);
     }
+    const int tiny_pv = __syncthreads_or(tp || tv);
+    // ---- u = P~ . V over the tile's keys in ascending order, then o = o*alpha + u ----
+    float2 u[8][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 8; ++i)
 #pragma unroll
-      for (int e = 0; e < 8; ++e) o[i][e] = fadd(fmul(o[i][e], alpha[i]), u[i][e]);
+      for (int e = 0; e < 4; ++e) u[i][e] = make_float2(0.0f, 0.0f);
+    const int kmax = min(FK, q0 + FQ - j0);
+    if (tiny_pv) mac_8x8<false>(Ps, KV, kmax, ty, tx, u);
+    else mac_8x8<true>(Ps, KV, kmax, ty, tx, u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float2 al = make_float2(alpha[i], alpha[i]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[i][e] = __fadd2_rn(__fmul2_rn(o[i][e], al), u[i][e]);
+    }
+    __syncthreads();  // V and P~ may be overwritten by the next tile
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int row = q0 + ty * 4 + i;
+  for (int i = 0; i < 8; ++i) {
+    const int row = q0 + (i >> 2) * 64 + ty * 4 + (i & 3);
+    if (row >= S) continue;
     const float il = fdiv(1.0f, l[i]);
     uint16_t* op = out + (row0 + row) * ld_out + (size_t)h * DH;
     uint2 w0, w1;
-    w0.x = pack_bf2(fmul(o[i][0], il), fmul(o[i][1], il)); w0.y = pack_bf2(fmul(o[i][2], il), fmul(o[i][3], il));
-    w1.x = pack_bf2(fmul(o[i][4], il), fmul(o[i][5], il)); w1.y = pack_bf2(fmul(o[i][6], il), fmul(o[i][7], il));
+    w0.x = pack_bf2(fmul(o[i][0].x, il), fmul(o[i][0].y, il)); w0.y = pack_bf2(fmul(o[i][1].x, il), fmul(o[i][1].y, il));
+    w1.x = pack_bf2(fmul(o[i][2].x, il), fmul(o[i][2].y, il)); w1.y = pack_bf2(fmul(o[i][3].x, il), fmul(o[i][3].y, il));
     *reinterpret_cast<uint2*>(op + tx * 4) = w0;
     *reinterpret_cast<uint2*>(op + 64 + tx * 4) = w1;
     if (tx == 0) lse[((size_t)b * H + h) * S + row] = fadd(m[i], det_log(l[i]));
@@ -313,7 +333,7 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
   static bool cfg = false;
   if (!cfg) { if (set_smem((const void*)k_attn_fwd, FWD_SMEM)) return DET_ERR_CUDA; cfg = true; }
-  dim3 grid(S / FQ, H, B);
+  dim3 grid((S + FQ - 1) / FQ, H, B);
   k_attn_fwd<<<DET_L(grid), 256, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
   DET_CHECK_LAUNCH();
   return DET_OK;
