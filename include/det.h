@@ -127,6 +127,10 @@ int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, cons
                    det_bf16* dX, float* dW, float* ds_x, void* ws, size_t ws_bytes, void* stream, int* status_dev);
 /* exact int8 x int8 -> int32 contraction C[i,j] = sum_k A[i,k] B[j,k] (tcgen05); test hook for the GEMM core.
  * I % 128 == 0, J % 128 == 0, K % 128 == 0. */
+/* Test hook: mode 0 lets the GEMM use two-CTA 256 x 256 tiles (tcgen05 cta_group::2) whenever both output dimensions
+ * are multiples of 256; mode 1 forces the one-CTA kernel.  Results are identical (integer accumulation is exact).
+ * Process-wide, not thread-safe. */
+int det_igemm_set_mode(int mode);
 int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream, int* status_dev);
 
 /* ---- RMSNorm (Sec. 3.1 "RMSNorm", FP32 internals) -------------------------------------------------

@@ -176,6 +176,10 @@ def det_linear_bwd(dY, X, qX, W, qWt_bwd, s_x, s_w, s_u, M, N, K, hadamard_block
         C.c_int(K), C.c_int(hadamard_block), _ptr(dX), _ptr(dW), _ptr(ds_x), *_ws(ws), _stream(), _ptr(status_dev)))
 
 
+def det_igemm_set_mode(mode):
+    _check("det_igemm_set_mode", load().det_igemm_set_mode(C.c_int(mode)))
+
+
 def det_igemm_tn(A, B, I, J, K, Cout, status_dev=None):
     _check("det_igemm_tn", load().det_igemm_tn(_ptr(A), _ptr(B), C.c_int(I), C.c_int(J), C.c_int(K), _ptr(Cout), _stream(),
                                                _ptr(status_dev)))

@@ -116,6 +116,116 @@ __device__ __forceinline__ void tile_origin(int tile, int tiles_i, int tiles_j, 
   else { i0 = (tile % tiles_i) * BM; j0 = (tile / tiles_i) * bn; }
 }
 
+// data-dependent scalars of the epilogue, read once per CTA from device memory
+template <int EPI>
+__device__ __forceinline__ void epi_scalars(const EpiParams& ep, float& cscale, float& inv_s, float& sx) {
+  cscale = 1.0f; inv_s = 1.0f; sx = 1.0f;
+    if (EPI == EPI_FWD) sx = ep.s_x[0];
+    if (EPI == EPI_DX) {
+      const float am = __uint_as_float(ep.amax1[0]);
+      const float s_a = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
+      cscale = fmul(fmul(s_a, ep.s_u[0]), ep.rot);
+      inv_s = fdiv(1.0f, ep.s_x[0]);
+    }
+    if (EPI == EPI_DW) {
+      const float am = __uint_as_float(ep.amax1[0]);
+      const float s_g = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
+      float s_z = 1.0f;
+      if (ep.amax2) {
+        const int az = (int)ep.amax2[0];
+        s_z = (az > 0) ? fdiv(__int2float_rn(az), 127.0f) : 0.0f;
+      }
+      cscale = fmul(fmul(fmul(s_g, s_z), ep.s_x[0]), ep.rot);
+    }
+}
+
+// Epilogue of one accumulator row: this lane owns TMEM lane `taddr`'s row (output row `row`), columns j0 .. j0+BN.
+template <int BN, int EPI>
+__device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int row, int J, int j0, float cscale,
+                                        float inv_s, float sx) {
+      const size_t rbase = (size_t)row * J + j0;
+      if (EPI == EPI_DW) inv_s = fdiv(1.0f, ep.s_w[row]);
+#pragma unroll 1
+      for (int h = 0; h < BN / 128; ++h) {
+      float grp[4];
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c0 = h * 128 + cc * 32;
+        uint32_t r[32];
+        tmem_ld32(taddr + (uint32_t)c0, r);
+        if (EPI == EPI_RAW) {
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<int32_t*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 8; ++v) o[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+        } else if (EPI == EPI_FWD) {
+          const float4* sw = reinterpret_cast<const float4*>(ep.s_w + j0 + c0);
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float4 w0 = __ldg(sw + 2 * v), w1 = __ldg(sw + 2 * v + 1);
+            float f[8];
+            f[0] = fmul(__int2float_rn((int)r[8 * v + 0]), fmul(sx, w0.x));
+            f[1] = fmul(__int2float_rn((int)r[8 * v + 1]), fmul(sx, w0.y));
+            f[2] = fmul(__int2float_rn((int)r[8 * v + 2]), fmul(sx, w0.z));
+            f[3] = fmul(__int2float_rn((int)r[8 * v + 3]), fmul(sx, w0.w));
+            f[4] = fmul(__int2float_rn((int)r[8 * v + 4]), fmul(sx, w1.x));
+            f[5] = fmul(__int2float_rn((int)r[8 * v + 5]), fmul(sx, w1.y));
+            f[6] = fmul(__int2float_rn((int)r[8 * v + 6]), fmul(sx, w1.z));
+            f[7] = fmul(__int2float_rn((int)r[8 * v + 7]), fmul(sx, w1.w));
+            o[v] = make_uint4(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]), pack_bf2(f[4], f[5]), pack_bf2(f[6], f[7]));
+          }
+        } else if (EPI == EPI_DX) {
+          const uint4* xr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
+          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+          float term[32];
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 xu = __ldg(xr + v);
+            const uint32_t xs[4] = {xu.x, xu.y, xu.z, xu.w};
+            float g[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float xv = (e & 1) ? bfhi(xs[e >> 1]) : bflo(xs[e >> 1]);
+              const float gx = fmul(__int2float_rn((int)r[8 * v + e]), cscale);
+              const float t = fmul(xv, inv_s);
+              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
+              const float phi = t < -128.0f ? -128.0f : (t > 127.0f ? 127.0f : fsub(rintf(t), t));
+              g[e] = in_range ? gx : 0.0f;
+              term[8 * v + e] = fmul(gx, phi);
+            }
+            o[v] = make_uint4(pack_bf2(g[0], g[1]), pack_bf2(g[2], g[3]), pack_bf2(g[4], g[5]), pack_bf2(g[6], g[7]));
+          }
+          // adjacent tree over this lane's 32 columns
+#pragma unroll
+          for (int w = 1; w < 32; w <<= 1)
+#pragma unroll
+            for (int e = 0; e < 32; e += 2 * w) term[e] = fadd(term[e], term[e + w]);
+          grp[cc] = term[0];
+        } else {  // EPI_DW
+          const uint4* wr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
+          float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out) + rbase + c0);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 wu = __ldg(wr + v);
+            const uint32_t wsr[4] = {wu.x, wu.y, wu.z, wu.w};
+            float g[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float wv = (e & 1) ? bfhi(wsr[e >> 1]) : bflo(wsr[e >> 1]);
+              const float t = fmul(wv, inv_s);
+              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
+              g[e] = in_range ? fmul(__int2float_rn((int)r[8 * v + e]), cscale) : 0.0f;
+            }
+            o[2 * v] = make_float4(g[0], g[1], g[2], g[3]);
+            o[2 * v + 1] = make_float4(g[4], g[5], g[6], g[7]);
+          }
+        }
+      }
+      if (EPI == EPI_DX)
+        ep.ds_partial[(size_t)row * (J / 128) + (j0 / 128) + h] = fadd(fadd(grp[0], grp[1]), fadd(grp[2], grp[3]));
+      }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
     k_igemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, EpiParams ep, int I, int J,
@@ -202,24 +312,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int it = 0;
     bool ok = true;
-    float cscale = 1.0f, inv_s = 1.0f, sx = 1.0f;
-    if (EPI == EPI_FWD) sx = ep.s_x[0];
-    if (EPI == EPI_DX) {
-      const float am = __uint_as_float(ep.amax1[0]);
-      const float s_a = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
-      cscale = fmul(fmul(s_a, ep.s_u[0]), ep.rot);
-      inv_s = fdiv(1.0f, ep.s_x[0]);
-    }
-    if (EPI == EPI_DW) {
-      const float am = __uint_as_float(ep.amax1[0]);
-      const float s_g = (am > 0.0f) ? fdiv(am, 127.0f) : 0.0f;
-      float s_z = 1.0f;
-      if (ep.amax2) {
-        const int az = (int)ep.amax2[0];
-        s_z = (az > 0) ? fdiv(__int2float_rn(az), 127.0f) : 0.0f;
-      }
-      cscale = fmul(fmul(fmul(s_g, s_z), ep.s_x[0]), ep.rot);
-    }
+    float cscale, inv_s, sx;
+    epi_scalars<EPI>(ep, cscale, inv_s, sx);
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -227,88 +321,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         tile_origin(tile, tiles_i, tiles_j, BN, i0, j0);
       if (!mbar_wait(&bar_tfull[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
-      const int row = i0 + q * 32 + lane;
-      const size_t rbase = (size_t)row * J + j0;
-      if (EPI == EPI_DW) inv_s = fdiv(1.0f, ep.s_w[row]);
-#pragma unroll 1
-      for (int h = 0; h < BN / 128; ++h) {
-      float grp[4];
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c0 = h * 128 + cc * 32;
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-        if (EPI == EPI_RAW) {
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<int32_t*>(ep.out) + rbase + c0);
-#pragma unroll
-          for (int v = 0; v < 8; ++v) o[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-        } else if (EPI == EPI_FWD) {
-          const float4* sw = reinterpret_cast<const float4*>(ep.s_w + j0 + c0);
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            float4 w0 = __ldg(sw + 2 * v), w1 = __ldg(sw + 2 * v + 1);
-            float f[8];
-            f[0] = fmul(__int2float_rn((int)r[8 * v + 0]), fmul(sx, w0.x));
-            f[1] = fmul(__int2float_rn((int)r[8 * v + 1]), fmul(sx, w0.y));
-            f[2] = fmul(__int2float_rn((int)r[8 * v + 2]), fmul(sx, w0.z));
-            f[3] = fmul(__int2float_rn((int)r[8 * v + 3]), fmul(sx, w0.w));
-            f[4] = fmul(__int2float_rn((int)r[8 * v + 4]), fmul(sx, w1.x));
-            f[5] = fmul(__int2float_rn((int)r[8 * v + 5]), fmul(sx, w1.y));
-            f[6] = fmul(__int2float_rn((int)r[8 * v + 6]), fmul(sx, w1.z));
-            f[7] = fmul(__int2float_rn((int)r[8 * v + 7]), fmul(sx, w1.w));
-            o[v] = make_uint4(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]), pack_bf2(f[4], f[5]), pack_bf2(f[6], f[7]));
-          }
-        } else if (EPI == EPI_DX) {
-          const uint4* xr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
-          float term[32];
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint4 xu = __ldg(xr + v);
-            const uint32_t xs[4] = {xu.x, xu.y, xu.z, xu.w};
-            float g[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const float xv = (e & 1) ? bfhi(xs[e >> 1]) : bflo(xs[e >> 1]);
-              const float gx = fmul(__int2float_rn((int)r[8 * v + e]), cscale);
-              const float t = fmul(xv, inv_s);
-              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
-              const float phi = t < -128.0f ? -128.0f : (t > 127.0f ? 127.0f : fsub(rintf(t), t));
-              g[e] = in_range ? gx : 0.0f;
-              term[8 * v + e] = fmul(gx, phi);
-            }
-            o[v] = make_uint4(pack_bf2(g[0], g[1]), pack_bf2(g[2], g[3]), pack_bf2(g[4], g[5]), pack_bf2(g[6], g[7]));
-          }
-          // adjacent tree over this lane's 32 columns
-#pragma unroll
-          for (int w = 1; w < 32; w <<= 1)
-#pragma unroll
-            for (int e = 0; e < 32; e += 2 * w) term[e] = fadd(term[e], term[e + w]);
-          grp[cc] = term[0];
-        } else {  // EPI_DW
-          const uint4* wr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
-          float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out) + rbase + c0);
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint4 wu = __ldg(wr + v);
-            const uint32_t wsr[4] = {wu.x, wu.y, wu.z, wu.w};
-            float g[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const float wv = (e & 1) ? bfhi(wsr[e >> 1]) : bflo(wsr[e >> 1]);
-              const float t = fmul(wv, inv_s);
-              const bool in_range = (t >= -128.0f) && (t <= 127.0f);
-              g[e] = in_range ? fmul(__int2float_rn((int)r[8 * v + e]), cscale) : 0.0f;
-            }
-            o[2 * v] = make_float4(g[0], g[1], g[2], g[3]);
-            o[2 * v + 1] = make_float4(g[4], g[5], g[6], g[7]);
-          }
-        }
-      }
-      if (EPI == EPI_DX)
-        ep.ds_partial[(size_t)row * (J / 128) + (j0 / 128) + h] = fadd(fadd(grp[0], grp[1]), fadd(grp[2], grp[3]));
-      }
+      epi_row<BN, EPI>(ep, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), i0 + q * 32 + lane, J, j0, cscale, inv_s, sx);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bar_tempty[acc]);
@@ -325,6 +338,188 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Two-CTA variant (tcgen05 cta_group::2).  A cluster of two CTAs on neighbouring SMs computes one 256 x 256 tile:
+// CTA r owns rows r*128 .. r*128+127 of the tile (its own A rows and its own 128 x 256 accumulator in TMEM) and stages
+// only half of the B tile (rows r*128 .. of the 256 B rows); the MMA, issued by the leader CTA for both, reads the two
+// halves of B from the two CTAs' shared memory.  Per CTA and K step that is 32 KiB staged and 32 KiB read by the tensor
+// core instead of 48 + 48 KiB, which matters because TMA writes and MMA operand reads share the shared-memory port.
+//   * each CTA's producer thread loads its own A / B-half tiles; the loads complete on the LEADER's full barrier
+//   * the leader's MMA thread waits on that barrier, issues the MMAs, and releases the ring slot in BOTH CTAs with a
+//     multicast tcgen05.commit; the same for "accumulator ready"
+//   * the epilogue warps of both CTAs drain their own TMEM and arrive on the leader's "accumulator free" barrier
+// No load uses cluster multicast.  All waits are bounded as in the one-CTA kernel.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int STAGES2 = 6;
+constexpr int BN2 = 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// tile load of this CTA whose completion is counted on the leader CTA's barrier (peer bit of the address cleared)
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+  const uint32_t leader_bar = smem_u32(bar) & 0xFEFFFFFFu;
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(leader_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this offset in both CTAs once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                   smem_u32(bar)),
+               "h"(mask)
+               : "memory");
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+    k_igemm2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, EpiParams ep, int I, int J,
+             int K, int* status) {
+  constexpr int STAGE_A = 128 * BK, STAGE_B = 128 * BK, STAGE_BYTES = STAGE_A + STAGE_B;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bar_full[STAGES2], bar_empty[STAGES2], bar_tfull[2], bar_tempty[2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&bar_tfull[a], 1); mbar_init(&bar_tempty[a], 8); }
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything can signal them
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  const int tiles_i = I / 256, tiles_j = J / BN2;
+  const int num_tiles = tiles_i * tiles_j;
+  const int kblocks = K / BK;
+  const int cluster_id = blockIdx.x >> 1, nclusters = gridDim.x >> 1;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += nclusters) {
+        int i0, j0;
+        if (tiles_j <= tiles_i) { j0 = (tile % tiles_j) * BN2; i0 = (tile / tiles_j) * 256; }
+        else { i0 = (tile % tiles_i) * 256; j0 = (tile / tiles_i) * BN2; }
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          if (leader) mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);  // both CTAs' tiles complete on this barrier
+          uint8_t* sa = smem + stage * STAGE_BYTES;
+          tma_load_2d_pair(sa, &tmA, kb * BK, i0 + (int)rank * 128, &bar_full[stage]);
+          tma_load_2d_pair(sa + STAGE_A, &tmB, kb * BK, j0 + (int)rank * 128, &bar_full[stage]);
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      // instruction descriptor: D = S32, A = B = signed 8-bit, both K-major, N = 256, M = 256 (two CTAs x 128)
+      constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN2 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += nclusters, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(&bar_tempty[acc], acc_phase ^ 1u, abort_flag, status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN2);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_full[stage], phase, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + STAGE_A);
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 32; ++k4)
+            umma_i8_pair(tmem_d, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+          umma_commit_pair(&bar_empty[stage]);
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit_pair(&bar_tfull[acc]);
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int it = 0;
+    bool ok = true;
+    float cscale, inv_s, sx;
+    epi_scalars<EPI>(ep, cscale, inv_s, sx);
+    const uint32_t tempty_leader0 = mapa_u32(smem_u32(&bar_tempty[0]), 0), tempty_leader1 = mapa_u32(smem_u32(&bar_tempty[1]), 0);
+    for (int tile = cluster_id; tile < num_tiles && ok; tile += nclusters, ++it) {
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      int i0, j0;
+      if (tiles_j <= tiles_i) { j0 = (tile % tiles_j) * BN2; i0 = (tile / tiles_j) * 256; }
+      else { i0 = (tile % tiles_i) * 256; j0 = (tile / tiles_i) * BN2; }
+      if (!mbar_wait(&bar_tfull[acc], acc_phase, abort_flag, status)) { ok = false; break; }
+      tc_fence_after();
+      epi_row<BN2, EPI>(ep, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN2), i0 + (int)rank * 128 + q * 32 + lane, J,
+                        j0, cscale, inv_s, sx);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(acc ? tempty_leader1 : tempty_leader0);
+    }
+  }
+
+  // teardown: both CTAs meet before either leaves (the peer may still signal this CTA's barriers or read its tiles)
+  __syncthreads();
+  if (abort_s) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+  }
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -378,6 +573,34 @@ static int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const EpiPar
   return DET_OK;
 }
 
+template <int EPI>
+static int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const EpiParams& ep, int I, int J, int K, int* status,
+                       cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES2 * (2 * 128 * BK) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(k_igemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return DET_ERR_CUDA;
+    configured = true;
+  }
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const int tiles = (I / 256) * (J / BN2);
+  int clusters = sms / 2;
+  if (tiles < clusters) clusters = tiles;
+  k_igemm2<EPI><<<DET_L(2 * clusters), GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
+  if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
+  return DET_OK;
+}
+
+// 0: automatic (two-CTA 256 x 256 tiles when both dimensions are multiples of 256); 1: always the one-CTA kernel
+static int g_gemm_mode = 0;
+void igemm_set_mode(int mode) { g_gemm_mode = mode; }
+
 int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
                  cudaStream_t st) {
   if (!A || !B || I <= 0 || J <= 0 || K <= 0) return DET_ERR_ARG;
@@ -386,6 +609,16 @@ int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K,
   if (!aligned16(A) || !aligned16(B)) return DET_ERR_ALIGN;
   const int bn = (J % 256 == 0) ? 256 : 128;
   CUtensorMap ta, tb;
+  if (g_gemm_mode == 0 && I % 256 == 0 && J % 256 == 0) {
+    if (!make_map(&ta, A, I, K, 128) || !make_map(&tb, B, J, K, 128)) return DET_ERR_CUDA;
+    switch (epi) {
+      case EPI_RAW: return launch_pair<EPI_RAW>(ta, tb, ep, I, J, K, status, st);
+      case EPI_FWD: return launch_pair<EPI_FWD>(ta, tb, ep, I, J, K, status, st);
+      case EPI_DX: return launch_pair<EPI_DX>(ta, tb, ep, I, J, K, status, st);
+      case EPI_DW: return launch_pair<EPI_DW>(ta, tb, ep, I, J, K, status, st);
+    }
+    return DET_ERR_ARG;
+  }
   if (!make_map(&ta, A, I, K, BM) || !make_map(&tb, B, J, K, bn)) return DET_ERR_CUDA;
 #define DET_GEMM_CASE(E)                                                     \
   case E:                                                                    \
@@ -404,6 +637,12 @@ int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K,
 }  // namespace det
 
 using namespace det;
+
+extern "C" int det_igemm_set_mode(int mode) {
+  if (mode != 0 && mode != 1) return DET_ERR_ARG;
+  igemm_set_mode(mode);
+  return DET_OK;
+}
 
 extern "C" int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream,
                             int* status_dev) {

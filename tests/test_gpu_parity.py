@@ -292,7 +292,8 @@ def test_tensor_hash(det, n):
 
 
 # ------------------------------------------------------------------ int8 GEMM and the LSQ linear layer
-@pytest.mark.parametrize("I,J,K", [(128, 128, 128), (256, 512, 512), (384, 256, 1024), (128, 384, 2048), (512, 768, 640)])
+@pytest.mark.parametrize("I,J,K", [(128, 128, 128), (256, 512, 512), (384, 256, 1024), (128, 384, 2048), (512, 768, 640),
+                                   (1024, 2048, 1152), (256, 256, 128)])
 def test_igemm_exact(det, I, J, K):
     import torch
     rng = np.random.default_rng(I + J + K)
@@ -342,9 +343,11 @@ def test_lsq_scales_quant_forward(det, M, N, K, per_tensor):
     assert_same_bits(host(Y, np.uint16), oY, "Y")
 
 
-@pytest.mark.parametrize("M,N,K,hb", [(256, 512, 512, 128), (256, 512, 512, 0), (384, 128, 256, 128), (128, 256, 640, 128)])
-def test_linear_backward(det, M, N, K, hb):
+@pytest.mark.parametrize("M,N,K,hb,mode", [(256, 512, 512, 128, 0), (256, 512, 512, 0, 0), (384, 128, 256, 128, 0),
+                                            (128, 256, 640, 128, 0), (256, 512, 512, 128, 1), (512, 256, 768, 128, 0)])
+def test_linear_backward(det, M, N, K, hb, mode):
     import torch
+    det.det_igemm_set_mode(mode)       # 0: two-CTA tiles where the shape allows, 1: one-CTA kernel only
     X, W, dY = _linear_case(M, N, K, 12)
     osw = oracle.lsq_weight_scale(W)
     osx = oracle.lsq_act_scale_init(X)
@@ -366,6 +369,7 @@ def test_linear_backward(det, M, N, K, hb):
     assert_same_bits(host(gX, np.uint16), odX, "dX")
     assert_same_bits(host(gW), odW, "dW")
     assert_same_bits(host(gs), ods, "ds_x")
+    det.det_igemm_set_mode(0)
 
 
 # ------------------------------------------------------------------ LM head and attention (ordered FP32)
