@@ -112,37 +112,57 @@ __global__ void __launch_bounds__(256) k_quantize(const uint16_t* __restrict__ X
 template <int PASS, bool ROT>
 __global__ void __launch_bounds__(256) k_rot_rows(const uint16_t* __restrict__ dY, const float* __restrict__ s_w, int M,
                                                   int N, uint32_t* __restrict__ amax, int8_t* __restrict__ Aq) {
+  // a warp owns RB consecutive 128-element blocks of one row and issues all its loads before any arithmetic
+  constexpr int RB = 8;
   const int lane = threadIdx.x & 31;
-  const size_t blk = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  const size_t nblk = (size_t)M * (N / 128);
+  const int gpr = (N / 128 + RB - 1) / RB;  // warp groups per row
+  const size_t grp = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   float local = 0.0f;
-  if (blk < nblk) {
-    const size_t m = blk / (N / 128);
-    const int n0 = (int)(blk % (N / 128)) * 128 + lane * 4;
-    uint2 u = __ldg(reinterpret_cast<const uint2*>(dY + m * N + n0));
-    float4 w = __ldg(reinterpret_cast<const float4*>(s_w + n0));
-    float v[4] = {fmul(bflo(u.x), w.x), fmul(bfhi(u.x), w.y), fmul(bflo(u.y), w.z), fmul(bfhi(u.y), w.w)};
-    if (ROT) {
-      float a0 = fadd(v[0], v[1]), a1 = fsub(v[0], v[1]), a2 = fadd(v[2], v[3]), a3 = fsub(v[2], v[3]);
-      v[0] = fadd(a0, a2); v[2] = fsub(a0, a2); v[1] = fadd(a1, a3); v[3] = fsub(a1, a3);
+  if (grp < (size_t)M * gpr) {
+    const size_t m = grp / gpr;
+    const int nb0 = (int)(grp % gpr) * RB;  // first 128-block of this group
+    uint2 u[RB];
+    float4 w[RB];
 #pragma unroll
-      for (int hl = 1; hl < 32; hl <<= 1) {
-        const bool upper = lane & hl;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float o = __shfl_xor_sync(0xffffffffu, v[e], hl);
-          v[e] = upper ? fsub(o, v[e]) : fadd(v[e], o);
-        }
+    for (int r = 0; r < RB; ++r) {
+      const int n0 = (nb0 + r) * 128 + lane * 4;
+      if (n0 < N) {
+        u[r] = __ldg(reinterpret_cast<const uint2*>(dY + m * N + n0));
+        w[r] = __ldg(reinterpret_cast<const float4*>(s_w + n0));
+      } else {
+        u[r] = make_uint2(0u, 0u);
+        w[r] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
-    if (PASS == 0) {
-      local = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
-    } else {
+    float inv = 0.0f;
+    if (PASS == 1) {
       const float am = __uint_as_float(amax[0]);
-      const float inv = (am > 0.0f) ? fdiv(127.0f, am) : 0.0f;
-      uint32_t o = ((uint32_t)(uint8_t)quant1(v[0], inv)) | ((uint32_t)(uint8_t)quant1(v[1], inv) << 8) |
-                   ((uint32_t)(uint8_t)quant1(v[2], inv) << 16) | ((uint32_t)(uint8_t)quant1(v[3], inv) << 24);
-      *reinterpret_cast<uint32_t*>(Aq + m * N + n0) = o;
+      inv = (am > 0.0f) ? fdiv(127.0f, am) : 0.0f;
+    }
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+      const int n0 = (nb0 + r) * 128 + lane * 4;
+      float v[4] = {fmul(bflo(u[r].x), w[r].x), fmul(bfhi(u[r].x), w[r].y), fmul(bflo(u[r].y), w[r].z), fmul(bfhi(u[r].y), w[r].w)};
+      if (ROT) {
+        float a0 = fadd(v[0], v[1]), a1 = fsub(v[0], v[1]), a2 = fadd(v[2], v[3]), a3 = fsub(v[2], v[3]);
+        v[0] = fadd(a0, a2); v[2] = fsub(a0, a2); v[1] = fadd(a1, a3); v[3] = fsub(a1, a3);
+#pragma unroll
+        for (int hl = 1; hl < 32; hl <<= 1) {
+          const bool upper = lane & hl;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float o = __shfl_xor_sync(0xffffffffu, v[e], hl);
+            v[e] = upper ? fsub(o, v[e]) : fadd(v[e], o);
+          }
+        }
+      }
+      if (PASS == 0) {
+        local = fmaxf(local, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+      } else if (n0 < N) {
+        uint32_t o = ((uint32_t)(uint8_t)quant1(v[0], inv)) | ((uint32_t)(uint8_t)quant1(v[1], inv) << 8) |
+                     ((uint32_t)(uint8_t)quant1(v[2], inv) << 16) | ((uint32_t)(uint8_t)quant1(v[3], inv) << 24);
+        *reinterpret_cast<uint32_t*>(Aq + m * N + n0) = o;
+      }
     }
   }
   if (PASS == 0) {
@@ -359,8 +379,8 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   float* sscr = (float*)(base + oS);
   const bool rot = hadamard_block != 0;
   cudaMemsetAsync(amax, 0, 256, st);
-  const size_t nblk = (size_t)M * (N / 128);
-  const unsigned g1 = (unsigned)((nblk + 7) / 8);
+  const size_t ngrp = (size_t)M * ((N / 128 + 7) / 8);  // warp groups of 8 blocks
+  const unsigned g1 = (unsigned)((ngrp + 7) / 8);
   dim3 gG(N / 128, M / 128), gZ(K / 128, M / 128);
   if (rot) {
     k_rot_rows<0, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);

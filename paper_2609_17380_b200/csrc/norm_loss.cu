@@ -89,71 +89,85 @@ __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x
 // Backward for rows of at most 2048 elements.  With DG, the CTA (8 adjacent rows) also leaves the column-wise
 // tree over its 8 rows of dy*xhat in partial8[blockIdx.x][D] (the first three levels of the row-direction tree).
 template <bool BF, bool DG>
-__global__ void __launch_bounds__(256) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
+__global__ void __launch_bounds__(512) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
                                                       const void* __restrict__ gamma, const float* __restrict__ rstd,
                                                       int rows, int D, float invD, void* __restrict__ dx,
                                                       float* __restrict__ partial8) {
+  // 16 warps = 8 rows x 2 warps; warp half hw owns leaves hw*4 .. hw*4+3 (elements hw*1024 ..) of its row
   extern __shared__ __align__(16) float srow[];  // DG: [8][D]
+  __shared__ float half_sum[8][2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.x * 8 + warp;
+  const int rl = warp >> 1, hw = warp & 1;
+  const int row = blockIdx.x * 8 + rl;
   const bool live = row < rows;
   const size_t rb = (size_t)row * D;
-  float w[8][8], xh[8][8];
+  float w[4][8], xh[4][8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int e0 = j * 256 + lane * 8;
+  for (int jj = 0; jj < 4; ++jj) {
+    const int e0 = (hw * 4 + jj) * 256 + lane * 8;
     if (live && e0 < D) {
-      load8<BF>(dy, rb + e0, w[j]);
-      load8<BF>(x, rb + e0, xh[j]);
+      load8<BF>(dy, rb + e0, w[jj]);
+      load8<BF>(x, rb + e0, xh[jj]);
     } else {
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { w[j][t] = 0.0f; xh[j][t] = 0.0f; }
+      for (int t = 0; t < 8; ++t) { w[jj][t] = 0.0f; xh[jj][t] = 0.0f; }
     }
   }
   const float rs = live ? rstd[row] : 0.0f;
   float mine = 0.0f;
   const bool full = (D & 255) == 0;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
+  for (int jj = 0; jj < 4; ++jj) {
+    const int j = hw * 4 + jj;
     const int e0 = j * 256 + lane * 8;
     float pr[8];
 #pragma unroll
-    for (int t = 0; t < 8; ++t) xh[j][t] = fmul(xh[j][t], rs);
+    for (int t = 0; t < 8; ++t) xh[jj][t] = fmul(xh[jj][t], rs);
     if (DG && e0 < D) {
       float dgt[8];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[j][t], xh[j][t]);
-      *reinterpret_cast<float4*>(&srow[warp * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
-      *reinterpret_cast<float4*>(&srow[warp * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
+      for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[jj][t], xh[jj][t]);
+      *reinterpret_cast<float4*>(&srow[rl * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
+      *reinterpret_cast<float4*>(&srow[rl * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
     }
     if (gamma && e0 < D) {
       float g[8];
       load8<BF>(gamma, e0, g);
 #pragma unroll
-      for (int t = 0; t < 8; ++t) w[j][t] = fmul(w[j][t], g[t]);
+      for (int t = 0; t < 8; ++t) w[jj][t] = fmul(w[jj][t], g[t]);
     }
 #pragma unroll
-    for (int t = 0; t < 8; ++t) pr[t] = fmul(w[j][t], xh[j][t]);
+    for (int t = 0; t < 8; ++t) pr[t] = fmul(w[jj][t], xh[jj][t]);
     const float t8 = tree8_full(pr);
     const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
-    if (lane == j) mine = leaf;
+    if (lane == jj) mine = leaf;
   }
-  const float c = fmul(warp_tree(mine, 0, 256, D), invD);
+  // tree over this warp's four leaf sums (lanes 0..3), then over the two halves of the row
+#pragma unroll
+  for (int wd = 1; wd < 4; wd <<= 1) {
+    const float o = __shfl_xor_sync(0xffffffffu, mine, wd);
+    const int right_leaf = hw * 4 + ((lane | wd) & ~(wd - 1));
+    const bool right_valid = (long long)right_leaf * 256 < D;
+    mine = right_valid ? fadd(mine, o) : ((lane & wd) ? o : mine);
+  }
+  if (lane == 0) half_sum[rl][hw] = mine;
+  __syncthreads();
+  const float tot = (D > 1024) ? fadd(half_sum[rl][0], half_sum[rl][1]) : half_sum[rl][0];
+  const float c = fmul(tot, invD);
   if (live) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int e0 = j * 256 + lane * 8;
+    for (int jj = 0; jj < 4; ++jj) {
+      const int e0 = (hw * 4 + jj) * 256 + lane * 8;
       if (e0 >= D) continue;
       float o[8];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[j][t], fmul(xh[j][t], c)));
+      for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[jj][t], fmul(xh[jj][t], c)));
       store8<BF>(dx, rb + e0, o);
     }
   }
   if (DG) {
-    __syncthreads();
     const long long r0 = (long long)blockIdx.x * 8;
-    for (int col = threadIdx.x; col < D; col += 256) {
+    for (int col = threadIdx.x; col < D; col += 512) {
       float v[8];
 #pragma unroll
       for (int r = 0; r < 8; ++r) v[r] = srow[r * D + col];
@@ -480,7 +494,7 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
                                float invD, void* dx, float* dgamma, float* ws, cudaStream_t st) {
   dim3 grid((rows + 7) / 8);
   if (!dgamma) {
-    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
+    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 512, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
     return DET_OK;
   }
   static bool cfg = false;
@@ -492,7 +506,7 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
   const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
   float* partial8 = ws;
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);
-  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 256, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
+  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 512, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
   dim3 g2((D + 255) / 256, nb256);
   k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256);
   k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>(partial256, nb256, D, dgamma, rows);
