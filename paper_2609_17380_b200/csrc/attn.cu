@@ -53,8 +53,12 @@ __device__ __forceinline__ void mac_8x8(const float (*As)[LQ], const float (*Bs)
       const float2 a = make_float2(av[i], av[i]);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        if (FUSED) acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
-        else acc[i][j] = __fadd2_rn(acc[i][j], __fmul2_rn(a, b[j]));
+        if (FUSED) {
+          acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
+        } else {  // scalar on purpose: a packed multiply + add pair would be contracted by ptxas
+          acc[i][j].x = fadd(acc[i][j].x, fmul(av[i], b[j].x));
+          acc[i][j].y = fadd(acc[i][j].y, fmul(av[i], b[j].y));
+        }
       }
     }
   }
@@ -191,9 +195,11 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     else mac_8x8<true>(Ps, KV, kmax, ty, tx, u);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float2 al = make_float2(alpha[i], alpha[i]);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) o[i][e] = __fadd2_rn(__fmul2_rn(o[i][e], al), u[i][e]);
+      for (int e = 0; e < 4; ++e) {  // scalar: the product o*alpha is rounded before the add
+        o[i][e].x = fadd(fmul(o[i][e].x, alpha[i]), u[i][e].x);
+        o[i][e].y = fadd(fmul(o[i][e].y, alpha[i]), u[i][e].y);
+      }
     }
     __syncthreads();  // V and P~ may be overwritten by the next tile
   }

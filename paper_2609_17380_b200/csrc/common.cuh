@@ -55,6 +55,13 @@ __device__ __forceinline__ float det_exp(float x) {
   return fmul(p, __int_as_float((k + 127) << 23));
 }
 
+// NOTE on the packed two-lane FP32 instructions (mul/add/fma .f32x2): each lane of a single packed instruction
+// rounds exactly like the scalar instruction, but ptxas contracts a packed multiply followed by a packed add into one
+// fused instruction even when both carry .rn and --fmad=false is given (measured on this toolchain: the result
+// equals the true fused multiply-add in every lane).  Packed arithmetic is therefore used only where a fused
+// multiply-add is wanted and proven identical; every multiply-then-add whose product must be rounded on its own is
+// written with the scalar intrinsics, which ptxas never contracts.
+
 // log for normal x > 0: x = 2^e m, m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1), z = s^2,
 // log m = 2 s (1 + z/3 + z^2/5 + z^3/7 + z^4/9).
 __device__ __forceinline__ float det_log(float x) {

@@ -109,8 +109,12 @@ __device__ __forceinline__ void slab_mac(const float (*As)[OT + 4], const float 
       const float2 a = make_float2(av[i], av[i]);
 #pragma unroll
       for (int j = 0; j < TN / 32; ++j) {
-        if (FUSED) acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
-        else acc[i][j] = __fadd2_rn(acc[i][j], __fmul2_rn(a, b[j]));
+        if (FUSED) {
+          acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
+        } else {  // scalar on purpose: a packed multiply + add pair would be contracted by ptxas
+          acc[i][j].x = fadd(acc[i][j].x, fmul(av[i], b[j].x));
+          acc[i][j].y = fadd(acc[i][j].y, fmul(av[i], b[j].y));
+        }
       }
     }
   }

@@ -414,3 +414,64 @@ def test_attention(det, B, H, S):
     got = host(dqkv, np.uint16)
     for name, c in (("dq", 0), ("dk", 1), ("dv", 2)):
         assert_same_bits(got[:, c * HD:(c + 1) * HD], want[:, c * HD:(c + 1) * HD], name)
+
+
+# ------------------------------------------------------------------ slabs whose products can underflow
+def _sprinkle_tiny(a, seed, frac=0.002):
+    """Overwrite a fraction of a bf16 tensor with magnitudes around 2^-64 .. 2^-62 (random signs)."""
+    rng = np.random.default_rng(seed)
+    flat = a.reshape(-1)
+    idx = rng.choice(flat.size, max(4, int(flat.size * frac)), replace=False)
+    vals = (2.0 ** rng.integers(-66, -61, idx.size)) * rng.choice([-1.0, 1.0, 1.5, -1.25], idx.size)
+    flat[idx] = synth.to_bf16(vals.astype(F))
+    return a
+
+
+def test_lmhead_subnormal_products(det):
+    # 1.5*2^-126 + 2^-127: the second product is subnormal, so multiply-flush-add keeps 1.5*2^-126 while a fused
+    # multiply-add would give 2^-125; the kernel must notice the tiny factors and take the unfused sequence
+    M, V, K = 128, 256, 64
+    Hh = synth.normal_bf16((M, K), 1.0, seed=21, tid=1)
+    W = synth.normal_bf16((V, K), 0.02, seed=21, tid=2)
+    Hh[0] = 0
+    W[0] = 0
+    Hh[0, :2] = synth.to_bf16(np.array([2.0 ** -63, 2.0 ** -64], F))
+    W[0, :2] = synth.to_bf16(np.array([1.5 * 2.0 ** -63, 2.0 ** -63], F))
+    _sprinkle_tiny(Hh[1:], 1)
+    _sprinkle_tiny(W[1:], 2)
+    lg = empty((M, V), F)
+    det.det_lmhead_fwd(dev(Hh), dev(W), M, V, K, lg)
+    _sync()
+    want = oracle.lmhead_fwd(Hh, W)
+    assert want[0, 0] == F(1.5 * 2.0 ** -126)
+    assert_same_bits(host(lg), want, "logits with subnormal products")
+    dl = synth.normal_f32((M, V), 1e-3, seed=21, tid=3)
+    dl.reshape(-1)[::97] = F(2.0 ** -65)
+    dH, dW = empty((M, K), np.uint16), empty((V, K), F)
+    det.det_lmhead_bwd(dev(dl), dev(Hh), dev(W), M, V, K, dH, dW, 1)
+    _sync()
+    oH, oW = oracle.lmhead_bwd(dl, Hh, W)
+    assert_same_bits(host(dH, np.uint16), oH, "dH")
+    assert_same_bits(host(dW), oW, "dW")
+
+
+def test_attention_subnormal_products(det):
+    B, H, S = 1, 2, 256
+    HD = H * 128
+    qkv = _sprinkle_tiny(synth.normal_bf16((B * S, 3 * HD), 1.0, seed=22, tid=1), 3, 0.01)
+    qkv[5:9, :] = synth.to_bf16(np.full((4, 3 * HD), 2.0 ** -64, F))       # whole rows of tiny q, k, v
+    dout = _sprinkle_tiny(synth.normal_bf16((B * S, HD), 0.1, seed=22, tid=2), 4, 0.01)
+    dqkv_in = dev(qkv)
+    base = dqkv_in.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    det.det_attn_fwd(base, base + 2 * HD, base + 4 * HD, 3 * HD, B, H, S, out, HD, lse)
+    _sync()
+    oout, olse = oracle.attn_fwd(qkv, B, H, S)
+    assert_same_bits(host(lse), olse, "lse")
+    assert_same_bits(host(out, np.uint16), oout, "out")
+    dqkv = empty((B * S, 3 * HD), np.uint16)
+    db = dqkv.data_ptr()
+    det.det_attn_bwd(dev(dout), base, base + 2 * HD, base + 4 * HD, out, lse, 3 * HD, HD, B, H, S, db, db + 2 * HD,
+                     db + 4 * HD, 3 * HD, ws(det.det_attn_bwd_ws_bytes(B, H, S)))
+    _sync()
+    assert_same_bits(host(dqkv, np.uint16), oracle.attn_bwd(dout, qkv, oout, olse, B, H, S), "dqkv")
