@@ -217,8 +217,11 @@ int det_adamw_step(const det_adamw_desc* h, int pdtype, void* p, const float* g,
                    void* stream);
 
 /* ---- tensor hash (Appendix B: per-step state hash, here on the device) --------------------------------
- * SHA-256 of every 64 KiB chunk of the raw bytes on the device; root = SHA-256(chunk digests || u64le(nbytes))
- * finished on the host.  out32_host receives 32 bytes.  Synchronises `stream`. */
+ * Level 1: SHA-256 of every 4 KiB chunk of the raw bytes (last chunk may be shorter).  While more than 2048
+ * digests remain, the concatenated digests are hashed again in 64 KiB blocks.  root = SHA-256(remaining digests
+ * || u64le(nbytes)), finished on the host; every level below it runs on the device.  p device, 16-byte aligned;
+ * ws device, 16-byte aligned, det_tensor_hash_ws_bytes(nbytes) bytes; out32_host receives 32 bytes.
+ * Synchronises `stream`. */
 size_t det_tensor_hash_ws_bytes(size_t nbytes);
 int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes, void* stream);
 

@@ -252,7 +252,9 @@ __global__ void __launch_bounds__(256) k_adamw(AdamScalars h, void* __restrict__
 }
 
 // ------------------------------------------------------------------------------------------------
-// SHA-256 of 64 KiB chunks: one thread per chunk, message words fetched with 128-bit loads.
+// SHA-256 of fixed-size chunks (4 KiB leaves of the data, 64 KiB blocks of digests above them): one thread per
+// chunk, message words fetched with 128-bit loads.  The small leaf gives a multi-gigabyte tensor hundreds of
+// thousands of independent chains, which is what fills the integer pipes.
 // ------------------------------------------------------------------------------------------------
 __constant__ uint32_t c_K[64] = {
     0x428a2f98, 0x71374491, 0xb5c0fbcf, 0xe9b5dba5, 0x3956c25b, 0x59f111f1, 0x923f82a4, 0xab1c5ed5, 0xd807aa98,
@@ -284,21 +286,30 @@ __device__ __forceinline__ void sha_rounds(uint32_t h[8], uint32_t w[16]) {
 }
 
 __global__ void __launch_bounds__(64) k_sha_chunks(const uint8_t* __restrict__ data, size_t nbytes, size_t nchunks,
-                                                   uint8_t* __restrict__ digests) {
+                                                   size_t CH, uint8_t* __restrict__ digests) {
   size_t c = (size_t)blockIdx.x * 64 + threadIdx.x;
   if (c >= nchunks) return;
-  const size_t CH = 65536;
   const uint8_t* p = data + c * CH;
   const size_t len = (c + 1) * CH <= nbytes ? CH : nbytes - c * CH;
   uint32_t h[8] = {0x6a09e667, 0xbb67ae85, 0x3c6ef372, 0xa54ff53a, 0x510e527f, 0x9b05688c, 0x1f83d9ab, 0x5be0cd19};
   uint32_t w[16];
   const size_t full = len / 64;
+  // the next 64-byte block is fetched while the 64 rounds of the current one run
+  uint4 nx[4];
+  if (full) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) nx[k] = __ldg(reinterpret_cast<const uint4*>(p) + k);
+  }
   for (size_t b = 0; b < full; ++b) {
-    const uint4* q = reinterpret_cast<const uint4*>(p + b * 64);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      uint4 u = __ldg(q + k);
+      const uint4 u = nx[k];
       w[4 * k] = bswap(u.x); w[4 * k + 1] = bswap(u.y); w[4 * k + 2] = bswap(u.z); w[4 * k + 3] = bswap(u.w);
+    }
+    if (b + 1 < full) {
+      const uint4* q = reinterpret_cast<const uint4*>(p + (b + 1) * 64);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) nx[k] = __ldg(q + k);
     }
     sha_rounds(h, w);
   }
@@ -317,10 +328,9 @@ __global__ void __launch_bounds__(64) k_sha_chunks(const uint8_t* __restrict__ d
              ((uint32_t)tail[b * 64 + 4 * k + 2] << 8) | (uint32_t)tail[b * 64 + 4 * k + 3];
     sha_rounds(h, w);
   }
-  for (int i = 0; i < 8; ++i) {
-    digests[c * 32 + 4 * i] = (uint8_t)(h[i] >> 24); digests[c * 32 + 4 * i + 1] = (uint8_t)(h[i] >> 16);
-    digests[c * 32 + 4 * i + 2] = (uint8_t)(h[i] >> 8); digests[c * 32 + 4 * i + 3] = (uint8_t)h[i];
-  }
+  uint4* o = reinterpret_cast<uint4*>(digests + c * 32);
+  o[0] = make_uint4(bswap(h[0]), bswap(h[1]), bswap(h[2]), bswap(h[3]));
+  o[1] = make_uint4(bswap(h[4]), bswap(h[5]), bswap(h[6]), bswap(h[7]));
 }
 
 // host-side SHA-256 for the root over the chunk digests
@@ -541,24 +551,34 @@ extern "C" int det_adamw_step(const det_adamw_desc* d, int pdtype, void* p, cons
   return DET_OK;
 }
 
-extern "C" size_t det_tensor_hash_ws_bytes(size_t nbytes) { return align_up(((nbytes + 65535) / 65536) * 32 + 32, 256); }
+// Workspace: the level-1 digests followed by the (much shorter) upper levels, ping-ponged in two areas.
+static inline size_t hash_l1_bytes(size_t nbytes) { return align_up(((nbytes + 4095) / 4096) * 32 + 32, 256); }
+static inline size_t hash_l2_bytes(size_t nbytes) { return align_up(((nbytes + 4095) / 4096) / 64 + 64, 256); }
+extern "C" size_t det_tensor_hash_ws_bytes(size_t nbytes) { return hash_l1_bytes(nbytes) + hash_l2_bytes(nbytes); }
 
 extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes,
                                void* stream) {
   if ((nbytes && !p) || !out32_host) return DET_ERR_ARG;
   if (nbytes && !aligned16(p)) return DET_ERR_ALIGN;
-  if (ws_bytes < det_tensor_hash_ws_bytes(nbytes) || !ws) return DET_ERR_WORKSPACE;
+  if (ws_bytes < det_tensor_hash_ws_bytes(nbytes) || !ws || !aligned16(ws)) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t nc = (nbytes + 65535) / 65536;
-  if (nc) k_sha_chunks<<<DET_L((unsigned)((nc + 63) / 64)), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, (uint8_t*)ws);
+  uint8_t* a = (uint8_t*)ws;
+  uint8_t* b = a + hash_l1_bytes(nbytes);
+  size_t nc = (nbytes + 4095) / 4096;
+  if (nc) k_sha_chunks<<<DET_L((unsigned)((nc + 63) / 64)), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, 4096, a);
   DET_CHECK_LAUNCH();
-  uint8_t* host = (uint8_t*)malloc(nc * 32 + 8);
-  if (!host) return DET_ERR_ARG;
-  if (nc && cudaMemcpyAsync(host, ws, nc * 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) { free(host); return DET_ERR_CUDA; }
-  if (cudaStreamSynchronize(st) != cudaSuccess) { free(host); return DET_ERR_CUDA; }
+  while (nc > 2048) {
+    const size_t lb = nc * 32, m = (lb + 65535) / 65536;
+    k_sha_chunks<<<DET_L((unsigned)((m + 63) / 64)), 64, 0, st>>>(a, lb, m, 65536, b);
+    DET_CHECK_LAUNCH();
+    uint8_t* t = a; a = b; b = t;
+    nc = m;
+  }
+  uint8_t host[2048 * 32 + 8];
+  if (nc && cudaMemcpyAsync(host, a, nc * 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DET_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DET_ERR_CUDA;
   unsigned long long nn = nbytes;
   for (int i = 0; i < 8; ++i) host[nc * 32 + i] = (uint8_t)(nn >> (8 * i));
   host_sha256(host, nc * 32 + 8, out32_host);
-  free(host);
   return DET_OK;
 }
