@@ -217,8 +217,8 @@ int det_adamw_step(const det_adamw_desc* h, int pdtype, void* p, const float* g,
                    void* stream);
 
 /* ---- tensor hash (Appendix B: per-step state hash, here on the device) --------------------------------
- * Level 1: SHA-256 of every 4 KiB chunk of the raw bytes (last chunk may be shorter).  While more than 2048
- * digests remain, the concatenated digests are hashed again in 64 KiB blocks.  root = SHA-256(remaining digests
+ * Level 1: SHA-256 of every 4 KiB chunk of the raw bytes (last chunk may be shorter).  While more than 128
+ * digests remain, the concatenated digests are hashed again in 4 KiB blocks (128 digests each).  root = SHA-256(remaining digests
  * || u64le(nbytes)), finished on the host; every level below it runs on the device.  p device, 16-byte aligned;
  * ws device, 16-byte aligned, det_tensor_hash_ws_bytes(nbytes) bytes; out32_host receives 32 bytes.
  * Synchronises `stream`. */

@@ -749,26 +749,24 @@ void orc_sha256(const uint8_t *data, size_t n, uint8_t out[32]) {
 }
 /* Tree hash of a tensor's raw bytes (the per-step state hash; Appendix B only says "sharded canonical hash"):
  *   level 1: SHA-256 of every 4 KiB chunk of the data (the last chunk may be shorter);
- *   while more than 2048 digests remain: SHA-256 of every 64 KiB block of the concatenated digests;
+ *   while more than 128 digests remain: SHA-256 of every 4 KiB block (128 digests) of the concatenated digests;
  *   root = SHA-256(remaining digests || u64le(nbytes)). */
-static size_t hash_level(const uint8_t *data, size_t n, size_t chunk, uint8_t *out) {
-  size_t nc = (n + chunk - 1) / chunk;
+static size_t hash_level(const uint8_t *data, size_t n, uint8_t *out) {
+  size_t nc = (n + 4095) / 4096;
 #pragma omp parallel for
   for (size_t c = 0; c < nc; ++c) {
-    size_t len = (c + 1) * chunk <= n ? chunk : n - c * chunk;
-    orc_sha256(data + c * chunk, len, out + 32 * c);
+    size_t len = (c + 1) * 4096 <= n ? 4096 : n - c * 4096;
+    orc_sha256(data + c * 4096, len, out + 32 * c);
   }
   return nc;
 }
 void orc_tensor_hash(const uint8_t *data, size_t n, uint8_t out[32]) {
-  size_t nc = (n + 4095) / 4096;
-  uint8_t *a = (uint8_t *)malloc(nc * 32 + 8), *b = (uint8_t *)malloc(nc / 64 + 64 + 8);
-  nc = hash_level(data, n, 4096, a);
-  while (nc > 2048) {
-    size_t m = hash_level(a, nc * 32, 65536, b);
+  size_t cap = ((n + 4095) / 4096) * 32 + 64;
+  uint8_t *a = (uint8_t *)malloc(cap), *b = (uint8_t *)malloc(cap);
+  size_t nc = hash_level(data, n, a);
+  while (nc > 128) {
+    nc = hash_level(a, nc * 32, b);
     uint8_t *t = a; a = b; b = t;
-    nc = m;
-    b = (uint8_t *)realloc(b, nc * 32 + 8 > 64 ? nc * 32 + 8 : 64);
   }
   uint64_t nn = n;
   for (int i = 0; i < 8; ++i) a[nc * 32 + i] = (uint8_t)(nn >> (8 * i));

@@ -252,9 +252,10 @@ __global__ void __launch_bounds__(256) k_adamw(AdamScalars h, void* __restrict__
 }
 
 // ------------------------------------------------------------------------------------------------
-// SHA-256 of fixed-size chunks (4 KiB leaves of the data, 64 KiB blocks of digests above them): one thread per
-// chunk, message words fetched with 128-bit loads.  The small leaf gives a multi-gigabyte tensor hundreds of
-// thousands of independent chains, which is what fills the integer pipes.
+// SHA-256 of 4 KiB chunks (of the data at level 1, of the concatenated digests above it): one thread per chunk,
+// message words fetched with 128-bit loads.  A chunk is one sequential chain of 64 compressions (~0.1 ms), so the
+// small chunk both bounds the latency of the short upper levels and gives a multi-gigabyte tensor hundreds of
+// thousands of independent chains to fill the integer pipes.
 // ------------------------------------------------------------------------------------------------
 __constant__ uint32_t c_K[64] = {
     0x428a2f98, 0x71374491, 0xb5c0fbcf, 0xe9b5dba5, 0x3956c25b, 0x59f111f1, 0x923f82a4, 0xab1c5ed5, 0xd807aa98,
@@ -286,9 +287,10 @@ __device__ __forceinline__ void sha_rounds(uint32_t h[8], uint32_t w[16]) {
 }
 
 __global__ void __launch_bounds__(64) k_sha_chunks(const uint8_t* __restrict__ data, size_t nbytes, size_t nchunks,
-                                                   size_t CH, uint8_t* __restrict__ digests) {
+                                                   uint8_t* __restrict__ digests) {
   size_t c = (size_t)blockIdx.x * 64 + threadIdx.x;
   if (c >= nchunks) return;
+  const size_t CH = 4096;
   const uint8_t* p = data + c * CH;
   const size_t len = (c + 1) * CH <= nbytes ? CH : nbytes - c * CH;
   uint32_t h[8] = {0x6a09e667, 0xbb67ae85, 0x3c6ef372, 0xa54ff53a, 0x510e527f, 0x9b05688c, 0x1f83d9ab, 0x5be0cd19};
@@ -551,10 +553,11 @@ extern "C" int det_adamw_step(const det_adamw_desc* d, int pdtype, void* p, cons
   return DET_OK;
 }
 
-// Workspace: the level-1 digests followed by the (much shorter) upper levels, ping-ponged in two areas.
+// Workspace: two areas of level-1 size, ping-ponged by the levels.
 static inline size_t hash_l1_bytes(size_t nbytes) { return align_up(((nbytes + 4095) / 4096) * 32 + 32, 256); }
-static inline size_t hash_l2_bytes(size_t nbytes) { return align_up(((nbytes + 4095) / 4096) / 64 + 64, 256); }
-extern "C" size_t det_tensor_hash_ws_bytes(size_t nbytes) { return hash_l1_bytes(nbytes) + hash_l2_bytes(nbytes); }
+extern "C" size_t det_tensor_hash_ws_bytes(size_t nbytes) {
+  return hash_l1_bytes(nbytes) + hash_l1_bytes(hash_l1_bytes(nbytes));
+}
 
 extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes,
                                void* stream) {
@@ -565,16 +568,16 @@ extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host
   uint8_t* a = (uint8_t*)ws;
   uint8_t* b = a + hash_l1_bytes(nbytes);
   size_t nc = (nbytes + 4095) / 4096;
-  if (nc) k_sha_chunks<<<DET_L((unsigned)((nc + 63) / 64)), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, 4096, a);
+  if (nc) k_sha_chunks<<<DET_L((unsigned)((nc + 63) / 64)), 64, 0, st>>>((const uint8_t*)p, nbytes, nc, a);
   DET_CHECK_LAUNCH();
-  while (nc > 2048) {
-    const size_t lb = nc * 32, m = (lb + 65535) / 65536;
-    k_sha_chunks<<<DET_L((unsigned)((m + 63) / 64)), 64, 0, st>>>(a, lb, m, 65536, b);
+  while (nc > 128) {
+    const size_t lb = nc * 32, m = (lb + 4095) / 4096;
+    k_sha_chunks<<<DET_L((unsigned)((m + 63) / 64)), 64, 0, st>>>(a, lb, m, b);
     DET_CHECK_LAUNCH();
     uint8_t* t = a; a = b; b = t;
     nc = m;
   }
-  uint8_t host[2048 * 32 + 8];
+  uint8_t host[128 * 32 + 8];
   if (nc && cudaMemcpyAsync(host, a, nc * 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DET_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return DET_ERR_CUDA;
   unsigned long long nn = nbytes;

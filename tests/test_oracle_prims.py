@@ -134,14 +134,14 @@ def test_sha256_and_tensor_hash():
     assert oracle.sha256(np.frombuffer(msg, np.uint8)) == \
         "248d6a61d20638b8e5c026930c3e6039a33ce45964ff2167f6ecedd419db06c1"      # FIPS 180-4 example
     rng = np.random.default_rng(0)
-    # 2048 * 4096 bytes is the largest input with a single level; beyond it the digests are hashed in 64 KiB blocks
-    for n in (0, 1, 55, 56, 63, 64, 65, 119, 120, 4095, 4096, 4097, 65537, 200001, 2048 * 4096, 2048 * 4096 + 1,
-              3 * 2048 * 4096 + 777):
+    # 128 * 4096 bytes is the largest input with a single level, 128 * 128 * 4096 the largest with two
+    for n in (0, 1, 55, 56, 63, 64, 65, 119, 120, 4095, 4096, 4097, 65537, 200001, 128 * 4096, 128 * 4096 + 1,
+              3 * 128 * 4096 + 777, 128 * 128 * 4096 + 5000):
         b = rng.integers(0, 256, n).astype(np.uint8)
         assert oracle.sha256(b) == hashlib.sha256(b.tobytes()).hexdigest()
         d = b"".join(hashlib.sha256(b[i:i + 4096].tobytes()).digest() for i in range(0, n, 4096))
-        while len(d) > 2048 * 32:
-            d = b"".join(hashlib.sha256(d[i:i + 65536]).digest() for i in range(0, len(d), 65536))
+        while len(d) > 128 * 32:
+            d = b"".join(hashlib.sha256(d[i:i + 4096]).digest() for i in range(0, len(d), 4096))
         root = hashlib.sha256(d + int(n).to_bytes(8, "little")).hexdigest()
         assert oracle.tensor_hash(b) == root
 
