@@ -267,10 +267,12 @@ __global__ void __launch_bounds__(256, 1)
 #pragma unroll
     for (int c = 0; c < 4; ++c) { sa[a][c] = make_float2(0.f, 0.f); da[a][c] = make_float2(0.f, 0.f); }
   float vq[8], vo[8], vk[8], vv[8];
-  slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, 0, vq);
-  slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, 0, vo);
-  slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, 0, vk);
-  slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, 0, vv);
+  Raw8<false> rq[1], ro[1], rk[1], rv[1];
+  slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, 0, rq);
+  slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, 0, ro);
+  slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, 0, rk);
+  slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, 0, rv);
+  unpack8<false>(rq[0], vq); unpack8<false>(ro[0], vo); unpack8<false>(rk[0], vk); unpack8<false>(rv[0], vv);
   slab_store<CONTIG, OT>(Qs[0], vq); slab_store<CONTIG, OT>(Os[0], vo);
   slab_store<CONTIG, OT>(Ks[0], vk); slab_store<CONTIG, OT>(Vs[0], vv);
   int tiny = __syncthreads_or(tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv));
@@ -278,15 +280,16 @@ __global__ void __launch_bounds__(256, 1)
   for (int s = 0; s < NS; ++s) {
     const int cur = s & 1;
     if (s + 1 < NS) {
-      slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, (s + 1) * OK, vq);
-      slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, (s + 1) * OK, vo);
-      slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, (s + 1) * OK, vk);
-      slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, (s + 1) * OK, vv);
+      slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, (s + 1) * OK, rq);
+      slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, (s + 1) * OK, ro);
+      slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, (s + 1) * OK, rk);
+      slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, (s + 1) * OK, rv);
     }
     if (tiny) { slab_mac<false, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<false, OT>(Os[cur], Vs[cur], ty, tx, da); }
     else { slab_mac<true, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<true, OT>(Os[cur], Vs[cur], ty, tx, da); }
     bool nt = false;
     if (s + 1 < NS) {
+      unpack8<false>(rq[0], vq); unpack8<false>(ro[0], vo); unpack8<false>(rk[0], vk); unpack8<false>(rv[0], vv);
       slab_store<CONTIG, OT>(Qs[cur ^ 1], vq); slab_store<CONTIG, OT>(Os[cur ^ 1], vo);
       slab_store<CONTIG, OT>(Ks[cur ^ 1], vk); slab_store<CONTIG, OT>(Vs[cur ^ 1], vv);
       nt = tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv);

@@ -15,21 +15,37 @@ constexpr int OK = 16;   // slab depth
 //   STRIDED: operand stored [contraction, rows] (row index contiguous)
 enum { CONTIG = 0, STRIDED = 1 };
 
+// Raw global data of 8 operand values: one 16-byte word of bf16, or two of f32.  The words stay packed in registers
+// while the current slab is multiplied and are only unpacked when they are stored to shared memory, so the unpacking
+// instructions (which wait for the load) sit after the multiply loop instead of in front of it.
 template <bool F32IN>
-__device__ __forceinline__ void load8_any(const void* base, size_t idx, bool ok, float v[8]) {
+struct Raw8 {
+  uint4 w[F32IN ? 2 : 1];
+};
+template <bool F32IN>
+__device__ __forceinline__ void load8_raw(const void* base, size_t idx, bool ok, Raw8<F32IN>& r) {
   if (!ok) {
 #pragma unroll
-    for (int t = 0; t < 8; ++t) v[t] = 0.0f;
+    for (int t = 0; t < (F32IN ? 2 : 1); ++t) r.w[t] = make_uint4(0u, 0u, 0u, 0u);
     return;
   }
   if (F32IN) {
-    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + idx);
-    float4 a = __ldg(p), b = __ldg(p + 1);
-    // operands of the gradient contractions are rounded to bf16 first
-    v[0] = bf2f(f2bf(a.x)); v[1] = bf2f(f2bf(a.y)); v[2] = bf2f(f2bf(a.z)); v[3] = bf2f(f2bf(a.w));
-    v[4] = bf2f(f2bf(b.x)); v[5] = bf2f(f2bf(b.y)); v[6] = bf2f(f2bf(b.z)); v[7] = bf2f(f2bf(b.w));
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(base) + idx);
+    r.w[0] = __ldg(p);
+    r.w[1] = __ldg(p + 1);
   } else {
-    uint4 u = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + idx));
+    r.w[0] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + idx));
+  }
+}
+template <bool F32IN>
+__device__ __forceinline__ void unpack8(const Raw8<F32IN>& r, float v[8]) {
+  if (F32IN) {
+    // operands of the gradient contractions are rounded to bf16 first
+    const uint32_t u[8] = {r.w[0].x, r.w[0].y, r.w[0].z, r.w[0].w, r.w[1].x, r.w[1].y, r.w[1].z, r.w[1].w};
+#pragma unroll
+    for (int t = 0; t < 8; ++t) v[t] = bf2f(f2bf(__uint_as_float(u[t])));
+  } else {
+    const uint4 u = r.w[0];
     v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
     v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
   }
@@ -38,20 +54,26 @@ __device__ __forceinline__ void load8_any(const void* base, size_t idx, bool ok,
 // fetch this thread's values of an operand slab of ROWS rows x 16 contraction steps:
 // ROWS == 128: 8 values per thread, ROWS == 256: 16 values per thread
 template <int MODE, bool F32IN, int ROWS>
-__device__ __forceinline__ void slab_fetch(const void* base, int rows, int C, int ld, int r0, int c0, float* v) {
+__device__ __forceinline__ void slab_fetch(const void* base, int rows, int C, int ld, int r0, int c0,
+                                           Raw8<F32IN> (&raw)[ROWS / 128]) {
   const int tid = threadIdx.x;
   constexpr int NV = ROWS / 16;  // values per thread
   if (MODE == CONTIG) {
     // thread -> (row, 8 or 16 consecutive contraction indices)
     const int r = r0 + (ROWS == 128 ? (tid & 127) : tid), c = c0 + (ROWS == 128 ? (tid >> 7) * 8 : 0);
 #pragma unroll
-    for (int h = 0; h < NV / 8; ++h) load8_any<F32IN>(base, (size_t)r * ld + c + 8 * h, r < rows && c + 8 * h < C, v + 8 * h);
+    for (int h = 0; h < NV / 8; ++h) load8_raw<F32IN>(base, (size_t)r * ld + c + 8 * h, r < rows && c + 8 * h < C, raw[h]);
   } else {
     // thread -> (contraction index, NV consecutive rows)
     const int c = c0 + (tid >> 4), r = r0 + (tid & 15) * NV;
 #pragma unroll
-    for (int h = 0; h < NV / 8; ++h) load8_any<F32IN>(base, (size_t)c * ld + r + 8 * h, c < C && r + 8 * h < rows, v + 8 * h);
+    for (int h = 0; h < NV / 8; ++h) load8_raw<F32IN>(base, (size_t)c * ld + r + 8 * h, c < C && r + 8 * h < rows, raw[h]);
   }
+}
+template <bool F32IN, int ROWS>
+__device__ __forceinline__ void slab_unpack(const Raw8<F32IN> (&raw)[ROWS / 128], float* v) {
+#pragma unroll
+  for (int h = 0; h < ROWS / 128; ++h) unpack8<F32IN>(raw[h], v + 8 * h);
 }
 template <int MODE, int ROWS>
 __device__ __forceinline__ void slab_store(float (*s)[ROWS + 4], const float* v) {
@@ -172,8 +194,12 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
     }
   }
   float va[8], vb[TN / 16];
-  slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, va);
-  slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo, vb);
+  Raw8<AF32> ra[1];
+  Raw8<false> rb[TN / 128];
+  slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, ra);
+  slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo, rb);
+  slab_unpack<AF32, OT>(ra, va);
+  slab_unpack<false, TN>(rb, vb);
   slab_store<AMODE, OT>(As[0], va);
   slab_store<BMODE, TN>(Bs[0], vb);
   int tiny = __syncthreads_or(tiny_any<8>(va) || tiny_any<TN / 16>(vb));
@@ -181,13 +207,15 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   for (int s = 0; s < nslab; ++s) {
     const int cur = s & 1;
     if (s + 1 < nslab) {
-      slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, va);
-      slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, vb);
+      slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, ra);
+      slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, rb);
     }
     if (tiny) slab_mac<false, TN>(As[cur], Bs[cur], ty, tx, acc);
     else slab_mac<true, TN>(As[cur], Bs[cur], ty, tx, acc);
     bool next_tiny = false;
     if (s + 1 < nslab) {
+      slab_unpack<AF32, OT>(ra, va);
+      slab_unpack<false, TN>(rb, vb);
       slab_store<AMODE, OT>(As[cur ^ 1], va);
       slab_store<BMODE, TN>(Bs[cur ^ 1], vb);
       next_tiny = tiny_any<8>(va) || tiny_any<TN / 16>(vb);
