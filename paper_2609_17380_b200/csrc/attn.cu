@@ -104,21 +104,36 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     for (int e = 0; e < 4; ++e) o[i][e] = make_float2(0.0f, 0.0f);
   }
   const int ntiles = q0 / FK + 1;
+  // one 128 x 128 bf16 tile in flight: 8 sixteen-byte words per thread
+  uint4 rw[8];
+  auto fetch_k = [&](int j0) {
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int idx = tid + 256 * it, key = idx & 127, ch = idx >> 7;
+      rw[it] = (j0 + key < S) ? __ldg(reinterpret_cast<const uint4*>(kp + (size_t)(j0 + key) * ld + ch * 8))
+                              : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  fetch_k(0);
   for (int jt = 0; jt < ntiles; ++jt) {
     const int j0 = jt * FK;
-    // ---- K tile, transposed ----
+    // ---- K tile (fetched during the previous tile's P.V), transposed ----
     bool tk = false;
-    for (int idx = tid; idx < FK * 16; idx += 256) {
-      const int key = idx & 127, ch = idx >> 7;
-      float t[8];
-      if (j0 + key < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(kp + (size_t)(j0 + key) * ld + ch * 8)), t);
-      else {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) t[e] = 0.0f;
-      }
+    for (int it = 0; it < 8; ++it) {
+      const int idx = tid + 256 * it, key = idx & 127, ch = idx >> 7;
+      float t[8];
+      unpack8a(rw[it], t);
       tk |= tiny8a(t);
 #pragma unroll
       for (int e = 0; e < 8; ++e) KV[ch * 8 + e][key] = t[e];
+    }
+    // V words of this tile travel while the logits are computed
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int idx = tid + 256 * it, key = idx >> 4, ch = idx & 15;
+      rw[it] = (j0 + key < S) ? __ldg(reinterpret_cast<const uint4*>(vp + (size_t)(j0 + key) * ld + ch * 8))
+                              : make_uint4(0u, 0u, 0u, 0u);
     }
     const int tiny_k = __syncthreads_or(tk);
     float2 s[8][4];
@@ -171,18 +186,17 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     __syncthreads();  // every thread is done with K; P~ is complete
     // ---- V tile, natural layout, into the same buffer ----
     bool tv = false;
-    for (int idx = tid; idx < FK * 16; idx += 256) {
-      const int key = idx >> 4, ch = idx & 15;
-      float t[8];
-      if (j0 + key < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(vp + (size_t)(j0 + key) * ld + ch * 8)), t);
-      else {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) t[e] = 0.0f;
-      }
+    for (int it = 0; it < 8; ++it) {
+      const int idx = tid + 256 * it, key = idx >> 4, ch = idx & 15;
+      float t[8];
+      unpack8a(rw[it], t);
       tv |= tiny8a(t);
       *reinterpret_cast<float4*>(&KV[key][ch * 8]) = make_float4(t[0], t[1], t[2], t[3]);
       *reinterpret_cast<float4*>(&KV[key][ch * 8 + 4]) = make_float4(t[4], t[5], t[6], t[7]);
     }
+    // K words of the next tile travel during P.V
+    if (jt + 1 < ntiles) fetch_k(j0 + FK);
     const int tiny_pv = __syncthreads_or(tp || tv);
     // ---- u = P~ . V over the tile's keys in ascending order, then o = o*alpha + u ----
     float2 u[8][4];
