@@ -21,35 +21,38 @@ __device__ __forceinline__ void unpack8a(const uint4& u, float v[8]) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// forward: CTA = 128 queries of one (batch, head); 256 threads, thread = 8 queries x 8 keys / 8 dims.
-// Shared memory (f32): Q [dim][query], one buffer that holds K [dim][key] during the logits and V [key][dim]
+// forward: CTA = 128 queries of one (batch, head); 512 threads (four warps per scheduler, so that the softmax and
+// staging phases, which are chains of dependent instructions, overlap across warps), thread = 4 queries x 8 keys /
+// 8 dims.  Shared memory (f32): Q [dim][query], one buffer that holds K [dim][key] during the logits and V [key][dim]
 // during P.V, and P~ [key][query].  Multiply-adds use the fused instruction whenever no factor of the tile is
 // below 2^-63 in magnitude (then the exact bf16 x bf16 product cannot be subnormal and fused = unfused bit for bit).
 // ---------------------------------------------------------------------------------------------
-constexpr int FQ = 128, FK = 128;
+constexpr int FQ = 128, FK = 128, FT = 512;
 constexpr int LQ = FQ + 4;
 constexpr size_t FWD_SMEM = (size_t)(3 * DH * LQ) * sizeof(float);
 
+// conservative test for 0 < |v| < 2^-63 (also true for subnormal v, which only selects the slower exact path)
+__device__ __forceinline__ bool tiny1(float v) { return (__float_as_uint(v) * 2u - 1u) < 0x3fffffffu; }
 __device__ __forceinline__ bool tiny8a(const float v[8]) {
   bool t = false;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) t |= (((__float_as_uint(v[i]) >> 23) & 0xffu) - 1u) < 63u;
+  for (int i = 0; i < 8; ++i) t |= tiny1(v[i]);
   return t;
 }
 
+// acc[i][j] += A[k][ty*4 + i] * B[k][{tx*4.., 64 + tx*4..}] for k ascending
 template <bool FUSED>
-__device__ __forceinline__ void mac_8x8(const float (*As)[LQ], const float (*Bs)[LQ], int n, int ty, int tx,
-                                        float2 (&acc)[8][4]) {
-#pragma unroll 4
+__device__ __forceinline__ void mac_4x8(const float (*As)[LQ], const float (*Bs)[LQ], int n, int ty, int tx,
+                                        float2 (&acc)[4][4]) {
+#pragma unroll 8
   for (int k = 0; k < n; ++k) {
     const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
-    const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
     const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
     const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
-    const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float av[4] = {a0.x, a0.y, a0.z, a0.w};
     const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 4; ++i) {
       const float2 a = make_float2(av[i], av[i]);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -64,15 +67,17 @@ __device__ __forceinline__ void mac_8x8(const float (*As)[LQ], const float (*Bs)
   }
 }
 
-__global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                                                     const uint16_t* __restrict__ v, int ld, int H, int S,
-                                                     uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse) {
+__global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                                                    const uint16_t* __restrict__ v, int ld, int H, int S,
+                                                    uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse) {
   extern __shared__ __align__(16) float sm[];
   float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                 // [dim][query]
   float(*KV)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + DH * LQ);       // K: [dim][key]; V: [key][dim]
   float(*Ps)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + 2 * DH * LQ);   // [key][query]
-  const int qb = gridDim.x - 1 - blockIdx.x;  // longest rows first
-  const int h = blockIdx.y, b = blockIdx.z;
+  // blocks are handed out in linear order: the query block is the slow index and runs from the longest rows to the
+  // shortest, so the blocks that are still running at the end are the short ones
+  const int qb = gridDim.y - 1 - blockIdx.y;
+  const int h = blockIdx.x % H, b = blockIdx.x / H;
   const int q0 = qb * FQ;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const size_t row0 = (size_t)b * S;
@@ -80,9 +85,21 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
   const uint16_t* kp = k + row0 * ld + (size_t)h * DH;
   const uint16_t* vp = v + row0 * ld + (size_t)h * DH;
 
+  // one 128 x 128 bf16 tile in flight: 4 sixteen-byte words per thread
+  uint4 rw[4];
+  auto fetch_k = [&](int j0) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + FT * it, key = idx & 127, ch = idx >> 7;
+      rw[it] = (j0 + key < S) ? __ldg(reinterpret_cast<const uint4*>(kp + (size_t)(j0 + key) * ld + ch * 8))
+                              : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  fetch_k(0);
   bool tq = false;
-  for (int idx = tid; idx < FQ * 16; idx += 256) {
-    const int r = idx & 127, ch = idx >> 7;
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int idx = tid + FT * it, r = idx & 127, ch = idx >> 7;
     float t[8];
     if (q0 + r < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(qp + (size_t)(q0 + r) * ld + ch * 8)), t);
     else {
@@ -94,34 +111,23 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     for (int e = 0; e < 8; ++e) Qs[ch * 8 + e][r] = t[e];
   }
   const int tiny_q = __syncthreads_or(tq);
-  float m[8], l[8];
-  float2 o[8][4];
+  float m[4], l[4];
+  float2 o[4][4];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
+  for (int i = 0; i < 4; ++i) {
     m[i] = __int_as_float(0xff800000);
     l[i] = 0.0f;
 #pragma unroll
     for (int e = 0; e < 4; ++e) o[i][e] = make_float2(0.0f, 0.0f);
   }
   const int ntiles = q0 / FK + 1;
-  // one 128 x 128 bf16 tile in flight: 8 sixteen-byte words per thread
-  uint4 rw[8];
-  auto fetch_k = [&](int j0) {
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int idx = tid + 256 * it, key = idx & 127, ch = idx >> 7;
-      rw[it] = (j0 + key < S) ? __ldg(reinterpret_cast<const uint4*>(kp + (size_t)(j0 + key) * ld + ch * 8))
-                              : make_uint4(0u, 0u, 0u, 0u);
-    }
-  };
-  fetch_k(0);
   for (int jt = 0; jt < ntiles; ++jt) {
     const int j0 = jt * FK;
     // ---- K tile (fetched during the previous tile's P.V), transposed ----
     bool tk = false;
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int idx = tid + 256 * it, key = idx & 127, ch = idx >> 7;
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + FT * it, key = idx & 127, ch = idx >> 7;
       float t[8];
       unpack8a(rw[it], t);
       tk |= tiny8a(t);
@@ -130,25 +136,26 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     }
     // V words of this tile travel while the logits are computed
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int idx = tid + 256 * it, key = idx >> 4, ch = idx & 15;
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + FT * it, key = idx >> 4, ch = idx & 15;
       rw[it] = (j0 + key < S) ? __ldg(reinterpret_cast<const uint4*>(vp + (size_t)(j0 + key) * ld + ch * 8))
                               : make_uint4(0u, 0u, 0u, 0u);
     }
     const int tiny_k = __syncthreads_or(tk);
-    float2 s[8][4];
+    float2 s[4][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int e = 0; e < 4; ++e) s[i][e] = make_float2(0.0f, 0.0f);
-    if (tiny_q || tiny_k) mac_8x8<false>(Qs, KV, DH, ty, tx, s);
-    else mac_8x8<true>(Qs, KV, DH, ty, tx, s);
+    if (tiny_q || tiny_k) mac_4x8<false>(Qs, KV, DH, ty, tx, s);
+    else mac_4x8<true>(Qs, KV, DH, ty, tx, s);
     // ---- online softmax statistics per row; P~ to shared memory ----
-    float alpha[8];
+    float alpha[4];
     bool tp = false;
+    const bool diag = (jt == ntiles - 1);  // only the last tile of a row block reaches past the diagonal
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int rl = (i >> 2) * 64 + ty * 4 + (i & 3);
+    for (int i = 0; i < 4; ++i) {
+      const int rl = ty * 4 + i;
       const int row = q0 + rl;
       float sv[8] = {s[i][0].x, s[i][0].y, s[i][1].x, s[i][1].y, s[i][2].x, s[i][2].y, s[i][3].x, s[i][3].y};
       float mt = m[i];
@@ -156,7 +163,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int key = j0 + ((e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4));
-        valid[e] = key <= row;
+        valid[e] = !diag || key <= row;
         sv[e] = fmul(sv[e], ATT_SCALE);
         if (valid[e]) mt = fmaxf(mt, sv[e]);
       }
@@ -170,7 +177,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
       for (int e = 0; e < 8; ++e) {
         const int kl = (e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4);
         const float pt = bf2f(f2bf(p[e]));
-        tp |= (((__float_as_uint(pt) >> 23) & 0xffu) - 1u) < 63u;
+        tp |= tiny1(pt);
         Ps[kl][rl] = pt;
       }
       float h0 = fadd(fadd(p[0], p[1]), fadd(p[2], p[3]));
@@ -187,8 +194,8 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     // ---- V tile, natural layout, into the same buffer ----
     bool tv = false;
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int idx = tid + 256 * it, key = idx >> 4, ch = idx & 15;
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + FT * it, key = idx >> 4, ch = idx & 15;
       float t[8];
       unpack8a(rw[it], t);
       tv |= tiny8a(t);
@@ -199,16 +206,16 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     if (jt + 1 < ntiles) fetch_k(j0 + FK);
     const int tiny_pv = __syncthreads_or(tp || tv);
     // ---- u = P~ . V over the tile's keys in ascending order, then o = o*alpha + u ----
-    float2 u[8][4];
+    float2 u[4][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int e = 0; e < 4; ++e) u[i][e] = make_float2(0.0f, 0.0f);
     const int kmax = min(FK, q0 + FQ - j0);
-    if (tiny_pv) mac_8x8<false>(Ps, KV, kmax, ty, tx, u);
-    else mac_8x8<true>(Ps, KV, kmax, ty, tx, u);
+    if (tiny_pv) mac_4x8<false>(Ps, KV, kmax, ty, tx, u);
+    else mac_4x8<true>(Ps, KV, kmax, ty, tx, u);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 4; ++i) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {  // scalar: the product o*alpha is rounded before the add
         o[i][e].x = fadd(fmul(o[i][e].x, alpha[i]), u[i][e].x);
@@ -218,8 +225,8 @@ __global__ void __launch_bounds__(256, 1) k_attn_fwd(const uint16_t* __restrict_
     __syncthreads();  // V and P~ may be overwritten by the next tile
   }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = q0 + (i >> 2) * 64 + ty * 4 + (i & 3);
+  for (int i = 0; i < 4; ++i) {
+    const int row = q0 + ty * 4 + i;
     if (row >= S) continue;
     const float il = fdiv(1.0f, l[i]);
     uint16_t* op = out + (row0 + row) * ld_out + (size_t)h * DH;
@@ -356,8 +363,8 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
   static bool cfg = false;
   if (!cfg) { if (set_smem((const void*)k_attn_fwd, FWD_SMEM)) return DET_ERR_CUDA; cfg = true; }
-  dim3 grid((S + FQ - 1) / FQ, H, B);
-  k_attn_fwd<<<DET_L(grid), 256, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
+  dim3 grid(H * B, (S + FQ - 1) / FQ);
+  k_attn_fwd<<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -161,7 +161,8 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
   float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
-  const int i0 = blockIdx.y * OT, j0 = blockIdx.x * TN;
+  // blocks are handed out in linear order; with a causal range the longest contractions are put first
+  const int i0 = (p.range_mode == 2 ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y) * OT, j0 = blockIdx.x * TN;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
   const long long zb = blockIdx.z / p.H, zh = blockIdx.z % p.H;
   const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + zh * p.a_h)
