@@ -96,10 +96,7 @@ template <int NV>
 __device__ __forceinline__ bool tiny_any(const float* v) {
   bool t = false;
 #pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    const uint32_t e = (__float_as_uint(v[i]) >> 23) & 0xffu;
-    t |= (e - 1u) < 63u;
-  }
+  for (int i = 0; i < NV; ++i) t |= (__float_as_uint(v[i]) * 2u - 1u) < 0x3fffffffu;  // also true for subnormals
   return t;
 }
 
