@@ -212,11 +212,21 @@ def run_ours(args):
     det.load()
     kw = full_config_kwargs(args.layers)
     cfg = dstep.ModelConfig(**kw)
-    r = dstep.Replay(cfg)
-    r.init_params_on_device(seed=rank)
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(1234 + rank)
     n_mb = cfg.n_microbatches
+    # N > 1: the micro-batches of the one global step are shared out over the ranks and the gradient is exchanged in
+    # the fixed order (same parameters, tokens and resulting hashes on every rank); if N does not divide the
+    # micro-batch count the ranks run independent replicas instead
+    sharded = world > 1 and n_mb % world == 0
+    if sharded:
+        from paper_2609_17380_b200.dist import ShardedReplay
+        rep = ShardedReplay(cfg, rank, world)
+        r = rep.r
+    else:
+        rep = r = dstep.Replay(cfg)
+    seed = 0 if sharded else rank
+    r.init_params_on_device(seed=seed)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + seed)
     tok_dev = torch.randint(0, cfg.vocab, (n_mb, cfg.micro_batch, cfg.seq + 1), generator=gen, device="cuda", dtype=torch.int32)
     tok_host = tok_dev.cpu().pin_memory()
     r.calibrate(tok_dev[0])
@@ -235,7 +245,7 @@ def run_ours(args):
                 tok = tok_host.to("cuda", non_blocking=True)
             else:
                 tok = tok_dev
-            out = r.step(tok, per_tensor_hashes=False, want_losses=host_inputs)
+            out = rep.step(tok, per_tensor_hashes=False, want_losses=host_inputs)
             r.cfg.step += 1
             outs.append(out)
         return outs
@@ -273,14 +283,21 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms, ms_e2e = float(t[0]), float(t[1])
     status = max(o["status"] for o in outs + outs2)
+    agree = None
+    if sharded:   # every rank must hold the same state after the same steps
+        hb = torch.tensor(list(bytes.fromhex(outs2[-1]["hashes"]["params_bf16"])), dtype=torch.uint8, device="cuda")
+        allh = torch.empty(world * 32, dtype=torch.uint8, device="cuda")
+        dist.all_gather_into_tensor(allh, hb)
+        agree = bool((allh.view(world, 32) == hb).all().item())
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
     peaks = measured_peaks()
     per_step = ms / args.steps
-    value = world * tokens_per_step * args.steps / (ms / 1e3)
-    e2e_val = world * tokens_per_step * args.steps / (ms_e2e / 1e3)
+    jobs = 1 if sharded else world          # sharded: all ranks together process one global batch per step
+    value = jobs * tokens_per_step * args.steps / (ms / 1e3)
+    e2e_val = jobs * tokens_per_step * args.steps / (ms_e2e / 1e3)
     # ---- roofline of the dominant kernel group (by device time inside the timed region) ----
     total_prof = sum(v[1] for v in prof.values()) or 1.0
     shares = {k: round(v[1] / total_prof, 4) for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}
@@ -323,16 +340,17 @@ def run_ours(args):
         extra["grad_accum_gbs"] = 3.0 * r.n_grad * 4 * n / (tot_ms / 1e3) / 1e9
         extra["grad_accum_frac_of_hbm"] = extra["grad_accum_gbs"] / peaks["hbm_gbs"]
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": per_step, "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": "int8 tensor-core GEMMs + f32 ordered arithmetic (bf16 storage)", "data": "synthetic",
             "config": {"workload": WORKLOAD if args.layers is None else WORKLOAD + " [REDUCED to %d layers]" % args.layers,
-                       "l2": "inputs_exceed_l2", "multi_gpu": "replicas only" if world > 1 else "single"},
+                       "l2": "inputs_exceed_l2", "multi_gpu": ("micro-batches sharded over ranks, ordered gradient exchange, replicated optimizer" if sharded
+                                     else "replicas only" if world > 1 else "single"), "ranks_agree": agree},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(tok_host.numel() * 4),
                     "d2h_bytes_per_step": int(n_mb * 4 + 8 + 5 * 32)},
             "roofline": roof, "alu_kernels": all_alu, "kernel_time_shares": shares, "component_rates": extra, "peaks": peaks,
             "wall_s_timed": wall, "device_status": status,
-            "state_hash": outs[-1]["hashes"].get("params_bf16")}
+            "state_hash": outs2[-1]["hashes"].get("params_bf16")}
     if world == 1 and not args.no_cpu_baseline:
         try:
             import oracle

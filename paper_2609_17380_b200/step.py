@@ -67,7 +67,10 @@ def _numel(shape):
 class Replay:
     """Device state of the replay: parameters, optimizer moments, gradient buffers, saved activations."""
 
-    def __init__(self, cfg, device="cuda"):
+    def __init__(self, cfg, device="cuda", accum_len=None, gout_len=None):
+        """accum_len: elements per buffer of the accumulation pool (default: the whole gradient); gout_len: allocated
+        length of the reduced-gradient buffer (default: the gradient length).  The sharded replay folds only a slice of
+        the gradient on each GPU and gathers the slices into a padded buffer."""
         self.cfg = cfg
         self.dev = device
         self.specs = param_specs(cfg)
@@ -88,9 +91,10 @@ class Replay:
         self.sx = z(L * 4, F32)                    # LSQ activation steps, [layer, (qkv, o, gu, down)]
         self.m, self.v = z(g, F32), z(g, F32)      # Adam moments, gradient layout
         self.gmb = z(g, F32)                       # gradient of the current micro-batch
-        self.gout = z(g, F32)                      # reduced gradient
+        self.gout_padded = z(max(g, gout_len or 0), F32)
+        self.gout = self.gout_padded[:g]           # reduced gradient
         self.nbufs = det.det_grad_accum_nbufs(cfg.mesh[2])
-        self.abufs = z(self.nbufs * g, F32)
+        self.abufs = z(self.nbufs * (accum_len or g), F32)
         self.lin = {}
         for l in range(L):
             for w, (N, K) in zip(LINEARS, ((3 * D, D), (D, D), (2 * Fh, D), (D, Fh))):

@@ -37,3 +37,63 @@ def test_step_hashes_match_oracle(kw):
     for name, arr in want["params"].items():
         assert np.array_equal(host[name].reshape(-1).view(np.uint8), np.ascontiguousarray(arr).reshape(-1).view(np.uint8)), name
     assert abs(got["loss"] - np.log(cfg.vocab)) < 0.5      # random init: loss ~ log V
+
+
+@pytest.mark.parametrize("world", [1, 2, 4, 8])
+def test_sharded_fold_on_device_matches_single_replay(world):
+    """The multi-GPU step with its transport replaced by plain copies, all ranks played one after the other on one
+    GPU: micro-batch gradients are cut into the ranks' slices, every slice is folded with the library's accumulator
+    at its own offset and length, and the state after clip + AdamW hashes like the single-device replay."""
+    import torch
+    import paper_2609_17380_b200 as det
+    from paper_2609_17380_b200 import step as dstep
+    from paper_2609_17380_b200.dist import ShardPlan, fold_slices
+    kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=512, seq=128, micro_batch=1, mesh=(2, 2, 2))
+    cfg = dstep.ModelConfig(**kw)
+    params = synth.model_params(cfg.as_dict(), seed=3)
+    tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=3)
+    want = dstep.run_step(cfg, params, tokens)
+    n = want["replay"].n_grad
+    plan = ShardPlan(cfg.n_microbatches, world, n)
+    r = dstep.Replay(cfg, accum_len=plan.chunk, gout_len=plan.padded)
+    r.load_params(params)
+    tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).cuda()
+    r.calibrate(tok[0])
+    r.prepare_weights()
+    recv = [torch.empty((plan.M, plan.chunk), dtype=torch.float32, device="cuda") for _ in range(world)]
+    for rank in range(world):
+        for m in plan.local_microbatches(rank):
+            r.forward(tok[m])
+            r.backward()
+            for c in range(world):
+                lo, hi = plan.bounds(c)
+                recv[c][m, :hi - lo].copy_(r.gmb[lo:hi])
+    for c in range(world):
+        lo, hi = plan.bounds(c)
+        if hi > lo:
+            fold_slices(det, cfg.mesh, r.abufs, [recv[c][m, :hi - lo] for m in range(plan.M)],
+                        r.gout_padded[c * plan.chunk:c * plan.chunk + hi - lo])
+    r.optimizer()
+    got = r.hashes()
+    bad = [k for k, h in want["hashes"].items() if got[k] != h]
+    assert not bad, bad
+
+
+def test_sharded_replay_class_single_rank():
+    """ShardedReplay with one rank takes no collective and must reproduce the plain replay."""
+    import torch
+    from paper_2609_17380_b200 import step as dstep
+    from paper_2609_17380_b200.dist import ShardedReplay
+    kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=512, seq=128, micro_batch=1, mesh=(2, 1, 3))
+    cfg = dstep.ModelConfig(**kw)
+    params = synth.model_params(cfg.as_dict(), seed=5)
+    tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=5)
+    want = dstep.run_step(cfg, params, tokens)
+    rep = ShardedReplay(cfg, 0, 1)
+    rep.r.load_params(params)
+    tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).cuda()
+    rep.calibrate(tok[0])
+    got = rep.step(tok)
+    assert got["status"] == 0 and got["losses"] == want["losses"]
+    bad = [k for k, h in want["hashes"].items() if got["hashes"][k] != h]
+    assert not bad, bad
