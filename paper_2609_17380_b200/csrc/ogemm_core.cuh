@@ -123,13 +123,14 @@ __device__ __forceinline__ void slab_mac(const float (*As)[OT + 4], const float 
       b[2 * g] = make_float2(bv.x, bv.y);
       b[2 * g + 1] = make_float2(bv.z, bv.w);
     }
+    // column pairs outermost: each pair of B values meets the eight rows back to back (measured a few percent faster
+    // than rows outermost); the order in which different accumulators are visited has no effect on any result
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float2 a = make_float2(av[i], av[i]);
+    for (int j = 0; j < TN / 32; ++j) {
 #pragma unroll
-      for (int j = 0; j < TN / 32; ++j) {
+      for (int i = 0; i < 8; ++i) {
         if (FUSED) {
-          acc[i][j] = __ffma2_rn(a, b[j], acc[i][j]);
+          acc[i][j] = __ffma2_rn(make_float2(av[i], av[i]), b[j], acc[i][j]);
         } else {  // scalar on purpose: a packed multiply + add pair would be contracted by ptxas
           acc[i][j].x = fadd(acc[i][j].x, fmul(av[i], b[j].x));
           acc[i][j].y = fadd(acc[i][j].y, fmul(av[i], b[j].y));
