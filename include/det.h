@@ -163,7 +163,7 @@ int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, i
 int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S,
                  det_bf16* out, int ld_out, float* lse, void* stream);
 /* dq, dk, dv with leading dimension ld_d; every contraction is a sequential ascending sum from +0.
- * ws holds bf16(P) and bf16(dS), [B*H, S, S] each, and Delta [B*H, S]: see det_attn_bwd_ws_bytes. */
+ * ws holds P (f32) and bf16(dS), [B*H, S, S] each, and Delta [B*H, S]: see det_attn_bwd_ws_bytes. */
 size_t det_attn_bwd_ws_bytes(int B, int H, int S);
 int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,
                  const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq, det_bf16* dk,

@@ -258,96 +258,6 @@ __global__ void __launch_bounds__(256) k_attn_delta(const uint16_t* __restrict__
   if (lane == 0) delta[w] = t;
 }
 
-// S = q.k^T and dP = dO.v^T for one 128 x 128 tile of one (batch, head), both sequential over the 128 head
-// dimensions; then P = exp(S*scale - L), dS = P (dP - Delta) scale, and bf16(P), bf16(dS) go to global scratch
-// [b*H+h][query][key] for the three gradient contractions.  Tiles above the diagonal are skipped and never read.
-constexpr size_t SDP_SMEM = (size_t)4 * 2 * OK * (OT + 4) * sizeof(float);
-__global__ void __launch_bounds__(256, 1)
-    k_attn_sdp(const uint16_t* __restrict__ dout, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-               const uint16_t* __restrict__ v, const float* __restrict__ lse, const float* __restrict__ delta, int ld,
-               int ld_out, int H, int S, uint16_t* __restrict__ Pt, uint16_t* __restrict__ dSt) {
-  const int jt = blockIdx.x, it = blockIdx.y;
-  if (jt > it) return;
-  extern __shared__ __align__(16) unsigned char osm[];
-  typedef float(*Slab)[OK][OT + 4];
-  Slab Qs = reinterpret_cast<Slab>(osm);
-  Slab Os = reinterpret_cast<Slab>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
-  Slab Ks = reinterpret_cast<Slab>(osm + (size_t)4 * OK * (OT + 4) * sizeof(float));
-  Slab Vs = reinterpret_cast<Slab>(osm + (size_t)6 * OK * (OT + 4) * sizeof(float));
-  const int b = blockIdx.z / H, h = blockIdx.z % H;
-  const int i0 = it * OT, j0 = jt * OT;
-  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-  const size_t row0 = (size_t)b * S;
-  const uint16_t* qp = q + row0 * ld + (size_t)h * DH;
-  const uint16_t* kp = k + row0 * ld + (size_t)h * DH;
-  const uint16_t* vp = v + row0 * ld + (size_t)h * DH;
-  const uint16_t* op = dout + row0 * ld_out + (size_t)h * DH;
-  float2 sa[8][4], da[8][4];
-#pragma unroll
-  for (int a = 0; a < 8; ++a)
-#pragma unroll
-    for (int c = 0; c < 4; ++c) { sa[a][c] = make_float2(0.f, 0.f); da[a][c] = make_float2(0.f, 0.f); }
-  float vq[8], vo[8], vk[8], vv[8];
-  Raw8<false> rq[1], ro[1], rk[1], rv[1];
-  slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, 0, rq);
-  slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, 0, ro);
-  slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, 0, rk);
-  slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, 0, rv);
-  unpack8<false>(rq[0], vq); unpack8<false>(ro[0], vo); unpack8<false>(rk[0], vk); unpack8<false>(rv[0], vv);
-  slab_store<CONTIG, OT>(Qs[0], vq); slab_store<CONTIG, OT>(Os[0], vo);
-  slab_store<CONTIG, OT>(Ks[0], vk); slab_store<CONTIG, OT>(Vs[0], vv);
-  int tiny = __syncthreads_or(tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv));
-  constexpr int NS = DH / OK;
-  for (int s = 0; s < NS; ++s) {
-    const int cur = s & 1;
-    if (s + 1 < NS) {
-      slab_fetch<CONTIG, false, OT>(qp, S, DH, ld, i0, (s + 1) * OK, rq);
-      slab_fetch<CONTIG, false, OT>(op, S, DH, ld_out, i0, (s + 1) * OK, ro);
-      slab_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0, (s + 1) * OK, rk);
-      slab_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0, (s + 1) * OK, rv);
-    }
-    if (tiny) { slab_mac<false, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<false, OT>(Os[cur], Vs[cur], ty, tx, da); }
-    else { slab_mac<true, OT>(Qs[cur], Ks[cur], ty, tx, sa); slab_mac<true, OT>(Os[cur], Vs[cur], ty, tx, da); }
-    bool nt = false;
-    if (s + 1 < NS) {
-      unpack8<false>(rq[0], vq); unpack8<false>(ro[0], vo); unpack8<false>(rk[0], vk); unpack8<false>(rv[0], vv);
-      slab_store<CONTIG, OT>(Qs[cur ^ 1], vq); slab_store<CONTIG, OT>(Os[cur ^ 1], vo);
-      slab_store<CONTIG, OT>(Ks[cur ^ 1], vk); slab_store<CONTIG, OT>(Vs[cur ^ 1], vv);
-      nt = tiny_any<8>(vq) || tiny_any<8>(vo) || tiny_any<8>(vk) || tiny_any<8>(vv);
-    }
-    tiny = __syncthreads_or(nt);
-  }
-  const size_t bh = (size_t)blockIdx.z;
-#pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    const int i = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
-    if (i >= S) continue;
-    const float L = lse[bh * S + i], dl = delta[bh * S + i];
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      const int jb = j0 + g * 64 + tx * 4;
-      if (jb >= S) continue;
-      const float sv[4] = {sa[a][2 * g].x, sa[a][2 * g].y, sa[a][2 * g + 1].x, sa[a][2 * g + 1].y};
-      const float dv4[4] = {da[a][2 * g].x, da[a][2 * g].y, da[a][2 * g + 1].x, da[a][2 * g + 1].y};
-      float pv[4], dsv[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        pv[e] = 0.0f; dsv[e] = 0.0f;
-        if (jb + e <= i) {
-          pv[e] = det_exp(fsub(fmul(sv[e], ATT_SCALE), L));
-          dsv[e] = fmul(fmul(pv[e], fsub(dv4[e], dl)), ATT_SCALE);
-        }
-      }
-      const size_t off = (bh * S + i) * S + jb;
-      uint2 u;
-      u.x = pack_bf2(pv[0], pv[1]); u.y = pack_bf2(pv[2], pv[3]);
-      *reinterpret_cast<uint2*>(Pt + off) = u;
-      u.x = pack_bf2(dsv[0], dsv[1]); u.y = pack_bf2(dsv[2], dsv[3]);
-      *reinterpret_cast<uint2*>(dSt + off) = u;
-    }
-  }
-}
-
 static int set_smem(const void* fn, size_t bytes) {
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? 0 : -1;
 }
@@ -369,8 +279,10 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   return DET_OK;
 }
 
+// workspace: P f32 [B*H, S, S], dS bf16 [B*H, S, S], Delta f32 [B*H, S]
 extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int S) {
-  return 2 * align_up((size_t)B * H * S * S * 2, 256) + align_up((size_t)B * H * S * 4, 256);
+  return align_up((size_t)B * H * S * S * 4, 256) + align_up((size_t)B * H * S * S * 2, 256) +
+         align_up((size_t)B * H * S * 4, 256);
 }
 
 extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
@@ -382,29 +294,36 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
       !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
     return DET_ERR_ALIGN;
   if (!ws || ws_bytes < det_attn_bwd_ws_bytes(B, H, S)) return DET_ERR_WORKSPACE;
-  static bool cfg = false;
-  if (!cfg) {
-    if (set_smem((const void*)k_attn_sdp, SDP_SMEM)) return DET_ERR_CUDA;
-    cfg = true;
-  }
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t mat = align_up((size_t)B * H * S * S * 2, 256);
-  uint16_t* Pt = (uint16_t*)ws;
-  uint16_t* dSt = (uint16_t*)((uint8_t*)ws + mat);
-  float* delta = (float*)((uint8_t*)ws + 2 * mat);
+  const size_t matP = align_up((size_t)B * H * S * S * 4, 256), matS = align_up((size_t)B * H * S * S * 2, 256);
+  float* Pf = (float*)ws;
+  uint16_t* dSt = (uint16_t*)((uint8_t*)ws + matP);
+  float* delta = (float*)((uint8_t*)ws + matP + matS);
   const size_t nrows = (size_t)B * H * S;
   k_attn_delta<<<DET_L((unsigned)((nrows + 7) / 8)), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
-  const int nt = (S + OT - 1) / OT;
-  dim3 grid(nt, nt, B * H);
-  k_attn_sdp<<<DET_L(grid), 256, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, S, Pt, dSt);
   DET_CHECK_LAUNCH();
+  // P[i,j] = exp(scale * sum_d q[i,d] k[j,d] - L_i) for j <= i (f32; tiles above the diagonal are never touched), then
+  // dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both contractions ascend over the 128 dims
+  OgemmArgs e = {};
+  e.I = S; e.J = S; e.C = DH; e.H = H; e.range_mode = 3; e.scale = ATT_SCALE;
+  e.ldo = S; e.o_b = (long long)H * S * S; e.o_h = (long long)S * S;
+  e.A = q; e.lda = ld; e.a_b = (long long)S * ld; e.a_h = DH;
+  e.B = k; e.ldb = ld; e.b_b = (long long)S * ld; e.b_h = DH;
+  e.out = Pf; e.rowv = lse;
+  int rc = ogemm_launch<CONTIG, CONTIG, false, false, 128, OEPI_P>(e, B * H, st);
+  if (rc != DET_OK) return rc;
+  e.A = dout; e.lda = ld_out; e.a_b = (long long)S * ld_out;
+  e.B = v;
+  e.out = dSt; e.rowv = delta; e.Pin = Pf;
+  rc = ogemm_launch<CONTIG, CONTIG, false, true, 128, OEPI_DS>(e, B * H, st);
+  if (rc != DET_OK) return rc;
   // dV[j,c] = sum over queries i >= j ascending of P~[i,j] dO[i,c];  dK[j,c] likewise with dS~ and q
   OgemmArgs p = {};
   p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
   p.range_mode = 1;
-  p.A = Pt; p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; p.b_h = DH;
+  p.A = Pf; p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; p.b_h = DH;
   p.out = dv; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
-  int rc = ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * H, st);
+  rc = ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * H, st);   // P is rounded to bf16 as it is read
   if (rc != DET_OK) return rc;
   p.A = dSt; p.B = q; p.ldb = ld; p.b_b = (long long)S * ld; p.out = dk;
   rc = ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * H, st);

@@ -150,17 +150,27 @@ struct OgemmArgs {
   int init;             // f32 output only: start from the values already in out
   int H;                // batching: blockIdx.z = b * H + h
   long long a_b, a_h, b_b, b_h, o_b, o_h;  // element offsets per batch index / head index
-  int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
+  int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile;
+                        // 3: whole contraction, but tiles entirely above the diagonal (j0 > i0) are skipped
+  // epilogues of the attention backward (EPI 1, 2); rowv and Pin are batched like the output
+  const float* rowv;    // one value per row i of each batch: the logsumexp L (EPI 1) or Delta (EPI 2)
+  const float* Pin;     // EPI 2: the f32 weights written by EPI 1, same layout as the output
+  float scale;          // softmax scale
 };
 
+// Output transforms.  OEPI_NONE: the accumulator.  OEPI_P: P[i,j] = exp(acc*scale - L_i) for j <= i, else +0 (f32 out).
+// OEPI_DS: dS[i,j] = (P[i,j] * (acc - Delta_i)) * scale (bf16 out; P = 0 above the diagonal makes dS = 0 there).
+enum { OEPI_NONE = 0, OEPI_P = 1, OEPI_DS = 2 };
+
 // CTA tile 128 x TN; thread (ty, tx) owns rows {ty*4.., 64+ty*4..} and columns {g*64 + tx*4..}, g < TN/64.
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN, int EPI = OEPI_NONE>
 __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
   float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
   // blocks are handed out in linear order; with a causal range the longest contractions are put first
   const int i0 = (p.range_mode == 2 ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y) * OT, j0 = blockIdx.x * TN;
+  if (p.range_mode == 3 && j0 > i0) return;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
   const long long zb = blockIdx.z / p.H, zh = blockIdx.z % p.H;
   const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + zh * p.a_h)
@@ -224,35 +234,47 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
     const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+    float rv = 0.0f;
+    if (EPI != OEPI_NONE && r < I) rv = p.rowv[(size_t)blockIdx.z * I + r];
 #pragma unroll
     for (int g = 0; g < TN / 64; ++g) {
       const int c = j0 + g * 64 + tx * 4;
       if (r < I && c < J) {
-        const float2 lo = acc[a][2 * g], hi = acc[a][2 * g + 1];
+        float w[4] = {acc[a][2 * g].x, acc[a][2 * g].y, acc[a][2 * g + 1].x, acc[a][2 * g + 1].y};
+        if (EPI == OEPI_P) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) w[e] = (c + e <= r) ? det_exp(fsub(fmul(w[e], p.scale), rv)) : 0.0f;
+        }
+        if (EPI == OEPI_DS) {
+          const float4 pw = *reinterpret_cast<const float4*>(p.Pin + zb * p.o_b + zh * p.o_h + (size_t)r * ldo + c);
+          const float pv[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) w[e] = fmul(fmul(pv[e], fsub(w[e], rv)), p.scale);
+        }
         if (OUT_BF16) {
           uint2 u;
-          u.x = pack_bf2(lo.x, lo.y);
-          u.y = pack_bf2(hi.x, hi.y);
+          u.x = pack_bf2(w[0], w[1]);
+          u.y = pack_bf2(w[2], w[3]);
           *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(out) + (size_t)r * ldo + c) = u;
         } else {
-          *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ldo + c) = make_float4(lo.x, lo.y, hi.x, hi.y);
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ldo + c) = make_float4(w[0], w[1], w[2], w[3]);
         }
       }
     }
   }
 }
 
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN, int EPI = OEPI_NONE>
 static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   static bool cfg = false;
   if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)ogemm_smem<TN>()) != cudaSuccess)
       return DET_ERR_CUDA;
     cfg = true;
   }
   dim3 grid((p.J + TN - 1) / TN, (p.I + OT - 1) / OT, batches);
-  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
+  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN, EPI><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
   return DET_OK;
 }
 
