@@ -5,9 +5,9 @@
 // ascending sum over the 128 head dimensions of exact bf16 products; the tile's row sum is the adjacent
 // pairwise tree over its 128 slots (masked slots are +0); P is rounded to bf16 before P.V; P.V is a
 // sequential ascending sum over the tile's keys from +0, then o = o*alpha + u.
-// Backward: P = exp(S - L) recomputed; dV, dK (per key) and dQ (per query) are single accumulators fed in
-// ascending order of the contraction index; bf16(dS) goes through global scratch from the dK/dV kernel to
-// the dQ kernel, so nothing is accumulated with atomics.
+// Backward: P = exp(S*scale - L) recomputed; every one of the five contractions (S, dP, dV, dK, dQ) is a batched
+// ordered contraction with one sequential accumulator per output (ogemm_core.cuh); P (f32) and bf16(dS) go through
+// global scratch, so nothing is accumulated with atomics.
 #include "ogemm_core.cuh"
 
 namespace det {
