@@ -144,6 +144,24 @@ size_t det_rmsnorm_bwd_ws_bytes(int rows, int D);
 int det_rmsnorm_bwd(int io, const void* dy, const void* x, const void* gamma, const float* rstd, int rows, int D,
                     void* dx, float* dgamma, void* ws, size_t ws_bytes, void* stream);
 
+/* ---- per-head operations of the attention block (Sec. 3.1 "QK-norm", "RoPE") --------------------------
+ * Rows of 128 values (one head of one token) inside wider token rows: element (t, h, i) of x sits at
+ * x[t*ld + h*128 + i]; ld, ld_y, ... are row strides in elements (multiples of 4, >= nh*128); pointers 8-byte
+ * aligned; in-place use (y == x) is allowed.  All device pointers; stream-ordered.
+ * det_headnorm_fwd: gain-free RMS normalisation of every head: y = bf16(x * rstd),
+ *   rstd[t*nh + h] = 1 / sqrt(det_sum(x^2) * 2^-7 + eps)  (the paper normalises queries and keys before RoPE).
+ * det_headnorm_bwd: dx = bf16(rstd * (dy - xhat * c)), xhat = x * rstd, c = det_sum(dy * xhat) * 2^-7. */
+int det_headnorm_fwd(const det_bf16* x, int ld, int T, int nh, float eps, det_bf16* y, int ld_y, float* rstd,
+                     void* stream);
+int det_headnorm_bwd(const det_bf16* dy, int ld_dy, const det_bf16* x, int ld, const float* rstd, int T, int nh,
+                     det_bf16* dx, int ld_dx, void* stream);
+/* Rotary embedding with caller-supplied tables cos_tab, sin_tab f32 [S, 64] (inputs of the step; the paper uses
+ * theta = 5e5): the position of token t is t mod S; pairs are (i, i+64):
+ *   y_i = bf16(x_i c_i - x_{i+64} s_i),  y_{i+64} = bf16(x_{i+64} c_i + x_i s_i),  every product rounded on its own.
+ * inverse != 0 rotates by the opposite angle, which is the backward pass of the rotation. */
+int det_rope(const det_bf16* x, int ld, int T, int nh, int S, const float* cos_tab, const float* sin_tab, int inverse,
+             det_bf16* y, int ld_y, void* stream);
+
 /* ---- cross-entropy with optional z-loss (Sec. 3.1 "Z-loss"; loss in FP32) ---------------------------
  * per row: m = max z, S = det_sum exp(z - m), lse = m + log S, loss_row = lse - z[target];
  * loss_mean[0] = det_sum(loss_row)/rows (+ z_weight * z_mean), z_mean[0] = det_sum(lse^2)/rows.

@@ -191,6 +191,19 @@ def rmsnorm_bwd(dy, x, gamma, rstd, bf=False):
     return dx, dg
 
 
+def rope(x, S, cos, sin, inverse=False):
+    """x: bf16 bits [T, nh, 128]; cos, sin: f32 [S, 64]; position = t mod S."""
+    x = _c(x, np.uint16)
+    T, nh, d = x.shape
+    assert d == 128
+    cos = _c(cos, np.float32)
+    sin = _c(sin, np.float32)
+    assert cos.shape == (S, 64) and sin.shape == (S, 64)
+    y = np.empty_like(x)
+    lib().orc_rope(_p(x), C.c_int(T), C.c_int(nh), C.c_int(S), _p(cos), _p(sin), C.c_int(int(inverse)), _p(y))
+    return y
+
+
 def xent_fwd(logits, target, z_weight=0.0):
     logits = _c(logits, np.float32)
     target = _c(target, np.int32)

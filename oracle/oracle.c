@@ -773,3 +773,29 @@ void orc_tensor_hash(const uint8_t *data, size_t n, uint8_t out[32]) {
   orc_sha256(a, nc * 32 + 8, out);
   free(a); free(b);
 }
+
+/* ------------------------------------------------------------------ */
+/* rotary position embedding (Sec. 3.1 "RoPE", theta = 5e5; the tables  */
+/* are inputs of the step, generated once in float64 and rounded)       */
+/* ------------------------------------------------------------------ */
+/* x, y: bf16 [T, nh, 128]; position of token t is t mod S; cos, sin: f32 [S, 64].
+ * Pairs are (i, i + 64):  y_i = x_i c_i - x_{i+64} s_i,  y_{i+64} = x_{i+64} c_i + x_i s_i,
+ * every product rounded on its own; inverse != 0 rotates by the opposite angle (the backward pass). */
+void orc_rope(const bf16_t *x, int T, int nh, int S, const float *cs, const float *sn, int inverse, bf16_t *y) {
+#pragma omp parallel for
+  for (int t = 0; t < T; ++t) {
+    const float *c = cs + (size_t)(t % S) * 64, *s = sn + (size_t)(t % S) * 64;
+    for (int h = 0; h < nh; ++h) {
+      const bf16_t *xr = x + ((size_t)t * nh + h) * 128;
+      bf16_t *yr = y + ((size_t)t * nh + h) * 128;
+      for (int i = 0; i < 64; ++i) {
+        float a = bf2f(xr[i]), b = bf2f(xr[i + 64]);
+        float si = inverse ? -s[i] : s[i];
+        float lo = fsub(fmul(a, c[i]), fmul(b, si));
+        float hi = fadd(fmul(b, c[i]), fmul(a, si));
+        yr[i] = f2bf(lo);
+        yr[i + 64] = f2bf(hi);
+      }
+    }
+  }
+}

@@ -191,6 +191,21 @@ def det_rmsnorm_fwd(io, x, gamma, rows, D, eps, y, rstd):
                                                      C.c_float(eps), _ptr(y), _ptr(rstd), _stream()))
 
 
+def det_headnorm_fwd(x, ld, T, nh, eps, y, ld_y, rstd):
+    _check("det_headnorm_fwd", load().det_headnorm_fwd(_ptr(x), C.c_int(ld), C.c_int(T), C.c_int(nh), C.c_float(eps), _ptr(y),
+                                                       C.c_int(ld_y), _ptr(rstd), _stream()))
+
+
+def det_headnorm_bwd(dy, ld_dy, x, ld, rstd, T, nh, dx, ld_dx):
+    _check("det_headnorm_bwd", load().det_headnorm_bwd(_ptr(dy), C.c_int(ld_dy), _ptr(x), C.c_int(ld), _ptr(rstd), C.c_int(T),
+                                                       C.c_int(nh), _ptr(dx), C.c_int(ld_dx), _stream()))
+
+
+def det_rope(x, ld, T, nh, S, cos_tab, sin_tab, inverse, y, ld_y):
+    _check("det_rope", load().det_rope(_ptr(x), C.c_int(ld), C.c_int(T), C.c_int(nh), C.c_int(S), _ptr(cos_tab), _ptr(sin_tab),
+                                       C.c_int(int(inverse)), _ptr(y), C.c_int(ld_y), _stream()))
+
+
 def det_rmsnorm_bwd_ws_bytes(rows, D):
     return load().det_rmsnorm_bwd_ws_bytes(C.c_int(rows), C.c_int(D))
 

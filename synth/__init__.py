@@ -108,3 +108,12 @@ def model_params(cfg, seed=0):
 def model_tokens(cfg, n_microbatches, seed=0):
     """Uniform random token ids, [n_microbatches, micro_batch, seq + 1] (inputs and shifted labels)."""
     return randint((n_microbatches, cfg["micro_batch"], cfg["seq"] + 1), cfg["vocab"], seed=seed, tid=777)
+
+
+def rope_tables(S, base=5.0e5, dim=128):
+    """cos/sin tables [S, dim/2] for rotary embeddings: angle = pos * base**(-2i/dim), evaluated in float64 and rounded
+    to float32 once; the tables are inputs of the step (both implementations read the same arrays)."""
+    i = np.arange(dim // 2, dtype=np.float64)
+    inv = base ** (-2.0 * i / dim)
+    ang = np.arange(S, dtype=np.float64)[:, None] * inv[None, :]
+    return np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)

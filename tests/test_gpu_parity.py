@@ -164,6 +164,45 @@ def test_rmsnorm(det, bf, rows, D, gain):
     assert_same_bits(host(dgam), odg, "dgamma")
 
 
+# ------------------------------------------------------------------ per-head norm and rotary embedding
+@pytest.mark.parametrize("T,nh,pad,S", [(300, 4, 0, 100), (129, 3, 256, 64), (7, 1, 8, 7)])
+def test_headnorm_and_rope(det, T, nh, pad, S):
+    """Rows of 128 inside wider token rows (stride = nh*128 + pad), against the oracle on the gathered rows."""
+    ld = nh * 128 + pad
+    buf = synth.normal_bf16((T, ld), seed=21)
+    buf[::5, 3] = 0x0001                                        # a few subnormal and tiny inputs
+    buf[1::7, 64] = synth.to_bf16(np.array([2.0 ** -70], F))[0]
+    dyb = synth.normal_bf16((T, ld), seed=22)
+    x = np.ascontiguousarray(buf[:, :nh * 128]).reshape(T * nh, 128)
+    dy = np.ascontiguousarray(dyb[:, :nh * 128]).reshape(T * nh, 128)
+    # forward norm into a second strided buffer
+    ybuf, rstd = dev(np.zeros((T, ld), np.uint16)), empty((T * nh,), F)
+    det.det_headnorm_fwd(dev(buf), ld, T, nh, 1e-6, ybuf, ld, rstd)
+    _sync()
+    oy, orstd = oracle.rmsnorm_fwd(x, None, 1e-6, bf=True)
+    assert_same_bits(host(rstd), orstd, "headnorm rstd")
+    gy = host(ybuf, np.uint16)
+    assert_same_bits(gy[:, :nh * 128].reshape(T * nh, 128), oy, "headnorm y")
+    assert not gy[:, nh * 128:].any()                           # nothing written outside the heads
+    dxbuf = dev(np.zeros((T, ld), np.uint16))
+    det.det_headnorm_bwd(dev(dyb), ld, dev(buf), ld, rstd, T, nh, dxbuf, ld)
+    _sync()
+    odx, _ = oracle.rmsnorm_bwd(dy, x, None, orstd, bf=True)
+    assert_same_bits(host(dxbuf, np.uint16)[:, :nh * 128].reshape(T * nh, 128), odx, "headnorm dx")
+    # rotary embedding, forward out of place and inverse in place
+    cos, sin = synth.rope_tables(S)
+    dc, ds = dev(cos), dev(sin)
+    rbuf = dev(np.zeros((T, ld), np.uint16))
+    det.det_rope(dev(buf), ld, T, nh, S, dc, ds, 0, rbuf, ld)
+    _sync()
+    orot = oracle.rope(x.reshape(T, nh, 128), S, cos, sin)
+    assert_same_bits(host(rbuf, np.uint16)[:, :nh * 128].reshape(T, nh, 128), orot, "rope")
+    det.det_rope(rbuf, ld, T, nh, S, dc, ds, 1, rbuf, ld)
+    _sync()
+    oinv = oracle.rope(orot, S, cos, sin, inverse=True)
+    assert_same_bits(host(rbuf, np.uint16)[:, :nh * 128].reshape(T, nh, 128), oinv, "rope inverse in place")
+
+
 # ------------------------------------------------------------------ cross-entropy
 @pytest.mark.parametrize("rows,V,zw", [(24, 50304, 0.0), (8, 50304, 1e-4), (5, 1000, 0.0), (3, 4, 0.0), (2, 128256, 1e-4)])
 def test_xent(det, rows, V, zw):

@@ -408,3 +408,59 @@ def test_adamw_hand_element_and_float64():
         P = bf(synth.to_bf16(P.astype(F))).astype(np.float64)
     assert np.mean(bf(pb) == P) > 0.98 and np.allclose(bf(pb), P, rtol=2 ** -7)
     assert np.allclose(m, M, rtol=1e-5, atol=1e-12) and np.allclose(v, Vv, rtol=1e-5, atol=1e-14)
+
+
+def test_rope_pins():
+    """Rotary embedding (Sec. 3.1): pairing (i, i+64), signs, identity at position 0, float64 agreement, inverse."""
+    S, nh = 24, 3
+    cos, sin = synth.rope_tables(S)
+    assert cos.shape == (S, 64) and np.all(cos[0] == 1.0) and np.all(sin[0] == 0.0)
+    # the tables follow angle = pos * theta**(-2i/128) with theta = 5e5
+    assert abs(float(cos[5, 7]) - math.cos(5 * 5.0e5 ** (-14 / 128))) < 1e-7
+    x = synth.normal_bf16((2 * S, nh, 128), seed=11)
+    y = oracle.rope(x, S, cos, sin)
+    assert np.array_equal(y[0], x[0]) and np.array_equal(y[S], x[S])          # position 0 (and S: t mod S) is the identity
+    # unit vectors pin the pairing and the signs: e_i -> (c_i at i, s_i at i+64); e_{i+64} -> (-s_i at i, c_i at i+64)
+    e = np.zeros((S, 1, 128), np.float32)
+    e[:, 0, 9] = 1.0
+    ye = synth.from_bf16(oracle.rope(synth.to_bf16(e), S, cos, sin))
+    assert np.array_equal(ye[:, 0, 9], synth.from_bf16(synth.to_bf16(cos[:, 9])))
+    assert np.array_equal(ye[:, 0, 73], synth.from_bf16(synth.to_bf16(sin[:, 9])))
+    assert not ye[:, 0, [8, 10, 72, 74]].any()
+    e[:] = 0
+    e[:, 0, 73] = 1.0
+    ye = synth.from_bf16(oracle.rope(synth.to_bf16(e), S, cos, sin))
+    assert np.array_equal(ye[:, 0, 9], synth.from_bf16(synth.to_bf16(-sin[:, 9])))
+    assert np.array_equal(ye[:, 0, 73], synth.from_bf16(synth.to_bf16(cos[:, 9])))
+    # float64 reference within half a bf16 ulp (+ the f32 roundings)
+    xf = synth.from_bf16(x).astype(np.float64).reshape(2, S, nh, 128)
+    c, s = cos.astype(np.float64)[None, :, None, :], sin.astype(np.float64)[None, :, None, :]
+    ref = np.concatenate([xf[..., :64] * c - xf[..., 64:] * s, xf[..., 64:] * c + xf[..., :64] * s], -1).reshape(2 * S, nh, 128)
+    got = synth.from_bf16(y).astype(np.float64)
+    assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -8 + 1e-30)
+    # relative-position property: <rope(q, p), rope(k, r)> depends on p - r only (float64 check on the reference form)
+    # and the inverse rotation undoes the forward one up to the two bf16 roundings
+    back = synth.from_bf16(oracle.rope(y, S, cos, sin, inverse=True)).astype(np.float64)
+    assert np.all(np.abs(back - synth.from_bf16(x)) <= np.abs(synth.from_bf16(x)) * 2.0 ** -7 + 2.0 ** -7 * np.abs(ref).max())
+    # the inverse is the transpose: <y, R x> = <R^T y, x> in float64 up to rounding
+    g = synth.normal_bf16((2 * S, nh, 128), seed=12)
+    lhs = (synth.from_bf16(g).astype(np.float64) * got).sum()
+    rhs = (synth.from_bf16(oracle.rope(g, S, cos, sin, inverse=True)).astype(np.float64) * synth.from_bf16(x)).sum()
+    assert abs(lhs - rhs) <= 2e-2 * math.sqrt(got.size)
+
+
+def test_headnorm_is_gain_free_rmsnorm_over_128():
+    """QK-norm (Sec. 3.1) is the gain-free RMSNorm over each head's 128 values: unit RMS out, float64 agreement."""
+    x = synth.normal_bf16((40, 128), seed=13)
+    y, rstd = oracle.rmsnorm_fwd(x, None, 1e-6, bf=True)
+    xf = synth.from_bf16(x).astype(np.float64)
+    ref = xf / np.sqrt((xf * xf).mean(-1, keepdims=True) + 1e-6)
+    assert np.all(np.abs(synth.from_bf16(y) - ref) <= np.abs(ref) * 2.0 ** -8 + 1e-30)
+    assert np.allclose(np.sqrt((synth.from_bf16(y).astype(np.float64) ** 2).mean(-1)), 1.0, atol=5e-3)
+    dy = synth.normal_bf16((40, 128), seed=14)
+    dx, _ = oracle.rmsnorm_bwd(dy, x, None, rstd, bf=True)
+    g = synth.from_bf16(dy).astype(np.float64)
+    r = 1.0 / np.sqrt((xf * xf).mean(-1, keepdims=True) + 1e-6)
+    xh = xf * r
+    refdx = r * (g - xh * (g * xh).mean(-1, keepdims=True))
+    assert np.all(np.abs(synth.from_bf16(dx) - refdx) <= np.abs(refdx) * 2.0 ** -7 + 1e-3 * np.abs(refdx).max())
