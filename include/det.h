@@ -174,18 +174,23 @@ int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, i
                  float scale, void* stream);
 
 /* ---- causal attention, head_dim 128 (Sec. 3.2: QK^T and softmax in higher precision; BF16 flash
- *      backward that recomputes the weights) ----------------------------------------------------------
- * q, k, v: bf16, row (b*S + i) of head h starts at element ld*(b*S+i) + h*128.  Online softmax over KV
- * tiles of 128 keys in ascending order; dot products are sequential over the 128 dimensions; tile row sums
- * are adjacent trees over the 128 slots; P is rounded to bf16 before P.V.  lse f32 [B,H,S]. */
-int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S,
-                 det_bf16* out, int ld_out, float* lse, void* stream);
-/* dq, dk, dv with leading dimension ld_d; every contraction is a sequential ascending sum from +0.
- * ws holds P (f32) and bf16(dS), [B*H, S, S] each, and Delta [B*H, S]: see det_attn_bwd_ws_bytes. */
-size_t det_attn_bwd_ws_bytes(int B, int H, int S);
+ *      backward that recomputes the weights; Sec. 3.1: grouped queries, sliding windows) -------------------
+ * q, k, v: bf16, row (b*S + i) of head h starts at element ld*(b*S+i) + h*128.  H query heads share Hkv
+ * key/value heads (H % Hkv == 0; query head h reads key/value head h / (H/Hkv); Hkv == H is multi-head
+ * attention).  window == 0: row i sees the keys j <= i; window = W > 0 (multiple of 128): the keys j in (i - W, i].
+ * Online softmax over KV tiles of 128 keys in ascending order (a row visits the tiles that hold one of its keys);
+ * dot products are sequential over the 128 dimensions; tile row sums are adjacent trees over the 128 slots; P is
+ * rounded to bf16 before P.V.  lse f32 [B,H,S].  S % 64 == 0. */
+int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                 int window, det_bf16* out, int ld_out, float* lse, void* stream);
+/* dq (H heads), dk, dv (Hkv heads) with leading dimension ld_d; every contraction is one sequential ascending sum
+ * from +0; the gradient of a shared key/value head runs over its query heads in ascending order and, within a
+ * head, over the queries in ascending order.  ws (16-byte aligned, det_attn_bwd_ws_bytes) holds P (f32) and
+ * bf16(dS), [B*H, S, S] each, Delta [B*H, S], and for Hkv < H the f32 accumulators carried between query heads. */
+size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S);
 int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,
-                 const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq, det_bf16* dk,
-                 det_bf16* dv, int ld_d, void* ws, size_t ws_bytes, void* stream);
+                 const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S, int window, det_bf16* dq,
+                 det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes, void* stream);
 
 /* ---- elementwise glue (Sec. 3.1: SwiGLU with fused gate/up projection, pre-norm residuals, embedding) */
 /* gu bf16 [rows, 2F] (gate | up), h bf16 [rows, F] = silu(gate) * up;  F % 8 == 0 */

@@ -228,32 +228,36 @@ def xent_bwd(logits, target, lse, z_weight=0.0, scale=1.0):
 
 
 # ---- attention ------------------------------------------------------------
-def attn_fwd(qkv, B, H, S):
-    """qkv: uint16 [B*S, 3*H*128] (q | k | v column blocks).  Returns out [B*S, H*128], lse [B,H,S]."""
+def attn_fwd(qkv, B, H, S, Hkv=None, window=0):
+    """qkv: uint16 [B*S, (H + 2*Hkv)*128] (q | k | v column blocks).  Returns out [B*S, H*128], lse [B,H,S].
+    Hkv < H: grouped-query attention; window > 0: sliding-window attention over the last `window` keys."""
     qkv = _c(qkv, np.uint16)
+    Hkv = H if Hkv is None else Hkv
     ld = qkv.shape[1]
-    HD = H * 128
+    assert ld == (H + 2 * Hkv) * 128 and H % Hkv == 0
+    HD, KD = H * 128, Hkv * 128
     out = np.empty((B * S, HD), np.uint16)
     lse = np.empty((B, H, S), np.float32)
     base = qkv.ctypes.data
-    lib().orc_attn_fwd(C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 4 * HD), C.c_int(ld), C.c_int(B),
-                       C.c_int(H), C.c_int(S), _p(out), C.c_int(HD), _p(lse))
+    lib().orc_attn_fwd(C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), C.c_int(ld), C.c_int(B),
+                       C.c_int(H), C.c_int(Hkv), C.c_int(S), C.c_int(window), _p(out), C.c_int(HD), _p(lse))
     return out, lse
 
 
-def attn_bwd(dout, qkv, out, lse, B, H, S):
+def attn_bwd(dout, qkv, out, lse, B, H, S, Hkv=None, window=0):
     dout = _c(dout, np.uint16)
     qkv = _c(qkv, np.uint16)
     out = _c(out, np.uint16)
     lse = _c(lse, np.float32)
+    Hkv = H if Hkv is None else Hkv
     ld = qkv.shape[1]
-    HD = H * 128
+    HD, KD = H * 128, Hkv * 128
     dqkv = np.empty_like(qkv)
     base = qkv.ctypes.data
     dbase = dqkv.ctypes.data
-    lib().orc_attn_bwd(_p(dout), C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 4 * HD), _p(out), _p(lse),
-                       C.c_int(ld), C.c_int(HD), C.c_int(B), C.c_int(H), C.c_int(S), C.c_void_p(dbase),
-                       C.c_void_p(dbase + 2 * HD), C.c_void_p(dbase + 4 * HD), C.c_int(ld))
+    lib().orc_attn_bwd(_p(dout), C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), _p(out), _p(lse),
+                       C.c_int(ld), C.c_int(HD), C.c_int(B), C.c_int(H), C.c_int(Hkv), C.c_int(S), C.c_int(window),
+                       C.c_void_p(dbase), C.c_void_p(dbase + 2 * HD), C.c_void_p(dbase + 2 * (HD + KD)), C.c_int(ld))
     return dqkv
 
 

@@ -404,27 +404,35 @@ static float tree128(float *v) { /* perfect adjacent tree, in place */
 }
 
 /* q,k,v: row (b*S+i) at element offset ld*(b*S+i) + h*128; out likewise with ld_out; lse [B,H,S] */
-void orc_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, int B, int H, int S, bf16_t *out,
-                  int ld_out, float *lse) {
+/* Hkv: number of key/value heads (grouped-query attention, Sec. 3.1: query head h reads key/value head
+ * h / (H/Hkv)); Hkv == H is ordinary multi-head attention.  W: sliding window (Sec. 3.1: local layers see the
+ * last W keys, j in (i - W, i]); W == 0 is full causal attention.  A row visits only the key tiles that hold at
+ * least one visible key, in ascending order. */
+static inline int visible(int i, int j, int W) { return j <= i && (W == 0 || j > i - W); }
+static inline int first_tile(int i, int W) { int lo = (W == 0 || i - W + 1 < 0) ? 0 : i - W + 1; return lo / KT * KT; }
+
+void orc_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, int B, int H, int Hkv, int S, int W,
+                  bf16_t *out, int ld_out, float *lse) {
+  const int G = H / Hkv;
 #pragma omp parallel for collapse(2) schedule(dynamic, 8)
   for (int bh = 0; bh < B * H; ++bh)
     for (int i = 0; i < S; ++i) {
-      int b = bh / H, h = bh % H;
+      int b = bh / H, h = bh % H, hk = h / G;
       const bf16_t *qi = q + (size_t)ldq * (b * S + i) + h * DH;
       float m = -INFINITY, l = 0.0f, o[DH], s[KT], p[KT], pt[KT];
       for (int c = 0; c < DH; ++c) o[c] = 0.0f;
-      for (int j0 = 0; j0 <= i; j0 += KT) {
+      for (int j0 = first_tile(i, W); j0 <= i; j0 += KT) {
         float mt = m;
         for (int jj = 0; jj < KT; ++jj) {
           int j = j0 + jj;
-          if (j <= i) {
-            s[jj] = fmul(dot128(qi, k + (size_t)ldq * (b * S + j) + h * DH), ATT_SCALE);
+          if (visible(i, j, W)) {
+            s[jj] = fmul(dot128(qi, k + (size_t)ldq * (b * S + j) + hk * DH), ATT_SCALE);
             mt = fmax2(mt, s[jj]);
           }
         }
         float alpha = det_exp(fsub(m, mt));
         for (int jj = 0; jj < KT; ++jj) {
-          p[jj] = (j0 + jj <= i) ? det_exp(fsub(s[jj], mt)) : 0.0f;
+          p[jj] = visible(i, j0 + jj, W) ? det_exp(fsub(s[jj], mt)) : 0.0f;
           pt[jj] = bf2f(f2bf(p[jj]));
         }
         float r = tree128(p);
@@ -432,7 +440,7 @@ void orc_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, in
         for (int c = 0; c < DH; ++c) {
           float u = 0.0f;
           for (int jj = 0; jj < KT && j0 + jj <= i; ++jj)
-            u = fadd(u, fmul(pt[jj], bf2f(v[(size_t)ldq * (b * S + j0 + jj) + h * DH + c])));
+            u = fadd(u, fmul(pt[jj], bf2f(v[(size_t)ldq * (b * S + j0 + jj) + hk * DH + c])));
           o[c] = fadd(fmul(o[c], alpha), u);
         }
         m = mt;
@@ -445,50 +453,67 @@ void orc_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, in
 
 /* backward: p_ij = exp(s_ij - L_i); Delta_i = tree_c(dO*O); dP = dO.v_j;
  * dS = p (dP - Delta) scale; contraction operands rounded to bf16; all three
- * gradient contractions are sequential ascending sums from +0. */
+ * gradient contractions are sequential ascending sums from +0.  With grouped
+ * queries the gradient of a shared key/value head is ONE sequential accumulator
+ * over its query heads in ascending order and, within a head, over the queries
+ * in ascending order. */
 void orc_attn_bwd(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf16_t *v, const bf16_t *out,
-                  const float *lse, int ldq, int ld_out, int B, int H, int S, bf16_t *dq, bf16_t *dk, bf16_t *dv,
-                  int ld_d) {
+                  const float *lse, int ldq, int ld_out, int B, int H, int Hkv, int S, int W, bf16_t *dq, bf16_t *dk,
+                  bf16_t *dv, int ld_d) {
+  const int G = H / Hkv;
 #pragma omp parallel for schedule(dynamic, 1)
-  for (int bh = 0; bh < B * H; ++bh) {
-    int b = bh / H, h = bh % H;
+  for (int bk = 0; bk < B * Hkv; ++bk) {
+    int b = bk / Hkv, hk = bk % Hkv;
     size_t SS = (size_t)S * S;
-    float *Pt = (float *)calloc(SS, sizeof(float));  /* bf16-rounded p, widened */
-    float *dSt = (float *)calloc(SS, sizeof(float)); /* bf16-rounded dS, widened */
-    for (int i = 0; i < S; ++i) {
-      const bf16_t *qi = q + (size_t)ldq * (b * S + i) + h * DH;
-      const bf16_t *doi = dout + (size_t)ld_out * (b * S + i) + h * DH;
-      const bf16_t *oi = out + (size_t)ld_out * (b * S + i) + h * DH;
-      float t[DH];
-      for (int c = 0; c < DH; ++c) t[c] = fmul(bf2f(doi[c]), bf2f(oi[c]));
-      float delta = tree128(t);
-      float L = lse[(size_t)bh * S + i];
-      for (int j = 0; j <= i; ++j) {
-        float s = fmul(dot128(qi, k + (size_t)ldq * (b * S + j) + h * DH), ATT_SCALE);
-        float p = det_exp(fsub(s, L));
-        float dP = dot128(doi, v + (size_t)ldq * (b * S + j) + h * DH);
-        float dS = fmul(fmul(p, fsub(dP, delta)), ATT_SCALE);
-        Pt[(size_t)i * S + j] = bf2f(f2bf(p));
-        dSt[(size_t)i * S + j] = bf2f(f2bf(dS));
+    float *Pt = (float *)calloc(SS * G, sizeof(float));  /* bf16-rounded p, widened, per query head of the group */
+    float *dSt = (float *)calloc(SS * G, sizeof(float)); /* bf16-rounded dS, widened */
+    for (int g = 0; g < G; ++g) {
+      int h = hk * G + g;
+      for (int i = 0; i < S; ++i) {
+        const bf16_t *qi = q + (size_t)ldq * (b * S + i) + h * DH;
+        const bf16_t *doi = dout + (size_t)ld_out * (b * S + i) + h * DH;
+        const bf16_t *oi = out + (size_t)ld_out * (b * S + i) + h * DH;
+        float t[DH];
+        for (int c = 0; c < DH; ++c) t[c] = fmul(bf2f(doi[c]), bf2f(oi[c]));
+        float delta = tree128(t);
+        float L = lse[((size_t)b * H + h) * S + i];
+        for (int j = 0; j <= i; ++j) {
+          if (!visible(i, j, W)) continue;
+          float s = fmul(dot128(qi, k + (size_t)ldq * (b * S + j) + hk * DH), ATT_SCALE);
+          float p = det_exp(fsub(s, L));
+          float dP = dot128(doi, v + (size_t)ldq * (b * S + j) + hk * DH);
+          float dS = fmul(fmul(p, fsub(dP, delta)), ATT_SCALE);
+          Pt[g * SS + (size_t)i * S + j] = bf2f(f2bf(p));
+          dSt[g * SS + (size_t)i * S + j] = bf2f(f2bf(dS));
+        }
       }
     }
     for (int j = 0; j < S; ++j)
       for (int c = 0; c < DH; ++c) {
         float av = 0.0f, ak = 0.0f;
-        for (int i = j; i < S; ++i) {
-          av = fadd(av, fmul(Pt[(size_t)i * S + j], bf2f(dout[(size_t)ld_out * (b * S + i) + h * DH + c])));
-          ak = fadd(ak, fmul(dSt[(size_t)i * S + j], bf2f(q[(size_t)ldq * (b * S + i) + h * DH + c])));
+        for (int g = 0; g < G; ++g) {
+          int h = hk * G + g;
+          for (int i = j; i < S; ++i) {
+            if (!visible(i, j, W)) continue;
+            av = fadd(av, fmul(Pt[g * SS + (size_t)i * S + j], bf2f(dout[(size_t)ld_out * (b * S + i) + h * DH + c])));
+            ak = fadd(ak, fmul(dSt[g * SS + (size_t)i * S + j], bf2f(q[(size_t)ldq * (b * S + i) + h * DH + c])));
+          }
         }
-        dv[(size_t)ld_d * (b * S + j) + h * DH + c] = f2bf(av);
-        dk[(size_t)ld_d * (b * S + j) + h * DH + c] = f2bf(ak);
+        dv[(size_t)ld_d * (b * S + j) + hk * DH + c] = f2bf(av);
+        dk[(size_t)ld_d * (b * S + j) + hk * DH + c] = f2bf(ak);
       }
-    for (int i = 0; i < S; ++i)
-      for (int c = 0; c < DH; ++c) {
-        float aq = 0.0f;
-        for (int j = 0; j <= i; ++j)
-          aq = fadd(aq, fmul(dSt[(size_t)i * S + j], bf2f(k[(size_t)ldq * (b * S + j) + h * DH + c])));
-        dq[(size_t)ld_d * (b * S + i) + h * DH + c] = f2bf(aq);
-      }
+    for (int g = 0; g < G; ++g) {
+      int h = hk * G + g;
+      for (int i = 0; i < S; ++i)
+        for (int c = 0; c < DH; ++c) {
+          float aq = 0.0f;
+          for (int j = 0; j <= i; ++j) {
+            if (!visible(i, j, W)) continue;
+            aq = fadd(aq, fmul(dSt[g * SS + (size_t)i * S + j], bf2f(k[(size_t)ldq * (b * S + j) + hk * DH + c])));
+          }
+          dq[(size_t)ld_d * (b * S + i) + h * DH + c] = f2bf(aq);
+        }
+    }
     free(Pt); free(dSt);
   }
 }

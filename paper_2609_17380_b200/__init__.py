@@ -231,19 +231,21 @@ def det_xent_bwd(logits_inout, target, lse, rows, V, z_weight, scale):
 
 
 # ---- attention ------------------------------------------------------------------------------------------------
-def det_attn_fwd(q, k, v, ld, B, H, S, out, ld_out, lse):
-    _check("det_attn_fwd", load().det_attn_fwd(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H), C.c_int(S),
-                                               _ptr(out), C.c_int(ld_out), _ptr(lse), _stream()))
+def det_attn_fwd(q, k, v, ld, B, H, S, out, ld_out, lse, Hkv=None, window=0):
+    _check("det_attn_fwd", load().det_attn_fwd(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H),
+                                               C.c_int(H if Hkv is None else Hkv), C.c_int(S), C.c_int(window), _ptr(out),
+                                               C.c_int(ld_out), _ptr(lse), _stream()))
 
 
-def det_attn_bwd_ws_bytes(B, H, S):
-    return load().det_attn_bwd_ws_bytes(C.c_int(B), C.c_int(H), C.c_int(S))
+def det_attn_bwd_ws_bytes(B, H, S, Hkv=None):
+    return load().det_attn_bwd_ws_bytes(C.c_int(B), C.c_int(H), C.c_int(H if Hkv is None else Hkv), C.c_int(S))
 
 
-def det_attn_bwd(dout, q, k, v, out, lse, ld, ld_out, B, H, S, dq, dk, dv, ld_d, ws):
+def det_attn_bwd(dout, q, k, v, out, lse, ld, ld_out, B, H, S, dq, dk, dv, ld_d, ws, Hkv=None, window=0):
     _check("det_attn_bwd", load().det_attn_bwd(_ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), C.c_int(ld),
-                                               C.c_int(ld_out), C.c_int(B), C.c_int(H), C.c_int(S), _ptr(dq), _ptr(dk),
-                                               _ptr(dv), C.c_int(ld_d), *_ws(ws), _stream()))
+                                               C.c_int(ld_out), C.c_int(B), C.c_int(H), C.c_int(H if Hkv is None else Hkv),
+                                               C.c_int(S), C.c_int(window), _ptr(dq), _ptr(dk), _ptr(dv), C.c_int(ld_d),
+                                               *_ws(ws), _stream()))
 
 
 # ---- glue --------------------------------------------------------------------------------------------------------

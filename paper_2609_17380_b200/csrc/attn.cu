@@ -67,9 +67,14 @@ __device__ __forceinline__ void mac_4x8(const float (*As)[LQ], const float (*Bs)
   }
 }
 
+// Hkv key/value heads serve H query heads (head h reads key/value head h / (H/Hkv)); W > 0 restricts row i to the keys
+// j in (i - W, i] (W a multiple of 128): the tile loop then starts at the tile of q0 - W, and a row skips a tile that
+// holds none of its keys (its statistics stay untouched: alpha = 1, all weights 0).
+template <bool WIN>
 __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                                                    const uint16_t* __restrict__ v, int ld, int H, int S,
+                                                    const uint16_t* __restrict__ v, int ld, int H, int Hkv, int S, int Warg,
                                                     uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse) {
+  const int W = WIN ? Warg : 0;
   extern __shared__ __align__(16) float sm[];
   float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                 // [dim][query]
   float(*KV)[LQ] = reinterpret_cast<float(*)[LQ]>(sm + DH * LQ);       // K: [dim][key]; V: [key][dim]
@@ -82,8 +87,9 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const size_t row0 = (size_t)b * S;
   const uint16_t* qp = q + row0 * ld + (size_t)h * DH;
-  const uint16_t* kp = k + row0 * ld + (size_t)h * DH;
-  const uint16_t* vp = v + row0 * ld + (size_t)h * DH;
+  const int hk = h / (H / Hkv);
+  const uint16_t* kp = k + row0 * ld + (size_t)hk * DH;
+  const uint16_t* vp = v + row0 * ld + (size_t)hk * DH;
 
   // one 128 x 128 bf16 tile in flight: 4 sixteen-byte words per thread
   uint4 rw[4];
@@ -95,7 +101,8 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
                               : make_uint4(0u, 0u, 0u, 0u);
     }
   };
-  fetch_k(0);
+  const int jt0 = (WIN && q0 > W) ? (q0 - W) / FK : 0;
+  fetch_k(jt0 * FK);
   bool tq = false;
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
@@ -121,7 +128,7 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
     for (int e = 0; e < 4; ++e) o[i][e] = make_float2(0.0f, 0.0f);
   }
   const int ntiles = q0 / FK + 1;
-  for (int jt = 0; jt < ntiles; ++jt) {
+  for (int jt = jt0; jt < ntiles; ++jt) {
     const int j0 = jt * FK;
     // ---- K tile (fetched during the previous tile's P.V), transposed ----
     bool tk = false;
@@ -153,23 +160,25 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
     float alpha[4];
     bool tp = false;
     const bool diag = (jt == ntiles - 1);  // only the last tile of a row block reaches past the diagonal
+    const bool edge = WIN && j0 <= q0 + FQ - 1 - W;  // some row's window starts inside or after this tile
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int rl = ty * 4 + i;
       const int row = q0 + rl;
+      const bool rowvalid = !(edge && j0 + FK - 1 <= row - W);
       float sv[8] = {s[i][0].x, s[i][0].y, s[i][1].x, s[i][1].y, s[i][2].x, s[i][2].y, s[i][3].x, s[i][3].y};
       float mt = m[i];
       bool valid[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int key = j0 + ((e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4));
-        valid[e] = !diag || key <= row;
+        valid[e] = (!diag || key <= row) && (!edge || key > row - W);
         sv[e] = fmul(sv[e], ATT_SCALE);
         if (valid[e]) mt = fmaxf(mt, sv[e]);
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
-      alpha[i] = det_exp(fsub(m[i], mt));
+      alpha[i] = rowvalid ? det_exp(fsub(m[i], mt)) : 1.0f;
       float p[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) p[e] = valid[e] ? det_exp(fsub(sv[e], mt)) : 0.0f;
@@ -266,46 +275,56 @@ static int set_smem(const void* fn, size_t bytes) {
 
 using namespace det;
 
-extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S,
-                            det_bf16* out, int ld_out, float* lse, void* stream) {
-  if (!q || !k || !v || !out || !lse || B <= 0 || H <= 0 || S <= 0) return DET_ERR_ARG;
-  if (S % 64 || ld % 8 || ld_out % 8 || ld < H * DH || ld_out < H * DH || H > 65535 || B > 65535) return DET_ERR_SHAPE;
+extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                            int window, det_bf16* out, int ld_out, float* lse, void* stream) {
+  if (!q || !k || !v || !out || !lse || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0) return DET_ERR_ARG;
+  if (S % 64 || ld % 8 || ld_out % 8 || ld < H * DH || ld_out < H * DH || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
   static bool cfg = false;
-  if (!cfg) { if (set_smem((const void*)k_attn_fwd, FWD_SMEM)) return DET_ERR_CUDA; cfg = true; }
+  if (!cfg) {
+    if (set_smem((const void*)k_attn_fwd<false>, FWD_SMEM) || set_smem((const void*)k_attn_fwd<true>, FWD_SMEM)) return DET_ERR_CUDA;
+    cfg = true;
+  }
   dim3 grid(H * B, (S + FQ - 1) / FQ);
-  k_attn_fwd<<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, S, out, ld_out, lse);
+  if (window) k_attn_fwd<true><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse);
+  else k_attn_fwd<false><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, 0, out, ld_out, lse);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
 
-// workspace: P f32 [B*H, S, S], dS bf16 [B*H, S, S], Delta f32 [B*H, S]
-extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int S) {
+// workspace: P f32 [B*H, S, S], dS bf16 [B*H, S, S], Delta f32 [B*H, S], and with grouped queries the f32 accumulators
+// [B*Hkv, S, 128] that carry dK / dV from one query head of a group to the next
+extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S) {
   return align_up((size_t)B * H * S * S * 4, 256) + align_up((size_t)B * H * S * S * 2, 256) +
-         align_up((size_t)B * H * S * 4, 256);
+         align_up((size_t)B * H * S * 4, 256) + (Hkv < H ? align_up((size_t)B * Hkv * S * DH * 4, 256) : 0);
 }
 
 extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
-                            const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int S, det_bf16* dq,
-                            det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes, void* stream) {
-  if (!dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv || B <= 0 || H <= 0 || S <= 0) return DET_ERR_ARG;
-  if (S % 64 || ld % 8 || ld_out % 8 || ld_d % 8 || (long long)B * H > 65535) return DET_ERR_SHAPE;
+                            const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
+                            int window, det_bf16* dq, det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes,
+                            void* stream) {
+  if (!dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0)
+    return DET_ERR_ARG;
+  if (S % 64 || ld % 8 || ld_out % 8 || ld_d % 8 || (long long)B * H > 65535 || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(dout) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
     return DET_ERR_ALIGN;
-  if (!ws || ws_bytes < det_attn_bwd_ws_bytes(B, H, S)) return DET_ERR_WORKSPACE;
+  if (!ws || ws_bytes < det_attn_bwd_ws_bytes(B, H, Hkv, S)) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
+  const int G = H / Hkv;
   const size_t matP = align_up((size_t)B * H * S * S * 4, 256), matS = align_up((size_t)B * H * S * S * 2, 256);
+  const size_t dl = align_up((size_t)B * H * S * 4, 256);
   float* Pf = (float*)ws;
   uint16_t* dSt = (uint16_t*)((uint8_t*)ws + matP);
   float* delta = (float*)((uint8_t*)ws + matP + matS);
+  float* carry = (float*)((uint8_t*)ws + matP + matS + dl);
   const size_t nrows = (size_t)B * H * S;
   k_attn_delta<<<DET_L((unsigned)((nrows + 7) / 8)), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
   DET_CHECK_LAUNCH();
-  // P[i,j] = exp(scale * sum_d q[i,d] k[j,d] - L_i) for j <= i (f32; tiles above the diagonal are never touched), then
-  // dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both contractions ascend over the 128 dims
+  // P[i,j] = exp(scale * sum_d q[i,d] k[j,d] - L_i) for visible (i,j) (f32; tiles without a visible pair are never
+  // touched), then dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both ascend over the 128 dims
   OgemmArgs e = {};
-  e.I = S; e.J = S; e.C = DH; e.H = H; e.range_mode = 3; e.scale = ATT_SCALE;
+  e.I = S; e.J = S; e.C = DH; e.H = H; e.range_mode = 3; e.scale = ATT_SCALE; e.window = window; e.b_div = G;
   e.ldo = S; e.o_b = (long long)H * S * S; e.o_h = (long long)S * S;
   e.A = q; e.lda = ld; e.a_b = (long long)S * ld; e.a_h = DH;
   e.B = k; e.ldb = ld; e.b_b = (long long)S * ld; e.b_h = DH;
@@ -317,19 +336,35 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   e.out = dSt; e.rowv = delta; e.Pin = Pf;
   rc = ogemm_launch<CONTIG, CONTIG, false, true, 128, OEPI_DS>(e, B * H, st);
   if (rc != DET_OK) return rc;
-  // dV[j,c] = sum over queries i >= j ascending of P~[i,j] dO[i,c];  dK[j,c] likewise with dS~ and q
+  // dV[j,c] = sum over the query heads g of the group, then over queries i >= j ascending, of P~[i,j] dO[i,c];
+  // dK[j,c] likewise with dS~ and q.  One accumulator per output: with G > 1 it travels through `carry` in f32.
+  for (int which = 0; which < 2; ++which) {
+    for (int g = 0; g < G; ++g) {
+      OgemmArgs p = {};
+      p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = Hkv; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
+      p.h_mul = G; p.h_add = g; p.range_mode = 1; p.window = window;
+      p.A = which == 0 ? (const void*)Pf : (const void*)dSt;
+      if (which == 0) { p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; }
+      else { p.B = q; p.ldb = ld; p.b_b = (long long)S * ld; }
+      p.b_h = DH;
+      if (g > 0) { p.acc_in = carry; p.acc_ld = DH; p.acc_b = (long long)Hkv * S * DH; p.acc_h = (long long)S * DH; }
+      if (g == G - 1) {
+        p.out = which == 0 ? dv : dk; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
+        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * Hkv, st)     // P is rounded to bf16 as read
+                        : ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * Hkv, st);
+      } else {
+        p.out = carry; p.ldo = DH; p.o_b = (long long)Hkv * S * DH; p.o_h = (long long)S * DH;
+        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, false, 128>(p, B * Hkv, st)
+                        : ogemm_launch<STRIDED, STRIDED, false, false, 128>(p, B * Hkv, st);
+      }
+      if (rc != DET_OK) return rc;
+    }
+  }
+  // dQ[i,c] = sum over visible keys j ascending of dS~[i,j] k[j,c]
   OgemmArgs p = {};
   p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
-  p.range_mode = 1;
-  p.A = Pf; p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; p.b_h = DH;
-  p.out = dv; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
-  rc = ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * H, st);   // P is rounded to bf16 as it is read
-  if (rc != DET_OK) return rc;
-  p.A = dSt; p.B = q; p.ldb = ld; p.b_b = (long long)S * ld; p.out = dk;
-  rc = ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * H, st);
-  if (rc != DET_OK) return rc;
-  // dQ[i,c] = sum over keys j <= i ascending of dS~[i,j] k[j,c]
-  p.B = k; p.out = dq; p.range_mode = 2;
+  p.A = dSt; p.B = k; p.ldb = ld; p.b_b = (long long)S * ld; p.b_h = DH; p.b_div = G;
+  p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
   rc = ogemm_launch<CONTIG, STRIDED, false, true, 128>(p, B * H, st);
   if (rc != DET_OK) return rc;
   DET_CHECK_LAUNCH();

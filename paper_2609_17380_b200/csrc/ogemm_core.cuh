@@ -150,8 +150,19 @@ struct OgemmArgs {
   int init;             // f32 output only: start from the values already in out
   int H;                // batching: blockIdx.z = b * H + h
   long long a_b, a_h, b_b, b_h, o_b, o_h;  // element offsets per batch index / head index
+  // head mapping for grouped-query attention (0 = identity): A reads head hA = h * h_mul + h_add, B reads head
+  // hA / b_div, the output (and rowv, Pin, acc_in) belongs to head h
+  int h_mul, h_add, b_div;
+  // optional f32 accumulators to start from (any output type): one sequential accumulator can be carried through
+  // several launches this way; batched with acc_b / acc_h, leading dimension acc_ld
+  const float* acc_in;
+  int acc_ld;
+  long long acc_b, acc_h;
+  int window;           // sliding window W (multiple of 128; 0 = none): only |query - key| < W contributes
   int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile;
-                        // 3: whole contraction, but tiles entirely above the diagonal (j0 > i0) are skipped
+                        // 3: whole contraction, but tiles entirely above the diagonal (j0 > i0) or entirely below the
+                        //    window are skipped
+                        // (with a window, mode 1 also stops at c < i0 + W + 128 and mode 2 starts at c >= i0 - W)
   // epilogues of the attention backward (EPI 1, 2); rowv and Pin are batched like the output
   const float* rowv;    // one value per row i of each batch: the logsumexp L (EPI 1) or Delta (EPI 2)
   const float* Pin;     // EPI 2: the f32 weights written by EPI 1, same layout as the output
@@ -170,24 +181,29 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
   // blocks are handed out in linear order; with a causal range the longest contractions are put first
   const int i0 = (p.range_mode == 2 ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y) * OT, j0 = blockIdx.x * TN;
-  if (p.range_mode == 3 && j0 > i0) return;
+  const int W = p.window;
+  if (p.range_mode == 3 && (j0 > i0 || (W && i0 >= j0 + W + OT))) return;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
   const long long zb = blockIdx.z / p.H, zh = blockIdx.z % p.H;
-  const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + zh * p.a_h)
-                       : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + zh * p.a_h);
-  const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + zh * p.b_h;
+  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
+  const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
+                       : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
+  const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
   void* out = OUT_BF16 ? (void*)(reinterpret_cast<uint16_t*>(p.out) + zb * p.o_b + zh * p.o_h)
                        : (void*)(reinterpret_cast<float*>(p.out) + zb * p.o_b + zh * p.o_h);
   const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
   int c_lo = 0, C = p.C;
-  if (p.range_mode == 1) c_lo = i0;
-  if (p.range_mode == 2) C = min(p.C, i0 + OT);
+  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
+  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
   float2 acc[8][TN / 32];
 #pragma unroll
   for (int a = 0; a < 8; ++a)
 #pragma unroll
     for (int b = 0; b < TN / 32; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
-  if (p.init && !OUT_BF16) {
+  const float* accp = p.acc_in ? p.acc_in + zb * p.acc_b + zh * p.acc_h
+                               : ((p.init && !OUT_BF16) ? reinterpret_cast<const float*>(out) : nullptr);
+  if (accp) {
+    const int ldacc = p.acc_in ? p.acc_ld : ldo;
 #pragma unroll
     for (int a = 0; a < 8; ++a) {
       const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
@@ -195,7 +211,7 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
       for (int g = 0; g < TN / 64; ++g) {
         const int c = j0 + g * 64 + tx * 4;
         if (r < I && c < J) {
-          float4 t = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(out) + (size_t)r * ldo + c);
+          float4 t = *reinterpret_cast<const float4*>(accp + (size_t)r * ldacc + c);
           acc[a][2 * g] = make_float2(t.x, t.y);
           acc[a][2 * g + 1] = make_float2(t.z, t.w);
         }
@@ -243,7 +259,8 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
         float w[4] = {acc[a][2 * g].x, acc[a][2 * g].y, acc[a][2 * g + 1].x, acc[a][2 * g + 1].y};
         if (EPI == OEPI_P) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) w[e] = (c + e <= r) ? det_exp(fsub(fmul(w[e], p.scale), rv)) : 0.0f;
+          for (int e = 0; e < 4; ++e)
+            w[e] = (c + e <= r && (!W || c + e > r - W)) ? det_exp(fsub(fmul(w[e], p.scale), rv)) : 0.0f;
         }
         if (EPI == OEPI_DS) {
           const float4 pw = *reinterpret_cast<const float4*>(p.Pin + zb * p.o_b + zh * p.o_h + (size_t)r * ldo + c);

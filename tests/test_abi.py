@@ -39,5 +39,7 @@ def test_host_side_argument_checks():
     assert lib.det_rmsnorm_fwd(0, a1, None, 4, 8, ctypes.c_float(0), a16, a16, None) == -3          # alignment
     assert lib.det_linear_fwd(a16, a16, a16, a16, 100, 128, 128, a16, a16, None, None) == -2        # M % 128
     assert lib.det_linear_fwd(a16, a16, a16, a16, 128, 128, 1 << 17, a16, a16, None, None) == -5    # int32 range
-    assert lib.det_attn_fwd(a16, a16, a16, 128, 1, 1, 100, a16, 128, a16, None) == -2               # S % 64
+    assert lib.det_attn_fwd(a16, a16, a16, 128, 1, 1, 1, 100, 0, a16, 128, a16, None) == -2         # S % 64
+    assert lib.det_attn_fwd(a16, a16, a16, 512, 1, 4, 3, 128, 0, a16, 512, a16, None) == -2         # H % Hkv
+    assert lib.det_attn_fwd(a16, a16, a16, 128, 1, 1, 1, 128, 100, a16, 128, a16, None) == -2       # window % 128
     assert lib.det_xent_fwd(a16, a16, 4, 8, ctypes.c_float(0), a16, a16, a16, a16, a16, ctypes.c_size_t(8), None, None) == -4

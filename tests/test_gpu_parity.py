@@ -456,6 +456,33 @@ def test_attention(det, B, H, S):
         assert_same_bits(got[:, c * HD:(c + 1) * HD], want[:, c * HD:(c + 1) * HD], name)
 
 
+@pytest.mark.parametrize("B,H,Hkv,S,W", [(1, 4, 2, 192, 0), (2, 4, 1, 128, 0), (1, 2, 2, 448, 128), (1, 1, 1, 640, 256),
+                                         (1, 4, 2, 384, 128), (1, 2, 2, 256, 512)])
+def test_attention_grouped_and_windowed(det, B, H, Hkv, S, W):
+    """Grouped-query heads (Hkv < H) and sliding windows: forward and all three gradients bit for bit."""
+    HD, KD = H * 128, Hkv * 128
+    ld = HD + 2 * KD
+    qkv = synth.normal_bf16((B * S, ld), 1.0, seed=15, tid=1)
+    dout = synth.normal_bf16((B * S, HD), 0.1, seed=15, tid=2)
+    dqkv_in = dev(qkv)
+    base = dqkv_in.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    det.det_attn_fwd(base, base + 2 * HD, base + 2 * (HD + KD), ld, B, H, S, out, HD, lse, Hkv=Hkv, window=W)
+    _sync()
+    oout, olse = oracle.attn_fwd(qkv, B, H, S, Hkv=Hkv, window=W)
+    assert_same_bits(host(lse), olse, "lse")
+    assert_same_bits(host(out, np.uint16), oout, "out")
+    dqkv = empty((B * S, ld), np.uint16)
+    db = dqkv.data_ptr()
+    det.det_attn_bwd(dev(dout), base, base + 2 * HD, base + 2 * (HD + KD), out, lse, ld, HD, B, H, S, db, db + 2 * HD,
+                     db + 2 * (HD + KD), ld, ws(det.det_attn_bwd_ws_bytes(B, H, S, Hkv)), Hkv=Hkv, window=W)
+    _sync()
+    want = oracle.attn_bwd(dout, qkv, oout, olse, B, H, S, Hkv=Hkv, window=W)
+    got = host(dqkv, np.uint16)
+    for name, lo, hi in (("dq", 0, HD), ("dk", HD, HD + KD), ("dv", HD + KD, ld)):
+        assert_same_bits(got[:, lo:hi], want[:, lo:hi], name)
+
+
 # ------------------------------------------------------------------ slabs whose products can underflow
 def _sprinkle_tiny(a, seed, frac=0.002):
     """Overwrite a fraction of a bf16 tensor with magnitudes around 2^-64 .. 2^-62 (random signs)."""

@@ -269,6 +269,76 @@ def test_attention_backward_against_float64():
     assert np.array_equal(d2[:S, :], dqkv[:S, :]) and np.array_equal(d2[S:S + 130 - 0, :H * 128], dqkv[S:S + 130, :H * 128])
 
 
+def _expand_kv(qkv, H, Hkv):
+    """grouped q|k|v rows -> multi-head rows with every key/value head repeated for its query heads"""
+    G = H // Hkv
+    q = qkv[:, :H * 128]
+    k = qkv[:, H * 128:(H + Hkv) * 128].reshape(-1, Hkv, 128).repeat(G, axis=1).reshape(-1, H * 128)
+    v = qkv[:, (H + Hkv) * 128:].reshape(-1, Hkv, 128).repeat(G, axis=1).reshape(-1, H * 128)
+    return np.ascontiguousarray(np.concatenate([q, k, v], 1))
+
+
+def test_grouped_query_attention_pins():
+    """Sec. 3.1 GQA: the forward of a query head is that of multi-head attention on its shared key/value head (bit
+    for bit); dq likewise; dk, dv of a shared head are the float64 sums over its query heads."""
+    B, H, Hkv, S = 1, 4, 2, 160
+    qkv = synth.normal_bf16((B * S, (H + 2 * Hkv) * 128), 1.0, seed=0, tid=65)
+    dout = synth.normal_bf16((B * S, H * 128), 0.1, seed=0, tid=66)
+    out, lse = oracle.attn_fwd(qkv, B, H, S, Hkv=Hkv)
+    full = _expand_kv(qkv, H, Hkv)
+    out_m, lse_m = oracle.attn_fwd(full, B, H, S)
+    assert np.array_equal(out, out_m) and np.array_equal(lse, lse_m)
+    d = oracle.attn_bwd(dout, qkv, out, lse, B, H, S, Hkv=Hkv)
+    d_m = oracle.attn_bwd(dout, full, out_m, lse_m, B, H, S)
+    assert np.array_equal(d[:, :H * 128], d_m[:, :H * 128])                     # dq is per query head
+    q, k, v, p, o, _ = _attn_ref(full, B, H, S)
+    do = bf(dout).astype(np.float64).reshape(B, S, H, 128).transpose(0, 2, 1, 3)
+    dv = p.transpose(0, 1, 3, 2) @ do
+    ds = p * (do @ v.transpose(0, 1, 3, 2) - (do * o).sum(-1, keepdims=True)) / math.sqrt(128)
+    dk = ds.transpose(0, 1, 3, 2) @ q
+    G = H // Hkv
+    for name, ref, off in (("dk", dk, H * 128), ("dv", dv, (H + Hkv) * 128)):
+        r = ref.reshape(B, Hkv, G, S, 128).sum(2).transpose(0, 2, 1, 3).reshape(B * S, Hkv * 128)
+        assert rel_err(bf(d[:, off:off + Hkv * 128]).astype(np.float64), r) < 0.01, name
+    # one group per head is plain multi-head attention
+    assert np.array_equal(oracle.attn_fwd(full, B, H, S, Hkv=H)[0], out_m)
+
+
+def test_sliding_window_attention_pins():
+    """Sec. 3.1 SWA: keys j in (i - W, i].  A window that covers the sequence is full causal attention bit for bit;
+    keys that left the window cannot change a bit of the row; float64 agreement with the banded softmax."""
+    B, H, S, W = 1, 1, 400, 128
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=67)
+    dout = synth.normal_bf16((B * S, H * 128), 0.1, seed=0, tid=68)
+    out_f, lse_f = oracle.attn_fwd(qkv, B, H, S)
+    out_w, lse_w = oracle.attn_fwd(qkv, B, H, S, window=512)
+    assert np.array_equal(out_f, out_w) and np.array_equal(lse_f, lse_w)
+    assert np.array_equal(oracle.attn_bwd(dout, qkv, out_f, lse_f, B, H, S), oracle.attn_bwd(dout, qkv, out_w, lse_w, B, H, S, window=512))
+    out, lse = oracle.attn_fwd(qkv, B, H, S, window=W)
+    assert np.array_equal(out[:W], out_f[:W]) and not np.array_equal(out[W:], out_f[W:])   # rows < W see everything
+    x = bf(qkv).astype(np.float64).reshape(S, 3, 128)
+    s = x[:, 0] @ x[:, 1].T / math.sqrt(128)
+    i, j = np.arange(S)[:, None], np.arange(S)[None, :]
+    s = np.where((j <= i) & (j > i - W), s, -np.inf)
+    l64 = np.log(np.exp(s - s.max(-1, keepdims=True)).sum(-1)) + s.max(-1)
+    p = np.exp(s - l64[:, None])
+    assert np.abs(bf(out) - p @ x[:, 2]).max() < 0.02 and np.allclose(lse[0, 0], l64, rtol=1e-5, atol=1e-5)
+    # locality: rows >= 300 do not depend on keys/values before 300 - W + 1 = 173
+    qkv2 = qkv.copy(); qkv2[:173, 128:] = synth.normal_bf16((173, 256), 1.0, seed=3, tid=69)
+    out2, lse2 = oracle.attn_fwd(qkv2, B, H, S, window=W)
+    assert np.array_equal(out2[300:], out[300:]) and np.array_equal(lse2[..., 300:], lse[..., 300:])
+    # backward against the banded float64 softmax
+    d = oracle.attn_bwd(dout, qkv, out, lse, B, H, S, window=W)
+    do = bf(dout).astype(np.float64)
+    o = p @ x[:, 2]
+    ds = p * (do @ x[:, 2].T - (do * o).sum(-1, keepdims=True)) / math.sqrt(128)
+    for c, ref in enumerate((ds @ x[:, 1], ds.T @ x[:, 0], p.T @ do)):
+        assert rel_err(bf(d[:, c * 128:(c + 1) * 128]).astype(np.float64), ref) < 0.01
+    # dk, dv of keys that no later query can see inside the window ... every key is seen by itself; key 0 only by rows < W
+    d3 = oracle.attn_bwd(dout, qkv2, out2, lse2, B, H, S, window=W)
+    assert np.array_equal(d3[300:, :128], d[300:, :128])                          # dq rows >= 300 unchanged
+
+
 # ---------------------------------------------------------------- glue
 def test_glue_ops():
     gu = synth.normal_bf16((9, 512), 2.0, seed=0, tid=70)
