@@ -11,11 +11,26 @@ import oracle as O
 LINEARS = ("w_qkv", "w_o", "w_gu", "w_down")
 
 
+def _kv(cfg):
+    return cfg.get("n_kv_heads") or cfg["n_heads"]
+
+
+def _window(cfg, l):
+    """Sliding-window layers (Sec. 3.1): every `full_every`-th layer and the last one attend to everything."""
+    W = cfg.get("window", 0)
+    if not W or l == cfg["n_layers"] - 1 or (l + 1) % cfg.get("full_every", 5) == 0:
+        return 0
+    return W
+
+
 def _specs(cfg):
     D, Fh, V, L = cfg["d_model"], cfg["ffn"], cfg["vocab"], cfg["n_layers"]
+    nq = D + 2 * 128 * _kv(cfg)
     s = [("embed", (V, D))]
+    if cfg.get("embed_norm"):
+        s += [("embed_norm", (D,))]
     for l in range(L):
-        s += [("l%d.attn_norm" % l, (D,)), ("l%d.w_qkv" % l, (3 * D, D)), ("l%d.w_o" % l, (D, D)),
+        s += [("l%d.attn_norm" % l, (D,)), ("l%d.w_qkv" % l, (nq, D)), ("l%d.w_o" % l, (D, D)),
               ("l%d.ffn_norm" % l, (D,)), ("l%d.w_gu" % l, (2 * Fh, D)), ("l%d.w_down" % l, (D, Fh)),
               ("l%d.s_x" % l, (4,))]
     return s + [("final_norm", (D,)), ("lm_head", (V, D))]
@@ -24,9 +39,14 @@ def _specs(cfg):
 def forward(cfg, P, sw, tok, calibrate=False):
     """Returns (saved activations, loss pieces).  With calibrate, every activation step is set from its input."""
     L, H, S, B = cfg["n_layers"], cfg["n_heads"], cfg["seq"], cfg["micro_batch"]
+    Hkv, D = _kv(cfg), cfg["d_model"]
     inp = tok[:, :-1].reshape(-1)
     x = O.embed_fwd(inp, P["embed"])
     saved = {"inp": inp, "layers": []}
+    if cfg.get("embed_norm"):
+        saved["x_emb"] = x
+        x, saved["rstd_emb"] = O.rmsnorm_fwd(x, P["embed_norm"], 1e-6, bf=True)
+    rope = cfg.get("rope_tables")
     for l in range(L):
         sx = P["l%d.s_x" % l]
         a = {"x": x}
@@ -34,7 +54,15 @@ def forward(cfg, P, sw, tok, calibrate=False):
         if calibrate:
             sx[0] = O.lsq_act_scale_init(a["n1"])[0]
         a["qkv"], _, _ = O.linear_fwd(a["n1"], P["l%d.w_qkv" % l], sx[0:1], sw["l%d.w_qkv" % l])
-        a["att"], a["lse"] = O.attn_fwd(a["qkv"], B, H, S)
+        # the paper's block: gain-free RMS norm of every query and key head, then the rotary embedding
+        qk = np.ascontiguousarray(a["qkv"][:, :D + 128 * Hkv]).reshape(-1, 128)
+        if cfg.get("qk_norm"):
+            a["qk_pre"] = qk
+            qk, a["rstd_qk"] = O.rmsnorm_fwd(qk, None, 1e-6, bf=True)
+        if rope is not None:
+            qk = O.rope(qk.reshape(B * S, H + Hkv, 128), S, rope[0], rope[1]).reshape(-1, 128)
+        a["qkr"] = np.ascontiguousarray(np.concatenate([qk.reshape(B * S, -1), a["qkv"][:, D + 128 * Hkv:]], 1))
+        a["att"], a["lse"] = O.attn_fwd(a["qkr"], B, H, S, Hkv=Hkv, window=_window(cfg, l))
         if calibrate:
             sx[1] = O.lsq_act_scale_init(a["att"])[0]
         o, _, _ = O.linear_fwd(a["att"], P["l%d.w_o" % l], sx[1:2], sw["l%d.w_o" % l])
@@ -59,6 +87,7 @@ def microbatch_grad(cfg, P, sw, tok):
     """Forward + backward of one micro-batch; returns (flat f32 gradient in canonical order, mean loss)."""
     L, H, S, B = cfg["n_layers"], cfg["n_heads"], cfg["seq"], cfg["micro_batch"]
     hb = cfg.get("hadamard_block", 128)
+    Hkv, D, rope = _kv(cfg), cfg["d_model"], cfg.get("rope_tables")
     sv = forward(cfg, P, sw, tok)
     labels = tok[:, 1:].reshape(-1).astype(np.int32)
     T = labels.size
@@ -77,12 +106,20 @@ def microbatch_grad(cfg, P, sw, tok):
         d_h2, G["l%d.ffn_norm" % l] = O.rmsnorm_bwd(d_n2, a["h"], P["l%d.ffn_norm" % l], a["rstd2"], bf=True)
         d_h = O.residual_add(dx, d_h2)
         d_att, G["l%d.w_o" % l], d1 = O.linear_bwd(d_h, a["att"], P["l%d.w_o" % l], sx[1:2], sw["l%d.w_o" % l], hb)
-        d_qkv = O.attn_bwd(d_att, a["qkv"], a["att"], a["lse"], B, H, S)
+        d_qkv = O.attn_bwd(d_att, a["qkr"], a["att"], a["lse"], B, H, S, Hkv=Hkv, window=_window(cfg, l))
+        dqk = np.ascontiguousarray(d_qkv[:, :D + 128 * Hkv]).reshape(-1, 128)
+        if rope is not None:
+            dqk = O.rope(dqk.reshape(B * S, H + Hkv, 128), S, rope[0], rope[1], inverse=True).reshape(-1, 128)
+        if cfg.get("qk_norm"):
+            dqk, _ = O.rmsnorm_bwd(dqk, a["qk_pre"], None, a["rstd_qk"], bf=True)
+        d_qkv = np.ascontiguousarray(np.concatenate([dqk.reshape(B * S, -1), d_qkv[:, D + 128 * Hkv:]], 1))
         d_n1, G["l%d.w_qkv" % l], d0 = O.linear_bwd(d_qkv, a["n1"], P["l%d.w_qkv" % l], sx[0:1], sw["l%d.w_qkv" % l], hb)
         d_x1, G["l%d.attn_norm" % l] = O.rmsnorm_bwd(d_n1, a["x"], P["l%d.attn_norm" % l], a["rstd1"], bf=True)
         dx = O.residual_add(d_h, d_x1)
         ds[0], ds[1], ds[2], ds[3] = d0[0], d1[0], d2[0], d3[0]
         G["l%d.s_x" % l] = ds
+    if cfg.get("embed_norm"):
+        dx, G["embed_norm"] = O.rmsnorm_bwd(dx, sv["x_emb"], P["embed_norm"], sv["rstd_emb"], bf=True)
     G["embed"] = O.embed_bwd(sv["inp"], dx, cfg["vocab"])
     flat = np.concatenate([np.asarray(G[name], np.float32).reshape(-1) for name, _ in _specs(cfg)])
     return flat, float(loss_mean[0])
@@ -90,7 +127,8 @@ def microbatch_grad(cfg, P, sw, tok):
 
 def run_step(cfg, params, tokens, opt=None, calibrate=True):
     """One optimizer step.  cfg: dict (n_layers, d_model, n_heads, ffn, vocab, seq, micro_batch, mesh=(accum,
-    dp_shard, dp_replicate), optional hadamard_block, z_weight, lr, betas, eps, wd, clip, step).
+    dp_shard, dp_replicate), optional hadamard_block, z_weight, lr, betas, eps, wd, clip, step; the paper's block:
+    n_kv_heads, qk_norm, rope_tables=(cos, sin) f32 [seq, 64], embed_norm, window, full_every).
     params: dict name -> numpy (uint16 bf16 bits / float32 steps).  tokens: [n_mb, micro_batch, seq+1]."""
     P = {k: np.array(v, copy=True) for k, v in params.items()}
     specs = _specs(cfg)

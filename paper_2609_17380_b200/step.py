@@ -34,6 +34,13 @@ class ModelConfig:
     wd: float = 0.1
     clip: float = 1.0
     step: int = 1
+    # the paper's block (Sec. 3.1); the defaults are the plain multi-head block of the benchmark configuration
+    n_kv_heads: int = 0              # 0 = n_heads (multi-head); 4 with 16 query heads in the paper
+    qk_norm: bool = False            # gain-free RMS norm of every query and key head before RoPE
+    rope_tables: tuple = None        # (cos, sin) float32 numpy arrays [seq, 64], inputs of the step
+    embed_norm: bool = False         # RMSNorm (with gain) on the embedding output
+    window: int = 0                  # sliding-window width of the local layers (multiple of 128), 0 = all layers full
+    full_every: int = 5              # every full_every-th layer and the last one attend to the whole prefix
 
     def as_dict(self):
         return dict(self.__dict__)
@@ -46,12 +53,27 @@ class ModelConfig:
     def n_microbatches(self):
         return self.mesh[0] * self.mesh[1] * self.mesh[2]
 
+    @property
+    def kv_heads(self):
+        return self.n_kv_heads or self.n_heads
+
+    @property
+    def qkv_width(self):
+        return (self.n_heads + 2 * self.kv_heads) * 128
+
+    def layer_window(self, l):
+        if not self.window or l == self.n_layers - 1 or (l + 1) % self.full_every == 0:
+            return 0
+        return self.window
+
 
 def param_specs(cfg):
     D, Fh, V, L = cfg.d_model, cfg.ffn, cfg.vocab, cfg.n_layers
     s = [("embed", (V, D), "bf16")]
+    if cfg.embed_norm:
+        s += [("embed_norm", (D,), "bf16")]
     for l in range(L):
-        s += [("l%d.attn_norm" % l, (D,), "bf16"), ("l%d.w_qkv" % l, (3 * D, D), "bf16"), ("l%d.w_o" % l, (D, D), "bf16"),
+        s += [("l%d.attn_norm" % l, (D,), "bf16"), ("l%d.w_qkv" % l, (cfg.qkv_width, D), "bf16"), ("l%d.w_o" % l, (D, D), "bf16"),
               ("l%d.ffn_norm" % l, (D,), "bf16"), ("l%d.w_gu" % l, (2 * Fh, D), "bf16"), ("l%d.w_down" % l, (D, Fh), "bf16"),
               ("l%d.s_x" % l, (4,), "f32")]
     return s + [("final_norm", (D,), "bf16"), ("lm_head", (V, D), "bf16")]
@@ -97,27 +119,35 @@ class Replay:
         self.abufs = z(self.nbufs * (accum_len or g), F32)
         self.lin = {}
         for l in range(L):
-            for w, (N, K) in zip(LINEARS, ((3 * D, D), (D, D), (2 * Fh, D), (D, Fh))):
+            for w, (N, K) in zip(LINEARS, ((cfg.qkv_width, D), (D, D), (2 * Fh, D), (D, Fh))):
                 self.lin[(l, w)] = dict(N=N, K=K, s_w=z(N, F32), qW=z(N * K, I8), qWt=z(N * K, I8), s_u=z(1, F32))
         e = lambda n, dt: torch.empty(n, dtype=dt, device=device)
-        self.act = [dict(x=e(T * D, I16), rstd1=e(T, F32), n1=e(T * D, I16), qx_qkv=e(T * D, I8), qkv=e(T * 3 * D, I16),
+        QW, Hkv = cfg.qkv_width, cfg.kv_heads
+        self.head_ops = cfg.qk_norm or cfg.rope_tables is not None
+        if cfg.rope_tables is not None:
+            self.rope_cos = torch.from_numpy(np.ascontiguousarray(cfg.rope_tables[0], dtype=np.float32)).to(device)
+            self.rope_sin = torch.from_numpy(np.ascontiguousarray(cfg.rope_tables[1], dtype=np.float32)).to(device)
+        self.act = [dict(x=e(T * D, I16), rstd1=e(T, F32), n1=e(T * D, I16), qx_qkv=e(T * D, I8), qkv=e(T * QW, I16),
+                         qkr=e(T * QW if self.head_ops else 0, I16),
+                         rstd_qk=e(T * (cfg.n_heads + Hkv) if cfg.qk_norm else 0, F32),
                          lse=e(T * cfg.n_heads, F32), att=e(T * D, I16), qx_o=e(T * D, I8), h=e(T * D, I16), rstd2=e(T, F32),
                          n2=e(T * D, I16), qx_gu=e(T * D, I8), gu=e(T * 2 * Fh, I16), a=e(T * Fh, I16),
                          qx_down=e(T * Fh, I8)) for _ in range(L)]
         self.xf, self.rstdf, self.nf = e(T * D, I16), e(T, F32), e(T * D, I16)
+        self.x_emb, self.rstd_emb = (e(T * D, I16), e(T, F32)) if cfg.embed_norm else (None, None)
         self.logits = e(T * V, F32)
         self.loss_row, self.lse_x = e(T, F32), e(T, F32)
         self.loss_mean, self.z_mean = e(1, F32), e(1, F32)
-        self.tmp = [e(T * max(3 * D, 2 * Fh), I16) for _ in range(3)]   # gradient scratch activations
+        self.tmp = [e(T * max(QW, 2 * Fh), I16) for _ in range(3)]   # gradient scratch activations
         self.tok = e(T, I32)
         self.lab = e(T, I32)
         self.norm, self.coef = e(1, F32), e(1, F32)
         self.status = z(1, I32)
         B, H, S = cfg.micro_batch, cfg.n_heads, cfg.seq
-        wsb = max(det.det_attn_bwd_ws_bytes(B, H, S), det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
+        wsb = max(det.det_attn_bwd_ws_bytes(B, H, S, Hkv), det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
                   det.det_lsq_weight_scale_ws_bytes(2 * Fh, D), det.det_lsq_act_scale_init_ws_bytes(T * max(Fh, D)),
                   det.det_tensor_hash_ws_bytes(g * 4), det.det_sum_ws_bytes(g), 1 << 20,
-                  *[det.det_linear_bwd_ws_bytes(T, N, K) for (N, K) in ((3 * D, D), (D, D), (2 * Fh, D), (D, Fh))])
+                  *[det.det_linear_bwd_ws_bytes(T, N, K) for (N, K) in ((QW, D), (D, D), (2 * Fh, D), (D, Fh))])
         self.ws = e(wsb + 4096, torch.uint8)
         self.losses = []
         self.prof = None
@@ -211,15 +241,31 @@ class Replay:
         self.tok.copy_(tokens_mb[:, :-1].reshape(-1))
         self.lab.copy_(tokens_mb[:, 1:].reshape(-1))
         x = self.tmp[0][:T * D]
-        det.det_embed_fwd(self.tok, T, self.p("embed"), V, D, x)
+        Hkv, QW = cfg.kv_heads, cfg.qkv_width
+        if cfg.embed_norm:
+            det.det_embed_fwd(self.tok, T, self.p("embed"), V, D, self.x_emb)
+            det.det_rmsnorm_fwd(det.DET_BF16, self.x_emb, self.p("embed_norm"), T, D, 1e-6, x, self.rstd_emb)
+        else:
+            det.det_embed_fwd(self.tok, T, self.p("embed"), V, D, x)
         for l in range(L):
             a = self.act[l]
             a["x"].copy_(x)
             det.det_rmsnorm_fwd(det.DET_BF16, a["x"], self.p("l%d.attn_norm" % l), T, D, 1e-6, a["n1"], a["rstd1"])
             self._linear(l, "w_qkv", 0, a["n1"], T, a["qkv"], a["qx_qkv"], calibrate)
-            qp = a["qkv"].data_ptr()
+            qp = vp = a["qkv"].data_ptr()
+            if self.head_ops:
+                # queries and keys (the first H + Hkv heads of every row) are normalised and rotated into qkr; the
+                # values are read from qkv, which has the same row stride
+                src = a["qkv"]
+                if cfg.qk_norm:
+                    det.det_headnorm_fwd(src, QW, T, H + Hkv, 1e-6, a["qkr"], QW, a["rstd_qk"])
+                    src = a["qkr"]
+                if cfg.rope_tables is not None:
+                    det.det_rope(src, QW, T, H + Hkv, S, self.rope_cos, self.rope_sin, 0, a["qkr"], QW)
+                qp = a["qkr"].data_ptr()
             with self.span("attn_fwd"):
-                det.det_attn_fwd(qp, qp + 2 * D, qp + 4 * D, 3 * D, B, H, S, a["att"], D, a["lse"])
+                det.det_attn_fwd(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"], Hkv=Hkv,
+                                 window=cfg.layer_window(l))
             o = self.tmp[1][:T * D]
             self._linear(l, "w_o", 1, a["att"], T, o, a["qx_o"], calibrate)
             det.det_residual_add(a["x"], o, T * D, a["h"])
@@ -274,17 +320,28 @@ class Replay:
             det.det_residual_add(dx, d_h2, T * D, d_h)            # in place over dx
             d_att = t0[:T * D]
             self._linear_bwd(l, "w_o", 1, d_h, a["att"], a["qx_o"], T, d_att)
-            d_qkv = t2[:T * 3 * D]
-            qp, dp = a["qkv"].data_ptr(), d_qkv.data_ptr()
+            Hkv, QW = cfg.kv_heads, cfg.qkv_width
+            d_qkv = t2[:T * QW]
+            vp, dp = a["qkv"].data_ptr(), d_qkv.data_ptr()
+            qp = a["qkr"].data_ptr() if self.head_ops else vp
             with self.span("attn_bwd"):
-                det.det_attn_bwd(d_att, qp, qp + 2 * D, qp + 4 * D, a["att"], a["lse"], 3 * D, D, B, H, S, dp, dp + 2 * D,
-                                 dp + 4 * D, 3 * D, self.ws)
+                det.det_attn_bwd(d_att, qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), a["att"], a["lse"], QW, D, B, H, S, dp,
+                                 dp + 2 * D, dp + 2 * (D + 128 * Hkv), QW, self.ws, Hkv=Hkv, window=cfg.layer_window(l))
+            if cfg.rope_tables is not None:
+                det.det_rope(d_qkv, QW, T, H + Hkv, S, self.rope_cos, self.rope_sin, 1, d_qkv, QW)
+            if cfg.qk_norm:
+                det.det_headnorm_bwd(d_qkv, QW, a["qkv"], QW, a["rstd_qk"], T, H + Hkv, d_qkv, QW)
             d_n1 = t0[:T * D]
             self._linear_bwd(l, "w_qkv", 0, d_qkv, a["n1"], a["qx_qkv"], T, d_n1)
             d_x1 = t2[:T * D]
             det.det_rmsnorm_bwd(det.DET_BF16, d_n1, a["x"], self.p("l%d.attn_norm" % l), a["rstd1"], T, D, d_x1,
                                 self.g(self.gmb, "l%d.attn_norm" % l), self.ws)
             det.det_residual_add(d_h, d_x1, T * D, dx)            # dx aliases d_h: in place
+        if cfg.embed_norm:
+            d_emb = t0[:T * D]
+            det.det_rmsnorm_bwd(det.DET_BF16, dx, self.x_emb, self.p("embed_norm"), self.rstd_emb, T, D, d_emb,
+                                self.g(self.gmb, "embed_norm"), self.ws)
+            dx = d_emb
         det.det_embed_bwd(self.tok, T, dx, V, D, self.g(self.gmb, "embed"))
 
     def optimizer(self):

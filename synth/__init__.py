@@ -78,12 +78,16 @@ def randint(shape, high, seed=0, tid=0):
 # ---- model-shaped inputs --------------------------------------------------------------------------------
 def model_param_specs(cfg):
     """Canonical parameter order: embedding; per layer attn-norm gain, W_qkv, W_o, ffn-norm gain, W_gate/up,
-    W_down, the four activation steps; final-norm gain; LM head.  cfg: dict with n_layers, d_model, ffn, vocab.
-    Returns a list of (name, shape, kind) with kind in {"embed", "gain", "linear", "step", "head"}."""
+    W_down, the four activation steps; final-norm gain; LM head.  cfg: dict with n_layers, d_model, ffn, vocab and
+    optionally n_kv_heads (grouped queries: W_qkv has (n_heads + 2 n_kv_heads) * 128 rows) and embed_norm (a gain
+    after the embedding).  Returns a list of (name, shape, kind), kind in {"embed", "gain", "linear", "step", "head"}."""
     D, Fh, V, L = cfg["d_model"], cfg["ffn"], cfg["vocab"], cfg["n_layers"]
+    nq = D + 2 * 128 * (cfg.get("n_kv_heads") or cfg["n_heads"]) if "n_heads" in cfg else 3 * D
     specs = [("embed", (V, D), "embed")]
+    if cfg.get("embed_norm"):
+        specs += [("embed_norm", (D,), "gain")]
     for l in range(L):
-        specs += [("l%d.attn_norm" % l, (D,), "gain"), ("l%d.w_qkv" % l, (3 * D, D), "linear"),
+        specs += [("l%d.attn_norm" % l, (D,), "gain"), ("l%d.w_qkv" % l, (nq, D), "linear"),
                   ("l%d.w_o" % l, (D, D), "linear"), ("l%d.ffn_norm" % l, (D,), "gain"),
                   ("l%d.w_gu" % l, (2 * Fh, D), "linear"), ("l%d.w_down" % l, (D, Fh), "linear"),
                   ("l%d.s_x" % l, (4,), "step")]

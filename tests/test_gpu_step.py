@@ -10,6 +10,9 @@ pytestmark = pytest.mark.gpu
 def _run(cfg_kwargs, seed=0):
     from oracle import step as ostep
     from paper_2609_17380_b200 import step as dstep
+    cfg_kwargs = dict(cfg_kwargs)
+    if cfg_kwargs.pop("rope", False):
+        cfg_kwargs["rope_tables"] = synth.rope_tables(cfg_kwargs["seq"])
     cfg = dstep.ModelConfig(**cfg_kwargs)
     params = synth.model_params(cfg.as_dict(), seed=seed)
     tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=seed)
@@ -23,6 +26,12 @@ def _run(cfg_kwargs, seed=0):
     dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=1024, seq=192, micro_batch=2, mesh=(1, 1, 3)),
     dict(n_layers=1, d_model=128, n_heads=1, ffn=256, vocab=256, seq=128, micro_batch=1, mesh=(1, 1, 1), hadamard_block=0,
          z_weight=1e-4),
+    # the paper's block in miniature: grouped queries 4/1, QK-norm, RoPE, embedding norm, a sliding-window layer
+    # followed by a full one, z-loss
+    dict(n_layers=2, d_model=512, n_heads=4, n_kv_heads=1, ffn=384, vocab=512, seq=256, micro_batch=1, mesh=(1, 2, 1),
+         qk_norm=True, rope=True, embed_norm=True, window=128, z_weight=1e-4),
+    dict(n_layers=1, d_model=256, n_heads=2, n_kv_heads=2, ffn=256, vocab=256, seq=128, micro_batch=2, mesh=(1, 1, 1),
+         qk_norm=True, rope=True),
 ])
 def test_step_hashes_match_oracle(kw):
     cfg, got, want = _run(kw)
