@@ -250,6 +250,100 @@ __global__ void __launch_bounds__(128) k_rotc(const void* __restrict__ in, int R
   }
 }
 
+// (3) both rotations of dY from one read: a CTA stages a 128 x 128 tile of dY in shared memory (f32), then every thread
+//     rotates one row of dY * s_w along n (the A operand of the input-gradient GEMM) and one column of dY along the
+//     token index (the G operand of the weight-gradient GEMM, written transposed).  128 values per thread in registers,
+//     butterflies on register pairs with packed arithmetic: a + b is one packed add, a - b one packed fused
+//     multiply-add b * (-1) + a, which rounds exactly like the subtraction.  PASS 0 records both absmax values,
+//     PASS 1 quantises with them.  dY is read twice per backward pass instead of four times.
+constexpr int PT = 128, PLD = 129;
+constexpr size_t PREP_SMEM = (size_t)(PT * PLD + PT) * sizeof(float);
+
+__device__ __forceinline__ void wht128_pairs(float2 (&v)[64]) {
+#pragma unroll
+  for (int p = 0; p < 64; ++p) v[p] = make_float2(fadd(v[p].x, v[p].y), fsub(v[p].x, v[p].y));   // stage h = 1
+  const float2 m1 = make_float2(-1.0f, -1.0f);
+#pragma unroll
+  for (int hp = 1; hp < 64; hp <<= 1) {                                                        // stages h = 2 .. 64
+#pragma unroll
+    for (int p = 0; p < 64; ++p) {
+      if (!(p & hp)) {
+        const float2 a = v[p], b = v[p + hp];
+        v[p] = __fadd2_rn(a, b);
+        v[p + hp] = __ffma2_rn(b, m1, a);
+      }
+    }
+  }
+}
+__device__ __forceinline__ float absmax128(const float2 (&v)[64]) {
+  float m = 0.0f;
+#pragma unroll
+  for (int p = 0; p < 64; ++p) m = fmaxf(m, fmaxf(fabsf(v[p].x), fabsf(v[p].y)));
+  return m;
+}
+__device__ __forceinline__ void quant_store128(const float2 (&v)[64], float inv, int8_t* dst) {
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float2 lo = v[g * 8 + k * 2], hi = v[g * 8 + k * 2 + 1];
+      w[k] = ((uint32_t)(uint8_t)quant1(lo.x, inv)) | ((uint32_t)(uint8_t)quant1(lo.y, inv) << 8) |
+             ((uint32_t)(uint8_t)quant1(hi.x, inv) << 16) | ((uint32_t)(uint8_t)quant1(hi.y, inv) << 24);
+    }
+    d4[g] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+__device__ __forceinline__ void amax_publish(float local, uint32_t* amax) {
+#pragma unroll
+  for (int w = 16; w; w >>= 1) local = fmaxf(local, __shfl_xor_sync(0xffffffffu, local, w));
+  if ((threadIdx.x & 31) == 0 && local > 0.0f && __float_as_uint(local) > *reinterpret_cast<volatile uint32_t*>(amax))
+    atomicMax(amax, __float_as_uint(local));
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(PT, 3) k_prep_dy(const uint16_t* __restrict__ dY, const float* __restrict__ s_w, int M, int N,
+                                                   uint32_t* __restrict__ amax, int8_t* __restrict__ Aq,
+                                                   int8_t* __restrict__ GqT) {
+  extern __shared__ __align__(16) float psm[];
+  float(*tile)[PLD] = reinterpret_cast<float(*)[PLD]>(psm);
+  float* sw = psm + PT * PLD;
+  const int t = threadIdx.x, n0 = blockIdx.x * PT, m0 = blockIdx.y * PT;
+  uint4 raw[16];
+#pragma unroll
+  for (int it = 0; it < 16; ++it)
+    raw[it] = __ldg(reinterpret_cast<const uint4*>(dY + (size_t)(m0 + it * 8 + (t >> 4)) * N + n0 + (t & 15) * 8));
+  sw[t] = __ldg(s_w + n0 + t);
+#pragma unroll
+  for (int it = 0; it < 16; ++it) {
+    float* d = &tile[it * 8 + (t >> 4)][(t & 15) * 8];
+    const uint4 u = raw[it];
+    d[0] = bflo(u.x); d[1] = bfhi(u.x); d[2] = bflo(u.y); d[3] = bfhi(u.y);
+    d[4] = bflo(u.z); d[5] = bfhi(u.z); d[6] = bflo(u.w); d[7] = bfhi(u.w);
+  }
+  __syncthreads();
+  float invA = 0.0f, invG = 0.0f;
+  if (PASS == 1) {
+    const float a = __uint_as_float(amax[0]), g = __uint_as_float(amax[1]);
+    invA = (a > 0.0f) ? fdiv(127.0f, a) : 0.0f;
+    invG = (g > 0.0f) ? fdiv(127.0f, g) : 0.0f;
+  }
+  float2 v[64];
+  // row t of the tile, scaled by the weight steps (scalar multiplies: the products are rounded before any add)
+#pragma unroll
+  for (int p = 0; p < 64; ++p) v[p] = make_float2(fmul(tile[t][2 * p], sw[2 * p]), fmul(tile[t][2 * p + 1], sw[2 * p + 1]));
+  wht128_pairs(v);
+  if (PASS == 0) amax_publish(absmax128(v), amax + 0);
+  else quant_store128(v, invA, Aq + (size_t)(m0 + t) * N + n0);
+  // column t of the tile, transposed output
+#pragma unroll
+  for (int p = 0; p < 64; ++p) v[p] = make_float2(tile[2 * p][t], tile[2 * p + 1][t]);
+  wht128_pairs(v);
+  if (PASS == 0) amax_publish(absmax128(v), amax + 1);
+  else quant_store128(v, invG, GqT + (size_t)(n0 + t) * M + m0);
+}
+
 __global__ void k_su_finish(const uint32_t* amax, int rotated, float* s_u) {
   if (!rotated) { s_u[0] = 1.0f; return; }
   const int am = (int)amax[0];
@@ -383,11 +477,16 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   const unsigned g1 = (unsigned)((ngrp + 7) / 8);
   dim3 gG(N / 128, M / 128), gZ(K / 128, M / 128);
   if (rot) {
-    k_rot_rows<0, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
-    k_rotc<true, 0, true><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, nullptr);
+    static bool cfg = false;
+    if (!cfg) {
+      if (cudaFuncSetAttribute(k_prep_dy<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+          cudaFuncSetAttribute(k_prep_dy<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess)
+        return DET_ERR_CUDA;
+      cfg = true;
+    }
+    k_prep_dy<0><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, nullptr, nullptr);
     k_rotc<false, 0, true><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, nullptr);
-    k_rot_rows<1, true><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
-    k_rotc<true, 1, true><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, GqT);
+    k_prep_dy<1><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, Aq, GqT);
     k_rotc<false, 1, true><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, ZqT);
   } else {
     k_rot_rows<0, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
