@@ -303,6 +303,26 @@ def embed_bwd(tok, dy, V):
     return dE
 
 
+def linear_bwd_rows(dY, X, W, s_x, s_w, rows_m, rows_n, hb=128):
+    """Rows rows_m of dX and rows rows_n of dW of linear_bwd (same bits), without the full contractions."""
+    dY = _c(dY, np.uint16)
+    X = _c(X, np.uint16)
+    W = _c(W, np.uint16)
+    s_x = _c(s_x, np.float32).reshape(1)
+    s_w = _c(s_w, np.float32)
+    rows_m = _c(rows_m, np.int32)
+    rows_n = _c(rows_n, np.int32)
+    M, K = X.shape
+    N = W.shape[0]
+    if hb:
+        assert M % 128 == 0 and N % 128 == 0
+    dX = np.empty((rows_m.size, K), np.uint16)
+    dW = np.empty((rows_n.size, K), np.float32)
+    lib().orc_linear_bwd_rows(_p(dY), _p(X), _p(W), C.c_int(M), C.c_int(N), C.c_int(K), _p(s_x), _p(s_w), C.c_int(hb),
+                              _p(rows_m), C.c_int(rows_m.size), _p(rows_n), C.c_int(rows_n.size), _p(dX), _p(dW))
+    return dX, dW
+
+
 def lmhead_fwd(Hh, W):
     Hh = _c(Hh, np.uint16)
     W = _c(W, np.uint16)

@@ -165,6 +165,84 @@ static void absmax_quant_f(const float *v, size_t n, int8_t *q, float *s) {
  * Outputs: dX bf16 [M,K], dW f32 [N,K], ds_x f32 scalar.
  * Optional (nullable) debug outputs: Aq [M,N], UqT [K,N], GqT [N,M], ZqT [K,M],
  * scales[4] = {s_a, s_u, s_g, s_z}. */
+/* integer operand after the rotation: exact int32 values -> int8 with s = absmax/127 (rotation on), or the values
+ * themselves with s = 1 (rotation off) */
+static void int_operand_quant(const int32_t *U, size_t n, int hb, int8_t *q, float *s) {
+  if (hb) {
+    int32_t am = 0;
+    for (size_t i = 0; i < n; ++i) { int32_t v = U[i] < 0 ? -U[i] : U[i]; if (v > am) am = v; }
+    float inv = 0.0f; *s = 0.0f;
+    if (am > 0) { *s = fdiv(i2f(am), 127.0f); inv = fdiv(127.0f, i2f(am)); }
+    for (size_t i = 0; i < n; ++i) {
+      float t = fmin2(fmax2(fmul(i2f(U[i]), inv), -128.0f), 127.0f);
+      q[i] = (int8_t)(int)frne(t);
+    }
+  } else {
+    *s = 1.0f;
+    for (size_t i = 0; i < n; ++i) q[i] = (int8_t)U[i];
+  }
+}
+
+/* operands of the input-gradient GEMM: Aq [M,N] = quant(rotate_n(dY * s_w)), UqT [K,N] = quant(rotate_n(qW)^T) */
+static void bwd_operands_x(const bf16_t *dY, const int8_t *qW, int M, int N, int K, const float *s_w, int hb,
+                           int8_t *Aq, int8_t *UqT, float *s_a, float *s_u) {
+  size_t MN = (size_t)M * N, NK = (size_t)N * K;
+  float *a = (float *)malloc(MN * sizeof(float));
+#pragma omp parallel for
+  for (int m = 0; m < M; ++m) {
+    for (int n = 0; n < N; ++n) a[(size_t)m * N + n] = fmul(bf2f(dY[(size_t)m * N + n]), s_w[n]);
+    if (hb) for (int n0 = 0; n0 < N; n0 += 128) wht128_f(a + (size_t)m * N + n0);
+  }
+  absmax_quant_f(a, MN, Aq, s_a);
+  free(a);
+  /* U = H * qW along n (exact integers), stored transposed [K,N] */
+  int32_t *U = (int32_t *)malloc(NK * sizeof(int32_t));
+#pragma omp parallel for
+  for (int k = 0; k < K; ++k) {
+    for (int n = 0; n < N; ++n) U[(size_t)k * N + n] = qW[(size_t)n * K + k];
+    if (hb) for (int n0 = 0; n0 < N; n0 += 128) wht128_i(U + (size_t)k * N + n0);
+  }
+  int_operand_quant(U, NK, hb, UqT, s_u);
+  free(U);
+}
+
+/* operands of the weight-gradient GEMM: GqT [N,M] = quant(rotate_m(dY)^T), ZqT [K,M] = quant(rotate_m(qX)^T) */
+static void bwd_operands_w(const bf16_t *dY, const int8_t *qX, int M, int N, int K, int hb, int8_t *GqT, int8_t *ZqT,
+                           float *s_g, float *s_z) {
+  size_t MN = (size_t)M * N, MK = (size_t)M * K;
+  float *GT = (float *)malloc(MN * sizeof(float)); /* [N,M] */
+#pragma omp parallel for
+  for (int n = 0; n < N; ++n) {
+    for (int m = 0; m < M; ++m) GT[(size_t)n * M + m] = bf2f(dY[(size_t)m * N + n]);
+    if (hb) for (int m0 = 0; m0 < M; m0 += 128) wht128_f(GT + (size_t)n * M + m0);
+  }
+  absmax_quant_f(GT, MN, GqT, s_g);
+  free(GT);
+  int32_t *Z = (int32_t *)malloc(MK * sizeof(int32_t)); /* [K,M] */
+#pragma omp parallel for
+  for (int k = 0; k < K; ++k) {
+    for (int m = 0; m < M; ++m) Z[(size_t)k * M + m] = qX[(size_t)m * K + k];
+    if (hb) for (int m0 = 0; m0 < M; m0 += 128) wht128_i(Z + (size_t)k * M + m0);
+  }
+  int_operand_quant(Z, MK, hb, ZqT, s_z);
+  free(Z);
+}
+
+/* dX element and its LSQ step-gradient term from the integer accumulator */
+static inline float dx_epilogue(int32_t acc, float cx, float x, float inv_sx, int8_t qx, bf16_t *dx) {
+  float gx = fmul(i2f(acc), cx);
+  float t = fmul(x, inv_sx);
+  int in_range = (t >= -128.0f) && (t <= 127.0f);
+  *dx = f2bf(in_range ? gx : 0.0f);
+  float phi = t < -128.0f ? -128.0f : (t > 127.0f ? 127.0f : fsub(i2f((int32_t)qx), t));
+  return fmul(gx, phi);
+}
+static inline float dw_epilogue(int32_t acc, float cw, float w, float inv_sw) {
+  float t = fmul(w, inv_sw);
+  int in_range = (t >= -128.0f) && (t <= 127.0f);
+  return in_range ? fmul(i2f(acc), cw) : 0.0f;
+}
+
 void orc_linear_bwd(const bf16_t *dY, const bf16_t *X, const bf16_t *W, int M, int N, int K,
                     const float *s_x, const float *s_w, int hb, bf16_t *dX, float *dW, float *ds_x,
                     int8_t *Aq_out, int8_t *UqT_out, int8_t *GqT_out, int8_t *ZqT_out, float *scales) {
@@ -176,83 +254,23 @@ void orc_linear_bwd(const bf16_t *dY, const bf16_t *X, const bf16_t *W, int M, i
   float s_a, s_u, s_g, s_z;
 
   /* ---- grad wrt x: contraction over n ---- */
-  float *a = (float *)malloc(MN * sizeof(float));
-#pragma omp parallel for
-  for (int m = 0; m < M; ++m) {
-    for (int n = 0; n < N; ++n) a[(size_t)m * N + n] = fmul(bf2f(dY[(size_t)m * N + n]), s_w[n]);
-    if (hb) for (int n0 = 0; n0 < N; n0 += 128) wht128_f(a + (size_t)m * N + n0);
-  }
-  int8_t *Aq = (int8_t *)malloc(MN);
-  absmax_quant_f(a, MN, Aq, &s_a);
-  /* U = H * qW along n (exact integers), stored transposed [K,N] */
-  int32_t *U = (int32_t *)malloc(NK * sizeof(int32_t));
-#pragma omp parallel for
-  for (int k = 0; k < K; ++k) {
-    for (int n = 0; n < N; ++n) U[(size_t)k * N + n] = qW[(size_t)n * K + k];
-    if (hb) for (int n0 = 0; n0 < N; n0 += 128) wht128_i(U + (size_t)k * N + n0);
-  }
-  int8_t *UqT = (int8_t *)malloc(NK);
-  if (hb) {
-    int32_t am = 0;
-    for (size_t i = 0; i < NK; ++i) { int32_t v = U[i] < 0 ? -U[i] : U[i]; if (v > am) am = v; }
-    float inv = 0.0f; s_u = 0.0f;
-    if (am > 0) { s_u = fdiv(i2f(am), 127.0f); inv = fdiv(127.0f, i2f(am)); }
-    for (size_t i = 0; i < NK; ++i) {
-      float t = fmin2(fmax2(fmul(i2f(U[i]), inv), -128.0f), 127.0f);
-      UqT[i] = (int8_t)(int)frne(t);
-    }
-  } else {
-    s_u = 1.0f;
-    for (size_t i = 0; i < NK; ++i) UqT[i] = (int8_t)U[i];
-  }
+  int8_t *Aq = (int8_t *)malloc(MN), *UqT = (int8_t *)malloc(NK);
+  bwd_operands_x(dY, qW, M, N, K, s_w, hb, Aq, UqT, &s_a, &s_u);
   int32_t *acc = (int32_t *)malloc(MK * sizeof(int32_t));
   igemm_tn(Aq, UqT, M, K, N, acc);
   float cx = fmul(fmul(s_a, s_u), rot);
   float inv_sx = fdiv(1.0f, *s_x);
   float *terms = (float *)malloc(MK * sizeof(float));
 #pragma omp parallel for
-  for (size_t i = 0; i < MK; ++i) {
-    float gx = fmul(i2f(acc[i]), cx);
-    float t = fmul(bf2f(X[i]), inv_sx);
-    int in_range = (t >= -128.0f) && (t <= 127.0f);
-    dX[i] = f2bf(in_range ? gx : 0.0f);
-    float phi = t < -128.0f ? -128.0f : (t > 127.0f ? 127.0f : fsub(i2f((int32_t)qX[i]), t));
-    terms[i] = fmul(gx, phi);
-  }
+  for (size_t i = 0; i < MK; ++i) terms[i] = dx_epilogue(acc[i], cx, bf2f(X[i]), inv_sx, qX[i], dX + i);
   /* LSQ step-size gradient, scaled by 1/sqrt(M*K*q_max) */
   float gs = (float)(1.0 / sqrt((double)M * (double)K * 127.0));
   *ds_x = fmul(gs, det_sum(terms, MK));
-  free(terms); free(acc); free(U); free(a);
+  free(terms); free(acc);
 
   /* ---- grad wrt W: contraction over tokens m ---- */
-  float *GT = (float *)malloc(MN * sizeof(float)); /* [N,M] */
-#pragma omp parallel for
-  for (int n = 0; n < N; ++n) {
-    for (int m = 0; m < M; ++m) GT[(size_t)n * M + m] = bf2f(dY[(size_t)m * N + n]);
-    if (hb) for (int m0 = 0; m0 < M; m0 += 128) wht128_f(GT + (size_t)n * M + m0);
-  }
-  int8_t *GqT = (int8_t *)malloc(MN);
-  absmax_quant_f(GT, MN, GqT, &s_g);
-  int32_t *Z = (int32_t *)malloc(MK * sizeof(int32_t)); /* [K,M] */
-#pragma omp parallel for
-  for (int k = 0; k < K; ++k) {
-    for (int m = 0; m < M; ++m) Z[(size_t)k * M + m] = qX[(size_t)m * K + k];
-    if (hb) for (int m0 = 0; m0 < M; m0 += 128) wht128_i(Z + (size_t)k * M + m0);
-  }
-  int8_t *ZqT = (int8_t *)malloc(MK);
-  if (hb) {
-    int32_t am = 0;
-    for (size_t i = 0; i < MK; ++i) { int32_t v = Z[i] < 0 ? -Z[i] : Z[i]; if (v > am) am = v; }
-    float inv = 0.0f; s_z = 0.0f;
-    if (am > 0) { s_z = fdiv(i2f(am), 127.0f); inv = fdiv(127.0f, i2f(am)); }
-    for (size_t i = 0; i < MK; ++i) {
-      float t = fmin2(fmax2(fmul(i2f(Z[i]), inv), -128.0f), 127.0f);
-      ZqT[i] = (int8_t)(int)frne(t);
-    }
-  } else {
-    s_z = 1.0f;
-    for (size_t i = 0; i < MK; ++i) ZqT[i] = (int8_t)Z[i];
-  }
+  int8_t *GqT = (int8_t *)malloc(MN), *ZqT = (int8_t *)malloc(MK);
+  bwd_operands_w(dY, qX, M, N, K, hb, GqT, ZqT, &s_g, &s_z);
   int32_t *accw = (int32_t *)malloc(NK * sizeof(int32_t));
   igemm_tn(GqT, ZqT, N, K, M, accw);
   float cw = fmul(fmul(fmul(s_g, s_z), *s_x), rot);
@@ -261,9 +279,7 @@ void orc_linear_bwd(const bf16_t *dY, const bf16_t *X, const bf16_t *W, int M, i
     float inv_sw = fdiv(1.0f, s_w[n]);
     for (int k = 0; k < K; ++k) {
       size_t i = (size_t)n * K + k;
-      float t = fmul(bf2f(W[i]), inv_sw);
-      int in_range = (t >= -128.0f) && (t <= 127.0f);
-      dW[i] = in_range ? fmul(i2f(accw[i]), cw) : 0.0f;
+      dW[i] = dw_epilogue(accw[i], cw, bf2f(W[i]), inv_sw);
     }
   }
   if (Aq_out) memcpy(Aq_out, Aq, MN);
@@ -271,7 +287,48 @@ void orc_linear_bwd(const bf16_t *dY, const bf16_t *X, const bf16_t *W, int M, i
   if (GqT_out) memcpy(GqT_out, GqT, MN);
   if (ZqT_out) memcpy(ZqT_out, ZqT, MK);
   if (scales) { scales[0] = s_a; scales[1] = s_u; scales[2] = s_g; scales[3] = s_z; }
-  free(accw); free(Z); free(ZqT); free(GT); free(GqT); free(Aq); free(UqT); free(qX); free(qW);
+  free(accw); free(ZqT); free(GqT); free(Aq); free(UqT); free(qX); free(qW);
+}
+
+/* The same backward, but only nm rows of dX (token indices rows_m) and nn rows of dW (output channels rows_n) are
+ * evaluated: the operands are prepared in full (their scales are whole-tensor maxima), the two integer contractions
+ * and epilogues only for the selected rows.  For checks at shapes whose full contractions are too slow on a CPU. */
+void orc_linear_bwd_rows(const bf16_t *dY, const bf16_t *X, const bf16_t *W, int M, int N, int K, const float *s_x,
+                         const float *s_w, int hb, const int32_t *rows_m, int nm, const int32_t *rows_n, int nn,
+                         bf16_t *dX_rows, float *dW_rows) {
+  size_t MN = (size_t)M * N, MK = (size_t)M * K, NK = (size_t)N * K;
+  int8_t *qX = (int8_t *)malloc(MK), *qW = (int8_t *)malloc(NK);
+  orc_lsq_quantize(X, M, K, s_x, 0, qX);
+  orc_lsq_quantize(W, N, K, s_w, 1, qW);
+  float rot = hb ? 0x1p-7f : 1.0f;
+  float s_a, s_u, s_g, s_z;
+  int8_t *Aq = (int8_t *)malloc(MN), *UqT = (int8_t *)malloc(NK);
+  bwd_operands_x(dY, qW, M, N, K, s_w, hb, Aq, UqT, &s_a, &s_u);
+  int8_t *Ar = (int8_t *)malloc((size_t)nm * N);
+  for (int i = 0; i < nm; ++i) memcpy(Ar + (size_t)i * N, Aq + (size_t)rows_m[i] * N, N);
+  int32_t *acc = (int32_t *)malloc((size_t)nm * K * sizeof(int32_t));
+  igemm_tn(Ar, UqT, nm, K, N, acc);
+  float cx = fmul(fmul(s_a, s_u), rot);
+  float inv_sx = fdiv(1.0f, *s_x);
+  for (int i = 0; i < nm; ++i)
+    for (int k = 0; k < K; ++k) {
+      size_t src = (size_t)rows_m[i] * K + k;
+      dx_epilogue(acc[(size_t)i * K + k], cx, bf2f(X[src]), inv_sx, qX[src], dX_rows + (size_t)i * K + k);
+    }
+  free(acc); free(Ar); free(Aq); free(UqT);
+  int8_t *GqT = (int8_t *)malloc(MN), *ZqT = (int8_t *)malloc(MK);
+  bwd_operands_w(dY, qX, M, N, K, hb, GqT, ZqT, &s_g, &s_z);
+  int8_t *Gr = (int8_t *)malloc((size_t)nn * M);
+  for (int i = 0; i < nn; ++i) memcpy(Gr + (size_t)i * M, GqT + (size_t)rows_n[i] * M, M);
+  int32_t *accw = (int32_t *)malloc((size_t)nn * K * sizeof(int32_t));
+  igemm_tn(Gr, ZqT, nn, K, M, accw);
+  float cw = fmul(fmul(fmul(s_g, s_z), *s_x), rot);
+  for (int i = 0; i < nn; ++i) {
+    float inv_sw = fdiv(1.0f, s_w[rows_n[i]]);
+    for (int k = 0; k < K; ++k)
+      dW_rows[(size_t)i * K + k] = dw_epilogue(accw[(size_t)i * K + k], cw, bf2f(W[(size_t)rows_n[i] * K + k]), inv_sw);
+  }
+  free(accw); free(Gr); free(GqT); free(ZqT); free(qX); free(qW);
 }
 
 /* ------------------------------------------------------------------ */

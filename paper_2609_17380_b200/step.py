@@ -383,11 +383,13 @@ class Replay:
         det.det_grad_accum_init(st, cfg.mesh[0], cfg.mesh[1], cfg.mesh[2], self.n_grad, self.abufs)
         losses = torch.empty(tokens.shape[0], dtype=F32, device=self.dev)
         for mb in range(tokens.shape[0]):
+            torch.cuda.nvtx.range_push("microbatch%d" % mb)      # lets a profiler select one micro-batch
             self.forward(tokens[mb])
             losses[mb:mb + 1].copy_(self.loss_mean)
             self.backward()
             with self.span("grad_accum"):
                 det.det_grad_accum_push(st, self.gmb)
+            torch.cuda.nvtx.range_pop()
         det.det_grad_accum_result(st, self.gout)
         with self.span("optimizer"):
             self.optimizer()

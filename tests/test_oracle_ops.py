@@ -116,6 +116,19 @@ def test_linear_bwd_against_float64(hb):
     assert np.all(bf(dX).reshape(-1)[:5] == 0)                               # STE range mask
 
 
+def test_linear_bwd_rows_is_a_view_of_the_full_backward():
+    """The row-sampled entry (used for checks at shapes too large for a CPU contraction) gives the bits of the full one."""
+    M, N, K = 256, 384, 256
+    X, W, dY = synth.normal_bf16((M, K), 1.0, seed=0, tid=90), synth.normal_bf16((N, K), 0.02, seed=0, tid=91), \
+        synth.normal_bf16((M, N), 0.01, seed=0, tid=92)
+    sw, sx = oracle.lsq_weight_scale(W), oracle.lsq_act_scale_init(X)
+    for hb in (128, 0):
+        full = oracle.linear_bwd(dY, X, W, sx, sw, hb)
+        rm, rn = np.array([0, 5, 130, 255], np.int32), np.array([1, 100, 383], np.int32)
+        dx, dw = oracle.linear_bwd_rows(dY, X, W, sx, sw, rm, rn, hb)
+        assert np.array_equal(dx, full[0][rm]) and np.array_equal(dw.view(np.uint32), full[1][rn].view(np.uint32))
+
+
 def test_hadamard_modes_agree_when_quantisation_is_exact():
     # one non-zero per 128-block, power-of-two magnitudes: rotated and unrotated operands both quantise exactly
     M = N = K = 128
