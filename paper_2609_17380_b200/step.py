@@ -210,6 +210,21 @@ class Replay:
                     c = min(1 << 26, n - o)
                     dst[o:o + c] = (torch.randn(c, generator=gen, device=self.dev) * 0.02).to(torch.bfloat16).view(I16)
 
+    # ---- state dump: everything a later step depends on (Appendix B: replay from a saved state) ------------------
+    def save_state(self, path):
+        """Parameters (bf16 bits), activation steps, both Adam moments and the step counter, as one .npz file."""
+        np.savez(path, pbf=self.pbf.cpu().numpy(), sx=self.sx.cpu().numpy(), m=self.m.cpu().numpy(), v=self.v.cpu().numpy(),
+                 step=np.array([self.cfg.step], np.int64))
+
+    def load_state(self, path):
+        z = np.load(path)
+        for name, dst in (("pbf", self.pbf), ("sx", self.sx), ("m", self.m), ("v", self.v)):
+            a = z[name]
+            if a.shape != tuple(dst.shape):
+                raise ValueError("state file does not match this configuration: %s %s vs %s" % (name, a.shape, tuple(dst.shape)))
+            dst.copy_(torch.from_numpy(a).to(self.dev))
+        self.cfg.step = int(z["step"][0])
+
     def params_to_host(self):
         out = {}
         for name, shape, kind in self.specs:

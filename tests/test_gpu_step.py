@@ -106,3 +106,37 @@ def test_sharded_replay_class_single_rank():
     assert got["status"] == 0 and got["losses"] == want["losses"]
     bad = [k for k, h in want["hashes"].items() if got["hashes"][k] != h]
     assert not bad, bad
+
+
+def test_two_steps_and_replay_from_a_dump(tmp_path):
+    """Two consecutive optimizer steps match the oracle's two steps; a replay that starts from the state dumped after
+    the first step reproduces the second step's hashes."""
+    import torch
+    from oracle import step as ostep
+    from paper_2609_17380_b200 import step as dstep
+    kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=256, vocab=512, seq=128, micro_batch=1, mesh=(2, 1, 2))
+    cfg = dstep.ModelConfig(**kw)
+    params = synth.model_params(cfg.as_dict(), seed=7)
+    toks = [synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=70 + i) for i in range(2)]
+    # oracle: step 1 (with calibration), then step 2 from its parameters and moments
+    o1 = ostep.run_step(cfg.as_dict(), params, toks[0])
+    c2 = dict(cfg.as_dict(), step=2)
+    o2 = ostep.run_step(c2, o1["params"], toks[1], opt={"m": o1["m"], "v": o1["v"]}, calibrate=False)
+    # device: two steps in one replay
+    r = dstep.Replay(cfg)
+    r.load_params(params)
+    t0, t1 = (torch.from_numpy(np.ascontiguousarray(t, dtype=np.int32)).cuda() for t in toks)
+    r.calibrate(t0[0])
+    g1 = r.step(t0)
+    dump = str(tmp_path / "after_step1.npz")
+    r.cfg.step = 2
+    r.save_state(dump)
+    g2 = r.step(t1)
+    assert not [k for k, h in o1["hashes"].items() if g1["hashes"][k] != h]
+    assert not [k for k, h in o2["hashes"].items() if g2["hashes"][k] != h]
+    # a fresh replay from the dump
+    r2 = dstep.Replay(dstep.ModelConfig(**kw))
+    r2.load_state(dump)
+    assert r2.cfg.step == 2
+    g2b = r2.step(t1)
+    assert g2b["hashes"] == g2["hashes"] and g2b["losses"] == g2["losses"]
