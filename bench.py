@@ -115,7 +115,7 @@ def cpu_baseline(kw):
     cores = os.cpu_count() or 1
     D, Fh, V, L, H = kw["d_model"], kw["ffn"], kw["vocab"], kw["n_layers"], kw["n_heads"]
     # (a) head: 8 tokens (weights drawn with numpy's seeded generator: only the timing is used here)
-    th = 8
+    th = 24
     c = dict(kw)
     c.update(seq=th, micro_batch=1, mesh=(1, 1, 1), n_layers=0)
     rng = np.random.default_rng(0)
@@ -126,8 +126,8 @@ def cpu_baseline(kw):
     t0 = time.time()
     ostep.microbatch_grad(c, P, {}, toks)
     t_head = time.time() - t0
-    # (b) one layer on 128 tokens
-    T = 128
+    # (b) one layer on 256 tokens (two sequences of 128; attention is timed apart because it grows with seq^2)
+    T = 256
     x = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32))
     dy = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32) * 0.01)
     gain = np.full(D, 0x3F80, np.uint16)
@@ -137,7 +137,9 @@ def cpu_baseline(kw):
     n1, r1 = O.rmsnorm_fwd(x, gain, 1e-6, bf=True)
     s0 = O.lsq_act_scale_init(n1)
     qkv, _, _ = O.linear_fwd(n1, Ws[0], s0, sws[0])
-    att, lse = O.attn_fwd(qkv, 1, H, T)
+    ta = time.time()
+    att, lse = O.attn_fwd(qkv, 2, H, 128)
+    t_att_small = time.time() - ta
     s1 = O.lsq_act_scale_init(att)
     o, _, _ = O.linear_fwd(att, Ws[1], s1, sws[1])
     h = O.residual_add(x, o)
@@ -154,11 +156,21 @@ def cpu_baseline(kw):
     d_h2, _ = O.rmsnorm_bwd(d_n2, h, gain, r2, bf=True)
     d_h = O.residual_add(dy, d_h2)
     d_att, _, _ = O.linear_bwd(d_h, att, Ws[1], s1, sws[1], 128)
-    d_qkv = O.attn_bwd(d_att, qkv, att, lse, 1, H, T)
+    ta = time.time()
+    d_qkv = O.attn_bwd(d_att, qkv, att, lse, 2, H, 128)
+    t_att_small += time.time() - ta
     d_n1, _, _ = O.linear_bwd(d_qkv, n1, Ws[0], s0, sws[0], 128)
     d_x1, _ = O.rmsnorm_bwd(d_n1, x, gain, r1, bf=True)
     O.residual_add(d_h, d_x1)
-    t_layer = time.time() - t0
+    t_layer = time.time() - t0 - t_att_small
+    # (b2) attention forward + backward of 16 heads at seq 512; the cost per sequence grows with seq^2
+    SA = 512
+    qa = synth.to_bf16(rng.standard_normal((SA, 3 * H * 128), dtype=np.float32))
+    da = synth.to_bf16(rng.standard_normal((SA, H * 128), dtype=np.float32) * 0.1)
+    t0 = time.time()
+    oa, la = O.attn_fwd(qa, 1, H, SA)
+    O.attn_bwd(da, qa, oa, la, 1, H, SA)
+    t_attn = time.time() - t0
     # (c) reduction + optimizer + hash on 4M parameters
     n_opt = 1 << 22
     g = rng.standard_normal(n_opt, dtype=np.float32) * np.float32(1e-3)
@@ -175,12 +187,16 @@ def cpu_baseline(kw):
     t_opt = time.time() - t0
     n_params = 2 * V * D + L * (4 * D * D + 3 * D * Fh + 2 * D + 4) + D
     tokens_step = 8 * kw["micro_batch"] * kw["seq"]
-    est = t_head * (tokens_step / th) + L * t_layer * (tokens_step / T) + (t_opt + 7 * t_push) * (n_params / n_opt)
+    n_seq = 8 * kw["micro_batch"]
+    est = t_head * (tokens_step / th) + L * t_layer * (tokens_step / T) + L * t_attn * n_seq * (kw["seq"] / SA) ** 2 + \
+        (t_opt + 7 * t_push) * (n_params / n_opt)
     return {"value": tokens_step / est, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "8 tokens through embed+norm+head+loss fwd/bwd (%.1fs); one full-width layer fwd/bwd on 128 tokens at "
-                      "seq 128 (%.1fs); accumulate+clip+AdamW+hash on 4M params (%.1fs); scaled linearly to %d layers, "
-                      "%d tokens, %.2fB params" % (t_head, t_layer, t_opt, L, tokens_step, n_params / 1e9),
-            "sample_seconds": t_head + t_layer + t_opt, "est_step_seconds": est}
+            "sample": "%d tokens through embed+norm+head+loss fwd/bwd (%.1fs); one full-width layer fwd/bwd without attention on "
+                      "%d tokens (%.1fs); attention fwd/bwd of one 16-head sequence at seq %d (%.1fs); accumulate+clip+AdamW+hash "
+                      "on 4M params (%.1fs); scaled linearly in tokens, layers and parameters and with seq^2 for attention to "
+                      "%d layers, %d tokens at seq %d, %.2fB params"
+                      % (th, t_head, T, t_layer, SA, t_attn, t_opt, L, tokens_step, kw["seq"], n_params / 1e9),
+            "sample_seconds": t_head + t_layer + t_att_small + t_attn + t_opt, "est_step_seconds": est}
 
 
 def run_reference(args):
@@ -333,8 +349,11 @@ def run_ours(args):
     if dom in alg:
         n, tot_ms = prof[dom]
         ach = alg[dom][1] / (tot_ms / n / 1e3) / 1e12
+        # DRAM traffic per launch group from one ncu capture of the same kernels at B = 1 (read + write, summed over the five
+        # backward contractions: 644.8 MB; it grows in proportion to the batch), see profiles/k_ogemm_attn_bwd_small.md
+        traffic = 644.8e6 * B if (dom == "attn_bwd" and args.workload == "config5") else None
         roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
-                     "traffic": None, "peak_source": "148 SMs x 128 FP32 lanes x 2 flop (fused multiply-add) x %.0f MHz"
+                     "traffic": traffic, "peak_source": "148 SMs x 128 FP32 lanes x 2 flop (fused multiply-add) x %.0f MHz"
                      % peaks["sm_max_mhz"]})
     all_alu = {}
     for kname, (bound, work, _) in alg.items():
