@@ -115,7 +115,7 @@ def cpu_baseline(kw):
     cores = os.cpu_count() or 1
     D, Fh, V, L, H = kw["d_model"], kw["ffn"], kw["vocab"], kw["n_layers"], kw["n_heads"]
     # (a) head: 8 tokens (weights drawn with numpy's seeded generator: only the timing is used here)
-    th = 24
+    th = 48
     c = dict(kw)
     c.update(seq=th, micro_batch=1, mesh=(1, 1, 1), n_layers=0)
     rng = np.random.default_rng(0)
@@ -126,8 +126,8 @@ def cpu_baseline(kw):
     t0 = time.time()
     ostep.microbatch_grad(c, P, {}, toks)
     t_head = time.time() - t0
-    # (b) one layer on 256 tokens (two sequences of 128; attention is timed apart because it grows with seq^2)
-    T = 256
+    # (b) one layer on 512 tokens (four sequences of 128; attention is timed apart because it grows with seq^2)
+    T = 512
     x = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32))
     dy = synth.to_bf16(rng.standard_normal((T, D), dtype=np.float32) * 0.01)
     gain = np.full(D, 0x3F80, np.uint16)
@@ -138,7 +138,7 @@ def cpu_baseline(kw):
     s0 = O.lsq_act_scale_init(n1)
     qkv, _, _ = O.linear_fwd(n1, Ws[0], s0, sws[0])
     ta = time.time()
-    att, lse = O.attn_fwd(qkv, 2, H, 128)
+    att, lse = O.attn_fwd(qkv, 4, H, 128)
     t_att_small = time.time() - ta
     s1 = O.lsq_act_scale_init(att)
     o, _, _ = O.linear_fwd(att, Ws[1], s1, sws[1])
@@ -157,14 +157,14 @@ def cpu_baseline(kw):
     d_h = O.residual_add(dy, d_h2)
     d_att, _, _ = O.linear_bwd(d_h, att, Ws[1], s1, sws[1], 128)
     ta = time.time()
-    d_qkv = O.attn_bwd(d_att, qkv, att, lse, 2, H, 128)
+    d_qkv = O.attn_bwd(d_att, qkv, att, lse, 4, H, 128)
     t_att_small += time.time() - ta
     d_n1, _, _ = O.linear_bwd(d_qkv, n1, Ws[0], s0, sws[0], 128)
     d_x1, _ = O.rmsnorm_bwd(d_n1, x, gain, r1, bf=True)
     O.residual_add(d_h, d_x1)
     t_layer = time.time() - t0 - t_att_small
-    # (b2) attention forward + backward of 16 heads at seq 512; the cost per sequence grows with seq^2
-    SA = 512
+    # (b2) attention forward + backward of 16 heads at seq 1024; the cost per sequence grows with seq^2
+    SA = 1024
     qa = synth.to_bf16(rng.standard_normal((SA, 3 * H * 128), dtype=np.float32))
     da = synth.to_bf16(rng.standard_normal((SA, H * 128), dtype=np.float32) * 0.1)
     t0 = time.time()
