@@ -228,9 +228,10 @@ def xent_bwd(logits, target, lse, z_weight=0.0, scale=1.0):
 
 
 # ---- attention ------------------------------------------------------------
-def attn_fwd(qkv, B, H, S, Hkv=None, window=0):
+def attn_fwd(qkv, B, H, S, Hkv=None, window=0, int8_pv=False):
     """qkv: uint16 [B*S, (H + 2*Hkv)*128] (q | k | v column blocks).  Returns out [B*S, H*128], lse [B,H,S].
-    Hkv < H: grouped-query attention; window > 0: sliding-window attention over the last `window` keys."""
+    Hkv < H: grouped-query attention; window > 0: sliding-window attention over the last `window` keys;
+    int8_pv: the P.V product of every block of 128 keys in int8 with per-block scales."""
     qkv = _c(qkv, np.uint16)
     Hkv = H if Hkv is None else Hkv
     ld = qkv.shape[1]
@@ -239,8 +240,9 @@ def attn_fwd(qkv, B, H, S, Hkv=None, window=0):
     out = np.empty((B * S, HD), np.uint16)
     lse = np.empty((B, H, S), np.float32)
     base = qkv.ctypes.data
-    lib().orc_attn_fwd(C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), C.c_int(ld), C.c_int(B),
-                       C.c_int(H), C.c_int(Hkv), C.c_int(S), C.c_int(window), _p(out), C.c_int(HD), _p(lse))
+    fn = lib().orc_attn_fwd_int8pv if int8_pv else lib().orc_attn_fwd
+    fn(C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), C.c_int(ld), C.c_int(B),
+       C.c_int(H), C.c_int(Hkv), C.c_int(S), C.c_int(window), _p(out), C.c_int(HD), _p(lse))
     return out, lse
 
 

@@ -508,6 +508,70 @@ void orc_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, in
     }
 }
 
+/* Forward with the P.V product of every KV block in int8 (Sec. 3.2: "int8 P.V per block; QK^T and softmax in
+ * higher precision").  The paper does not state the scales; this version fixes them as follows.  Per (batch, key/value
+ * head, block of 128 keys): s_v = absmax(V block)/127, q_v = rne(clamp(v * (127/absmax))).  Per row and block:
+ * q_p = rne(p * 127) with p = exp(s - m) in [0,1] (masked slots 0).  u_c = float(sum_j q_p[j] q_v[j,c]) * (s_v/127)
+ * (the integer sum is exact and order-free), then o = o*alpha + u as before.  The row sum l and the logsumexp use
+ * the unquantised p, so lse equals that of orc_attn_fwd; the backward pass is unchanged (it recomputes P in full
+ * precision and does not see the quantisation).  The scale of a block is shared by all rows that touch it. */
+void orc_attn_fwd_int8pv(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ldq, int B, int H, int Hkv, int S, int W,
+                         bf16_t *out, int ld_out, float *lse) {
+  const int G = H / Hkv, NT = (S + KT - 1) / KT;
+  float *sv = (float *)malloc((size_t)B * Hkv * NT * sizeof(float));   /* absmax of every V block */
+#pragma omp parallel for
+  for (int t = 0; t < B * Hkv * NT; ++t) {
+    int b = t / (Hkv * NT), hk = (t / NT) % Hkv, j0 = (t % NT) * KT;
+    float am = 0.0f;
+    for (int j = j0; j < j0 + KT && j < S; ++j)
+      for (int c = 0; c < DH; ++c) am = fmax2(am, fabs1(bf2f(v[(size_t)ldq * (b * S + j) + hk * DH + c])));
+    sv[t] = am;
+  }
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+  for (int bh = 0; bh < B * H; ++bh)
+    for (int i = 0; i < S; ++i) {
+      int b = bh / H, h = bh % H, hk = h / G;
+      const bf16_t *qi = q + (size_t)ldq * (b * S + i) + h * DH;
+      float m = -INFINITY, l = 0.0f, o[DH], s[KT], p[KT];
+      int32_t qp[KT];
+      for (int c = 0; c < DH; ++c) o[c] = 0.0f;
+      for (int j0 = first_tile(i, W); j0 <= i; j0 += KT) {
+        float mt = m;
+        for (int jj = 0; jj < KT; ++jj) {
+          int j = j0 + jj;
+          if (visible(i, j, W)) {
+            s[jj] = fmul(dot128(qi, k + (size_t)ldq * (b * S + j) + hk * DH), ATT_SCALE);
+            mt = fmax2(mt, s[jj]);
+          }
+        }
+        float alpha = det_exp(fsub(m, mt));
+        for (int jj = 0; jj < KT; ++jj) {
+          p[jj] = visible(i, j0 + jj, W) ? det_exp(fsub(s[jj], mt)) : 0.0f;
+          qp[jj] = (int32_t)frne(fmul(p[jj], 127.0f));
+        }
+        float r = tree128(p);
+        l = fadd(fmul(l, alpha), r);
+        float am = sv[((size_t)b * Hkv + hk) * NT + j0 / KT];
+        float s_v = 0.0f, inv_v = 0.0f;
+        if (am > 0.0f) { s_v = fdiv(am, 127.0f); inv_v = fdiv(127.0f, am); }
+        float cs = fdiv(s_v, 127.0f);
+        for (int c = 0; c < DH; ++c) {
+          int32_t acc = 0;
+          for (int jj = 0; jj < KT && j0 + jj <= i; ++jj) {
+            float t = fmin2(fmax2(fmul(bf2f(v[(size_t)ldq * (b * S + j0 + jj) + hk * DH + c]), inv_v), -128.0f), 127.0f);
+            acc += qp[jj] * (int32_t)frne(t);
+          }
+          o[c] = fadd(fmul(o[c], alpha), fmul(i2f(acc), cs));
+        }
+        m = mt;
+      }
+      float il = fdiv(1.0f, l);
+      for (int c = 0; c < DH; ++c) out[(size_t)ld_out * (b * S + i) + h * DH + c] = f2bf(fmul(o[c], il));
+      lse[(size_t)bh * S + i] = fadd(m, det_log(l));
+    }
+  free(sv);
+}
+
 /* backward: p_ij = exp(s_ij - L_i); Delta_i = tree_c(dO*O); dP = dO.v_j;
  * dS = p (dP - Delta) scale; contraction operands rounded to bf16; all three
  * gradient contractions are sequential ascending sums from +0.  With grouped

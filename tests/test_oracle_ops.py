@@ -352,6 +352,46 @@ def test_sliding_window_attention_pins():
     assert np.array_equal(d3[300:, :128], d[300:, :128])                          # dq rows >= 300 unchanged
 
 
+def test_attention_int8_pv_pins():
+    """int8 P.V per block (Sec. 3.2): same logsumexp as the full-precision forward, output within the quantisation
+    error of it and of the float64 softmax, exact where the quantisers are exact, causal at block granularity."""
+    B, H, S = 1, 2, 300
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=93)
+    out_f, lse_f = oracle.attn_fwd(qkv, B, H, S)
+    out_q, lse_q = oracle.attn_fwd(qkv, B, H, S, int8_pv=True)
+    assert np.array_equal(lse_f, lse_q)                                   # statistics are not quantised
+    q, k, v, p, o, _ = _attn_ref(qkv, B, H, S)
+    o = o.transpose(0, 2, 1, 3).reshape(B * S, H * 128)
+    err_q, err_f = np.abs(bf(out_q) - o).max(), np.abs(bf(out_f) - o).max()
+    assert err_q < 0.08 and err_q > err_f                                  # coarser than the f32 path, but close
+    # float64 emulation of the defined formula (quantised p and v, per-block scale): much closer than to the exact softmax
+    x = bf(qkv).astype(np.float64).reshape(S, 3, H, 128)
+    for h in range(H):
+        ref = np.zeros((S, 128))
+        sc = x[:, 0, h] @ x[:, 1, h].T / math.sqrt(128)
+        for i in (0, 1, 127, 128, 200, 299):
+            mrun, orow, l = -np.inf, np.zeros(128), 0.0
+            for j0 in range(0, i + 1, 128):
+                js = np.arange(j0, min(j0 + 128, i + 1))
+                mt = max(mrun, sc[i, js].max())
+                pj = np.exp(sc[i, js] - mt)
+                blk = x[j0:min(j0 + 128, S), 2, h]
+                am = np.abs(blk).max()
+                qv = np.clip(np.rint(x[js, 2, h] * (127.0 / am)), -128, 127)
+                u = (np.rint(pj * 127.0)[:, None] * qv).sum(0) * (am / 127.0 / 127.0)
+                a = np.exp(mrun - mt) if np.isfinite(mrun) else 0.0
+                orow, l, mrun = orow * a + u, l * a + pj.sum(), mt
+            got = bf(out_q)[i, h * 128:(h + 1) * 128]
+            assert np.abs(got - orow / l).max() < 0.02
+    # row 0 sees one key with p = 1: out_0 = v_0 up to the two quantisers' rounding
+    assert np.abs(bf(out_q)[0] - bf(qkv)[0, 2 * H * 128:]).max() < np.abs(bf(qkv)[:128, 2 * H * 128:]).max() / 127 + 1e-2
+    # changing keys/values of later blocks leaves the rows of earlier blocks bit-identical (the block scale is shared
+    # inside a block, so the guarantee is per block of 128 keys)
+    qkv2 = qkv.copy(); qkv2[256:, H * 128:] = synth.normal_bf16((S - 256, 2 * H * 128), 1.0, seed=1, tid=94)
+    out2, _ = oracle.attn_fwd(qkv2, B, H, S, int8_pv=True)
+    assert np.array_equal(out2[:256], out_q[:256]) and not np.array_equal(out2[256:], out_q[256:])
+
+
 # ---------------------------------------------------------------- glue
 def test_glue_ops():
     gu = synth.normal_bf16((9, 512), 2.0, seed=0, tid=70)
