@@ -183,6 +183,14 @@ int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, i
  * rounded to bf16 before P.V.  lse f32 [B,H,S].  S % 64 == 0. */
 int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
                  int window, det_bf16* out, int ld_out, float* lse, void* stream);
+/* The same forward with the P.V product of every block of 128 keys on the int8 tensor cores (Sec. 3.2: "int8 P.V
+ * per block"; the scales are this library's reading): per (batch, key/value head, block) s_v = absmax(V block)/127,
+ * q_v = rne(clamp(v * (127/absmax))); per row and block q_p = rne(p * 127) with p = exp(s - m) in [0,1];
+ * u = float(sum_j q_p q_v) * (s_v/127); logits, statistics, row sums and o = o*alpha + u as in det_attn_fwd, so lse is
+ * identical to det_attn_fwd's and det_attn_bwd applies unchanged.  status_dev (device int, may be NULL) receives
+ * DET_DEV_TIMEOUT if the bounded wait for the tensor-core product expires; the output is then undefined. */
+int det_attn_fwd_int8pv(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                        int window, det_bf16* out, int ld_out, float* lse, void* stream, int* status_dev);
 /* dq (H heads), dk, dv (Hkv heads) with leading dimension ld_d; every contraction is one sequential ascending sum
  * from +0; the gradient of a shared key/value head runs over its query heads in ascending order and, within a
  * head, over the queries in ascending order.  ws (16-byte aligned, det_attn_bwd_ws_bytes) holds P (f32) and

@@ -62,7 +62,7 @@ def forward(cfg, P, sw, tok, calibrate=False):
         if rope is not None:
             qk = O.rope(qk.reshape(B * S, H + Hkv, 128), S, rope[0], rope[1]).reshape(-1, 128)
         a["qkr"] = np.ascontiguousarray(np.concatenate([qk.reshape(B * S, -1), a["qkv"][:, D + 128 * Hkv:]], 1))
-        a["att"], a["lse"] = O.attn_fwd(a["qkr"], B, H, S, Hkv=Hkv, window=_window(cfg, l))
+        a["att"], a["lse"] = O.attn_fwd(a["qkr"], B, H, S, Hkv=Hkv, window=_window(cfg, l), int8_pv=bool(cfg.get("pv_int8")))
         if calibrate:
             sx[1] = O.lsq_act_scale_init(a["att"])[0]
         o, _, _ = O.linear_fwd(a["att"], P["l%d.w_o" % l], sx[1:2], sw["l%d.w_o" % l])

@@ -237,6 +237,12 @@ def det_attn_fwd(q, k, v, ld, B, H, S, out, ld_out, lse, Hkv=None, window=0):
                                                C.c_int(ld_out), _ptr(lse), _stream()))
 
 
+def det_attn_fwd_int8pv(q, k, v, ld, B, H, S, out, ld_out, lse, status_dev=None, Hkv=None, window=0):
+    _check("det_attn_fwd_int8pv", load().det_attn_fwd_int8pv(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H),
+                                                             C.c_int(H if Hkv is None else Hkv), C.c_int(S), C.c_int(window),
+                                                             _ptr(out), C.c_int(ld_out), _ptr(lse), _stream(), _ptr(status_dev)))
+
+
 def det_attn_bwd_ws_bytes(B, H, S, Hkv=None):
     return load().det_attn_bwd_ws_bytes(C.c_int(B), C.c_int(H), C.c_int(H if Hkv is None else Hkv), C.c_int(S))
 

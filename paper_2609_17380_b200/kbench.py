@@ -125,7 +125,7 @@ def case_linear(small, which, bwd):
         2.0 * M * N * K, "op"
 
 
-def case_attn(small, bwd):
+def case_attn(small, bwd, int8pv=False):
     B, H, S = (1, 16, 2048) if small else (4, 16, 2048)
     HD = H * 128
     qkv = randn_bf16(B * S * 3 * HD)
@@ -133,6 +133,9 @@ def case_attn(small, bwd):
     p = qkv.data_ptr()
     fwd = lambda: det.det_attn_fwd(p, p + 2 * HD, p + 4 * HD, 3 * HD, B, H, S, out, HD, lse)
     unit = B * H * (S * S // 2) * 128 * 2.0
+    if int8pv:   # same nominal work as the full-precision forward (one of the two contractions runs on the tensor cores)
+        st = torch.zeros(1, dtype=I32, device="cuda")
+        return (lambda: det.det_attn_fwd_int8pv(p, p + 2 * HD, p + 4 * HD, 3 * HD, B, H, S, out, HD, lse, st)), 2 * unit, "flop"
     if not bwd:
         return fwd, 2 * unit, "flop"
     fwd()
@@ -185,6 +188,7 @@ def build_cases():
     c = {"sumsq": case_sumsq, "rmsnorm_fwd": lambda s: case_rmsnorm(s, False), "rmsnorm_bwd": lambda s: case_rmsnorm(s, True),
          "xent_fwd": lambda s: case_xent(s, False), "xent_bwd": lambda s: case_xent(s, True),
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
+         "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
          "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_bwd": lambda s: case_lmhead(s, True),
          "accum": case_accum, "adamw": case_adamw, "hash": case_hash}
     for k in LINEAR_SHAPES:

@@ -41,6 +41,7 @@ class ModelConfig:
     embed_norm: bool = False         # RMSNorm (with gain) on the embedding output
     window: int = 0                  # sliding-window width of the local layers (multiple of 128), 0 = all layers full
     full_every: int = 5              # every full_every-th layer and the last one attend to the whole prefix
+    pv_int8: bool = False            # forward P.V of every block of 128 keys on the int8 tensor cores
 
     def as_dict(self):
         return dict(self.__dict__)
@@ -279,8 +280,12 @@ class Replay:
                     det.det_rope(src, QW, T, H + Hkv, S, self.rope_cos, self.rope_sin, 0, a["qkr"], QW)
                 qp = a["qkr"].data_ptr()
             with self.span("attn_fwd"):
-                det.det_attn_fwd(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"], Hkv=Hkv,
-                                 window=cfg.layer_window(l))
+                if cfg.pv_int8:
+                    det.det_attn_fwd_int8pv(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"],
+                                            self.status, Hkv=Hkv, window=cfg.layer_window(l))
+                else:
+                    det.det_attn_fwd(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"], Hkv=Hkv,
+                                     window=cfg.layer_window(l))
             o = self.tmp[1][:T * D]
             self._linear(l, "w_o", 1, a["att"], T, o, a["qx_o"], calibrate)
             det.det_residual_add(a["x"], o, T * D, a["h"])

@@ -483,6 +483,26 @@ def test_attention_grouped_and_windowed(det, B, H, Hkv, S, W):
         assert_same_bits(got[:, lo:hi], want[:, lo:hi], name)
 
 
+@pytest.mark.parametrize("B,H,Hkv,S,W", [(1, 1, 1, 128, 0), (1, 2, 2, 320, 0), (2, 4, 2, 256, 0), (1, 2, 1, 512, 128)])
+def test_attention_forward_int8_pv(det, B, H, Hkv, S, W):
+    """P.V of every block on the int8 tensor cores: output and logsumexp bit for bit against the oracle's definition."""
+    import torch
+    HD, KD = H * 128, Hkv * 128
+    ld = HD + 2 * KD
+    qkv = synth.normal_bf16((B * S, ld), 1.0, seed=16, tid=1)
+    qkv[5, HD + KD:] = 0                                         # a zero value row
+    dq = dev(qkv)
+    base = dq.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_attn_fwd_int8pv(base, base + 2 * HD, base + 2 * (HD + KD), ld, B, H, S, out, HD, lse, status, Hkv=Hkv, window=W)
+    _sync()
+    assert int(status.item()) == 0
+    oout, olse = oracle.attn_fwd(qkv, B, H, S, Hkv=Hkv, window=W, int8_pv=True)
+    assert_same_bits(host(lse), olse, "lse")
+    assert_same_bits(host(out, np.uint16), oout, "out")
+
+
 # ------------------------------------------------------------------ slabs whose products can underflow
 def _sprinkle_tiny(a, seed, frac=0.002):
     """Overwrite a fraction of a bf16 tensor with magnitudes around 2^-64 .. 2^-62 (random signs)."""

@@ -32,6 +32,9 @@ def _run(cfg_kwargs, seed=0):
          qk_norm=True, rope=True, embed_norm=True, window=128, z_weight=1e-4),
     dict(n_layers=1, d_model=256, n_heads=2, n_kv_heads=2, ffn=256, vocab=256, seq=128, micro_batch=2, mesh=(1, 1, 1),
          qk_norm=True, rope=True),
+    # forward P.V on the int8 tensor cores (the backward recomputes the weights in full precision)
+    dict(n_layers=2, d_model=256, n_heads=2, n_kv_heads=1, ffn=256, vocab=256, seq=256, micro_batch=1, mesh=(2, 1, 1),
+         pv_int8=True, window=128),
 ])
 def test_step_hashes_match_oracle(kw):
     cfg, got, want = _run(kw)
