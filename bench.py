@@ -246,7 +246,7 @@ def run_ours(args):
     sharded = world > 1 and n_mb % world == 0
     if sharded:
         from paper_2609_17380_b200.dist import ShardedReplay
-        rep = ShardedReplay(cfg, rank, world)
+        rep = ShardedReplay(cfg, rank, world, peer_fold=args.peer_fold)
         r = rep.r
     else:
         rep = r = dstep.Replay(cfg)
@@ -402,6 +402,9 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--peer-fold", action="store_true",
+                    help="N > 1: fold the gradient slices straight out of the peers' buffers (symmetric memory) instead of "
+                         "exchanging them with point-to-point copies first")
     ap.add_argument("--workload", choices=("config5", "paper"), default="config5",
                     help="config5 (default) is the benchmark configuration; paper is the paper's own block and shapes")
     ap.add_argument("--steps", type=int, default=3)

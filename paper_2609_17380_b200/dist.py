@@ -106,6 +106,70 @@ class ShardedReducer:
         return out_padded[:p.n]
 
 
+class PeerReducer:
+    """The same exchange without staging copies: every rank keeps the gradients of its micro-batches in a buffer that its
+    peers can address (symmetric memory over NVLink / NVSwitch), and the fold reads slice `rank` of every micro-batch
+    straight out of the owners' buffers, so the accumulate kernel itself moves the data (plain peer loads, no multicast)
+    and the arithmetic order is untouched.  Two barriers per step delimit the window in which peers read a buffer.
+
+    `peer_view(owner, j, lo, hi)` returns what `fold` consumes for micro-batch j of rank `owner`, elements [lo, hi):
+    a device address on GPUs, a tensor view in the CPU tests.  `barrier()` is a process-group barrier ordered with the
+    device work of every rank."""
+
+    def __init__(self, plan, rank, stash, peer_view, barrier, group=None):
+        self.plan, self.rank, self.group = plan, rank, group
+        self.stash_buf, self.peer_view, self.barrier = stash, peer_view, barrier
+        lo, hi = plan.bounds(rank)
+        self.len = hi - lo
+
+    def wait(self):
+        pass
+
+    def scatter(self, j, grad):
+        """Keep the j-th local micro-batch gradient where the peers can read it."""
+        self.stash_buf[j].copy_(grad)
+
+    def fold_and_gather(self, fold, out_padded):
+        p = self.plan
+        lo, hi = p.bounds(self.rank)
+        self.barrier()                       # every rank's gradients are complete
+        mine = out_padded[self.rank * p.chunk:(self.rank + 1) * p.chunk]
+        if self.len:
+            fold([self.peer_view(m // p.per_rank, m % p.per_rank, lo, hi) for m in range(p.M)], mine[:self.len])
+        if self.len < p.chunk:
+            mine[self.len:].zero_()
+        self.barrier()                       # nobody reads a peer's buffer past this point
+        if p.W > 1:
+            if dist.get_backend(self.group) == "nccl":
+                dist.all_gather_into_tensor(out_padded, mine, group=self.group)
+            else:
+                views = [out_padded[c * p.chunk:(c + 1) * p.chunk] for c in range(p.W)]
+                dist.all_gather(views, mine.clone(), group=self.group)
+        return out_padded[:p.n]
+
+
+def make_peer_reducer(plan, rank, device, group=None):
+    """GPU construction of a PeerReducer on torch's symmetric memory (one allocation of per_rank x n floats per rank)."""
+    import torch.distributed._symmetric_memory as symm_mem
+    n = plan.n
+    flat = symm_mem.empty(plan.per_rank * n, dtype=torch.float32, device=device)
+    hdl = symm_mem.rendezvous(flat, group if group is not None else dist.group.WORLD)
+    ptrs = [int(x) for x in hdl.buffer_ptrs]
+    stash = flat.view(plan.per_rank, n)
+
+    def peer_view(owner, j, lo, hi):
+        return ptrs[owner] + 4 * (j * n + lo)
+
+    def barrier():
+        # an NCCL collective on the compute stream: it starts on a rank only after that rank's earlier kernels, and
+        # completes only when every rank has started it
+        dist.barrier(group=group)
+
+    red = PeerReducer(plan, rank, stash, peer_view, barrier, group)
+    red._keepalive = (flat, hdl)
+    return red
+
+
 def fold_slices(det, mesh, pool, slices, out):
     """The single-device push sequence (Algorithm 1 + TreeFold) on one slice: `slices` are the M micro-batch slices in
     mesh order, `pool` the accumulation buffers (det_grad_accum_nbufs x len(out) floats), `out` the reduced slice."""
@@ -121,7 +185,9 @@ class ShardedReplay:
     pool is sized for this rank's slice only; parameters, moments and the reduced gradient are replicated, so the
     state hashes of all ranks are equal to each other and to those of the single-device replay."""
 
-    def __init__(self, cfg, rank, world, group=None, device="cuda"):
+    def __init__(self, cfg, rank, world, group=None, device="cuda", peer_fold=False):
+        """peer_fold: fold straight out of the peers' gradient buffers (symmetric memory, plain peer loads inside the
+        accumulate kernel) instead of exchanging slices with point-to-point copies first."""
         import paper_2609_17380_b200 as det
         from .step import Replay, param_specs, _numel
         n_grad = sum(_numel(sh) for _, sh, _ in param_specs(cfg))
@@ -129,9 +195,14 @@ class ShardedReplay:
         self.plan = ShardPlan(cfg.n_microbatches, world, n_grad)
         self.rank, self.world, self.group = rank, world, group
         self.r = Replay(cfg, device, accum_len=self.plan.chunk, gout_len=self.plan.padded)
-        self.red = ShardedReducer(self.plan, rank, device, group)
-        # the fresh gradient is copied here so that the next backward pass can overwrite gmb while it travels
-        self.stage = torch.empty(n_grad, dtype=torch.float32, device=device)
+        self.peer_fold = bool(peer_fold) and world > 1
+        if self.peer_fold:
+            self.red = make_peer_reducer(self.plan, rank, device, group)
+            self.stage = None
+        else:
+            self.red = ShardedReducer(self.plan, rank, device, group)
+            # the fresh gradient is copied here so that the next backward pass can overwrite gmb while it travels
+            self.stage = torch.empty(n_grad, dtype=torch.float32, device=device)
 
     def _fold(self, slices, out):
         fold_slices(self.det, self.r.cfg.mesh, self.r.abufs, slices, out)
@@ -150,9 +221,12 @@ class ShardedReplay:
             losses[m:m + 1].copy_(r.loss_mean)
             r.backward()
             with r.span("grad_exchange"):
-                self.red.wait()
-                self.stage.copy_(r.gmb)
-                self.red.scatter(j, self.stage)
+                if self.peer_fold:
+                    self.red.scatter(j, r.gmb)
+                else:
+                    self.red.wait()
+                    self.stage.copy_(r.gmb)
+                    self.red.scatter(j, self.stage)
         with r.span("grad_accum"):
             self.red.fold_and_gather(self._fold, r.gout_padded)
         with r.span("optimizer"):

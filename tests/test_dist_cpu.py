@@ -11,7 +11,7 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 import oracle
-from paper_2609_17380_b200.dist import ShardPlan, ShardedReducer
+from paper_2609_17380_b200.dist import PeerReducer, ShardPlan, ShardedReducer
 
 
 def _grad(m, n):
@@ -52,6 +52,41 @@ def _worker(rank, world, port, mesh, n, outdir):
         np.save(os.path.join(outdir, "rank%d.npy" % rank), got)
     finally:
         dist.destroy_process_group()
+
+
+def _peer_worker(rank, world, port, mesh, n, outdir, stashes):
+    """The peer-memory variant: `stashes` are shared-memory tensors standing in for the ranks' symmetric buffers."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        M = mesh[0] * mesh[1] * mesh[2]
+        plan = ShardPlan(M, world, n)
+        red = PeerReducer(plan, rank, stashes[rank], lambda owner, j, lo, hi: stashes[owner][j, lo:hi], dist.barrier)
+        for j, m in enumerate(plan.local_microbatches(rank)):
+            red.scatter(j, torch.from_numpy(_grad(m, n)))
+
+        def fold(slices, out):
+            acc = oracle.Accum(mesh[0], mesh[1], mesh[2], out.numel())
+            for s in slices:
+                acc.push(s.numpy())
+            out.copy_(torch.from_numpy(acc.result()))
+
+        out = torch.full((plan.padded,), float("nan"))
+        np.save(os.path.join(outdir, "rank%d.npy" % rank), red.fold_and_gather(fold, out).numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,mesh,n", [(2, (2, 2, 2), 1000), (4, (2, 2, 2), 300), (3, (1, 2, 3), 5000)])
+def test_peer_fold_equals_single_process(tmp_path, world, mesh, n):
+    M = mesh[0] * mesh[1] * mesh[2]
+    stashes = [torch.zeros((M // world, n), dtype=torch.float32).share_memory_() for _ in range(world)]
+    mp.spawn(_peer_worker, args=(world, _free_port(), mesh, n, str(tmp_path), stashes), nprocs=world, join=True)
+    want = _single(mesh, n)
+    for r in range(world):
+        got = np.load(tmp_path / ("rank%d.npy" % r))
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), "rank %d differs" % r
 
 
 def _free_port():
