@@ -131,6 +131,11 @@ int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, cons
  * are multiples of 256; mode 1 forces the one-CTA kernel.  Results are identical (integer accumulation is exact).
  * Process-wide, not thread-safe. */
 int det_igemm_set_mode(int mode);
+/* Self-test of the bounded wait used by every kernel that waits on an mbarrier (TMA loads, tensor-core commits): one
+ * warp waits on a barrier that nothing completes; after limit_cycles SM clocks (at most 4e9) the wait gives up, ORs
+ * DET_DEV_TIMEOUT into *status_dev (device int) and the kernel returns, leaving the context usable.  No counterpart in
+ * the paper: it exists so that the time-out path can be exercised without making a real kernel hang. */
+int det_selftest_wait_timeout(int* status_dev, long long limit_cycles, void* stream);
 int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream, int* status_dev);
 
 /* ---- RMSNorm (Sec. 3.1 "RMSNorm", FP32 internals) -------------------------------------------------

@@ -15,6 +15,7 @@ _SO = os.path.join(_DIR, "libdet.so")
 
 DET_OK = 0
 DET_F32, DET_BF16 = 0, 1
+DET_DEV_TARGET, DET_DEV_TIMEOUT, DET_DEV_NONFINITE = 1, 2, 4   # bits of a device status word
 DEV_TARGET, DEV_TIMEOUT, DEV_NONFINITE = 1, 2, 4
 STATUS_NAMES = {0: "DET_OK", -1: "DET_ERR_ARG", -2: "DET_ERR_SHAPE", -3: "DET_ERR_ALIGN", -4: "DET_ERR_WORKSPACE",
                 -5: "DET_ERR_RANGE", -6: "DET_ERR_CUDA"}
@@ -174,6 +175,10 @@ def det_linear_bwd(dY, X, qX, W, qWt_bwd, s_x, s_w, s_u, M, N, K, hadamard_block
     _check("det_linear_bwd", load().det_linear_bwd(
         _ptr(dY), _ptr(X), _ptr(qX), _ptr(W), _ptr(qWt_bwd), _ptr(s_x), _ptr(s_w), _ptr(s_u), C.c_int(M), C.c_int(N),
         C.c_int(K), C.c_int(hadamard_block), _ptr(dX), _ptr(dW), _ptr(ds_x), *_ws(ws), _stream(), _ptr(status_dev)))
+
+
+def det_selftest_wait_timeout(status_dev, limit_cycles):
+    _check("det_selftest_wait_timeout", load().det_selftest_wait_timeout(_ptr(status_dev), C.c_longlong(limit_cycles), _stream()))
 
 
 def det_igemm_set_mode(mode):

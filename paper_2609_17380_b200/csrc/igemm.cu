@@ -550,6 +550,27 @@ int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K,
 
 using namespace det;
 
+// Self-test of the bounded wait every tensor-core kernel relies on: one warp waits on an mbarrier that nothing ever
+// completes; after `limit_cycles` the wait gives up, raises DET_DEV_TIMEOUT in *status_dev and the kernel returns.
+__global__ void k_selftest_wait(int* status, long long limit) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_s;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  mbar_wait(&bar, 0, &abort_s, status, limit);
+}
+
+extern "C" int det_selftest_wait_timeout(int* status_dev, long long limit_cycles, void* stream) {
+  if (!status_dev || limit_cycles <= 0 || limit_cycles > 4000000000ll) return DET_ERR_ARG;
+  k_selftest_wait<<<DET_L(1), 32, 0, (cudaStream_t)stream>>>(status_dev, limit_cycles);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
 extern "C" int det_igemm_set_mode(int mode) {
   if (mode != 0 && mode != 1) return DET_ERR_ARG;
   igemm_set_mode(mode);

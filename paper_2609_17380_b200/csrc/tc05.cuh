@@ -34,7 +34,8 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // bounded wait; returns false when the limit expired or another role already gave up
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit = WAIT_LIMIT_CYCLES) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   int polls = 0;
@@ -42,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try(bar, parity)) return true;
     if ((++polls & 63) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         or_status(status, DET_DEV_TIMEOUT);
         return false;

@@ -562,3 +562,18 @@ def test_attention_subnormal_products(det):
                      db + 4 * HD, 3 * HD, ws(det.det_attn_bwd_ws_bytes(B, H, S)))
     _sync()
     assert_same_bits(host(dqkv, np.uint16), oracle.attn_bwd(dout, qkv, oout, olse, B, H, S), "dqkv")
+
+
+def test_bounded_wait_times_out_and_context_survives(det):
+    """A wait on a barrier that nothing completes gives up after its limit, reports DET_DEV_TIMEOUT through the status
+    word and returns; the next launches run normally."""
+    import torch
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_selftest_wait_timeout(status, 2000000)              # about a millisecond
+    _sync()
+    assert int(status.item()) == det.DET_DEV_TIMEOUT
+    x = np.arange(1000, dtype=F)
+    out = empty((1,), F)
+    det.det_sum(dev(x), 1000, 0, out, ws(det.det_sum_ws_bytes(1000)))
+    _sync()
+    assert_same_bits(host(out), np.array([oracle.det_sum(x)], F), "sum after a timed-out wait")
