@@ -295,4 +295,220 @@ static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   return DET_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Warp-specialised variant for the long contractions of the LM head: 128 x 256 tile, eight consumer warps that only
+// multiply (8 x 16 register tiles fed from shared memory) and four producer warps that only stage (global loads,
+// unpacking, the below-2^-63 test, shared-memory stores) into a three-slab ring.  Producers and consumers meet at named
+// barriers (one "full" and one "empty" barrier per ring slot), so the multiply pipe never waits for staging
+// instructions of its own warp.  Plain contraction only (no batching, ranges or epilogues).
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int WS_STAGES = 3, WS_CONS = 256, WS_PROD = 128, WS_THREADS = WS_CONS + WS_PROD, WS_TN = 256;
+constexpr size_t WS_SMEM = (size_t)WS_STAGES * OK * ((OT + 4) + (WS_TN + 4)) * sizeof(float);
+
+__device__ __forceinline__ void nbar_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(WS_THREADS) : "memory"); }
+__device__ __forceinline__ void nbar_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(WS_THREADS) : "memory"); }
+
+// One producer thread's share of a slab of ROWS rows x 16 contraction steps, as raw words.
+//   CONTIG : rows pt + 128*g (g < ROWS/128), all 16 contraction indices (two 16-byte words of bf16, four of f32, per row)
+//   STRIDED: four consecutive rows 4f .. 4f+3 (f = pt mod ROWS/4) at the contraction indices kk + KPP*i, kk = pt / (ROWS/4),
+//            KPP = 512/ROWS, i < 16/KPP: consecutive lanes read and store consecutive words, so the shared-memory stores
+//            are free of bank conflicts
+template <int MODE, bool F32IN, int ROWS>
+struct WsRaw {
+  static constexpr int NW = MODE == CONTIG ? (ROWS / 128) * 2 * (F32IN ? 2 : 1) : (16 * ROWS / 512) / (F32IN ? 1 : 2);
+  uint4 w[NW];   // STRIDED bf16: two passes share one 16-byte register group (8 bytes each)
+};
+template <int MODE, bool F32IN, int ROWS>
+__device__ __forceinline__ void ws_fetch(const void* base, int rows, int C, int ld, int r0, int c0, int pt,
+                                         WsRaw<MODE, F32IN, ROWS>& raw) {
+  constexpr int ESZ = F32IN ? 4 : 2;
+  const char* b = reinterpret_cast<const char*>(base);
+  if (MODE == CONTIG) {
+    constexpr int EPW = F32IN ? 4 : 8;    // elements per 16-byte word
+    constexpr int WPR = 16 / EPW;        // words per row
+#pragma unroll
+    for (int g = 0; g < ROWS / 128; ++g) {
+      const int r = r0 + pt + 128 * g;
+#pragma unroll
+      for (int w = 0; w < WPR; ++w) {
+        const int c = c0 + w * EPW;
+        raw.w[g * WPR + w] = (r < rows && c < C) ? __ldg(reinterpret_cast<const uint4*>(b + ((size_t)r * ld + c) * ESZ))
+                                                 : make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+  } else {
+    constexpr int F4 = ROWS / 4, KPP = 128 / F4, NP = 16 / KPP;
+    const int f = pt % F4, kk = pt / F4;
+    const int r = r0 + 4 * f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      const int c = c0 + kk + KPP * i;
+      const bool ok = c < C && r < rows;
+      const char* src = b + ((size_t)c * ld + r) * ESZ;
+      if (F32IN) {
+        raw.w[i] = ok ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0u, 0u, 0u, 0u);
+      } else {
+        const uint2 u = ok ? __ldg(reinterpret_cast<const uint2*>(src)) : make_uint2(0u, 0u);
+        if (i & 1) { raw.w[i >> 1].z = u.x; raw.w[i >> 1].w = u.y; }
+        else { raw.w[i >> 1].x = u.x; raw.w[i >> 1].y = u.y; }
+      }
+    }
+  }
+}
+template <bool F32IN>
+__device__ __forceinline__ void ws_unpack_word(const uint4& u, float* v) {   // 8 (bf16) or 4 (f32, rounded to bf16) values
+  if (F32IN) {
+    v[0] = bf2f(f2bf(__uint_as_float(u.x))); v[1] = bf2f(f2bf(__uint_as_float(u.y)));
+    v[2] = bf2f(f2bf(__uint_as_float(u.z))); v[3] = bf2f(f2bf(__uint_as_float(u.w)));
+  } else {
+    v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
+    v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
+  }
+}
+// unpack, test and store one thread's share; returns the below-2^-63 flag of its values
+template <int MODE, bool F32IN, int ROWS>
+__device__ __forceinline__ bool ws_store(float (*s)[ROWS + 4], int pt, const WsRaw<MODE, F32IN, ROWS>& raw) {
+  bool tiny = false;
+  if (MODE == CONTIG) {
+    constexpr int EPW = F32IN ? 4 : 8;
+    constexpr int WPR = 16 / EPW;
+#pragma unroll
+    for (int g = 0; g < ROWS / 128; ++g)
+#pragma unroll
+      for (int w = 0; w < WPR; ++w) {
+        float v[8];
+        ws_unpack_word<F32IN>(raw.w[g * WPR + w], v);
+#pragma unroll
+        for (int e = 0; e < EPW; ++e) {
+          tiny |= (__float_as_uint(v[e]) * 2u - 1u) < 0x3fffffffu;
+          s[w * EPW + e][pt + 128 * g] = v[e];
+        }
+      }
+  } else {
+    constexpr int F4 = ROWS / 4, KPP = 128 / F4, NP = 16 / KPP;
+    const int f = pt % F4, kk = pt / F4;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      float v[4];
+      if (F32IN) {
+        float t[8];
+        ws_unpack_word<true>(raw.w[i], t);
+        v[0] = t[0]; v[1] = t[1]; v[2] = t[2]; v[3] = t[3];
+      } else {
+        const uint32_t lo = (i & 1) ? raw.w[i >> 1].z : raw.w[i >> 1].x, hi = (i & 1) ? raw.w[i >> 1].w : raw.w[i >> 1].y;
+        v[0] = bflo(lo); v[1] = bfhi(lo); v[2] = bflo(hi); v[3] = bfhi(hi);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) tiny |= (__float_as_uint(v[e]) * 2u - 1u) < 0x3fffffffu;
+      *reinterpret_cast<float4*>(&s[kk + KPP * i][4 * f]) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+  }
+  return tiny;
+}
+
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+__global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
+  extern __shared__ __align__(16) unsigned char osm[];
+  float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
+  float(*Bs)[OK][WS_TN + 4] = reinterpret_cast<float(*)[OK][WS_TN + 4]>(osm + (size_t)WS_STAGES * OK * (OT + 4) * sizeof(float));
+  __shared__ int tiny_s[WS_STAGES][WS_PROD / 32];
+  const int i0 = blockIdx.y * OT, j0 = blockIdx.x * WS_TN;
+  const int I = p.I, J = p.J, C = p.C, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
+  const int nslab = (C + OK - 1) / OK;
+  const int tid = threadIdx.x;
+  // barrier ids: 1 + s = slot s is full, 1 + WS_STAGES + s = slot s is empty (id 0 is __syncthreads)
+  if (tid >= WS_CONS) {
+    // ------------------------------- producers -------------------------------
+    // the producer warpgroup hands most of its registers to the two consumer warpgroups
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    const int pt = tid - WS_CONS, pw = pt >> 5;
+    WsRaw<AMODE, AF32, OT> ra;
+    WsRaw<BMODE, false, WS_TN> rb;
+    ws_fetch<AMODE, AF32, OT>(p.A, I, C, lda, i0, 0, pt, ra);
+    ws_fetch<BMODE, false, WS_TN>(p.B, J, C, ldb, j0, 0, pt, rb);
+    for (int s = 0; s < nslab; ++s) {
+      const int slot = s % WS_STAGES;
+      if (s >= WS_STAGES) nbar_sync(1 + WS_STAGES + slot);          // the consumers have left this slot
+      bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
+      tiny |= ws_store<BMODE, false, WS_TN>(Bs[slot], pt, rb);
+      if (s + 1 < nslab) {                                           // next slab's words travel during the handshake
+        ws_fetch<AMODE, AF32, OT>(p.A, I, C, lda, i0, (s + 1) * OK, pt, ra);
+        ws_fetch<BMODE, false, WS_TN>(p.B, J, C, ldb, j0, (s + 1) * OK, pt, rb);
+      }
+      const int any = __any_sync(0xffffffffu, tiny);
+      if ((pt & 31) == 0) tiny_s[slot][pw] = any;
+      nbar_arrive(1 + slot);                                         // slot is full (orders the stores above)
+    }
+    // every "empty" barrier the consumers still arrive at needs its partner: drain them
+    for (int s = nslab; s < nslab + WS_STAGES; ++s)
+      if (s >= WS_STAGES) nbar_sync(1 + WS_STAGES + (s % WS_STAGES));
+    return;
+  }
+  // --------------------------------- consumers ---------------------------------
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  const int ty = tid >> 4, tx = tid & 15;
+  float2 acc[8][WS_TN / 32];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < WS_TN / 32; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
+  float* outf = reinterpret_cast<float*>(p.out);
+  if (p.init && !OUT_BF16) {
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+      for (int g = 0; g < WS_TN / 64; ++g) {
+        const int c = j0 + g * 64 + tx * 4;
+        if (r < I && c < J) {
+          const float4 t = *reinterpret_cast<const float4*>(outf + (size_t)r * ldo + c);
+          acc[a][2 * g] = make_float2(t.x, t.y);
+          acc[a][2 * g + 1] = make_float2(t.z, t.w);
+        }
+      }
+    }
+  }
+  for (int s = 0; s < nslab; ++s) {
+    const int slot = s % WS_STAGES;
+    nbar_sync(1 + slot);                                             // slot is full
+    const int tiny = tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
+    if (tiny) slab_mac<false, WS_TN>(As[slot], Bs[slot], ty, tx, acc);
+    else slab_mac<true, WS_TN>(As[slot], Bs[slot], ty, tx, acc);
+    nbar_arrive(1 + WS_STAGES + slot);                               // slot may be refilled
+  }
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+    for (int g = 0; g < WS_TN / 64; ++g) {
+      const int c = j0 + g * 64 + tx * 4;
+      if (r < I && c < J) {
+        const float2 lo = acc[a][2 * g], hi = acc[a][2 * g + 1];
+        if (OUT_BF16) {
+          uint2 u;
+          u.x = pack_bf2(lo.x, lo.y);
+          u.y = pack_bf2(hi.x, hi.y);
+          *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out) + (size_t)r * ldo + c) = u;
+        } else {
+          *reinterpret_cast<float4*>(outf + (size_t)r * ldo + c) = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+      }
+    }
+  }
+}
+
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+static int ogemm_ws_launch(const OgemmArgs& p, cudaStream_t st) {
+  static bool cfg = false;
+  if (!cfg) {
+    if (cudaFuncSetAttribute(k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)WS_SMEM) != cudaSuccess)
+      return DET_ERR_CUDA;
+    cfg = true;
+  }
+  dim3 grid((p.J + WS_TN - 1) / WS_TN, (p.I + OT - 1) / OT, 1);
+  k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WS_THREADS, WS_SMEM, st>>>(p);
+  return DET_OK;
+}
+
 }  // namespace det
