@@ -179,12 +179,17 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
   float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
-  // blocks are handed out in linear order; with a causal range the longest contractions are put first
-  const int i0 = (p.range_mode == 2 ? (gridDim.y - 1 - blockIdx.y) : blockIdx.y) * OT, j0 = blockIdx.x * TN;
+  // Blocks are handed out in linear order.  With a causal range (modes 1, 2) the row tile sits on the slowest grid index
+  // and runs from the longest contraction to the shortest, so that the blocks still running at the end of the grid are
+  // the short ones of every batch entry; otherwise the batch index is the slowest.
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
+  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
+  const int i0 = ti * OT, j0 = blockIdx.x * TN;
   const int W = p.window;
   if (p.range_mode == 3 && (j0 > i0 || (W && i0 >= j0 + W + OT))) return;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-  const long long zb = blockIdx.z / p.H, zh = blockIdx.z % p.H;
+  const long long zb = zidx / p.H, zh = zidx % p.H;
   const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
   const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
                        : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
@@ -251,7 +256,7 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   for (int a = 0; a < 8; ++a) {
     const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
     float rv = 0.0f;
-    if (EPI != OEPI_NONE && r < I) rv = p.rowv[(size_t)blockIdx.z * I + r];
+    if (EPI != OEPI_NONE && r < I) rv = p.rowv[(size_t)zidx * I + r];
 #pragma unroll
     for (int g = 0; g < TN / 64; ++g) {
       const int c = j0 + g * 64 + tx * 4;
@@ -290,7 +295,9 @@ static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
       return DET_ERR_CUDA;
     cfg = true;
   }
-  dim3 grid((p.J + TN - 1) / TN, (p.I + OT - 1) / OT, batches);
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
+  dim3 grid((p.J + TN - 1) / TN, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
   k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN, EPI><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
   return DET_OK;
 }
