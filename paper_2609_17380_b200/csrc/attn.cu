@@ -337,8 +337,13 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   rc = ogemm_launch<CONTIG, CONTIG, false, true, 128, OEPI_DS>(e, B * H, st);
   if (rc != DET_OK) return rc;
   // dV[j,c] = sum over the query heads g of the group, then over queries i >= j ascending, of P~[i,j] dO[i,c];
-  // dK[j,c] likewise with dS~ and q.  One accumulator per output: with G > 1 it travels through `carry` in f32.
+  // dK[j,c] likewise with dS~ and q.  One accumulator per output: with G > 1 it travels through `carry` in f32, and
+  // the two chains then share that scratch and run one after the other.  dV, dK (for G == 1) and dQ are independent of
+  // each other and run side by side on auxiliary streams, so that the short blocks at the end of one grid overlap
+  // with the long blocks at the start of the next.
+  AuxStreams* aux = aux_fork(st);
   for (int which = 0; which < 2; ++which) {
+    cudaStream_t sk = (aux && G == 1 && which == 1) ? aux->s[0] : st;
     for (int g = 0; g < G; ++g) {
       OgemmArgs p = {};
       p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = Hkv; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
@@ -350,12 +355,12 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
       if (g > 0) { p.acc_in = carry; p.acc_ld = DH; p.acc_b = (long long)Hkv * S * DH; p.acc_h = (long long)S * DH; }
       if (g == G - 1) {
         p.out = which == 0 ? dv : dk; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
-        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * Hkv, st)     // P is rounded to bf16 as read
-                        : ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * Hkv, st);
+        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * Hkv, sk)     // P is rounded to bf16 as read
+                        : ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * Hkv, sk);
       } else {
         p.out = carry; p.ldo = DH; p.o_b = (long long)Hkv * S * DH; p.o_h = (long long)S * DH;
-        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, false, 128>(p, B * Hkv, st)
-                        : ogemm_launch<STRIDED, STRIDED, false, false, 128>(p, B * Hkv, st);
+        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, false, 128>(p, B * Hkv, sk)
+                        : ogemm_launch<STRIDED, STRIDED, false, false, 128>(p, B * Hkv, sk);
       }
       if (rc != DET_OK) return rc;
     }
@@ -365,8 +370,9 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
   p.A = dSt; p.B = k; p.ldb = ld; p.b_b = (long long)S * ld; p.b_h = DH; p.b_div = G;
   p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
-  rc = ogemm_launch<CONTIG, STRIDED, false, true, 128>(p, B * H, st);
+  rc = ogemm_launch<CONTIG, STRIDED, false, true, 128>(p, B * H, aux ? aux->s[1] : st);
   if (rc != DET_OK) return rc;
+  if (!aux_join(st, aux)) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -27,6 +27,18 @@ struct EpiParams {
   float* ds_partial;      // DX: [I, J/128] partial sums of dXhat * phi
 };
 
+// Independent kernels of one call may run side by side so that the partial last wave of one grid is filled by blocks of
+// another.  aux_fork makes up to two auxiliary streams of the current device start where `st` stands now; aux_join makes
+// `st` wait for them, so the caller still sees plain stream order.  Returns NULL / false when the streams cannot be
+// had (the caller then launches everything on `st`).
+struct AuxStreams {
+  cudaStream_t s[2];
+  cudaEvent_t fork, join[2];
+  bool ok;
+};
+AuxStreams* aux_fork(cudaStream_t st);
+bool aux_join(cudaStream_t st, AuxStreams* a);
+
 // C[i,j] = sum_k A[i,k] B[j,k] on the tensor cores with the chosen epilogue; host-side checks included
 int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
                  cudaStream_t st);

@@ -10,39 +10,13 @@
 // once and give the same bits, unless the product is subnormal (the unfused product is then flushed to zero,
 // the fused one is not).  Each slab is therefore checked for factors below 2^-63 while it is staged; clean
 // slabs use the fused instruction, the others the two-instruction sequence.
-#include <mutex>
-
 #include "ogemm_core.cuh"
 
 using namespace det;
 
 // The two gradient contractions of the LM head are independent; the input-gradient grid (512 blocks on 148 SMs at
 // the benchmark shape) ends in a partial wave, so the weight-gradient kernel runs beside it on an auxiliary stream
-// and fills the idle SMs.  The caller still sees plain stream order: the auxiliary stream starts after everything
-// queued on the caller's stream and the caller's stream waits for it before anything queued later.
-namespace {
-struct AuxStream {
-  cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
-  bool ok = false;
-};
-AuxStream* aux_for_current_device() {
-  static std::mutex mu;
-  static AuxStream table[64];
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  std::lock_guard<std::mutex> lock(mu);
-  AuxStream& a = table[dev];
-  if (!a.ok) {
-    if (cudaStreamCreateWithFlags(&a.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    a.ok = true;
-  }
-  return &a;
-}
-}  // namespace
-
+// and fills the idle SMs (aux_fork / aux_join keep plain stream order for the caller).
 static OgemmArgs plain_args(const void* A, const void* B, void* out, int I, int J, int C, int lda, int ldb, int ldo, int init) {
   OgemmArgs p = {};
   p.A = A; p.B = B; p.out = out; p.I = I; p.J = J; p.C = C; p.lda = lda; p.ldb = ldb; p.ldo = ldo; p.init = init; p.H = 1;
@@ -65,22 +39,15 @@ extern "C" int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det
   if (K % 16 || V % 16 || M % 8) return DET_ERR_SHAPE;
   if (!aligned16(dlogits) || !aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW)) return DET_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
-  // the auxiliary stream starts where the caller's stream stands now
-  AuxStream* aux = aux_for_current_device();
-  cudaStream_t sw = st;
-  if (aux) {
-    if (cudaEventRecord(aux->fork, st) != cudaSuccess || cudaStreamWaitEvent(aux->stream, aux->fork, 0) != cudaSuccess) return DET_ERR_CUDA;
-    sw = aux->stream;
-  }
+  AuxStreams* aux = aux_fork(st);   // the auxiliary stream starts where the caller's stream stands now
   // dH[m,k] = sum over v ascending of bf16(dlogits[m,v]) * W[v,k]
   int rc = ogemm_ws_launch<CONTIG, STRIDED, true, true>(plain_args(dlogits, W, dH, M, K, V, V, K, K, 0), st);
   if (rc != DET_OK) return rc;
   // dW[v,k] (+)= sum over m ascending of bf16(dlogits[m,v]) * H[m,k], beside the first kernel
-  rc = ogemm_ws_launch<STRIDED, STRIDED, true, false>(plain_args(dlogits, H, dW, V, K, M, V, K, K, first_chunk ? 0 : 1), sw);
+  rc = ogemm_ws_launch<STRIDED, STRIDED, true, false>(plain_args(dlogits, H, dW, V, K, M, V, K, K, first_chunk ? 0 : 1),
+                                                      aux ? aux->s[0] : st);
   if (rc != DET_OK) return rc;
-  if (aux) {
-    if (cudaEventRecord(aux->join, aux->stream) != cudaSuccess || cudaStreamWaitEvent(st, aux->join, 0) != cudaSuccess) return DET_ERR_CUDA;
-  }
+  if (!aux_join(st, aux)) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

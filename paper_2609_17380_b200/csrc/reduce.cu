@@ -5,6 +5,8 @@
 // a warp butterfly finishes the 256-element leaf, eight leaf sums are paired in registers, and the
 // eight warp sums in shared memory.  The chunk sums are reduced by the same kernel until one value
 // is left, so the tree depends on n only.
+#include <mutex>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -12,6 +14,35 @@ namespace det {
 
 static unsigned long long g_launches = 0;
 int note_launch() { ++g_launches; return 0; }
+
+AuxStreams* aux_fork(cudaStream_t st) {
+  static std::mutex mu;
+  static AuxStreams table[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  AuxStreams* a = &table[dev];
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!a->ok) {
+      for (int i = 0; i < 2; ++i) {
+        if (cudaStreamCreateWithFlags(&a->s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&a->join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      }
+      if (cudaEventCreateWithFlags(&a->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      a->ok = true;
+    }
+  }
+  if (cudaEventRecord(a->fork, st) != cudaSuccess) return nullptr;
+  for (int i = 0; i < 2; ++i)
+    if (cudaStreamWaitEvent(a->s[i], a->fork, 0) != cudaSuccess) return nullptr;
+  return a;
+}
+bool aux_join(cudaStream_t st, AuxStreams* a) {
+  if (!a) return true;
+  for (int i = 0; i < 2; ++i)
+    if (cudaEventRecord(a->join[i], a->s[i]) != cudaSuccess || cudaStreamWaitEvent(st, a->join[i], 0) != cudaSuccess) return false;
+  return true;
+}
 unsigned long long launches() { return g_launches; }
 
 constexpr int SUM_CHUNK = 16384;
