@@ -59,6 +59,9 @@ class ShardedReducer:
         # (rows are a whole chunk apart, so every row starts 16-byte aligned)
         self.recv = torch.empty((plan.M, plan.chunk), dtype=dtype, device=device)
         self.pending = []
+        # a process group that cannot move device memory (gloo) gets the slices through host copies
+        self.host_stage = torch.device(device).type == "cuda" and dist.is_initialized() and dist.get_backend(group) != "nccl"
+        self.landing = []       # (host tensor, device destination) pairs of receives in flight
 
     def scatter(self, j, grad):
         """Send the slices of the j-th local micro-batch gradient (flat tensor of n elements) to their finishers and post
@@ -74,9 +77,15 @@ class ShardedReducer:
                 continue
             clo, chi = p.bounds(c)
             if chi > clo:
-                ops.append(dist.P2POp(dist.isend, grad[clo:chi], c, group=self.group))
+                src = grad[clo:chi].cpu() if self.host_stage else grad[clo:chi]
+                ops.append(dist.P2POp(dist.isend, src, c, group=self.group))
             if hi > lo:
-                ops.append(dist.P2POp(dist.irecv, self.recv[c * p.per_rank + j, :hi - lo], c, group=self.group))
+                dst = self.recv[c * p.per_rank + j, :hi - lo]
+                if self.host_stage:
+                    land = torch.empty(hi - lo, dtype=dst.dtype)
+                    self.landing.append((land, dst))
+                    dst = land
+                ops.append(dist.P2POp(dist.irecv, dst, c, group=self.group))
         if ops:
             self.pending += dist.batch_isend_irecv(ops)
 
@@ -84,6 +93,23 @@ class ShardedReducer:
         for w in self.pending:
             w.wait()
         self.pending = []
+        for land, dst in self.landing:
+            dst.copy_(land)
+        self.landing = []
+
+    def _gather(self, out_padded, mine):
+        p = self.plan
+        if dist.get_backend(self.group) == "nccl":
+            # in place: this rank's slice already sits at its position of the output
+            dist.all_gather_into_tensor(out_padded, mine, group=self.group)
+        elif out_padded.is_cuda:
+            host = [torch.empty(p.chunk, dtype=mine.dtype) for _ in range(p.W)]
+            dist.all_gather(host, mine.cpu(), group=self.group)
+            for c in range(p.W):
+                out_padded[c * p.chunk:(c + 1) * p.chunk].copy_(host[c])
+        else:
+            views = [out_padded[c * p.chunk:(c + 1) * p.chunk] for c in range(p.W)]
+            dist.all_gather(views, mine.clone(), group=self.group)
 
     def fold_and_gather(self, fold, out_padded):
         """fold(list of M slice tensors in mesh order, out) writes the reduced slice (self.len elements) into out.  The
@@ -97,12 +123,7 @@ class ShardedReducer:
         if self.len < p.chunk:
             mine[self.len:].zero_()
         if p.W > 1:
-            if dist.get_backend(self.group) == "nccl":
-                # in place: this rank's slice already sits at its position of the output
-                dist.all_gather_into_tensor(out_padded, mine, group=self.group)
-            else:
-                views = [out_padded[c * p.chunk:(c + 1) * p.chunk] for c in range(p.W)]
-                dist.all_gather(views, mine.clone(), group=self.group)
+            self._gather(out_padded, mine)
         return out_padded[:p.n]
 
 
@@ -235,8 +256,13 @@ class ShardedReplay:
             h = r.hashes(per_tensor_hashes)
         res = {"hashes": h, "status": int(r.status.item())}
         if want_losses:
-            if self.world > 1:
-                dist.all_reduce(losses, group=self.group)   # every entry is non-zero on exactly one rank
+            if self.world > 1:   # every entry is non-zero on exactly one rank
+                if dist.get_backend(self.group) == "nccl":
+                    dist.all_reduce(losses, group=self.group)
+                else:
+                    host = losses.cpu()
+                    dist.all_reduce(host, group=self.group)
+                    losses = host
             ls = losses.cpu().numpy()
             res.update(losses=[float(x) for x in ls], grad_norm=float(r.norm.item()), coef=float(r.coef.item()))
         return res

@@ -143,3 +143,50 @@ def test_two_steps_and_replay_from_a_dump(tmp_path):
     assert r2.cfg.step == 2
     g2b = r2.step(t1)
     assert g2b["hashes"] == g2["hashes"] and g2b["losses"] == g2["losses"]
+
+
+def _sharded_worker(rank, world, port, kw, outdir):
+    """One rank of the sharded replay; both ranks share the one GPU (their kernels never wait on each other, only the
+    host blocks in the process group), gloo carries the CUDA tensors."""
+    import os
+    import torch
+    import torch.distributed as dist
+    from paper_2609_17380_b200 import step as dstep
+    from paper_2609_17380_b200.dist import ShardedReplay
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        torch.cuda.set_device(0)
+        cfg = dstep.ModelConfig(**kw)
+        params = synth.model_params(cfg.as_dict(), seed=9)
+        tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=9)
+        rep = ShardedReplay(cfg, rank, world)
+        rep.r.load_params(params)
+        tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).cuda()
+        rep.calibrate(tok[0])
+        out = rep.step(tok)
+        with open(os.path.join(outdir, "rank%d.txt" % rank), "w") as f:
+            f.write(repr((out["hashes"], out["losses"], out["status"])))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sharded_replay_two_ranks_on_one_gpu(tmp_path):
+    """The whole ShardedReplay step on two ranks (point-to-point slice exchange, fold, gather, replicated optimizer):
+    both ranks end with the single-replay hashes."""
+    import socket
+    import torch.multiprocessing as mp
+    from paper_2609_17380_b200 import step as dstep
+    kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=512, seq=128, micro_batch=1, mesh=(2, 2, 2))
+    cfg = dstep.ModelConfig(**kw)
+    want = dstep.run_step(cfg, synth.model_params(cfg.as_dict(), seed=9), synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=9))
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    mp.spawn(_sharded_worker, args=(2, port, kw, str(tmp_path)), nprocs=2, join=True)
+    for rank in range(2):
+        hashes, losses, status = eval(open(tmp_path / ("rank%d.txt" % rank)).read())
+        assert status == 0 and losses == want["losses"]
+        assert not [k for k, h in want["hashes"].items() if hashes[k] != h], "rank %d" % rank
