@@ -190,3 +190,57 @@ def test_sharded_replay_two_ranks_on_one_gpu(tmp_path):
         hashes, losses, status = eval(open(tmp_path / ("rank%d.txt" % rank)).read())
         assert status == 0 and losses == want["losses"]
         assert not [k for k, h in want["hashes"].items() if hashes[k] != h], "rank %d" % rank
+
+
+def _peer_worker_gpu(rank, world, port, outdir):
+    """Symmetric-memory construction of the peer-fold reducer with a one-rank NCCL group: the stash is allocated and
+    rendezvoused through torch's symmetric memory and the fold reads it through the raw addresses it reports."""
+    import os
+    import torch
+    import torch.distributed as dist
+    import paper_2609_17380_b200 as det
+    from paper_2609_17380_b200.dist import ShardPlan, fold_slices, make_peer_reducer
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", 0))
+    try:
+        mesh, n = (2, 2, 2), 100000
+        plan = ShardPlan(8, 1, n)
+        red = make_peer_reducer(plan, 0, "cuda")
+        g = [torch.from_numpy(np.random.default_rng(50 + m).standard_normal(n).astype(np.float32)).cuda() for m in range(8)]
+        for j in range(8):
+            red.scatter(j, g[j])
+        pool = torch.empty(det.det_grad_accum_nbufs(2) * plan.chunk, dtype=torch.float32, device="cuda")
+        out = torch.zeros(plan.padded, dtype=torch.float32, device="cuda")
+        got = red.fold_and_gather(lambda sl, o: fold_slices(det, mesh, pool, sl, o), out).cpu().numpy()
+        st = det.det_accum()
+        bufs = torch.empty(det.det_grad_accum_nbufs(2) * n, dtype=torch.float32, device="cuda")
+        det.det_grad_accum_init(st, 2, 2, 2, n, bufs)
+        for j in range(8):
+            det.det_grad_accum_push(st, g[j])
+        want = torch.empty(n, dtype=torch.float32, device="cuda")
+        det.det_grad_accum_result(st, want)
+        same = np.array_equal(got.view(np.uint32), want.cpu().numpy().view(np.uint32))
+        # the NCCL in-place all-gather of the slice exchange accepts a slice of its own output (one rank: a no-op copy)
+        from paper_2609_17380_b200.dist import ShardedReducer
+        sr = ShardedReducer(plan, 0, "cuda")
+        before = out.clone()
+        sr._gather(out, out[:plan.chunk])
+        torch.cuda.synchronize()
+        same = same and bool((out == before).all().item()) and not sr.host_stage
+        with open(os.path.join(outdir, "ok.txt"), "w") as f:
+            f.write("1" if same else "0")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_peer_fold_symmetric_memory_one_rank(tmp_path):
+    import socket
+    import torch.multiprocessing as mp
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    mp.spawn(_peer_worker_gpu, args=(1, port, str(tmp_path)), nprocs=1, join=True)
+    assert open(tmp_path / "ok.txt").read() == "1"
