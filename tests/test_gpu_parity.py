@@ -412,6 +412,48 @@ def test_linear_backward(det, M, N, K, hb, mode):
     det.det_igemm_set_mode(0)
 
 
+@pytest.mark.parametrize("case", ["zero_grad", "zero_weight", "zero_input", "heavy_tail", "saturated_input"])
+def test_linear_backward_degenerate(det, case):
+    """Degenerate operands of the LSQ linear: all-zero tensors (absmax 0 -> scale 0, codes 0), a gradient with a few
+    huge entries (everything else quantises to 0 without the rotation's spreading), activations far outside the
+    quantiser's range (straight-through mask zeroes their gradient)."""
+    import torch
+    M, N, K = 256, 256, 256
+    X, W, dY = _linear_case(M, N, K, 13)
+    if case == "zero_grad":
+        dY[:] = 0
+    if case == "zero_weight":
+        W[:] = 0
+    if case == "zero_input":
+        X[:] = 0
+    if case == "heavy_tail":
+        dY[::37, ::41] = synth.to_bf16(np.array([3.0e4], F))[0]
+    osw = oracle.lsq_weight_scale(W)
+    osx = oracle.lsq_act_scale_init(X)
+    if case == "saturated_input":
+        X[::3, ::5] = synth.to_bf16(np.array([1.0e3], F))[0]      # far beyond 127 steps, after the step was fixed
+    odX, odW, ods, dbg = oracle.linear_bwd(dY, X, W, osx, osw, hb=128, debug=True)
+    dX_, dW_, dY_ = dev(X), dev(W), dev(dY)
+    s_w, s_x = dev(osw), dev(osx)
+    qW, qWt, s_u = empty((N, K), np.int8), empty((K, N), np.int8), empty((1,), F)
+    det.det_lsq_quantize_weight(dW_, s_w, N, K, 128, qW, qWt, s_u, ws(det.det_lsq_quantize_weight_ws_bytes(N, K)))
+    Y, qX = empty((M, N), np.uint16), empty((M, K), np.int8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_linear_fwd(dX_, qW, s_x, s_w, M, N, K, Y, qX, status)
+    oY, _, _ = oracle.linear_fwd(X, W, osx, osw)
+    gX, gW, gs = empty((M, K), np.uint16), empty((N, K), F), empty((1,), F)
+    det.det_linear_bwd(dY_, dX_, qX, dW_, qWt, s_x, s_w, s_u, M, N, K, 128, gX, gW, gs, ws(det.det_linear_bwd_ws_bytes(M, N, K)),
+                       status)
+    _sync()
+    assert int(status.item()) == 0
+    assert_same_bits(host(Y, np.uint16), oY, "Y")
+    assert_same_bits(host(gX, np.uint16), odX, "dX")
+    assert_same_bits(host(gW), odW, "dW")
+    assert_same_bits(host(gs), ods, "ds_x")
+    if case == "zero_grad":
+        assert not host(gX, np.uint16).any() and not host(gW).view(np.uint32).any()
+
+
 # ------------------------------------------------------------------ LM head and attention (ordered FP32)
 @pytest.mark.parametrize("M,V,K", [(128, 256, 256), (72, 1008, 64), (256, 50304 // 8, 128)])
 def test_lmhead(det, M, V, K):
