@@ -619,3 +619,66 @@ def test_bounded_wait_times_out_and_context_survives(det):
     det.det_sum(dev(x), 1000, 0, out, ws(det.det_sum_ws_bytes(1000)))
     _sync()
     assert_same_bits(host(out), np.array([oracle.det_sum(x)], F), "sum after a timed-out wait")
+
+
+def test_extreme_inputs(det):
+    """Saturated softmax, zero rows and non-finite gradients: the degenerate corners of the floating-point ops."""
+    import torch
+    # attention with logits so large that most weights underflow to exactly 0 (flush-to-zero results of det_exp)
+    B, H, S = 1, 1, 256
+    HD = 128
+    qkv = synth.normal_bf16((B * S, 3 * HD), 1.0, seed=17, tid=1)
+    qkv[:, :HD] = synth.to_bf16(synth.from_bf16(qkv[:, :HD]) * F(40.0))          # logits of order +-400
+    qkv[7, :HD] = 0                                                              # one all-zero query: uniform weights
+    dout = synth.normal_bf16((B * S, HD), 0.1, seed=17, tid=2)
+    dq = dev(qkv)
+    base = dq.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    det.det_attn_fwd(base, base + 2 * HD, base + 4 * HD, 3 * HD, B, H, S, out, HD, lse)
+    dqkv = empty((B * S, 3 * HD), np.uint16)
+    db = dqkv.data_ptr()
+    det.det_attn_bwd(dev(dout), base, base + 2 * HD, base + 4 * HD, out, lse, 3 * HD, HD, B, H, S, db, db + 2 * HD, db + 4 * HD,
+                     3 * HD, ws(det.det_attn_bwd_ws_bytes(B, H, S)))
+    _sync()
+    oout, olse = oracle.attn_fwd(qkv, B, H, S)
+    assert_same_bits(host(out, np.uint16), oout, "saturated attention out")
+    assert_same_bits(host(lse), olse, "saturated attention lse")
+    assert_same_bits(host(dqkv, np.uint16), oracle.attn_bwd(dout, qkv, oout, olse, B, H, S), "saturated attention grads")
+    # RMSNorm of an all-zero row: rstd = 1/sqrt(eps), outputs 0
+    x = synth.normal_f32((16, 256), 1.0, seed=18, tid=1)
+    x[3] = 0
+    y, rstd = empty((16, 256), F), empty((16,), F)
+    det.det_rmsnorm_fwd(0, dev(x), None, 16, 256, 1e-6, y, rstd)
+    _sync()
+    oy, orstd = oracle.rmsnorm_fwd(x, None, 1e-6)
+    assert_same_bits(host(y), oy, "rmsnorm zero row")
+    assert_same_bits(host(rstd), orstd, "rstd zero row")
+    assert not host(y)[3].any()
+    # cross-entropy with a dominant logit and with huge negative logits
+    z = synth.normal_f32((6, 1000), 1.0, seed=19, tid=1)
+    z[0, 5] = 1.0e4
+    z[1] = -3.0e4
+    z[2, :] = 0.0
+    tgt = np.array([5, 7, 9, 11, 13, 999], np.int32)
+    loss_row, l2, lm, zm = empty((6,), F), empty((6,), F), empty((1,), F), empty((1,), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_xent_fwd(dev(z), dev(tgt), 6, 1000, 0.0, loss_row, l2, lm, zm, ws(det.det_xent_ws_bytes(6, 1000)), status)
+    _sync()
+    olr, ol2, olm, _, _ = oracle.xent_fwd(z, tgt, 0.0)
+    assert_same_bits(host(loss_row), olr, "xent extreme rows")
+    assert_same_bits(host(lm), olm, "xent mean")
+    assert host(loss_row)[0] == 0.0                                             # dominant logit at the target
+    # gradient norm: all zeros -> norm 0, coefficient 1; a NaN raises the non-finite flag
+    g0 = dev(np.zeros(5000, F))
+    norm, coef = empty((1,), F), empty((1,), F)
+    det.det_grad_norm([g0], 1.0, norm, coef, ws(det.det_grad_norm_ws_bytes([g0])), status)
+    _sync()
+    on, oc = oracle.grad_norm([np.zeros(5000, F)], 1.0)
+    assert_same_bits(host(norm), np.array([on], F), "zero norm")
+    assert_same_bits(host(coef), np.array([oc], F), "zero-norm coefficient")
+    bad = np.zeros(5000, F)
+    bad[123] = np.nan
+    status.zero_()
+    det.det_grad_norm([dev(bad)], 1.0, norm, coef, ws(det.det_grad_norm_ws_bytes([g0])), status)
+    _sync()
+    assert int(status.item()) & det.DET_DEV_NONFINITE
