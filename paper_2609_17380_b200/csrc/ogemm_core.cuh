@@ -2,7 +2,7 @@
 // shared memory as f32, an 8 x (TN/16) register tile per thread, packed two-lane arithmetic, and the per-slab check
 // that decides between the fused and the two-instruction multiply-add (identical bits, see ogemm.cu).
 #pragma once
-#include "common.cuh"
+#include "tc05.cuh"
 #include "internal.h"
 
 namespace det {
@@ -305,15 +305,15 @@ static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
 // ---------------------------------------------------------------------------------------------------------------
 // Warp-specialised variant for the long contractions of the LM head: 128 x 256 tile, eight consumer warps that only
 // multiply (8 x 16 register tiles fed from shared memory) and four producer warps that only stage (global loads,
-// unpacking, the below-2^-63 test, shared-memory stores) into a three-slab ring.  Producers and consumers meet at named
-// barriers (one "full" and one "empty" barrier per ring slot), so the multiply pipe never waits for staging
-// instructions of its own warp.  Plain contraction only (no batching, ranges or epilogues).
+// unpacking, the below-2^-63 test, shared-memory stores) into a three-slab ring.  Each ring slot has a "full" and an
+// "empty" mbarrier: a producer warp arrives on "full" after its stores, a consumer warp arrives on "empty" after its
+// last read, and everybody only waits for the other side, so consumer warps are not coupled to each other and the
+// multiply pipe never waits for staging instructions of its own warp.  All waits are bounded.  Plain contraction only
+// (no batching, ranges or epilogues).
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int WS_STAGES = 3, WS_CONS = 256, WS_PROD = 128, WS_THREADS = WS_CONS + WS_PROD, WS_TN = 256;
 constexpr size_t WS_SMEM = (size_t)WS_STAGES * OK * ((OT + 4) + (WS_TN + 4)) * sizeof(float);
 
-__device__ __forceinline__ void nbar_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(WS_THREADS) : "memory"); }
-__device__ __forceinline__ void nbar_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(WS_THREADS) : "memory"); }
 
 // One producer thread's share of a slab of ROWS rows x 16 contraction steps, as raw words.
 //   CONTIG : rows pt + 128*g (g < ROWS/128), all 16 contraction indices (two 16-byte words of bf16, four of f32, per row)
@@ -419,11 +419,20 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
   float(*Bs)[OK][WS_TN + 4] = reinterpret_cast<float(*)[OK][WS_TN + 4]>(osm + (size_t)WS_STAGES * OK * (OT + 4) * sizeof(float));
   __shared__ int tiny_s[WS_STAGES][WS_PROD / 32];
+  __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
   const int i0 = blockIdx.y * OT, j0 = blockIdx.x * WS_TN;
   const int I = p.I, J = p.J, C = p.C, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
   const int nslab = (C + OK - 1) / OK;
-  const int tid = threadIdx.x;
-  // barrier ids: 1 + s = slot s is full, 1 + WS_STAGES + s = slot s is empty (id 0 is __syncthreads)
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WS_CONS / 32); }
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // use n of a slot (slabs slot, slot + 3, ...) completes phase n of its barriers: the wait parity is n & 1
   if (tid >= WS_CONS) {
     // ------------------------------- producers -------------------------------
     // the producer warpgroup hands most of its registers to the two consumer warpgroups
@@ -435,7 +444,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
     ws_fetch<BMODE, false, WS_TN>(p.B, J, C, ldb, j0, 0, pt, rb);
     for (int s = 0; s < nslab; ++s) {
       const int slot = s % WS_STAGES;
-      if (s >= WS_STAGES) nbar_sync(1 + WS_STAGES + slot);          // the consumers have left this slot
+      if (s >= WS_STAGES &&                                          // the consumers have left this slot
+          !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr))
+        break;
       bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
       tiny |= ws_store<BMODE, false, WS_TN>(Bs[slot], pt, rb);
       if (s + 1 < nslab) {                                           // next slab's words travel during the handshake
@@ -443,12 +454,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
         ws_fetch<BMODE, false, WS_TN>(p.B, J, C, ldb, j0, (s + 1) * OK, pt, rb);
       }
       const int any = __any_sync(0xffffffffu, tiny);
-      if ((pt & 31) == 0) tiny_s[slot][pw] = any;
-      nbar_arrive(1 + slot);                                         // slot is full (orders the stores above)
+      if (lane == 0) tiny_s[slot][pw] = any;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_full[slot]);                   // slot is full (releases the warp's stores)
     }
-    // every "empty" barrier the consumers still arrive at needs its partner: drain them
-    for (int s = nslab; s < nslab + WS_STAGES; ++s)
-      if (s >= WS_STAGES) nbar_sync(1 + WS_STAGES + (s % WS_STAGES));
     return;
   }
   // --------------------------------- consumers ---------------------------------
@@ -477,11 +486,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
   }
   for (int s = 0; s < nslab; ++s) {
     const int slot = s % WS_STAGES;
-    nbar_sync(1 + slot);                                             // slot is full
+    if (!mbar_wait(&bar_full[slot], (uint32_t)((s / WS_STAGES) & 1), abort_flag, nullptr)) break;   // slot is full
     const int tiny = tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
     if (tiny) slab_mac<false, WS_TN>(As[slot], Bs[slot], ty, tx, acc);
     else slab_mac<true, WS_TN>(As[slot], Bs[slot], ty, tx, acc);
-    nbar_arrive(1 + WS_STAGES + slot);                               // slot may be refilled
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_empty[slot]);                    // slot may be refilled
   }
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
