@@ -8,11 +8,15 @@
  *  - returns DET_OK (0) or a negative det_status; errors that the host can see (bad shape, misaligned
  *    pointer, workspace too small) return before anything is launched;
  *  - every tensor pointer is a DEVICE pointer owned by the caller, row-major and contiguous unless a
- *    leading dimension is given; the library allocates nothing, frees nothing and keeps no pointer after
+ *    leading dimension is given; the library allocates no device memory, frees nothing and keeps no pointer after
  *    it returns.  Scratch comes from the caller's `ws` buffer of `ws_bytes` bytes (256-byte aligned),
  *    sized by the matching det_*_ws_bytes() query;
  *  - work is asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream), except
- *    det_tensor_hash which synchronises that stream;
+ *    det_tensor_hash which synchronises that stream.  det_linear_bwd, det_attn_bwd and det_lmhead_bwd run
+ *    independent kernels of the call side by side on two auxiliary streams per device that the library creates
+ *    on first use: they start where `stream` stands when the call is made and `stream` waits for them before
+ *    the call returns, so the caller still sees plain stream order.  The library keeps per-device state for this
+ *    (and for kernel attributes); calls for one device must not be issued from several host threads at once;
  *  - data-dependent scalars (LSQ steps, norms, losses) are device scalars so that no call forces a sync;
  *  - device-detected conditions (bad target index, a bounded wait that expired, a non-finite norm) are
  *    OR-ed into *status_dev (device int, may be NULL) as DET_DEV_* bits; kernels never trap;
