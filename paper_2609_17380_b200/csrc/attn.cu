@@ -267,6 +267,151 @@ __global__ void __launch_bounds__(256) k_attn_delta(const uint16_t* __restrict__
   if (lane == 0) delta[w] = t;
 }
 
+// ---------------------------------------------------------------------------------------------
+// backward, first half: P and dS of one block of 128 queries against every visible block of 128 keys.
+// Warp-specialised like the LM-head kernel: the CTA keeps q^T and dO^T of its query block in shared memory; four
+// producer warps stream the key and value blocks through a three-slot ring of 16-dimension slabs (a "full" and an
+// "empty" mbarrier per slot, bounded waits); eight consumer warps accumulate S = q.k^T and dP = dO.v^T together (two
+// 8 x 8 register tiles per thread, each logit one ascending sum over the 128 dimensions) and, per key block, apply
+// P = exp(S*scale - L) and dS = (P (dP - Delta)) scale and store P (f32) and bf16(dS).  The producers already fetch
+// the next key block while the consumers are in that epilogue, and consumer warps are not coupled to each other.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t SDP_SMEM = (size_t)(2 * DH * (OT + 4) + 2 * WS_STAGES * OK * (OT + 4)) * sizeof(float);
+
+__global__ void __launch_bounds__(WS_THREADS, 1)
+    k_attn_sdp_ws(const uint16_t* __restrict__ dout, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                  const uint16_t* __restrict__ v, const float* __restrict__ lse, const float* __restrict__ delta, int ld,
+                  int ld_out, int H, int Hkv, int S, int W, float* __restrict__ Pf, uint16_t* __restrict__ dSt) {
+  extern __shared__ __align__(16) unsigned char osm[];
+  typedef float(*Full)[OT + 4];
+  Full Qs = reinterpret_cast<Full>(osm);                                            // [dim][query]
+  Full Os = reinterpret_cast<Full>(osm + (size_t)DH * (OT + 4) * sizeof(float));    // [dim][query] of dO
+  float(*Ks)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm + (size_t)2 * DH * (OT + 4) * sizeof(float));
+  float(*Vs)[OK][OT + 4] = Ks + WS_STAGES;
+  __shared__ int tiny_s[WS_STAGES][WS_PROD / 32];
+  __shared__ int tiny_qo, abort_s;
+  __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
+  volatile int* abort_flag = &abort_s;
+  const int it = gridDim.y - 1 - blockIdx.y;        // longest rows first
+  const int h = blockIdx.x % H, b = blockIdx.x / H, hk = h / (H / Hkv);
+  const int i0 = it * OT;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const size_t row0 = (size_t)b * S;
+  const uint16_t* qp = q + row0 * ld + (size_t)h * DH;
+  const uint16_t* op = dout + row0 * ld_out + (size_t)h * DH;
+  const uint16_t* kp = k + row0 * ld + (size_t)hk * DH;
+  const uint16_t* vp = v + row0 * ld + (size_t)hk * DH;
+  const int jt_lo = (W > 0 && i0 > W) ? (i0 - W) / OT : 0;
+  const int ntile = it - jt_lo + 1, nslab = ntile * (DH / OK);
+  if (tid == 0) {
+    for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WS_CONS / 32); }
+    tiny_qo = 0;
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  {  // q^T and dO^T of the query block, staged once by everybody
+    bool tq = false;
+    for (int idx = tid; idx < 2 * OT * 16; idx += WS_THREADS) {
+      const int which = idx >= OT * 16, e = idx - which * OT * 16, r = e & 127, ch = e >> 7;
+      const uint16_t* src = which ? op + (size_t)(i0 + r) * ld_out : qp + (size_t)(i0 + r) * ld;
+      float t[8];
+      if (i0 + r < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(src + ch * 8)), t);
+      else {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) t[x] = 0.0f;
+      }
+      Full dst = which ? Os : Qs;
+#pragma unroll
+      for (int x = 0; x < 8; ++x) { tq |= tiny1(t[x]); dst[ch * 8 + x][r] = t[x]; }
+    }
+    if (__any_sync(0xffffffffu, tq) && lane == 0) atomicOr(&tiny_qo, 1);
+  }
+  __syncthreads();
+  if (tid >= WS_CONS) {
+    // ------------------------------- producers -------------------------------
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    const int pt = tid - WS_CONS, pw = pt >> 5;
+    WsRaw<CONTIG, false, OT> rk, rv;
+    ws_fetch<CONTIG, false, OT>(kp, S, DH, ld, jt_lo * OT, 0, pt, rk);
+    ws_fetch<CONTIG, false, OT>(vp, S, DH, ld, jt_lo * OT, 0, pt, rv);
+    for (int s = 0; s < nslab; ++s) {
+      const int slot = s % WS_STAGES;
+      if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
+      bool tiny = ws_store<CONTIG, false, OT>(Ks[slot], pt, rk);
+      tiny |= ws_store<CONTIG, false, OT>(Vs[slot], pt, rv);
+      if (s + 1 < nslab) {
+        const int j0n = (jt_lo + (s + 1) / (DH / OK)) * OT, c0n = ((s + 1) % (DH / OK)) * OK;
+        ws_fetch<CONTIG, false, OT>(kp, S, DH, ld, j0n, c0n, pt, rk);
+        ws_fetch<CONTIG, false, OT>(vp, S, DH, ld, j0n, c0n, pt, rv);
+      }
+      const int any = __any_sync(0xffffffffu, tiny);
+      if (lane == 0) tiny_s[slot][pw] = any;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_full[slot]);
+    }
+    return;
+  }
+  // --------------------------------- consumers ---------------------------------
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  const int ty = tid >> 4, tx = tid & 15;
+  const int tqo = tiny_qo;
+  const size_t bh = (size_t)b * H + h;
+  float Lr[8], Dr[8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int i = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+    Lr[a] = i < S ? lse[bh * S + i] : 0.0f;
+    Dr[a] = i < S ? delta[bh * S + i] : 0.0f;
+  }
+  int s = 0;
+  bool ok = true;
+  for (int jt = jt_lo; jt <= it && ok; ++jt) {
+    const int j0 = jt * OT;
+    float2 sa[8][4], da[8][4];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { sa[a][c] = make_float2(0.f, 0.f); da[a][c] = make_float2(0.f, 0.f); }
+    for (int sl = 0; sl < DH / OK; ++sl, ++s) {
+      const int slot = s % WS_STAGES;
+      if (!mbar_wait(&bar_full[slot], (uint32_t)((s / WS_STAGES) & 1), abort_flag, nullptr)) { ok = false; break; }
+      const int tiny = tqo | tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
+      if (tiny) { slab_mac<false, OT>(Qs + sl * OK, Ks[slot], ty, tx, sa); slab_mac<false, OT>(Os + sl * OK, Vs[slot], ty, tx, da); }
+      else { slab_mac<true, OT>(Qs + sl * OK, Ks[slot], ty, tx, sa); slab_mac<true, OT>(Os + sl * OK, Vs[slot], ty, tx, da); }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    }
+    if (!ok) break;
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      const int i = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+      if (i >= S) continue;
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        const int jb = j0 + g * 64 + tx * 4;
+        if (jb >= S) continue;
+        const float sv[4] = {sa[a][2 * g].x, sa[a][2 * g].y, sa[a][2 * g + 1].x, sa[a][2 * g + 1].y};
+        const float dv4[4] = {da[a][2 * g].x, da[a][2 * g].y, da[a][2 * g + 1].x, da[a][2 * g + 1].y};
+        float pv[4], dsv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          pv[e] = 0.0f; dsv[e] = 0.0f;
+          if (jb + e <= i && (W == 0 || jb + e > i - W)) {
+            pv[e] = det_exp(fsub(fmul(sv[e], ATT_SCALE), Lr[a]));
+            dsv[e] = fmul(fmul(pv[e], fsub(dv4[e], Dr[a])), ATT_SCALE);
+          }
+        }
+        const size_t off = (bh * S + i) * S + jb;
+        *reinterpret_cast<float4*>(Pf + off) = make_float4(pv[0], pv[1], pv[2], pv[3]);
+        uint2 u;
+        u.x = pack_bf2(dsv[0], dsv[1]); u.y = pack_bf2(dsv[2], dsv[3]);
+        *reinterpret_cast<uint2*>(dSt + off) = u;
+      }
+    }
+  }
+}
+
 static int set_smem(const void* fn, size_t bytes) {
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? 0 : -1;
 }
@@ -322,20 +467,13 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   k_attn_delta<<<DET_L((unsigned)((nrows + 7) / 8)), 256, 0, st>>>(dout, out, ld_out, H, S, nrows, delta);
   DET_CHECK_LAUNCH();
   // P[i,j] = exp(scale * sum_d q[i,d] k[j,d] - L_i) for visible (i,j) (f32; tiles without a visible pair are never
-  // touched), then dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both ascend over the 128 dims
-  OgemmArgs e = {};
-  e.I = S; e.J = S; e.C = DH; e.H = H; e.range_mode = 3; e.scale = ATT_SCALE; e.window = window; e.b_div = G;
-  e.ldo = S; e.o_b = (long long)H * S * S; e.o_h = (long long)S * S;
-  e.A = q; e.lda = ld; e.a_b = (long long)S * ld; e.a_h = DH;
-  e.B = k; e.ldb = ld; e.b_b = (long long)S * ld; e.b_h = DH;
-  e.out = Pf; e.rowv = lse;
-  int rc = ogemm_launch<CONTIG, CONTIG, false, false, 128, OEPI_P>(e, B * H, st);
-  if (rc != DET_OK) return rc;
-  e.A = dout; e.lda = ld_out; e.a_b = (long long)S * ld_out;
-  e.B = v;
-  e.out = dSt; e.rowv = delta; e.Pin = Pf;
-  rc = ogemm_launch<CONTIG, CONTIG, false, true, 128, OEPI_DS>(e, B * H, st);
-  if (rc != DET_OK) return rc;
+  // touched) and dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both sums ascend over the 128 dims
+  static bool cfg = false;
+  if (!cfg) { if (set_smem((const void*)k_attn_sdp_ws, SDP_SMEM)) return DET_ERR_CUDA; cfg = true; }
+  dim3 gsdp(H * B, (S + OT - 1) / OT);
+  k_attn_sdp_ws<<<DET_L(gsdp), WS_THREADS, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, Hkv, S, window, Pf, dSt);
+  DET_CHECK_LAUNCH();
+  int rc = DET_OK;
   // dV[j,c] = sum over the query heads g of the group, then over queries i >= j ascending, of P~[i,j] dO[i,c];
   // dK[j,c] likewise with dS~ and q.  One accumulator per output: with G > 1 it travels through `carry` in f32, and
   // the two chains then share that scratch and run one after the other.  dV, dK (for G == 1) and dQ are independent of

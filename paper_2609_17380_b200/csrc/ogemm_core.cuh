@@ -151,7 +151,7 @@ struct OgemmArgs {
   int H;                // batching: blockIdx.z = b * H + h
   long long a_b, a_h, b_b, b_h, o_b, o_h;  // element offsets per batch index / head index
   // head mapping for grouped-query attention (0 = identity): A reads head hA = h * h_mul + h_add, B reads head
-  // hA / b_div, the output (and rowv, Pin, acc_in) belongs to head h
+  // hA / b_div, the output (and acc_in) belongs to head h
   int h_mul, h_add, b_div;
   // optional f32 accumulators to start from (any output type): one sequential accumulator can be carried through
   // several launches this way; batched with acc_b / acc_h, leading dimension acc_ld
@@ -159,22 +159,12 @@ struct OgemmArgs {
   int acc_ld;
   long long acc_b, acc_h;
   int window;           // sliding window W (multiple of 128; 0 = none): only |query - key| < W contributes
-  int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile;
-                        // 3: whole contraction, but tiles entirely above the diagonal (j0 > i0) or entirely below the
-                        //    window are skipped
+  int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
                         // (with a window, mode 1 also stops at c < i0 + W + 128 and mode 2 starts at c >= i0 - W)
-  // epilogues of the attention backward (EPI 1, 2); rowv and Pin are batched like the output
-  const float* rowv;    // one value per row i of each batch: the logsumexp L (EPI 1) or Delta (EPI 2)
-  const float* Pin;     // EPI 2: the f32 weights written by EPI 1, same layout as the output
-  float scale;          // softmax scale
 };
 
-// Output transforms.  OEPI_NONE: the accumulator.  OEPI_P: P[i,j] = exp(acc*scale - L_i) for j <= i, else +0 (f32 out).
-// OEPI_DS: dS[i,j] = (P[i,j] * (acc - Delta_i)) * scale (bf16 out; P = 0 above the diagonal makes dS = 0 there).
-enum { OEPI_NONE = 0, OEPI_P = 1, OEPI_DS = 2 };
-
 // CTA tile 128 x TN; thread (ty, tx) owns rows {ty*4.., 64+ty*4..} and columns {g*64 + tx*4..}, g < TN/64.
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN, int EPI = OEPI_NONE>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
 __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
@@ -187,7 +177,6 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
   const int i0 = ti * OT, j0 = blockIdx.x * TN;
   const int W = p.window;
-  if (p.range_mode == 3 && (j0 > i0 || (W && i0 >= j0 + W + OT))) return;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
   const long long zb = zidx / p.H, zh = zidx % p.H;
   const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
@@ -255,24 +244,11 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
     const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
-    float rv = 0.0f;
-    if (EPI != OEPI_NONE && r < I) rv = p.rowv[(size_t)zidx * I + r];
 #pragma unroll
     for (int g = 0; g < TN / 64; ++g) {
       const int c = j0 + g * 64 + tx * 4;
       if (r < I && c < J) {
         float w[4] = {acc[a][2 * g].x, acc[a][2 * g].y, acc[a][2 * g + 1].x, acc[a][2 * g + 1].y};
-        if (EPI == OEPI_P) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            w[e] = (c + e <= r && (!W || c + e > r - W)) ? det_exp(fsub(fmul(w[e], p.scale), rv)) : 0.0f;
-        }
-        if (EPI == OEPI_DS) {
-          const float4 pw = *reinterpret_cast<const float4*>(p.Pin + zb * p.o_b + zh * p.o_h + (size_t)r * ldo + c);
-          const float pv[4] = {pw.x, pw.y, pw.z, pw.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) w[e] = fmul(fmul(pv[e], fsub(w[e], rv)), p.scale);
-        }
         if (OUT_BF16) {
           uint2 u;
           u.x = pack_bf2(w[0], w[1]);
@@ -286,11 +262,11 @@ __global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
   }
 }
 
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN, int EPI = OEPI_NONE>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
 static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   static bool cfg = false;
   if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)ogemm_smem<TN>()) != cudaSuccess)
       return DET_ERR_CUDA;
     cfg = true;
@@ -298,7 +274,7 @@ static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   const bool causal = p.range_mode == 1 || p.range_mode == 2;
   const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
   dim3 grid((p.J + TN - 1) / TN, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
-  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN, EPI><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
+  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
   return DET_OK;
 }
 
