@@ -493,12 +493,12 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
       if (g > 0) { p.acc_in = carry; p.acc_ld = DH; p.acc_b = (long long)Hkv * S * DH; p.acc_h = (long long)S * DH; }
       if (g == G - 1) {
         p.out = which == 0 ? dv : dk; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
-        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, true, 128>(p, B * Hkv, sk)     // P is rounded to bf16 as read
-                        : ogemm_launch<STRIDED, STRIDED, false, true, 128>(p, B * Hkv, sk);
+        rc = which == 0 ? ogemm_wb_launch<STRIDED, STRIDED, true, true>(p, B * Hkv, sk)     // P is rounded to bf16 as read
+                        : ogemm_wb_launch<STRIDED, STRIDED, false, true>(p, B * Hkv, sk);
       } else {
         p.out = carry; p.ldo = DH; p.o_b = (long long)Hkv * S * DH; p.o_h = (long long)S * DH;
-        rc = which == 0 ? ogemm_launch<STRIDED, STRIDED, true, false, 128>(p, B * Hkv, sk)
-                        : ogemm_launch<STRIDED, STRIDED, false, false, 128>(p, B * Hkv, sk);
+        rc = which == 0 ? ogemm_wb_launch<STRIDED, STRIDED, true, false>(p, B * Hkv, sk)
+                        : ogemm_wb_launch<STRIDED, STRIDED, false, false>(p, B * Hkv, sk);
       }
       if (rc != DET_OK) return rc;
     }
@@ -508,7 +508,7 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
   p.A = dSt; p.B = k; p.ldb = ld; p.b_b = (long long)S * ld; p.b_h = DH; p.b_div = G;
   p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
-  rc = ogemm_launch<CONTIG, STRIDED, false, true, 128>(p, B * H, aux ? aux->s[1] : st);
+  rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux ? aux->s[1] : st);
   if (rc != DET_OK) return rc;
   if (!aux_join(st, aux)) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();

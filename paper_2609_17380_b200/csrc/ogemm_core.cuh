@@ -1,6 +1,7 @@
-// Building blocks of the ordered FP32-ALU contractions (LM head, attention backward): operand slabs staged through
-// shared memory as f32, an 8 x (TN/16) register tile per thread, packed two-lane arithmetic, and the per-slab check
-// that decides between the fused and the two-instruction multiply-add (identical bits, see ogemm.cu).
+// The ordered FP32-ALU contractions (LM head, attention backward): C[i,j] = sum over c ascending of A(i,c) B(j,c), one
+// sequential accumulator per output.  Operand slabs are staged through shared memory as f32 by producer warps, consumer
+// warps hold 8 x 16 (or two 8 x 8) register tiles and use packed two-lane arithmetic; a per-slab check decides between the
+// fused and the two-instruction multiply-add (identical bits, see ogemm.cu).
 #pragma once
 #include "tc05.cuh"
 #include "internal.h"
@@ -14,95 +15,6 @@ constexpr int OK = 16;   // slab depth
 //   CONTIG : operand stored [rows, contraction] (contraction index contiguous)
 //   STRIDED: operand stored [contraction, rows] (row index contiguous)
 enum { CONTIG = 0, STRIDED = 1 };
-
-// Raw global data of 8 operand values: one 16-byte word of bf16, or two of f32.  The words stay packed in registers
-// while the current slab is multiplied and are only unpacked when they are stored to shared memory, so the unpacking
-// instructions (which wait for the load) sit after the multiply loop instead of in front of it.
-template <bool F32IN>
-struct Raw8 {
-  uint4 w[F32IN ? 2 : 1];
-};
-template <bool F32IN>
-__device__ __forceinline__ void load8_raw(const void* base, size_t idx, bool ok, Raw8<F32IN>& r) {
-  if (!ok) {
-#pragma unroll
-    for (int t = 0; t < (F32IN ? 2 : 1); ++t) r.w[t] = make_uint4(0u, 0u, 0u, 0u);
-    return;
-  }
-  if (F32IN) {
-    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(base) + idx);
-    r.w[0] = __ldg(p);
-    r.w[1] = __ldg(p + 1);
-  } else {
-    r.w[0] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + idx));
-  }
-}
-template <bool F32IN>
-__device__ __forceinline__ void unpack8(const Raw8<F32IN>& r, float v[8]) {
-  if (F32IN) {
-    // operands of the gradient contractions are rounded to bf16 first
-    const uint32_t u[8] = {r.w[0].x, r.w[0].y, r.w[0].z, r.w[0].w, r.w[1].x, r.w[1].y, r.w[1].z, r.w[1].w};
-#pragma unroll
-    for (int t = 0; t < 8; ++t) v[t] = bf2f(f2bf(__uint_as_float(u[t])));
-  } else {
-    const uint4 u = r.w[0];
-    v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
-    v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
-  }
-}
-
-// fetch this thread's values of an operand slab of ROWS rows x 16 contraction steps:
-// ROWS == 128: 8 values per thread, ROWS == 256: 16 values per thread
-template <int MODE, bool F32IN, int ROWS>
-__device__ __forceinline__ void slab_fetch(const void* base, int rows, int C, int ld, int r0, int c0,
-                                           Raw8<F32IN> (&raw)[ROWS / 128]) {
-  const int tid = threadIdx.x;
-  constexpr int NV = ROWS / 16;  // values per thread
-  if (MODE == CONTIG) {
-    // thread -> (row, 8 or 16 consecutive contraction indices)
-    const int r = r0 + (ROWS == 128 ? (tid & 127) : tid), c = c0 + (ROWS == 128 ? (tid >> 7) * 8 : 0);
-#pragma unroll
-    for (int h = 0; h < NV / 8; ++h) load8_raw<F32IN>(base, (size_t)r * ld + c + 8 * h, r < rows && c + 8 * h < C, raw[h]);
-  } else {
-    // thread -> (contraction index, NV consecutive rows)
-    const int c = c0 + (tid >> 4), r = r0 + (tid & 15) * NV;
-#pragma unroll
-    for (int h = 0; h < NV / 8; ++h) load8_raw<F32IN>(base, (size_t)c * ld + r + 8 * h, c < C && r + 8 * h < rows, raw[h]);
-  }
-}
-template <bool F32IN, int ROWS>
-__device__ __forceinline__ void slab_unpack(const Raw8<F32IN> (&raw)[ROWS / 128], float* v) {
-#pragma unroll
-  for (int h = 0; h < ROWS / 128; ++h) unpack8<F32IN>(raw[h], v + 8 * h);
-}
-template <int MODE, int ROWS>
-__device__ __forceinline__ void slab_store(float (*s)[ROWS + 4], const float* v) {
-  const int tid = threadIdx.x;
-  constexpr int NV = ROWS / 16;
-  if (MODE == CONTIG) {
-    const int r = (ROWS == 128 ? (tid & 127) : tid), k0 = (ROWS == 128 ? (tid >> 7) * 8 : 0);
-#pragma unroll
-    for (int t = 0; t < NV; ++t) s[k0 + t][r] = v[t];
-  } else {
-    const int k = tid >> 4, r = (tid & 15) * NV;
-#pragma unroll
-    for (int t = 0; t < NV; t += 4) *reinterpret_cast<float4*>(&s[k][r + t]) = make_float4(v[t], v[t + 1], v[t + 2], v[t + 3]);
-  }
-}
-
-// true if some value v has 0 < |v| < 2^-63 (biased exponent field in 1..63): a product with such a factor could
-// fall below 2^-126, where "multiply, flush, add" and a fused multiply-add differ
-template <int NV>
-__device__ __forceinline__ bool tiny_any(const float* v) {
-  bool t = false;
-#pragma unroll
-  for (int i = 0; i < NV; ++i) t |= (__float_as_uint(v[i]) * 2u - 1u) < 0x3fffffffu;  // also true for subnormals
-  return t;
-}
-
-
-template <int TN>
-constexpr size_t ogemm_smem() { return (size_t)2 * OK * ((OT + 4) + (TN + 4)) * sizeof(float); }
 
 // One 16-deep slab for this thread's 8 x (TN/16) outputs.  FUSED: a*b+acc in one instruction, used only for slabs in
 // which no product can be subnormal (every non-zero factor is at least 2^-63 in magnitude), where it gives exactly the
@@ -162,121 +74,6 @@ struct OgemmArgs {
   int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
                         // (with a window, mode 1 also stops at c < i0 + W + 128 and mode 2 starts at c >= i0 - W)
 };
-
-// CTA tile 128 x TN; thread (ty, tx) owns rows {ty*4.., 64+ty*4..} and columns {g*64 + tx*4..}, g < TN/64.
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
-__global__ void __launch_bounds__(256, TN == 128 ? 2 : 1) k_ogemm(OgemmArgs p) {
-  extern __shared__ __align__(16) unsigned char osm[];
-  float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
-  float(*Bs)[OK][TN + 4] = reinterpret_cast<float(*)[OK][TN + 4]>(osm + (size_t)2 * OK * (OT + 4) * sizeof(float));
-  // Blocks are handed out in linear order.  With a causal range (modes 1, 2) the row tile sits on the slowest grid index
-  // and runs from the longest contraction to the shortest, so that the blocks still running at the end of the grid are
-  // the short ones of every batch entry; otherwise the batch index is the slowest.
-  const bool causal = p.range_mode == 1 || p.range_mode == 2;
-  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
-  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
-  const int i0 = ti * OT, j0 = blockIdx.x * TN;
-  const int W = p.window;
-  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-  const long long zb = zidx / p.H, zh = zidx % p.H;
-  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
-  const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
-                       : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
-  const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
-  void* out = OUT_BF16 ? (void*)(reinterpret_cast<uint16_t*>(p.out) + zb * p.o_b + zh * p.o_h)
-                       : (void*)(reinterpret_cast<float*>(p.out) + zb * p.o_b + zh * p.o_h);
-  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
-  int c_lo = 0, C = p.C;
-  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
-  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
-  float2 acc[8][TN / 32];
-#pragma unroll
-  for (int a = 0; a < 8; ++a)
-#pragma unroll
-    for (int b = 0; b < TN / 32; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
-  const float* accp = p.acc_in ? p.acc_in + zb * p.acc_b + zh * p.acc_h
-                               : ((p.init && !OUT_BF16) ? reinterpret_cast<const float*>(out) : nullptr);
-  if (accp) {
-    const int ldacc = p.acc_in ? p.acc_ld : ldo;
-#pragma unroll
-    for (int a = 0; a < 8; ++a) {
-      const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
-#pragma unroll
-      for (int g = 0; g < TN / 64; ++g) {
-        const int c = j0 + g * 64 + tx * 4;
-        if (r < I && c < J) {
-          float4 t = *reinterpret_cast<const float4*>(accp + (size_t)r * ldacc + c);
-          acc[a][2 * g] = make_float2(t.x, t.y);
-          acc[a][2 * g + 1] = make_float2(t.z, t.w);
-        }
-      }
-    }
-  }
-  float va[8], vb[TN / 16];
-  Raw8<AF32> ra[1];
-  Raw8<false> rb[TN / 128];
-  slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, ra);
-  slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo, rb);
-  slab_unpack<AF32, OT>(ra, va);
-  slab_unpack<false, TN>(rb, vb);
-  slab_store<AMODE, OT>(As[0], va);
-  slab_store<BMODE, TN>(Bs[0], vb);
-  int tiny = __syncthreads_or(tiny_any<8>(va) || tiny_any<TN / 16>(vb));
-  const int nslab = (C - c_lo + OK - 1) / OK;
-  for (int s = 0; s < nslab; ++s) {
-    const int cur = s & 1;
-    if (s + 1 < nslab) {
-      slab_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, ra);
-      slab_fetch<BMODE, false, TN>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, rb);
-    }
-    if (tiny) slab_mac<false, TN>(As[cur], Bs[cur], ty, tx, acc);
-    else slab_mac<true, TN>(As[cur], Bs[cur], ty, tx, acc);
-    bool next_tiny = false;
-    if (s + 1 < nslab) {
-      slab_unpack<AF32, OT>(ra, va);
-      slab_unpack<false, TN>(rb, vb);
-      slab_store<AMODE, OT>(As[cur ^ 1], va);
-      slab_store<BMODE, TN>(Bs[cur ^ 1], vb);
-      next_tiny = tiny_any<8>(va) || tiny_any<TN / 16>(vb);
-    }
-    tiny = __syncthreads_or(next_tiny);
-  }
-#pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
-#pragma unroll
-    for (int g = 0; g < TN / 64; ++g) {
-      const int c = j0 + g * 64 + tx * 4;
-      if (r < I && c < J) {
-        float w[4] = {acc[a][2 * g].x, acc[a][2 * g].y, acc[a][2 * g + 1].x, acc[a][2 * g + 1].y};
-        if (OUT_BF16) {
-          uint2 u;
-          u.x = pack_bf2(w[0], w[1]);
-          u.y = pack_bf2(w[2], w[3]);
-          *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(out) + (size_t)r * ldo + c) = u;
-        } else {
-          *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ldo + c) = make_float4(w[0], w[1], w[2], w[3]);
-        }
-      }
-    }
-  }
-}
-
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, int TN>
-static int ogemm_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)ogemm_smem<TN>()) != cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
-  const bool causal = p.range_mode == 1 || p.range_mode == 2;
-  const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
-  dim3 grid((p.J + TN - 1) / TN, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
-  k_ogemm<AMODE, BMODE, AF32, OUT_BF16, TN><<<DET_L(grid), 256, ogemm_smem<TN>(), st>>>(p);
-  return DET_OK;
-}
 
 // ---------------------------------------------------------------------------------------------------------------
 // Warp-specialised variant for the long contractions of the LM head: 128 x 256 tile, eight consumer warps that only
@@ -501,6 +298,177 @@ static int ogemm_ws_launch(const OgemmArgs& p, cudaStream_t st) {
   }
   dim3 grid((p.J + WS_TN - 1) / WS_TN, (p.I + OT - 1) / OT, 1);
   k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WS_THREADS, WS_SMEM, st>>>(p);
+  return DET_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Warp-specialised batched variant for the causal contractions of the attention backward: 128 x 128 tile, four consumer
+// warps with 8 x 16 register tiles (rows {ty*4.., 64 + ty*4..}, columns g*32 + tx*4.., g < 4, eight threads across the
+// columns), four producer warps, the same mbarrier-guarded ring; two CTAs per SM.  Batching, head mapping, causal ranges,
+// windows and carried accumulators as in k_ogemm.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int WB_CONS = 128, WB_THREADS = WB_CONS + WS_PROD;
+constexpr size_t WB_SMEM = (size_t)WS_STAGES * OK * 2 * (OT + 4) * sizeof(float);
+
+template <bool FUSED>
+__device__ __forceinline__ void slab_mac_8x16n(const float (*As)[OT + 4], const float (*Bs)[OT + 4], int ty, int tx,
+                                               float2 (&acc)[8][8]) {
+#pragma unroll
+  for (int k = 0; k < OK; ++k) {
+    const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+    const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
+    const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    float2 b[8];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[k][g * 32 + tx * 4]);
+      b[2 * g] = make_float2(bv.x, bv.y);
+      b[2 * g + 1] = make_float2(bv.z, bv.w);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (FUSED) {
+          acc[i][j] = __ffma2_rn(make_float2(av[i], av[i]), b[j], acc[i][j]);
+        } else {  // scalar on purpose: a packed multiply + add pair would be contracted by ptxas
+          acc[i][j].x = fadd(acc[i][j].x, fmul(av[i], b[j].x));
+          acc[i][j].y = fadd(acc[i][j].y, fmul(av[i], b[j].y));
+        }
+      }
+    }
+  }
+}
+
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+__global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
+  extern __shared__ __align__(16) unsigned char osm[];
+  float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
+  float(*Bs)[OK][OT + 4] = As + WS_STAGES;
+  __shared__ int tiny_s[WS_STAGES][WS_PROD / 32];
+  __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+  // row tile on the slowest grid index, longest contraction first (see k_ogemm)
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
+  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
+  const int i0 = ti * OT, j0 = blockIdx.x * OT;
+  const int W = p.window;
+  const long long zb = zidx / p.H, zh = zidx % p.H;
+  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
+  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
+  int c_lo = 0, C = p.C;
+  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
+  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
+  const int nslab = (C - c_lo + OK - 1) / OK;
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WB_CONS / 32); }
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid >= WB_CONS) {
+    // ------------------------------- producers -------------------------------
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
+                         : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
+    const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
+    const int pt = tid - WB_CONS, pw = pt >> 5;
+    WsRaw<AMODE, AF32, OT> ra;
+    WsRaw<BMODE, false, OT> rb;
+    if (nslab > 0) {
+      ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, pt, ra);
+      ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo, pt, rb);
+    }
+    for (int s = 0; s < nslab; ++s) {
+      const int slot = s % WS_STAGES;
+      if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
+      bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
+      tiny |= ws_store<BMODE, false, OT>(Bs[slot], pt, rb);
+      if (s + 1 < nslab) {
+        ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, pt, ra);
+        ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, pt, rb);
+      }
+      const int any = __any_sync(0xffffffffu, tiny);
+      if (lane == 0) tiny_s[slot][pw] = any;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_full[slot]);
+    }
+    return;
+  }
+  // --------------------------------- consumers ---------------------------------
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  const int ty = tid >> 3, tx = tid & 7;
+  void* out = OUT_BF16 ? (void*)(reinterpret_cast<uint16_t*>(p.out) + zb * p.o_b + zh * p.o_h)
+                       : (void*)(reinterpret_cast<float*>(p.out) + zb * p.o_b + zh * p.o_h);
+  float2 acc[8][8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 8; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
+  const float* accp = p.acc_in ? p.acc_in + zb * p.acc_b + zh * p.acc_h
+                               : ((p.init && !OUT_BF16) ? reinterpret_cast<const float*>(out) : nullptr);
+  if (accp) {
+    const int ldacc = p.acc_in ? p.acc_ld : ldo;
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int c = j0 + g * 32 + tx * 4;
+        if (r < I && c < J) {
+          const float4 t = *reinterpret_cast<const float4*>(accp + (size_t)r * ldacc + c);
+          acc[a][2 * g] = make_float2(t.x, t.y);
+          acc[a][2 * g + 1] = make_float2(t.z, t.w);
+        }
+      }
+    }
+  }
+  for (int s = 0; s < nslab; ++s) {
+    const int slot = s % WS_STAGES;
+    if (!mbar_wait(&bar_full[slot], (uint32_t)((s / WS_STAGES) & 1), abort_flag, nullptr)) break;
+    const int tiny = tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
+    if (tiny) slab_mac_8x16n<false>(As[slot], Bs[slot], ty, tx, acc);
+    else slab_mac_8x16n<true>(As[slot], Bs[slot], ty, tx, acc);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_empty[slot]);
+  }
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const int c = j0 + g * 32 + tx * 4;
+      if (r < I && c < J) {
+        const float2 lo = acc[a][2 * g], hi = acc[a][2 * g + 1];
+        if (OUT_BF16) {
+          uint2 u;
+          u.x = pack_bf2(lo.x, lo.y);
+          u.y = pack_bf2(hi.x, hi.y);
+          *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(out) + (size_t)r * ldo + c) = u;
+        } else {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ldo + c) = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+      }
+    }
+  }
+}
+
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
+  static bool cfg = false;
+  if (!cfg) {
+    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)WB_SMEM) != cudaSuccess)
+      return DET_ERR_CUDA;
+    cfg = true;
+  }
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
+  dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
+  k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WB_THREADS, WB_SMEM, st>>>(p);
   return DET_OK;
 }
 
