@@ -51,27 +51,91 @@ __device__ __forceinline__ void epi_scalars(const EpiParams& ep, float& cscale, 
     }
 }
 
+// A warp's 32 rows x 32 columns of output, held one row per lane (`w`: NW sixteen-byte words), go through a 32 x NW*16
+// byte staging tile in shared memory (sixteen-byte pieces XOR-swizzled, conflict-free both ways) so that every store
+// instruction writes whole 64- or 128-byte row segments instead of 16 bytes in each of 32 rows.
+template <int NW>
+__device__ __forceinline__ void store_rows32(uint8_t* stage, uint8_t* gbase, size_t row_pitch_bytes, const uint4 (&w)[NW]) {
+  const int lane = threadIdx.x & 31;
+  constexpr int SH = (NW == 4) ? 1 : 0;  // NW = 4: two rows share a 128-byte bank window, so the swizzle uses row >> 1
+  __syncwarp();                          // the previous chunk's reads are done
+#pragma unroll
+  for (int v = 0; v < NW; ++v)
+    *reinterpret_cast<uint4*>(stage + lane * (NW * 16) + ((v ^ ((lane >> SH) & (NW - 1))) << 4)) = w[v];
+  __syncwarp();
+  constexpr int RPI = 32 / NW;           // rows per store instruction
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    const int r = i * RPI + lane / NW, piece = lane % NW;
+    const uint4 x = *reinterpret_cast<const uint4*>(stage + r * (NW * 16) + ((piece ^ ((r >> SH) & (NW - 1))) << 4));
+    *reinterpret_cast<uint4*>(gbase + (size_t)r * row_pitch_bytes + piece * 16) = x;
+  }
+}
+
+// The reverse for the bf16 reference operand of the gradient epilogues: `pre` holds sixteen-byte pieces fetched with whole
+// 64-byte row segments per quad of lanes (fetch_rows32); rows32_to_lanes hands every lane the four words of its own row.
+__device__ __forceinline__ void fetch_rows32(const uint8_t* gbase, size_t row_pitch_bytes, uint4 (&pre)[4]) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    pre[i] = __ldg(reinterpret_cast<const uint4*>(gbase + (size_t)(i * 8 + (lane >> 2)) * row_pitch_bytes + (lane & 3) * 16));
+}
+__device__ __forceinline__ void rows32_to_lanes(uint8_t* stage, const uint4 (&pre)[4], uint4 (&w)[4]) {
+  const int lane = threadIdx.x & 31;
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), piece = lane & 3;
+    *reinterpret_cast<uint4*>(stage + r * 64 + ((piece ^ ((r >> 1) & 3)) << 4)) = pre[i];
+  }
+  __syncwarp();
+#pragma unroll
+  for (int v = 0; v < 4; ++v) w[v] = *reinterpret_cast<const uint4*>(stage + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4));
+}
+
 // Epilogue of one accumulator row: this lane owns TMEM lane `taddr`'s row (output row `row`), columns j0 .. j0+BN.
+// With a staging tile (`stage`, 4 KiB per warp) the outputs are written through store_rows32.
 template <int BN, int EPI>
 __device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int row, int J, int j0, float cscale,
-                                        float inv_s, float sx) {
+                                        float inv_s, float sx, uint8_t* stage = nullptr) {
       const size_t rbase = (size_t)row * J + j0;
+      const size_t wbase = (size_t)(row - (int)(threadIdx.x & 31)) * J + j0;  // the warp's first row
       if (EPI == EPI_DW) inv_s = fdiv(1.0f, ep.s_w[row]);
 #pragma unroll 1
       for (int h = 0; h < BN / 128; ++h) {
       float grp[4];
+      uint4 pre[4];
+      const bool staged_ref = (EPI == EPI_DX || EPI == EPI_DW) && stage != nullptr;
+      if (staged_ref) fetch_rows32(reinterpret_cast<const uint8_t*>(ep.ref + wbase + h * 128), (size_t)J * 2, pre);
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         const int c0 = h * 128 + cc * 32;
         uint32_t r[32];
         tmem_ld32(taddr + (uint32_t)c0, r);
+        uint4 refw[4];
+        if (EPI == EPI_DX || EPI == EPI_DW) {
+          if (staged_ref) {
+            rows32_to_lanes(stage, pre, refw);
+            if (cc < 3) fetch_rows32(reinterpret_cast<const uint8_t*>(ep.ref + wbase + c0 + 32), (size_t)J * 2, pre);
+          } else {
+            const uint4* rr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) refw[v] = __ldg(rr + v);
+          }
+        }
         if (EPI == EPI_RAW) {
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<int32_t*>(ep.out) + rbase + c0);
+          uint4 o[8];
 #pragma unroll
           for (int v = 0; v < 8; ++v) o[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          if (stage) store_rows32<8>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<int32_t*>(ep.out) + wbase + c0), (size_t)J * 4, o);
+          else {
+            uint4* og = reinterpret_cast<uint4*>(reinterpret_cast<int32_t*>(ep.out) + rbase + c0);
+#pragma unroll
+            for (int v = 0; v < 8; ++v) og[v] = o[v];
+          }
         } else if (EPI == EPI_FWD) {
           const float4* sw = reinterpret_cast<const float4*>(ep.s_w + j0 + c0);
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+          uint4 o[4];
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             float4 w0 = __ldg(sw + 2 * v), w1 = __ldg(sw + 2 * v + 1);
@@ -86,13 +150,18 @@ __device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int
             f[7] = fmul(__int2float_rn((int)r[8 * v + 7]), fmul(sx, w1.w));
             o[v] = make_uint4(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]), pack_bf2(f[4], f[5]), pack_bf2(f[6], f[7]));
           }
+          if (stage) store_rows32<4>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(ep.out) + wbase + c0), (size_t)J * 2, o);
+          else {
+            uint4* og = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) og[v] = o[v];
+          }
         } else if (EPI == EPI_DX) {
-          const uint4* xr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
-          uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+          uint4 o[4];
           float term[32];
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
-            uint4 xu = __ldg(xr + v);
+            uint4 xu = refw[v];
             const uint32_t xs[4] = {xu.x, xu.y, xu.z, xu.w};
             float g[8];
 #pragma unroll
@@ -107,6 +176,12 @@ __device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int
             }
             o[v] = make_uint4(pack_bf2(g[0], g[1]), pack_bf2(g[2], g[3]), pack_bf2(g[4], g[5]), pack_bf2(g[6], g[7]));
           }
+          if (stage) store_rows32<4>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(ep.out) + wbase + c0), (size_t)J * 2, o);
+          else {
+            uint4* og = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(ep.out) + rbase + c0);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) og[v] = o[v];
+          }
           // adjacent tree over this lane's 32 columns
 #pragma unroll
           for (int w = 1; w < 32; w <<= 1)
@@ -114,11 +189,10 @@ __device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int
             for (int e = 0; e < 32; e += 2 * w) term[e] = fadd(term[e], term[e + w]);
           grp[cc] = term[0];
         } else {  // EPI_DW
-          const uint4* wr = reinterpret_cast<const uint4*>(ep.ref + rbase + c0);
-          float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out) + rbase + c0);
+          uint4 o[8];
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
-            uint4 wu = __ldg(wr + v);
+            uint4 wu = refw[v];
             const uint32_t wsr[4] = {wu.x, wu.y, wu.z, wu.w};
             float g[8];
 #pragma unroll
@@ -128,8 +202,14 @@ __device__ __forceinline__ void epi_row(const EpiParams& ep, uint32_t taddr, int
               const bool in_range = (t >= -128.0f) && (t <= 127.0f);
               g[e] = in_range ? fmul(__int2float_rn((int)r[8 * v + e]), cscale) : 0.0f;
             }
-            o[2 * v] = make_float4(g[0], g[1], g[2], g[3]);
-            o[2 * v + 1] = make_float4(g[4], g[5], g[6], g[7]);
+            o[2 * v] = make_uint4(__float_as_uint(g[0]), __float_as_uint(g[1]), __float_as_uint(g[2]), __float_as_uint(g[3]));
+            o[2 * v + 1] = make_uint4(__float_as_uint(g[4]), __float_as_uint(g[5]), __float_as_uint(g[6]), __float_as_uint(g[7]));
+          }
+          if (stage) store_rows32<8>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<float*>(ep.out) + wbase + c0), (size_t)J * 4, o);
+          else {
+            uint4* og = reinterpret_cast<uint4*>(reinterpret_cast<float*>(ep.out) + rbase + c0);
+#pragma unroll
+            for (int v = 0; v < 8; ++v) og[v] = o[v];
           }
         }
       }
@@ -267,6 +347,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 // ------------------------------------------------------------------------------------------------------------
 constexpr int STAGES2 = 6;
 constexpr int BN2 = 256;
+// warps 0 / 1 load and multiply; eight epilogue warps: warp & 3 is the TMEM lane quarter a warp may read, the two
+// warps of a quarter take one half (128 columns) of the accumulator each
+constexpr int GEMM2_THREADS = 64 + 8 * 32;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -313,7 +396,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
 }
 
 template <int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     k_igemm2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, EpiParams ep, int I, int J,
              int K, int* status) {
   constexpr int STAGE_A = 128 * BK, STAGE_B = 128 * BK, STAGE_BYTES = STAGE_A + STAGE_B;
@@ -329,7 +412,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
   const bool leader = rank == 0;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&bar_tfull[a], 1); mbar_init(&bar_tempty[a], 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&bar_tfull[a], 1); mbar_init(&bar_tempty[a], 16); }
     abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -400,7 +483,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
       }
     }
   } else {
-    const int q = warp & 3;
+    const int q = warp & 3, half = (warp - 2) >> 2;
+    uint8_t* stage = smem + STAGES2 * STAGE_BYTES + (warp - 2) * 4096;  // this warp's 32 x 128-byte staging tile
     int it = 0;
     bool ok = true;
     float cscale, inv_s, sx;
@@ -414,8 +498,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
       else { i0 = (tile % tiles_i) * 256; j0 = (tile / tiles_i) * BN2; }
       if (!mbar_wait(&bar_tfull[acc], acc_phase, abort_flag, status)) { ok = false; break; }
       tc_fence_after();
-      epi_row<BN2, EPI>(ep, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN2), i0 + (int)rank * 128 + q * 32 + lane, J,
-                        j0, cscale, inv_s, sx);
+      epi_row<BN2 / 2, EPI>(ep, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN2 + half * (BN2 / 2)),
+                            i0 + (int)rank * 128 + q * 32 + lane, J, j0 + half * (BN2 / 2), cscale, inv_s, sx, stage);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(acc ? tempty_leader1 : tempty_leader0);
@@ -488,7 +572,7 @@ static int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const EpiPar
 template <int EPI>
 static int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const EpiParams& ep, int I, int J, int K, int* status,
                        cudaStream_t st) {
-  constexpr size_t smem = (size_t)STAGES2 * (2 * 128 * BK) + 1024;
+  constexpr size_t smem = (size_t)STAGES2 * (2 * 128 * BK) + 8 * 4096 + 1024;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(k_igemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -504,7 +588,7 @@ static int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const EpiPa
   const int tiles = (I / 256) * (J / BN2);
   int clusters = sms / 2;
   if (tiles < clusters) clusters = tiles;
-  k_igemm2<EPI><<<DET_L(2 * clusters), GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
+  k_igemm2<EPI><<<DET_L(2 * clusters), GEMM2_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
   if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
   return DET_OK;
 }

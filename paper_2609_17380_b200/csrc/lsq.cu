@@ -256,7 +256,10 @@ __global__ void __launch_bounds__(128) k_rotc(const void* __restrict__ in, int R
 //     butterflies on register pairs with packed arithmetic: a + b is one packed add, a - b one packed fused
 //     multiply-add b * (-1) + a, which rounds exactly like the subtraction.  PASS 0 records both absmax values,
 //     PASS 1 quantises with them.  dY is read twice per backward pass instead of four times.
-constexpr int PT = 128, PLD = 129;
+//     The kernel is bound by the shared-memory / L1 pipeline, so every shared-memory access is a conflict-free
+//     sixteen-byte one where the layout allows (rows padded to 132 floats), and PASS 1 hands its int8 rows over through
+//     the (then dead) tile so that every global store instruction writes four whole 128-byte rows.
+constexpr int PT = 128, PLD = 132;
 constexpr size_t PREP_SMEM = (size_t)(PT * PLD + PT) * sizeof(float);
 
 __device__ __forceinline__ void wht128_pairs(float2 (&v)[64]) {
@@ -281,20 +284,31 @@ __device__ __forceinline__ float absmax128(const float2 (&v)[64]) {
   for (int p = 0; p < 64; ++p) m = fmaxf(m, fmaxf(fabsf(v[p].x), fabsf(v[p].y)));
   return m;
 }
-__device__ __forceinline__ void quant_store128(const float2 (&v)[64], float inv, int8_t* dst) {
-  uint4* d4 = reinterpret_cast<uint4*>(dst);
+// 128 rotated values -> 32 words of int8 codes clamp(rne(v * inv), -128, 127).
+// FAST: every product is finite and at most 127 (1 + 2^-22) in magnitude (the caller checked: the step comes from the
+// absmax of these very values, and the first rotated value, the plain sum that every input reaches through additions
+// only, is finite), so the clamp cannot act; adding 1.5 * 2^23 rounds to nearest-even exactly like the conversion and
+// leaves the code in the low byte of the float's bits.  The multiply stays a scalar instruction of its own (rounded
+// before the add); otherwise the generic path.
+template <bool FAST>
+__device__ __forceinline__ void quant_pack128(const float2 (&v)[64], float inv, uint32_t (&w)[32]) {
+  const float2 magic = make_float2(12582912.0f, 12582912.0f);
 #pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    uint32_t w[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float2 lo = v[g * 8 + k * 2], hi = v[g * 8 + k * 2 + 1];
+  for (int k = 0; k < 32; ++k) {
+    const float2 lo = v[2 * k], hi = v[2 * k + 1];
+    if (FAST) {
+      const float2 a = __fadd2_rn(make_float2(fmul(lo.x, inv), fmul(lo.y, inv)), magic);
+      const float2 b = __fadd2_rn(make_float2(fmul(hi.x, inv), fmul(hi.y, inv)), magic);
+      const uint32_t t1 = __byte_perm(__float_as_uint(a.x), __float_as_uint(a.y), 0x0040);
+      const uint32_t t2 = __byte_perm(__float_as_uint(b.x), __float_as_uint(b.y), 0x0040);
+      w[k] = __byte_perm(t1, t2, 0x5410);
+    } else {
       w[k] = ((uint32_t)(uint8_t)quant1(lo.x, inv)) | ((uint32_t)(uint8_t)quant1(lo.y, inv) << 8) |
              ((uint32_t)(uint8_t)quant1(hi.x, inv) << 16) | ((uint32_t)(uint8_t)quant1(hi.y, inv) << 24);
     }
-    d4[g] = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
+__device__ __forceinline__ bool finite1(float x) { return (__float_as_uint(x) & 0x7f800000u) != 0x7f800000u; }
 __device__ __forceinline__ void amax_publish(float local, uint32_t* amax) {
 #pragma unroll
   for (int w = 16; w; w >>= 1) local = fmaxf(local, __shfl_xor_sync(0xffffffffu, local, w));
@@ -315,33 +329,66 @@ __global__ void __launch_bounds__(PT, 3) k_prep_dy(const uint16_t* __restrict__ 
   for (int it = 0; it < 16; ++it)
     raw[it] = __ldg(reinterpret_cast<const uint4*>(dY + (size_t)(m0 + it * 8 + (t >> 4)) * N + n0 + (t & 15) * 8));
   sw[t] = __ldg(s_w + n0 + t);
+  // eight values per thread and row as two sixteen-byte stores; lanes 0-3 of every eight store their first half while
+  // lanes 4-7 store their second, then the other way round: each store instruction covers all banks once
+  const int sel = (t >> 2) & 1;
 #pragma unroll
   for (int it = 0; it < 16; ++it) {
     float* d = &tile[it * 8 + (t >> 4)][(t & 15) * 8];
     const uint4 u = raw[it];
-    d[0] = bflo(u.x); d[1] = bfhi(u.x); d[2] = bflo(u.y); d[3] = bfhi(u.y);
-    d[4] = bflo(u.z); d[5] = bfhi(u.z); d[6] = bflo(u.w); d[7] = bfhi(u.w);
+    const float4 f0 = make_float4(bflo(u.x), bfhi(u.x), bflo(u.y), bfhi(u.y));
+    const float4 f1 = make_float4(bflo(u.z), bfhi(u.z), bflo(u.w), bfhi(u.w));
+    *reinterpret_cast<float4*>(d + 4 * sel) = sel ? f1 : f0;
+    *reinterpret_cast<float4*>(d + 4 * (sel ^ 1)) = sel ? f0 : f1;
   }
   __syncthreads();
   float invA = 0.0f, invG = 0.0f;
+  bool fastA = false, fastG = false;
   if (PASS == 1) {
     const float a = __uint_as_float(amax[0]), g = __uint_as_float(amax[1]);
     invA = (a > 0.0f) ? fdiv(127.0f, a) : 0.0f;
     invG = (g > 0.0f) ? fdiv(127.0f, g) : 0.0f;
+    fastA = finite1(a) && finite1(invA);
+    fastG = finite1(g) && finite1(invG);
   }
   float2 v[64];
+  uint32_t qa[32], qg[32];
   // row t of the tile, scaled by the weight steps (scalar multiplies: the products are rounded before any add)
 #pragma unroll
-  for (int p = 0; p < 64; ++p) v[p] = make_float2(fmul(tile[t][2 * p], sw[2 * p]), fmul(tile[t][2 * p + 1], sw[2 * p + 1]));
+  for (int q = 0; q < 32; ++q) {
+    const float4 x = *reinterpret_cast<const float4*>(&tile[t][4 * q]);
+    const float4 c = *reinterpret_cast<const float4*>(&sw[4 * q]);
+    v[2 * q] = make_float2(fmul(x.x, c.x), fmul(x.y, c.y));
+    v[2 * q + 1] = make_float2(fmul(x.z, c.z), fmul(x.w, c.w));
+  }
   wht128_pairs(v);
   if (PASS == 0) amax_publish(absmax128(v), amax + 0);
-  else quant_store128(v, invA, Aq + (size_t)(m0 + t) * N + n0);
+  else if (fastA && finite1(v[0].x)) quant_pack128<true>(v, invA, qa);
+  else quant_pack128<false>(v, invA, qa);
   // column t of the tile, transposed output
 #pragma unroll
   for (int p = 0; p < 64; ++p) v[p] = make_float2(tile[2 * p][t], tile[2 * p + 1][t]);
   wht128_pairs(v);
-  if (PASS == 0) amax_publish(absmax128(v), amax + 1);
-  else quant_store128(v, invG, GqT + (size_t)(n0 + t) * M + m0);
+  if (PASS == 0) { amax_publish(absmax128(v), amax + 1); return; }
+  if (fastG && finite1(v[0].x)) quant_pack128<true>(v, invG, qg);
+  else quant_pack128<false>(v, invG, qg);
+  // hand-over through the tile's memory: two tiles of 128 rows x 128 bytes, sixteen-byte pieces XOR-swizzled by row
+  __syncthreads();
+  uint8_t* stg = reinterpret_cast<uint8_t*>(psm);
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    const int off = t * 128 + ((g ^ (t & 7)) << 4);
+    *reinterpret_cast<uint4*>(stg + off) = make_uint4(qa[4 * g], qa[4 * g + 1], qa[4 * g + 2], qa[4 * g + 3]);
+    *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(qg[4 * g], qg[4 * g + 1], qg[4 * g + 2], qg[4 * g + 3]);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int idx = i * PT + t, r = idx >> 3, piece = idx & 7;
+    const int off = r * 128 + ((piece ^ (r & 7)) << 4);
+    *reinterpret_cast<uint4*>(Aq + (size_t)(m0 + r) * N + n0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + off);
+    *reinterpret_cast<uint4*>(GqT + (size_t)(n0 + r) * M + m0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + 16384 + off);
+  }
 }
 
 __global__ void k_su_finish(const uint32_t* amax, int rotated, float* s_u) {
