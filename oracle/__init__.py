@@ -246,7 +246,8 @@ def attn_fwd(qkv, B, H, S, Hkv=None, window=0, int8_pv=False):
     return out, lse
 
 
-def attn_bwd(dout, qkv, out, lse, B, H, S, Hkv=None, window=0):
+def attn_bwd(dout, qkv, out, lse, B, H, S, Hkv=None, window=0, fixq=False):
+    """fixq: the query gradient accumulated over the key blocks in 64-bit fixed point (48 fractional bits)."""
     dout = _c(dout, np.uint16)
     qkv = _c(qkv, np.uint16)
     out = _c(out, np.uint16)
@@ -257,10 +258,24 @@ def attn_bwd(dout, qkv, out, lse, B, H, S, Hkv=None, window=0):
     dqkv = np.empty_like(qkv)
     base = qkv.ctypes.data
     dbase = dqkv.ctypes.data
-    lib().orc_attn_bwd(_p(dout), C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), _p(out), _p(lse),
+    fn = lib().orc_attn_bwd_fixq if fixq else lib().orc_attn_bwd
+    fn(_p(dout), C.c_void_p(base), C.c_void_p(base + 2 * HD), C.c_void_p(base + 2 * (HD + KD)), _p(out), _p(lse),
                        C.c_int(ld), C.c_int(HD), C.c_int(B), C.c_int(H), C.c_int(Hkv), C.c_int(S), C.c_int(window),
                        C.c_void_p(dbase), C.c_void_p(dbase + 2 * HD), C.c_void_p(dbase + 2 * (HD + KD)), C.c_int(ld))
     return dqkv
+
+
+def fix48(u):
+    """float32 -> the 64-bit fixed-point contribution (48 fractional bits) of the query-gradient accumulator."""
+    f = lib().orc_fix48
+    f.restype, f.argtypes = C.c_int64, [C.c_float]
+    return int(f(C.c_float(float(np.float32(u)))))
+
+
+def unfix48(a):
+    f = lib().orc_unfix48
+    f.restype, f.argtypes = C.c_float, [C.c_int64]
+    return np.float32(f(C.c_int64(int(a))))
 
 
 # ---- glue -----------------------------------------------------------------

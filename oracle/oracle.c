@@ -578,9 +578,23 @@ void orc_attn_fwd_int8pv(const bf16_t *q, const bf16_t *k, const bf16_t *v, int 
  * queries the gradient of a shared key/value head is ONE sequential accumulator
  * over its query heads in ascending order and, within a head, over the queries
  * in ascending order. */
-void orc_attn_bwd(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf16_t *v, const bf16_t *out,
-                  const float *lse, int ldq, int ld_out, int B, int H, int Hkv, int S, int W, bf16_t *dq, bf16_t *dk,
-                  bf16_t *dv, int ld_d) {
+/* Sec. 3.2 names a second accumulator for the query gradient: 64-bit fixed point, so that the sum over the key blocks
+   does not depend on their order.  Reading: the contribution of one block of 128 keys is the ordered fp32 sum over the
+   block's keys from +0 (the same per-block arithmetic as P.V in the forward); it enters a signed 64-bit accumulator
+   with 48 fractional bits as rne(u * 2^48), saturated at the ends of the range (a NaN contributes 0); integer
+   additions wrap; the result is the accumulator converted to fp32 (round to nearest even) times 2^-48, then bf16. */
+int64_t orc_fix48(float u) {
+  float t = fmul(u, 0x1p48f);
+  if (t != t) return 0;
+  if (t >= 0x1p63f) return INT64_MAX;
+  if (t <= -0x1p63f) return INT64_MIN;
+  return (int64_t)llrintf(t);
+}
+float orc_unfix48(int64_t a) { return fmul((float)a, 0x1p-48f); }
+
+static void attn_bwd_impl(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf16_t *v, const bf16_t *out,
+                          const float *lse, int ldq, int ld_out, int B, int H, int Hkv, int S, int W, bf16_t *dq,
+                          bf16_t *dk, bf16_t *dv, int ld_d, int fixq) {
   const int G = H / Hkv;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int bk = 0; bk < B * Hkv; ++bk) {
@@ -628,15 +642,38 @@ void orc_attn_bwd(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf
       for (int i = 0; i < S; ++i)
         for (int c = 0; c < DH; ++c) {
           float aq = 0.0f;
-          for (int j = 0; j <= i; ++j) {
-            if (!visible(i, j, W)) continue;
-            aq = fadd(aq, fmul(dSt[g * SS + (size_t)i * S + j], bf2f(k[(size_t)ldq * (b * S + j) + hk * DH + c])));
+          if (!fixq) {
+            for (int j = 0; j <= i; ++j) {
+              if (!visible(i, j, W)) continue;
+              aq = fadd(aq, fmul(dSt[g * SS + (size_t)i * S + j], bf2f(k[(size_t)ldq * (b * S + j) + hk * DH + c])));
+            }
+          } else {
+            uint64_t fx = 0;
+            for (int j0 = 0; j0 <= i; j0 += 128) {   /* blocks of 128 keys; a block without visible keys adds 0 */
+              float u = 0.0f;
+              for (int j = j0; j < j0 + 128 && j <= i; ++j) {
+                if (!visible(i, j, W)) continue;
+                u = fadd(u, fmul(dSt[g * SS + (size_t)i * S + j], bf2f(k[(size_t)ldq * (b * S + j) + hk * DH + c])));
+              }
+              fx += (uint64_t)orc_fix48(u);
+            }
+            aq = orc_unfix48((int64_t)fx);
           }
           dq[(size_t)ld_d * (b * S + i) + h * DH + c] = f2bf(aq);
         }
     }
     free(Pt); free(dSt);
   }
+}
+void orc_attn_bwd(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf16_t *v, const bf16_t *out,
+                  const float *lse, int ldq, int ld_out, int B, int H, int Hkv, int S, int W, bf16_t *dq, bf16_t *dk,
+                  bf16_t *dv, int ld_d) {
+  attn_bwd_impl(dout, q, k, v, out, lse, ldq, ld_out, B, H, Hkv, S, W, dq, dk, dv, ld_d, 0);
+}
+void orc_attn_bwd_fixq(const bf16_t *dout, const bf16_t *q, const bf16_t *k, const bf16_t *v, const bf16_t *out,
+                       const float *lse, int ldq, int ld_out, int B, int H, int Hkv, int S, int W, bf16_t *dq, bf16_t *dk,
+                       bf16_t *dv, int ld_d) {
+  attn_bwd_impl(dout, q, k, v, out, lse, ldq, ld_out, B, H, Hkv, S, W, dq, dk, dv, ld_d, 1);
 }
 
 /* ------------------------------------------------------------------ */

@@ -40,7 +40,11 @@ __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
 __device__ __forceinline__ float det_exp(float x) {
   if (x > 0x1.62e42ep+6f) return __int_as_float(0x7f800000);
   if (x < -0x1.5d58a0p+6f) return 0.0f;
-  float kf = rintf(fmul(x, 0x1.715476p+0f));
+  // k = rne(x log2 e): adding 1.5 * 2^23 rounds to the nearest even integer exactly like rintf for |t| < 2^22 (here
+  // |t| < 2^8) and leaves k in the low bits of the sum, so neither the rounding nor the conversion needs the
+  // conversion pipe
+  const float km = fadd(fmul(x, 0x1.715476p+0f), 12582912.0f);
+  const float kf = fsub(km, 12582912.0f);
   float r = fsub(fsub(x, fmul(kf, 0x1.62e400p-1f)), fmul(kf, 0x1.7f7d1cp-20f));
   float p = 0x1.a01a02p-13f;
   p = fadd(fmul(p, r), 0x1.6c16c2p-10f);
@@ -50,7 +54,7 @@ __device__ __forceinline__ float det_exp(float x) {
   p = fadd(fmul(p, r), 0.5f);
   p = fadd(fmul(p, r), 1.0f);
   p = fadd(fmul(p, r), 1.0f);
-  int k = (int)kf;
+  const int k = (int)__float_as_uint(km) - 0x4B400000;
   if (k > 127) return fmul(fmul(p, 0x1p127f), 2.0f);
   return fmul(p, __int_as_float((k + 127) << 23));
 }

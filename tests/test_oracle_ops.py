@@ -282,6 +282,63 @@ def test_attention_backward_against_float64():
     assert np.array_equal(d2[:S, :], dqkv[:S, :]) and np.array_equal(d2[S:S + 130 - 0, :H * 128], dqkv[S:S + 130, :H * 128])
 
 
+def test_fixed_point_query_gradient_pins():
+    """The 64-bit fixed-point accumulator of the query gradient (Sec. 3.2).  Hand values of the conversion; one block of
+    keys: identical to the plain ordered sum wherever that sum is a multiple of 2^-48; several blocks: float64 reference,
+    the other two gradients untouched, and the bf16 results at most one step away from the plain accumulator's."""
+    two48 = 1 << 48
+    assert oracle.fix48(1.0) == two48 and oracle.fix48(-0.75) == -3 * (1 << 46)
+    assert oracle.fix48(2.0 ** -49) == 0 and oracle.fix48(3 * 2.0 ** -49) == 2      # ties go to the even integer
+    assert oracle.fix48(-(2.0 ** -49)) == 0 and oracle.fix48(-3 * 2.0 ** -49) == -2
+    assert oracle.fix48(5 * 2.0 ** -50) == 1 and oracle.fix48(7 * 2.0 ** -50) == 2   # 1.25 -> 1, 1.75 -> 2
+    assert oracle.fix48(2.0 ** 15) == (1 << 63) - 1 and oracle.fix48(-(2.0 ** 15)) == -(1 << 63)   # saturation
+    assert oracle.fix48(1e30) == (1 << 63) - 1 and oracle.fix48(-1e30) == -(1 << 63)
+    assert oracle.fix48(float("nan")) == 0 and oracle.fix48(32767.5) == 32767 * two48 + (two48 >> 1)
+    assert oracle.unfix48(two48) == 1.0 and oracle.unfix48(-3 * (1 << 46)) == -0.75
+    assert oracle.unfix48(two48 + 1) == 1.0                            # 2^48 + 1 rounds to 2^48 in binary32
+    assert oracle.unfix48((1 << 24) + 1) == np.float32(2.0 ** -24)     # 2^24 + 1 ties to even
+    assert oracle.unfix48((1 << 24) + 3) == np.float32((2 ** 24 + 4) * 2.0 ** -48)
+
+    B, H = 1, 2
+    for S in (96, 128):                       # a single block of keys: sums far above 2^-25 convert exactly
+        qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=66)
+        dout = synth.normal_bf16((B * S, H * 128), 1.0, seed=0, tid=67)
+        out, lse = oracle.attn_fwd(qkv, B, H, S)
+        plain = oracle.attn_bwd(dout, qkv, out, lse, B, H, S)
+        fixed = oracle.attn_bwd(dout, qkv, out, lse, B, H, S, fixq=True)
+        assert np.array_equal(fixed[:, H * 128:], plain[:, H * 128:])        # dK, dV do not use the accumulator
+        big = np.abs(bf(plain[:, :H * 128])) >= 2.0 ** -20
+        assert big.mean() > 0.9 and np.array_equal(fixed[:, :H * 128][big], plain[:, :H * 128][big])
+
+    S = 300                                   # three blocks (the last one ragged)
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=68)
+    dout = synth.normal_bf16((B * S, H * 128), 0.1, seed=0, tid=69)
+    out, lse = oracle.attn_fwd(qkv, B, H, S)
+    plain = oracle.attn_bwd(dout, qkv, out, lse, B, H, S)
+    fixed = oracle.attn_bwd(dout, qkv, out, lse, B, H, S, fixq=True)
+    assert np.array_equal(fixed[:, H * 128:], plain[:, H * 128:])
+    q, k, v, pr, o, _ = _attn_ref(qkv, B, H, S)
+    do = bf(dout).astype(np.float64).reshape(B, S, H, 128).transpose(0, 2, 1, 3)
+    ds = pr * (do @ v.transpose(0, 1, 3, 2) - (do * o).sum(-1, keepdims=True)) / math.sqrt(128)
+    ref = (ds @ k).transpose(0, 2, 1, 3).reshape(B * S, H * 128)
+    assert rel_err(bf(fixed[:, :H * 128]).astype(np.float64), ref) < 0.01
+    # rows below 128 see one block only; all rows: neighbouring bf16 values at worst (the two accumulators differ by
+    # far less than a bf16 step, so they can only fall on either side of a rounding boundary)
+    assert np.array_equal(fixed[:128, :H * 128], plain[:128, :H * 128])
+    fa, pa = fixed[:, :H * 128].astype(np.int32), plain[:, :H * 128].astype(np.int32)
+    assert np.abs(fa - pa).max() <= 1 and (fa != pa).mean() < 0.02
+    # a sliding window and grouped heads go through the same accumulator
+    Hq, Hkv, W = 4, 2, 128
+    qkv = synth.normal_bf16((B * S, (Hq + 2 * Hkv) * 128), 1.0, seed=0, tid=70)
+    dout = synth.normal_bf16((B * S, Hq * 128), 0.1, seed=0, tid=71)
+    out, lse = oracle.attn_fwd(qkv, B, Hq, S, Hkv=Hkv, window=W)
+    plain = oracle.attn_bwd(dout, qkv, out, lse, B, Hq, S, Hkv=Hkv, window=W)
+    fixed = oracle.attn_bwd(dout, qkv, out, lse, B, Hq, S, Hkv=Hkv, window=W, fixq=True)
+    assert np.array_equal(fixed[:, Hq * 128:], plain[:, Hq * 128:])
+    fa, pa = fixed[:, :Hq * 128].astype(np.int32), plain[:, :Hq * 128].astype(np.int32)
+    assert np.abs(fa - pa).max() <= 1 and np.array_equal(fa[:128], pa[:128])
+
+
 def _expand_kv(qkv, H, Hkv):
     """grouped q|k|v rows -> multi-head rows with every key/value head repeated for its query heads"""
     G = H // Hkv
