@@ -29,7 +29,7 @@ WORKLOAD = "config5: full 1B-shaped step, 24 layers, d_model 2048, 16 heads, FFN
 
 
 WORKLOAD_PAPER = "paper block (not the default): 24 layers, d_model 2048, 16 query / 4 key-value heads, QK-norm, RoPE 5e5, " \
-                 "embedding norm, sliding window 512 with every 5th and the last layer full, int8 P.V, z-loss 1e-4, FFN 5632, vocab 128256, " \
+                 "embedding norm, sliding window 512 with every 5th and the last layer full, int8 P.V, fixed-point query gradient, z-loss 1e-4, FFN 5632, vocab 128256, " \
                  "seq 4096, 8 micro-batches of 4 sequences, mesh (2,2,2), AdamW, SHA-256 of post-step state"
 
 
@@ -41,7 +41,7 @@ def full_config_kwargs(layers=None, workload="config5"):
         i = np.arange(64, dtype=np.float64)
         ang = np.arange(4096, dtype=np.float64)[:, None] * (5.0e5 ** (-2.0 * i / 128))[None, :]
         kw.update(n_kv_heads=4, ffn=5632, vocab=128256, seq=4096, qk_norm=True, embed_norm=True, window=512, full_every=5,
-                  z_weight=1e-4, lr=4.5e-4, pv_int8=True, rope_tables=(np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)))
+                  z_weight=1e-4, lr=4.5e-4, pv_int8=True, dq_fixed=True, rope_tables=(np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)))
     if layers is not None:
         kw["n_layers"] = layers
     return kw

@@ -106,7 +106,8 @@ def microbatch_grad(cfg, P, sw, tok):
         d_h2, G["l%d.ffn_norm" % l] = O.rmsnorm_bwd(d_n2, a["h"], P["l%d.ffn_norm" % l], a["rstd2"], bf=True)
         d_h = O.residual_add(dx, d_h2)
         d_att, G["l%d.w_o" % l], d1 = O.linear_bwd(d_h, a["att"], P["l%d.w_o" % l], sx[1:2], sw["l%d.w_o" % l], hb)
-        d_qkv = O.attn_bwd(d_att, a["qkr"], a["att"], a["lse"], B, H, S, Hkv=Hkv, window=_window(cfg, l))
+        d_qkv = O.attn_bwd(d_att, a["qkr"], a["att"], a["lse"], B, H, S, Hkv=Hkv, window=_window(cfg, l),
+                           fixq=bool(cfg.get("dq_fixed")))
         dqk = np.ascontiguousarray(d_qkv[:, :D + 128 * Hkv]).reshape(-1, 128)
         if rope is not None:
             dqk = O.rope(dqk.reshape(B * S, H + Hkv, 128), S, rope[0], rope[1], inverse=True).reshape(-1, 128)

@@ -52,7 +52,8 @@ def load():
         _lib = C.CDLL(_SO)
         for name in ("det_sum_ws_bytes", "det_grad_norm_ws_bytes", "det_lsq_weight_scale_ws_bytes",
                      "det_lsq_act_scale_init_ws_bytes", "det_lsq_quantize_weight_ws_bytes", "det_linear_bwd_ws_bytes",
-                     "det_rmsnorm_bwd_ws_bytes", "det_xent_ws_bytes", "det_attn_bwd_ws_bytes", "det_tensor_hash_ws_bytes"):
+                     "det_rmsnorm_bwd_ws_bytes", "det_xent_ws_bytes", "det_attn_bwd_ws_bytes", "det_attn_bwd_fixq_ws_bytes",
+                     "det_tensor_hash_ws_bytes"):
             getattr(_lib, name).restype = C.c_size_t
         _lib.det_launch_count.restype = C.c_ulonglong
     return _lib
@@ -257,6 +258,17 @@ def det_attn_bwd(dout, q, k, v, out, lse, ld, ld_out, B, H, S, dq, dk, dv, ld_d,
                                                C.c_int(ld_out), C.c_int(B), C.c_int(H), C.c_int(H if Hkv is None else Hkv),
                                                C.c_int(S), C.c_int(window), _ptr(dq), _ptr(dk), _ptr(dv), C.c_int(ld_d),
                                                *_ws(ws), _stream()))
+
+
+def det_attn_bwd_fixq_ws_bytes(B, H, S, Hkv=None):
+    return load().det_attn_bwd_fixq_ws_bytes(C.c_int(B), C.c_int(H), C.c_int(H if Hkv is None else Hkv), C.c_int(S))
+
+
+def det_attn_bwd_fixq(dout, q, k, v, out, lse, ld, ld_out, B, H, S, dq, dk, dv, ld_d, ws, Hkv=None, window=0):
+    _check("det_attn_bwd_fixq", load().det_attn_bwd_fixq(_ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse),
+                                                         C.c_int(ld), C.c_int(ld_out), C.c_int(B), C.c_int(H),
+                                                         C.c_int(H if Hkv is None else Hkv), C.c_int(S), C.c_int(window),
+                                                         _ptr(dq), _ptr(dk), _ptr(dv), C.c_int(ld_d), *_ws(ws), _stream()))
 
 
 # ---- glue --------------------------------------------------------------------------------------------------------

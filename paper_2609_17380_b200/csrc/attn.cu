@@ -444,17 +444,23 @@ extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S) {
          align_up((size_t)B * H * S * 4, 256) + (Hkv < H ? align_up((size_t)B * Hkv * S * DH * 4, 256) : 0);
 }
 
-extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
-                            const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
-                            int window, det_bf16* dq, det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes,
-                            void* stream) {
+// the fixed-point variant adds the signed 64-bit accumulators of the query gradient [B*H, S, 128]
+extern "C" size_t det_attn_bwd_fixq_ws_bytes(int B, int H, int Hkv, int S) {
+  return det_attn_bwd_ws_bytes(B, H, Hkv, S) + align_up((size_t)B * H * S * DH * 8, 256);
+}
+
+static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
+                         const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
+                         int window, det_bf16* dq, det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes,
+                         void* stream, bool fixq) {
   if (!dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0)
     return DET_ERR_ARG;
   if (S % 64 || ld % 8 || ld_out % 8 || ld_d % 8 || (long long)B * H > 65535 || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(dout) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
     return DET_ERR_ALIGN;
-  if (!ws || ws_bytes < det_attn_bwd_ws_bytes(B, H, Hkv, S)) return DET_ERR_WORKSPACE;
+  if (!ws || ws_bytes < (fixq ? det_attn_bwd_fixq_ws_bytes(B, H, Hkv, S) : det_attn_bwd_ws_bytes(B, H, Hkv, S)))
+    return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const int G = H / Hkv;
   const size_t matP = align_up((size_t)B * H * S * S * 4, 256), matS = align_up((size_t)B * H * S * S * 2, 256);
@@ -508,9 +514,28 @@ extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_b
   p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = H; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
   p.A = dSt; p.B = k; p.ldb = ld; p.b_b = (long long)S * ld; p.b_h = DH; p.b_div = G;
   p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
-  rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux ? aux->s[1] : st);
+  if (fixq) {
+    // per block of 128 keys the ordered f32 sum, accumulated over the blocks in 64-bit fixed point (Sec. 3.2)
+    p.fix = reinterpret_cast<long long*>((uint8_t*)ws + det_attn_bwd_ws_bytes(B, H, Hkv, S));
+    rc = ogemm_wb_launch<CONTIG, STRIDED, false, true, true>(p, B * H, aux ? aux->s[1] : st);
+  } else {
+    rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux ? aux->s[1] : st);
+  }
   if (rc != DET_OK) return rc;
   if (!aux_join(st, aux)) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();
   return DET_OK;
+}
+
+extern "C" int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
+                            const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
+                            int window, det_bf16* dq, det_bf16* dk, det_bf16* dv, int ld_d, void* ws, size_t ws_bytes,
+                            void* stream) {
+  return attn_bwd_impl(dout, q, k, v, out, lse, ld, ld_out, B, H, Hkv, S, window, dq, dk, dv, ld_d, ws, ws_bytes, stream, false);
+}
+extern "C" int det_attn_bwd_fixq(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
+                                 const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
+                                 int window, det_bf16* dq, det_bf16* dk, det_bf16* dv, int ld_d, void* ws,
+                                 size_t ws_bytes, void* stream) {
+  return attn_bwd_impl(dout, q, k, v, out, lse, ld, ld_out, B, H, Hkv, S, window, dq, dk, dv, ld_d, ws, ws_bytes, stream, true);
 }

@@ -73,6 +73,9 @@ struct OgemmArgs {
   int window;           // sliding window W (multiple of 128; 0 = none): only |query - key| < W contributes
   int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
                         // (with a window, mode 1 also stops at c < i0 + W + 128 and mode 2 starts at c >= i0 - W)
+  // fixed-point variant (k_ogemm_wb<..., FIXQ = true>): scratch of I * J signed 64-bit words per batch index; every 128
+  // contraction indices the f32 accumulators are converted (48 fractional bits) and added to it
+  long long* fix;
 };
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -340,7 +343,20 @@ __device__ __forceinline__ void slab_mac_8x16n(const float (*As)[OT + 4], const 
   }
 }
 
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+// f32 -> signed 64-bit fixed point with 48 fractional bits: round to nearest even, saturate, NaN -> 0
+__device__ __forceinline__ long long fix48(float u) {
+  const float t = fmul(u, 0x1p48f);
+  if (t != t) return 0;
+  if (t >= 0x1p63f) return 0x7fffffffffffffffll;
+  if (t <= -0x1p63f) return (long long)0x8000000000000000ull;
+  return __float2ll_rn(t);
+}
+__device__ __forceinline__ float unfix48(long long a) { return fmul(__ll2float_rn(a), 0x1p-48f); }
+
+// FIXQ: the contraction is cut into blocks of 128 indices (from the first index of the tile's range); each block's
+// ordered f32 sum starts from +0 and is added, converted to 64-bit fixed point, to a thread-private accumulator in
+// global scratch (it stays in L2 between the blocks); the output is the converted total.
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, bool FIXQ = false>
 __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
@@ -434,6 +450,35 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
     else slab_mac_8x16n<true>(As[slot], Bs[slot], ty, tx, acc);
     __syncwarp();
     if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    if (FIXQ && ((s & 7) == 7 || s == nslab - 1)) {
+      const bool first = s < 8, last = s == nslab - 1;
+      long long* fx = p.fix + (size_t)zidx * I * J;
+#pragma unroll
+      for (int a = 0; a < 8; ++a) {
+        const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int c = j0 + g * 32 + tx * 4;
+          if (r < I && c < J) {
+            longlong2* f2 = reinterpret_cast<longlong2*>(fx + (size_t)r * J + c);
+            longlong2 v0 = make_longlong2(0, 0), v1 = make_longlong2(0, 0);
+            if (!first) { v0 = f2[0]; v1 = f2[1]; }
+            v0.x = (long long)((unsigned long long)v0.x + (unsigned long long)fix48(acc[a][2 * g].x));
+            v0.y = (long long)((unsigned long long)v0.y + (unsigned long long)fix48(acc[a][2 * g].y));
+            v1.x = (long long)((unsigned long long)v1.x + (unsigned long long)fix48(acc[a][2 * g + 1].x));
+            v1.y = (long long)((unsigned long long)v1.y + (unsigned long long)fix48(acc[a][2 * g + 1].y));
+            if (last) {
+              acc[a][2 * g] = make_float2(unfix48(v0.x), unfix48(v0.y));
+              acc[a][2 * g + 1] = make_float2(unfix48(v1.x), unfix48(v1.y));
+            } else {
+              f2[0] = v0; f2[1] = v1;
+              acc[a][2 * g] = make_float2(0.0f, 0.0f);
+              acc[a][2 * g + 1] = make_float2(0.0f, 0.0f);
+            }
+          }
+        }
+      }
+    }
   }
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
@@ -456,11 +501,11 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   }
 }
 
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, bool FIXQ = false>
 static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   static bool cfg = false;
   if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16, FIXQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)WB_SMEM) != cudaSuccess)
       return DET_ERR_CUDA;
     cfg = true;
@@ -468,7 +513,7 @@ static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   const bool causal = p.range_mode == 1 || p.range_mode == 2;
   const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
   dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
-  k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WB_THREADS, WB_SMEM, st>>>(p);
+  k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16, FIXQ><<<DET_L(grid), WB_THREADS, WB_SMEM, st>>>(p);
   return DET_OK;
 }
 

@@ -125,7 +125,7 @@ def case_linear(small, which, bwd):
         2.0 * M * N * K, "op"
 
 
-def case_attn(small, bwd, int8pv=False):
+def case_attn(small, bwd, int8pv=False, fixq=False):
     B, H, S = (1, 16, 2048) if small else (4, 16, 2048)
     HD = H * 128
     qkv = randn_bf16(B * S * 3 * HD)
@@ -140,10 +140,11 @@ def case_attn(small, bwd, int8pv=False):
         return fwd, 2 * unit, "flop"
     fwd()
     dout, dqkv = randn_bf16(B * S * HD, 0.1), torch.empty(B * S * 3 * HD, dtype=I16, device="cuda")
-    w = ws(det.det_attn_bwd_ws_bytes(B, H, S))
+    w = ws(det.det_attn_bwd_fixq_ws_bytes(B, H, S) if fixq else det.det_attn_bwd_ws_bytes(B, H, S))
     dp = dqkv.data_ptr()
-    return (lambda: det.det_attn_bwd(dout, p, p + 2 * HD, p + 4 * HD, out, lse, 3 * HD, HD, B, H, S, dp, dp + 2 * HD,
-                                     dp + 4 * HD, 3 * HD, w)), 5 * unit, "flop"
+    bwd_fn = det.det_attn_bwd_fixq if fixq else det.det_attn_bwd
+    return (lambda: bwd_fn(dout, p, p + 2 * HD, p + 4 * HD, out, lse, 3 * HD, HD, B, H, S, dp, dp + 2 * HD,
+                           dp + 4 * HD, 3 * HD, w)), 5 * unit, "flop"
 
 
 def case_lmhead(small, bwd):
@@ -189,6 +190,7 @@ def build_cases():
          "xent_fwd": lambda s: case_xent(s, False), "xent_bwd": lambda s: case_xent(s, True),
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
          "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
+         "attn_bwd_fixq": lambda s: case_attn(s, True, False, True),
          "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_bwd": lambda s: case_lmhead(s, True),
          "accum": case_accum, "adamw": case_adamw, "hash": case_hash}
     for k in LINEAR_SHAPES:

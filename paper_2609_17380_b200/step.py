@@ -42,6 +42,7 @@ class ModelConfig:
     window: int = 0                  # sliding-window width of the local layers (multiple of 128), 0 = all layers full
     full_every: int = 5              # every full_every-th layer and the last one attend to the whole prefix
     pv_int8: bool = False            # forward P.V of every block of 128 keys on the int8 tensor cores
+    dq_fixed: bool = False           # query gradient accumulated over the key blocks in 64-bit fixed point
 
     def as_dict(self):
         return dict(self.__dict__)
@@ -145,7 +146,8 @@ class Replay:
         self.norm, self.coef = e(1, F32), e(1, F32)
         self.status = z(1, I32)
         B, H, S = cfg.micro_batch, cfg.n_heads, cfg.seq
-        wsb = max(det.det_attn_bwd_ws_bytes(B, H, S, Hkv), det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
+        wsb = max(det.det_attn_bwd_fixq_ws_bytes(B, H, S, Hkv) if cfg.dq_fixed else det.det_attn_bwd_ws_bytes(B, H, S, Hkv),
+                  det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
                   det.det_lsq_weight_scale_ws_bytes(2 * Fh, D), det.det_lsq_act_scale_init_ws_bytes(T * max(Fh, D)),
                   det.det_tensor_hash_ws_bytes(g * 4), det.det_sum_ws_bytes(g), 1 << 20,
                   *[det.det_linear_bwd_ws_bytes(T, N, K) for (N, K) in ((QW, D), (D, D), (2 * Fh, D), (D, Fh))])
@@ -345,8 +347,9 @@ class Replay:
             vp, dp = a["qkv"].data_ptr(), d_qkv.data_ptr()
             qp = a["qkr"].data_ptr() if self.head_ops else vp
             with self.span("attn_bwd"):
-                det.det_attn_bwd(d_att, qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), a["att"], a["lse"], QW, D, B, H, S, dp,
-                                 dp + 2 * D, dp + 2 * (D + 128 * Hkv), QW, self.ws, Hkv=Hkv, window=cfg.layer_window(l))
+                bwd = det.det_attn_bwd_fixq if cfg.dq_fixed else det.det_attn_bwd
+                bwd(d_att, qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), a["att"], a["lse"], QW, D, B, H, S, dp,
+                    dp + 2 * D, dp + 2 * (D + 128 * Hkv), QW, self.ws, Hkv=Hkv, window=cfg.layer_window(l))
             if cfg.rope_tables is not None:
                 det.det_rope(d_qkv, QW, T, H + Hkv, S, self.rope_cos, self.rope_sin, 1, d_qkv, QW)
             if cfg.qk_norm:

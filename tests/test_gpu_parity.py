@@ -525,6 +525,35 @@ def test_attention_grouped_and_windowed(det, B, H, Hkv, S, W):
         assert_same_bits(got[:, lo:hi], want[:, lo:hi], name)
 
 
+@pytest.mark.parametrize("B,H,Hkv,S,W,scale", [(1, 2, 2, 64, 0, 0.1), (2, 2, 2, 192, 0, 0.1), (1, 4, 2, 448, 0, 1e-6),
+                                               (1, 2, 1, 640, 256, 0.1), (1, 1, 1, 384, 128, 1e-9),
+                                               (1, 1, 1, 320, 0, 3e4)])
+def test_attention_backward_fixed_point_query_gradient(det, B, H, Hkv, S, W, scale):
+    """dQ accumulated over the key blocks in 64-bit fixed point: all three gradients bit for bit, from gradients so small
+    that most contributions round to a few units of 2^-48 up to ones that saturate the accumulator."""
+    HD, KD = H * 128, Hkv * 128
+    ld = HD + 2 * KD
+    qkv = synth.normal_bf16((B * S, ld), 1.0, seed=16, tid=1)
+    dout = synth.normal_bf16((B * S, HD), scale, seed=16, tid=2)
+    dqkv_in = dev(qkv)
+    base = dqkv_in.data_ptr()
+    out, lse = empty((B * S, HD), np.uint16), empty((B, H, S), F)
+    det.det_attn_fwd(base, base + 2 * HD, base + 2 * (HD + KD), ld, B, H, S, out, HD, lse, Hkv=Hkv, window=W)
+    _sync()
+    oout, olse = oracle.attn_fwd(qkv, B, H, S, Hkv=Hkv, window=W)
+    dqkv = empty((B * S, ld), np.uint16)
+    db = dqkv.data_ptr()
+    w = ws(det.det_attn_bwd_fixq_ws_bytes(B, H, S, Hkv))
+    w.fill_(255)                                       # stale scratch must not leak into the accumulators
+    det.det_attn_bwd_fixq(dev(dout), base, base + 2 * HD, base + 2 * (HD + KD), out, lse, ld, HD, B, H, S, db, db + 2 * HD,
+                          db + 2 * (HD + KD), ld, w, Hkv=Hkv, window=W)
+    _sync()
+    want = oracle.attn_bwd(dout, qkv, oout, olse, B, H, S, Hkv=Hkv, window=W, fixq=True)
+    got = host(dqkv, np.uint16)
+    for name, lo, hi in (("dq", 0, HD), ("dk", HD, HD + KD), ("dv", HD + KD, ld)):
+        assert_same_bits(got[:, lo:hi], want[:, lo:hi], name)
+
+
 @pytest.mark.parametrize("B,H,Hkv,S,W", [(1, 1, 1, 128, 0), (1, 2, 2, 320, 0), (2, 4, 2, 256, 0), (1, 2, 1, 512, 128)])
 def test_attention_forward_int8_pv(det, B, H, Hkv, S, W):
     """P.V of every block on the int8 tensor cores: output and logsumexp bit for bit against the oracle's definition."""

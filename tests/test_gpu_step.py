@@ -35,6 +35,9 @@ def _run(cfg_kwargs, seed=0):
     # forward P.V on the int8 tensor cores (the backward recomputes the weights in full precision)
     dict(n_layers=2, d_model=256, n_heads=2, n_kv_heads=1, ffn=256, vocab=256, seq=256, micro_batch=1, mesh=(2, 1, 1),
          pv_int8=True, window=128),
+    # both integer devices of the attention: int8 P.V forward, query gradient in 64-bit fixed point backward
+    dict(n_layers=2, d_model=256, n_heads=2, n_kv_heads=1, ffn=256, vocab=256, seq=384, micro_batch=1, mesh=(1, 2, 1),
+         pv_int8=True, dq_fixed=True, qk_norm=True, rope=True),
 ])
 def test_step_hashes_match_oracle(kw):
     cfg, got, want = _run(kw)
