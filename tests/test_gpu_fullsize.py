@@ -145,6 +145,18 @@ def test_attention_full_shape_one_head(det):
         assert_same_bits(glse[b, h], ol[i, 0], "lse head")
         for c, name in enumerate(("dq", "dk", "dv")):
             assert_same_bits(gd[r, c * HD + h * 128:c * HD + (h + 1) * 128], od[ro, c * 128:(c + 1) * 128], name)
+    # the same backward with the query gradient accumulated over the 16 key blocks in 64-bit fixed point
+    dqkv2 = empty((B * S, 3 * HD), np.uint16)
+    db2 = dqkv2.data_ptr()
+    det.det_attn_bwd_fixq(dev(dout), base, base + 2 * HD, base + 4 * HD, out, lse, 3 * HD, HD, B, H, S, db2, db2 + 2 * HD,
+                          db2 + 4 * HD, 3 * HD, ws(det.det_attn_bwd_fixq_ws_bytes(B, H, S)))
+    _sync()
+    gd2 = host(dqkv2, np.uint16)
+    assert_same_bits(gd2[:, HD:], gd[:, HD:], "dk, dv of the fixed-point variant")
+    od2 = oracle.attn_bwd(do1, one, oo, ol, 2, 1, S, fixq=True)
+    for i, (b, h) in enumerate(picks):
+        r, ro = slice(b * S, (b + 1) * S), slice(i * S, (i + 1) * S)
+        assert_same_bits(gd2[r, h * 128:(h + 1) * 128], od2[ro, :128], "dq fixed point")
 
 
 def test_norm_and_loss_full_shape(det):
