@@ -8,7 +8,9 @@
  * Conventions (each primitive is one IEEE-754 binary32 round-to-nearest-even
  * operation with flush-to-zero applied to its inputs and to its result):
  *   fadd/fsub/fmul/fdiv/fsqrt  - separate roundings, never fused
- *   fmax2/fmin2                - -0 orders below +0
+ *   fmax2/fmin2                - -0 orders below +0; a NaN operand is ignored (the
+ *                                other operand is returned), so a running maximum
+ *                                does not depend on where a NaN sits in the scan
  *   bf16 widen                 - exact;  narrow - RN-even on the top 16 bits
  *   det_sum                    - level-by-level adjacent pairwise tree; an odd
  *                                trailing element is carried up unchanged
@@ -58,11 +60,15 @@ static inline float fabs1(float a) { return u2f(f2u(ftz(a)) & 0x7fffffffu); }
 static inline float fneg(float a) { return u2f(f2u(ftz(a)) ^ 0x80000000u); }
 static inline float fmax2(float a, float b) {
   a = ftz(a); b = ftz(b);
+  if (a != a) return b;                    /* a NaN operand is ignored (maxNum); two NaNs give NaN */
+  if (b != b) return a;
   if (a == b) return u2f(f2u(a) & f2u(b)); /* max(-0,+0) = +0 */
   return a > b ? a : b;
 }
 static inline float fmin2(float a, float b) {
   a = ftz(a); b = ftz(b);
+  if (a != a) return b;
+  if (b != b) return a;
   if (a == b) return u2f(f2u(a) | f2u(b)); /* min(-0,+0) = -0 */
   return a < b ? a : b;
 }

@@ -412,7 +412,8 @@ def test_linear_backward(det, M, N, K, hb, mode):
     det.det_igemm_set_mode(0)
 
 
-@pytest.mark.parametrize("case", ["zero_grad", "zero_weight", "zero_input", "heavy_tail", "saturated_input"])
+@pytest.mark.parametrize("case", ["zero_grad", "zero_weight", "zero_input", "heavy_tail", "saturated_input", "inf_grad",
+                                  "nan_grad"])
 def test_linear_backward_degenerate(det, case):
     """Degenerate operands of the LSQ linear: all-zero tensors (absmax 0 -> scale 0, codes 0), a gradient with a few
     huge entries (everything else quantises to 0 without the rotation's spreading), activations far outside the
@@ -428,6 +429,10 @@ def test_linear_backward_degenerate(det, case):
         X[:] = 0
     if case == "heavy_tail":
         dY[::37, ::41] = synth.to_bf16(np.array([3.0e4], F))[0]
+    if case == "inf_grad":        # an infinite gradient: both absmax values are infinite, every code is 0 or the clamp of a NaN
+        dY[5, 9] = 0x7F80
+    if case == "nan_grad":        # a NaN does not enter the absmax; its 128-block rotates to NaNs, which quantise like the oracle's
+        dY[100, 200] = 0x7FC0
     osw = oracle.lsq_weight_scale(W)
     osx = oracle.lsq_act_scale_init(X)
     if case == "saturated_input":
@@ -447,6 +452,16 @@ def test_linear_backward_degenerate(det, case):
     _sync()
     assert int(status.item()) == 0
     assert_same_bits(host(Y, np.uint16), oY, "Y")
+    if case == "inf_grad":
+        # infinite steps turn almost every gradient into a NaN; NaNs are compared as NaNs (their payload is not part of
+        # the arithmetic's definition), everything else bit for bit
+        for got, want, name in ((synth.from_bf16(host(gX, np.uint16)), synth.from_bf16(odX), "dX"), (host(gW), odW, "dW"),
+                                (host(gs), ods, "ds_x")):
+            gn, wn = np.isnan(got), np.isnan(want)
+            assert np.array_equal(gn, wn), name + ": NaN positions differ"
+            assert np.array_equal(got[~gn].view(np.uint32), want[~wn].view(np.uint32)), name
+        assert np.isnan(odW).mean() > 0.9
+        return
     assert_same_bits(host(gX, np.uint16), odX, "dX")
     assert_same_bits(host(gW), odW, "dW")
     assert_same_bits(host(gs), ods, "ds_x")

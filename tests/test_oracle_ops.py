@@ -82,6 +82,27 @@ def test_hadamard_butterflies():
     assert np.array_equal(oracle.wht128_f(oracle.wht128_f(x)), 128 * x)
 
 
+def test_gradient_absmax_ignores_nan_wherever_it_sits():
+    """The per-tensor absmax of the rotated gradient operands skips NaNs, so the steps do not depend on the order in which
+    the tensor is scanned: with one NaN in dY the step of each operand is the absmax over the finite rotated values / 127,
+    recomputed here with a Hadamard matrix product (small integers times powers of two: exact in float64)."""
+    M = N = K = 256
+    rng = np.random.default_rng(7)
+    dY = synth.to_bf16((rng.integers(-64, 64, (M, N)) * 2.0 ** -10).astype(F))
+    X = synth.normal_bf16((M, K), 1.0, seed=0, tid=80)
+    W = synth.normal_bf16((N, K), 0.02, seed=0, tid=81)
+    s_x, s_w = oracle.lsq_act_scale_init(X), np.full(N, 2.0 ** -6, F)
+    H = hadamard(128).astype(np.float64)
+    for (r, c) in ((3, 5), (200, 250)):                      # early and late in either scan order
+        d = dY.copy(); d[r, c] = 0x7FC0
+        _, _, _, dbg = oracle.linear_bwd(d, X, W, s_x, s_w, hb=128, debug=True)
+        g = bf(d).astype(np.float64)
+        a = (g * 2.0 ** -6).reshape(M, N // 128, 128) @ H                    # rotation along n, rows scaled by s_w
+        gt = np.einsum("ij,bjn->bin", H, g.reshape(M // 128, 128, N))        # rotation along the token index
+        assert dbg["scales"][0] == F(np.nanmax(np.abs(a))) / F(127.0)
+        assert dbg["scales"][2] == F(np.nanmax(np.abs(gt))) / F(127.0)
+
+
 def _ref_linear_bwd(dY, X, W, s_x, s_w):
     """float64 straight-through reference with exact (unquantised-gradient) contractions."""
     inv = F(1) / s_x[0]

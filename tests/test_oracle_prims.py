@@ -49,6 +49,10 @@ def test_flush_to_zero():
     assert oracle.prim("mul", [F(1 + 2.0 ** -23)], [tiny])[0] == F((1 + 2.0 ** -23) * 2.0 ** -126)
     assert oracle.prim("max", [-0.0], [0.0]).view(np.uint32)[0] == 0
     assert oracle.prim("max", [0.0], [-0.0]).view(np.uint32)[0] == 0
+    # a NaN operand of max is ignored, whichever side it is on (maxNum); only two NaNs give a NaN
+    nan = F("nan")
+    assert oracle.prim("max", [nan], [F(-3.0)])[0] == F(-3.0) and oracle.prim("max", [F(-3.0)], [nan])[0] == F(-3.0)
+    assert np.isnan(oracle.prim("max", [nan], [nan])[0])
 
 
 def test_bf16_roundtrip_and_ties():
