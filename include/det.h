@@ -24,7 +24,11 @@
  *    inputs and results flushed to zero (Sec. 2.1).  Sums run in the fixed pairwise tree "det_sum":
  *    level by level, adjacent elements paired, an odd last element carried up unchanged, so the tree
  *    shape depends only on the length, never on the launch configuration.
- *  - bf16 tensors are passed as uint16_t bit patterns.
+ *  - bf16 tensors are passed as uint16_t bit patterns;
+ *  - operands are expected to be finite.  The LSQ linears, norms, losses and reductions propagate an infinity or a NaN
+ *    exactly as the definition does (max/min ignore a NaN operand; NaN payloads are unspecified); the attention calls
+ *    multiply masked pairs in with weight +0, so a non-finite q, k, v or dout entry can turn more elements of its block
+ *    into NaN than the definition names.  Every finite element is still exact.
  */
 #ifndef DET_H
 #define DET_H
