@@ -127,10 +127,14 @@ static inline float det_exp(float x) {
   return fmul(p, u2f((uint32_t)(k + 127) << 23));
 }
 
-/* log for normal x > 0: x = 2^e m, m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1),
+/* log: the ends of the domain first (0 -> -inf, +inf -> +inf, negative or NaN -> NaN; a flushed subnormal is 0), so that
+ * a non-finite operand stays visible instead of turning into an arbitrary finite number; then for normal x > 0: x = 2^e m, m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1),
  * log m = 2s (1 + z/3 + z^2/5 + z^3/7 + z^4/9), z = s^2. */
 static inline float det_log(float x) {
-  uint32_t u = f2u(ftz(x));
+  x = ftz(x);
+  if (!(x > 0.0f)) return x == 0.0f ? -INFINITY : NAN;   /* log 0 = -inf; a negative argument or a NaN gives NaN */
+  if (x == INFINITY) return x;
+  uint32_t u = f2u(x);
   int e = (int)(u >> 23) - 127;
   float m = u2f((u & 0x007fffffu) | 0x3f800000u);
   if (m > 0x1.6a09e6p+0f) { m = fmul(m, 0.5f); e += 1; }

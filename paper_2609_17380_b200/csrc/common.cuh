@@ -66,9 +66,13 @@ __device__ __forceinline__ float det_exp(float x) {
 // multiply-add is wanted and proven identical; every multiply-then-add whose product must be rounded on its own is
 // written with the scalar intrinsics, which ptxas never contracts.
 
-// log for normal x > 0: x = 2^e m, m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1), z = s^2,
+// log: for normal x > 0, x = 2^e m, m in (sqrt(1/2), sqrt(2)], s = (m-1)/(m+1), z = s^2,
 // log m = 2 s (1 + z/3 + z^2/5 + z^3/7 + z^4/9).
 __device__ __forceinline__ float det_log(float x) {
+  // the ends of the domain first: 0 (a flushed subnormal included) -> -inf, +inf -> +inf, negative or NaN -> NaN
+  // (comparisons flush subnormal operands like every other instruction here)
+  if (!(x > 0.0f)) return x == 0.0f ? __int_as_float(0xff800000) : __int_as_float(0x7fffffff);
+  if (x == __int_as_float(0x7f800000)) return x;
   uint32_t u = __float_as_uint(x);
   int e = (int)(u >> 23) - 127;
   float m = __uint_as_float((u & 0x007fffffu) | 0x3f800000u);

@@ -86,6 +86,35 @@ def test_exp_all_bf16_arguments(det):
     assert_same_bits(host(out), oracle.prim("exp", x), "exp")
 
 
+def test_log_ends_of_the_domain_and_nan_logits(det):
+    """det_log keeps a non-finite or non-positive argument visible; a NaN logit therefore gives a NaN loss, not a finite
+    number that depends on the NaN's payload.  NaNs are compared as NaNs, everything else bit for bit."""
+    import torch
+    x = np.array([0.0, -0.0, 1e-40, np.inf, -1.0, -np.inf, np.nan, 1.0, 2.5, 50304.0], F)
+    out = empty(x.shape, F)
+    det.det_prim(oracle.OPS["log"], dev(x), None, out)
+    _sync()
+    got, want = host(out), oracle.prim("log", x)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.array_equal(got[~np.isnan(got)].view(np.uint32), want[~np.isnan(want)].view(np.uint32))
+    z = synth.normal_f32((6, 1000), 1.0, seed=31, tid=1)
+    z[1, 10] = np.nan
+    z[2, 20] = np.inf
+    z[3, 30] = -np.inf
+    z[4, :] = -np.inf
+    tgt = np.array([5, 7, 9, 11, 13, 999], np.int32)
+    lr, l2, lm, zm = empty((6,), F), empty((6,), F), empty((1,), F), empty((1,), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_xent_fwd(dev(z), dev(tgt), 6, 1000, 1e-4, lr, l2, lm, zm, ws(det.det_xent_ws_bytes(6, 1000)), status)
+    _sync()
+    olr, ol2, olm, ozm, _ = oracle.xent_fwd(z, tgt, 1e-4)
+    for g, w, name in ((host(lr), olr, "loss_row"), (host(l2), ol2, "lse"), (host(lm), olm, "mean")):
+        w = np.asarray(w, F).reshape(g.shape)
+        assert np.array_equal(np.isnan(g), np.isnan(w)), name
+        assert np.array_equal(g[~np.isnan(g)].view(np.uint32), w[~np.isnan(w)].view(np.uint32)), name
+    assert np.isnan(host(lr)[1]) and np.isnan(host(lm)[0])
+
+
 # ------------------------------------------------------------------ sums
 @pytest.mark.parametrize("n", [0, 1, 2, 7, 255, 256, 257, 16383, 16384, 16385, 50304, 1000003, 16384 * 300 + 17])
 def test_det_sum_lengths(det, n):

@@ -118,6 +118,10 @@ def test_log_pins():
     assert ulp_diff(got, F(math.log(50304.0))) <= 2                     # 10.82583988
     x = np.concatenate([np.linspace(1.0, 4.0, 200001), np.logspace(0, 30, 100001)]).astype(F)
     assert ulp_diff(oracle.prim("log", x), np.log(x.astype(np.float64)).astype(F)).max() <= 4
+    # the ends of the domain: a non-finite or non-positive argument stays visible (a NaN logit must not become a finite loss)
+    edge = oracle.prim("log", np.array([0.0, -0.0, 1e-40, np.inf, -1.0, -np.inf, np.nan], F))
+    assert edge[0] == -np.inf and edge[1] == -np.inf and edge[2] == -np.inf and edge[3] == np.inf   # 1e-40 is flushed to 0
+    assert np.isnan(edge[4:]).all()
 
 
 def test_reciprocal_multiply_vs_division():
