@@ -217,7 +217,7 @@ int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, con
  * reading): per block of 128 keys the ordered f32 sum u over the block's keys from +0; its contribution is
  * rne(u * 2^48) as a signed 64-bit integer (saturated at the ends of the range, NaN -> 0); integer additions wrap, so
  * the order of the blocks cannot matter; dq = bf16(f32(acc) * 2^-48) with the conversion rounding to nearest even.
- * dk and dv as in det_attn_bwd.  The workspace (det_attn_bwd_fixq_ws_bytes) adds the accumulators [B*H, S, 128]. */
+ * dk and dv as in det_attn_bwd; the 64-bit accumulators live in registers, so the workspace has det_attn_bwd's size. */
 size_t det_attn_bwd_fixq_ws_bytes(int B, int H, int Hkv, int S);
 int det_attn_bwd_fixq(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,
                       const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S, int window, det_bf16* dq,

@@ -444,10 +444,8 @@ extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S) {
          align_up((size_t)B * H * S * 4, 256) + (Hkv < H ? align_up((size_t)B * Hkv * S * DH * 4, 256) : 0);
 }
 
-// the fixed-point variant adds the signed 64-bit accumulators of the query gradient [B*H, S, 128]
-extern "C" size_t det_attn_bwd_fixq_ws_bytes(int B, int H, int Hkv, int S) {
-  return det_attn_bwd_ws_bytes(B, H, Hkv, S) + align_up((size_t)B * H * S * DH * 8, 256);
-}
+// the fixed-point variant keeps its 64-bit accumulators in registers: no extra scratch
+extern "C" size_t det_attn_bwd_fixq_ws_bytes(int B, int H, int Hkv, int S) { return det_attn_bwd_ws_bytes(B, H, Hkv, S); }
 
 static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v,
                          const det_bf16* out, const float* lse, int ld, int ld_out, int B, int H, int Hkv, int S,
@@ -516,8 +514,7 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
   p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
   if (fixq) {
     // per block of 128 keys the ordered f32 sum, accumulated over the blocks in 64-bit fixed point (Sec. 3.2)
-    p.fix = reinterpret_cast<long long*>((uint8_t*)ws + det_attn_bwd_ws_bytes(B, H, Hkv, S));
-    rc = ogemm_wb_launch<CONTIG, STRIDED, false, true, true>(p, B * H, aux ? aux->s[1] : st);
+    rc = ogemm_fix_launch<CONTIG, STRIDED, false>(p, B * H, aux ? aux->s[1] : st);
   } else {
     rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux ? aux->s[1] : st);
   }

@@ -73,9 +73,6 @@ struct OgemmArgs {
   int window;           // sliding window W (multiple of 128; 0 = none): only |query - key| < W contributes
   int range_mode;       // 0: whole contraction; 1: c >= first row of the tile (causal, per key); 2: c < last row + 1 of the tile
                         // (with a window, mode 1 also stops at c < i0 + W + 128 and mode 2 starts at c >= i0 - W)
-  // fixed-point variant (k_ogemm_wb<..., FIXQ = true>): scratch of I * J signed 64-bit words per batch index; every 128
-  // contraction indices the f32 accumulators are converted (48 fractional bits) and added to it
-  long long* fix;
 };
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -353,10 +350,7 @@ __device__ __forceinline__ long long fix48(float u) {
 }
 __device__ __forceinline__ float unfix48(long long a) { return fmul(__ll2float_rn(a), 0x1p-48f); }
 
-// FIXQ: the contraction is cut into blocks of 128 indices (from the first index of the tile's range); each block's
-// ordered f32 sum starts from +0 and is added, converted to 64-bit fixed point, to a thread-private accumulator in
-// global scratch (it stays in L2 between the blocks); the output is the converted total.
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, bool FIXQ = false>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
 __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   extern __shared__ __align__(16) unsigned char osm[];
   float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
@@ -450,35 +444,6 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
     else slab_mac_8x16n<true>(As[slot], Bs[slot], ty, tx, acc);
     __syncwarp();
     if (lane == 0) mbar_arrive(&bar_empty[slot]);
-    if (FIXQ && ((s & 7) == 7 || s == nslab - 1)) {
-      const bool first = s < 8, last = s == nslab - 1;
-      long long* fx = p.fix + (size_t)zidx * I * J;
-#pragma unroll
-      for (int a = 0; a < 8; ++a) {
-        const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const int c = j0 + g * 32 + tx * 4;
-          if (r < I && c < J) {
-            longlong2* f2 = reinterpret_cast<longlong2*>(fx + (size_t)r * J + c);
-            longlong2 v0 = make_longlong2(0, 0), v1 = make_longlong2(0, 0);
-            if (!first) { v0 = f2[0]; v1 = f2[1]; }
-            v0.x = (long long)((unsigned long long)v0.x + (unsigned long long)fix48(acc[a][2 * g].x));
-            v0.y = (long long)((unsigned long long)v0.y + (unsigned long long)fix48(acc[a][2 * g].y));
-            v1.x = (long long)((unsigned long long)v1.x + (unsigned long long)fix48(acc[a][2 * g + 1].x));
-            v1.y = (long long)((unsigned long long)v1.y + (unsigned long long)fix48(acc[a][2 * g + 1].y));
-            if (last) {
-              acc[a][2 * g] = make_float2(unfix48(v0.x), unfix48(v0.y));
-              acc[a][2 * g + 1] = make_float2(unfix48(v1.x), unfix48(v1.y));
-            } else {
-              f2[0] = v0; f2[1] = v1;
-              acc[a][2 * g] = make_float2(0.0f, 0.0f);
-              acc[a][2 * g + 1] = make_float2(0.0f, 0.0f);
-            }
-          }
-        }
-      }
-    }
   }
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
@@ -501,11 +466,11 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   }
 }
 
-template <int AMODE, int BMODE, bool AF32, bool OUT_BF16, bool FIXQ = false>
+template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
 static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   static bool cfg = false;
   if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16, FIXQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)WB_SMEM) != cudaSuccess)
       return DET_ERR_CUDA;
     cfg = true;
@@ -513,7 +478,132 @@ static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
   const bool causal = p.range_mode == 1 || p.range_mode == 2;
   const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
   dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
-  k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16, FIXQ><<<DET_L(grid), WB_THREADS, WB_SMEM, st>>>(p);
+  k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WB_THREADS, WB_SMEM, st>>>(p);
+  return DET_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Fixed-point variant with the 64-bit accumulators in registers: 128 x 128 tile, eight consumer warps with 8 x 8 register
+// tiles (64 f32 partial sums + 64 signed 64-bit accumulators per thread), four producer warps, one CTA per SM.  After
+// every block of 128 contraction indices the partial sums are converted (48 fractional bits) and added; nothing leaves
+// the registers until the converted total is written.  Same arguments, ranges and batching as k_ogemm_wb.
+// ---------------------------------------------------------------------------------------------------------------
+template <int AMODE, int BMODE, bool AF32>
+__global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_fix(OgemmArgs p) {
+  extern __shared__ __align__(16) unsigned char osm[];
+  float(*As)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(osm);
+  float(*Bs)[OK][OT + 4] = As + WS_STAGES;
+  __shared__ int tiny_s[WS_STAGES][WS_PROD / 32];
+  __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
+  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
+  const int i0 = ti * OT, j0 = blockIdx.x * OT;
+  const int W = p.window;
+  const long long zb = zidx / p.H, zh = zidx % p.H;
+  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
+  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
+  int c_lo = 0, C = p.C;
+  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
+  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
+  const int nslab = (C - c_lo + OK - 1) / OK;
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WS_CONS / 32); }
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid >= WS_CONS) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
+                         : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
+    const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
+    const int pt = tid - WS_CONS, pw = pt >> 5;
+    WsRaw<AMODE, AF32, OT> ra;
+    WsRaw<BMODE, false, OT> rb;
+    if (nslab > 0) {
+      ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, pt, ra);
+      ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo, pt, rb);
+    }
+    for (int s = 0; s < nslab; ++s) {
+      const int slot = s % WS_STAGES;
+      if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
+      bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
+      tiny |= ws_store<BMODE, false, OT>(Bs[slot], pt, rb);
+      if (s + 1 < nslab) {
+        ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, pt, ra);
+        ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, pt, rb);
+      }
+      const int any = __any_sync(0xffffffffu, tiny);
+      if (lane == 0) tiny_s[slot][pw] = any;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_full[slot]);
+    }
+    return;
+  }
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+  const int ty = tid >> 4, tx = tid & 15;
+  float2 acc[8][4];
+  long long fx[8][8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int b = 0; b < 8; ++b) fx[a][b] = 0;
+  }
+  for (int s = 0; s < nslab; ++s) {
+    const int slot = s % WS_STAGES;
+    if (!mbar_wait(&bar_full[slot], (uint32_t)((s / WS_STAGES) & 1), abort_flag, nullptr)) return;
+    const int tiny = tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
+    if (tiny) slab_mac<false, OT>(As[slot], Bs[slot], ty, tx, acc);
+    else slab_mac<true, OT>(As[slot], Bs[slot], ty, tx, acc);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    if ((s & 7) == 7 || s == nslab - 1) {
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          fx[a][2 * b] = (long long)((unsigned long long)fx[a][2 * b] + (unsigned long long)fix48(acc[a][b].x));
+          fx[a][2 * b + 1] = (long long)((unsigned long long)fx[a][2 * b + 1] + (unsigned long long)fix48(acc[a][b].y));
+          acc[a][b] = make_float2(0.0f, 0.0f);
+        }
+    }
+  }
+  uint16_t* out = reinterpret_cast<uint16_t*>(p.out) + zb * p.o_b + zh * p.o_h;
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int r = i0 + (a >> 2) * 64 + ty * 4 + (a & 3);
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      const int c = j0 + g * 64 + tx * 4;
+      if (r < I && c < J) {
+        uint2 u;
+        u.x = pack_bf2(unfix48(fx[a][4 * g]), unfix48(fx[a][4 * g + 1]));
+        u.y = pack_bf2(unfix48(fx[a][4 * g + 2]), unfix48(fx[a][4 * g + 3]));
+        *reinterpret_cast<uint2*>(out + (size_t)r * ldo + c) = u;
+      }
+    }
+  }
+}
+
+template <int AMODE, int BMODE, bool AF32>
+static int ogemm_fix_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
+  static bool cfg = false;
+  if (!cfg) {
+    if (cudaFuncSetAttribute(k_ogemm_fix<AMODE, BMODE, AF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WB_SMEM) !=
+        cudaSuccess)
+      return DET_ERR_CUDA;
+    cfg = true;
+  }
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
+  dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
+  k_ogemm_fix<AMODE, BMODE, AF32><<<DET_L(grid), WS_THREADS, WB_SMEM, st>>>(p);
   return DET_OK;
 }
 
