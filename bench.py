@@ -350,9 +350,9 @@ def run_ours(args):
         n, tot_ms = prof[dom]
         ach = alg[dom][1] / (tot_ms / n / 1e3) / 1e12
         # DRAM traffic per launch group from one ncu capture of the same kernels at B = 1 (read + write, summed over the
-        # P/dS kernel and the three causal contractions: 524.8 MB; it grows in proportion to the batch), see
+        # P/dS kernel and the three causal contractions: 379.3 MB; it grows in proportion to the batch), see
         # profiles/k_attn_sdp_ws_k_ogemm_wb_attn_bwd_small.md
-        traffic = 524.8e6 * B if (dom == "attn_bwd" and args.workload == "config5") else None
+        traffic = 379.3e6 * B if (dom == "attn_bwd" and args.workload == "config5") else None
         roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
                      "traffic": traffic, "peak_source": "148 SMs x 128 FP32 lanes x 2 flop (fused multiply-add) x %.0f MHz"
                      % peaks["sm_max_mhz"]})

@@ -206,7 +206,7 @@ int det_attn_fwd_int8pv(const det_bf16* q, const det_bf16* k, const det_bf16* v,
                         int window, det_bf16* out, int ld_out, float* lse, void* stream, int* status_dev);
 /* dq (H heads), dk, dv (Hkv heads) with leading dimension ld_d; every contraction is one sequential ascending sum
  * from +0; the gradient of a shared key/value head runs over its query heads in ascending order and, within a
- * head, over the queries in ascending order.  ws (16-byte aligned, det_attn_bwd_ws_bytes) holds P (f32) and
+ * head, over the queries in ascending order.  ws (16-byte aligned, det_attn_bwd_ws_bytes) holds bf16(P) and
  * bf16(dS), [B*H, S, S] each, Delta [B*H, S], and for Hkv < H the f32 accumulators carried between query heads. */
 size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S);
 int det_attn_bwd(const det_bf16* dout, const det_bf16* q, const det_bf16* k, const det_bf16* v, const det_bf16* out,

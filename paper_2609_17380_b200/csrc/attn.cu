@@ -6,7 +6,7 @@
 // pairwise tree over its 128 slots (masked slots are +0); P is rounded to bf16 before P.V; P.V is a
 // sequential ascending sum over the tile's keys from +0, then o = o*alpha + u.
 // Backward: P = exp(S*scale - L) recomputed; every one of the five contractions (S, dP, dV, dK, dQ) is a batched
-// ordered contraction with one sequential accumulator per output (ogemm_core.cuh); P (f32) and bf16(dS) go through
+// ordered contraction with one sequential accumulator per output (ogemm_core.cuh); bf16(P) and bf16(dS) go through
 // global scratch, so nothing is accumulated with atomics.
 #include "ogemm_core.cuh"
 
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(256) k_attn_delta(const uint16_t* __restrict__
 // producer warps stream the key and value blocks through a three-slot ring of 16-dimension slabs (a "full" and an
 // "empty" mbarrier per slot, bounded waits); eight consumer warps accumulate S = q.k^T and dP = dO.v^T together (two
 // 8 x 8 register tiles per thread, each logit one ascending sum over the 128 dimensions) and, per key block, apply
-// P = exp(S*scale - L) and dS = (P (dP - Delta)) scale and store P (f32) and bf16(dS).  The producers already fetch
+// P = exp(S*scale - L) and dS = (P (dP - Delta)) scale and store bf16(P) and bf16(dS).  The producers already fetch
 // the next key block while the consumers are in that epilogue, and consumer warps are not coupled to each other.
 // ---------------------------------------------------------------------------------------------
 constexpr size_t SDP_SMEM = (size_t)(2 * DH * (OT + 4) + 2 * WS_STAGES * OK * (OT + 4)) * sizeof(float);
@@ -281,7 +281,7 @@ constexpr size_t SDP_SMEM = (size_t)(2 * DH * (OT + 4) + 2 * WS_STAGES * OK * (O
 __global__ void __launch_bounds__(WS_THREADS, 1)
     k_attn_sdp_ws(const uint16_t* __restrict__ dout, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                   const uint16_t* __restrict__ v, const float* __restrict__ lse, const float* __restrict__ delta, int ld,
-                  int ld_out, int H, int Hkv, int S, int W, float* __restrict__ Pf, uint16_t* __restrict__ dSt) {
+                  int ld_out, int H, int Hkv, int S, int W, uint16_t* __restrict__ Pb, uint16_t* __restrict__ dSt) {
   extern __shared__ __align__(16) unsigned char osm[];
   typedef float(*Full)[OT + 4];
   Full Qs = reinterpret_cast<Full>(osm);                                            // [dim][query]
@@ -403,8 +403,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
           }
         }
         const size_t off = (bh * S + i) * S + jb;
-        *reinterpret_cast<float4*>(Pf + off) = make_float4(pv[0], pv[1], pv[2], pv[3]);
         uint2 u;
+        u.x = pack_bf2(pv[0], pv[1]); u.y = pack_bf2(pv[2], pv[3]);        // P~ = bf16(P) is all the value gradient needs
+        *reinterpret_cast<uint2*>(Pb + off) = u;
         u.x = pack_bf2(dsv[0], dsv[1]); u.y = pack_bf2(dsv[2], dsv[3]);
         *reinterpret_cast<uint2*>(dSt + off) = u;
       }
@@ -437,10 +438,10 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   return DET_OK;
 }
 
-// workspace: P f32 [B*H, S, S], dS bf16 [B*H, S, S], Delta f32 [B*H, S], and with grouped queries the f32 accumulators
+// workspace: bf16(P) and bf16(dS), [B*H, S, S] each, Delta f32 [B*H, S], and with grouped queries the f32 accumulators
 // [B*Hkv, S, 128] that carry dK / dV from one query head of a group to the next
 extern "C" size_t det_attn_bwd_ws_bytes(int B, int H, int Hkv, int S) {
-  return align_up((size_t)B * H * S * S * 4, 256) + align_up((size_t)B * H * S * S * 2, 256) +
+  return 2 * align_up((size_t)B * H * S * S * 2, 256) +
          align_up((size_t)B * H * S * 4, 256) + (Hkv < H ? align_up((size_t)B * Hkv * S * DH * 4, 256) : 0);
 }
 
@@ -461,9 +462,9 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
     return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const int G = H / Hkv;
-  const size_t matP = align_up((size_t)B * H * S * S * 4, 256), matS = align_up((size_t)B * H * S * S * 2, 256);
+  const size_t matP = align_up((size_t)B * H * S * S * 2, 256), matS = matP;
   const size_t dl = align_up((size_t)B * H * S * 4, 256);
-  float* Pf = (float*)ws;
+  uint16_t* Pb = (uint16_t*)ws;
   uint16_t* dSt = (uint16_t*)((uint8_t*)ws + matP);
   float* delta = (float*)((uint8_t*)ws + matP + matS);
   float* carry = (float*)((uint8_t*)ws + matP + matS + dl);
@@ -475,7 +476,7 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
   static bool cfg = false;
   if (!cfg) { if (set_smem((const void*)k_attn_sdp_ws, SDP_SMEM)) return DET_ERR_CUDA; cfg = true; }
   dim3 gsdp(H * B, (S + OT - 1) / OT);
-  k_attn_sdp_ws<<<DET_L(gsdp), WS_THREADS, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, Hkv, S, window, Pf, dSt);
+  k_attn_sdp_ws<<<DET_L(gsdp), WS_THREADS, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, Hkv, S, window, Pb, dSt);
   DET_CHECK_LAUNCH();
   int rc = DET_OK;
   // dV[j,c] = sum over the query heads g of the group, then over queries i >= j ascending, of P~[i,j] dO[i,c];
@@ -490,19 +491,17 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
       OgemmArgs p = {};
       p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = Hkv; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
       p.h_mul = G; p.h_add = g; p.range_mode = 1; p.window = window;
-      p.A = which == 0 ? (const void*)Pf : (const void*)dSt;
+      p.A = which == 0 ? (const void*)Pb : (const void*)dSt;
       if (which == 0) { p.B = dout; p.ldb = ld_out; p.b_b = (long long)S * ld_out; }
       else { p.B = q; p.ldb = ld; p.b_b = (long long)S * ld; }
       p.b_h = DH;
       if (g > 0) { p.acc_in = carry; p.acc_ld = DH; p.acc_b = (long long)Hkv * S * DH; p.acc_h = (long long)S * DH; }
       if (g == G - 1) {
         p.out = which == 0 ? dv : dk; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH;
-        rc = which == 0 ? ogemm_wb_launch<STRIDED, STRIDED, true, true>(p, B * Hkv, sk)     // P is rounded to bf16 as read
-                        : ogemm_wb_launch<STRIDED, STRIDED, false, true>(p, B * Hkv, sk);
+        rc = ogemm_wb_launch<STRIDED, STRIDED, false, true>(p, B * Hkv, sk);
       } else {
         p.out = carry; p.ldo = DH; p.o_b = (long long)Hkv * S * DH; p.o_h = (long long)S * DH;
-        rc = which == 0 ? ogemm_wb_launch<STRIDED, STRIDED, true, false>(p, B * Hkv, sk)
-                        : ogemm_wb_launch<STRIDED, STRIDED, false, false>(p, B * Hkv, sk);
+        rc = ogemm_wb_launch<STRIDED, STRIDED, false, false>(p, B * Hkv, sk);
       }
       if (rc != DET_OK) return rc;
     }
