@@ -310,6 +310,62 @@ static int ogemm_ws_launch(const OgemmArgs& p, cudaStream_t st) {
 constexpr int WB_CONS = 128, WB_THREADS = WB_CONS + WS_PROD;
 constexpr size_t WB_SMEM = (size_t)WS_STAGES * OK * 2 * (OT + 4) * sizeof(float);
 
+// Which tile a CTA of the batched kernels works on, and over which part of the contraction.
+struct WbTile {
+  int i0, j0, zidx, c_lo, C, nslab;
+  long long zb, zh, hA, hB;
+};
+__device__ __forceinline__ WbTile wb_tile(const OgemmArgs& p) {
+  WbTile t;
+  // row tile on the slowest grid index, longest contraction first
+  const bool causal = p.range_mode == 1 || p.range_mode == 2;
+  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
+  t.zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
+  t.i0 = ti * OT;
+  t.j0 = blockIdx.x * OT;
+  const int W = p.window;
+  t.zb = t.zidx / p.H;
+  t.zh = t.zidx % p.H;
+  t.hA = t.zh * (p.h_mul ? p.h_mul : 1) + p.h_add;
+  t.hB = t.hA / (p.b_div ? p.b_div : 1);
+  t.c_lo = 0;
+  t.C = p.C;
+  if (p.range_mode == 1) { t.c_lo = t.i0; if (W) t.C = min(p.C, t.i0 + W + OT); }
+  if (p.range_mode == 2) { t.C = min(p.C, t.i0 + OT); if (W) t.c_lo = max(0, t.i0 - W); }
+  t.nslab = (t.C - t.c_lo + OK - 1) / OK;
+  return t;
+}
+// The producer warps of the batched kernels: 16-deep slabs of both operands into the ring, one slab ahead in registers.
+template <int AMODE, int BMODE, bool AF32>
+__device__ __forceinline__ void wb_produce(const OgemmArgs& p, const WbTile& t, float (*As)[OK][OT + 4], float (*Bs)[OK][OT + 4],
+                                           int (*tiny_s)[WS_PROD / 32], uint64_t* bar_full, uint64_t* bar_empty,
+                                           volatile int* abort_flag, int pt) {
+  const int lane = pt & 31, pw = pt >> 5;
+  const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + t.zb * p.a_b + t.hA * p.a_h)
+                       : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + t.zb * p.a_b + t.hA * p.a_h);
+  const void* B = reinterpret_cast<const uint16_t*>(p.B) + t.zb * p.b_b + t.hB * p.b_h;
+  WsRaw<AMODE, AF32, OT> ra;
+  WsRaw<BMODE, false, OT> rb;
+  if (t.nslab > 0) {
+    ws_fetch<AMODE, AF32, OT>(A, p.I, t.C, p.lda, t.i0, t.c_lo, pt, ra);
+    ws_fetch<BMODE, false, OT>(B, p.J, t.C, p.ldb, t.j0, t.c_lo, pt, rb);
+  }
+  for (int s = 0; s < t.nslab; ++s) {
+    const int slot = s % WS_STAGES;
+    if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
+    bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
+    tiny |= ws_store<BMODE, false, OT>(Bs[slot], pt, rb);
+    if (s + 1 < t.nslab) {
+      ws_fetch<AMODE, AF32, OT>(A, p.I, t.C, p.lda, t.i0, t.c_lo + (s + 1) * OK, pt, ra);
+      ws_fetch<BMODE, false, OT>(B, p.J, t.C, p.ldb, t.j0, t.c_lo + (s + 1) * OK, pt, rb);
+    }
+    const int any = __any_sync(0xffffffffu, tiny);
+    if (lane == 0) tiny_s[slot][pw] = any;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_full[slot]);
+  }
+}
+
 template <bool FUSED>
 __device__ __forceinline__ void slab_mac_8x16n(const float (*As)[OT + 4], const float (*Bs)[OT + 4], int ty, int tx,
                                                float2 (&acc)[8][8]) {
@@ -359,19 +415,10 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
-  // row tile on the slowest grid index, longest contraction first (see k_ogemm)
-  const bool causal = p.range_mode == 1 || p.range_mode == 2;
-  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
-  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
-  const int i0 = ti * OT, j0 = blockIdx.x * OT;
-  const int W = p.window;
-  const long long zb = zidx / p.H, zh = zidx % p.H;
-  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
-  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
-  int c_lo = 0, C = p.C;
-  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
-  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
-  const int nslab = (C - c_lo + OK - 1) / OK;
+  const WbTile t = wb_tile(p);
+  const int i0 = t.i0, j0 = t.j0, nslab = t.nslab;
+  const long long zb = t.zb, zh = t.zh;
+  const int I = p.I, J = p.J, ldo = p.ldo;
   const int tid = threadIdx.x, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WB_CONS / 32); }
@@ -380,32 +427,8 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
   }
   __syncthreads();
   if (tid >= WB_CONS) {
-    // ------------------------------- producers -------------------------------
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-    const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
-                         : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
-    const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
-    const int pt = tid - WB_CONS, pw = pt >> 5;
-    WsRaw<AMODE, AF32, OT> ra;
-    WsRaw<BMODE, false, OT> rb;
-    if (nslab > 0) {
-      ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, pt, ra);
-      ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo, pt, rb);
-    }
-    for (int s = 0; s < nslab; ++s) {
-      const int slot = s % WS_STAGES;
-      if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
-      bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
-      tiny |= ws_store<BMODE, false, OT>(Bs[slot], pt, rb);
-      if (s + 1 < nslab) {
-        ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, pt, ra);
-        ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, pt, rb);
-      }
-      const int any = __any_sync(0xffffffffu, tiny);
-      if (lane == 0) tiny_s[slot][pw] = any;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_full[slot]);
-    }
+    wb_produce<AMODE, BMODE, AF32>(p, t, As, Bs, tiny_s, bar_full, bar_empty, abort_flag, tid - WB_CONS);
     return;
   }
   // --------------------------------- consumers ---------------------------------
@@ -497,18 +520,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_fix(OgemmArgs p) {
   __shared__ __align__(8) uint64_t bar_full[WS_STAGES], bar_empty[WS_STAGES];
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
-  const bool causal = p.range_mode == 1 || p.range_mode == 2;
-  const int ti = causal ? (p.range_mode == 2 ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z) : (int)blockIdx.y;
-  const int zidx = causal ? (int)blockIdx.y : (int)blockIdx.z;
-  const int i0 = ti * OT, j0 = blockIdx.x * OT;
-  const int W = p.window;
-  const long long zb = zidx / p.H, zh = zidx % p.H;
-  const long long hA = zh * (p.h_mul ? p.h_mul : 1) + p.h_add, hB = hA / (p.b_div ? p.b_div : 1);
-  const int I = p.I, J = p.J, lda = p.lda, ldb = p.ldb, ldo = p.ldo;
-  int c_lo = 0, C = p.C;
-  if (p.range_mode == 1) { c_lo = i0; if (W) C = min(p.C, i0 + W + OT); }
-  if (p.range_mode == 2) { C = min(p.C, i0 + OT); if (W) c_lo = max(0, i0 - W); }
-  const int nslab = (C - c_lo + OK - 1) / OK;
+  const WbTile t = wb_tile(p);
+  const int i0 = t.i0, j0 = t.j0, nslab = t.nslab;
+  const long long zb = t.zb, zh = t.zh;
+  const int I = p.I, J = p.J, ldo = p.ldo;
   const int tid = threadIdx.x, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < WS_STAGES; ++s) { mbar_init(&bar_full[s], WS_PROD / 32); mbar_init(&bar_empty[s], WS_CONS / 32); }
@@ -518,30 +533,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_fix(OgemmArgs p) {
   __syncthreads();
   if (tid >= WS_CONS) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-    const void* A = AF32 ? (const void*)(reinterpret_cast<const float*>(p.A) + zb * p.a_b + hA * p.a_h)
-                         : (const void*)(reinterpret_cast<const uint16_t*>(p.A) + zb * p.a_b + hA * p.a_h);
-    const void* B = reinterpret_cast<const uint16_t*>(p.B) + zb * p.b_b + hB * p.b_h;
-    const int pt = tid - WS_CONS, pw = pt >> 5;
-    WsRaw<AMODE, AF32, OT> ra;
-    WsRaw<BMODE, false, OT> rb;
-    if (nslab > 0) {
-      ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo, pt, ra);
-      ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo, pt, rb);
-    }
-    for (int s = 0; s < nslab; ++s) {
-      const int slot = s % WS_STAGES;
-      if (s >= WS_STAGES && !mbar_wait(&bar_empty[slot], (uint32_t)((s / WS_STAGES - 1) & 1), abort_flag, nullptr)) break;
-      bool tiny = ws_store<AMODE, AF32, OT>(As[slot], pt, ra);
-      tiny |= ws_store<BMODE, false, OT>(Bs[slot], pt, rb);
-      if (s + 1 < nslab) {
-        ws_fetch<AMODE, AF32, OT>(A, I, C, lda, i0, c_lo + (s + 1) * OK, pt, ra);
-        ws_fetch<BMODE, false, OT>(B, J, C, ldb, j0, c_lo + (s + 1) * OK, pt, rb);
-      }
-      const int any = __any_sync(0xffffffffu, tiny);
-      if (lane == 0) tiny_s[slot][pw] = any;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_full[slot]);
-    }
+    wb_produce<AMODE, BMODE, AF32>(p, t, As, Bs, tiny_s, bar_full, bar_empty, abort_flag, tid - WS_CONS);
     return;
   }
   asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
