@@ -99,15 +99,112 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0, "source": "fallback"}
 
 
+def profile_traffic(name):
+    """DRAM read + write bytes summed over the launches of one committed ncu summary under profiles/ (the lines
+    `dram__bytes_read.sum` / `dram__bytes_write.sum`), or None if the file is missing."""
+    path = os.path.join(ROOT, "profiles", name)
+    if not os.path.exists(path):
+        return None
+    mult = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    tot, seen = 0.0, 0
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 3 and f[0] in ("dram__bytes_read.sum", "dram__bytes_write.sum") and f[2] in mult:
+            tot += float(f[1]) * mult[f[2]]
+            seen += 1
+    return tot if seen else None
+
+
+def accum_bytes_per_element(accum, shard, rep):
+    """Bytes per gradient element that the pushes of one step really move (Algorithm 1 + 2 as det_grad_accum_push runs
+    them): every push reads the fresh gradient and writes one buffer; it also reads the rank's running sum (k > 0), the
+    running shard sum (end of a rank, shard > 0) and one stacked partial per TreeFold carry (end of a replica)."""
+    streams, stack = 0, []
+    for r in range(shard * rep):
+        for k in range(accum):
+            streams += 2 + (1 if k > 0 else 0)
+            if k == accum - 1:
+                s_ = r % shard
+                streams += 1 if s_ > 0 else 0
+                if s_ == shard - 1:
+                    level = 0
+                    while stack and stack[-1] == level:
+                        stack.pop()
+                        level += 1
+                        streams += 1
+                    stack.append(level)
+    return 4.0 * streams
+
+
+def component_rates_configs_2_3(peaks, iters=5):
+    """The kernel-level workloads of the metric, timed one call at a time (CUDA events, L2 flushed between iterations):
+    the order-fixed reductions (RMSNorm forward/backward on 16384 x 2048 f32, cross-entropy forward/backward on
+    4096 x 50304, global gradient norm over 1.2e9 f32) as GB/s and fraction of the measured copy bandwidth, and the
+    1B-shaped linear set at 16384 tokens, forward and backward, as int8 POP/s and fraction of 4.5 POP/s nominal and of
+    2 x the measured bf16 rate."""
+    import torch
+    from paper_2609_17380_b200 import kbench
+    out = {}
+    for name, fn in (("rmsnorm_fwd", lambda: kbench.case_rmsnorm(False, False)), ("rmsnorm_bwd", lambda: kbench.case_rmsnorm(False, True)),
+                     ("xent_fwd", lambda: kbench.case_xent(False, False)), ("xent_bwd", lambda: kbench.case_xent(False, True)),
+                     ("grad_norm_1.2e9", lambda: kbench.case_grad_norm(False))):
+        call, work, _ = fn()
+        torch.cuda.synchronize()
+        ms = kbench.timeit(call, iters)
+        gbs = work / (ms / 1e3) / 1e9
+        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+        del call
+        torch.cuda.empty_cache()
+    tot = {"fwd": [0.0, 0.0], "bwd": [0.0, 0.0]}
+    for which in kbench.LINEAR_SHAPES:
+        for bwd in (False, True):
+            call, work, _ = kbench.case_linear(False, which, bwd, M=16384)
+            torch.cuda.synchronize()
+            ms = kbench.timeit(call, iters)
+            tops = work / (ms / 1e3) / 1e12
+            key = "linear16k_%s_%s" % ("bwd" if bwd else "fwd", which)
+            out[key] = {"ms": round(ms, 4), "int8_tops": round(tops, 1), "frac_of_4.5POPs": round(tops / 4500.0, 3),
+                        "frac_of_2x_measured_bf16": round(tops / (2.0 * peaks["bf16_tflops"]), 3)}
+            t = tot["bwd" if bwd else "fwd"]
+            t[0] += work
+            t[1] += ms
+            del call
+            torch.cuda.empty_cache()
+    for k, (work, ms) in tot.items():
+        tops = work / (ms / 1e3) / 1e12
+        out["linear16k_%s_set" % k] = {"ms": round(ms, 4), "int8_tops": round(tops, 1), "frac_of_4.5POPs": round(tops / 4500.0, 3),
+                                       "frac_of_2x_measured_bf16": round(tops / (2.0 * peaks["bf16_tflops"]), 3)}
+    out["hbm_peak_used_gbs"] = peaks["hbm_gbs"]
+    out["note"] = "hbm fraction is against the measured copy bandwidth (%s); a read-mostly kernel can read a little above it" % peaks["source"]
+    return out
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start N local ranks, one GPU each, NCCL over 127.0.0.1."""
+    import socket
+    import torch
+    have = torch.cuda.device_count()
+    if have < args.gpus:
+        print("bench.py: --gpus %d asked for, %d visible" % (args.gpus, have), file=sys.stderr)
+        return 2
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus), "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 # ---------------------------------------------------------------------------------------------------------
 def cpu_baseline(kw):
     """The oracle, as it stands, on the host cores: a bounded sample of the same workload, scaled to tokens/s.
 
-    Sample: (a) 8 tokens through embedding + final norm + LM head + loss, forward and backward; (b) one full-width
-    decoder layer (norms, four LSQ int8 linears, 16-head attention at seq 128, SwiGLU, residuals) on 128 tokens,
-    forward and backward; (c) accumulate + clip + AdamW + hash on 4M parameters.  Scaled linearly in tokens, layers
-    and parameters to the full step.  Attention is sampled at seq 128 instead of 2048, so its quadratic part is
-    under-counted: the figure flatters the CPU."""
+    Sample: (a) 48 tokens through embedding + final norm + LM head + loss, forward and backward; (b) one full-width
+    decoder layer (norms, four LSQ int8 linears, SwiGLU, residuals) on 512 tokens, forward and backward, with its
+    attention (four sequences of 128) timed apart and left out; (b2) attention forward + backward of one 16-head sequence
+    at seq 1024; (c) accumulate + clip + AdamW + hash on 4M parameters.  (a), (b) and (c) are scaled linearly in tokens,
+    layers and parameters, (b2) with the number of sequences and with (seq / 1024)^2."""
     import numpy as np
     import oracle as O
     import synth
@@ -349,10 +446,12 @@ def run_ours(args):
     if dom in alg:
         n, tot_ms = prof[dom]
         ach = alg[dom][1] / (tot_ms / n / 1e3) / 1e12
-        # DRAM traffic per launch group from one ncu capture of the same kernels at B = 1 (read + write, summed over the
-        # P/dS kernel and the three causal contractions: 379.3 MB; it grows in proportion to the batch), see
-        # profiles/k_attn_sdp_ws_k_ogemm_wb_attn_bwd_small.md
-        traffic = 379.3e6 * B if (dom == "attn_bwd" and args.workload == "config5") else None
+        # DRAM traffic per launch group from the committed ncu capture of the same kernels at B = 1 (read + write, summed
+        # over the launches of the summary; it grows in proportion to the batch)
+        prof_file = {"attn_bwd": "k_attn_sdp_ws_k_ogemm_wb_attn_bwd_small.md", "attn_fwd": "k_attn_fwd_attn_fwd_small.md"}.get(dom)
+        t1 = profile_traffic(prof_file) if (prof_file and args.workload == "config5") else None
+        traffic = t1 * B if t1 is not None else None
+        roof["traffic_source"] = ("profiles/%s x batch %d" % (prof_file, B)) if t1 is not None else None
         roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
                      "traffic": traffic, "peak_source": "148 SMs x 128 FP32 lanes x 2 flop (fused multiply-add) x %.0f MHz"
                      % peaks["sm_max_mhz"]})
@@ -371,10 +470,17 @@ def run_ours(args):
     if "linear_bwd" in prof:
         n, tot_ms = prof["linear_bwd"]
         extra["linear_bwd_int8_tops"] = 2.0 * 2 * lin_macs_fwd / 4 * n / (tot_ms / 1e3) / 1e12
+        extra["linear_bwd_frac_of_4.5POPs"] = extra["linear_bwd_int8_tops"] / 4500.0
     if "grad_accum" in prof:
         n, tot_ms = prof["grad_accum"]
-        extra["grad_accum_gbs"] = 3.0 * r.n_grad * 4 * n / (tot_ms / 1e3) / 1e9
+        # bytes the pushes really move: single GPU, n timed pushes = n / n_mb steps over the whole gradient; sharded, one
+        # timed fold per step over this rank's slice (the gather that follows it is inside the same span)
+        bpe = accum_bytes_per_element(*cfg.mesh)
+        elems, nsteps = (rep.plan.chunk, n) if sharded else (r.n_grad, n / n_mb)
+        extra["grad_accum_bytes_per_element_per_step"] = bpe
+        extra["grad_accum_gbs"] = bpe * elems * nsteps / (tot_ms / 1e3) / 1e9
         extra["grad_accum_frac_of_hbm"] = extra["grad_accum_gbs"] / peaks["hbm_gbs"]
+        extra["grad_accum_peak_note"] = "against the measured copy bandwidth; a kernel with three or four read streams per write stream can read a little above a 1:1 copy"
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": per_step, "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": "int8 tensor-core GEMMs + f32 ordered arithmetic (bf16 storage)", "data": "synthetic",
@@ -388,6 +494,16 @@ def run_ours(args):
             "roofline": roof, "alu_kernels": all_alu, "kernel_time_shares": shares, "component_rates": extra, "peaks": peaks,
             "wall_s_timed": wall, "device_status": status,
             "state_hash": outs2[-1]["hashes"].get("params_bf16")}
+    if world == 1 and not args.no_component_rates:
+        # free the step's buffers, then time the kernel-level workloads of the metric on their own
+        hash_keep = line["state_hash"]
+        del rep, r, outs, outs2, tok_dev
+        torch.cuda.empty_cache()
+        try:
+            line["component_rates"].update(component_rates_configs_2_3(peaks))
+        except Exception as ex:
+            line["component_rates"]["configs_2_3_error"] = repr(ex)
+        line["state_hash"] = hash_keep
     if world == 1 and not args.no_cpu_baseline:
         try:
             import oracle
@@ -413,9 +529,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=None, help="debug only: fewer layers (the line says REDUCED)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-component-rates", action="store_true",
+                    help="skip the kernel-level workloads (reductions, 16384-token linear set) timed after the step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args)
 

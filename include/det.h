@@ -12,11 +12,15 @@
  *    it returns.  Scratch comes from the caller's `ws` buffer of `ws_bytes` bytes (256-byte aligned),
  *    sized by the matching det_*_ws_bytes() query;
  *  - work is asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream), except
- *    det_tensor_hash which synchronises that stream.  det_linear_bwd, det_attn_bwd and det_lmhead_bwd run
- *    independent kernels of the call side by side on two auxiliary streams per device that the library creates
- *    on first use: they start where `stream` stands when the call is made and `stream` waits for them before
- *    the call returns, so the caller still sees plain stream order.  The library keeps per-device state for this
- *    (and for kernel attributes); calls for one device must not be issued from several host threads at once;
+ *    det_tensor_hash which synchronises that stream (det_tensor_hash_async does not).  det_linear_bwd, det_attn_bwd
+ *    and det_lmhead_bwd run independent kernels of the call side by side on two auxiliary streams per device that
+ *    the library creates on first use: they start where `stream` stands when the call is made and `stream` waits
+ *    for them on every way out of the call (error returns included), so the caller still sees plain stream order.
+ *    What the library keeps between calls is per DEVICE and set up under a lock on first use there: those two streams,
+ *    the one-time opt-in of each kernel for large shared memory, the SM count, and the address of det_sum_static's
+ *    scratch.  None of it outlives a cudaDeviceReset (do not call the library again after one).  No mode or option
+ *    is process-wide.  Calls for one device may come from several host threads, except that two calls of the three
+ *    functions above on one device at the same time would share the auxiliary streams: give those one thread per device;
  *  - data-dependent scalars (LSQ steps, norms, losses) are device scalars so that no call forces a sync;
  *  - device-detected conditions (bad target index, a bounded wait that expired, a non-finite norm) are
  *    OR-ed into *status_dev (device int, may be NULL) as DET_DEV_* bits; kernels never trap;
@@ -60,14 +64,8 @@ typedef enum { DET_F32 = 0, DET_BF16 = 1 } det_dtype;
 
 /* library / device information: returns the number of SMs of the current device (or a negative status) */
 int det_device_sm_count(void);
-/* number of kernels this library has launched in this process so far (host-side counter, not thread-safe) */
+/* number of kernels this library has launched in this process so far (host-side atomic counter) */
 unsigned long long det_launch_count(void);
-
-/* ---- primitives (test hook) ---------------------------------------------------------------------
- * Elementwise evaluation of one primitive of Sec. 2.1 on device arrays: op 0 add, 1 sub, 2 mul, 3 div,
- * 4 sqrt(a), 5 det_exp(a), 6 det_log(a), 7 max, 8 bf16 round trip of a, 9 unfused a*b+b.  b may be NULL
- * for unary ops.  Lets a test compare the device arithmetic with the CPU statement of the same rule. */
-int det_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream);
 
 /* ---- order-fixed sums (Sec. 2.1 "Reduction order") ----------------------------------------------- */
 /* out[0] = det_sum_i x[i]^2 (squares == 1) or det_sum_i x[i] (squares == 0).  n >= 0. */
@@ -133,19 +131,6 @@ size_t det_linear_bwd_ws_bytes(int M, int N, int K);
 int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, const det_bf16* W, const int8_t* qWt_bwd,
                    const float* s_x, const float* s_w, const float* s_u, int M, int N, int K, int hadamard_block,
                    det_bf16* dX, float* dW, float* ds_x, void* ws, size_t ws_bytes, void* stream, int* status_dev);
-/* exact int8 x int8 -> int32 contraction C[i,j] = sum_k A[i,k] B[j,k] (tcgen05); test hook for the GEMM core.
- * I % 128 == 0, J % 128 == 0, K % 128 == 0. */
-/* Test hook: mode 0 lets the GEMM use two-CTA 256 x 256 tiles (tcgen05 cta_group::2) whenever both output dimensions
- * are multiples of 256; mode 1 forces the one-CTA kernel.  Results are identical (integer accumulation is exact).
- * Process-wide, not thread-safe. */
-int det_igemm_set_mode(int mode);
-/* Self-test of the bounded wait used by every kernel that waits on an mbarrier (TMA loads, tensor-core commits): one
- * warp waits on a barrier that nothing completes; after limit_cycles SM clocks (at most 4e9) the wait gives up, ORs
- * DET_DEV_TIMEOUT into *status_dev (device int) and the kernel returns, leaving the context usable.  No counterpart in
- * the paper: it exists so that the time-out path can be exercised without making a real kernel hang. */
-int det_selftest_wait_timeout(int* status_dev, long long limit_cycles, void* stream);
-int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream, int* status_dev);
-
 /* ---- RMSNorm (Sec. 3.1 "RMSNorm", FP32 internals) -------------------------------------------------
  * y = (x * rstd) * gamma, rstd = 1 / sqrt(det_sum(x^2) * (1/D) + eps); gamma NULL = gain-free.
  * io: dtype of x, y, gamma, dy, dx (DET_F32 or DET_BF16); rstd f32 [rows]; D % 8 == 0, D <= 8192. */

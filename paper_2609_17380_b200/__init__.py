@@ -90,8 +90,8 @@ def det_launch_count():
     return load().det_launch_count()
 
 
-def det_prim(op, a, b, out):
-    _check("det_prim", load().det_prim(C.c_int(op), _ptr(a), _ptr(b), _ptr(out), C.c_size_t(a.numel()), _stream()))
+def det_test_prim(op, a, b, out):
+    _check("det_test_prim", load().det_test_prim(C.c_int(op), _ptr(a), _ptr(b), _ptr(out), C.c_size_t(a.numel()), _stream()))
 
 
 # ---- sums, norm, clip -----------------------------------------------------------------------------------
@@ -178,17 +178,13 @@ def det_linear_bwd(dY, X, qX, W, qWt_bwd, s_x, s_w, s_u, M, N, K, hadamard_block
         C.c_int(K), C.c_int(hadamard_block), _ptr(dX), _ptr(dW), _ptr(ds_x), *_ws(ws), _stream(), _ptr(status_dev)))
 
 
-def det_selftest_wait_timeout(status_dev, limit_cycles):
-    _check("det_selftest_wait_timeout", load().det_selftest_wait_timeout(_ptr(status_dev), C.c_longlong(limit_cycles), _stream()))
+def det_test_wait_timeout(status_dev, limit_cycles):
+    _check("det_test_wait_timeout", load().det_test_wait_timeout(_ptr(status_dev), C.c_longlong(limit_cycles), _stream()))
 
 
-def det_igemm_set_mode(mode):
-    _check("det_igemm_set_mode", load().det_igemm_set_mode(C.c_int(mode)))
-
-
-def det_igemm_tn(A, B, I, J, K, Cout, status_dev=None):
-    _check("det_igemm_tn", load().det_igemm_tn(_ptr(A), _ptr(B), C.c_int(I), C.c_int(J), C.c_int(K), _ptr(Cout), _stream(),
-                                               _ptr(status_dev)))
+def det_test_igemm_tn(A, B, I, J, K, Cout, force_one_cta=0, status_dev=None):
+    _check("det_test_igemm_tn", load().det_test_igemm_tn(_ptr(A), _ptr(B), C.c_int(I), C.c_int(J), C.c_int(K), _ptr(Cout),
+                                                         C.c_int(force_one_cta), _stream(), _ptr(status_dev)))
 
 
 # ---- RMSNorm, cross-entropy ---------------------------------------------------------------------------------
@@ -326,6 +322,12 @@ def det_adamw_step(desc, pdtype, p, g, m, v, n):
 
 def det_tensor_hash_ws_bytes(nbytes):
     return load().det_tensor_hash_ws_bytes(C.c_size_t(nbytes))
+
+
+def det_tensor_hash_async(p, nbytes, out32_dev, ws):
+    """Queues the hash; the 32-byte root lands in out32_dev (device) in stream order, nothing synchronises."""
+    _check("det_tensor_hash_async", load().det_tensor_hash_async(_ptr(p), C.c_size_t(nbytes), _ptr(out32_dev), *_ws(ws),
+                                                                 _stream()))
 
 
 def det_tensor_hash(p, nbytes, ws):

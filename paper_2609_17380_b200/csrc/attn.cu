@@ -413,9 +413,6 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
   }
 }
 
-static int set_smem(const void* fn, size_t bytes) {
-  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? 0 : -1;
-}
 
 }  // namespace det
 
@@ -426,11 +423,10 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
   if (!q || !k || !v || !out || !lse || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0) return DET_ERR_ARG;
   if (S % 64 || ld % 8 || ld_out % 8 || ld < H * DH || ld_out < H * DH || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
-  static bool cfg = false;
-  if (!cfg) {
-    if (set_smem((const void*)k_attn_fwd<false>, FWD_SMEM) || set_smem((const void*)k_attn_fwd<true>, FWD_SMEM)) return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once_full = {}, once_win = {};
+  if (dev_ensure_smem(once_full, (const void*)k_attn_fwd<false>, FWD_SMEM) != DET_OK ||
+      dev_ensure_smem(once_win, (const void*)k_attn_fwd<true>, FWD_SMEM) != DET_OK)
+    return DET_ERR_CUDA;
   dim3 grid(H * B, (S + FQ - 1) / FQ);
   if (window) k_attn_fwd<true><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse);
   else k_attn_fwd<false><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, 0, out, ld_out, lse);
@@ -473,8 +469,8 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
   DET_CHECK_LAUNCH();
   // P[i,j] = exp(scale * sum_d q[i,d] k[j,d] - L_i) for visible (i,j) (f32; tiles without a visible pair are never
   // touched) and dS[i,j] = bf16((P[i,j] * (sum_d dO[i,d] v[j,d] - Delta_i)) * scale); both sums ascend over the 128 dims
-  static bool cfg = false;
-  if (!cfg) { if (set_smem((const void*)k_attn_sdp_ws, SDP_SMEM)) return DET_ERR_CUDA; cfg = true; }
+  static DevOnce once_sdp = {};
+  if (dev_ensure_smem(once_sdp, (const void*)k_attn_sdp_ws, SDP_SMEM) != DET_OK) return DET_ERR_CUDA;
   dim3 gsdp(H * B, (S + OT - 1) / OT);
   k_attn_sdp_ws<<<DET_L(gsdp), WS_THREADS, SDP_SMEM, st>>>(dout, q, k, v, lse, delta, ld, ld_out, H, Hkv, S, window, Pb, dSt);
   DET_CHECK_LAUNCH();
@@ -484,9 +480,9 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
   // the two chains then share that scratch and run one after the other.  dV, dK (for G == 1) and dQ are independent of
   // each other and run side by side on auxiliary streams, so that the short blocks at the end of one grid overlap
   // with the long blocks at the start of the next.
-  AuxStreams* aux = aux_fork(st);
+  AuxScope aux(st);   // joined again on every way out
   for (int which = 0; which < 2; ++which) {
-    cudaStream_t sk = (aux && G == 1 && which == 1) ? aux->s[0] : st;
+    cudaStream_t sk = (G == 1 && which == 1) ? aux.aux(0) : st;
     for (int g = 0; g < G; ++g) {
       OgemmArgs p = {};
       p.I = S; p.J = DH; p.C = S; p.lda = S; p.H = Hkv; p.a_b = (long long)H * S * S; p.a_h = (long long)S * S;
@@ -513,12 +509,12 @@ static int attn_bwd_impl(const det_bf16* dout, const det_bf16* q, const det_bf16
   p.out = dq; p.ldo = ld_d; p.o_b = (long long)S * ld_d; p.o_h = DH; p.range_mode = 2; p.window = window;
   if (fixq) {
     // per block of 128 keys the ordered f32 sum, accumulated over the blocks in 64-bit fixed point (Sec. 3.2)
-    rc = ogemm_fix_launch<CONTIG, STRIDED, false>(p, B * H, aux ? aux->s[1] : st);
+    rc = ogemm_fix_launch<CONTIG, STRIDED, false>(p, B * H, aux.aux(1));
   } else {
-    rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux ? aux->s[1] : st);
+    rc = ogemm_wb_launch<CONTIG, STRIDED, false, true>(p, B * H, aux.aux(1));
   }
   if (rc != DET_OK) return rc;
-  if (!aux_join(st, aux)) return DET_ERR_CUDA;
+  if (!aux.join()) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

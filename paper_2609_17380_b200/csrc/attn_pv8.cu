@@ -293,12 +293,8 @@ extern "C" int det_attn_fwd_int8pv(const det_bf16* q, const det_bf16* k, const d
   if (!q || !k || !v || !out || !lse || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0) return DET_ERR_ARG;
   if (S % 64 || ld % 8 || ld_out % 8 || ld < H * PD || ld_out < H * PD || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_attn_fwd_pv8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PV8_SMEM) != cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_attn_fwd_pv8, PV8_SMEM) != DET_OK) return DET_ERR_CUDA;
   dim3 grid(H * B, (S + PQ - 1) / PQ);
   k_attn_fwd_pv8<<<DET_L(grid), PTH, PV8_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse, status_dev);
   DET_CHECK_LAUNCH();

@@ -335,46 +335,41 @@ __global__ void __launch_bounds__(64) k_sha_chunks(const uint8_t* __restrict__ d
   o[1] = make_uint4(bswap(h[4]), bswap(h[5]), bswap(h[6]), bswap(h[7]));
 }
 
-// host-side SHA-256 for the root over the chunk digests
-static const uint32_t hK[64] = {
-    0x428a2f98, 0x71374491, 0xb5c0fbcf, 0xe9b5dba5, 0x3956c25b, 0x59f111f1, 0x923f82a4, 0xab1c5ed5, 0xd807aa98,
-    0x12835b01, 0x243185be, 0x550c7dc3, 0x72be5d74, 0x80deb1fe, 0x9bdc06a7, 0xc19bf174, 0xe49b69c1, 0xefbe4786,
-    0x0fc19dc6, 0x240ca1cc, 0x2de92c6f, 0x4a7484aa, 0x5cb0a9dc, 0x76f988da, 0x983e5152, 0xa831c66d, 0xb00327c8,
-    0xbf597fc7, 0xc6e00bf3, 0xd5a79147, 0x06ca6351, 0x14292967, 0x27b70a85, 0x2e1b2138, 0x4d2c6dfc, 0x53380d13,
-    0x650a7354, 0x766a0abb, 0x81c2c92e, 0x92722c85, 0xa2bfe8a1, 0xa81a664b, 0xc24b8b70, 0xc76c51a3, 0xd192e819,
-    0xd6990624, 0xf40e3585, 0x106aa070, 0x19a4c116, 0x1e376c08, 0x2748774c, 0x34b0bcb5, 0x391c0cb3, 0x4ed8aa4a,
-    0x5b9cca4f, 0x682e6ff3, 0x748f82ee, 0x78a5636f, 0x84c87814, 0x8cc70208, 0x90befffa, 0xa4506ceb, 0xbef9a3f7,
-    0xc67178f2};
-static inline uint32_t hrotr(uint32_t x, int r) { return (x >> r) | (x << (32 - r)); }
-static void host_sha_block(uint32_t h[8], const uint8_t* blk) {
-  uint32_t w[64];
-  for (int i = 0; i < 16; ++i)
-    w[i] = ((uint32_t)blk[4 * i] << 24) | ((uint32_t)blk[4 * i + 1] << 16) | ((uint32_t)blk[4 * i + 2] << 8) | blk[4 * i + 3];
-  for (int i = 16; i < 64; ++i)
-    w[i] = w[i - 16] + (hrotr(w[i - 15], 7) ^ hrotr(w[i - 15], 18) ^ (w[i - 15] >> 3)) + w[i - 7] +
-           (hrotr(w[i - 2], 17) ^ hrotr(w[i - 2], 19) ^ (w[i - 2] >> 10));
-  uint32_t a = h[0], b = h[1], c = h[2], d = h[3], e = h[4], f = h[5], g = h[6], hh = h[7];
-  for (int i = 0; i < 64; ++i) {
-    uint32_t t1 = hh + (hrotr(e, 6) ^ hrotr(e, 11) ^ hrotr(e, 25)) + ((e & f) ^ (~e & g)) + hK[i] + w[i];
-    uint32_t t2 = (hrotr(a, 2) ^ hrotr(a, 13) ^ hrotr(a, 22)) + ((a & b) ^ (a & c) ^ (b & c));
-    hh = g; g = f; f = e; e = d + t1; d = c; c = b; b = a; a = t1 + t2;
-  }
-  h[0] += a; h[1] += b; h[2] += c; h[3] += d; h[4] += e; h[5] += f; h[6] += g; h[7] += hh;
-}
-static void host_sha256(const uint8_t* data, size_t n, uint8_t out[32]) {
+// Root of the tree: SHA-256(the nd <= 128 remaining digests || u64le(nbytes)), one thread (at most 65 compressions).
+__global__ void k_sha_root(const uint8_t* __restrict__ digests, int nd, unsigned long long nbytes, uint8_t* __restrict__ out32) {
   uint32_t h[8] = {0x6a09e667, 0xbb67ae85, 0x3c6ef372, 0xa54ff53a, 0x510e527f, 0x9b05688c, 0x1f83d9ab, 0x5be0cd19};
-  size_t full = n / 64;
-  for (size_t i = 0; i < full; ++i) host_sha_block(h, data + 64 * i);
-  uint8_t tail[128] = {0};
-  size_t rem = n - 64 * full;
-  for (size_t i = 0; i < rem; ++i) tail[i] = data[64 * full + i];
-  tail[rem] = 0x80;
-  size_t tl = (rem + 9 <= 64) ? 64 : 128;
-  unsigned long long bits = (unsigned long long)n * 8ull;
-  for (int i = 0; i < 8; ++i) tail[tl - 1 - i] = (uint8_t)(bits >> (8 * i));
-  host_sha_block(h, tail);
-  if (tl == 128) host_sha_block(h, tail + 64);
-  for (int i = 0; i < 8; ++i) { out[4 * i] = h[i] >> 24; out[4 * i + 1] = h[i] >> 16; out[4 * i + 2] = h[i] >> 8; out[4 * i + 3] = h[i]; }
+  uint32_t w[16];
+  const uint4* d4 = reinterpret_cast<const uint4*>(digests);
+  for (int b = 0; b < nd / 2; ++b) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint4 u = d4[4 * b + k];
+      w[4 * k] = bswap(u.x); w[4 * k + 1] = bswap(u.y); w[4 * k + 2] = bswap(u.z); w[4 * k + 3] = bswap(u.w);
+    }
+    sha_rounds(h, w);
+  }
+  // last block: an odd digest (32 bytes), the length word (8 bytes, little endian), 0x80, zeros, the bit count
+#pragma unroll
+  for (int k = 0; k < 16; ++k) w[k] = 0;
+  int pos = 0;   // words filled
+  if (nd & 1) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const uint4 u = d4[2 * (nd - 1) + k];
+      w[4 * k] = bswap(u.x); w[4 * k + 1] = bswap(u.y); w[4 * k + 2] = bswap(u.z); w[4 * k + 3] = bswap(u.w);
+    }
+    pos = 8;
+  }
+  const uint32_t lo = (uint32_t)nbytes, hi = (uint32_t)(nbytes >> 32);
+  const uint32_t wl = bswap(lo), wh = bswap(hi), pad = 0x80000000u;
+  if (pos == 0) { w[0] = wl; w[1] = wh; w[2] = pad; } else { w[8] = wl; w[9] = wh; w[10] = pad; }
+  const unsigned long long bits = ((unsigned long long)nd * 32ull + 8ull) * 8ull;
+  w[14] = (uint32_t)(bits >> 32);
+  w[15] = (uint32_t)bits;
+  sha_rounds(h, w);
+  uint4* o = reinterpret_cast<uint4*>(out32);
+  o[0] = make_uint4(bswap(h[0]), bswap(h[1]), bswap(h[2]), bswap(h[3]));
+  o[1] = make_uint4(bswap(h[4]), bswap(h[5]), bswap(h[6]), bswap(h[7]));
 }
 
 static double ipow(double b, int e) {
@@ -553,16 +548,16 @@ extern "C" int det_adamw_step(const det_adamw_desc* d, int pdtype, void* p, cons
   return DET_OK;
 }
 
-// Workspace: two areas of level-1 size, ping-ponged by the levels.
+// Workspace: two areas of level-1 size, ping-ponged by the levels, and 256 bytes for the root of the synchronising call.
 static inline size_t hash_l1_bytes(size_t nbytes) { return align_up(((nbytes + 4095) / 4096) * 32 + 32, 256); }
 extern "C" size_t det_tensor_hash_ws_bytes(size_t nbytes) {
-  return hash_l1_bytes(nbytes) + hash_l1_bytes(hash_l1_bytes(nbytes));
+  return hash_l1_bytes(nbytes) + hash_l1_bytes(hash_l1_bytes(nbytes)) + 256;
 }
 
-extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes,
-                               void* stream) {
-  if ((nbytes && !p) || !out32_host) return DET_ERR_ARG;
-  if (nbytes && !aligned16(p)) return DET_ERR_ALIGN;
+extern "C" int det_tensor_hash_async(const void* p, size_t nbytes, uint8_t* out32_dev, void* ws, size_t ws_bytes,
+                                     void* stream) {
+  if ((nbytes && !p) || !out32_dev) return DET_ERR_ARG;
+  if ((nbytes && !aligned16(p)) || !aligned16(out32_dev)) return DET_ERR_ALIGN;
   if (ws_bytes < det_tensor_hash_ws_bytes(nbytes) || !ws || !aligned16(ws)) return DET_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* a = (uint8_t*)ws;
@@ -577,11 +572,20 @@ extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host
     uint8_t* t = a; a = b; b = t;
     nc = m;
   }
-  uint8_t host[128 * 32 + 8];
-  if (nc && cudaMemcpyAsync(host, a, nc * 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DET_ERR_CUDA;
+  k_sha_root<<<DET_L(1), 1, 0, st>>>(a, (int)nc, (unsigned long long)nbytes, out32_dev);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" int det_tensor_hash(const void* p, size_t nbytes, uint8_t* out32_host, void* ws, size_t ws_bytes,
+                               void* stream) {
+  if (!out32_host) return DET_ERR_ARG;
+  if (ws_bytes < det_tensor_hash_ws_bytes(nbytes) || !ws || !aligned16(ws)) return DET_ERR_WORKSPACE;
+  uint8_t* root = (uint8_t*)ws + det_tensor_hash_ws_bytes(nbytes) - 256;
+  int rc = det_tensor_hash_async(p, nbytes, root, ws, ws_bytes, stream);
+  if (rc != DET_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(out32_host, root, 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DET_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return DET_ERR_CUDA;
-  unsigned long long nn = nbytes;
-  for (int i = 0; i < 8; ++i) host[nc * 32 + i] = (uint8_t)(nn >> (8 * i));
-  host_sha256(host, nc * 32 + 8, out32_host);
   return DET_OK;
 }

@@ -14,6 +14,7 @@
 // work, lets in-flight copies land, frees its TMEM and returns.
 #include "tc05.cuh"
 #include "internal.h"
+#include "../../include/det_test.h"
 
 namespace det {
 
@@ -550,18 +551,10 @@ template <int BN, int EPI>
 static int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const EpiParams& ep, int I, int J, int K, int* status,
                       cudaStream_t st) {
   constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 1024;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(k_igemm<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return DET_ERR_CUDA;
-    configured = true;
-  }
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_igemm<BN, EPI>, smem) != DET_OK) return DET_ERR_CUDA;
+  const int sms = dev_sm_count();
+  if (sms <= 0) return DET_ERR_CUDA;
   const int tiles = (I / BM) * (J / BN);
   const int grid = tiles < sms ? tiles : sms;
   k_igemm<BN, EPI><<<DET_L(grid), GEMM_THREADS, smem, st>>>(ta, tb, ep, I, J, K, status);
@@ -573,18 +566,10 @@ template <int EPI>
 static int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const EpiParams& ep, int I, int J, int K, int* status,
                        cudaStream_t st) {
   constexpr size_t smem = (size_t)STAGES2 * (2 * 128 * BK) + 8 * 4096 + 1024;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(k_igemm2<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return DET_ERR_CUDA;
-    configured = true;
-  }
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_igemm2<EPI>, smem) != DET_OK) return DET_ERR_CUDA;
+  const int sms = dev_sm_count();
+  if (sms < 2) return DET_ERR_CUDA;
   const int tiles = (I / 256) * (J / BN2);
   int clusters = sms / 2;
   if (tiles < clusters) clusters = tiles;
@@ -593,19 +578,16 @@ static int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const EpiPa
   return DET_OK;
 }
 
-// 0: automatic (two-CTA 256 x 256 tiles when both dimensions are multiples of 256); 1: always the one-CTA kernel
-static int g_gemm_mode = 0;
-void igemm_set_mode(int mode) { g_gemm_mode = mode; }
-
+// Two-CTA 256 x 256 tiles when both output dimensions are multiples of 256 (unless force_one_cta), else the one-CTA kernel.
 int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
-                 cudaStream_t st) {
+                 cudaStream_t st, int force_one_cta) {
   if (!A || !B || I <= 0 || J <= 0 || K <= 0) return DET_ERR_ARG;
   if (I % BM || J % 128 || K % BK) return DET_ERR_SHAPE;
   if (K >= (1 << 17)) return DET_ERR_RANGE;
   if (!aligned16(A) || !aligned16(B)) return DET_ERR_ALIGN;
   const int bn = (J % 256 == 0) ? 256 : 128;
   CUtensorMap ta, tb;
-  if (g_gemm_mode == 0 && I % 256 == 0 && J % 256 == 0) {
+  if (!force_one_cta && I % 256 == 0 && J % 256 == 0) {
     if (!make_map(&ta, A, I, K, 128) || !make_map(&tb, B, J, K, 128)) return DET_ERR_CUDA;
     switch (epi) {
       case EPI_RAW: return launch_pair<EPI_RAW>(ta, tb, ep, I, J, K, status, st);
@@ -648,24 +630,18 @@ __global__ void k_selftest_wait(int* status, long long limit) {
   mbar_wait(&bar, 0, &abort_s, status, limit);
 }
 
-extern "C" int det_selftest_wait_timeout(int* status_dev, long long limit_cycles, void* stream) {
+extern "C" int det_test_wait_timeout(int* status_dev, long long limit_cycles, void* stream) {
   if (!status_dev || limit_cycles <= 0 || limit_cycles > 4000000000ll) return DET_ERR_ARG;
   k_selftest_wait<<<DET_L(1), 32, 0, (cudaStream_t)stream>>>(status_dev, limit_cycles);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }
 
-extern "C" int det_igemm_set_mode(int mode) {
-  if (mode != 0 && mode != 1) return DET_ERR_ARG;
-  igemm_set_mode(mode);
-  return DET_OK;
-}
-
-extern "C" int det_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, void* stream,
-                            int* status_dev) {
+extern "C" int det_test_igemm_tn(const int8_t* A, const int8_t* B, int I, int J, int K, int32_t* C, int force_one_cta,
+                                 void* stream, int* status_dev) {
   if (!C) return DET_ERR_ARG;
   if (!aligned16(C)) return DET_ERR_ALIGN;
   EpiParams ep = {};
   ep.out = C;
-  return igemm_launch(EPI_RAW, A, B, I, J, K, ep, status_dev, (cudaStream_t)stream);
+  return igemm_launch(EPI_RAW, A, B, I, J, K, ep, status_dev, (cudaStream_t)stream, force_one_cta);
 }

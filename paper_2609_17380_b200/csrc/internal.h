@@ -38,8 +38,26 @@ struct AuxStreams {
 };
 AuxStreams* aux_fork(cudaStream_t st);
 bool aux_join(cudaStream_t st, AuxStreams* a);
+// Joins the auxiliary streams on every way out of a call that forked them (error returns included), so that the
+// caller's stream never keeps an unjoined fork.
+struct AuxScope {
+  cudaStream_t st;
+  AuxStreams* a;
+  AuxScope(cudaStream_t s) : st(s), a(aux_fork(s)) {}
+  ~AuxScope() { if (a) aux_join(st, a); }
+  cudaStream_t aux(int i) const { return a ? a->s[i] : st; }
+  bool join() { AuxStreams* t = a; a = nullptr; return aux_join(st, t); }
+};
+
+// Kernel attributes and the SM count belong to a device, not to the process: DevOnce remembers per device whether a
+// kernel's opt-in for large dynamic shared memory has been made there.  Both helpers act on the CURRENT device.
+constexpr int MAX_DEVICES = 64;
+struct DevOnce { bool done[MAX_DEVICES]; };
+int dev_ensure_smem(DevOnce& once, const void* fn, size_t bytes);  // DET_OK or DET_ERR_CUDA
+int dev_sm_count();                                                 // SMs of the current device (0 on error)
 
 // C[i,j] = sum_k A[i,k] B[j,k] on the tensor cores with the chosen epilogue; host-side checks included
+// force_one_cta != 0 keeps the one-CTA kernel even where the two-CTA tiles would apply (the results are identical)
 int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
-                 cudaStream_t st);
+                 cudaStream_t st, int force_one_cta = 0);
 }  // namespace det

@@ -524,21 +524,18 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   const unsigned g1 = (unsigned)((ngrp + 7) / 8);
   dim3 gG(N / 128, M / 128), gZ(K / 128, M / 128);
   if (rot) {
-    static bool cfg = false;
-    if (!cfg) {
-      if (cudaFuncSetAttribute(k_prep_dy<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-          cudaFuncSetAttribute(k_prep_dy<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess)
-        return DET_ERR_CUDA;
-      cfg = true;
-    }
+    static DevOnce once0 = {}, once1 = {};
+    if (dev_ensure_smem(once0, (const void*)k_prep_dy<0>, PREP_SMEM) != DET_OK ||
+        dev_ensure_smem(once1, (const void*)k_prep_dy<1>, PREP_SMEM) != DET_OK)
+      return DET_ERR_CUDA;
     // the rotation of the saved int8 activations does not depend on dY: it runs beside the two passes over dY
-    AuxStreams* az = aux_fork(st);
-    cudaStream_t sz = az ? az->s[1] : st;
+    AuxScope az(st);
+    cudaStream_t sz = az.aux(1);
     k_prep_dy<0><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, nullptr, nullptr);
     k_rotc<false, 0, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, nullptr);
     k_prep_dy<1><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, Aq, GqT);
     k_rotc<false, 1, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, ZqT);
-    if (!aux_join(st, az)) return DET_ERR_CUDA;
+    if (!az.join()) return DET_ERR_CUDA;
   } else {
     k_rot_rows<0, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
     k_rotc<true, 0, false><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, nullptr);
@@ -551,7 +548,7 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   // The two gradient GEMMs are independent.  Each is a persistent grid whose blocks leave as their tiles run out, so the
   // weight-gradient GEMM, queued on an auxiliary stream, moves onto the SMs that the input-gradient GEMM's last
   // partial round leaves idle.
-  AuxStreams* aux = aux_fork(st);
+  AuxScope aux(st);   // joined again on every way out
   // grad wrt W: [N,K] = G_q^T [N,M] . (Z_q^T [K,M])^T
   EpiParams ew = {};
   ew.out = dW; ew.s_x = s_x; ew.s_w = s_w; ew.amax1 = amax + 1; ew.amax2 = rot ? amax + 2 : nullptr; ew.ref = W; ew.rot = rotf;
@@ -560,12 +557,12 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   ex.out = dX; ex.s_x = s_x; ex.amax1 = amax + 0; ex.s_u = s_u; ex.ref = X; ex.rot = rotf; ex.ds_partial = partial;
   int rc = igemm_launch(EPI_DX, Aq, qWt_bwd, M, K, N, ex, status_dev, st);
   if (rc != DET_OK) return rc;
-  rc = igemm_launch(EPI_DW, GqT, ZqT, N, K, M, ew, status_dev, aux ? aux->s[0] : st);
+  rc = igemm_launch(EPI_DW, GqT, ZqT, N, K, M, ew, status_dev, aux.aux(0));
   if (rc != DET_OK) return rc;
   const size_t np = (size_t)M * (K / 128);
   sum_launch(partial, np, 0, sscr, sscr + 64, st);
   k_dsx_finish<<<DET_L(1), 1, 0, st>>>(sscr, (float)(1.0 / sqrt((double)M * (double)K * 127.0)), ds_x);
   DET_CHECK_LAUNCH();
-  if (!aux_join(st, aux)) return DET_ERR_CUDA;
+  if (!aux.join()) return DET_ERR_CUDA;
   return DET_OK;
 }

@@ -497,12 +497,8 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
     k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 512, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
     return DET_OK;
   }
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_rmsnorm_bwd8<BF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 2048 * 4) != cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_rmsnorm_bwd8<BF, true>, 8 * 2048 * 4) != DET_OK) return DET_ERR_CUDA;
   const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
   float* partial8 = ws;
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);

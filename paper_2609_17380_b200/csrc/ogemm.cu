@@ -39,15 +39,15 @@ extern "C" int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det
   if (K % 16 || V % 16 || M % 8) return DET_ERR_SHAPE;
   if (!aligned16(dlogits) || !aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW)) return DET_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
-  AuxStreams* aux = aux_fork(st);   // the auxiliary stream starts where the caller's stream stands now
+  AuxScope aux(st);   // the auxiliary streams start where the caller's stream stands now; joined on every way out
   // dH[m,k] = sum over v ascending of bf16(dlogits[m,v]) * W[v,k]
   int rc = ogemm_ws_launch<CONTIG, STRIDED, true, true>(plain_args(dlogits, W, dH, M, K, V, V, K, K, 0), st);
   if (rc != DET_OK) return rc;
   // dW[v,k] (+)= sum over m ascending of bf16(dlogits[m,v]) * H[m,k], beside the first kernel
   rc = ogemm_ws_launch<STRIDED, STRIDED, true, false>(plain_args(dlogits, H, dW, V, K, M, V, K, K, first_chunk ? 0 : 1),
-                                                      aux ? aux->s[0] : st);
+                                                      aux.aux(0));
   if (rc != DET_OK) return rc;
-  if (!aux_join(st, aux)) return DET_ERR_CUDA;
+  if (!aux.join()) return DET_ERR_CUDA;
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -289,13 +289,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_ws(OgemmArgs p) {
 
 template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
 static int ogemm_ws_launch(const OgemmArgs& p, cudaStream_t st) {
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)WS_SMEM) != cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16>, WS_SMEM) != DET_OK) return DET_ERR_CUDA;
   dim3 grid((p.J + WS_TN - 1) / WS_TN, (p.I + OT - 1) / OT, 1);
   k_ogemm_ws<AMODE, BMODE, AF32, OUT_BF16><<<DET_L(grid), WS_THREADS, WS_SMEM, st>>>(p);
   return DET_OK;
@@ -491,13 +486,8 @@ __global__ void __launch_bounds__(WB_THREADS, 2) k_ogemm_wb(OgemmArgs p) {
 
 template <int AMODE, int BMODE, bool AF32, bool OUT_BF16>
 static int ogemm_wb_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)WB_SMEM) != cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_ogemm_wb<AMODE, BMODE, AF32, OUT_BF16>, WB_SMEM) != DET_OK) return DET_ERR_CUDA;
   const bool causal = p.range_mode == 1 || p.range_mode == 2;
   const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
   dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);
@@ -585,13 +575,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) k_ogemm_fix(OgemmArgs p) {
 
 template <int AMODE, int BMODE, bool AF32>
 static int ogemm_fix_launch(const OgemmArgs& p, int batches, cudaStream_t st) {
-  static bool cfg = false;
-  if (!cfg) {
-    if (cudaFuncSetAttribute(k_ogemm_fix<AMODE, BMODE, AF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WB_SMEM) !=
-        cudaSuccess)
-      return DET_ERR_CUDA;
-    cfg = true;
-  }
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_ogemm_fix<AMODE, BMODE, AF32>, WB_SMEM) != DET_OK) return DET_ERR_CUDA;
   const bool causal = p.range_mode == 1 || p.range_mode == 2;
   const unsigned ni = (unsigned)((p.I + OT - 1) / OT);
   dim3 grid((p.J + OT - 1) / OT, causal ? (unsigned)batches : ni, causal ? ni : (unsigned)batches);

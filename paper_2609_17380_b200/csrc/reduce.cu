@@ -5,45 +5,86 @@
 // a warp butterfly finishes the 256-element leaf, eight leaf sums are paired in registers, and the
 // eight warp sums in shared memory.  The chunk sums are reduced by the same kernel until one value
 // is left, so the tree depends on n only.
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
 #include "internal.h"
+#include "../../include/det_test.h"
 
 namespace det {
 
-static unsigned long long g_launches = 0;
-int note_launch() { ++g_launches; return 0; }
+static std::atomic<unsigned long long> g_launches{0};
+int note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); return 0; }
+
+static std::mutex g_dev_mutex;
 
 AuxStreams* aux_fork(cudaStream_t st) {
-  static std::mutex mu;
-  static AuxStreams table[64] = {};
+  static AuxStreams table[MAX_DEVICES] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
   AuxStreams* a = &table[dev];
   {
-    std::lock_guard<std::mutex> lock(mu);
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!a->ok) {
-      for (int i = 0; i < 2; ++i) {
-        if (cudaStreamCreateWithFlags(&a->s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&a->join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      // all or nothing: what a failed attempt created is destroyed again, so a later call starts from scratch
+      AuxStreams t = {};
+      int ns = 0, ne = 0;
+      bool good = true, have_fork = false;
+      for (int i = 0; i < 2 && good; ++i) {
+        good = cudaStreamCreateWithFlags(&t.s[i], cudaStreamNonBlocking) == cudaSuccess;
+        if (good) ++ns;
+        if (good) { good = cudaEventCreateWithFlags(&t.join[i], cudaEventDisableTiming) == cudaSuccess; if (good) ++ne; }
       }
-      if (cudaEventCreateWithFlags(&a->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-      a->ok = true;
+      if (good) { good = cudaEventCreateWithFlags(&t.fork, cudaEventDisableTiming) == cudaSuccess; have_fork = good; }
+      if (!good) {
+        for (int i = 0; i < ns; ++i) cudaStreamDestroy(t.s[i]);
+        for (int i = 0; i < ne; ++i) cudaEventDestroy(t.join[i]);
+        if (have_fork) cudaEventDestroy(t.fork);
+        cudaGetLastError();
+        return nullptr;
+      }
+      t.ok = true;
+      *a = t;
     }
   }
   if (cudaEventRecord(a->fork, st) != cudaSuccess) return nullptr;
+  // if the second wait fails the first auxiliary stream already depends on `st`: still hand the streams out, the
+  // join below is what the caller's stream order needs
   for (int i = 0; i < 2; ++i)
-    if (cudaStreamWaitEvent(a->s[i], a->fork, 0) != cudaSuccess) return nullptr;
+    if (cudaStreamWaitEvent(a->s[i], a->fork, 0) != cudaSuccess) { cudaGetLastError(); return nullptr; }
   return a;
 }
 bool aux_join(cudaStream_t st, AuxStreams* a) {
   if (!a) return true;
+  bool ok = true;
   for (int i = 0; i < 2; ++i)
-    if (cudaEventRecord(a->join[i], a->s[i]) != cudaSuccess || cudaStreamWaitEvent(st, a->join[i], 0) != cudaSuccess) return false;
-  return true;
+    if (cudaEventRecord(a->join[i], a->s[i]) != cudaSuccess || cudaStreamWaitEvent(st, a->join[i], 0) != cudaSuccess) ok = false;
+  return ok;
 }
-unsigned long long launches() { return g_launches; }
+
+int dev_ensure_smem(DevOnce& once, const void* fn, size_t bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return DET_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  if (!once.done[dev]) {
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return DET_ERR_CUDA;
+    }
+    once.done[dev] = true;
+  }
+  return DET_OK;
+}
+int dev_sm_count() {
+  static int sms[MAX_DEVICES] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 0;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms[dev] = 0;
+  return sms[dev];
+}
+unsigned long long launches() { return g_launches.load(std::memory_order_relaxed); }
 
 constexpr int SUM_CHUNK = 16384;
 
@@ -201,7 +242,7 @@ extern "C" int det_device_sm_count(void) {
   return sms;
 }
 
-extern "C" int det_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream) {
+extern "C" int det_test_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream) {
   if (!a || !out || op < 0 || op > 9) return DET_ERR_ARG;
   if (n == 0) return DET_OK;
   k_prim<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(op, a, b, out, n);

@@ -18,7 +18,6 @@ constexpr size_t STATIC_SCRATCH_FLOATS = 65536;  // 256 KiB
 // cudaGetSymbolAddress for the address and hand that to kernels.
 static __device__ __align__(256) float g_sum_scratch[STATIC_SCRATCH_FLOATS];
 
-constexpr int MAX_DEVICES = 64;
 static float* g_scratch_addr[MAX_DEVICES];  // device address of g_sum_scratch on each device, filled on first use
 static std::mutex g_scratch_mutex;
 

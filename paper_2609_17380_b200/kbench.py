@@ -58,6 +58,15 @@ def case_sumsq(small):
     return (lambda: det.det_sum(x, n, 1, out, w)), 4.0 * n, "B"
 
 
+def case_grad_norm(small):
+    """Global L2 norm and clip coefficient over one flat gradient of 1.2e9 f32 ~ N(0, 1e-3)."""
+    n = 100_000_000 if small else 1_200_000_000
+    x = torch.randn(n, device="cuda") * 1e-3
+    norm, coef = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    w = ws(det.det_grad_norm_ws_bytes([x]))
+    return (lambda: det.det_grad_norm([x], 1.0, norm, coef, w)), 4.0 * n, "B"
+
+
 def case_rmsnorm(small, bwd):
     rows, D = 16384, 2048
     x, dy = torch.randn(rows * D, device="cuda"), torch.randn(rows * D, device="cuda")
@@ -109,11 +118,11 @@ def case_igemm(small, which):
     B = torch.randint(-128, 128, (N * K,), dtype=I8, device="cuda")
     C = torch.empty(M * N, dtype=I32, device="cuda")
     status = torch.zeros(1, dtype=I32, device="cuda")
-    return (lambda: det.det_igemm_tn(A, B, M, N, K, C, status)), 2.0 * M * N * K, "op"
+    return (lambda: det.det_test_igemm_tn(A, B, M, N, K, C, 0, status)), 2.0 * M * N * K, "op"
 
 
-def case_linear(small, which, bwd):
-    M = 2048 if small else 8192
+def case_linear(small, which, bwd, M=None):
+    M = M or (2048 if small else 8192)
     N, K = LINEAR_SHAPES[which]
     d = _linear_setup(M, N, K)
     if bwd:
@@ -186,7 +195,7 @@ def case_hash(small):
 
 
 def build_cases():
-    c = {"sumsq": case_sumsq, "rmsnorm_fwd": lambda s: case_rmsnorm(s, False), "rmsnorm_bwd": lambda s: case_rmsnorm(s, True),
+    c = {"sumsq": case_sumsq, "grad_norm": case_grad_norm, "rmsnorm_fwd": lambda s: case_rmsnorm(s, False), "rmsnorm_bwd": lambda s: case_rmsnorm(s, True),
          "xent_fwd": lambda s: case_xent(s, False), "xent_bwd": lambda s: case_xent(s, True),
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
          "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
@@ -197,6 +206,9 @@ def build_cases():
         c["igemm_" + k] = (lambda s, k=k: case_igemm(s, k))
         c["linear_fwd_" + k] = (lambda s, k=k: case_linear(s, k, False))
         c["linear_bwd_" + k] = (lambda s, k=k: case_linear(s, k, True))
+        # the 1B-shaped linear set at 16384 tokens
+        c["linear16k_fwd_" + k] = (lambda s, k=k: case_linear(s, k, False, M=16384))
+        c["linear16k_bwd_" + k] = (lambda s, k=k: case_linear(s, k, True, M=16384))
     return c
 
 

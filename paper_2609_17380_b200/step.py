@@ -145,6 +145,7 @@ class Replay:
         self.lab = e(T, I32)
         self.norm, self.coef = e(1, F32), e(1, F32)
         self.status = z(1, I32)
+        self.roots = z(32 * 8, torch.uint8)        # hash roots of one step, read back with one copy
         B, H, S = cfg.micro_batch, cfg.n_heads, cfg.seq
         wsb = max(det.det_attn_bwd_fixq_ws_bytes(B, H, S, Hkv) if cfg.dq_fixed else det.det_attn_bwd_ws_bytes(B, H, S, Hkv),
                   det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
@@ -379,18 +380,23 @@ class Replay:
                                self.g(self.m, name), self.g(self.v, name), _numel(shape))
 
     def hashes(self, per_tensor=True):
-        out = {}
+        """State hashes of the step (Appendix B).  Every hash is queued on the stream with its root finished on the
+        device; the roots come back in ONE copy, so the whole set costs one synchronisation."""
+        jobs = []
         if per_tensor:
             for name, shape, kind in self.specs:
                 t = self.p(name)
-                out[name] = det.det_tensor_hash(t, t.numel() * t.element_size(), self.ws)
+                jobs.append((name, t, t.numel() * t.element_size()))
         else:
-            out["params_bf16"] = det.det_tensor_hash(self.pbf, self.pbf.numel() * 2, self.ws)
-            out["steps_f32"] = det.det_tensor_hash(self.sx, self.sx.numel() * 4, self.ws)
-        out["grad"] = det.det_tensor_hash(self.gout, self.n_grad * 4, self.ws)
-        out["adam_m"] = det.det_tensor_hash(self.m, self.n_grad * 4, self.ws)
-        out["adam_v"] = det.det_tensor_hash(self.v, self.n_grad * 4, self.ws)
-        return out
+            jobs.append(("params_bf16", self.pbf, self.pbf.numel() * 2))
+            jobs.append(("steps_f32", self.sx, self.sx.numel() * 4))
+        jobs += [("grad", self.gout, self.n_grad * 4), ("adam_m", self.m, self.n_grad * 4), ("adam_v", self.v, self.n_grad * 4)]
+        if self.roots.numel() < 32 * len(jobs):
+            self.roots = torch.empty(32 * len(jobs), dtype=torch.uint8, device=self.dev)
+        for i, (_, t, nbytes) in enumerate(jobs):
+            det.det_tensor_hash_async(t, nbytes, self.roots[32 * i:32 * i + 32], self.ws)
+        raw = self.roots[:32 * len(jobs)].cpu().numpy().tobytes()
+        return {name: raw[32 * i:32 * i + 32].hex() for i, (name, _, _) in enumerate(jobs)}
 
     def calibrate(self, tokens_mb):
         """Untimed: set every activation step from the first micro-batch (LSQ initialisation rule)."""

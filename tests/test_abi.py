@@ -1,4 +1,4 @@
-"""The C-ABI library loads and exports every symbol that include/det.h declares (no GPU needed)."""
+"""The C-ABI library loads and exports every symbol that include/det.h and include/det_test.h declare (no GPU needed)."""
 import ctypes
 import os
 import re
@@ -7,9 +7,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    src = open(os.path.join(ROOT, "include", "det.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(det_[a-z0-9_]+)\s*\(", src)))
+    names = set()
+    for h in ("det.h", "det_test.h"):
+        src = open(os.path.join(ROOT, "include", h)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names |= set(re.findall(r"\b(det_[a-z0-9_]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_header_symbols_are_exported():

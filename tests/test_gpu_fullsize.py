@@ -33,8 +33,10 @@ def _bf16_normal(shape, std, seed):
     return synth.to_bf16((np.random.default_rng(seed).standard_normal(shape, dtype=np.float32) * F(std)))
 
 
-@pytest.mark.parametrize("N,K", [(2 * FF, D), (D, FF)])          # gate/up (one-CTA-pair tiles, short K) and down (long K)
-def test_linear_forward_full_shape_sampled(det, N, K):
+# gate/up (CTA-pair tiles, short K) and down (long K) at the micro-batch's 8192 tokens, and both again at the 16384
+# tokens of the 1B-shaped linear set
+@pytest.mark.parametrize("T,N,K", [(8192, 2 * FF, D), (8192, D, FF), (16384, 2 * FF, D), (16384, D, FF)])
+def test_linear_forward_full_shape_sampled(det, T, N, K):
     import torch
     X, W = _bf16_normal((T, K), 1.0, 1), _bf16_normal((N, K), 0.02, 2)
     dX_, dW_ = dev(X), dev(W)
@@ -63,11 +65,12 @@ def test_linear_forward_full_shape_sampled(det, N, K):
     assert_same_bits(host(Y, np.uint16)[np.ix_(rows, cols)], oY, "Y sample")
 
 
-def test_linear_backward_full_shape_sampled(det):
-    """Gate/up projection backward at 8192 x 16384 x 2048 with the Hadamard rotation: the operands' scales are maxima
-    over whole tensors, so the oracle prepares them in full and evaluates the two contractions for sampled rows."""
+@pytest.mark.parametrize("T,N,K", [(8192, 2 * FF, D), (16384, 3 * D, D)])
+def test_linear_backward_full_shape_sampled(det, T, N, K):
+    """Gate/up projection backward at 8192 x 16384 x 2048 and the QKV projection backward at 16384 x 6144 x 2048 (the token
+    count of the 1B-shaped linear set) with the Hadamard rotation: the operands' scales are maxima over whole tensors, so
+    the oracle prepares them in full and evaluates the two contractions for sampled rows."""
     import torch
-    N, K = 2 * FF, D
     X, W, dY = _bf16_normal((T, K), 1.0, 21), _bf16_normal((N, K), 0.02, 22), _bf16_normal((T, N), 0.01, 23)
     dX_, dW_, dY_ = dev(X), dev(W), dev(dY)
     s_w, s_x = empty((N,), F), empty((1,), F)
@@ -198,6 +201,33 @@ def test_norm_and_loss_full_shape(det):
     _sync()
     odz = oracle.xent_bwd(z[rows], tgt[rows], glse[rows], 1e-4, F(1.0 / T))
     assert_same_bits(dz[rows.tolist()].cpu().numpy(), odz, "dlogits rows")
+
+
+def test_grad_norm_1p2e9_elements(det):
+    """Global gradient norm over 1.2e9 f32 ~ N(0, 1e-3) (the reductions configuration), split into three tensors of ragged
+    lengths so that the per-tensor trees (four levels of 16384-element chunks for the largest) and the tree over the
+    per-tensor sums both run: norm and clip coefficient bit for bit against the oracle's trees."""
+    import torch
+    n = 1_200_000_000
+    g = np.random.default_rng(31).standard_normal(n, dtype=np.float32)
+    g *= F(1e-3)
+    cuts = [0, 700_000_000, 1_000_000_128, n]      # lengths 700000000, 300000128, 199999872; every start 16-byte aligned
+    dg = dev(g)
+    views = [dg[cuts[i]:cuts[i + 1]] for i in range(3)]
+    norm, coef = empty((1,), F), empty((1,), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_grad_norm(views, 1.0, norm, coef, ws(det.det_grad_norm_ws_bytes(views)), status)
+    _sync()
+    onorm, ocoef = oracle.grad_norm([g[cuts[i]:cuts[i + 1]] for i in range(3)], 1.0)
+    assert int(status.item()) == 0
+    assert_same_bits(host(norm), np.array([onorm], F), "norm")
+    assert_same_bits(host(coef), np.array([ocoef], F), "clip coefficient")
+    assert abs(float(onorm) - 34.64) < 0.05                        # sqrt(1.2e9) * 1e-3
+    # the whole vector as one tensor: one tree of five levels
+    out = empty((1,), F)
+    det.det_sum(dg, n, 1, out, ws(det.det_sum_ws_bytes(n)))
+    _sync()
+    assert_same_bits(host(out), np.array([oracle.sumsq(g)], F), "sum of squares, 1.2e9 elements")
 
 
 def test_reduction_and_optimizer_at_scale(det):

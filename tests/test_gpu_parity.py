@@ -44,7 +44,7 @@ def test_primitives_bitwise(det):
             da = dev(x)
         else:
             da = dev(a)
-        det.det_prim(op, da, db, out)
+        det.det_test_prim(op, da, db, out)
         _sync()
         assert_same_bits(host(out), oracle.prim(name, x, y), "prim " + name)
 
@@ -53,7 +53,7 @@ def test_max_of_signed_zeros(det):
     a = np.array([0.0, -0.0, -0.0, 0.0], F)
     b = np.array([-0.0, 0.0, -0.0, 0.0], F)
     out = empty(a.shape, F)
-    det.det_prim(oracle.OPS["max"], dev(a), dev(b), out)
+    det.det_test_prim(oracle.OPS["max"], dev(a), dev(b), out)
     _sync()
     assert_same_bits(host(out), oracle.prim("max", a, b), "max of zeros")
 
@@ -64,14 +64,14 @@ def test_flush_boundary_probe(det):
     a = np.array([fh('0x1.fffffep-1'), fh('0x1.fffffcp-1'), fh('0x1.000002p+0'), fh('0x1.8p-1')], F)
     b = np.array([2.0 ** -126, 2.0 ** -126, fh('0x1.fffffep-1') * 2.0 ** -126, 2.0 ** -126], F)
     out = empty(a.shape, F)
-    det.det_prim(oracle.OPS["mul"], dev(a), dev(b), out)
+    det.det_test_prim(oracle.OPS["mul"], dev(a), dev(b), out)
     _sync()
     assert_same_bits(host(out), oracle.prim("mul", a, b), "ftz boundary")
     # quotients: exact value (1 - 2^-24) * 2^-126 is a tie that IEEE would round up to the minimum normal
     a = np.array([fh('0x1.fffffep-1'), fh('0x1.fffffep-1'), 1.0, fh('0x1.fffffep-100'), 3.0], F)
     b = np.array([2.0 ** 126, 2.0 ** 125, 2.0 ** 126, 2.0 ** 27, fh('0x1.8p+127')], F)
     out = empty(a.shape, F)
-    det.det_prim(oracle.OPS["div"], dev(a), dev(b), out)
+    det.det_test_prim(oracle.OPS["div"], dev(a), dev(b), out)
     _sync()
     assert_same_bits(host(out), oracle.prim("div", a, b), "ftz boundary (div)")
 
@@ -81,7 +81,7 @@ def test_exp_all_bf16_arguments(det):
     x = oracle.bf2f(h)
     x = x[np.isfinite(x)]
     out = empty(x.shape, F)
-    det.det_prim(oracle.OPS["exp"], dev(x), None, out)
+    det.det_test_prim(oracle.OPS["exp"], dev(x), None, out)
     _sync()
     assert_same_bits(host(out), oracle.prim("exp", x), "exp")
 
@@ -92,7 +92,7 @@ def test_log_ends_of_the_domain_and_nan_logits(det):
     import torch
     x = np.array([0.0, -0.0, 1e-40, np.inf, -1.0, -np.inf, np.nan, 1.0, 2.5, 50304.0], F)
     out = empty(x.shape, F)
-    det.det_prim(oracle.OPS["log"], dev(x), None, out)
+    det.det_test_prim(oracle.OPS["log"], dev(x), None, out)
     _sync()
     got, want = host(out), oracle.prim("log", x)
     assert np.array_equal(np.isnan(got), np.isnan(want))
@@ -361,16 +361,17 @@ def test_tensor_hash(det, n):
 
 
 # ------------------------------------------------------------------ int8 GEMM and the LSQ linear layer
-@pytest.mark.parametrize("I,J,K", [(128, 128, 128), (256, 512, 512), (384, 256, 1024), (128, 384, 2048), (512, 768, 640),
-                                   (1024, 2048, 1152), (256, 256, 128)])
-def test_igemm_exact(det, I, J, K):
+@pytest.mark.parametrize("I,J,K,one_cta", [(128, 128, 128, 0), (256, 512, 512, 0), (384, 256, 1024, 0), (128, 384, 2048, 0),
+                                           (512, 768, 640, 0), (1024, 2048, 1152, 0), (256, 256, 128, 0), (256, 512, 512, 1),
+                                           (1024, 2048, 1152, 1)])
+def test_igemm_exact(det, I, J, K, one_cta):
     import torch
     rng = np.random.default_rng(I + J + K)
     A = rng.integers(-128, 128, (I, K)).astype(np.int8)
     B = rng.integers(-128, 128, (J, K)).astype(np.int8)
     Cd = empty((I, J), np.int32)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    det.det_igemm_tn(dev(A), dev(B), I, J, K, Cd, status)
+    det.det_test_igemm_tn(dev(A), dev(B), I, J, K, Cd, one_cta, status)   # one_cta: the one-CTA kernel where CTA pairs would apply
     _sync()
     assert int(status.item()) == 0
     want = A.astype(np.int32) @ B.astype(np.int32).T       # brute force, exact
@@ -412,11 +413,13 @@ def test_lsq_scales_quant_forward(det, M, N, K, per_tensor):
     assert_same_bits(host(Y, np.uint16), oY, "Y")
 
 
-@pytest.mark.parametrize("M,N,K,hb,mode", [(256, 512, 512, 128, 0), (256, 512, 512, 0, 0), (384, 128, 256, 128, 0),
-                                            (128, 256, 640, 128, 0), (256, 512, 512, 128, 1), (512, 256, 768, 128, 0)])
-def test_linear_backward(det, M, N, K, hb, mode):
+@pytest.mark.parametrize("M,N,K,hb", [(256, 512, 512, 128), (256, 512, 512, 0), (384, 128, 256, 128), (128, 256, 640, 128),
+                                       (384, 512, 512, 128), (512, 256, 768, 128), (128, 384, 256, 128)])
+def test_linear_backward(det, M, N, K, hb):
+    """Shapes whose output dimensions are multiples of 256 run on CTA pairs, the others on the one-CTA kernel with 128- or
+    256-wide tiles: (384, 512, 512) takes the one-CTA kernel with 256-wide tiles for the input gradient and CTA pairs for the
+    weight gradient."""
     import torch
-    det.det_igemm_set_mode(mode)       # 0: two-CTA tiles where the shape allows, 1: one-CTA kernel only
     X, W, dY = _linear_case(M, N, K, 12)
     osw = oracle.lsq_weight_scale(W)
     osx = oracle.lsq_act_scale_init(X)
@@ -438,7 +441,38 @@ def test_linear_backward(det, M, N, K, hb, mode):
     assert_same_bits(host(gX, np.uint16), odX, "dX")
     assert_same_bits(host(gW), odW, "dW")
     assert_same_bits(host(gs), ods, "ds_x")
-    det.det_igemm_set_mode(0)
+
+
+def test_linear_backward_per_tensor_weight_step(det):
+    """The single-linear configuration (256 tokens, 512 -> 512) with ONE weight step for the whole tensor: the backward
+    folds that step into dY and uses it in the weight mask exactly as it does a per-channel vector."""
+    import torch
+    M, N, K = 256, 512, 512
+    X, W, dY = _linear_case(M, N, K, 0)
+    osw = oracle.lsq_weight_scale(W, True)
+    assert np.all(osw == osw[0])
+    osx = oracle.lsq_act_scale_init(X)
+    for hb in (128, 0):
+        odX, odW, ods, dbg = oracle.linear_bwd(dY, X, W, osx, osw, hb=hb, debug=True)
+        dX_, dW_, dY_ = dev(X), dev(W), dev(dY)
+        s_w, s_x = empty((N,), F), dev(osx)
+        det.det_lsq_weight_scale(dW_, N, K, 1, s_w, ws(det.det_lsq_weight_scale_ws_bytes(N, K)))
+        qW, qWt, s_u = empty((N, K), np.int8), empty((K, N), np.int8), empty((1,), F)
+        det.det_lsq_quantize_weight(dW_, s_w, N, K, hb, qW, qWt, s_u, ws(det.det_lsq_quantize_weight_ws_bytes(N, K)))
+        Y, qX = empty((M, N), np.uint16), empty((M, K), np.int8)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        det.det_linear_fwd(dX_, qW, s_x, s_w, M, N, K, Y, qX, status)
+        gX, gW, gs = empty((M, K), np.uint16), empty((N, K), F), empty((1,), F)
+        det.det_linear_bwd(dY_, dX_, qX, dW_, qWt, s_x, s_w, s_u, M, N, K, hb, gX, gW, gs,
+                           ws(det.det_linear_bwd_ws_bytes(M, N, K)), status)
+        _sync()
+        assert int(status.item()) == 0
+        assert_same_bits(host(s_w), osw, "per-tensor s_w")
+        oY, _, _ = oracle.linear_fwd(X, W, osx, osw)
+        assert_same_bits(host(Y, np.uint16), oY, "Y")
+        assert_same_bits(host(gX, np.uint16), odX, "dX hb=%d" % hb)
+        assert_same_bits(host(gW), odW, "dW hb=%d" % hb)
+        assert_same_bits(host(gs), ods, "ds_x hb=%d" % hb)
 
 
 @pytest.mark.parametrize("case", ["zero_grad", "zero_weight", "zero_input", "heavy_tail", "saturated_input", "inf_grad",
@@ -684,7 +718,7 @@ def test_bounded_wait_times_out_and_context_survives(det):
     word and returns; the next launches run normally."""
     import torch
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    det.det_selftest_wait_timeout(status, 2000000)              # about a millisecond
+    det.det_test_wait_timeout(status, 2000000)              # about a millisecond
     _sync()
     assert int(status.item()) == det.DET_DEV_TIMEOUT
     x = np.arange(1000, dtype=F)

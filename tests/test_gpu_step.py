@@ -21,6 +21,15 @@ def _run(cfg_kwargs, seed=0):
     return cfg, got, want
 
 
+def _oracle_step(kw, seed):
+    """The oracle's step for a configuration given as keyword arguments of ModelConfig (seeded inputs from synth)."""
+    from oracle import step as ostep
+    from paper_2609_17380_b200 import step as dstep
+    cfg = dstep.ModelConfig(**kw).as_dict()
+    n_mb = cfg["mesh"][0] * cfg["mesh"][1] * cfg["mesh"][2]
+    return ostep.run_step(cfg, synth.model_params(cfg, seed=seed), synth.model_tokens(cfg, n_mb, seed=seed))
+
+
 @pytest.mark.parametrize("kw", [
     dict(n_layers=2, d_model=256, n_heads=2, ffn=512, vocab=512, seq=128, micro_batch=1, mesh=(2, 2, 2)),
     dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=1024, seq=192, micro_batch=2, mesh=(1, 1, 3)),
@@ -54,6 +63,39 @@ def test_step_hashes_match_oracle(kw):
     assert abs(got["loss"] - np.log(cfg.vocab)) < 0.5      # random init: loss ~ log V
 
 
+def test_full_width_step_matches_oracle():
+    """One replayed step at the benchmark's full width (d_model 2048, 16 heads, FFN 8192, sequence 2048, micro-batch 4,
+    Hadamard 128, CTA-pair GEMMs on every linear, the 268 MB attention workspace, the driver's shared scratch buffers at
+    their real sizes), one layer and an 8192-entry vocabulary so that the oracle's step takes minutes, not hours.  The
+    expected hashes are the oracle's: read from tests/golden/full_width_step.json (written by make_full_width_step.py,
+    which imports only the oracle and the input generator) while the oracle's sources are the ones that file was made
+    from, recomputed with the oracle otherwise."""
+    import importlib.util
+    import json
+    import os
+    from paper_2609_17380_b200 import step as dstep
+    gdir = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_full_width_step", os.path.join(gdir, "make_full_width_step.py"))
+    mk = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mk)
+    want = None
+    if os.path.exists(mk.OUT):
+        stored = json.load(open(mk.OUT))
+        if stored.get("key") == mk.source_key():
+            want = stored
+    if want is None:
+        want = mk.compute()
+    cfg = dstep.ModelConfig(**mk.CASE)
+    params = synth.model_params(cfg.as_dict(), seed=mk.SEED)
+    tokens = synth.model_tokens(cfg.as_dict(), 1, seed=mk.SEED)
+    got = dstep.run_step(cfg, params, tokens)
+    assert got["status"] == 0
+    assert [np.float32(x) for x in got["losses"]] == [np.float32(x) for x in want["losses"]]
+    assert np.float32(got["grad_norm"]) == np.float32(want["grad_norm"])
+    bad = [k for k, h in want["hashes"].items() if got["hashes"][k] != h]
+    assert not bad, bad
+
+
 @pytest.mark.parametrize("world", [1, 2, 4, 8])
 def test_sharded_fold_on_device_matches_single_replay(world):
     """The multi-GPU step with its transport replaced by plain copies, all ranks played one after the other on one
@@ -67,8 +109,8 @@ def test_sharded_fold_on_device_matches_single_replay(world):
     cfg = dstep.ModelConfig(**kw)
     params = synth.model_params(cfg.as_dict(), seed=3)
     tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=3)
-    want = dstep.run_step(cfg, params, tokens)
-    n = want["replay"].n_grad
+    want = _oracle_step(kw, 3)                      # the expectation is the oracle's single-process step
+    n = want["grad"].size
     plan = ShardPlan(cfg.n_microbatches, world, n)
     r = dstep.Replay(cfg, accum_len=plan.chunk, gout_len=plan.padded)
     r.load_params(params)
@@ -103,13 +145,13 @@ def test_sharded_replay_class_single_rank():
     cfg = dstep.ModelConfig(**kw)
     params = synth.model_params(cfg.as_dict(), seed=5)
     tokens = synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=5)
-    want = dstep.run_step(cfg, params, tokens)
+    want = _oracle_step(kw, 5)
     rep = ShardedReplay(cfg, 0, 1)
     rep.r.load_params(params)
     tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).cuda()
     rep.calibrate(tok[0])
     got = rep.step(tok)
-    assert got["status"] == 0 and got["losses"] == want["losses"]
+    assert got["status"] == 0 and got["losses"] == [np.float32(x) for x in want["losses"]]
     bad = [k for k, h in want["hashes"].items() if got["hashes"][k] != h]
     assert not bad, bad
 
@@ -182,8 +224,7 @@ def test_sharded_replay_two_ranks_on_one_gpu(tmp_path):
     import torch.multiprocessing as mp
     from paper_2609_17380_b200 import step as dstep
     kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=384, vocab=512, seq=128, micro_batch=1, mesh=(2, 2, 2))
-    cfg = dstep.ModelConfig(**kw)
-    want = dstep.run_step(cfg, synth.model_params(cfg.as_dict(), seed=9), synth.model_tokens(cfg.as_dict(), cfg.n_microbatches, seed=9))
+    want = _oracle_step(kw, 9)
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
     port = s.getsockname()[1]
@@ -191,7 +232,7 @@ def test_sharded_replay_two_ranks_on_one_gpu(tmp_path):
     mp.spawn(_sharded_worker, args=(2, port, kw, str(tmp_path)), nprocs=2, join=True)
     for rank in range(2):
         hashes, losses, status = eval(open(tmp_path / ("rank%d.txt" % rank)).read())
-        assert status == 0 and losses == want["losses"]
+        assert status == 0 and losses == [np.float32(x) for x in want["losses"]]
         assert not [k for k, h in want["hashes"].items() if hashes[k] != h], "rank %d" % rank
 
 
@@ -217,14 +258,11 @@ def _peer_worker_gpu(rank, world, port, outdir):
         pool = torch.empty(det.det_grad_accum_nbufs(2) * plan.chunk, dtype=torch.float32, device="cuda")
         out = torch.zeros(plan.padded, dtype=torch.float32, device="cuda")
         got = red.fold_and_gather(lambda sl, o: fold_slices(det, mesh, pool, sl, o), out).cpu().numpy()
-        st = det.det_accum()
-        bufs = torch.empty(det.det_grad_accum_nbufs(2) * n, dtype=torch.float32, device="cuda")
-        det.det_grad_accum_init(st, 2, 2, 2, n, bufs)
+        import oracle                                   # the expectation is the oracle's accumulator (Algorithm 1 + 2)
+        oa = oracle.Accum(2, 2, 2, n)
         for j in range(8):
-            det.det_grad_accum_push(st, g[j])
-        want = torch.empty(n, dtype=torch.float32, device="cuda")
-        det.det_grad_accum_result(st, want)
-        same = np.array_equal(got.view(np.uint32), want.cpu().numpy().view(np.uint32))
+            oa.push(g[j].cpu().numpy())
+        same = np.array_equal(got[:n].view(np.uint32), oa.result().view(np.uint32))
         # the NCCL in-place all-gather of the slice exchange accepts a slice of its own output (one rank: a no-op copy)
         from paper_2609_17380_b200.dist import ShardedReducer
         sr = ShardedReducer(plan, 0, "cuda")
