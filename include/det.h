@@ -121,6 +121,15 @@ int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int N, int K, i
  * X bf16 [M,K], qW int8 [N,K], Y bf16 [M,N].  M % 128 == 0, N % 128 == 0, K % 128 == 0, K < 2^17. */
 int det_linear_fwd(const det_bf16* X, const int8_t* qW, const float* s_x, const float* s_w, int M, int N, int K,
                    det_bf16* Y, int8_t* qX_save, void* stream, int* status_dev);
+/* The activation quantiser fused into the kernel that produces the activation (Sec. 3.2 "int8 computation": the
+ * linears consume int8 activations).  In a step the step size s_x of a linear is known before its input is produced,
+ * so the producer can write the int8 codes beside its bf16 output and the linear takes them ready-made:
+ *   det_rmsnorm_fwd_q / det_swiglu_fwd_q / det_attn_fwd_q  =  the plain call, plus q = rne(clamp(y * (1/s_q), -128, 127))
+ *   of the bf16 values y it stores (s_q: device scalar; q: int8, same shape and leading dimension as y, 8-byte
+ *   aligned, 4-byte for the attention); det_linear_fwd_q = det_linear_fwd without its quantiser pass (qX given).
+ * Every output has exactly the bits of the unfused sequence det_<producer>, det_linear_fwd. */
+int det_linear_fwd_q(const int8_t* qX, const int8_t* qW, const float* s_x, const float* s_w, int M, int N, int K,
+                     det_bf16* Y, void* stream, int* status_dev);
 /* Backward (straight-through estimator; both gradient GEMMs in int8 after a block-`hadamard_block`
  * Walsh-Hadamard rotation along the contraction dimension, 0 = no rotation):
  *   dX bf16 [M,K]  = mask_x ? 2^-7 s_a s_u (A_q . U_q) : 0,   A = rotate_n(dY * s_w[n]) quantised per tensor
@@ -136,6 +145,9 @@ int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_t* qX, cons
  * io: dtype of x, y, gamma, dy, dx (DET_F32 or DET_BF16); rstd f32 [rows]; D % 8 == 0, D <= 8192. */
 int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int rows, int D, float eps, void* y, float* rstd,
                     void* stream);
+/* bf16 in and out, D <= 2048; also writes the next linear's int8 input (see det_linear_fwd_q) */
+int det_rmsnorm_fwd_q(const det_bf16* x, const det_bf16* gamma, int rows, int D, float eps, det_bf16* y, float* rstd,
+                      const float* s_q, int8_t* qy, void* stream);
 /* dx = rstd * (w - xhat * c), w = dy*gamma, xhat = x*rstd, c = det_sum(w*xhat) * (1/D);
  * dgamma[j] = det_sum over rows of dy[r,j] * xhat[r,j] (f32 [D], may be NULL). */
 size_t det_rmsnorm_bwd_ws_bytes(int rows, int D);
@@ -181,6 +193,9 @@ int det_xent_bwd(float* logits_inout, const int32_t* target, const float* lse, i
  * rounded to bf16 before P.V.  lse f32 [B,H,S].  S % 64 == 0. */
 int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
                  int window, det_bf16* out, int ld_out, float* lse, void* stream);
+/* det_attn_fwd that also writes the output projection's int8 input qout [B*S, ld_out] (see det_linear_fwd_q) */
+int det_attn_fwd_q(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                   int window, det_bf16* out, int ld_out, float* lse, const float* s_q, int8_t* qout, void* stream);
 /* The same forward with the P.V product of every block of 128 keys on the int8 tensor cores (Sec. 3.2: "int8 P.V
  * per block"; the scales are this library's reading): per (batch, key/value head, block) s_v = absmax(V block)/127,
  * q_v = rne(clamp(v * (127/absmax))); per row and block q_p = rne(p * 127) with p = exp(s - m) in [0,1];
@@ -211,6 +226,8 @@ int det_attn_bwd_fixq(const det_bf16* dout, const det_bf16* q, const det_bf16* k
 /* ---- elementwise glue (Sec. 3.1: SwiGLU with fused gate/up projection, pre-norm residuals, embedding) */
 /* gu bf16 [rows, 2F] (gate | up), h bf16 [rows, F] = silu(gate) * up;  F % 8 == 0 */
 int det_swiglu_fwd(const det_bf16* gu, int rows, int F, det_bf16* h, void* stream);
+/* det_swiglu_fwd that also writes the down projection's int8 input qh [rows, F] (see det_linear_fwd_q) */
+int det_swiglu_fwd_q(const det_bf16* gu, int rows, int F, det_bf16* h, const float* s_q, int8_t* qh, void* stream);
 int det_swiglu_bwd(const det_bf16* dh, const det_bf16* gu, int rows, int F, det_bf16* dgu, void* stream);
 /* y = bf16(a + b); y may alias a or b; n % 8 == 0 */
 int det_residual_add(const det_bf16* a, const det_bf16* b, size_t n, det_bf16* y, void* stream);

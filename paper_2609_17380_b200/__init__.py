@@ -168,6 +168,11 @@ def det_linear_fwd(X, qW, s_x, s_w, M, N, K, Y, qX_save, status_dev=None):
                                                    C.c_int(K), _ptr(Y), _ptr(qX_save), _stream(), _ptr(status_dev)))
 
 
+def det_linear_fwd_q(qX, qW, s_x, s_w, M, N, K, Y, status_dev=None):
+    _check("det_linear_fwd_q", load().det_linear_fwd_q(_ptr(qX), _ptr(qW), _ptr(s_x), _ptr(s_w), C.c_int(M), C.c_int(N),
+                                                       C.c_int(K), _ptr(Y), _stream(), _ptr(status_dev)))
+
+
 def det_linear_bwd_ws_bytes(M, N, K):
     return load().det_linear_bwd_ws_bytes(C.c_int(M), C.c_int(N), C.c_int(K))
 
@@ -191,6 +196,11 @@ def det_test_igemm_tn(A, B, I, J, K, Cout, force_one_cta=0, status_dev=None):
 def det_rmsnorm_fwd(io, x, gamma, rows, D, eps, y, rstd):
     _check("det_rmsnorm_fwd", load().det_rmsnorm_fwd(C.c_int(io), _ptr(x), _ptr(gamma), C.c_int(rows), C.c_int(D),
                                                      C.c_float(eps), _ptr(y), _ptr(rstd), _stream()))
+
+
+def det_rmsnorm_fwd_q(x, gamma, rows, D, eps, y, rstd, s_q, qy):
+    _check("det_rmsnorm_fwd_q", load().det_rmsnorm_fwd_q(_ptr(x), _ptr(gamma), C.c_int(rows), C.c_int(D), C.c_float(eps),
+                                                         _ptr(y), _ptr(rstd), _ptr(s_q), _ptr(qy), _stream()))
 
 
 def det_headnorm_fwd(x, ld, T, nh, eps, y, ld_y, rstd):
@@ -239,6 +249,12 @@ def det_attn_fwd(q, k, v, ld, B, H, S, out, ld_out, lse, Hkv=None, window=0):
                                                C.c_int(ld_out), _ptr(lse), _stream()))
 
 
+def det_attn_fwd_q(q, k, v, ld, B, H, S, out, ld_out, lse, s_q, qout, Hkv=None, window=0):
+    _check("det_attn_fwd_q", load().det_attn_fwd_q(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H),
+                                                   C.c_int(H if Hkv is None else Hkv), C.c_int(S), C.c_int(window), _ptr(out),
+                                                   C.c_int(ld_out), _ptr(lse), _ptr(s_q), _ptr(qout), _stream()))
+
+
 def det_attn_fwd_int8pv(q, k, v, ld, B, H, S, out, ld_out, lse, status_dev=None, Hkv=None, window=0):
     _check("det_attn_fwd_int8pv", load().det_attn_fwd_int8pv(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H),
                                                              C.c_int(H if Hkv is None else Hkv), C.c_int(S), C.c_int(window),
@@ -270,6 +286,10 @@ def det_attn_bwd_fixq(dout, q, k, v, out, lse, ld, ld_out, B, H, S, dq, dk, dv, 
 # ---- glue --------------------------------------------------------------------------------------------------------
 def det_swiglu_fwd(gu, rows, F, h):
     _check("det_swiglu_fwd", load().det_swiglu_fwd(_ptr(gu), C.c_int(rows), C.c_int(F), _ptr(h), _stream()))
+
+
+def det_swiglu_fwd_q(gu, rows, F, h, s_q, qh):
+    _check("det_swiglu_fwd_q", load().det_swiglu_fwd_q(_ptr(gu), C.c_int(rows), C.c_int(F), _ptr(h), _ptr(s_q), _ptr(qh), _stream()))
 
 
 def det_swiglu_bwd(dh, gu, rows, F, dgu):

@@ -73,7 +73,8 @@ __device__ __forceinline__ void mac_4x8(const float (*As)[LQ], const float (*Bs)
 template <bool WIN>
 __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                                                     const uint16_t* __restrict__ v, int ld, int H, int Hkv, int S, int Warg,
-                                                    uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse) {
+                                                    uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse,
+                                                    const float* __restrict__ s_q, int8_t* __restrict__ qout) {
   const int W = WIN ? Warg : 0;
   extern __shared__ __align__(16) float sm[];
   float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                 // [dim][query]
@@ -233,6 +234,7 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
     }
     __syncthreads();  // V and P~ may be overwritten by the next tile
   }
+  const float inv_q = qout ? fdiv(1.0f, s_q[0]) : 0.0f;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int row = q0 + ty * 4 + i;
@@ -244,6 +246,13 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
     w1.x = pack_bf2(fmul(o[i][2].x, il), fmul(o[i][2].y, il)); w1.y = pack_bf2(fmul(o[i][3].x, il), fmul(o[i][3].y, il));
     *reinterpret_cast<uint2*>(op + tx * 4) = w0;
     *reinterpret_cast<uint2*>(op + 64 + tx * 4) = w1;
+    if (qout) {   // the output projection's quantiser, applied to the bf16 values just stored
+      const float f[8] = {bflo(w0.x), bfhi(w0.x), bflo(w0.y), bfhi(w0.y), bflo(w1.x), bfhi(w1.x), bflo(w1.y), bfhi(w1.y)};
+      const uint2 c = quant8(f, inv_q);
+      int8_t* qp8 = qout + (row0 + row) * ld_out + (size_t)h * DH;
+      *reinterpret_cast<uint32_t*>(qp8 + tx * 4) = c.x;
+      *reinterpret_cast<uint32_t*>(qp8 + 64 + tx * 4) = c.y;
+    }
     if (tx == 0) lse[((size_t)b * H + h) * S + row] = fadd(m[i], det_log(l[i]));
   }
 }
@@ -418,9 +427,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
 
 using namespace det;
 
-extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
-                            int window, det_bf16* out, int ld_out, float* lse, void* stream) {
+static int attn_fwd_impl(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                         int window, det_bf16* out, int ld_out, float* lse, const float* s_q, int8_t* qout, void* stream) {
   if (!q || !k || !v || !out || !lse || B <= 0 || H <= 0 || Hkv <= 0 || S <= 0 || window < 0) return DET_ERR_ARG;
+  if (qout && (!s_q || (((uintptr_t)qout) & 3u))) return qout && !s_q ? DET_ERR_ARG : DET_ERR_ALIGN;
   if (S % 64 || ld % 8 || ld_out % 8 || ld < H * DH || ld_out < H * DH || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
   static DevOnce once_full = {}, once_win = {};
@@ -428,10 +438,20 @@ extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16
       dev_ensure_smem(once_win, (const void*)k_attn_fwd<true>, FWD_SMEM) != DET_OK)
     return DET_ERR_CUDA;
   dim3 grid(H * B, (S + FQ - 1) / FQ);
-  if (window) k_attn_fwd<true><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse);
-  else k_attn_fwd<false><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, 0, out, ld_out, lse);
+  if (window) k_attn_fwd<true><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse, s_q, qout);
+  else k_attn_fwd<false><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, 0, out, ld_out, lse, s_q, qout);
   DET_CHECK_LAUNCH();
   return DET_OK;
+}
+
+extern "C" int det_attn_fwd(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                            int window, det_bf16* out, int ld_out, float* lse, void* stream) {
+  return attn_fwd_impl(q, k, v, ld, B, H, Hkv, S, window, out, ld_out, lse, nullptr, nullptr, stream);
+}
+extern "C" int det_attn_fwd_q(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int Hkv, int S,
+                              int window, det_bf16* out, int ld_out, float* lse, const float* s_q, int8_t* qout, void* stream) {
+  if (!s_q || !qout) return DET_ERR_ARG;
+  return attn_fwd_impl(q, k, v, ld, B, H, Hkv, S, window, out, ld_out, lse, s_q, qout, stream);
 }
 
 // workspace: bf16(P) and bf16(dS), [B*H, S, S] each, Delta f32 [B*H, S], and with grouped queries the f32 accumulators

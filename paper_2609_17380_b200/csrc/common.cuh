@@ -35,6 +35,21 @@ __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
   return (uint32_t)f2bf(lo) | ((uint32_t)f2bf(hi) << 16);
 }
 
+// LSQ quantiser (Sec. 3.1): code = rne(clamp(v * (1/s), -128, 127)); the reciprocal is one division per step size.
+__device__ __forceinline__ int8_t quant1(float v, float inv_s) {
+  float t = fminf(fmaxf(__fmul_rn(v, inv_s), -128.0f), 127.0f);
+  return (int8_t)__float2int_rn(t);
+}
+// eight values -> eight codes packed low byte first
+__device__ __forceinline__ uint2 quant8(const float v[8], float inv_s) {
+  uint2 o;
+  o.x = ((uint32_t)(uint8_t)quant1(v[0], inv_s)) | ((uint32_t)(uint8_t)quant1(v[1], inv_s) << 8) |
+        ((uint32_t)(uint8_t)quant1(v[2], inv_s) << 16) | ((uint32_t)(uint8_t)quant1(v[3], inv_s) << 24);
+  o.y = ((uint32_t)(uint8_t)quant1(v[4], inv_s)) | ((uint32_t)(uint8_t)quant1(v[5], inv_s) << 8) |
+        ((uint32_t)(uint8_t)quant1(v[6], inv_s) << 16) | ((uint32_t)(uint8_t)quant1(v[7], inv_s) << 24);
+  return o;
+}
+
 // exp: x = k ln2 + r, degree-7 Taylor polynomial in Horner form, one multiply and one add per step,
 // scaled through the exponent field.  Results below 2^-126 flush to +0; above FLT_MAX give +inf.
 __device__ __forceinline__ float det_exp(float x) {

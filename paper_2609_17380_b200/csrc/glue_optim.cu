@@ -21,7 +21,8 @@ __device__ __forceinline__ uint4 pack8(const float v[8]) {
 }
 
 __global__ void __launch_bounds__(256) k_swiglu_fwd(const uint16_t* __restrict__ gu, int rows, int F,
-                                                    uint16_t* __restrict__ h) {
+                                                    uint16_t* __restrict__ h, const float* __restrict__ s_q = nullptr,
+                                                    int8_t* __restrict__ qh = nullptr) {
   const size_t per_row = (size_t)F / 8;
   size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= per_row * rows) return;
@@ -32,6 +33,12 @@ __global__ void __launch_bounds__(256) k_swiglu_fwd(const uint16_t* __restrict__
 #pragma unroll
   for (int t = 0; t < 8; ++t) o[t] = fmul(fmul(g[t], sigmoid_det(g[t])), u[t]);
   *reinterpret_cast<uint4*>(h + r * F + c) = pack8(o);
+  if (qh) {   // the next linear's quantiser, applied to the bf16 values just stored
+    const float inv_q = fdiv(1.0f, s_q[0]);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) o[t] = bf2f(f2bf(o[t]));
+    *reinterpret_cast<uint2*>(qh + r * F + c) = quant8(o, inv_q);
+  }
 }
 
 __global__ void __launch_bounds__(256) k_swiglu_bwd(const uint16_t* __restrict__ dh, const uint16_t* __restrict__ gu,
@@ -389,6 +396,16 @@ extern "C" int det_swiglu_fwd(const det_bf16* gu, int rows, int F, det_bf16* h, 
   size_t n = (size_t)rows * (F / 8);
   if (!n) return DET_OK;
   k_swiglu_fwd<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(gu, rows, F, h);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+extern "C" int det_swiglu_fwd_q(const det_bf16* gu, int rows, int F, det_bf16* h, const float* s_q, int8_t* qh, void* stream) {
+  if (!gu || !h || !s_q || !qh || rows < 0 || F <= 0) return DET_ERR_ARG;
+  if (F % 8) return DET_ERR_SHAPE;
+  if (!aligned16(gu) || !aligned16(h) || (((uintptr_t)qh) & 7u)) return DET_ERR_ALIGN;
+  size_t n = (size_t)rows * (F / 8);
+  if (!n) return DET_OK;
+  k_swiglu_fwd<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(gu, rows, F, h, s_q, qh);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

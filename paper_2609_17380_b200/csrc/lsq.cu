@@ -8,10 +8,6 @@ namespace det {
 
 #define C127 0x1.6b7612p-4f
 
-__device__ __forceinline__ int8_t quant1(float v, float inv_s) {
-  float t = fminf(fmaxf(fmul(v, inv_s), -128.0f), 127.0f);
-  return (int8_t)__float2int_rn(t);
-}
 __device__ __forceinline__ void unpack8u(const uint4& u, float v[8]) {
   v[0] = bflo(u.x); v[1] = bfhi(u.x); v[2] = bflo(u.y); v[3] = bfhi(u.y);
   v[4] = bflo(u.z); v[5] = bfhi(u.z); v[6] = bflo(u.w); v[7] = bfhi(u.w);
@@ -481,6 +477,17 @@ extern "C" int det_linear_fwd(const det_bf16* X, const int8_t* qW, const float* 
   EpiParams ep = {};
   ep.out = Y; ep.s_x = s_x; ep.s_w = s_w;
   return igemm_launch(EPI_FWD, qX_save, qW, M, N, K, ep, status_dev, st);
+}
+
+extern "C" int det_linear_fwd_q(const int8_t* qX, const int8_t* qW, const float* s_x, const float* s_w, int M, int N, int K,
+                                det_bf16* Y, void* stream, int* status_dev) {
+  if (!qX || !qW || !s_x || !s_w || !Y || M <= 0 || N <= 0 || K <= 0) return DET_ERR_ARG;
+  if (M % 128 || N % 128 || K % 128) return DET_ERR_SHAPE;
+  if (K >= (1 << 17)) return DET_ERR_RANGE;
+  if (!aligned16(qX) || !aligned16(qW) || !aligned16(Y) || !aligned16(s_w)) return DET_ERR_ALIGN;
+  EpiParams ep = {};
+  ep.out = Y; ep.s_x = s_x; ep.s_w = s_w;
+  return igemm_launch(EPI_FWD, qX, qW, M, N, K, ep, status_dev, (cudaStream_t)stream);
 }
 
 static size_t bwd_ws_layout(int M, int N, int K, size_t* oA, size_t* oG, size_t* oZ, size_t* oP, size_t* oS) {

@@ -39,11 +39,13 @@ __device__ __forceinline__ void store8(void* p, size_t idx, const float v[8]) {
 template <bool BF>
 __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
                                                       int D, float eps, float invD, void* __restrict__ y,
-                                                      float* __restrict__ rstd) {
+                                                      float* __restrict__ rstd, const float* __restrict__ s_q = nullptr,
+                                                      int8_t* __restrict__ qy = nullptr) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * 8 + warp;
   if (row >= rows) return;
   const size_t rb = (size_t)row * D;
+  const float inv_q = (BF && qy) ? fdiv(1.0f, s_q[0]) : 0.0f;
   float xr[8][8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -83,6 +85,11 @@ __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x
       for (int t = 0; t < 8; ++t) o[t] = fmul(xr[j][t], rs);
     }
     store8<BF>(y, rb + e0, o);
+    if (BF && qy) {   // the next linear's quantiser, applied to the bf16 values just stored
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = bf2f(f2bf(o[t]));
+      *reinterpret_cast<uint2*>(qy + rb + e0) = quant8(o, inv_q);
+    }
   }
 }
 
@@ -480,6 +487,18 @@ extern "C" int det_rmsnorm_fwd(int io, const void* x, const void* gamma, int row
     if (D <= 2048) k_rmsnorm_fwd8<false><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
     else k_rmsnorm_fwd<false, 0><<<DET_L(grid), 256, 0, st>>>(x, gamma, rows, D, eps, invD, y, rstd);
   }
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}
+
+extern "C" int det_rmsnorm_fwd_q(const det_bf16* x, const det_bf16* gamma, int rows, int D, float eps, det_bf16* y,
+                                 float* rstd, const float* s_q, int8_t* qy, void* stream) {
+  if (!x || !y || !rstd || !s_q || !qy || rows < 0 || D <= 0) return DET_ERR_ARG;
+  if (D % 8 || D > 2048) return DET_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y) || (gamma && !aligned16(gamma)) || (((uintptr_t)qy) & 7u)) return DET_ERR_ALIGN;
+  if (rows == 0) return DET_OK;
+  k_rmsnorm_fwd8<true><<<DET_L((rows + 7) / 8), 256, 0, (cudaStream_t)stream>>>(x, gamma, rows, D, eps, (float)(1.0 / (double)D), y,
+                                                                              rstd, s_q, qy);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -155,6 +155,7 @@ class Replay:
         self.ws = e(wsb + 4096, torch.uint8)
         self.losses = []
         self.prof = None
+        self.fuse_quant = True       # producers write the linears' int8 inputs (False: separate quantiser pass per linear)
 
     # ---- optional per-call-site device timing (CUDA events on the launching stream) --------------------
     class _Span:
@@ -245,13 +246,17 @@ class Replay:
             det.det_lsq_weight_scale(W, d["N"], d["K"], 0, d["s_w"], self.ws)
             det.det_lsq_quantize_weight(W, d["s_w"], d["N"], d["K"], hb, d["qW"], d["qWt"], d["s_u"], self.ws)
 
-    def _linear(self, l, w, idx, X, M, Y, qx, calibrate):
+    def _linear(self, l, w, idx, X, M, Y, qx, calibrate, prequantised=False):
+        """prequantised: the kernel that produced X already wrote its int8 codes into qx."""
         d = self.lin[(l, w)]
         sx = self.sx[4 * l + idx:4 * l + idx + 1]
         if calibrate:
             det.det_lsq_act_scale_init(X, M * d["K"], sx, self.ws)
         with self.span("linear_fwd"):
-            det.det_linear_fwd(X, d["qW"], sx, d["s_w"], M, d["N"], d["K"], Y, qx, self.status)
+            if prequantised:
+                det.det_linear_fwd_q(qx, d["qW"], sx, d["s_w"], M, d["N"], d["K"], Y, self.status)
+            else:
+                det.det_linear_fwd(X, d["qW"], sx, d["s_w"], M, d["N"], d["K"], Y, qx, self.status)
 
     def forward(self, tokens_mb, calibrate=False):
         cfg = self.cfg
@@ -269,8 +274,15 @@ class Replay:
         for l in range(L):
             a = self.act[l]
             a["x"].copy_(x)
-            det.det_rmsnorm_fwd(det.DET_BF16, a["x"], self.p("l%d.attn_norm" % l), T, D, 1e-6, a["n1"], a["rstd1"])
-            self._linear(l, "w_qkv", 0, a["n1"], T, a["qkv"], a["qx_qkv"], calibrate)
+            # outside the calibration pass every activation step is known before its activation is produced, so the
+            # producers write the next linear's int8 input themselves (same bits as the separate quantiser pass)
+            fuse = self.fuse_quant and not calibrate and D <= 2048
+            sxl = self.sx[4 * l:4 * l + 4]
+            if fuse:
+                det.det_rmsnorm_fwd_q(a["x"], self.p("l%d.attn_norm" % l), T, D, 1e-6, a["n1"], a["rstd1"], sxl[0:1], a["qx_qkv"])
+            else:
+                det.det_rmsnorm_fwd(det.DET_BF16, a["x"], self.p("l%d.attn_norm" % l), T, D, 1e-6, a["n1"], a["rstd1"])
+            self._linear(l, "w_qkv", 0, a["n1"], T, a["qkv"], a["qx_qkv"], calibrate, fuse)
             qp = vp = a["qkv"].data_ptr()
             if self.head_ops:
                 # queries and keys (the first H + Hkv heads of every row) are normalised and rotated into qkr; the
@@ -286,17 +298,26 @@ class Replay:
                 if cfg.pv_int8:
                     det.det_attn_fwd_int8pv(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"],
                                             self.status, Hkv=Hkv, window=cfg.layer_window(l))
+                elif fuse:
+                    det.det_attn_fwd_q(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"], sxl[1:2],
+                                       a["qx_o"], Hkv=Hkv, window=cfg.layer_window(l))
                 else:
                     det.det_attn_fwd(qp, qp + 2 * D, vp + 2 * (D + 128 * Hkv), QW, B, H, S, a["att"], D, a["lse"], Hkv=Hkv,
                                      window=cfg.layer_window(l))
             o = self.tmp[1][:T * D]
-            self._linear(l, "w_o", 1, a["att"], T, o, a["qx_o"], calibrate)
+            self._linear(l, "w_o", 1, a["att"], T, o, a["qx_o"], calibrate, fuse and not cfg.pv_int8)
             det.det_residual_add(a["x"], o, T * D, a["h"])
-            det.det_rmsnorm_fwd(det.DET_BF16, a["h"], self.p("l%d.ffn_norm" % l), T, D, 1e-6, a["n2"], a["rstd2"])
-            self._linear(l, "w_gu", 2, a["n2"], T, a["gu"], a["qx_gu"], calibrate)
-            det.det_swiglu_fwd(a["gu"], T, Fh, a["a"])
+            if fuse:
+                det.det_rmsnorm_fwd_q(a["h"], self.p("l%d.ffn_norm" % l), T, D, 1e-6, a["n2"], a["rstd2"], sxl[2:3], a["qx_gu"])
+            else:
+                det.det_rmsnorm_fwd(det.DET_BF16, a["h"], self.p("l%d.ffn_norm" % l), T, D, 1e-6, a["n2"], a["rstd2"])
+            self._linear(l, "w_gu", 2, a["n2"], T, a["gu"], a["qx_gu"], calibrate, fuse)
+            if fuse:
+                det.det_swiglu_fwd_q(a["gu"], T, Fh, a["a"], sxl[3:4], a["qx_down"])
+            else:
+                det.det_swiglu_fwd(a["gu"], T, Fh, a["a"])
             dn = self.tmp[1][:T * D]
-            self._linear(l, "w_down", 3, a["a"], T, dn, a["qx_down"], calibrate)
+            self._linear(l, "w_down", 3, a["a"], T, dn, a["qx_down"], calibrate, fuse)
             det.det_residual_add(a["h"], dn, T * D, x)
         self.xf.copy_(x)
         det.det_rmsnorm_fwd(det.DET_BF16, self.xf, self.p("final_norm"), T, D, 1e-6, self.nf, self.rstdf)

@@ -292,6 +292,62 @@ def test_glue(det):
     assert_same_bits(host(y, np.uint16), oracle.residual_add(a, b), "residual")
 
 
+def test_producers_write_the_next_linears_int8_input(det):
+    """The activation quantiser fused into RMSNorm, SwiGLU and the attention forward: the int8 copy equals the oracle's
+    quantiser applied to the producer's bf16 output, the bf16 output itself is untouched, and the linear that takes the
+    codes ready-made equals the oracle's linear forward.  Steps are chosen so that values saturate on both sides."""
+    import torch
+    rows, D = 264, 512
+    x = synth.normal_bf16((rows, D), 3.0, seed=41, tid=1)
+    g = synth.to_bf16(1 + synth.normal_f32(D, 0.02, seed=41, tid=2))
+    s = np.array([0.021], F)
+    y, rstd, qy = empty((rows, D), np.uint16), empty((rows,), F), empty((rows, D), np.int8)
+    det.det_rmsnorm_fwd_q(dev(x), dev(g), rows, D, 1e-6, y, rstd, dev(s), qy)
+    _sync()
+    oy, orstd = oracle.rmsnorm_fwd(x, g, 1e-6, bf=True)
+    assert_same_bits(host(y, np.uint16), oy, "rmsnorm y")
+    assert_same_bits(host(rstd), orstd, "rstd")
+    assert_same_bits(host(qy), oracle.lsq_quantize(oy, s, False), "rmsnorm int8 copy")
+    assert (host(qy) == 127).any() and (host(qy) == -128).any()
+    # SwiGLU
+    Fd = 768
+    gu = synth.normal_bf16((rows, 2 * Fd), 2.0, seed=41, tid=3)
+    s2 = np.array([0.013], F)
+    h, qh = empty((rows, Fd), np.uint16), empty((rows, Fd), np.int8)
+    det.det_swiglu_fwd_q(dev(gu), rows, Fd, h, dev(s2), qh)
+    _sync()
+    oh = oracle.swiglu_fwd(gu)
+    assert_same_bits(host(h, np.uint16), oh, "swiglu h")
+    assert_same_bits(host(qh), oracle.lsq_quantize(oh, s2, False), "swiglu int8 copy")
+    # attention (full causal and a sliding window), then the output projection on the ready-made codes
+    B, H, S = 2, 2, 320
+    HD = H * 128
+    qkv = synth.normal_bf16((B * S, 3 * HD), 1.0, seed=41, tid=4)
+    dq = dev(qkv)
+    base = dq.data_ptr()
+    s3 = np.array([0.004], F)
+    for window in (0, 128):
+        out, lse, qo = empty((B * S, HD), np.uint16), empty((B, H, S), F), empty((B * S, HD), np.int8)
+        det.det_attn_fwd_q(base, base + 2 * HD, base + 4 * HD, 3 * HD, B, H, S, out, HD, lse, dev(s3), qo, window=window)
+        _sync()
+        oout, olse = oracle.attn_fwd(qkv, B, H, S, window=window)
+        assert_same_bits(host(out, np.uint16), oout, "attention out")
+        assert_same_bits(host(lse), olse, "lse")
+        assert_same_bits(host(qo), oracle.lsq_quantize(oout, s3, False), "attention int8 copy")
+    N = 384
+    W = synth.normal_bf16((N, HD), 0.02, seed=41, tid=5)
+    osw = oracle.lsq_weight_scale(W)
+    qW = empty((N, HD), np.int8)
+    det.det_lsq_quantize_weight(dev(W), dev(osw), N, HD, 128, qW, None, None, ws(256))
+    Y = empty((B * S, N), np.uint16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_linear_fwd_q(qo, qW, dev(s3), dev(osw), B * S, N, HD, Y, status)
+    _sync()
+    oY, _, _ = oracle.linear_fwd(oout, W, s3, osw)
+    assert int(status.item()) == 0
+    assert_same_bits(host(Y, np.uint16), oY, "linear on ready-made codes")
+
+
 def test_embedding(det):
     V, D, T = 1000, 512, 700
     E = synth.normal_bf16((V, D), 0.02, seed=7, tid=1)

@@ -63,6 +63,26 @@ def test_step_hashes_match_oracle(kw):
     assert abs(got["loss"] - np.log(cfg.vocab)) < 0.5      # random init: loss ~ log V
 
 
+def test_step_with_separate_quantiser_passes_gives_the_same_hashes():
+    """The step driver lets the producers write the linears' int8 inputs; with that switched off every linear runs its own
+    quantiser pass (the unfused definition): same hashes, and both equal the oracle's."""
+    import torch
+    from paper_2609_17380_b200 import step as dstep
+    kw = dict(n_layers=2, d_model=256, n_heads=2, ffn=512, vocab=512, seq=128, micro_batch=1, mesh=(1, 2, 1))
+    want = _oracle_step(kw, 11)
+    cfg = dstep.ModelConfig(**kw)
+    params = synth.model_params(cfg.as_dict(), seed=11)
+    tok = torch.from_numpy(np.ascontiguousarray(synth.model_tokens(cfg.as_dict(), 2, seed=11), dtype=np.int32)).cuda()
+    for fuse in (False, True):
+        r = dstep.Replay(cfg)
+        r.fuse_quant = fuse
+        r.load_params(params)
+        r.calibrate(tok[0])
+        got = r.step(tok)
+        assert got["status"] == 0
+        assert not [k for k, h in want["hashes"].items() if got["hashes"][k] != h], fuse
+
+
 def test_full_width_step_matches_oracle():
     """One replayed step at the benchmark's full width (d_model 2048, 16 heads, FFN 8192, sequence 2048, micro-batch 4,
     Hadamard 128, CTA-pair GEMMs on every linear, the 268 MB attention workspace, the driver's shared scratch buffers at
