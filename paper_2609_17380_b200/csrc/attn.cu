@@ -179,10 +179,13 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
-      alpha[i] = rowvalid ? det_exp(fsub(m[i], mt)) : 1.0f;
+      const float al = det_exp_sel(fsub(m[i], mt));
+      alpha[i] = rowvalid ? al : 1.0f;
       float p[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) p[e] = valid[e] ? det_exp(fsub(sv[e], mt)) : 0.0f;
+      for (int e = 0; e < 8; ++e) p[e] = det_exp_sel(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
+#pragma unroll
+      for (int e = 0; e < 8; ++e) p[e] = valid[e] ? p[e] : 0.0f;
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int kl = (e < 4) ? (tx * 4 + e) : (64 + tx * 4 + e - 4);
@@ -256,6 +259,345 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
     if (tx == 0) lse[((size_t)b * H + h) * S + row] = fadd(m[i], det_log(l[i]));
   }
 }
+
+// ---------------------------------------------------------------------------------------------
+// forward, warp-specialised (full causal attention; the windowed layers keep k_attn_fwd<true>).
+//
+// What bounds the kernel above is shared-memory bandwidth: a 16-byte load costs the port one cycle per 128 distinct
+// bytes of every half-warp, its 4 x 8 register tiles need three such loads (10 port cycles per warp) for 16 packed
+// multiply-adds, and its phases (logits, softmax, P.V) are block-wide, so the FP32 pipe idles during every softmax.
+// Here a consumer warp owns 16 whole query rows: a lane holds 16 rows x 4 adjacent columns (keys while the logits are
+// formed, head dimensions during P.V), so the row operand is one address for the whole warp (q^T [dim][query] and
+// P~ [key][query] in shared memory) and the column operand one 16-byte word per lane: five loads (12 port cycles) per 32
+// packed multiply-adds.  A row's 128 logits of a key block sit in one warp, so its maximum and its row sum (the
+// adjacent pairwise tree: four slots in the lane, then lanes 1, 2, 4, 8, 16 apart) are warp shuffles, P~ of the warp's
+// rows is written and read by that warp alone, and the running maximum, sum and rescale factor of row i live in lane i.
+// K and V arrive through an mbarrier-guarded ring of 16-deep slabs filled by four producer warps (K: 16 head dimensions
+// x 128 keys, eight per block; V: 16 keys x 128 dimensions, eight per block), so no block-wide barrier is left in the
+// loop and consumer warps are not coupled to each other.  The softmax evaluates its 64 exponentials per lane as one
+// straight-line block of branch-free chains (det_exp_sel) and reduces the 16 rows with 16 shuffles per reduction.
+// On the diagonal block a warp stops P.V after the last key any of its rows may see.
+// Arithmetic and order per output are exactly those of k_attn_fwd (and of the definition): bit-identical results.
+// ---------------------------------------------------------------------------------------------
+constexpr int AF_SLOTS = 8, AF_PF = 4, AF_CONS = 256, AF_PROD = 128, AF_THREADS = AF_CONS + AF_PROD;
+constexpr size_t AFW_SMEM = (size_t)(DH * LQ + FK * FQ + AF_SLOTS * OK * (OT + 4)) * sizeof(float);
+
+// one 16-deep slab: acc[i/2][c].{x,y} += A[k][rows i, i+1 of the warp] * B[k][4 lane + c]: the accumulators pair two ROWS, so
+// the row operand's register pairs come straight out of its 16-byte loads and only the four column values are duplicated
+// into pairs.  A chunk g (rows 4g..4g+3) of step k is at ap + k * a_ld + ((chunk0 + g) ^ (PSWZ ? swizzle of the key : 0)) * 4.
+template <bool FUSED, bool PSWZ>
+__device__ __forceinline__ void mac_16x4(const float* __restrict__ ap, int a_ld, int chunk0, int key0,
+                                         const float (*Bs)[OT + 4], int lane, float2 (&acc)[8][4]) {
+#pragma unroll
+  for (int k = 0; k < OK; ++k) {
+    const int sw = PSWZ ? (((key0 + k) >> 2) & 7) : 0;
+    float4 a[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) a[g] = *reinterpret_cast<const float4*>(ap + (size_t)k * a_ld + (((chunk0 + g) ^ sw) << 2));
+    const float4 bv = *reinterpret_cast<const float4*>(&Bs[k][4 * lane]);
+    const float bs[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float2 bb = make_float2(bs[c], bs[c]);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        if (FUSED) {
+          acc[2 * g][c] = __ffma2_rn(make_float2(a[g].x, a[g].y), bb, acc[2 * g][c]);
+          acc[2 * g + 1][c] = __ffma2_rn(make_float2(a[g].z, a[g].w), bb, acc[2 * g + 1][c]);
+        } else {  // scalar on purpose: a packed multiply + add pair would be contracted by ptxas
+          acc[2 * g][c].x = fadd(acc[2 * g][c].x, fmul(a[g].x, bs[c]));
+          acc[2 * g][c].y = fadd(acc[2 * g][c].y, fmul(a[g].y, bs[c]));
+          acc[2 * g + 1][c].x = fadd(acc[2 * g + 1][c].x, fmul(a[g].z, bs[c]));
+          acc[2 * g + 1][c].y = fadd(acc[2 * g + 1][c].y, fmul(a[g].w, bs[c]));
+        }
+      }
+    }
+  }
+}
+// element (row i, column c) of a row-paired accumulator set; i is a compile-time constant wherever this is used
+#define RP(acc, i, c) (((i) & 1) ? (acc)[(i) >> 1][c].y : (acc)[(i) >> 1][c].x)
+// Reduction of 16 rows across the warp (x[i]: this lane's value for row i) with partners 1, 2, 4, 8, 16 lanes apart in that
+// order, which for sums is the adjacent pairwise tree over the lanes.  Instead of 16 butterflies of five shuffles every
+// stage halves the rows a lane carries (it sends its partner the half the partner keeps): 8 + 4 + 2 + 1 + 1 shuffles, and
+// lane L ends with the result of row ROW_OF_LANE(L); both operand orders of an addition or a maximum give the same bits.
+#define ROW_OF_LANE(L) ((((L) & 1) << 3) | (((L) & 2) << 1) | (((L) & 4) >> 1) | (((L) & 8) >> 3))
+#define ROW_LANE(i) ROW_OF_LANE(i)   /* a lane that holds row i (the bit reversal is its own inverse) */
+template <bool SUM>
+__device__ __forceinline__ float rows16_reduce(const float (&x)[16], int lane) {
+  auto op = [](float a, float b) { return SUM ? fadd(a, b) : fmaxf(a, b); };
+  float a[8], b[4], c[2];
+  const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4, b3 = lane & 8;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a[j] = op(b0 ? x[8 + j] : x[j], __shfl_xor_sync(0xffffffffu, b0 ? x[j] : x[8 + j], 1));
+#pragma unroll
+  for (int j = 0; j < 4; ++j) b[j] = op(b1 ? a[4 + j] : a[j], __shfl_xor_sync(0xffffffffu, b1 ? a[j] : a[4 + j], 2));
+#pragma unroll
+  for (int j = 0; j < 2; ++j) c[j] = op(b2 ? b[2 + j] : b[j], __shfl_xor_sync(0xffffffffu, b2 ? b[j] : b[2 + j], 4));
+  float d = op(b3 ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, b3 ? c[0] : c[1], 8));
+  return op(d, __shfl_xor_sync(0xffffffffu, d, 16));
+}
+__global__ void __launch_bounds__(AF_THREADS, 1)
+    k_attn_fwd_ws(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k, const uint16_t* __restrict__ v, int ld,
+                  int H, int Hkv, int S, uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse,
+                  const float* __restrict__ s_q, int8_t* __restrict__ qout) {
+  extern __shared__ __align__(16) float sm[];
+  float(*Qs)[LQ] = reinterpret_cast<float(*)[LQ]>(sm);                         // [dim][query]
+  float* Ps = sm + DH * LQ;                                                    // [key][query], 16-byte chunks swizzled
+  float(*Ring)[OK][OT + 4] = reinterpret_cast<float(*)[OK][OT + 4]>(sm + DH * LQ + FK * FQ);
+  __shared__ int tiny_s[AF_SLOTS][AF_PROD / 32];
+  __shared__ int tiny_q_s, abort_s;
+  __shared__ __align__(8) uint64_t bar_full[AF_SLOTS], bar_empty[AF_SLOTS];
+  volatile int* abort_flag = &abort_s;
+  const int qb = gridDim.y - 1 - blockIdx.y;          // longest rows first
+  const int h = blockIdx.x % H, b = blockIdx.x / H, hk = h / (H / Hkv);
+  const int q0 = qb * FQ;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const size_t row0 = (size_t)b * S;
+  const uint16_t* qp = q + row0 * ld + (size_t)h * DH;
+  const uint16_t* kp = k + row0 * ld + (size_t)hk * DH;
+  const uint16_t* vp = v + row0 * ld + (size_t)hk * DH;
+  const int ntiles = q0 / FK + 1, nslab = ntiles * 16;
+  if (tid == 0) {
+    for (int s = 0; s < AF_SLOTS; ++s) { mbar_init(&bar_full[s], AF_PROD / 32); mbar_init(&bar_empty[s], AF_CONS / 32); }
+    tiny_q_s = 0;
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  {  // q^T of the query block, staged once by everybody
+    bool tq = false;
+    for (int idx = tid; idx < FQ * 16; idx += AF_THREADS) {
+      const int r = idx & 127, ch = idx >> 7;
+      float t[8];
+      if (q0 + r < S) unpack8a(__ldg(reinterpret_cast<const uint4*>(qp + (size_t)(q0 + r) * ld + ch * 8)), t);
+      else {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) t[x] = 0.0f;
+      }
+#pragma unroll
+      for (int x = 0; x < 8; ++x) { tq |= tiny1(t[x]); Qs[ch * 8 + x][r] = t[x]; }
+    }
+    if (__any_sync(0xffffffffu, tq) && lane == 0) atomicOr(&tiny_q_s, 1);
+  }
+  __syncthreads();
+  if (tid >= AF_CONS) {
+    // ------------------------------- producers -------------------------------
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    const int pt = tid - AF_CONS, pw = pt >> 5;
+    // Slab s of the block sequence: block s / 16; s % 16 < 8: K, head dimensions 16 (s % 16) .. (thread = key, two
+    // 16-byte words); else V, keys 16 (s % 16 - 8) .. (thread = four dimensions of keys kk, kk + 4, kk + 8, kk + 12).
+    // AF_PF slabs are in flight in registers, so that the latency of a global load is spread over several slabs.
+    // Both kinds are two 16-byte words per thread, so one register array holds whichever kind slab s is.
+    uint4 raw[AF_PF][2];
+    const int vf = pt & 31, vk = pt >> 5;            // V: dimensions 4 vf .. 4 vf + 3 of keys vk, vk + 4, vk + 8, vk + 12
+    auto fetch = [&](int sn, uint4 (&w)[2]) {
+      if (sn >= nslab) return;
+      const int j0n = (sn >> 4) * FK, phn = sn & 15;
+      if (phn < 8) {
+        const int key = j0n + pt;
+        const uint4* src = reinterpret_cast<const uint4*>(kp + (size_t)key * ld + phn * OK);
+        const bool in = key < S;
+        w[0] = in ? __ldg(src) : make_uint4(0u, 0u, 0u, 0u);
+        w[1] = in ? __ldg(src + 1) : make_uint4(0u, 0u, 0u, 0u);
+      } else {
+        const int key0 = j0n + (phn - 8) * OK + vk;
+        uint2 u[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int key = key0 + 4 * i;
+          u[i] = key < S ? __ldg(reinterpret_cast<const uint2*>(vp + (size_t)key * ld + 4 * vf)) : make_uint2(0u, 0u);
+        }
+        w[0] = make_uint4(u[0].x, u[0].y, u[1].x, u[1].y);
+        w[1] = make_uint4(u[2].x, u[2].y, u[3].x, u[3].y);
+      }
+    };
+    // unpack, test for factors below 2^-63 and store: K as [dimension][key] (thread = key), V as [key][dimension]
+    auto store = [&](int ph, float (*dst)[OT + 4], const uint4 (&w)[2]) -> bool {
+      bool tiny = false;
+      if (ph < 8) {
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          float t[8];
+          unpack8a(w[x], t);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) { tiny |= tiny1(t[e]); dst[x * 8 + e][pt] = t[e]; }
+        }
+      } else {
+        const uint32_t words[8] = {w[0].x, w[0].y, w[0].z, w[0].w, w[1].x, w[1].y, w[1].z, w[1].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 t = make_float4(bflo(words[2 * i]), bfhi(words[2 * i]), bflo(words[2 * i + 1]), bfhi(words[2 * i + 1]));
+          tiny |= tiny1(t.x) | tiny1(t.y) | tiny1(t.z) | tiny1(t.w);
+          *reinterpret_cast<float4*>(&dst[vk + 4 * i][4 * vf]) = t;
+        }
+      }
+      return tiny;
+    };
+#pragma unroll
+    for (int d = 0; d < AF_PF; ++d) fetch(d, raw[d]);
+    for (int s0 = 0; s0 < nslab; s0 += AF_PF) {
+#pragma unroll
+      for (int d = 0; d < AF_PF; ++d) {
+        const int s = s0 + d, slot = s % AF_SLOTS, ph = s & 15;
+        if (s >= AF_SLOTS && !mbar_wait(&bar_empty[slot], (uint32_t)((s / AF_SLOTS - 1) & 1), abort_flag, nullptr)) return;
+        const bool tiny = store(ph, Ring[slot], raw[d]);
+        fetch(s + AF_PF, raw[d]);
+        const int any = __any_sync(0xffffffffu, tiny);
+        if (lane == 0) tiny_s[slot][pw] = any;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_full[slot]);
+      }
+    }
+    return;
+  }
+  // --------------------------------- consumers ---------------------------------
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  const int tiny_q = tiny_q_s;
+  const int wrow = warp * 16;                       // first row of this warp inside the query block
+  float m_mine = __int_as_float(0xff800000), l_mine = 0.0f, alpha_mine = 0.0f;   // row (lane & 15) of the warp
+  float2 o[8][4];                                   // rows (2a, 2a+1) x column c
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) o[a][c] = make_float2(0.0f, 0.0f);
+  int s = 0;
+  bool ok = true;
+  // slab s is waited for (and its below-2^-63 flags fetched) one slab ahead of its use
+  int tiny_cur = 0;
+  auto acquire = [&](int sn) -> bool {
+    if (sn >= nslab) return true;
+    const int slot = sn % AF_SLOTS;
+    if (!mbar_wait(&bar_full[slot], (uint32_t)((sn / AF_SLOTS) & 1), abort_flag, nullptr)) return false;
+    tiny_cur = tiny_s[slot][0] | tiny_s[slot][1] | tiny_s[slot][2] | tiny_s[slot][3];
+    return true;
+  };
+  ok = acquire(0);
+  for (int jt = 0; jt < ntiles && ok; ++jt) {
+    const int j0 = jt * FK;
+    const bool diag = (jt == ntiles - 1);           // only the last block of a row block reaches past the diagonal
+    // ---- logits: acc[i] = sum over the 128 dimensions ascending of q[row i][d] k[key][d], keys 4 lane .. 4 lane + 3 ----
+    float2 acc[8][4];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][c] = make_float2(0.0f, 0.0f);
+    for (int sl = 0; sl < 8; ++sl, ++s) {
+      const int slot = s % AF_SLOTS;
+      const int tiny = tiny_q | tiny_cur;
+      if (!acquire(s + 1)) { ok = false; break; }     // the next slab's flags travel while this one is multiplied
+      const float* ap = &Qs[sl * OK][wrow];
+      if (tiny) mac_16x4<false, false>(ap, LQ, 0, 0, Ring[slot], lane, acc);
+      else mac_16x4<true, false>(ap, LQ, 0, 0, Ring[slot], lane, acc);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    }
+    if (!ok) break;
+    // ---- online softmax of the warp's 16 rows ----
+    float rm[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int row = q0 + wrow + i;
+      float mt = __int_as_float(0xff800000);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float sv = fmul(RP(acc, i, e), ATT_SCALE);
+        RP(acc, i, e) = sv;
+        if (!diag || j0 + 4 * lane + e <= row) mt = fmaxf(mt, sv);
+      }
+      rm[i] = mt;
+    }
+    // the lane that owns row r (see rows16_reduce) updates its running maximum (every row sees at least key 0 of the
+    // first block, so the maximum of a block it visits is a number) and the rescale factor of what it has accumulated
+    const float m_new = fmaxf(m_mine, rows16_reduce<false>(rm, lane));
+    alpha_mine = det_exp(fsub(m_mine, m_new));
+    m_mine = m_new;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) rm[i] = __shfl_sync(0xffffffffu, m_new, ROW_LANE(i));
+    bool tp = false;
+    // 64 independent exponentials in one straight-line block (no branch, no shuffle in between), so that their
+    // dependent chains interleave; invisible pairs are zeroed afterwards (their arguments may be anything)
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp_sel(fsub(RP(acc, i, e), rm[i]));
+    if (diag) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (j0 + 4 * lane + e > q0 + wrow + i) RP(acc, i, e) = 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float p[4] = {RP(acc, i, 0), RP(acc, i, 1), RP(acc, i, 2), RP(acc, i, 3)};
+      rm[i] = fadd(fadd(p[0], p[1]), fadd(p[2], p[3]));      // the lane's four adjacent slots of the block's row sum
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { p[e] = bf2f(f2bf(p[e])); tp |= tiny1(p[e]); RP(acc, i, e) = p[e]; }
+    }
+    // the rest of the adjacent tree over the block's 128 slots: lanes 1, 2, 4, 8, 16 apart
+    l_mine = fadd(fmul(l_mine, alpha_mine), rows16_reduce<true>(rm, lane));
+    // P~ of the warp's rows: key row 4 lane + e, chunk of rows 4g .. 4g+3
+    __syncwarp();                                    // the previous block's P.V loads are done
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float* prow = Ps + (size_t)(4 * lane + e) * FQ;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const float4 t = make_float4(acc[2 * g][e].x, acc[2 * g][e].y, acc[2 * g + 1][e].x, acc[2 * g + 1][e].y);
+        *reinterpret_cast<float4*>(prow + ((((wrow >> 2) + g) ^ (lane & 7)) << 2)) = t;
+      }
+    }
+    const int tiny_p = __any_sync(0xffffffffu, tp);  // also orders the stores before the loads below
+    __syncwarp();
+    // ---- u = P~ . V over the block's keys ascending from +0, then o = o * alpha + u ----
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][c] = make_float2(0.0f, 0.0f);
+    const int last_slab = diag ? warp : 7;           // on the diagonal the warp's rows see no key past 16 (warp + 1)
+    for (int sl = 0; sl < 8; ++sl, ++s) {
+      const int slot = s % AF_SLOTS;
+      const int tiny = tiny_p | tiny_cur;
+      if (!acquire(s + 1)) { ok = false; break; }
+      if (sl <= last_slab) {
+        const float* ap = Ps + (size_t)(sl * OK) * FQ;
+        if (tiny) mac_16x4<false, true>(ap, FQ, wrow >> 2, sl * OK, Ring[slot], lane, acc);
+        else mac_16x4<true, true>(ap, FQ, wrow >> 2, sl * OK, Ring[slot], lane, acc);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    }
+    if (!ok) break;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {  // scalar: the product o * alpha is rounded before the add
+      const float al = __shfl_sync(0xffffffffu, alpha_mine, ROW_LANE(i));
+#pragma unroll
+      for (int c = 0; c < 4; ++c) RP(o, i, c) = fadd(fmul(RP(o, i, c), al), RP(acc, i, c));
+    }
+  }
+  if (!ok) return;
+  const float il_mine = fdiv(1.0f, l_mine);
+  const float lse_mine = fadd(m_mine, det_log(l_mine));
+  if (lane < 16 && q0 + wrow + ROW_OF_LANE(lane) < S) lse[((size_t)b * H + h) * S + q0 + wrow + ROW_OF_LANE(lane)] = lse_mine;
+  const float inv_q = qout ? fdiv(1.0f, s_q[0]) : 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int row = q0 + wrow + i;
+    const float il = __shfl_sync(0xffffffffu, il_mine, ROW_LANE(i));
+    if (row >= S) continue;
+    uint2 w0;
+    w0.x = pack_bf2(fmul(RP(o, i, 0), il), fmul(RP(o, i, 1), il));
+    w0.y = pack_bf2(fmul(RP(o, i, 2), il), fmul(RP(o, i, 3), il));
+    *reinterpret_cast<uint2*>(out + (row0 + row) * ld_out + (size_t)h * DH + 4 * lane) = w0;
+    if (qout) {   // the output projection's quantiser, applied to the bf16 values just stored
+      const float f0 = bflo(w0.x), f1 = bfhi(w0.x), f2 = bflo(w0.y), f3 = bfhi(w0.y);
+      const uint32_t c = ((uint32_t)(uint8_t)quant1(f0, inv_q)) | ((uint32_t)(uint8_t)quant1(f1, inv_q) << 8) |
+                         ((uint32_t)(uint8_t)quant1(f2, inv_q) << 16) | ((uint32_t)(uint8_t)quant1(f3, inv_q) << 24);
+      *reinterpret_cast<uint32_t*>(qout + (row0 + row) * ld_out + (size_t)h * DH + 4 * lane) = c;
+    }
+  }
+}
+
 
 // ---------------------------------------------------------------------------------------------
 // backward
@@ -404,12 +746,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
         const float dv4[4] = {da[a][2 * g].x, da[a][2 * g].y, da[a][2 * g + 1].x, da[a][2 * g + 1].y};
         float pv[4], dsv[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          pv[e] = 0.0f; dsv[e] = 0.0f;
-          if (jb + e <= i && (W == 0 || jb + e > i - W)) {
-            pv[e] = det_exp(fsub(fmul(sv[e], ATT_SCALE), Lr[a]));
-            dsv[e] = fmul(fmul(pv[e], fsub(dv4[e], Dr[a])), ATT_SCALE);
-          }
+        for (int e = 0; e < 4; ++e) {   // branch-free (selects), so that the exponentials' chains interleave
+          const bool vis = jb + e <= i && (W == 0 || jb + e > i - W);
+          const float pe = det_exp_sel(fsub(fmul(sv[e], ATT_SCALE), Lr[a]));
+          const float de = fmul(fmul(pe, fsub(dv4[e], Dr[a])), ATT_SCALE);
+          pv[e] = vis ? pe : 0.0f;
+          dsv[e] = vis ? de : 0.0f;
         }
         const size_t off = (bh * S + i) * S + jb;
         uint2 u;
@@ -433,13 +775,13 @@ static int attn_fwd_impl(const det_bf16* q, const det_bf16* k, const det_bf16* v
   if (qout && (!s_q || (((uintptr_t)qout) & 3u))) return qout && !s_q ? DET_ERR_ARG : DET_ERR_ALIGN;
   if (S % 64 || ld % 8 || ld_out % 8 || ld < H * DH || ld_out < H * DH || H % Hkv || window % 128) return DET_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DET_ERR_ALIGN;
-  static DevOnce once_full = {}, once_win = {};
-  if (dev_ensure_smem(once_full, (const void*)k_attn_fwd<false>, FWD_SMEM) != DET_OK ||
-      dev_ensure_smem(once_win, (const void*)k_attn_fwd<true>, FWD_SMEM) != DET_OK)
-    return DET_ERR_CUDA;
+  static DevOnce once_win = {};
+  if (dev_ensure_smem(once_win, (const void*)k_attn_fwd<true>, FWD_SMEM) != DET_OK) return DET_ERR_CUDA;
   dim3 grid(H * B, (S + FQ - 1) / FQ);
+  static DevOnce once_ws = {};
+  if (dev_ensure_smem(once_ws, (const void*)k_attn_fwd_ws, AFW_SMEM) != DET_OK) return DET_ERR_CUDA;
   if (window) k_attn_fwd<true><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, window, out, ld_out, lse, s_q, qout);
-  else k_attn_fwd<false><<<DET_L(grid), FT, FWD_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, 0, out, ld_out, lse, s_q, qout);
+  else k_attn_fwd_ws<<<DET_L(grid), AF_THREADS, AFW_SMEM, (cudaStream_t)stream>>>(q, k, v, ld, H, Hkv, S, out, ld_out, lse, s_q, qout);
   DET_CHECK_LAUNCH();
   return DET_OK;
 }

@@ -74,6 +74,30 @@ __device__ __forceinline__ float det_exp(float x) {
   return fmul(p, __int_as_float((k + 127) << 23));
 }
 
+// det_exp without branches: the same operations and the same results for every input, with the special ranges chosen by
+// selects, so that several independent evaluations interleave in one instruction stream (a kernel that evaluates many
+// exponentials per thread is bound by the latency of this chain, not by its instruction count).
+__device__ __forceinline__ float det_exp_sel(float x) {
+  const float km = fadd(fmul(x, 0x1.715476p+0f), 12582912.0f);
+  const float kf = fsub(km, 12582912.0f);
+  const float r = fsub(fsub(x, fmul(kf, 0x1.62e400p-1f)), fmul(kf, 0x1.7f7d1cp-20f));
+  float p = 0x1.a01a02p-13f;
+  p = fadd(fmul(p, r), 0x1.6c16c2p-10f);
+  p = fadd(fmul(p, r), 0x1.111112p-7f);
+  p = fadd(fmul(p, r), 0x1.555556p-5f);
+  p = fadd(fmul(p, r), 0x1.555556p-3f);
+  p = fadd(fmul(p, r), 0.5f);
+  p = fadd(fmul(p, r), 1.0f);
+  p = fadd(fmul(p, r), 1.0f);
+  const int k = (int)__float_as_uint(km) - 0x4B400000;
+  const float big = fmul(fmul(p, 0x1p127f), 2.0f);                              // k = 128
+  float v = fmul(p, __int_as_float((min(max(k, -127), 127) + 127) << 23));      // k in [-126, 127] wherever v is kept
+  v = (k > 127) ? big : v;
+  v = (x < -0x1.5d58a0p+6f) ? 0.0f : v;
+  v = (x > 0x1.62e42ep+6f) ? __int_as_float(0x7f800000) : v;
+  return v;
+}
+
 // NOTE on the packed two-lane FP32 instructions (mul/add/fma .f32x2): each lane of a single packed instruction
 // rounds exactly like the scalar instruction, but ptxas contracts a packed multiply followed by a packed add into one
 // fused instruction even when both carry .rn and --fmad=false is given (measured on this toolchain: the result
