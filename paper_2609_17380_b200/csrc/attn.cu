@@ -179,11 +179,11 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
-      const float al = det_exp_sel(fsub(m[i], mt));
+      const float al = det_exp(fsub(m[i], mt));
       alpha[i] = rowvalid ? al : 1.0f;
       float p[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) p[e] = det_exp_sel(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
+      for (int e = 0; e < 8; ++e) p[e] = det_exp(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
 #pragma unroll
       for (int e = 0; e < 8; ++e) p[e] = valid[e] ? p[e] : 0.0f;
 #pragma unroll
@@ -275,7 +275,7 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
 // K and V arrive through an mbarrier-guarded ring of 16-deep slabs filled by four producer warps (K: 16 head dimensions
 // x 128 keys, eight per block; V: 16 keys x 128 dimensions, eight per block), so no block-wide barrier is left in the
 // loop and consumer warps are not coupled to each other.  The softmax evaluates its 64 exponentials per lane as one
-// straight-line block of branch-free chains (det_exp_sel) and reduces the 16 rows with 16 shuffles per reduction.
+// straight-line block of branch-free chains and reduces the 16 rows with 16 shuffles per reduction.
 // On the diagonal block a warp stops P.V after the last key any of its rows may see.
 // Arithmetic and order per output are exactly those of k_attn_fwd (and of the definition): bit-identical results.
 // ---------------------------------------------------------------------------------------------
@@ -519,7 +519,7 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
 #pragma unroll
     for (int i = 0; i < 16; ++i)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp_sel(fsub(RP(acc, i, e), rm[i]));
+      for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp(fsub(RP(acc, i, e), rm[i]));
     if (diag) {
 #pragma unroll
       for (int i = 0; i < 16; ++i)
@@ -748,7 +748,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {   // branch-free (selects), so that the exponentials' chains interleave
           const bool vis = jb + e <= i && (W == 0 || jb + e > i - W);
-          const float pe = det_exp_sel(fsub(fmul(sv[e], ATT_SCALE), Lr[a]));
+          const float pe = det_exp(fsub(fmul(sv[e], ATT_SCALE), Lr[a]));
           const float de = fmul(fmul(pe, fsub(dv4[e], Dr[a])), ATT_SCALE);
           pv[e] = vis ? pe : 0.0f;
           dsv[e] = vis ? de : 0.0f;

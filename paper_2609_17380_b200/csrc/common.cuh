@@ -52,32 +52,13 @@ __device__ __forceinline__ uint2 quant8(const float v[8], float inv_s) {
 
 // exp: x = k ln2 + r, degree-7 Taylor polynomial in Horner form, one multiply and one add per step,
 // scaled through the exponent field.  Results below 2^-126 flush to +0; above FLT_MAX give +inf.
+// Written without branches: the special ranges are chosen by selects, so that several independent evaluations
+// interleave in one instruction stream (a kernel that evaluates many exponentials per thread is bound by the latency
+// of this chain, not by its instruction count).
+//   k = rne(x log2 e): adding 1.5 * 2^23 rounds to the nearest even integer exactly like rintf for |t| < 2^22 (here
+//   |t| < 2^8 wherever the result is kept) and leaves k in the low bits of the sum, so neither the rounding nor the
+//   conversion needs the conversion pipe.
 __device__ __forceinline__ float det_exp(float x) {
-  if (x > 0x1.62e42ep+6f) return __int_as_float(0x7f800000);
-  if (x < -0x1.5d58a0p+6f) return 0.0f;
-  // k = rne(x log2 e): adding 1.5 * 2^23 rounds to the nearest even integer exactly like rintf for |t| < 2^22 (here
-  // |t| < 2^8) and leaves k in the low bits of the sum, so neither the rounding nor the conversion needs the
-  // conversion pipe
-  const float km = fadd(fmul(x, 0x1.715476p+0f), 12582912.0f);
-  const float kf = fsub(km, 12582912.0f);
-  float r = fsub(fsub(x, fmul(kf, 0x1.62e400p-1f)), fmul(kf, 0x1.7f7d1cp-20f));
-  float p = 0x1.a01a02p-13f;
-  p = fadd(fmul(p, r), 0x1.6c16c2p-10f);
-  p = fadd(fmul(p, r), 0x1.111112p-7f);
-  p = fadd(fmul(p, r), 0x1.555556p-5f);
-  p = fadd(fmul(p, r), 0x1.555556p-3f);
-  p = fadd(fmul(p, r), 0.5f);
-  p = fadd(fmul(p, r), 1.0f);
-  p = fadd(fmul(p, r), 1.0f);
-  const int k = (int)__float_as_uint(km) - 0x4B400000;
-  if (k > 127) return fmul(fmul(p, 0x1p127f), 2.0f);
-  return fmul(p, __int_as_float((k + 127) << 23));
-}
-
-// det_exp without branches: the same operations and the same results for every input, with the special ranges chosen by
-// selects, so that several independent evaluations interleave in one instruction stream (a kernel that evaluates many
-// exponentials per thread is bound by the latency of this chain, not by its instruction count).
-__device__ __forceinline__ float det_exp_sel(float x) {
   const float km = fadd(fmul(x, 0x1.715476p+0f), 12582912.0f);
   const float kf = fsub(km, 12582912.0f);
   const float r = fsub(fsub(x, fmul(kf, 0x1.62e400p-1f)), fmul(kf, 0x1.7f7d1cp-20f));
@@ -97,6 +78,8 @@ __device__ __forceinline__ float det_exp_sel(float x) {
   v = (x > 0x1.62e42ep+6f) ? __int_as_float(0x7f800000) : v;
   return v;
 }
+
+
 
 // NOTE on the packed two-lane FP32 instructions (mul/add/fma .f32x2): each lane of a single packed instruction
 // rounds exactly like the scalar instruction, but ptxas contracts a packed multiply followed by a packed add into one

@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
     for (int h = 0; h < 2; ++h) {
       if (e0 + 4 * h < V) {
         float4 a = *reinterpret_cast<const float4*>(z + e0 + 4 * h);
-        e[4 * h] = det_exp(fsub(a.x, m)); e[4 * h + 1] = det_exp(fsub(a.y, m));
+        e[4 * h] = det_exp(fsub(a.x, m)); e[4 * h + 1] = det_exp(fsub(a.y, m));     // branch-free: the chains interleave
         e[4 * h + 2] = det_exp(fsub(a.z, m)); e[4 * h + 3] = det_exp(fsub(a.w, m));
       } else {
         e[4 * h] = e[4 * h + 1] = e[4 * h + 2] = e[4 * h + 3] = 0.0f;

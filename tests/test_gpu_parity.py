@@ -86,6 +86,23 @@ def test_exp_all_bf16_arguments(det):
     assert_same_bits(host(out), oracle.prim("exp", x), "exp")
 
 
+def test_exp_dense_grid_and_ends_of_the_range(det):
+    """A dense f32 grid over [-100, 100], every float within a few ULP of the two thresholds of the definition (the
+    largest argument with a finite result, the smallest with a non-zero one), of 0 and of the points where k changes,
+    and the infinities: bit for bit (the device evaluates the sequence with selects instead of branches)."""
+    grid = np.linspace(-100.0, 100.0, 400001).astype(F)
+    ends = []
+    for c in (float.fromhex("0x1.62e42ep+6"), float.fromhex("-0x1.5d58a0p+6"), 0.0, 0.34657359, -0.34657359, 88.0, -87.0, 1.0, -1.0):
+        b = np.array([c], F).view(np.int32)[0]
+        ends.append((np.arange(-40, 41, dtype=np.int64) + int(b)).astype(np.int32).view(F))
+    x = np.concatenate([grid] + ends + [np.array([np.inf, -np.inf, 3.0e38, -3.0e38, 1e-45, -1e-45, 1e-30], F)])
+    x = x[~np.isnan(x)]                       # the patterns just below +0 are NaNs; their payloads are not defined
+    out = empty(x.shape, F)
+    det.det_test_prim(oracle.OPS["exp"], dev(x), None, out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("exp", x), "exp")
+
+
 def test_log_ends_of_the_domain_and_nan_logits(det):
     """det_log keeps a non-finite or non-positive argument visible; a NaN logit therefore gives a NaN loss, not a finite
     number that depends on the NaN's payload.  NaNs are compared as NaNs, everything else bit for bit."""
