@@ -279,28 +279,27 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
 // On the diagonal block a warp stops P.V after the last key any of its rows may see.
 // Arithmetic and order per output are exactly those of k_attn_fwd (and of the definition): bit-identical results.
 // ---------------------------------------------------------------------------------------------
-constexpr int AF_SLOTS = 8, AF_PF = 4, AF_CONS = 256, AF_PROD = 128, AF_THREADS = AF_CONS + AF_PROD;
+constexpr int AF_RW = 8;                      // query rows per consumer warp (8: sixteen consumer warps, 16: eight)
+constexpr int AF_SLOTS = 8, AF_PF = 4, AF_CONS = (FQ / AF_RW) * 32, AF_PROD = 128, AF_THREADS = AF_CONS + AF_PROD;
 constexpr size_t AFW_SMEM = (size_t)(DH * LQ + FK * FQ + AF_SLOTS * OK * (OT + 4)) * sizeof(float);
 
-// one 16-deep slab: acc[i/2][c].{x,y} += A[k][rows i, i+1 of the warp] * B[k][4 lane + c]: the accumulators pair two ROWS, so
-// the row operand's register pairs come straight out of its 16-byte loads and only the four column values are duplicated
-// into pairs.  A chunk g (rows 4g..4g+3) of step k is at ap + k * a_ld + ((chunk0 + g) ^ (PSWZ ? swizzle of the key : 0)) * 4.
+// one 16-deep slab: (row i, column c) += A[k][row i of the warp] * B[k][4 lane + c], accumulators laid out as RP() says.  A chunk g (rows 4g..4g+3) of step k is at ap + k * a_ld + ((chunk0 + g) ^ (PSWZ ? swizzle of the key : 0)) * 4.
 template <bool FUSED, bool PSWZ>
 __device__ __forceinline__ void mac_16x4(const float* __restrict__ ap, int a_ld, int chunk0, int key0,
-                                         const float (*Bs)[OT + 4], int lane, float2 (&acc)[8][4]) {
+                                         const float (*Bs)[OT + 4], int lane, float2 (&acc)[AF_RW / 2][4]) {
 #pragma unroll
   for (int k = 0; k < OK; ++k) {
     const int sw = PSWZ ? (((key0 + k) >> 2) & 7) : 0;
-    float4 a[4];
+    float4 a[AF_RW / 4];
 #pragma unroll
-    for (int g = 0; g < 4; ++g) a[g] = *reinterpret_cast<const float4*>(ap + (size_t)k * a_ld + (((chunk0 + g) ^ sw) << 2));
+    for (int g = 0; g < AF_RW / 4; ++g) a[g] = *reinterpret_cast<const float4*>(ap + (size_t)k * a_ld + (((chunk0 + g) ^ sw) << 2));
     const float4 bv = *reinterpret_cast<const float4*>(&Bs[k][4 * lane]);
     const float bs[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       const float2 bb = make_float2(bs[c], bs[c]);
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
+      for (int g = 0; g < AF_RW / 4; ++g) {
         if (FUSED) {
           acc[2 * g][c] = __ffma2_rn(make_float2(a[g].x, a[g].y), bb, acc[2 * g][c]);
           acc[2 * g + 1][c] = __ffma2_rn(make_float2(a[g].z, a[g].w), bb, acc[2 * g + 1][c]);
@@ -314,28 +313,46 @@ __device__ __forceinline__ void mac_16x4(const float* __restrict__ ap, int a_ld,
     }
   }
 }
-// element (row i, column c) of a row-paired accumulator set; i is a compile-time constant wherever this is used
+// element (row i, column c) of a row-paired accumulator set (pair [i/2][c] holds rows i, i+1 of column c, so the row
+// operand's register pairs come straight out of its 16-byte loads and only the four column values are duplicated into
+// pairs); i is a compile-time constant wherever this is used
 #define RP(acc, i, c) (((i) & 1) ? (acc)[(i) >> 1][c].y : (acc)[(i) >> 1][c].x)
 // Reduction of 16 rows across the warp (x[i]: this lane's value for row i) with partners 1, 2, 4, 8, 16 lanes apart in that
 // order, which for sums is the adjacent pairwise tree over the lanes.  Instead of 16 butterflies of five shuffles every
 // stage halves the rows a lane carries (it sends its partner the half the partner keeps): 8 + 4 + 2 + 1 + 1 shuffles, and
 // lane L ends with the result of row ROW_OF_LANE(L); both operand orders of an addition or a maximum give the same bits.
-#define ROW_OF_LANE(L) ((((L) & 1) << 3) | (((L) & 2) << 1) | (((L) & 4) >> 1) | (((L) & 8) >> 3))
+#define ROW_OF_LANE(L) (AF_RW == 16 ? ((((L) & 1) << 3) | (((L) & 2) << 1) | (((L) & 4) >> 1) | (((L) & 8) >> 3)) \
+                                    : ((((L) & 1) << 2) | ((L) & 2) | (((L) & 4) >> 2)))
 #define ROW_LANE(i) ROW_OF_LANE(i)   /* a lane that holds row i (the bit reversal is its own inverse) */
 template <bool SUM>
-__device__ __forceinline__ float rows16_reduce(const float (&x)[16], int lane) {
+__device__ __forceinline__ float rows_reduce(const float (&x)[AF_RW], int lane) {
   auto op = [](float a, float b) { return SUM ? fadd(a, b) : fmaxf(a, b); };
-  float a[8], b[4], c[2];
   const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4, b3 = lane & 8;
+  float d;
+  if (AF_RW == 16) {
+    float a[8], b[4], c[2];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) a[j] = op(b0 ? x[8 + j] : x[j], __shfl_xor_sync(0xffffffffu, b0 ? x[j] : x[8 + j], 1));
+    for (int j = 0; j < 8; ++j) a[j] = op(b0 ? x[(8 + j) % AF_RW] : x[j], __shfl_xor_sync(0xffffffffu, b0 ? x[j] : x[(8 + j) % AF_RW], 1));
 #pragma unroll
-  for (int j = 0; j < 4; ++j) b[j] = op(b1 ? a[4 + j] : a[j], __shfl_xor_sync(0xffffffffu, b1 ? a[j] : a[4 + j], 2));
+    for (int j = 0; j < 4; ++j) b[j] = op(b1 ? a[4 + j] : a[j], __shfl_xor_sync(0xffffffffu, b1 ? a[j] : a[4 + j], 2));
 #pragma unroll
-  for (int j = 0; j < 2; ++j) c[j] = op(b2 ? b[2 + j] : b[j], __shfl_xor_sync(0xffffffffu, b2 ? b[j] : b[2 + j], 4));
-  float d = op(b3 ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, b3 ? c[0] : c[1], 8));
+    for (int j = 0; j < 2; ++j) c[j] = op(b2 ? b[2 + j] : b[j], __shfl_xor_sync(0xffffffffu, b2 ? b[j] : b[2 + j], 4));
+    d = op(b3 ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, b3 ? c[0] : c[1], 8));
+  } else {
+    float b[4], c[2];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) b[j] = op(b0 ? x[4 + j] : x[j], __shfl_xor_sync(0xffffffffu, b0 ? x[j] : x[4 + j], 1));
+#pragma unroll
+    for (int j = 0; j < 2; ++j) c[j] = op(b1 ? b[2 + j] : b[j], __shfl_xor_sync(0xffffffffu, b1 ? b[j] : b[2 + j], 2));
+    d = op(b2 ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, b2 ? c[0] : c[1], 4));
+    d = op(d, __shfl_xor_sync(0xffffffffu, d, 8));
+  }
   return op(d, __shfl_xor_sync(0xffffffffu, d, 16));
 }
+// Register hand-over between the roles (setmaxnreg): the counts after it must fit into what the block was launched with
+// (threads x the launch-time register count: 384 x 168 for 16 rows per warp, 640 x 96 for 8), or the increase never returns.
+static_assert(AF_RW == 16 ? (AF_CONS * 216 + AF_PROD * 72 <= AF_THREADS * 168) : (AF_CONS * 104 + AF_PROD * 64 <= AF_THREADS * 96),
+              "register hand-over exceeds the block's allocation");
 __global__ void __launch_bounds__(AF_THREADS, 1)
     k_attn_fwd_ws(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k, const uint16_t* __restrict__ v, int ld,
                   int H, int Hkv, int S, uint16_t* __restrict__ out, int ld_out, float* __restrict__ lse,
@@ -382,7 +399,7 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
   __syncthreads();
   if (tid >= AF_CONS) {
     // ------------------------------- producers -------------------------------
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(AF_RW == 16 ? 72 : 64));
     const int pt = tid - AF_CONS, pw = pt >> 5;
     // Slab s of the block sequence: block s / 16; s % 16 < 8: K, head dimensions 16 (s % 16) .. (thread = key, two
     // 16-byte words); else V, keys 16 (s % 16 - 8) .. (thread = four dimensions of keys kk, kk + 4, kk + 8, kk + 12).
@@ -451,13 +468,13 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     return;
   }
   // --------------------------------- consumers ---------------------------------
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(AF_RW == 16 ? 216 : 104));
   const int tiny_q = tiny_q_s;
-  const int wrow = warp * 16;                       // first row of this warp inside the query block
+  const int wrow = warp * AF_RW;                      // first row of this warp inside the query block
   float m_mine = __int_as_float(0xff800000), l_mine = 0.0f, alpha_mine = 0.0f;   // row (lane & 15) of the warp
-  float2 o[8][4];                                   // rows (2a, 2a+1) x column c
+  float2 o[AF_RW / 2][4];                                   // rows (2a, 2a+1) x column c
 #pragma unroll
-  for (int a = 0; a < 8; ++a)
+  for (int a = 0; a < AF_RW / 2; ++a)
 #pragma unroll
     for (int c = 0; c < 4; ++c) o[a][c] = make_float2(0.0f, 0.0f);
   int s = 0;
@@ -476,9 +493,9 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     const int j0 = jt * FK;
     const bool diag = (jt == ntiles - 1);           // only the last block of a row block reaches past the diagonal
     // ---- logits: acc[i] = sum over the 128 dimensions ascending of q[row i][d] k[key][d], keys 4 lane .. 4 lane + 3 ----
-    float2 acc[8][4];
+    float2 acc[AF_RW / 2][4];
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
+    for (int a = 0; a < AF_RW / 2; ++a)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[a][c] = make_float2(0.0f, 0.0f);
     for (int sl = 0; sl < 8; ++sl, ++s) {
@@ -493,9 +510,9 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     }
     if (!ok) break;
     // ---- online softmax of the warp's 16 rows ----
-    float rm[16];
+    float rm[AF_RW];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < AF_RW; ++i) {
       const int row = q0 + wrow + i;
       float mt = __int_as_float(0xff800000);
 #pragma unroll
@@ -508,42 +525,42 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     }
     // the lane that owns row r (see rows16_reduce) updates its running maximum (every row sees at least key 0 of the
     // first block, so the maximum of a block it visits is a number) and the rescale factor of what it has accumulated
-    const float m_new = fmaxf(m_mine, rows16_reduce<false>(rm, lane));
+    const float m_new = fmaxf(m_mine, rows_reduce<false>(rm, lane));
     alpha_mine = det_exp(fsub(m_mine, m_new));
     m_mine = m_new;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) rm[i] = __shfl_sync(0xffffffffu, m_new, ROW_LANE(i));
+    for (int i = 0; i < AF_RW; ++i) rm[i] = __shfl_sync(0xffffffffu, m_new, ROW_LANE(i));
     bool tp = false;
     // 64 independent exponentials in one straight-line block (no branch, no shuffle in between), so that their
     // dependent chains interleave; invisible pairs are zeroed afterwards (their arguments may be anything)
 #pragma unroll
-    for (int i = 0; i < 16; ++i)
+    for (int i = 0; i < AF_RW; ++i)
 #pragma unroll
       for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp(fsub(RP(acc, i, e), rm[i]));
     if (diag) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
+      for (int i = 0; i < AF_RW; ++i)
 #pragma unroll
         for (int e = 0; e < 4; ++e)
           if (j0 + 4 * lane + e > q0 + wrow + i) RP(acc, i, e) = 0.0f;
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < AF_RW; ++i) {
       float p[4] = {RP(acc, i, 0), RP(acc, i, 1), RP(acc, i, 2), RP(acc, i, 3)};
       rm[i] = fadd(fadd(p[0], p[1]), fadd(p[2], p[3]));      // the lane's four adjacent slots of the block's row sum
 #pragma unroll
       for (int e = 0; e < 4; ++e) { p[e] = bf2f(f2bf(p[e])); tp |= tiny1(p[e]); RP(acc, i, e) = p[e]; }
     }
     // the rest of the adjacent tree over the block's 128 slots: lanes 1, 2, 4, 8, 16 apart
-    l_mine = fadd(fmul(l_mine, alpha_mine), rows16_reduce<true>(rm, lane));
+    l_mine = fadd(fmul(l_mine, alpha_mine), rows_reduce<true>(rm, lane));
     // P~ of the warp's rows: key row 4 lane + e, chunk of rows 4g .. 4g+3
     __syncwarp();                                    // the previous block's P.V loads are done
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       float* prow = Ps + (size_t)(4 * lane + e) * FQ;
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        const float4 t = make_float4(acc[2 * g][e].x, acc[2 * g][e].y, acc[2 * g + 1][e].x, acc[2 * g + 1][e].y);
+      for (int g = 0; g < AF_RW / 4; ++g) {
+        const float4 t = make_float4(RP(acc, 4 * g, e), RP(acc, 4 * g + 1, e), RP(acc, 4 * g + 2, e), RP(acc, 4 * g + 3, e));
         *reinterpret_cast<float4*>(prow + ((((wrow >> 2) + g) ^ (lane & 7)) << 2)) = t;
       }
     }
@@ -551,10 +568,10 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     __syncwarp();
     // ---- u = P~ . V over the block's keys ascending from +0, then o = o * alpha + u ----
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
+    for (int a = 0; a < AF_RW / 2; ++a)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[a][c] = make_float2(0.0f, 0.0f);
-    const int last_slab = diag ? warp : 7;           // on the diagonal the warp's rows see no key past 16 (warp + 1)
+    const int last_slab = diag ? (wrow + AF_RW - 1) / OK : 7;          // on the diagonal the warp's rows see no key past 16 (warp + 1)
     for (int sl = 0; sl < 8; ++sl, ++s) {
       const int slot = s % AF_SLOTS;
       const int tiny = tiny_p | tiny_cur;
@@ -569,7 +586,7 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     }
     if (!ok) break;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {  // scalar: the product o * alpha is rounded before the add
+    for (int i = 0; i < AF_RW; ++i) {  // scalar: the product o * alpha is rounded before the add
       const float al = __shfl_sync(0xffffffffu, alpha_mine, ROW_LANE(i));
 #pragma unroll
       for (int c = 0; c < 4; ++c) RP(o, i, c) = fadd(fmul(RP(o, i, c), al), RP(acc, i, c));
@@ -578,10 +595,10 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
   if (!ok) return;
   const float il_mine = fdiv(1.0f, l_mine);
   const float lse_mine = fadd(m_mine, det_log(l_mine));
-  if (lane < 16 && q0 + wrow + ROW_OF_LANE(lane) < S) lse[((size_t)b * H + h) * S + q0 + wrow + ROW_OF_LANE(lane)] = lse_mine;
+  if (lane < AF_RW && q0 + wrow + ROW_OF_LANE(lane) < S) lse[((size_t)b * H + h) * S + q0 + wrow + ROW_OF_LANE(lane)] = lse_mine;
   const float inv_q = qout ? fdiv(1.0f, s_q[0]) : 0.0f;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < AF_RW; ++i) {
     const int row = q0 + wrow + i;
     const float il = __shfl_sync(0xffffffffu, il_mine, ROW_LANE(i));
     if (row >= S) continue;
