@@ -1,0 +1,57 @@
+"""CPU oracle, arithmetic version 2 -- TEST INFRASTRUCTURE ONLY.
+
+Version 2 replaces one definition of version 1: the LM-head contraction becomes an order-free, exactly defined sum of
+integer products of aligned bf16 significands with a single rounding (see v2.c).  It lives in files of its own so that
+version 1 and everything keyed to its sources stay untouched.  bf16 tensors are numpy uint16 bit patterns.
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_DIR, "liboracle_v2.so")
+_SRC = os.path.join(_DIR, "v2.c")
+_lib = None
+
+
+def build(force=False):
+    if not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC):
+        return _SO
+    subprocess.check_call(["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-msse4.1", "-fopenmp", "-shared", "-fPIC", "-o", _SO,
+                           _SRC, "-lm"])
+    return _SO
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = C.CDLL(_SO)
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def slice_rows(X):
+    """X bf16 [R,K] -> (hi int8 [R,K], lo int8 [R,K], E int32 [R]); bit 30 of E marks a row with a non-finite value."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    R, K = X.shape
+    hi, lo, E = np.empty((R, K), np.int8), np.empty((R, K), np.int8), np.empty(R, np.int32)
+    lib().orc2_slice_rows(_p(X), C.c_int(R), C.c_int(K), _p(hi), _p(lo), _p(E))
+    return hi, lo, E
+
+
+def lmhead_fwd(Hh, W):
+    """logits f32 [M,V]: version-2 contraction of the rows of Hh [M,K] with the rows of W [V,K]."""
+    Hh = np.ascontiguousarray(Hh, dtype=np.uint16)
+    W = np.ascontiguousarray(W, dtype=np.uint16)
+    M, K = Hh.shape
+    V = W.shape[0]
+    assert W.shape[1] == K
+    out = np.empty((M, V), np.float32)
+    lib().orc2_lmhead_fwd(_p(Hh), _p(W), C.c_int(M), C.c_int(V), C.c_int(K), _p(out))
+    return out

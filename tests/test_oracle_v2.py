@@ -1,0 +1,133 @@
+"""Pins of the version-2 oracle (order-free, exactly defined LM-head contraction): hand-worked slices, a brute-force
+restatement in exact rational arithmetic that starts from the VALUES (not the bit fields), the case in which nothing is
+truncated and the result must be the correctly rounded exact dot product, order-freedom, an error bound against float64,
+and the special rows."""
+from fractions import Fraction
+
+import numpy as np
+
+import synth
+from oracle import v2
+
+F = np.float32
+
+
+def _val(h):
+    return float(synth.from_bf16(np.array([h], np.uint16))[0])
+
+
+def _rn_f32(fr):
+    """Exactly representable-in-double rational -> binary32, nearest even (one rounding), flushed below 2^-126."""
+    d = float(fr)
+    assert Fraction(d) == fr
+    r = F(d)
+    return F(np.copysign(0.0, r)) if abs(r) < 2.0 ** -126 else r
+
+
+def _brute(a_bits, b_bits):
+    """Version-2 contraction of two rows from their values: scale = 2^(floor(log2 max|x|) - 13), T = trunc(x / scale)."""
+    def aligned(bits):
+        vals = [Fraction(_val(h)) for h in bits]
+        vals = [v if abs(v) >= Fraction(2) ** -126 else Fraction(0) for v in vals]      # flushed subnormals
+        mx = max(abs(v) for v in vals)
+        if mx == 0:
+            return [0] * len(vals), Fraction(1)
+        e = 0
+        while Fraction(2) ** (e + 1) <= mx:
+            e += 1
+        while Fraction(2) ** e > mx:
+            e -= 1
+        scale = Fraction(2) ** (e - 13)
+        T = [int(abs(v) / scale) * (1 if v >= 0 else -1) for v in vals]                  # truncation toward zero
+        return T, scale
+    Ta, sa = aligned(a_bits)
+    Tb, sb = aligned(b_bits)
+    return _rn_f32(sum(x * y for x, y in zip(Ta, Tb)) * sa * sb)
+
+
+def test_slices_by_hand():
+    x = synth.to_bf16(np.array([[1.0, 0.5, -3.0, 0.0, 3.0 * 2.0 ** -7, -2.0 ** -13, 2.0 ** -14]], F))
+    hi, lo, E = v2.slice_rows(x)
+    assert E[0] == 128                                   # 3.0 = 1.5 * 2^1
+    T = hi.astype(np.int32) * 128 + lo.astype(np.int32)
+    # units of 2^(128 - 140) = 2^-12: 1.0 -> 4096, 0.5 -> 2048, -3.0 -> -12288, 3 * 2^-7 -> 96, -2^-13 -> -0 (half a unit,
+    # truncated), 2^-14 -> 0
+    assert T[0].tolist() == [4096, 2048, -12288, 0, 96, 0, 0]
+    assert hi[0].tolist() == [32, 16, -96, 0, 0, 0, 0] and lo[0].tolist() == [0, 0, 0, 0, 96, 0, 0]
+    assert np.abs(hi.astype(np.int32)).max() <= 127 and np.abs(lo.astype(np.int32)).max() <= 127
+
+
+def test_slices_reconstruct_the_truncated_values():
+    x = synth.normal_bf16((5, 256), 1.0, seed=3, tid=1)
+    x[1] = synth.to_bf16((synth.normal_f32(256, 1.0, seed=3, tid=2) * np.exp2(np.arange(256) % 20 - 10.0)).astype(F))   # wide range
+    hi, lo, E = v2.slice_rows(x)
+    T = hi.astype(np.int64) * 128 + lo.astype(np.int64)
+    xv = synth.from_bf16(x).astype(np.float64)
+    for r in range(5):
+        unit = 2.0 ** (int(E[r]) - 140)
+        want = np.trunc(xv[r] / unit)
+        assert np.array_equal(T[r], want.astype(np.int64)), r
+        assert np.max(np.abs(xv[r] - T[r] * unit)) < unit
+        assert (hi[r].astype(np.int32) * lo[r].astype(np.int32) >= 0).all()      # both slices carry the sign
+
+
+def test_brute_force_in_exact_rational_arithmetic():
+    rng = np.random.default_rng(0)
+    for trial in range(6):
+        K = [1, 3, 8, 17, 32, 40][trial]
+        a = synth.to_bf16((rng.standard_normal((3, K)) * np.exp2(rng.integers(-9, 9, (3, K)))).astype(F))
+        b = synth.to_bf16((rng.standard_normal((4, K)) * np.exp2(rng.integers(-20, 3, (4, K)))).astype(F))
+        got = v2.lmhead_fwd(a, b)
+        for m in range(3):
+            for n in range(4):
+                want = _brute(a[m], b[n])
+                assert got[m, n].view(np.uint32) == F(want).view(np.uint32), (trial, m, n, got[m, n], want)
+
+
+def test_without_truncation_the_result_is_the_correctly_rounded_dot_product():
+    """Rows whose values all lie within a factor 64 of the row's largest are kept exactly, so the contraction is the exact
+    dot product of the bf16 values rounded once: a closed form that no ordered binary32 chain reaches in general."""
+    rng = np.random.default_rng(1)
+    K = 96
+    a = synth.to_bf16((rng.uniform(1.0, 1.99, (4, K)) * np.exp2(rng.integers(-6, 1, (4, K))) * rng.choice([-1, 1], (4, K))).astype(F))
+    b = synth.to_bf16((rng.uniform(1.0, 1.99, (5, K)) * np.exp2(rng.integers(-9, -3, (5, K))) * rng.choice([-1, 1], (5, K))).astype(F))
+    a[:, 0] = synth.to_bf16(np.array([1.5], F))[0]          # pins the row exponents at the top of the range
+    b[:, 0] = synth.to_bf16(np.array([2.0 ** -4 * 1.25], F))[0]
+    got = v2.lmhead_fwd(a, b)
+    av, bv = synth.from_bf16(a), synth.from_bf16(b)
+    for m in range(4):
+        for n in range(5):
+            exact = sum(Fraction(float(x)) * Fraction(float(y)) for x, y in zip(av[m], bv[n]))
+            assert got[m, n].view(np.uint32) == _rn_f32(exact).view(np.uint32), (m, n)
+
+
+def test_order_free_and_close_to_float64():
+    a = synth.normal_bf16((6, 512), 1.0, seed=5, tid=1)
+    b = synth.normal_bf16((7, 512), 0.02, seed=5, tid=2)
+    got = v2.lmhead_fwd(a, b)
+    perm = np.random.default_rng(2).permutation(512)
+    assert np.array_equal(v2.lmhead_fwd(a[:, perm], b[:, perm]).view(np.uint32), got.view(np.uint32))
+    av, bv = synth.from_bf16(a).astype(np.float64), synth.from_bf16(b).astype(np.float64)
+    ref = av @ bv.T
+    _, _, Ea = v2.slice_rows(a)
+    _, _, Eb = v2.slice_rows(b)
+    ua, ub = np.exp2(Ea.astype(np.float64) - 140), np.exp2(Eb.astype(np.float64) - 140)
+    # every operand is off by less than one unit of its row: |error| <= sum(|a| ub + |b| ua + ua ub) + half an ulp of the result
+    bound = np.abs(av).sum(1)[:, None] * ub[None, :] + ua[:, None] * np.abs(bv).sum(1)[None, :] + 512 * ua[:, None] * ub[None, :]
+    assert np.all(np.abs(got - ref) <= bound + np.abs(ref) * 2.0 ** -24)
+    assert np.max(np.abs(got - ref)) < 2e-3 * np.max(np.abs(ref))      # and in practice far inside it
+
+
+def test_special_rows():
+    a = synth.normal_bf16((4, 64), 1.0, seed=6, tid=1)
+    b = synth.normal_bf16((3, 64), 1.0, seed=6, tid=2)
+    a[1] = 0
+    a[2, 5] = 0x7F80                                   # +inf
+    b[1, 9] = 0x7FC0                                   # NaN
+    a[3, :] = 0x0001                                   # subnormal bf16 values count as zero
+    got = v2.lmhead_fwd(a, b)
+    assert got[1, 0].view(np.uint32) == 0 and got[3, 2].view(np.uint32) == 0        # +0
+    assert np.isnan(got[2]).all() and np.isnan(got[:, 1]).all()
+    assert np.isfinite(got[0, 0]) and np.isfinite(got[0, 2])
+    _, _, E = v2.slice_rows(a)
+    assert E[1] == 0 and E[3] == 0 and (E[2] >> 30) == 1
