@@ -244,6 +244,20 @@ int det_lmhead_fwd(const det_bf16* H, const det_bf16* W, int M, int V, int K, fl
 int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH,
                    float* dW, int first_chunk, void* stream);
 
+/* Arithmetic version 2 of the forward contraction (optional mode; version 1 above stays the default and the benchmark's
+ * arithmetic).  Built from the paper's two integer devices (Sec. 3.2: int8 products accumulated exactly in int32; a wide
+ * exact integer total "for bitwise reproducibility"): the result does not depend on the order of the terms at all.
+ *   per row x of H and of W:  E = largest biased bf16 exponent of the row (0 for an all-zero row; subnormals count as 0);
+ *     T_k = ((128 + fraction_k) << 6) >> (E - E_k) with the sign of x_k: x_k is replaced by T_k 2^(E - 140) (values within
+ *     2^-6 of the row's largest are exact, smaller ones truncated toward zero); T_k = 128 hi_k + lo_k, two signed int8 slices
+ *   logits[m,n] = binary32 nearest-even rounding of I 2^(E(H_m) + E(W_n) - 280),  I = sum_k Ta_k Tb_k
+ *     = 2^14 sum(ha hb) + 2^7 (sum(ha lb) + sum(la hb)) + sum(la lb), the four sums exact in int32 on the tensor cores;
+ *     ONE rounding; a result below 2^-126 after it is a signed zero; a row with an infinity or a NaN gives NaN.
+ * M % 128 == 0, V % 128 == 0, K % 128 == 0, K < 2^17.  ws: det_lmhead_fwd_v2_ws_bytes (the int8 slices and row exponents). */
+size_t det_lmhead_fwd_v2_ws_bytes(int M, int V, int K);
+int det_lmhead_fwd_v2(const det_bf16* H, const det_bf16* W, int M, int V, int K, float* logits, void* ws, size_t ws_bytes,
+                      void* stream, int* status_dev);
+
 /* ---- gradient accumulation = single-device replay of the data-parallel reduction
  *      (Sec. 6, Algorithm 1; Appendix A, Algorithm 2 "TreeFold"; A.3 reciprocal-multiply averages) -------
  * The state is a caller-owned POD; bufs holds det_grad_accum_nbufs(dp_replicate) * n floats on the device. */

@@ -536,7 +536,7 @@ static EncodeTiledFn get_encode() {
   }
   return fn;
 }
-static bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows) {
+bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return false;
   cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};

@@ -1,0 +1,253 @@
+// LM head, arithmetic version 2 (optional mode): an order-free, exactly defined contraction on the int8 tensor cores.
+//
+// Version 1 defines every logit as an ordered chain of binary32 roundings, which only the FP32 ALUs can replay.  Version 2
+// uses the paper's own two devices instead (Sec. 3.2: int8 products accumulated exactly in int32; a wide exact integer
+// total "for bitwise reproducibility"): every row of H and of W is aligned to its largest exponent and cut into two signed
+// 7-bit slices (T = 128 hi + lo, a 14-bit magnitude: values within 2^-6 of the row's largest are kept exactly, smaller
+// ones truncated toward zero), the four slice products are exact int32 sums on tcgen05.mma.kind::i8 in whatever order the
+// hardware takes them, and the epilogue forms I = 2^14 hh + 2^7 (hl + lh) + ll in 64 bits and rounds I 2^(Ea + Eb - 280)
+// to binary32 ONCE.  Nothing about the result depends on tiling, order or hardware.
+//
+//   k_slice_rows   one warp per row: row exponent (integer maximum), then the two int8 slices
+//   k_igemm_sl     persistent, one CTA per SM, 128 x 128 output tile; warp 0 streams the FOUR operand tiles of a 128-deep
+//                  step (H hi, H lo, W hi, W lo: 64 KiB) through a three-stage TMA ring, warp 1 issues the sixteen MMAs of
+//                  the step into three TMEM accumulators (hh | hl + lh | ll, 128 columns each), warps 2-5 combine and round.
+// Every mbarrier wait is bounded (DET_DEV_TIMEOUT), as in igemm.cu.
+#include "tc05.cuh"
+#include "internal.h"
+
+namespace det {
+
+// ---- slicing ----------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_slice_rows(const uint16_t* __restrict__ X, int R, int K, int8_t* __restrict__ hi,
+                                                    int8_t* __restrict__ lo, int32_t* __restrict__ E) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  const uint4* x = reinterpret_cast<const uint4*>(X + (size_t)row * K);
+  int e = 0, bad = 0;
+  for (int i = lane; i < K / 8; i += 32) {
+    const uint4 u = __ldg(x + i);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int e0 = (w[j] >> 7) & 0xFF, e1 = (w[j] >> 23) & 0xFF;
+      bad |= (e0 == 255) | (e1 == 255);
+      e = max(e, max(e0, e1));
+    }
+  }
+#pragma unroll
+  for (int s = 16; s; s >>= 1) {
+    e = max(e, __shfl_xor_sync(0xffffffffu, e, s));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, s);
+  }
+  if (lane == 0) E[row] = e | (bad ? (1 << 30) : 0);
+  for (int i = lane; i < K / 8; i += 32) {
+    const uint4 u = __ldg(x + i);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    uint32_t h8[2] = {0u, 0u}, l8[2] = {0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t b = (j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu);
+      const int ek = (b >> 7) & 0xFF, d = e - ek;
+      int t = (ek == 0 || d >= 14) ? 0 : (int)(((128u + (b & 0x7Fu)) << 6) >> d);
+      int h = t >> 7, l = t & 127;
+      if (b & 0x8000u) { h = -h; l = -l; }
+      h8[j >> 2] |= (uint32_t)(uint8_t)(int8_t)h << (8 * (j & 3));
+      l8[j >> 2] |= (uint32_t)(uint8_t)(int8_t)l << (8 * (j & 3));
+    }
+    *reinterpret_cast<uint2*>(hi + (size_t)row * K + 8 * i) = make_uint2(h8[0], h8[1]);
+    *reinterpret_cast<uint2*>(lo + (size_t)row * K + 8 * i) = make_uint2(l8[0], l8[1]);
+  }
+}
+
+// ---- sliced contraction -------------------------------------------------------------------------------------------------
+constexpr int SL_T = 128;                     // tile edge (rows of H x rows of W)
+constexpr int SL_BK = 128;                    // bytes (= int8 elements) per step along K
+constexpr int SL_STAGES = 3;
+constexpr int SL_TILE = SL_T * SL_BK;         // one operand tile: 16 KiB
+constexpr int SL_STAGE_BYTES = 4 * SL_TILE;   // H hi | H lo | W hi | W lo
+constexpr int SL_THREADS = 192;
+constexpr size_t SL_SMEM = (size_t)SL_STAGES * SL_STAGE_BYTES + 1024;
+
+// the one rounding of the definition: I 2^e as binary32, nearest even; results below 2^-126 after the rounding are zeros
+__device__ __forceinline__ float round_scaled(long long I, int e) {
+  const double v = (double)I * __longlong_as_double((long long)(e + 1023) << 52);   // exact: |I| < 2^53, e + 1023 in [745, 1253]
+  float r = __double2float_rn(v);
+  if (fabsf(r) < 0x1p-126f) r = copysignf(0.0f, r);
+  return r;
+}
+
+__global__ void __launch_bounds__(SL_THREADS, 1)
+    k_igemm_sl(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
+               const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const int32_t* __restrict__ Ea,
+               const int32_t* __restrict__ Eb, float* __restrict__ out, int I, int J, int K, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bar_full[SL_STAGES], bar_empty[SL_STAGES], bar_tfull, bar_tempty;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SL_STAGES; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+    mbar_init(&bar_tfull, 1);
+    mbar_init(&bar_tempty, 4);
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  const int tiles_i = I / SL_T, tiles_j = J / SL_T, num_tiles = tiles_i * tiles_j, kblocks = K / SL_BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        // the rows of H run fastest: the CTAs resident at one time share a tile of W and stream H through L2
+        const int i0 = (tile % tiles_i) * SL_T, j0 = (tile / tiles_i) * SL_T;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          mbar_expect_tx(&bar_full[stage], SL_STAGE_BYTES);
+          uint8_t* sa = smem + stage * SL_STAGE_BYTES;
+          tma_load_2d(sa, &tmAh, kb * SL_BK, i0, &bar_full[stage]);
+          tma_load_2d(sa + SL_TILE, &tmAl, kb * SL_BK, i0, &bar_full[stage]);
+          tma_load_2d(sa + 2 * SL_TILE, &tmBh, kb * SL_BK, j0, &bar_full[stage]);
+          tma_load_2d(sa + 3 * SL_TILE, &tmBl, kb * SL_BK, j0, &bar_full[stage]);
+          if (++stage == SL_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: D = S32, A = B = signed 8-bit, both K-major, N = 128, M = 128
+      constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(SL_T >> 3) << 17) | ((uint32_t)(SL_T >> 4) << 24);
+      int stage = 0, it = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        if (!mbar_wait(&bar_tempty, ((uint32_t)it & 1u) ^ 1u, abort_flag, status)) { ok = false; break; }   // accumulators drained
+        tc_fence_after();
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&bar_full[stage], phase, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * SL_STAGE_BYTES);
+          const uint64_t ah = make_smem_desc(sa), al = make_smem_desc(sa + SL_TILE);
+          const uint64_t bh = make_smem_desc(sa + 2 * SL_TILE), bl = make_smem_desc(sa + 3 * SL_TILE);
+#pragma unroll
+          for (int k4 = 0; k4 < SL_BK / 32; ++k4) {
+            const uint64_t o = (uint64_t)(k4 * 2);
+            const uint32_t first = (kb | k4) ? 1u : 0u;
+            umma_i8(tmem_base, ah + o, bh + o, idesc, first);              // hh
+            umma_i8(tmem_base + 128u, ah + o, bl + o, idesc, first);       // hl starts the cross accumulator ...
+            umma_i8(tmem_base + 128u, al + o, bh + o, idesc, 1u);          // ... lh adds to it
+            umma_i8(tmem_base + 256u, al + o, bl + o, idesc, first);       // ll
+          }
+          umma_commit(&bar_empty[stage]);
+          if (++stage == SL_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(&bar_tfull);
+      }
+    }
+  } else {
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int i0 = (tile % tiles_i) * SL_T, j0 = (tile / tiles_i) * SL_T;
+      if (!mbar_wait(&bar_tfull, (uint32_t)it & 1u, abort_flag, status)) { ok = false; break; }
+      tc_fence_after();
+      const int row = i0 + q * 32 + lane;
+      const int ea = Ea[row];
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      float* orow = out + (size_t)row * J + j0;
+#pragma unroll 1
+      for (int c0 = 0; c0 < SL_T; c0 += 32) {
+        uint32_t hh[32], cr[32], ll[32];
+        tmem_ld32(taddr + (uint32_t)c0, hh);
+        tmem_ld32(taddr + 128u + (uint32_t)c0, cr);
+        tmem_ld32(taddr + 256u + (uint32_t)c0, ll);
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          float f[4];
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            const int c = 4 * v + x;
+            const int eb = __ldg(Eb + j0 + c0 + c);
+            const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
+            f[x] = ((ea | eb) >> 30) ? __int_as_float(0x7FC00000) : round_scaled(Iv, (ea & 0xFF) + (eb & 0xFF) - 280);
+          }
+          *reinterpret_cast<float4*>(orow + c0 + 4 * v) = make_float4(f[0], f[1], f[2], f[3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_tempty);
+    }
+  }
+  __syncthreads();
+  if (abort_s) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace det
+
+using namespace det;
+
+static size_t v2_layout(int M, int V, int K, size_t* oAh, size_t* oAl, size_t* oBh, size_t* oBl, size_t* oEa, size_t* oEb) {
+  size_t off = 0;
+  *oAh = off; off += align_up((size_t)M * K, 256);
+  *oAl = off; off += align_up((size_t)M * K, 256);
+  *oBh = off; off += align_up((size_t)V * K, 256);
+  *oBl = off; off += align_up((size_t)V * K, 256);
+  *oEa = off; off += align_up((size_t)M * 4, 256);
+  *oEb = off; off += align_up((size_t)V * 4, 256);
+  return off;
+}
+extern "C" size_t det_lmhead_fwd_v2_ws_bytes(int M, int V, int K) {
+  size_t a, b, c, d, e, f;
+  return v2_layout(M, V, K, &a, &b, &c, &d, &e, &f);
+}
+extern "C" int det_lmhead_fwd_v2(const det_bf16* H, const det_bf16* W, int M, int V, int K, float* logits, void* ws,
+                                 size_t ws_bytes, void* stream, int* status_dev) {
+  if (!H || !W || !logits || M <= 0 || V <= 0 || K <= 0) return DET_ERR_ARG;
+  if (M % SL_T || V % SL_T || K % SL_BK) return DET_ERR_SHAPE;
+  if (K >= (1 << 17)) return DET_ERR_RANGE;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(logits) || !aligned16(ws)) return DET_ERR_ALIGN;
+  size_t oAh, oAl, oBh, oBl, oEa, oEb;
+  if (!ws || ws_bytes < v2_layout(M, V, K, &oAh, &oAl, &oBh, &oBl, &oEa, &oEb)) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* base = (uint8_t*)ws;
+  int8_t *Ah = (int8_t*)(base + oAh), *Al = (int8_t*)(base + oAl), *Bh = (int8_t*)(base + oBh), *Bl = (int8_t*)(base + oBl);
+  int32_t *Ea = (int32_t*)(base + oEa), *Eb = (int32_t*)(base + oEb);
+  k_slice_rows<<<DET_L((M + 7) / 8), 256, 0, st>>>(H, M, K, Ah, Al, Ea);
+  k_slice_rows<<<DET_L((V + 7) / 8), 256, 0, st>>>(W, V, K, Bh, Bl, Eb);
+  DET_CHECK_LAUNCH();
+  CUtensorMap tAh, tAl, tBh, tBl;
+  if (!make_map(&tAh, Ah, M, K, SL_T) || !make_map(&tAl, Al, M, K, SL_T) || !make_map(&tBh, Bh, V, K, SL_T) ||
+      !make_map(&tBl, Bl, V, K, SL_T))
+    return DET_ERR_CUDA;
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_igemm_sl, SL_SMEM) != DET_OK) return DET_ERR_CUDA;
+  const int sms = dev_sm_count();
+  if (sms <= 0) return DET_ERR_CUDA;
+  const int tiles = (M / SL_T) * (V / SL_T);
+  k_igemm_sl<<<DET_L(tiles < sms ? tiles : sms), SL_THREADS, SL_SMEM, st>>>(tAh, tAl, tBh, tBl, Ea, Eb, logits, M, V, K, status_dev);
+  DET_CHECK_LAUNCH();
+  return DET_OK;
+}

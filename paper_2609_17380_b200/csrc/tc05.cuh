@@ -93,6 +93,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// host: tensor map of a row-major int8 matrix [rows, K] with boxes of box_rows x 128 bytes, 128-byte swizzle (igemm.cu)
+bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows);
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 

@@ -167,6 +167,16 @@ def case_lmhead(small, bwd):
     return (lambda: det.det_lmhead_bwd(lg, Hh, W, M, V, K, dH, dW, 1)), 4.0 * M * V * K, "flop"
 
 
+def case_lmhead_v2(small):
+    """The order-free LM-head forward (arithmetic version 2) on the int8 tensor cores; same nominal work as lmhead_fwd."""
+    M, V, K = (1024 if small else 8192), 50304, 2048
+    Hh, W = randn_bf16(M * K), randn_bf16(V * K, 0.02)
+    lg = torch.empty(M * V, device="cuda")
+    w = ws(det.det_lmhead_fwd_v2_ws_bytes(M, V, K))
+    st = torch.zeros(1, dtype=I32, device="cuda")
+    return (lambda: det.det_lmhead_fwd_v2(Hh, W, M, V, K, lg, w, st)), 2.0 * M * V * K, "flop"
+
+
 def case_accum(small):
     n = (1 << 26) if small else (1 << 28)
     g = torch.randn(n, device="cuda")
@@ -200,7 +210,7 @@ def build_cases():
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
          "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
          "attn_bwd_fixq": lambda s: case_attn(s, True, False, True),
-         "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_bwd": lambda s: case_lmhead(s, True),
+         "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_fwd_v2": case_lmhead_v2, "lmhead_bwd": lambda s: case_lmhead(s, True),
          "accum": case_accum, "adamw": case_adamw, "hash": case_hash}
     for k in LINEAR_SHAPES:
         c["igemm_" + k] = (lambda s, k=k: case_igemm(s, k))

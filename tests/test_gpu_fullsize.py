@@ -120,6 +120,21 @@ def test_lmhead_full_shape_sampled(det):
     assert_same_bits(dW[vs.tolist()].cpu().numpy(), odW, "dW rows")
 
 
+def test_lmhead_version_2_full_shape_sampled(det):
+    """The order-free forward contraction (arithmetic version 2) at 8192 x 50304 x 2048: sampled rows against its oracle."""
+    import torch
+    from oracle import v2
+    Hh, W = _bf16_normal((T, D), 1.0, 41), _bf16_normal((V, D), 0.02, 42)
+    logits = empty((T, V), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_lmhead_fwd_v2(dev(Hh), dev(W), T, V, D, logits, ws(det.det_lmhead_fwd_v2_ws_bytes(T, V, D)), status)
+    _sync()
+    assert int(status.item()) == 0
+    rows = np.sort(np.random.default_rng(43).choice(T, 6, replace=False))
+    rows[0], rows[-1] = 0, T - 1
+    assert_same_bits(logits[rows.tolist()].cpu().numpy(), v2.lmhead_fwd(Hh[rows], W), "version-2 logit rows")
+
+
 def test_attention_full_shape_one_head(det):
     HD = H * 128
     qkv = _bf16_normal((B * S, 3 * HD), 1.0, 8)

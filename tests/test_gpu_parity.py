@@ -365,6 +365,33 @@ def test_producers_write_the_next_linears_int8_input(det):
     assert_same_bits(host(Y, np.uint16), oY, "linear on ready-made codes")
 
 
+@pytest.mark.parametrize("M,V,K", [(128, 128, 128), (256, 384, 1024), (384, 256, 2048)])
+def test_lmhead_forward_version_2(det, M, V, K):
+    """The order-free contraction of arithmetic version 2 on the int8 tensor cores against its oracle, bit for bit: values
+    over a wide range of exponents (so that slices are truncated), an all-zero row, subnormal inputs, a row with an
+    infinity and one with a NaN."""
+    import torch
+    from oracle import v2
+    rng = np.random.default_rng(M + V + K)
+    Hh = synth.to_bf16((rng.standard_normal((M, K)) * np.exp2(rng.integers(-10, 4, (M, K)))).astype(F))
+    W = synth.to_bf16((rng.standard_normal((V, K)) * 0.02 * np.exp2(rng.integers(-8, 3, (V, K)))).astype(F))
+    Hh[3] = 0
+    Hh[5, ::3] = 0x0001
+    W[7, 11] = 0x7F80
+    Hh[9, 0] = 0x7FC0
+    lg = empty((M, V), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_lmhead_fwd_v2(dev(Hh), dev(W), M, V, K, lg, ws(det.det_lmhead_fwd_v2_ws_bytes(M, V, K)), status)
+    _sync()
+    assert int(status.item()) == 0
+    got, want = host(lg), v2.lmhead_fwd(Hh, W)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.isnan(want[9]).all() and np.isnan(want[:, 7]).all()
+    ok = ~np.isnan(want)
+    assert_same_bits(got[ok], want[ok], "version-2 logits")
+    assert np.all(np.delete(got[3], 7).view(np.uint32) == 0)          # the all-zero row: +0 against every finite row of W
+
+
 def test_embedding(det):
     V, D, T = 1000, 512, 700
     E = synth.normal_bf16((V, D), 0.02, seed=7, tid=1)
