@@ -448,7 +448,7 @@ def run_ours(args):
         ach = alg[dom][1] / (tot_ms / n / 1e3) / 1e12
         # DRAM traffic per launch group from the committed ncu capture of the same kernels at B = 1 (read + write, summed
         # over the launches of the summary; it grows in proportion to the batch)
-        prof_file = {"attn_bwd": "k_attn_sdp_ws_k_ogemm_wb_attn_bwd_small.md", "attn_fwd": "k_attn_fwd_attn_fwd_small.md"}.get(dom)
+        prof_file = {"attn_bwd": "k_attn_sdp_ws_k_ogemm_wb_attn_bwd_small.md", "attn_fwd": "k_attn_fwd_ws_attn_fwd_small.md"}.get(dom)
         t1 = profile_traffic(prof_file) if (prof_file and args.workload == "config5") else None
         traffic = t1 * B if t1 is not None else None
         roof["traffic_source"] = ("profiles/%s x batch %d" % (prof_file, B)) if t1 is not None else None
