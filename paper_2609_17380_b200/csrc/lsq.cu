@@ -246,6 +246,76 @@ __global__ void __launch_bounds__(128) k_rotc(const void* __restrict__ in, int R
   }
 }
 
+// (2b) the int8 operands (Z = qX, U = qW) through shared memory: the CTA loads its 128 x 128 tile with whole 128-byte row
+//      segments (eight lanes per row), every thread takes one column from the tile (a warp reads 32 adjacent bytes of a
+//      row: one wavefront), rotates it in registers (exact integers, |value| <= 2^14), and in PASS 1 the quantised columns
+//      go back through the tile so that the transposed output is written as whole 128-byte lines as well (the version this
+//      replaced read one byte and wrote sixteen per lane in 32 different lines per instruction; the values are the same).
+template <int PASS, bool ROT>
+__global__ void __launch_bounds__(128) k_rotc8(const int8_t* __restrict__ in, int R, int C, uint32_t* __restrict__ amax,
+                                               int8_t* __restrict__ outT) {
+  __shared__ __align__(16) uint8_t tile[128 * 128];
+  const int t = threadIdx.x, c0 = blockIdx.x * 128, r0 = blockIdx.y * 128;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = i * 16 + (t >> 3), ch = t & 7;
+    *reinterpret_cast<uint4*>(tile + r * 128 + ch * 16) =
+        __ldg(reinterpret_cast<const uint4*>(in + (size_t)(r0 + r) * C + c0 + ch * 16));
+  }
+  __syncthreads();
+  int vi[128];
+#pragma unroll
+  for (int i = 0; i < 128; ++i) vi[i] = (int)(int8_t)tile[i * 128 + t];
+  if (ROT) {
+#pragma unroll
+    for (int h = 1; h < 128; h <<= 1) {
+#pragma unroll
+      for (int i = 0; i < 128; ++i) {
+        if (!(i & h)) { const int a = vi[i], b = vi[i + h]; vi[i] = a + b; vi[i + h] = a - b; }
+      }
+    }
+  }
+  if (PASS == 0) {
+    uint32_t local = 0;
+#pragma unroll
+    for (int i = 0; i < 128; ++i) local = max(local, (uint32_t)abs(vi[i]));
+#pragma unroll
+    for (int w = 16; w; w >>= 1) local = max(local, __shfl_xor_sync(0xffffffffu, local, w));
+    if ((t & 31) == 0 && local > *reinterpret_cast<volatile uint32_t*>(amax)) atomicMax(amax, local);
+    return;
+  }
+  float inv = 0.0f;
+  if (ROT) {
+    const int am = (int)amax[0];
+    inv = (am > 0) ? fdiv(127.0f, __int2float_rn(am)) : 0.0f;
+  }
+  __syncthreads();                       // everybody has read its column: the tile becomes the transposed output tile
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint32_t o = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int i = g * 16 + k * 4 + e;
+        const int8_t qv = ROT ? quant1(__int2float_rn(vi[i]), inv) : (int8_t)vi[i];
+        o |= ((uint32_t)(uint8_t)qv) << (8 * e);
+      }
+      w[k] = o;
+    }
+    // row t of the transposed tile (column c0 + t of the input), sixteen-byte pieces XOR-swizzled by row
+    *reinterpret_cast<uint4*>(tile + t * 128 + ((g ^ (t & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = i * 16 + (t >> 3), ch = t & 7;
+    *reinterpret_cast<uint4*>(outT + (size_t)(c0 + r) * R + r0 + ch * 16) =
+        *reinterpret_cast<const uint4*>(tile + r * 128 + ((ch ^ (r & 7)) << 4));
+  }
+}
+
 // (3) both rotations of dY from one read: a CTA stages a 128 x 128 tile of dY in shared memory (f32), then every thread
 //     rotates one row of dY * s_w along n (the A operand of the input-gradient GEMM) and one column of dY along the
 //     token index (the G operand of the weight-gradient GEMM, written transposed).  128 values per thread in registers,
@@ -453,10 +523,10 @@ extern "C" int det_lsq_quantize_weight(const det_bf16* W, const float* s_w, int 
     cudaMemsetAsync(amax, 0, 256, st);
     dim3 grid(K / 128, N / 128);
     if (hadamard_block) {
-      k_rotc<false, 0, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, nullptr);
-      k_rotc<false, 1, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rotc8<0, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, nullptr);
+      k_rotc8<1, true><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
     } else {
-      k_rotc<false, 1, false><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
+      k_rotc8<1, false><<<DET_L(grid), 128, 0, st>>>(qW, N, K, amax, qWt_bwd);
     }
     k_su_finish<<<DET_L(1), 1, 0, st>>>(amax, hadamard_block != 0, s_u);
   }
@@ -539,16 +609,16 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
     AuxScope az(st);
     cudaStream_t sz = az.aux(1);
     k_prep_dy<0><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, nullptr, nullptr);
-    k_rotc<false, 0, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, nullptr);
+    k_rotc8<0, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, nullptr);
     k_prep_dy<1><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, Aq, GqT);
-    k_rotc<false, 1, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, ZqT);
+    k_rotc8<1, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, ZqT);
     if (!az.join()) return DET_ERR_CUDA;
   } else {
     k_rot_rows<0, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, nullptr);
     k_rotc<true, 0, false><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, nullptr);
     k_rot_rows<1, false><<<DET_L(g1), 256, 0, st>>>(dY, s_w, M, N, amax + 0, Aq);
     k_rotc<true, 1, false><<<DET_L(gG), 128, 0, st>>>(dY, M, N, amax + 1, GqT);
-    k_rotc<false, 1, false><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, ZqT);
+    k_rotc8<1, false><<<DET_L(gZ), 128, 0, st>>>(qX, M, K, amax + 2, ZqT);
   }
   DET_CHECK_LAUNCH();
   const float rotf = rot ? 0x1p-7f : 1.0f;
