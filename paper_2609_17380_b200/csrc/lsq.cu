@@ -316,17 +316,13 @@ __global__ void __launch_bounds__(128) k_rotc8(const int8_t* __restrict__ in, in
   }
 }
 
-// (3) both rotations of dY from one read: a CTA stages a 128 x 128 tile of dY in shared memory (f32), then every thread
+// (3) both rotations of dY from one read: a CTA stages a 128 x 128 tile of dY in shared memory (raw bf16), then every thread
 //     rotates one row of dY * s_w along n (the A operand of the input-gradient GEMM) and one column of dY along the
 //     token index (the G operand of the weight-gradient GEMM, written transposed).  128 values per thread in registers,
 //     butterflies on register pairs with packed arithmetic: a + b is one packed add, a - b one packed fused
 //     multiply-add b * (-1) + a, which rounds exactly like the subtraction.  PASS 0 records both absmax values,
 //     PASS 1 quantises with them.  dY is read twice per backward pass instead of four times.
-//     The kernel is bound by the shared-memory / L1 pipeline, so every shared-memory access is a conflict-free
-//     sixteen-byte one where the layout allows (rows padded to 132 floats), and PASS 1 hands its int8 rows over through
-//     the (then dead) tile so that every global store instruction writes four whole 128-byte rows.
-constexpr int PT = 128, PLD = 132;
-constexpr size_t PREP_SMEM = (size_t)(PT * PLD + PT) * sizeof(float);
+constexpr int PT = 128;
 
 __device__ __forceinline__ void wht128_pairs(float2 (&v)[64]) {
 #pragma unroll
@@ -382,32 +378,39 @@ __device__ __forceinline__ void amax_publish(float local, uint32_t* amax) {
     atomicMax(amax, __float_as_uint(local));
 }
 
+//     The kernel is persistent and software-pipelined: a CTA walks over tiles, the raw bf16 tile of the NEXT step travels
+//     into the other half of a double buffer (16-byte asynchronous copies, chunks XOR-swizzled by row so that a thread reads
+//     its row with conflict-free 16-byte loads and its column with 2-byte loads) while the current one is rotated, so no
+//     global-load latency and no convert-and-store pass sits between the butterflies; the finished int8 rows leave through
+//     the buffer that has just been consumed, as whole 128-byte lines.
+constexpr size_t PREP2_SMEM = (size_t)2 * PT * 256 + 2 * PT * sizeof(float);
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+
 template <int PASS>
-__global__ void __launch_bounds__(PT, 3) k_prep_dy(const uint16_t* __restrict__ dY, const float* __restrict__ s_w, int M, int N,
-                                                   uint32_t* __restrict__ amax, int8_t* __restrict__ Aq,
-                                                   int8_t* __restrict__ GqT) {
-  extern __shared__ __align__(16) float psm[];
-  float(*tile)[PLD] = reinterpret_cast<float(*)[PLD]>(psm);
-  float* sw = psm + PT * PLD;
-  const int t = threadIdx.x, n0 = blockIdx.x * PT, m0 = blockIdx.y * PT;
-  uint4 raw[16];
+__global__ void __launch_bounds__(PT, 3) k_prep_dy2(const uint16_t* __restrict__ dY, const float* __restrict__ s_w, int M, int N,
+                                                    uint32_t* __restrict__ amax, int8_t* __restrict__ Aq,
+                                                    int8_t* __restrict__ GqT) {
+  extern __shared__ __align__(16) uint8_t pbuf[];
+  float* swb = reinterpret_cast<float*>(pbuf + 2 * PT * 256);      // [2][128]
+  const int t = threadIdx.x;
+  const int ntn = N / PT, ntiles = ntn * (M / PT);
+  auto issue = [&](int tile, int b) {
+    const int n0 = (tile % ntn) * PT, m0 = (tile / ntn) * PT;
+    uint8_t* dst = pbuf + b * (PT * 256);
 #pragma unroll
-  for (int it = 0; it < 16; ++it)
-    raw[it] = __ldg(reinterpret_cast<const uint4*>(dY + (size_t)(m0 + it * 8 + (t >> 4)) * N + n0 + (t & 15) * 8));
-  sw[t] = __ldg(s_w + n0 + t);
-  // eight values per thread and row as two sixteen-byte stores; lanes 0-3 of every eight store their first half while
-  // lanes 4-7 store their second, then the other way round: each store instruction covers all banks once
-  const int sel = (t >> 2) & 1;
-#pragma unroll
-  for (int it = 0; it < 16; ++it) {
-    float* d = &tile[it * 8 + (t >> 4)][(t & 15) * 8];
-    const uint4 u = raw[it];
-    const float4 f0 = make_float4(bflo(u.x), bfhi(u.x), bflo(u.y), bfhi(u.y));
-    const float4 f1 = make_float4(bflo(u.z), bfhi(u.z), bflo(u.w), bfhi(u.w));
-    *reinterpret_cast<float4*>(d + 4 * sel) = sel ? f1 : f0;
-    *reinterpret_cast<float4*>(d + 4 * (sel ^ 1)) = sel ? f0 : f1;
-  }
-  __syncthreads();
+    for (int it = 0; it < 16; ++it) {
+      const int r = it * 8 + (t >> 4), c = t & 15;
+      cp_async16(dst + r * 256 + ((c ^ (r & 7)) << 4), dY + (size_t)(m0 + r) * N + n0 + c * 8);
+    }
+    cp_async4(swb + b * PT + t, s_w + n0 + t);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
   float invA = 0.0f, invG = 0.0f;
   bool fastA = false, fastG = false;
   if (PASS == 1) {
@@ -417,43 +420,71 @@ __global__ void __launch_bounds__(PT, 3) k_prep_dy(const uint16_t* __restrict__ 
     fastA = finite1(a) && finite1(invA);
     fastG = finite1(g) && finite1(invG);
   }
-  float2 v[64];
-  uint32_t qa[32], qg[32];
-  // row t of the tile, scaled by the weight steps (scalar multiplies: the products are rounded before any add)
+  float maxA = 0.0f, maxG = 0.0f;
+  if ((int)blockIdx.x < ntiles) issue(blockIdx.x, 0);
+  int i = 0;
+  for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
+    const int b = i & 1, next = tile + gridDim.x;
+    __syncthreads();                                   // the other buffer (tile i - 1: operands and staging) is free
+    if (next < ntiles) {
+      issue(next, b ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();                                   // tile i has landed for every thread
+    const uint8_t* buf = pbuf + b * (PT * 256);
+    const float* sw = swb + b * PT;
+    const int n0 = (tile % ntn) * PT, m0 = (tile / ntn) * PT;
+    float2 v[64];
+    uint32_t qa[32], qg[32];
+    // row t of the tile, scaled by the weight steps (scalar multiplies: the products are rounded before any add)
 #pragma unroll
-  for (int q = 0; q < 32; ++q) {
-    const float4 x = *reinterpret_cast<const float4*>(&tile[t][4 * q]);
-    const float4 c = *reinterpret_cast<const float4*>(&sw[4 * q]);
-    v[2 * q] = make_float2(fmul(x.x, c.x), fmul(x.y, c.y));
-    v[2 * q + 1] = make_float2(fmul(x.z, c.z), fmul(x.w, c.w));
+    for (int c = 0; c < 16; ++c) {
+      const uint4 u = *reinterpret_cast<const uint4*>(buf + t * 256 + ((c ^ (t & 7)) << 4));
+      const float4 w0 = *reinterpret_cast<const float4*>(&sw[8 * c]), w1 = *reinterpret_cast<const float4*>(&sw[8 * c + 4]);
+      v[4 * c] = make_float2(fmul(bflo(u.x), w0.x), fmul(bfhi(u.x), w0.y));
+      v[4 * c + 1] = make_float2(fmul(bflo(u.y), w0.z), fmul(bfhi(u.y), w0.w));
+      v[4 * c + 2] = make_float2(fmul(bflo(u.z), w1.x), fmul(bfhi(u.z), w1.y));
+      v[4 * c + 3] = make_float2(fmul(bflo(u.w), w1.z), fmul(bfhi(u.w), w1.w));
+    }
+    wht128_pairs(v);
+    if (PASS == 0) maxA = fmaxf(maxA, absmax128(v));
+    else if (fastA && finite1(v[0].x)) quant_pack128<true>(v, invA, qa);
+    else quant_pack128<false>(v, invA, qa);
+    // column t of the tile, transposed output
+    const int cc = t >> 3, cw = (t & 7) * 2;
+#pragma unroll
+    for (int p = 0; p < 64; ++p) {
+      const uint16_t lo = *reinterpret_cast<const uint16_t*>(buf + (2 * p) * 256 + ((cc ^ ((2 * p) & 7)) << 4) + cw);
+      const uint16_t hi = *reinterpret_cast<const uint16_t*>(buf + (2 * p + 1) * 256 + ((cc ^ ((2 * p + 1) & 7)) << 4) + cw);
+      v[p] = make_float2(bf2f(lo), bf2f(hi));
+    }
+    wht128_pairs(v);
+    if (PASS == 0) { maxG = fmaxf(maxG, absmax128(v)); continue; }
+    if (fastG && finite1(v[0].x)) quant_pack128<true>(v, invG, qg);
+    else quant_pack128<false>(v, invG, qg);
+    // hand-over through the consumed buffer: two tiles of 128 rows x 128 bytes, sixteen-byte pieces XOR-swizzled by row
+    __syncthreads();
+    uint8_t* stg = pbuf + b * (PT * 256);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const int off = t * 128 + ((g ^ (t & 7)) << 4);
+      *reinterpret_cast<uint4*>(stg + off) = make_uint4(qa[4 * g], qa[4 * g + 1], qa[4 * g + 2], qa[4 * g + 3]);
+      *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(qg[4 * g], qg[4 * g + 1], qg[4 * g + 2], qg[4 * g + 3]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int idx = k * PT + t, r = idx >> 3, piece = idx & 7;
+      const int off = r * 128 + ((piece ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(Aq + (size_t)(m0 + r) * N + n0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + off);
+      *reinterpret_cast<uint4*>(GqT + (size_t)(n0 + r) * M + m0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + 16384 + off);
+    }
   }
-  wht128_pairs(v);
-  if (PASS == 0) amax_publish(absmax128(v), amax + 0);
-  else if (fastA && finite1(v[0].x)) quant_pack128<true>(v, invA, qa);
-  else quant_pack128<false>(v, invA, qa);
-  // column t of the tile, transposed output
-#pragma unroll
-  for (int p = 0; p < 64; ++p) v[p] = make_float2(tile[2 * p][t], tile[2 * p + 1][t]);
-  wht128_pairs(v);
-  if (PASS == 0) { amax_publish(absmax128(v), amax + 1); return; }
-  if (fastG && finite1(v[0].x)) quant_pack128<true>(v, invG, qg);
-  else quant_pack128<false>(v, invG, qg);
-  // hand-over through the tile's memory: two tiles of 128 rows x 128 bytes, sixteen-byte pieces XOR-swizzled by row
-  __syncthreads();
-  uint8_t* stg = reinterpret_cast<uint8_t*>(psm);
-#pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    const int off = t * 128 + ((g ^ (t & 7)) << 4);
-    *reinterpret_cast<uint4*>(stg + off) = make_uint4(qa[4 * g], qa[4 * g + 1], qa[4 * g + 2], qa[4 * g + 3]);
-    *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(qg[4 * g], qg[4 * g + 1], qg[4 * g + 2], qg[4 * g + 3]);
-  }
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int idx = i * PT + t, r = idx >> 3, piece = idx & 7;
-    const int off = r * 128 + ((piece ^ (r & 7)) << 4);
-    *reinterpret_cast<uint4*>(Aq + (size_t)(m0 + r) * N + n0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + off);
-    *reinterpret_cast<uint4*>(GqT + (size_t)(n0 + r) * M + m0 + piece * 16) = *reinterpret_cast<const uint4*>(stg + 16384 + off);
+  if (PASS == 0) {
+    amax_publish(maxA, amax + 0);
+    amax_publish(maxG, amax + 1);
   }
 }
 
@@ -602,15 +633,19 @@ extern "C" int det_linear_bwd(const det_bf16* dY, const det_bf16* X, const int8_
   dim3 gG(N / 128, M / 128), gZ(K / 128, M / 128);
   if (rot) {
     static DevOnce once0 = {}, once1 = {};
-    if (dev_ensure_smem(once0, (const void*)k_prep_dy<0>, PREP_SMEM) != DET_OK ||
-        dev_ensure_smem(once1, (const void*)k_prep_dy<1>, PREP_SMEM) != DET_OK)
+    if (dev_ensure_smem(once0, (const void*)k_prep_dy2<0>, PREP2_SMEM) != DET_OK ||
+        dev_ensure_smem(once1, (const void*)k_prep_dy2<1>, PREP2_SMEM) != DET_OK)
       return DET_ERR_CUDA;
+    const int sms = dev_sm_count();
+    if (sms <= 0) return DET_ERR_CUDA;
+    const int ptiles = (M / PT) * (N / PT);
+    const unsigned gP = (unsigned)(ptiles < 3 * sms ? ptiles : 3 * sms);   // persistent: three CTAs per SM
     // the rotation of the saved int8 activations does not depend on dY: it runs beside the two passes over dY
     AuxScope az(st);
     cudaStream_t sz = az.aux(1);
-    k_prep_dy<0><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, nullptr, nullptr);
+    k_prep_dy2<0><<<DET_L(gP), PT, PREP2_SMEM, st>>>(dY, s_w, M, N, amax, nullptr, nullptr);
     k_rotc8<0, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, nullptr);
-    k_prep_dy<1><<<DET_L(gG), PT, PREP_SMEM, st>>>(dY, s_w, M, N, amax, Aq, GqT);
+    k_prep_dy2<1><<<DET_L(gP), PT, PREP2_SMEM, st>>>(dY, s_w, M, N, amax, Aq, GqT);
     k_rotc8<1, true><<<DET_L(gZ), 128, 0, sz>>>(qX, M, K, amax + 2, ZqT);
     if (!az.join()) return DET_ERR_CUDA;
   } else {
