@@ -96,22 +96,24 @@ __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x
 // Backward for rows of at most 2048 elements.  With DG, the CTA (8 adjacent rows) also leaves the column-wise
 // tree over its 8 rows of dy*xhat in partial8[blockIdx.x][D] (the first three levels of the row-direction tree).
 template <bool BF, bool DG>
-__global__ void __launch_bounds__(512) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
+__global__ void __launch_bounds__(1024, 1) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
                                                       const void* __restrict__ gamma, const float* __restrict__ rstd,
                                                       int rows, int D, float invD, void* __restrict__ dx,
                                                       float* __restrict__ partial8) {
-  // 16 warps = 8 rows x 2 warps; warp half hw owns leaves hw*4 .. hw*4+3 (elements hw*1024 ..) of its row
+  // 32 warps = 8 rows x 4 warps; warp quarter hw owns leaves 2 hw, 2 hw + 1 (elements hw*512 ..) of its row: 16 values of
+  // dy and of x per lane, so that a whole SM's worth of warps fits (with two warps per row the 64 live values per lane
+  // left room for one 16-warp block per SM and the kernel ran at half the copy bandwidth)
   extern __shared__ __align__(16) float srow[];  // DG: [8][D]
-  __shared__ float half_sum[8][2];
+  __shared__ float half_sum[8][4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rl = warp >> 1, hw = warp & 1;
+  const int rl = warp >> 2, hw = warp & 3;
   const int row = blockIdx.x * 8 + rl;
   const bool live = row < rows;
   const size_t rb = (size_t)row * D;
-  float w[4][8], xh[4][8];
+  float w[2][8], xh[2][8];
 #pragma unroll
-  for (int jj = 0; jj < 4; ++jj) {
-    const int e0 = (hw * 4 + jj) * 256 + lane * 8;
+  for (int jj = 0; jj < 2; ++jj) {
+    const int e0 = (hw * 2 + jj) * 256 + lane * 8;
     if (live && e0 < D) {
       load8<BF>(dy, rb + e0, w[jj]);
       load8<BF>(x, rb + e0, xh[jj]);
@@ -124,8 +126,8 @@ __global__ void __launch_bounds__(512) k_rmsnorm_bwd8(const void* __restrict__ d
   float mine = 0.0f;
   const bool full = (D & 255) == 0;
 #pragma unroll
-  for (int jj = 0; jj < 4; ++jj) {
-    const int j = hw * 4 + jj;
+  for (int jj = 0; jj < 2; ++jj) {
+    const int j = hw * 2 + jj;
     const int e0 = j * 256 + lane * 8;
     float pr[8];
 #pragma unroll
@@ -149,22 +151,23 @@ __global__ void __launch_bounds__(512) k_rmsnorm_bwd8(const void* __restrict__ d
     const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
     if (lane == jj) mine = leaf;
   }
-  // tree over this warp's four leaf sums (lanes 0..3), then over the two halves of the row
-#pragma unroll
-  for (int wd = 1; wd < 4; wd <<= 1) {
-    const float o = __shfl_xor_sync(0xffffffffu, mine, wd);
-    const int right_leaf = hw * 4 + ((lane | wd) & ~(wd - 1));
-    const bool right_valid = (long long)right_leaf * 256 < D;
-    mine = right_valid ? fadd(mine, o) : ((lane & wd) ? o : mine);
+  // tree over this warp's two leaf sums (lanes 0, 1), then over the four quarters of the row (a node whose first element
+  // lies beyond D does not exist and its left neighbour is carried up unchanged)
+  {
+    const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
+    const bool right_valid = (long long)(hw * 2 + 1) * 256 < D;
+    mine = right_valid ? fadd(mine, o) : ((lane & 1) ? o : mine);
   }
   if (lane == 0) half_sum[rl][hw] = mine;
   __syncthreads();
-  const float tot = (D > 1024) ? fadd(half_sum[rl][0], half_sum[rl][1]) : half_sum[rl][0];
+  const float h01 = (D > 512) ? fadd(half_sum[rl][0], half_sum[rl][1]) : half_sum[rl][0];
+  const float h23 = (D > 1536) ? fadd(half_sum[rl][2], half_sum[rl][3]) : half_sum[rl][2];
+  const float tot = (D > 1024) ? fadd(h01, h23) : h01;
   const float c = fmul(tot, invD);
   if (live) {
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      const int e0 = (hw * 4 + jj) * 256 + lane * 8;
+    for (int jj = 0; jj < 2; ++jj) {
+      const int e0 = (hw * 2 + jj) * 256 + lane * 8;
       if (e0 >= D) continue;
       float o[8];
 #pragma unroll
@@ -174,7 +177,7 @@ __global__ void __launch_bounds__(512) k_rmsnorm_bwd8(const void* __restrict__ d
   }
   if (DG) {
     const long long r0 = (long long)blockIdx.x * 8;
-    for (int col = threadIdx.x; col < D; col += 512) {
+    for (int col = threadIdx.x; col < D; col += 1024) {
       float v[8];
 #pragma unroll
       for (int r = 0; r < 8; ++r) v[r] = srow[r * D + col];
@@ -513,7 +516,7 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
                                float invD, void* dx, float* dgamma, float* ws, cudaStream_t st) {
   dim3 grid((rows + 7) / 8);
   if (!dgamma) {
-    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 512, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
+    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 1024, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
     return DET_OK;
   }
   static DevOnce once = {};
@@ -521,7 +524,7 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
   const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
   float* partial8 = ws;
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);
-  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 512, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
+  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 1024, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
   dim3 g2((D + 255) / 256, nb256);
   k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256);
   k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>(partial256, nb256, D, dgamma, rows);
