@@ -253,10 +253,19 @@ int det_lmhead_bwd(const float* dlogits, const det_bf16* H, const det_bf16* W, i
  *   logits[m,n] = binary32 nearest-even rounding of I 2^(E(H_m) + E(W_n) - 280),  I = sum_k Ta_k Tb_k
  *     = 2^14 sum(ha hb) + 2^7 (sum(ha lb) + sum(la hb)) + sum(la lb), the four sums exact in int32 on the tensor cores;
  *     ONE rounding; a result below 2^-126 after it is a signed zero; a row with an infinity or a NaN gives NaN.
- * M % 128 == 0, V % 128 == 0, K % 128 == 0, K < 2^17.  ws: det_lmhead_fwd_v2_ws_bytes (the int8 slices and row exponents). */
+ * M % 128 == 0, V % 128 == 0, K % 128 == 0, contraction length < 2^16 (the accumulator of the two cross products holds
+ * 2 K 127^2).  ws: det_lmhead_fwd_v2_ws_bytes (the int8 slices and row exponents). */
 size_t det_lmhead_fwd_v2_ws_bytes(int M, int V, int K);
 int det_lmhead_fwd_v2(const det_bf16* H, const det_bf16* W, int M, int V, int K, float* logits, void* ws, size_t ws_bytes,
                       void* stream, int* status_dev);
+/* The two gradient contractions in version 2: the same contraction on transposed operands, the shared exponent always taken
+ * over the contracted index.  g = bf16(dlogits) (rounded once, as in version 1);
+ *   dH[m,k] bf16 = bf16(contraction over the vocabulary of row m of g with column k of W),
+ *   dW[v,k] f32  = contraction over the tokens of column v of g with column k of H (overwritten; a micro-batch is one call).
+ * Same shape limits; M, V < 2^16.  ws: det_lmhead_bwd_v2_ws_bytes (about 4 M V + 2 K (M + V) bytes). */
+size_t det_lmhead_bwd_v2_ws_bytes(int M, int V, int K);
+int det_lmhead_bwd_v2(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH, float* dW,
+                      void* ws, size_t ws_bytes, void* stream, int* status_dev);
 
 /* ---- gradient accumulation = single-device replay of the data-parallel reduction
  *      (Sec. 6, Algorithm 1; Appendix A, Algorithm 2 "TreeFold"; A.3 reciprocal-multiply averages) -------

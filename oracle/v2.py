@@ -55,3 +55,29 @@ def lmhead_fwd(Hh, W):
     out = np.empty((M, V), np.float32)
     lib().orc2_lmhead_fwd(_p(Hh), _p(W), C.c_int(M), C.c_int(V), C.c_int(K), _p(out))
     return out
+
+
+def _f2bf(x):
+    """binary32 -> bf16 bit patterns: subnormal inputs flushed to signed zero, then round to nearest even on the upper 16 bits."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = np.where((u & 0x7F800000) == 0, u & 0x80000000, u)
+    r = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    nan = ((u & 0x7F800000) == 0x7F800000) & ((u & 0x007FFFFF) != 0)
+    r = np.where(nan, (u >> 16) | 0x0040, r)
+    return r.astype(np.uint16)
+
+
+def lmhead_bwd(dlogits, Hh, W):
+    """Version-2 gradients of the LM head: the two contractions are the version-2 contraction itself on transposed
+    operands (the definition is symmetric in its two rows and order-free, so a transpose is all it takes).
+      g  = bf16(dlogits)                                    (rounded once, as in version 1)
+      dH = bf16(contraction of row m of g with column k of W over the vocabulary)     [M,K] bf16
+      dW = contraction of column v of g with column k of Hh over the tokens           [V,K] f32
+    Row exponents are taken over the contracted index: per token for g and per input dimension for W in dH, per
+    vocabulary entry for g and per input dimension for Hh in dW."""
+    g = _f2bf(dlogits)
+    Hh = np.ascontiguousarray(Hh, dtype=np.uint16)
+    W = np.ascontiguousarray(W, dtype=np.uint16)
+    dH = _f2bf(lmhead_fwd(g, np.ascontiguousarray(W.T)))
+    dW = lmhead_fwd(np.ascontiguousarray(g.T), np.ascontiguousarray(Hh.T))
+    return dH, dW

@@ -53,7 +53,7 @@ def load():
         for name in ("det_sum_ws_bytes", "det_grad_norm_ws_bytes", "det_lsq_weight_scale_ws_bytes",
                      "det_lsq_act_scale_init_ws_bytes", "det_lsq_quantize_weight_ws_bytes", "det_linear_bwd_ws_bytes",
                      "det_rmsnorm_bwd_ws_bytes", "det_xent_ws_bytes", "det_attn_bwd_ws_bytes", "det_attn_bwd_fixq_ws_bytes",
-                     "det_tensor_hash_ws_bytes", "det_lmhead_fwd_v2_ws_bytes"):
+                     "det_tensor_hash_ws_bytes", "det_lmhead_fwd_v2_ws_bytes", "det_lmhead_bwd_v2_ws_bytes"):
             getattr(_lib, name).restype = C.c_size_t
         _lib.det_launch_count.restype = C.c_ulonglong
     return _lib
@@ -319,6 +319,15 @@ def det_lmhead_fwd_v2_ws_bytes(M, V, K):
 def det_lmhead_fwd_v2(H, W, M, V, K, logits, ws, status_dev=None):
     _check("det_lmhead_fwd_v2", load().det_lmhead_fwd_v2(_ptr(H), _ptr(W), C.c_int(M), C.c_int(V), C.c_int(K), _ptr(logits),
                                                          *_ws(ws), _stream(), _ptr(status_dev)))
+
+
+def det_lmhead_bwd_v2_ws_bytes(M, V, K):
+    return load().det_lmhead_bwd_v2_ws_bytes(C.c_int(M), C.c_int(V), C.c_int(K))
+
+
+def det_lmhead_bwd_v2(dlogits, H, W, M, V, K, dH, dW, ws, status_dev=None):
+    _check("det_lmhead_bwd_v2", load().det_lmhead_bwd_v2(_ptr(dlogits), _ptr(H), _ptr(W), C.c_int(M), C.c_int(V), C.c_int(K),
+                                                         _ptr(dH), _ptr(dW), *_ws(ws), _stream(), _ptr(status_dev)))
 
 
 def det_lmhead_bwd(dlogits, H, W, M, V, K, dH, dW, first_chunk):

@@ -19,15 +19,40 @@
 namespace det {
 
 // ---- slicing ----------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_slice_rows(const uint16_t* __restrict__ X, int R, int K, int8_t* __restrict__ hi,
+// bf16 bit pattern of a binary32 value (subnormal inputs flushed first), as the gradient of the logits is rounded
+__device__ __forceinline__ uint32_t bf_bits(float x) {
+  if (!(__float_as_uint(x) & 0x7f800000u)) x = __uint_as_float(__float_as_uint(x) & 0x80000000u);
+  return (uint32_t)f2bf(x);
+}
+// signed 14-bit aligned value of one bf16 pattern against the exponent e of its row, as two int8 slices
+__device__ __forceinline__ void slice1(uint32_t b, int e, int& h, int& l) {
+  const int ek = (b >> 7) & 0xFF, d = e - ek;
+  const int t = (ek == 0 || d >= 14) ? 0 : (int)(((128u + (b & 0x7Fu)) << 6) >> d);
+  h = t >> 7; l = t & 127;
+  if (b & 0x8000u) { h = -h; l = -l; }
+}
+// eight values of a row as four words of packed bf16 patterns: bf16 source as stored, f32 source rounded to bf16
+template <bool F32>
+__device__ __forceinline__ void load8_bits(const void* X, size_t idx, uint32_t (&w)[4]) {
+  if (F32) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + idx));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + idx) + 1);
+    w[0] = bf_bits(a.x) | (bf_bits(a.y) << 16); w[1] = bf_bits(a.z) | (bf_bits(a.w) << 16);
+    w[2] = bf_bits(b.x) | (bf_bits(b.y) << 16); w[3] = bf_bits(b.z) | (bf_bits(b.w) << 16);
+  } else {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + idx));
+    w[0] = u.x; w[1] = u.y; w[2] = u.z; w[3] = u.w;
+  }
+}
+template <bool F32>
+__global__ void __launch_bounds__(256) k_slice_rows(const void* __restrict__ X, int R, int K, int8_t* __restrict__ hi,
                                                     int8_t* __restrict__ lo, int32_t* __restrict__ E) {
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (row >= R) return;
-  const uint4* x = reinterpret_cast<const uint4*>(X + (size_t)row * K);
   int e = 0, bad = 0;
   for (int i = lane; i < K / 8; i += 32) {
-    const uint4 u = __ldg(x + i);
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    uint32_t w[4];
+    load8_bits<F32>(X, (size_t)row * K + 8 * (size_t)i, w);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int e0 = (w[j] >> 7) & 0xFF, e1 = (w[j] >> 23) & 0xFF;
@@ -42,21 +67,70 @@ __global__ void __launch_bounds__(256) k_slice_rows(const uint16_t* __restrict__
   }
   if (lane == 0) E[row] = e | (bad ? (1 << 30) : 0);
   for (int i = lane; i < K / 8; i += 32) {
-    const uint4 u = __ldg(x + i);
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    uint32_t w[4];
+    load8_bits<F32>(X, (size_t)row * K + 8 * (size_t)i, w);
     uint32_t h8[2] = {0u, 0u}, l8[2] = {0u, 0u};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const uint32_t b = (j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu);
-      const int ek = (b >> 7) & 0xFF, d = e - ek;
-      int t = (ek == 0 || d >= 14) ? 0 : (int)(((128u + (b & 0x7Fu)) << 6) >> d);
-      int h = t >> 7, l = t & 127;
-      if (b & 0x8000u) { h = -h; l = -l; }
+      int h, l;
+      slice1(b, e, h, l);
       h8[j >> 2] |= (uint32_t)(uint8_t)(int8_t)h << (8 * (j & 3));
       l8[j >> 2] |= (uint32_t)(uint8_t)(int8_t)l << (8 * (j & 3));
     }
     *reinterpret_cast<uint2*>(hi + (size_t)row * K + 8 * i) = make_uint2(h8[0], h8[1]);
     *reinterpret_cast<uint2*>(lo + (size_t)row * K + 8 * i) = make_uint2(l8[0], l8[1]);
+  }
+}
+
+// Slicing along the OTHER index, for the gradient contractions: the exponent of column c is taken over the rows r, and the
+// slices are written transposed ([C, R], so that the contracted index r is contiguous for the tensor core).
+//   k_col_exp     E[c] = max over r (integer maximum through atomicMax: order-free); E must be zero before
+//   k_slice_cols  a CTA takes a 128 x 128 tile: thread = column (a warp reads 32 adjacent values of a row), 128 rows in
+//                 registers as packed bytes, out through a swizzled shared-memory tile as whole 128-byte lines
+template <bool F32>
+__global__ void __launch_bounds__(128) k_col_exp(const void* __restrict__ X, int R, int C, int32_t* __restrict__ E) {
+  const int c = blockIdx.x * 128 + threadIdx.x, r0 = blockIdx.y * 128;
+  int key = 0;
+#pragma unroll 8
+  for (int i = 0; i < 128; ++i) {
+    const size_t idx = (size_t)(r0 + i) * C + c;
+    const uint32_t b = F32 ? bf_bits(__ldg(reinterpret_cast<const float*>(X) + idx)) : (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(X) + idx);
+    const int e = (b >> 7) & 0xFF;
+    key = max(key, e | (e == 255 ? (1 << 30) : 0));
+  }
+  if (key > *reinterpret_cast<volatile int32_t*>(E + c)) atomicMax(E + c, key);
+}
+template <bool F32>
+__global__ void __launch_bounds__(128) k_slice_cols(const void* __restrict__ X, int R, int C, const int32_t* __restrict__ E,
+                                                    int8_t* __restrict__ hiT, int8_t* __restrict__ loT) {
+  __shared__ __align__(16) uint8_t tile[2][128 * 128];
+  const int t = threadIdx.x, c0 = blockIdx.x * 128, r0 = blockIdx.y * 128;
+  const int e = E[c0 + t] & 0xFF;
+  uint32_t hw[32], lw[32];
+#pragma unroll
+  for (int i = 0; i < 128; ++i) {
+    const size_t idx = (size_t)(r0 + i) * C + c0 + t;
+    const uint32_t b = F32 ? bf_bits(__ldg(reinterpret_cast<const float*>(X) + idx)) : (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(X) + idx);
+    int h, l;
+    slice1(b, e, h, l);
+    if ((i & 3) == 0) { hw[i >> 2] = 0u; lw[i >> 2] = 0u; }
+    hw[i >> 2] |= (uint32_t)(uint8_t)(int8_t)h << (8 * (i & 3));
+    lw[i >> 2] |= (uint32_t)(uint8_t)(int8_t)l << (8 * (i & 3));
+  }
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {   // row t of the transposed tiles, sixteen-byte pieces XOR-swizzled by row
+    const int off = t * 128 + ((g ^ (t & 7)) << 4);
+    *reinterpret_cast<uint4*>(tile[0] + off) = make_uint4(hw[4 * g], hw[4 * g + 1], hw[4 * g + 2], hw[4 * g + 3]);
+    *reinterpret_cast<uint4*>(tile[1] + off) = make_uint4(lw[4 * g], lw[4 * g + 1], lw[4 * g + 2], lw[4 * g + 3]);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = i * 16 + (t >> 3), ch = t & 7;
+    const int off = r * 128 + ((ch ^ (r & 7)) << 4);
+    *reinterpret_cast<uint4*>(hiT + (size_t)(c0 + r) * R + r0 + ch * 16) = *reinterpret_cast<const uint4*>(tile[0] + off);
+    *reinterpret_cast<uint4*>(loT + (size_t)(c0 + r) * R + r0 + ch * 16) = *reinterpret_cast<const uint4*>(tile[1] + off);
   }
 }
 
@@ -77,10 +151,11 @@ __device__ __forceinline__ float round_scaled(long long I, int e) {
   return r;
 }
 
+template <bool OUT_BF16>
 __global__ void __launch_bounds__(SL_THREADS, 1)
     k_igemm_sl(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
                const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const int32_t* __restrict__ Ea,
-               const int32_t* __restrict__ Eb, float* __restrict__ out, int I, int J, int K, int* status) {
+               const int32_t* __restrict__ Eb, void* __restrict__ out, int I, int J, int K, int* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ __align__(8) uint64_t bar_full[SL_STAGES], bar_empty[SL_STAGES], bar_tfull, bar_tempty;
@@ -168,7 +243,8 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       const int row = i0 + q * 32 + lane;
       const int ea = Ea[row];
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-      float* orow = out + (size_t)row * J + j0;
+      float* orow = reinterpret_cast<float*>(out) + (size_t)row * J + j0;
+      uint16_t* brow = reinterpret_cast<uint16_t*>(out) + (size_t)row * J + j0;
 #pragma unroll 1
       for (int c0 = 0; c0 < SL_T; c0 += 32) {
         uint32_t hh[32], cr[32], ll[32];
@@ -185,7 +261,8 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
             const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
             f[x] = ((ea | eb) >> 30) ? __int_as_float(0x7FC00000) : round_scaled(Iv, (ea & 0xFF) + (eb & 0xFF) - 280);
           }
-          *reinterpret_cast<float4*>(orow + c0 + 4 * v) = make_float4(f[0], f[1], f[2], f[3]);
+          if (OUT_BF16) *reinterpret_cast<uint2*>(brow + c0 + 4 * v) = make_uint2(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]));
+          else *reinterpret_cast<float4*>(orow + c0 + 4 * v) = make_float4(f[0], f[1], f[2], f[3]);
         }
       }
       tc_fence_before();
@@ -209,6 +286,24 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
 
 using namespace det;
 
+// one sliced contraction out[i,j] = round(I 2^(Ea[i] + Eb[j] - 280)) from the slices of both operands ([I,K] and [J,K] int8)
+template <bool OUT_BF16>
+static int sliced_gemm(const int8_t* Ah, const int8_t* Al, const int8_t* Bh, const int8_t* Bl, const int32_t* Ea, const int32_t* Eb,
+                       void* out, int I, int J, int K, int* status, cudaStream_t st) {
+  CUtensorMap tAh, tAl, tBh, tBl;
+  if (!make_map(&tAh, Ah, I, K, SL_T) || !make_map(&tAl, Al, I, K, SL_T) || !make_map(&tBh, Bh, J, K, SL_T) ||
+      !make_map(&tBl, Bl, J, K, SL_T))
+    return DET_ERR_CUDA;
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_igemm_sl<OUT_BF16>, SL_SMEM) != DET_OK) return DET_ERR_CUDA;
+  const int sms = dev_sm_count();
+  if (sms <= 0) return DET_ERR_CUDA;
+  const int tiles = (I / SL_T) * (J / SL_T);
+  k_igemm_sl<OUT_BF16><<<DET_L(tiles < sms ? tiles : sms), SL_THREADS, SL_SMEM, st>>>(tAh, tAl, tBh, tBl, Ea, Eb, out, I, J, K, status);
+  if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
+  return DET_OK;
+}
+
 static size_t v2_layout(int M, int V, int K, size_t* oAh, size_t* oAl, size_t* oBh, size_t* oBl, size_t* oEa, size_t* oEb) {
   size_t off = 0;
   *oAh = off; off += align_up((size_t)M * K, 256);
@@ -227,7 +322,7 @@ extern "C" int det_lmhead_fwd_v2(const det_bf16* H, const det_bf16* W, int M, in
                                  size_t ws_bytes, void* stream, int* status_dev) {
   if (!H || !W || !logits || M <= 0 || V <= 0 || K <= 0) return DET_ERR_ARG;
   if (M % SL_T || V % SL_T || K % SL_BK) return DET_ERR_SHAPE;
-  if (K >= (1 << 17)) return DET_ERR_RANGE;
+  if (K >= (1 << 16)) return DET_ERR_RANGE;   // the cross accumulator holds two products: 2 K 127^2 must stay below 2^31
   if (!aligned16(H) || !aligned16(W) || !aligned16(logits) || !aligned16(ws)) return DET_ERR_ALIGN;
   size_t oAh, oAl, oBh, oBl, oEa, oEb;
   if (!ws || ws_bytes < v2_layout(M, V, K, &oAh, &oAl, &oBh, &oBl, &oEa, &oEb)) return DET_ERR_WORKSPACE;
@@ -235,19 +330,52 @@ extern "C" int det_lmhead_fwd_v2(const det_bf16* H, const det_bf16* W, int M, in
   uint8_t* base = (uint8_t*)ws;
   int8_t *Ah = (int8_t*)(base + oAh), *Al = (int8_t*)(base + oAl), *Bh = (int8_t*)(base + oBh), *Bl = (int8_t*)(base + oBl);
   int32_t *Ea = (int32_t*)(base + oEa), *Eb = (int32_t*)(base + oEb);
-  k_slice_rows<<<DET_L((M + 7) / 8), 256, 0, st>>>(H, M, K, Ah, Al, Ea);
-  k_slice_rows<<<DET_L((V + 7) / 8), 256, 0, st>>>(W, V, K, Bh, Bl, Eb);
+  k_slice_rows<false><<<DET_L((M + 7) / 8), 256, 0, st>>>(H, M, K, Ah, Al, Ea);
+  k_slice_rows<false><<<DET_L((V + 7) / 8), 256, 0, st>>>(W, V, K, Bh, Bl, Eb);
   DET_CHECK_LAUNCH();
-  CUtensorMap tAh, tAl, tBh, tBl;
-  if (!make_map(&tAh, Ah, M, K, SL_T) || !make_map(&tAl, Al, M, K, SL_T) || !make_map(&tBh, Bh, V, K, SL_T) ||
-      !make_map(&tBl, Bl, V, K, SL_T))
-    return DET_ERR_CUDA;
-  static DevOnce once = {};
-  if (dev_ensure_smem(once, (const void*)k_igemm_sl, SL_SMEM) != DET_OK) return DET_ERR_CUDA;
-  const int sms = dev_sm_count();
-  if (sms <= 0) return DET_ERR_CUDA;
-  const int tiles = (M / SL_T) * (V / SL_T);
-  k_igemm_sl<<<DET_L(tiles < sms ? tiles : sms), SL_THREADS, SL_SMEM, st>>>(tAh, tAl, tBh, tBl, Ea, Eb, logits, M, V, K, status_dev);
+  return sliced_gemm<false>(Ah, Al, Bh, Bl, Ea, Eb, logits, M, V, K, status_dev, st);
+}
+
+// ---- gradients (version 2): the same contraction on transposed operands -------------------------------------------------
+static size_t v2b_layout(int M, int V, int K, size_t (&o)[12]) {
+  size_t off = 0;
+  const size_t sz[12] = {(size_t)M * V, (size_t)M * V,      // g = bf16(dlogits), rows (exponent per token): hi, lo [M,V]
+                         (size_t)M * V, (size_t)M * V,      // g columns, transposed (exponent per vocabulary entry): hi, lo [V,M]
+                         (size_t)V * K, (size_t)V * K,      // W columns, transposed: hi, lo [K,V]
+                         (size_t)M * K, (size_t)M * K,      // H columns, transposed: hi, lo [K,M]
+                         (size_t)M * 4, (size_t)V * 4, (size_t)K * 4, (size_t)K * 4};   // exponents: g rows, g columns, W columns, H columns
+  for (int i = 0; i < 12; ++i) { o[i] = off; off += align_up(sz[i], 256); }
+  return off;
+}
+extern "C" size_t det_lmhead_bwd_v2_ws_bytes(int M, int V, int K) {
+  size_t o[12];
+  return v2b_layout(M, V, K, o);
+}
+extern "C" int det_lmhead_bwd_v2(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH,
+                                 float* dW, void* ws, size_t ws_bytes, void* stream, int* status_dev) {
+  if (!dlogits || !H || !W || !dH || !dW || M <= 0 || V <= 0 || K <= 0) return DET_ERR_ARG;
+  if (M % SL_T || V % SL_T || K % SL_BK) return DET_ERR_SHAPE;
+  if (M >= (1 << 16) || V >= (1 << 16)) return DET_ERR_RANGE;   // contraction lengths of the two gradients
+  if (!aligned16(dlogits) || !aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW) || !aligned16(ws)) return DET_ERR_ALIGN;
+  size_t o[12];
+  if (!ws || ws_bytes < v2b_layout(M, V, K, o)) return DET_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* b = (uint8_t*)ws;
+  int8_t *gh = (int8_t*)(b + o[0]), *gl = (int8_t*)(b + o[1]), *gTh = (int8_t*)(b + o[2]), *gTl = (int8_t*)(b + o[3]);
+  int8_t *WTh = (int8_t*)(b + o[4]), *WTl = (int8_t*)(b + o[5]), *HTh = (int8_t*)(b + o[6]), *HTl = (int8_t*)(b + o[7]);
+  int32_t *Eg = (int32_t*)(b + o[8]), *EgT = (int32_t*)(b + o[9]), *EWT = (int32_t*)(b + o[10]), *EHT = (int32_t*)(b + o[11]);
+  cudaMemsetAsync(EgT, 0, o[11] - o[9] + align_up((size_t)K * 4, 256), st);        // the three column-exponent arrays
+  k_slice_rows<true><<<DET_L((M + 7) / 8), 256, 0, st>>>(dlogits, M, V, gh, gl, Eg);
+  k_col_exp<true><<<DET_L(dim3(V / 128, M / 128)), 128, 0, st>>>(dlogits, M, V, EgT);
+  k_col_exp<false><<<DET_L(dim3(K / 128, V / 128)), 128, 0, st>>>(W, V, K, EWT);
+  k_col_exp<false><<<DET_L(dim3(K / 128, M / 128)), 128, 0, st>>>(H, M, K, EHT);
+  k_slice_cols<true><<<DET_L(dim3(V / 128, M / 128)), 128, 0, st>>>(dlogits, M, V, EgT, gTh, gTl);
+  k_slice_cols<false><<<DET_L(dim3(K / 128, V / 128)), 128, 0, st>>>(W, V, K, EWT, WTh, WTl);
+  k_slice_cols<false><<<DET_L(dim3(K / 128, M / 128)), 128, 0, st>>>(H, M, K, EHT, HTh, HTl);
   DET_CHECK_LAUNCH();
-  return DET_OK;
+  // dH[m,k] = bf16(contraction over the vocabulary of row m of g with column k of W)
+  int rc = sliced_gemm<true>(gh, gl, WTh, WTl, Eg, EWT, dH, M, K, V, status_dev, st);
+  if (rc != DET_OK) return rc;
+  // dW[v,k] = contraction over the tokens of column v of g with column k of H
+  return sliced_gemm<false>(gTh, gTl, HTh, HTl, EgT, EHT, dW, V, K, M, status_dev, st);
 }

@@ -177,6 +177,17 @@ def case_lmhead_v2(small):
     return (lambda: det.det_lmhead_fwd_v2(Hh, W, M, V, K, lg, w, st)), 2.0 * M * V * K, "flop"
 
 
+def case_lmhead_bwd_v2(small):
+    """Both gradient contractions of the LM head in arithmetic version 2; same nominal work as lmhead_bwd."""
+    M, V, K = (1024 if small else 8192), 50304, 2048
+    Hh, W = randn_bf16(M * K), randn_bf16(V * K, 0.02)
+    lg = torch.empty(M * V, device="cuda").normal_(0, 1e-3)
+    dH, dW = torch.empty(M * K, dtype=I16, device="cuda"), torch.empty(V * K, device="cuda")
+    w = ws(det.det_lmhead_bwd_v2_ws_bytes(M, V, K))
+    st = torch.zeros(1, dtype=I32, device="cuda")
+    return (lambda: det.det_lmhead_bwd_v2(lg, Hh, W, M, V, K, dH, dW, w, st)), 4.0 * M * V * K, "flop"
+
+
 def case_accum(small):
     n = (1 << 26) if small else (1 << 28)
     g = torch.randn(n, device="cuda")
@@ -210,7 +221,7 @@ def build_cases():
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
          "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
          "attn_bwd_fixq": lambda s: case_attn(s, True, False, True),
-         "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_fwd_v2": case_lmhead_v2, "lmhead_bwd": lambda s: case_lmhead(s, True),
+         "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_fwd_v2": case_lmhead_v2, "lmhead_bwd_v2": case_lmhead_bwd_v2, "lmhead_bwd": lambda s: case_lmhead(s, True),
          "accum": case_accum, "adamw": case_adamw, "hash": case_hash}
     for k in LINEAR_SHAPES:
         c["igemm_" + k] = (lambda s, k=k: case_igemm(s, k))

@@ -392,6 +392,34 @@ def test_lmhead_forward_version_2(det, M, V, K):
     assert np.all(np.delete(got[3], 7).view(np.uint32) == 0)          # the all-zero row: +0 against every finite row of W
 
 
+@pytest.mark.parametrize("M,V,K", [(128, 128, 128), (256, 384, 256), (384, 1152, 128)])
+def test_lmhead_backward_version_2(det, M, V, K):
+    """Both gradient contractions of arithmetic version 2 (column slicing with transposed output, f32 source rounded to
+    bf16 first, bf16 and f32 results) against the oracle, bit for bit; gradients over a wide range of exponents, a
+    subnormal one, an all-zero token, a non-finite one."""
+    import torch
+    from oracle import v2
+    rng = np.random.default_rng(M + V + K + 1)
+    Hh = synth.to_bf16((rng.standard_normal((M, K)) * np.exp2(rng.integers(-6, 4, (M, K)))).astype(F))
+    W = synth.to_bf16((rng.standard_normal((V, K)) * 0.02 * np.exp2(rng.integers(-8, 3, (V, K)))).astype(F))
+    dl = (rng.standard_normal((M, V)) * 1e-3 * np.exp2(rng.integers(-12, 2, (M, V)))).astype(F)
+    dl[2] = 0
+    dl[4, 5] = 1e-41
+    dl[6, 9] = np.inf
+    dH, dW = empty((M, K), np.uint16), empty((V, K), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_lmhead_bwd_v2(dev(dl), dev(Hh), dev(W), M, V, K, dH, dW, ws(det.det_lmhead_bwd_v2_ws_bytes(M, V, K)), status)
+    _sync()
+    assert int(status.item()) == 0
+    wH, wW = v2.lmhead_bwd(dl, Hh, W)
+    gH, gW = host(dH, np.uint16), host(dW)
+    nanH, nanW = np.isnan(synth.from_bf16(wH)), np.isnan(wW)
+    assert nanH[6].all() and nanW[9].all() and nanH.sum() == K and nanW.sum() == K
+    assert np.array_equal(np.isnan(synth.from_bf16(gH)), nanH) and np.array_equal(np.isnan(gW), nanW)
+    assert_same_bits(gH[~nanH], wH[~nanH], "version-2 dH")
+    assert_same_bits(gW[~nanW], wW[~nanW], "version-2 dW")
+
+
 def test_embedding(det):
     V, D, T = 1000, 512, 700
     E = synth.normal_bf16((V, D), 0.02, seed=7, tid=1)

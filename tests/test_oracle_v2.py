@@ -131,3 +131,29 @@ def test_special_rows():
     assert np.isfinite(got[0, 0]) and np.isfinite(got[0, 2])
     _, _, E = v2.slice_rows(a)
     assert E[1] == 0 and E[3] == 0 and (E[2] >> 30) == 1
+
+
+def test_backward_is_the_contraction_on_transposed_operands_and_close_to_float64():
+    """dH and dW of version 2 against float64 (the bound of the forward applies), bf16 rounding of dlogits pinned against
+    the shared input generator's converter, and shapes / dtypes."""
+    rng = np.random.default_rng(7)
+    M, V, K = 24, 40, 32
+    Hh = synth.normal_bf16((M, K), 1.0, seed=8, tid=1)
+    W = synth.normal_bf16((V, K), 0.02, seed=8, tid=2)
+    dl = (rng.standard_normal((M, V)) * 1e-3).astype(F)
+    dl[0, 0] = 1e-41                                       # a subnormal gradient is flushed before it is rounded
+    assert np.array_equal(v2._f2bf(dl[1:]), synth.to_bf16(dl[1:])) and v2._f2bf(dl[:1])[0, 0] == 0
+    dH, dW = v2.lmhead_bwd(dl, Hh, W)
+    assert dH.shape == (M, K) and dH.dtype == np.uint16 and dW.shape == (V, K) and dW.dtype == F
+    g = synth.from_bf16(v2._f2bf(dl)).astype(np.float64)
+    rH = g @ synth.from_bf16(W).astype(np.float64)
+    rW = g.T @ synth.from_bf16(Hh).astype(np.float64)
+    assert np.max(np.abs(synth.from_bf16(dH) - rH)) <= np.max(np.abs(rH)) * 2.0 ** -8
+    assert np.max(np.abs(dW - rW)) <= np.max(np.abs(rW)) * 1e-3
+    # brute force of single elements in exact rational arithmetic from the values
+    for (m, k) in ((0, 0), (5, 7), (23, 31)):
+        want = _brute(v2._f2bf(dl)[m], np.ascontiguousarray(W[:, k]))
+        assert synth.from_bf16(dH[m:m + 1, k:k + 1])[0, 0] == synth.from_bf16(synth.to_bf16(np.array([want], F)))[0]
+    for (v, k) in ((0, 0), (11, 3), (39, 31)):
+        want = _brute(np.ascontiguousarray(v2._f2bf(dl)[:, v]), np.ascontiguousarray(Hh[:, k]))
+        assert dW[v, k].view(np.uint32) == F(want).view(np.uint32)
