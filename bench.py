@@ -335,6 +335,7 @@ def run_ours(args):
     from paper_2609_17380_b200 import step as dstep
     det.load()
     kw = full_config_kwargs(args.layers, args.workload)
+    kw["arith"] = args.arith
     cfg = dstep.ModelConfig(**kw)
     n_mb = cfg.n_microbatches
     # N > 1: the micro-batches of the one global step are shared out over the ranks and the gradient is exchanged in
@@ -485,7 +486,8 @@ def run_ours(args):
             "ms_per_step": per_step, "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": "int8 tensor-core GEMMs + f32 ordered arithmetic (bf16 storage)", "data": "synthetic",
             "config": {"workload": (WORKLOAD if args.workload == "config5" else WORKLOAD_PAPER) +
-                       ("" if args.layers is None else " [REDUCED to %d layers]" % args.layers),
+                       ("" if args.layers is None else " [REDUCED to %d layers]" % args.layers) +
+                       ("" if args.arith == 1 else " [LM-head contractions in arithmetic version 2: NOT the benchmark's arithmetic]"),
                        "l2": "inputs_exceed_l2", "multi_gpu": ("micro-batches sharded over ranks, ordered gradient exchange, replicated optimizer" if sharded
                                      else "replicas only" if world > 1 else "single"), "ranks_agree": agree},
             "clocks": clocks, "gpu_launches": int(launches),
@@ -524,6 +526,8 @@ def main():
                          "exchanging them with point-to-point copies first")
     ap.add_argument("--workload", choices=("config5", "paper"), default="config5",
                     help="config5 (default) is the benchmark configuration; paper is the paper's own block and shapes")
+    ap.add_argument("--arith", type=int, choices=(1, 2), default=1,
+                    help="2: the LM-head contractions in arithmetic version 2 (order-free, int8 tensor cores); not the default metric")
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -7,6 +7,7 @@ hash.  Written independently of the CUDA-side driver; they share only the seeded
 import numpy as np
 
 import oracle as O
+from oracle import v2 as O2
 
 LINEARS = ("w_qkv", "w_o", "w_gu", "w_down")
 
@@ -79,7 +80,8 @@ def forward(cfg, P, sw, tok, calibrate=False):
         saved["layers"].append(a)
     saved["xf"] = x
     saved["nf"], saved["rstdf"] = O.rmsnorm_fwd(x, P["final_norm"], 1e-6, bf=True)
-    saved["logits"] = O.lmhead_fwd(saved["nf"], P["lm_head"])
+    # arithmetic version 2 (cfg["arith"] == 2) replaces the LM-head contractions by the order-free ones of oracle/v2
+    saved["logits"] = (O2 if cfg.get("arith", 1) == 2 else O).lmhead_fwd(saved["nf"], P["lm_head"])
     return saved
 
 
@@ -94,7 +96,7 @@ def microbatch_grad(cfg, P, sw, tok):
     _, lse, loss_mean, _, _ = O.xent_fwd(sv["logits"], labels, cfg.get("z_weight", 0.0))
     dlog = O.xent_bwd(sv["logits"], labels, lse, cfg.get("z_weight", 0.0), np.float32(1.0 / T))
     G = {}
-    d_nf, G["lm_head"] = O.lmhead_bwd(dlog, sv["nf"], P["lm_head"])
+    d_nf, G["lm_head"] = (O2 if cfg.get("arith", 1) == 2 else O).lmhead_bwd(dlog, sv["nf"], P["lm_head"])
     dx, G["final_norm"] = O.rmsnorm_bwd(d_nf, sv["xf"], P["final_norm"], sv["rstdf"], bf=True)
     for l in reversed(range(L)):
         a = sv["layers"][l]

@@ -43,6 +43,7 @@ class ModelConfig:
     full_every: int = 5              # every full_every-th layer and the last one attend to the whole prefix
     pv_int8: bool = False            # forward P.V of every block of 128 keys on the int8 tensor cores
     dq_fixed: bool = False           # query gradient accumulated over the key blocks in 64-bit fixed point
+    arith: int = 1                   # 2: the LM-head contractions in arithmetic version 2 (order-free, int8 tensor cores)
 
     def as_dict(self):
         return dict(self.__dict__)
@@ -151,6 +152,7 @@ class Replay:
                   det.det_xent_ws_bytes(T, V), det.det_rmsnorm_bwd_ws_bytes(T, D),
                   det.det_lsq_weight_scale_ws_bytes(2 * Fh, D), det.det_lsq_act_scale_init_ws_bytes(T * max(Fh, D)),
                   det.det_tensor_hash_ws_bytes(g * 4), det.det_sum_ws_bytes(g), 1 << 20,
+                  (max(det.det_lmhead_fwd_v2_ws_bytes(T, V, D), det.det_lmhead_bwd_v2_ws_bytes(T, V, D)) if cfg.arith == 2 else 0),
                   *[det.det_linear_bwd_ws_bytes(T, N, K) for (N, K) in ((QW, D), (D, D), (2 * Fh, D), (D, Fh))])
         self.ws = e(wsb + 4096, torch.uint8)
         self.losses = []
@@ -322,7 +324,10 @@ class Replay:
         self.xf.copy_(x)
         det.det_rmsnorm_fwd(det.DET_BF16, self.xf, self.p("final_norm"), T, D, 1e-6, self.nf, self.rstdf)
         with self.span("lmhead_fwd"):
-            det.det_lmhead_fwd(self.nf, self.p("lm_head"), T, V, D, self.logits)
+            if cfg.arith == 2:
+                det.det_lmhead_fwd_v2(self.nf, self.p("lm_head"), T, V, D, self.logits, self.ws, self.status)
+            else:
+                det.det_lmhead_fwd(self.nf, self.p("lm_head"), T, V, D, self.logits)
         with self.span("xent_fwd"):
             det.det_xent_fwd(self.logits, self.lab, T, V, cfg.z_weight, self.loss_row, self.lse_x, self.loss_mean,
                              self.z_mean, self.ws, self.status)
@@ -345,7 +350,11 @@ class Replay:
         t0, t1, t2 = self.tmp
         d_nf = t0[:T * D]
         with self.span("lmhead_bwd"):
-            det.det_lmhead_bwd(self.logits, self.nf, self.p("lm_head"), T, V, D, d_nf, self.g(self.gmb, "lm_head"), 1)
+            if cfg.arith == 2:
+                det.det_lmhead_bwd_v2(self.logits, self.nf, self.p("lm_head"), T, V, D, d_nf, self.g(self.gmb, "lm_head"),
+                                      self.ws, self.status)
+            else:
+                det.det_lmhead_bwd(self.logits, self.nf, self.p("lm_head"), T, V, D, d_nf, self.g(self.gmb, "lm_head"), 1)
         dx = t1[:T * D]
         det.det_rmsnorm_bwd(det.DET_BF16, d_nf, self.xf, self.p("final_norm"), self.rstdf, T, D, dx,
                             self.g(self.gmb, "final_norm"), self.ws)

@@ -83,6 +83,19 @@ def test_step_with_separate_quantiser_passes_gives_the_same_hashes():
         assert not [k for k, h in want["hashes"].items() if got["hashes"][k] != h], fuse
 
 
+def test_step_in_arithmetic_version_2_matches_its_oracle():
+    """The step with the LM-head contractions in arithmetic version 2 (order-free, on the int8 tensor cores) against the
+    oracle's step in the same version: every hash; and it is a different arithmetic from version 1 (the hashes differ)."""
+    kw = dict(n_layers=1, d_model=256, n_heads=2, ffn=512, vocab=512, seq=128, micro_batch=2, mesh=(2, 1, 2))
+    cfg, got, want = _run(dict(kw, arith=2), seed=12)
+    assert got["status"] == 0
+    assert got["losses"] == [np.float32(x) for x in want["losses"]]
+    assert not [k for k, h in want["hashes"].items() if got["hashes"][k] != h]
+    v1 = _oracle_step(kw, 12)
+    assert v1["hashes"]["grad"] != want["hashes"]["grad"]
+    assert abs(v1["loss"] - want["loss"]) < 1e-3
+
+
 def test_full_width_step_matches_oracle():
     """One replayed step at the benchmark's full width (d_model 2048, 16 heads, FFN 8192, sequence 2048, micro-batch 4,
     Hadamard 128, CTA-pair GEMMs on every linear, the 268 MB attention workspace, the driver's shared scratch buffers at
