@@ -10,8 +10,8 @@ extern "C" {
 #endif
 
 /* Elementwise evaluation of one primitive of Sec. 2.1 ("Reproducible Operations") on device arrays: op 0 add, 1 sub,
- * 2 mul, 3 div, 4 sqrt(a), 5 det_exp(a), 6 det_log(a), 7 max, 8 bf16 round trip of a, 9 unfused a*b+b.  b may be NULL
- * for unary ops.  Lets a test compare the device arithmetic with the CPU statement of the same rule. */
+ * 2 mul, 3 div, 4 sqrt(a), 5 det_exp(a), 6 det_log(a), 7 max, 8 bf16 round trip of a, 9 unfused a*b+b, 10 the form of
+ * det_exp the softmax kernels use for arguments a <= 0 or NaN (same bits as op 5 there).  b may be NULL for unary ops.  Lets a test compare the device arithmetic with the CPU statement of the same rule. */
 int det_test_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream);
 
 /* The GEMM core of the LSQ linears alone (Sec. 3.2 "int8 computation"): exact int8 x int8 -> int32 contraction

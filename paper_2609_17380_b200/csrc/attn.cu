@@ -179,11 +179,11 @@ __global__ void __launch_bounds__(FT, 1) k_attn_fwd(const uint16_t* __restrict__
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
-      const float al = det_exp(fsub(m[i], mt));
+      const float al = det_exp_le0(fsub(m[i], mt));
       alpha[i] = rowvalid ? al : 1.0f;
       float p[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) p[e] = det_exp(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
+      for (int e = 0; e < 8; ++e) p[e] = det_exp_le0(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
 #pragma unroll
       for (int e = 0; e < 8; ++e) p[e] = valid[e] ? p[e] : 0.0f;
 #pragma unroll
@@ -526,7 +526,7 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
     // the lane that owns row r (see rows16_reduce) updates its running maximum (every row sees at least key 0 of the
     // first block, so the maximum of a block it visits is a number) and the rescale factor of what it has accumulated
     const float m_new = fmaxf(m_mine, rows_reduce<false>(rm, lane));
-    alpha_mine = det_exp(fsub(m_mine, m_new));
+    alpha_mine = det_exp_le0(fsub(m_mine, m_new));
     m_mine = m_new;
 #pragma unroll
     for (int i = 0; i < AF_RW; ++i) rm[i] = __shfl_sync(0xffffffffu, m_new, ROW_LANE(i));
@@ -536,7 +536,7 @@ __global__ void __launch_bounds__(AF_THREADS, 1)
 #pragma unroll
     for (int i = 0; i < AF_RW; ++i)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp(fsub(RP(acc, i, e), rm[i]));
+      for (int e = 0; e < 4; ++e) RP(acc, i, e) = det_exp_le0(fsub(RP(acc, i, e), rm[i]));
     if (diag) {
 #pragma unroll
       for (int i = 0; i < AF_RW; ++i)

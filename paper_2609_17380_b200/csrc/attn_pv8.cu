@@ -194,11 +194,11 @@ __global__ void __launch_bounds__(PTH, 1)
       }
 #pragma unroll
       for (int w = 1; w < 16; w <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
-      const float al0 = det_exp(fsub(m[i], mt));
+      const float al0 = det_exp_le0(fsub(m[i], mt));
       const float al = rowvalid ? al0 : 1.0f;
       float p[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) p[e] = det_exp(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
+      for (int e = 0; e < 8; ++e) p[e] = det_exp_le0(fsub(sv[e], mt));   // branch-free, so the eight chains interleave
 #pragma unroll
       for (int e = 0; e < 8; ++e) p[e] = valid[e] ? p[e] : 0.0f;
       uint32_t w0 = 0, w1 = 0;

@@ -79,7 +79,26 @@ __device__ __forceinline__ float det_exp(float x) {
   return v;
 }
 
-
+// The same function for arguments that are never positive (x <= 0, or NaN): a softmax argument z - max.  There k <= 0, so
+// neither the k = 128 product nor the overflow select can be chosen and the upper clamp of k never binds; what is left
+// is the same sequence, so every result has the bits det_exp gives.  For x > 0 the value is unspecified (no trap).
+__device__ __forceinline__ float det_exp_le0(float x) {
+  const float km = fadd(fmul(x, 0x1.715476p+0f), 12582912.0f);
+  const float kf = fsub(km, 12582912.0f);
+  const float r = fsub(fsub(x, fmul(kf, 0x1.62e400p-1f)), fmul(kf, 0x1.7f7d1cp-20f));
+  float p = 0x1.a01a02p-13f;
+  p = fadd(fmul(p, r), 0x1.6c16c2p-10f);
+  p = fadd(fmul(p, r), 0x1.111112p-7f);
+  p = fadd(fmul(p, r), 0x1.555556p-5f);
+  p = fadd(fmul(p, r), 0x1.555556p-3f);
+  p = fadd(fmul(p, r), 0.5f);
+  p = fadd(fmul(p, r), 1.0f);
+  p = fadd(fmul(p, r), 1.0f);
+  // 2^k: the bits of km are 0x4B400000 + k and 0x4B400000 << 23 is 0 mod 2^32, so k << 23 needs no subtraction; and
+  // wherever the result is kept (x at or above the flush threshold) k >= -126, so k needs no lower clamp either
+  const float v = fmul(p, __int_as_float((int)(__float_as_uint(km) << 23) + 0x3f800000));
+  return (x < -0x1.5d58a0p+6f) ? 0.0f : v;
+}
 
 // NOTE on the packed two-lane FP32 instructions (mul/add/fma .f32x2): each lane of a single packed instruction
 // rounds exactly like the scalar instruction, but ptxas contracts a packed multiply followed by a packed add into one

@@ -394,9 +394,19 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* z = logits + (size_t)blockIdx.x * V;
   float m = __int_as_float(0xff800000);
-  for (int i = threadIdx.x * 4; i < V; i += XT * 4) {
-    float4 a = *reinterpret_cast<const float4*>(z + i);
-    m = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
+  {
+    int i = threadIdx.x * 4;
+    for (; i + 3 * XT * 4 < V; i += 4 * XT * 4) {      // four loads in flight per thread
+      float4 a[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) a[u] = *reinterpret_cast<const float4*>(z + i + u * XT * 4);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) m = fmaxf(fmaxf(m, fmaxf(a[u].x, a[u].y)), fmaxf(a[u].z, a[u].w));
+    }
+    for (; i < V; i += XT * 4) {
+      float4 a = *reinterpret_cast<const float4*>(z + i);
+      m = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
+    }
   }
 #pragma unroll
   for (int w = 16; w; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
@@ -406,15 +416,38 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
 #pragma unroll
   for (int w = 1; w < XT / 32; ++w) m = fmaxf(m, red[w]);
   const int nl = (V + 255) >> 8;
-  for (int leaf = warp; leaf < nl; leaf += XT / 32) {
+  // every argument z - m is <= 0 (or NaN), so the exponential without the overflow range applies
+  const int nfull = V >> 8;  // leaves that lie wholly inside the row: no existence tests in their tree
+  float4 n0 = make_float4(0.f, 0.f, 0.f, 0.f), n1 = n0;
+  if (warp < nfull) {
+    n0 = *reinterpret_cast<const float4*>(z + warp * 256 + lane * 8);
+    n1 = *reinterpret_cast<const float4*>(z + warp * 256 + lane * 8 + 4);
+  }
+  for (int leaf = warp; leaf < nfull; leaf += XT / 32) {
+    const float4 a0 = n0, a1 = n1;
+    if (leaf + XT / 32 < nfull) {                     // the next leaf's values travel while this one is evaluated
+      const int e1 = (leaf + XT / 32) * 256 + lane * 8;
+      n0 = *reinterpret_cast<const float4*>(z + e1);
+      n1 = *reinterpret_cast<const float4*>(z + e1 + 4);
+    }
+    float e[8];
+    e[0] = det_exp_le0(fsub(a0.x, m)); e[1] = det_exp_le0(fsub(a0.y, m));          // branch-free: the chains interleave
+    e[2] = det_exp_le0(fsub(a0.z, m)); e[3] = det_exp_le0(fsub(a0.w, m));
+    e[4] = det_exp_le0(fsub(a1.x, m)); e[5] = det_exp_le0(fsub(a1.y, m));
+    e[6] = det_exp_le0(fsub(a1.z, m)); e[7] = det_exp_le0(fsub(a1.w, m));
+    const float s = warp_tree_full(tree8_full(e));
+    if (lane == 0) leafs[leaf] = s;
+  }
+  if (nfull < nl && warp == (nfull % (XT / 32))) {  // the ragged last leaf
+    const int leaf = nfull;
     const int e0 = leaf * 256 + lane * 8;
     float e[8];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (e0 + 4 * h < V) {
         float4 a = *reinterpret_cast<const float4*>(z + e0 + 4 * h);
-        e[4 * h] = det_exp(fsub(a.x, m)); e[4 * h + 1] = det_exp(fsub(a.y, m));     // branch-free: the chains interleave
-        e[4 * h + 2] = det_exp(fsub(a.z, m)); e[4 * h + 3] = det_exp(fsub(a.w, m));
+        e[4 * h] = det_exp_le0(fsub(a.x, m)); e[4 * h + 1] = det_exp_le0(fsub(a.y, m));
+        e[4 * h + 2] = det_exp_le0(fsub(a.z, m)); e[4 * h + 3] = det_exp_le0(fsub(a.w, m));
       } else {
         e[4 * h] = e[4 * h + 1] = e[4 * h + 2] = e[4 * h + 3] = 0.0f;
       }

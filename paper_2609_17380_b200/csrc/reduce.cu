@@ -224,6 +224,7 @@ __global__ void k_prim(int op, const float* a, const float* b, float* out, size_
       break;
     }
     case 9: r = fadd(fmul(x, y), y); break;
+    case 10: r = det_exp_le0(x); break;
     default: r = 0.0f;
   }
   out[i] = r;
@@ -243,7 +244,7 @@ extern "C" int det_device_sm_count(void) {
 }
 
 extern "C" int det_test_prim(int op, const float* a, const float* b, float* out, size_t n, void* stream) {
-  if (!a || !out || op < 0 || op > 9) return DET_ERR_ARG;
+  if (!a || !out || op < 0 || op > 10) return DET_ERR_ARG;
   if (n == 0) return DET_OK;
   k_prim<<<DET_L((unsigned)((n + 255) / 256)), 256, 0, (cudaStream_t)stream>>>(op, a, b, out, n);
   DET_CHECK_LAUNCH();

@@ -86,6 +86,27 @@ def test_exp_all_bf16_arguments(det):
     assert_same_bits(host(out), oracle.prim("exp", x), "exp")
 
 
+def test_exp_for_softmax_arguments_has_the_bits_of_exp(det):
+    """The softmax kernels evaluate the exponential of z - max <= 0 with the overflow range left out (test op 10): on
+    every non-positive bf16 value, a dense grid over [-110, 0], every float near the flush threshold, near 0 and near
+    the points where k changes, -inf and the negative subnormals it must give exactly the oracle's exp."""
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    xb = oracle.bf2f(h)
+    xb = xb[np.isfinite(xb) & (xb <= 0)]
+    grid = np.linspace(-110.0, 0.0, 400001).astype(F)
+    ends = []
+    for c in (float.fromhex("-0x1.5d58a0p+6"), -0.0, -0.34657359, -1.0397208, -87.0, -1.0, -86.98):
+        b = np.array([c], F).view(np.int32)[0]
+        ends.append((np.arange(-40, 41, dtype=np.int64) + int(b)).astype(np.int32).view(F))
+    x = np.concatenate([xb, grid] + ends + [np.array([-np.inf, -3.0e38, -1e-45, -1e-30, -0.0, 0.0], F)])
+    x = x[~np.isnan(x)]
+    x = x[x <= 0]
+    out = empty(x.shape, F)
+    det.det_test_prim(10, dev(x), None, out)
+    _sync()
+    assert_same_bits(host(out), oracle.prim("exp", x), "exp for arguments <= 0")
+
+
 def test_exp_dense_grid_and_ends_of_the_range(det):
     """A dense f32 grid over [-100, 100], every float within a few ULP of the two thresholds of the definition (the
     largest argument with a finite result, the smallest with a non-zero one), of 0 and of the points where k changes,
