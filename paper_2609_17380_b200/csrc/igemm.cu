@@ -346,13 +346,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 //   * the epilogue warps of both CTAs drain their own TMEM and arrive on the leader's "accumulator free" barrier
 // No load uses cluster multicast.  All waits are bounded as in the one-CTA kernel.
 // ------------------------------------------------------------------------------------------------------------
-#ifndef DET_STAGES2
-#define DET_STAGES2 6
-#endif
-constexpr int STAGES2 = DET_STAGES2;
-#ifndef DET_PROBE
-#define DET_PROBE 0
-#endif
+constexpr int STAGES2 = 6;
 constexpr int BN2 = 256;
 // warps 0 / 1 load and multiply; eight epilogue warps: warp & 3 is the TMEM lane quarter a warp may read, the two
 // warps of a quarter take one half (128 columns) of the accumulator each
@@ -453,14 +447,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
         else { i0 = (tile % tiles_i) * 256; j0 = (tile / tiles_i) * BN2; }
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
-#if DET_PROBE == 1
-          if (leader) mbar_arrive_remote(mapa_u32(smem_u32(&bar_full[stage]), 0));
-#else
           if (leader) mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);  // both CTAs' tiles complete on this barrier
           uint8_t* sa = smem + stage * STAGE_BYTES;
           tma_load_2d_pair(sa, &tmA, kb * BK, i0 + (int)rank * 128, &bar_full[stage]);
           tma_load_2d_pair(sa + STAGE_A, &tmB, kb * BK, j0 + (int)rank * 128, &bar_full[stage]);
-#endif
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
         }
       }
@@ -485,10 +475,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
           const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + STAGE_A);
 #pragma unroll
-#if DET_PROBE != 2
           for (int k4 = 0; k4 < BK / 32; ++k4)
             umma_i8_pair(tmem_d, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
-#endif
           umma_commit_pair(&bar_empty[stage]);
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
         }

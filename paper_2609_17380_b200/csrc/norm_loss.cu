@@ -93,91 +93,103 @@ __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x
   }
 }
 
-// Backward for rows of at most 2048 elements.  With DG, the CTA (8 adjacent rows) also leaves the column-wise
-// tree over its 8 rows of dy*xhat in partial8[blockIdx.x][D] (the first three levels of the row-direction tree).
-template <bool BF, bool DG>
-__global__ void __launch_bounds__(1024, 1) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
-                                                      const void* __restrict__ gamma, const float* __restrict__ rstd,
-                                                      int rows, int D, float invD, void* __restrict__ dx,
-                                                      float* __restrict__ partial8) {
-  // 32 warps = 8 rows x 4 warps; warp quarter hw owns leaves 2 hw, 2 hw + 1 (elements hw*512 ..) of its row: 16 values of
-  // dy and of x per lane, so that a whole SM's worth of warps fits (with two warps per row the 64 live values per lane
-  // left room for one 16-warp block per SM and the kernel ran at half the copy bandwidth)
+// Backward for rows of at most 2048 elements.  A CTA takes a block of 8 adjacent rows in passes of RP rows (RP * 4
+// warps: warp quarter hw of a row owns its leaves 2 hw, 2 hw + 1, i.e. 16 values of dy and of x per lane), so that
+// two CTAs share an SM and one loads or stores while the other stands at a barrier (one CTA of 8 x 4 warps per SM
+// ran 20 % slower; without the gain gradient this kernel moves its bytes at 0.9 of the copy bandwidth).  With DG the
+// CTA also leaves the column-wise tree over its 8 rows of dy*xhat in partial8[block][D] (the first three levels of
+// the row-direction tree).
+#ifndef RMS_RP
+#define RMS_RP 4
+#endif
+template <bool BF, bool DG, int RP>
+__global__ void __launch_bounds__(RP * 128, 8 / RP) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
+                                                                const void* __restrict__ gamma,
+                                                                const float* __restrict__ rstd, int rows, int D, float invD,
+                                                                void* __restrict__ dx, float* __restrict__ partial8,
+                                                                int* __restrict__ tickets) {
+  constexpr int NT = RP * 128, NPASS = 8 / RP;
   extern __shared__ __align__(16) float srow[];  // DG: [8][D]
-  __shared__ float half_sum[8][4];
+  __shared__ float half_sum[2][RP][4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rl = warp >> 2, hw = warp & 3;
-  const int row = blockIdx.x * 8 + rl;
-  const bool live = row < rows;
-  const size_t rb = (size_t)row * D;
-  float w[2][8], xh[2][8];
-#pragma unroll
-  for (int jj = 0; jj < 2; ++jj) {
-    const int e0 = (hw * 2 + jj) * 256 + lane * 8;
-    if (live && e0 < D) {
-      load8<BF>(dy, rb + e0, w[jj]);
-      load8<BF>(x, rb + e0, xh[jj]);
-    } else {
-#pragma unroll
-      for (int t = 0; t < 8; ++t) { w[jj][t] = 0.0f; xh[jj][t] = 0.0f; }
-    }
-  }
-  const float rs = live ? rstd[row] : 0.0f;
-  float mine = 0.0f;
+  const int hw = warp & 3;
   const bool full = (D & 255) == 0;
-#pragma unroll
-  for (int jj = 0; jj < 2; ++jj) {
-    const int j = hw * 2 + jj;
-    const int e0 = j * 256 + lane * 8;
-    float pr[8];
-#pragma unroll
-    for (int t = 0; t < 8; ++t) xh[jj][t] = fmul(xh[jj][t], rs);
-    if (DG && e0 < D) {
-      float dgt[8];
-#pragma unroll
-      for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[jj][t], xh[jj][t]);
-      *reinterpret_cast<float4*>(&srow[rl * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
-      *reinterpret_cast<float4*>(&srow[rl * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
-    }
-    if (gamma && e0 < D) {
-      float g[8];
-      load8<BF>(gamma, e0, g);
-#pragma unroll
-      for (int t = 0; t < 8; ++t) w[jj][t] = fmul(w[jj][t], g[t]);
-    }
-#pragma unroll
-    for (int t = 0; t < 8; ++t) pr[t] = fmul(w[jj][t], xh[jj][t]);
-    const float t8 = tree8_full(pr);
-    const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
-    if (lane == jj) mine = leaf;
-  }
-  // tree over this warp's two leaf sums (lanes 0, 1), then over the four quarters of the row (a node whose first element
-  // lies beyond D does not exist and its left neighbour is carried up unchanged)
-  {
-    const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
-    const bool right_valid = (long long)(hw * 2 + 1) * 256 < D;
-    mine = right_valid ? fadd(mine, o) : ((lane & 1) ? o : mine);
-  }
-  if (lane == 0) half_sum[rl][hw] = mine;
-  __syncthreads();
-  const float h01 = (D > 512) ? fadd(half_sum[rl][0], half_sum[rl][1]) : half_sum[rl][0];
-  const float h23 = (D > 1536) ? fadd(half_sum[rl][2], half_sum[rl][3]) : half_sum[rl][2];
-  const float tot = (D > 1024) ? fadd(h01, h23) : h01;
-  const float c = fmul(tot, invD);
-  if (live) {
+  const long long r0 = (long long)blockIdx.x * 8;
+  if (DG && blockIdx.x == 0 && (int)threadIdx.x < ((D + 255) >> 8)) tickets[threadIdx.x] = 0;   // for the kernel that follows
+#pragma unroll 1
+  for (int pass = 0; pass < NPASS; ++pass) {
+    const int rl = pass * RP + (warp >> 2);       // row of the block, 0 .. 7
+    float (*hs)[4] = half_sum[pass & 1];
+    const int row = blockIdx.x * 8 + rl;
+    const bool live = row < rows;
+    const size_t rb = (size_t)row * D;
+    float w[2][8], xh[2][8];
 #pragma unroll
     for (int jj = 0; jj < 2; ++jj) {
       const int e0 = (hw * 2 + jj) * 256 + lane * 8;
-      if (e0 >= D) continue;
-      float o[8];
+      if (live && e0 < D) {
+        load8<BF>(dy, rb + e0, w[jj]);
+        load8<BF>(x, rb + e0, xh[jj]);
+      } else {
 #pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[jj][t], fmul(xh[jj][t], c)));
-      store8<BF>(dx, rb + e0, o);
+        for (int t = 0; t < 8; ++t) { w[jj][t] = 0.0f; xh[jj][t] = 0.0f; }
+      }
+    }
+    const float rs = live ? rstd[row] : 0.0f;
+    float mine = 0.0f;
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj) {
+      const int j = hw * 2 + jj;
+      const int e0 = j * 256 + lane * 8;
+      float pr[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xh[jj][t] = fmul(xh[jj][t], rs);
+      if (DG && e0 < D) {
+        float dgt[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[jj][t], xh[jj][t]);
+        *reinterpret_cast<float4*>(&srow[rl * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
+        *reinterpret_cast<float4*>(&srow[rl * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
+      }
+      if (gamma && e0 < D) {
+        float g[8];
+        load8<BF>(gamma, e0, g);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) w[jj][t] = fmul(w[jj][t], g[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) pr[t] = fmul(w[jj][t], xh[jj][t]);
+      const float t8 = tree8_full(pr);
+      const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
+      if (lane == jj) mine = leaf;
+    }
+    // tree over this warp's two leaf sums (lanes 0, 1), then over the four quarters of the row (a node whose first
+    // element lies beyond D does not exist and its left neighbour is carried up unchanged)
+    {
+      const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
+      const bool right_valid = (long long)(hw * 2 + 1) * 256 < D;
+      mine = right_valid ? fadd(mine, o) : ((lane & 1) ? o : mine);
+    }
+    if (lane == 0) hs[warp >> 2][hw] = mine;
+    __syncthreads();
+    const float h01 = (D > 512) ? fadd(hs[warp >> 2][0], hs[warp >> 2][1]) : hs[warp >> 2][0];
+    const float h23 = (D > 1536) ? fadd(hs[warp >> 2][2], hs[warp >> 2][3]) : hs[warp >> 2][2];
+    const float tot = (D > 1024) ? fadd(h01, h23) : h01;
+    const float c = fmul(tot, invD);
+    if (live) {
+#pragma unroll
+      for (int jj = 0; jj < 2; ++jj) {
+        const int e0 = (hw * 2 + jj) * 256 + lane * 8;
+        if (e0 >= D) continue;
+        float o[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[jj][t], fmul(xh[jj][t], c)));
+        store8<BF>(dx, rb + e0, o);
+      }
     }
   }
-  if (DG) {
-    const long long r0 = (long long)blockIdx.x * 8;
-    for (int col = threadIdx.x; col < D; col += 1024) {
+  if (DG) {   // the last pass's barrier has published all eight rows of products
+    for (int col = threadIdx.x; col < D; col += NT) {
       float v[8];
 #pragma unroll
       for (int r = 0; r < 8; ++r) v[r] = srow[r * D + col];
@@ -185,19 +197,47 @@ __global__ void __launch_bounds__(1024, 1) k_rmsnorm_bwd8(const void* __restrict
     }
   }
 }
-// partial8 [nb8][D] (node = 8 rows) -> partial256 [nb256][D]: tree over 32 adjacent 8-row nodes per column
+// partial8 [nb8][D] (node = 8 rows) -> partial256 [nb256][D]: tree over 32 adjacent 8-row nodes per column; the CTA
+// that completes a block of 256 columns (a ticket counter per column block, zeroed by the kernel before, says which
+// one it is) goes on to the levels above for those columns, 32 nodes at a time, and writes dgamma.  The counter
+// decides only WHO evaluates those levels; operands and order are the fixed tree's.
 __global__ void __launch_bounds__(256) k_colsum32(const float* __restrict__ partial8, int nb8, int rows, int D,
-                                                  float* __restrict__ partial256) {
+                                                  float* __restrict__ partial256, int nb256, int* __restrict__ tickets,
+                                                  float* __restrict__ dgamma) {
+  __shared__ int last_s;
   const int col = blockIdx.x * 256 + threadIdx.x;
-  if (col >= D) return;
   const int g = blockIdx.y;
-  float s[32];
+  if (col < D) {
+    float s[32];
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const int b = g * 32 + i;
-    s[i] = (b < nb8) ? partial8[(size_t)b * D + col] : 0.0f;
+    for (int i = 0; i < 32; ++i) {
+      const int b = g * 32 + i;
+      s[i] = (b < nb8) ? partial8[(size_t)b * D + col] : 0.0f;
+    }
+    partial256[(size_t)g * D + col] = reg_tree<32>(s, (long long)g * 256, 8, rows);
   }
-  partial256[(size_t)g * D + col] = reg_tree<32>(s, (long long)g * 256, 8, rows);
+  __syncthreads();
+  if (threadIdx.x == 0) {   // the barrier orders the CTA's stores before this thread's fence, which is cumulative
+    __threadfence();
+    last_s = (atomicAdd(&tickets[blockIdx.x], 1) == nb256 - 1);
+    __threadfence();
+  }
+  __syncthreads();
+  if (!last_s || col >= D) return;
+  int n = nb256;
+  long long stride = 256;
+  while (n > 1) {
+    const int groups = (n + 31) / 32;
+    for (int gg = 0; gg < groups; ++gg) {
+      float s[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) s[i] = (gg * 32 + i < n) ? __ldcg(&partial256[(size_t)(gg * 32 + i) * D + col]) : 0.0f;
+      partial256[(size_t)gg * D + col] = reg_tree<32>(s, (long long)gg * 32 * stride, stride, rows);
+    }
+    n = groups;
+    stride *= 32;
+  }
+  dgamma[col] = __ldcg(&partial256[col]);
 }
 
 // generic two-pass variants (rows longer than 2048 elements)
@@ -418,18 +458,9 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
   const int nl = (V + 255) >> 8;
   // every argument z - m is <= 0 (or NaN), so the exponential without the overflow range applies
   const int nfull = V >> 8;  // leaves that lie wholly inside the row: no existence tests in their tree
-  float4 n0 = make_float4(0.f, 0.f, 0.f, 0.f), n1 = n0;
-  if (warp < nfull) {
-    n0 = *reinterpret_cast<const float4*>(z + warp * 256 + lane * 8);
-    n1 = *reinterpret_cast<const float4*>(z + warp * 256 + lane * 8 + 4);
-  }
   for (int leaf = warp; leaf < nfull; leaf += XT / 32) {
-    const float4 a0 = n0, a1 = n1;
-    if (leaf + XT / 32 < nfull) {                     // the next leaf's values travel while this one is evaluated
-      const int e1 = (leaf + XT / 32) * 256 + lane * 8;
-      n0 = *reinterpret_cast<const float4*>(z + e1);
-      n1 = *reinterpret_cast<const float4*>(z + e1 + 4);
-    }
+    const int e0 = leaf * 256 + lane * 8;
+    const float4 a0 = *reinterpret_cast<const float4*>(z + e0), a1 = *reinterpret_cast<const float4*>(z + e0 + 4);
     float e[8];
     e[0] = det_exp_le0(fsub(a0.x, m)); e[1] = det_exp_le0(fsub(a0.y, m));          // branch-free: the chains interleave
     e[2] = det_exp_le0(fsub(a0.z, m)); e[3] = det_exp_le0(fsub(a0.w, m));
@@ -547,20 +578,20 @@ extern "C" size_t det_rmsnorm_bwd_ws_bytes(int rows, int D) {
 template <bool BF>
 static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma, const float* rstd, int rows, int D,
                                float invD, void* dx, float* dgamma, float* ws, cudaStream_t st) {
-  dim3 grid((rows + 7) / 8);
+  constexpr int RP = RMS_RP;
+  const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
   if (!dgamma) {
-    k_rmsnorm_bwd8<BF, false><<<DET_L(grid), 1024, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr);
+    k_rmsnorm_bwd8<BF, false, RP><<<DET_L(nb8), RP * 128, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr, nullptr);
     return DET_OK;
   }
   static DevOnce once = {};
-  if (dev_ensure_smem(once, (const void*)k_rmsnorm_bwd8<BF, true>, 8 * 2048 * 4) != DET_OK) return DET_ERR_CUDA;
-  const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
+  if (dev_ensure_smem(once, (const void*)k_rmsnorm_bwd8<BF, true, RP>, 8 * 2048 * 4) != DET_OK) return DET_ERR_CUDA;
   float* partial8 = ws;
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);
-  k_rmsnorm_bwd8<BF, true><<<DET_L(grid), 1024, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8);
+  int* tickets = reinterpret_cast<int*>(partial256 + align_up((size_t)nb256 * D, 64));   // one per block of 256 columns (<= 8)
+  k_rmsnorm_bwd8<BF, true, RP><<<DET_L(nb8), RP * 128, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8, tickets);
   dim3 g2((D + 255) / 256, nb256);
-  k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256);
-  k_col_tree<<<DET_L((D + 127) / 128), 128, 0, st>>>(partial256, nb256, D, dgamma, rows);
+  k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256, nb256, tickets, dgamma);
   return DET_OK;
 }
 
