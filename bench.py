@@ -137,9 +137,7 @@ def accum_bytes_per_element(accum, shard, rep):
 
 
 def component_rates_configs_2_3(peaks, iters=5):
-    """The kernel-level workloads of the metric, timed one call at a time with CUDA events.  The reductions read
-    268 MB to 4.8 GB per call, more than twice L2, so nothing of one call is left for the next and L2 is not flushed
-    between their iterations (`l2` in each entry says so); the linear set is timed with L2 flushed between iterations:
+    """The kernel-level workloads of the metric, timed one call at a time (CUDA events, L2 flushed between iterations):
     the order-fixed reductions (RMSNorm forward/backward on 16384 x 2048 f32, cross-entropy forward/backward on
     4096 x 50304, global gradient norm over 1.2e9 f32) as GB/s and fraction of the measured copy bandwidth, and the
     1B-shaped linear set at 16384 tokens, forward and backward, as int8 POP/s and fraction of 4.5 POP/s nominal and of
@@ -152,10 +150,9 @@ def component_rates_configs_2_3(peaks, iters=5):
                      ("grad_norm_1.2e9", lambda: kbench.case_grad_norm(False))):
         call, work, _ = fn()
         torch.cuda.synchronize()
-        ms = kbench.timeit(call, iters, flush=False)
+        ms = kbench.timeit(call, iters)
         gbs = work / (ms / 1e3) / 1e9
-        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 3),
-                     "l2": "inputs larger than L2, no flush"}
+        out[name] = {"ms": round(ms, 4), "gbs": round(gbs, 1), "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 3)}
         del call
         torch.cuda.empty_cache()
     tot = {"fwd": [0.0, 0.0], "bwd": [0.0, 0.0]}

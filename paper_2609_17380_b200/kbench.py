@@ -1,7 +1,4 @@
-"""Per-kernel timing of libdet on one GPU: CUDA events around each C-ABI call; between iterations L2 is flushed (a
-256 MB buffer is written), except for the cases in STREAMING, whose inputs are more than twice the 126 MB of L2 and are
-read once per call, so that nothing of one call is left for the next (flushing by writing would instead leave up to
-126 MB of dirty lines whose write-back competes with the timed kernel).
+"""Per-kernel timing of libdet on one GPU: CUDA events around each C-ABI call, L2 flushed between iterations.
 
     python -m paper_2609_17380_b200.kbench [--case NAME ...] [--iters N] [--small] [--json]
 
@@ -29,17 +26,12 @@ def flush_l2():
     _flush.zero_()
 
 
-# full-size cases whose inputs exceed L2 more than twice over (RMSNorm 268 MB, cross-entropy 824 MB, 4.8 GB of gradients)
-STREAMING = {"rmsnorm_fwd", "rmsnorm_bwd", "xent_fwd", "xent_bwd", "grad_norm", "sumsq"}
-
-
-def timeit(fn, iters, warm=2, flush=True):
+def timeit(fn, iters, warm=2):
     for _ in range(warm):
         fn()
     ts = []
     for _ in range(iters):
-        if flush:
-            flush_l2()
+        flush_l2()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn()
@@ -255,8 +247,7 @@ def main():
     for name in names:
         fn, work, unit = cases[name](args.small)
         torch.cuda.synchronize()
-        ms = timeit(fn, args.iters, warm=1 if args.iters == 1 else 2,
-                    flush=not (args.no_flush or (name in STREAMING and not args.small)))
+        ms = timeit(fn, args.iters, warm=1 if args.iters == 1 else 2)
         rate = work / (ms / 1e3)
         res[name] = {"ms": round(ms, 4), "rate": rate / 1e9 if unit == "B" else rate / 1e12,
                      "unit": "GB/s" if unit == "B" else ("TOP/s" if unit == "op" else "TFLOP/s")}
