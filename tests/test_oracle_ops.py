@@ -279,6 +279,128 @@ def test_attention_forward_pins():
     assert np.allclose(lse3[0, 0], np.log(np.arange(1, S + 1)), atol=1e-5)
 
 
+def _qkv_rows(S, H=1):
+    return np.zeros((S, 3 * H * 128), np.uint16)
+
+
+def _bfrow(vals):
+    return synth.to_bf16(np.asarray(vals, F))
+
+
+def test_attention_logit_is_a_sequential_ascending_dot():
+    """One key, q = k = (4096, 1, 1, ..., 1): the products are 2^24, 1, ..., 1.  Added in ascending order every 1 is
+    lost against 2^24 (ties to even), so the logit is 2^24/sqrt(128); a pairwise tree or a descending sum collects the
+    127 ones first and gives (2^24 + 128)/sqrt(128).  With a single key the weight is 1, so lse is the logit itself."""
+    qkv = _qkv_rows(1)
+    r = _bfrow([4096.0] + [1.0] * 127)
+    qkv[0, :128] = r; qkv[0, 128:256] = r; qkv[0, 256:] = _bfrow(np.arange(128) - 60.0)
+    out, lse = oracle.attn_fwd(qkv, 1, 1, 1)
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    assert lse[0, 0, 0] == F(F(2.0 ** 24) * scale) and lse[0, 0, 0] != F(F(2.0 ** 24 + 128) * scale)
+    assert np.array_equal(out[0], qkv[0, 256:])
+    # the same for the backward's recomputed logit: dV_0 = bf16(P) dO with P = exp(s - lse) = exp(0) = 1
+    dout = _bfrow(np.linspace(-1, 1, 128)).reshape(1, 128)
+    d = oracle.attn_bwd(dout, qkv, out, lse, 1, 1, 1)
+    assert np.array_equal(d[0, 256:], dout[0])
+
+
+def test_attention_rounds_the_weights_to_bf16_for_pv_but_not_for_the_row_sum():
+    """Two keys seen by row 1, logits (s0, 0) through one-hot dimensions, v0 = 1, v1 = 0: the output is
+    bf16(p0) / (p0 + 1) with p0 = exp(s0) (the oracle's exp, pinned on its own), the division being a reciprocal and a
+    product in binary32, the result rounded to bf16.  Leaving out the rounding of p0, or summing the rounded weights,
+    gives another bf16 value for most of the arguments below."""
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    seen_unrounded = seen_roundsum = 0
+    for x0 in (-1.0, -3.0, -5.0, -7.0, -9.0, -11.0, -13.0, -19.0, -23.0, -29.0):
+        qkv = _qkv_rows(2)
+        qkv[1, 0] = _bfrow([1.0])[0]                      # q_1 = e_0
+        qkv[0, 128] = _bfrow([x0])[0]                     # k_0 = x0 e_0, k_1 = 0
+        qkv[0, 256:] = _bfrow(np.ones(128))               # v_0 = 1, v_1 = 0
+        out, lse = oracle.attn_fwd(qkv, 1, 1, 2)
+        s0 = F(F(x0) * scale)
+        p0 = oracle.prim("exp", np.array([s0], F))[0]
+        l = F(p0 + F(1.0))
+        il = F(F(1.0) / l)
+        pt = bf(synth.to_bf16(np.array([p0], F)))[0]
+        want = synth.to_bf16(np.array([F(pt * il)], F))[0]
+        assert np.all(out[1] == want), x0
+        assert lse[0, 0, 1] == F(F(0.0) + oracle.prim("log", np.array([l], F))[0])
+        seen_unrounded += synth.to_bf16(np.array([F(p0 * il)], F))[0] != want
+        seen_roundsum += synth.to_bf16(np.array([F(pt * F(F(1.0) / F(pt + F(1.0))))], F))[0] != want
+    assert seen_unrounded >= 2 and seen_roundsum >= 1     # the cases do tell the readings apart
+
+
+def test_attention_key_tile_is_128_and_earlier_tiles_are_rescaled():
+    """Row 128 sees keys 0..128 with logits s_A0 > s_A1 at keys 0 and 1, a dominant logit 0 at key B, and logits so low
+    everywhere else that their weights are exactly 0.  With B = 127 all three share the first tile:
+    l = (exp(s_A0) + exp(s_A1)) + 1.  With B = 128 the first tile is normalised by its own maximum s_A0 and rescaled when
+    the second tile arrives: l = (1 + exp(s_A1 - s_A0)) * exp(s_A0) + 1.  The two differ in the last bits, and a tile of
+    64 or of 256 keys would put the boundary elsewhere.  exp and log are the oracle's own (pinned separately)."""
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    ex = lambda x: oracle.prim("exp", np.array([x], F))[0]
+    lg = lambda x: oracle.prim("log", np.array([x], F))[0]
+    differ = 0
+    for xa0, xa1 in ((-8.0, -16.0), (-16.0, -17.0), (-15.75, -16.5), (-15.5, -16.0), (-15.25, -20.0), (-1.0, -2.0)):
+        sA0, sA1 = F(F(xa0) * scale), F(F(xa1) * scale)
+        got = {}
+        for Bk in (127, 128):
+            S = 129
+            qkv = _qkv_rows(S)
+            qkv[128, 0] = _bfrow([1.0])[0]                            # q_128 = e_0
+            qkv[:, 128] = _bfrow([-30000.0])[0]                       # every key far below ...
+            qkv[0, 128] = _bfrow([xa0])[0]; qkv[1, 128] = _bfrow([xa1])[0]
+            qkv[Bk, 128] = 0                                          # ... except A0, A1 and B
+            out, lse = oracle.attn_fwd(qkv, 1, 1, S)
+            got[Bk] = lse[0, 0, 128]
+        same_tile = F(F(ex(sA0) + ex(sA1)) + F(1.0))
+        two_tiles = F(F(F(F(1.0) + ex(F(sA1 - sA0))) * ex(F(sA0 - F(0.0)))) + F(1.0))
+        assert got[127] == F(F(0.0) + lg(same_tile)), (xa0, xa1)
+        assert got[128] == F(F(0.0) + lg(two_tiles)), (xa0, xa1)
+        differ += same_tile != two_tiles
+    assert differ >= 4
+
+
+def test_attention_value_gradient_sums_queries_in_ascending_order():
+    """Every row puts weight exactly 1 on key 0 (its logit is 0, every other logit is far below), so
+    dV_0 = sum_i dO_i in binary32, queries ascending from +0.  Column 0 of dO is (2^24, 1, ..., 1, -2^24): ascending, the
+    ones are lost and the total is 0; any other order keeps some of them.  Column 1 is (1, ..., 1, 2^24, -2^24): the 62
+    ones are exact before the large terms arrive, total 62.  Column 2 is (2^24, -2^24, 1, ..., 1): total 62 as well."""
+    S = 64
+    qkv = _qkv_rows(S)
+    qkv[:, 0] = _bfrow([1.0])[0]                                      # q_i = e_0
+    qkv[1:, 128] = _bfrow([-30000.0])[0]                              # k_0 = 0, the others far below
+    qkv[:, 256:] = synth.normal_bf16((S, 128), 1.0, seed=0, tid=68)
+    out, lse = oracle.attn_fwd(qkv, 1, 1, S)
+    assert np.all(lse == 0) and np.array_equal(out, np.tile(qkv[0, 256:], (S, 1)))
+    dO = np.zeros((S, 128), F)
+    dO[:, 0] = 1.0; dO[0, 0] = 2.0 ** 24; dO[S - 1, 0] = -2.0 ** 24
+    dO[:, 1] = 1.0; dO[S - 2, 1] = 2.0 ** 24; dO[S - 1, 1] = -2.0 ** 24
+    dO[:, 2] = 1.0; dO[0, 2] = 2.0 ** 24; dO[1, 2] = -2.0 ** 24
+    d = oracle.attn_bwd(synth.to_bf16(dO), qkv, out, lse, 1, 1, S)
+    dv0 = bf(d[0, 256:])
+    assert dv0[0] == 0.0 and dv0[1] == 62.0 and dv0[2] == 62.0 and np.all(dv0[3:] == 0.0)
+    assert np.all(bf(d[1:, 256:]) == 0.0)                             # no weight on the other keys
+
+
+def test_attention_backward_recomputes_the_weights_from_lse():
+    """Two keys, dO_0 = 0, dO_1 = e_c: dV_0 = bf16(P_10) in column c, with P_10 = exp(s_0 - lse_1) recomputed from the
+    stored logsumexp (not the forward's p / l) and rounded to bf16 once more by the output."""
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    for x0 in (-2.0, -5.0, -9.0, 3.0):
+        qkv = _qkv_rows(2)
+        qkv[1, 0] = _bfrow([1.0])[0]
+        qkv[0, 128] = _bfrow([x0])[0]
+        qkv[:, 256:] = synth.normal_bf16((2, 128), 1.0, seed=0, tid=69)
+        out, lse = oracle.attn_fwd(qkv, 1, 1, 2)
+        dO = np.zeros((2, 128), F); dO[1, 5] = 1.0
+        d = oracle.attn_bwd(synth.to_bf16(dO), qkv, out, lse, 1, 1, 2)
+        s0 = F(F(x0) * scale)
+        P10 = oracle.prim("exp", np.array([F(s0 - lse[0, 0, 1])], F))[0]
+        assert d[0, 256 + 5] == synth.to_bf16(np.array([P10], F))[0], x0
+        P11 = oracle.prim("exp", np.array([F(F(0.0) - lse[0, 0, 1])], F))[0]
+        assert d[1, 256 + 5] == synth.to_bf16(np.array([P11], F))[0], x0
+
+
 def test_attention_backward_against_float64():
     B, H, S = 2, 1, 160
     qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=62)
