@@ -435,16 +435,17 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
   const float* z = logits + (size_t)blockIdx.x * V;
   float m = __int_as_float(0xff800000);
   {
+    auto ld4 = [&](const float* p) { return *reinterpret_cast<const float4*>(p); };
     int i = threadIdx.x * 4;
     for (; i + 3 * XT * 4 < V; i += 4 * XT * 4) {      // four loads in flight per thread
       float4 a[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) a[u] = *reinterpret_cast<const float4*>(z + i + u * XT * 4);
+      for (int u = 0; u < 4; ++u) a[u] = ld4(z + i + u * XT * 4);
 #pragma unroll
       for (int u = 0; u < 4; ++u) m = fmaxf(fmaxf(m, fmaxf(a[u].x, a[u].y)), fmaxf(a[u].z, a[u].w));
     }
     for (; i < V; i += XT * 4) {
-      float4 a = *reinterpret_cast<const float4*>(z + i);
+      float4 a = ld4(z + i);
       m = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
     }
   }
@@ -460,7 +461,9 @@ __global__ void __launch_bounds__(XT) k_xent_fwd(const float* __restrict__ logit
   const int nfull = V >> 8;  // leaves that lie wholly inside the row: no existence tests in their tree
   for (int leaf = warp; leaf < nfull; leaf += XT / 32) {
     const int e0 = leaf * 256 + lane * 8;
-    const float4 a0 = *reinterpret_cast<const float4*>(z + e0), a1 = *reinterpret_cast<const float4*>(z + e0 + 4);
+    // second and last read of the row: streaming loads, so that these lines leave L2 before the rows still waiting
+    // between their two sweeps (the rows in flight on all SMs together fill most of L2)
+    const float4 a0 = __ldcs(reinterpret_cast<const float4*>(z + e0)), a1 = __ldcs(reinterpret_cast<const float4*>(z + e0 + 4));
     float e[8];
     e[0] = det_exp_le0(fsub(a0.x, m)); e[1] = det_exp_le0(fsub(a0.y, m));          // branch-free: the chains interleave
     e[2] = det_exp_le0(fsub(a0.z, m)); e[3] = det_exp_le0(fsub(a0.w, m));
