@@ -22,7 +22,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-typedef uint16_t bf16_t;
+#include "prim.h" /* the version-1 primitives that version 2 keeps: binary32 operations with flushing, det_sum, det_exp, det_log */
 
 /* row exponent; *bad is set when the row holds an infinity or a NaN */
 static int row_exponent(const bf16_t *x, int K, int *bad) {
@@ -101,4 +101,83 @@ void orc2_lmhead_fwd(const bf16_t *H, const bf16_t *W, int M, int V, int K, floa
       logits[(size_t)m * V + n] = round_scaled(I, Ea[m] + Eb[n] - 280);
     }
   free(Ta); free(Tb); free(Ea); free(Eb); free(Ba); free(Bb);
+}
+
+/* ------------------------------------------------------------------------------------------------------------------
+ * Causal attention in arithmetic version 2 (head dimension 128, one key/value head per query head, no window).
+ *
+ * Version 1 defines the logits, P.V and the online rescaling as ordered chains of binary32 roundings.  Version 2 keeps the
+ * softmax arithmetic of version 1 (binary32, det_exp, det_sum, det_log) and replaces the two contractions by the
+ * order-free contraction defined at the top of this file; with no order to respect there are no key tiles and no
+ * rescaling: a row takes its maximum over all of its keys first.
+ *
+ *   s_ij  = fmul(C(q_i, k_j), 2^-3.5 rounded to binary32)        j <= i; C = the version-2 contraction over the 128 dimensions,
+ *                                                                row exponents over the 128 values of q_i and of k_j
+ *   m_i   = max_j s_ij,  p_ij = det_exp(s_ij - m_i),  l_i = det_sum(p_i0 .. p_ii),  lse_i = m_i + det_log(l_i)
+ *   P~_ij = bf16(p_ij)                                            (as in version 1; 0 for j > i)
+ *   u_ic  = C(P~_i., v_.c) over the keys 0 .. i                   exponent of row i of P~ over its keys, exponent of column c
+ *                                                                of v over ALL keys of the sequence (so that it is shared
+ *                                                                by every query)
+ *   o_ic  = bf16(fmul(u_ic, fdiv(1, l_i)))
+ * ------------------------------------------------------------------------------------------------------------------ */
+#define A2_SCALE 0x1.6a09e6p-4f /* 1/sqrt(128) rounded to binary32 */
+
+/* exponent over n values spaced `stride` apart; *bad as in row_exponent */
+static int strided_exponent(const bf16_t *x, size_t stride, int n, int *bad) {
+  int e = 0;
+  *bad = 0;
+  for (int k = 0; k < n; ++k) {
+    int ek = (x[(size_t)k * stride] >> 7) & 0xFF;
+    if (ek == 255) *bad = 1;
+    if (ek > e) e = ek;
+  }
+  return e;
+}
+/* the version-2 contraction of n values of a (stride sa, exponent ea) with n values of b (stride sb, exponent eb) */
+static float contract2(const bf16_t *a, size_t sa, int ea, const bf16_t *b, size_t sb, int eb, int n) {
+  int64_t I = 0;
+  for (int k = 0; k < n; ++k) I += (int64_t)aligned(a[(size_t)k * sa], ea) * (int64_t)aligned(b[(size_t)k * sb], eb);
+  return round_scaled(I, ea + eb - 280);
+}
+static float quiet_nan(void) { uint32_t q = 0x7FC00000u; float f; memcpy(&f, &q, 4); return f; }
+
+void orc2_attn_fwd(const bf16_t *q, const bf16_t *k, const bf16_t *v, int ld, int B, int H, int S, bf16_t *out, int ld_out,
+                   float *lse) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int bh = 0; bh < B * H; ++bh) {
+    const int b = bh / H, h = bh % H;
+    const bf16_t *qb = q + (size_t)ld * b * S + h * 128, *kb = k + (size_t)ld * b * S + h * 128;
+    const bf16_t *vb = v + (size_t)ld * b * S + h * 128;
+    int *Eq = (int *)malloc(S * sizeof(int)), *Ek = (int *)malloc(S * sizeof(int));
+    int *Bq = (int *)malloc(S * sizeof(int)), *Bk = (int *)malloc(S * sizeof(int));
+    int Ev[128], Bv[128];
+    for (int i = 0; i < S; ++i) {
+      Eq[i] = row_exponent(qb + (size_t)ld * i, 128, &Bq[i]);
+      Ek[i] = row_exponent(kb + (size_t)ld * i, 128, &Bk[i]);
+    }
+    for (int c = 0; c < 128; ++c) Ev[c] = strided_exponent(vb + c, (size_t)ld, S, &Bv[c]);
+    float *s = (float *)malloc(S * sizeof(float)), *p = (float *)malloc(S * sizeof(float));
+    bf16_t *pt = (bf16_t *)malloc(S * sizeof(bf16_t));
+    for (int i = 0; i < S; ++i) {
+      float m = -INFINITY;
+      for (int j = 0; j <= i; ++j) {
+        float c = (Bq[i] || Bk[j]) ? quiet_nan() : contract2(qb + (size_t)ld * i, 1, Eq[i], kb + (size_t)ld * j, 1, Ek[j], 128);
+        s[j] = fmul(c, A2_SCALE);
+        m = fmax2(m, s[j]);
+      }
+      for (int j = 0; j <= i; ++j) {
+        p[j] = det_exp(fsub(s[j], m));
+        pt[j] = f2bf(p[j]);
+      }
+      float l = det_sum(p, (size_t)i + 1);
+      int bp, ep = row_exponent(pt, i + 1, &bp);
+      float il = fdiv(1.0f, l);
+      for (int c = 0; c < 128; ++c) {
+        float u = (bp || Bv[c]) ? quiet_nan() : contract2(pt, 1, ep, vb + c, (size_t)ld, Ev[c], i + 1);
+        out[(size_t)ld_out * (b * S + i) + h * 128 + c] = f2bf(fmul(u, il));
+      }
+      lse[(size_t)bh * S + i] = fadd(m, det_log(l));
+    }
+    free(Eq); free(Ek); free(Bq); free(Bk); free(s); free(p); free(pt);
+  }
 }

@@ -13,11 +13,12 @@ import numpy as np
 _DIR = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_DIR, "liboracle_v2.so")
 _SRC = os.path.join(_DIR, "v2.c")
+_HDR = os.path.join(_DIR, "prim.h")
 _lib = None
 
 
 def build(force=False):
-    if not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC):
+    if not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)):
         return _SO
     subprocess.check_call(["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-msse4.1", "-fopenmp", "-shared", "-fPIC", "-o", _SO,
                            _SRC, "-lm"])
@@ -55,6 +56,21 @@ def lmhead_fwd(Hh, W):
     out = np.empty((M, V), np.float32)
     lib().orc2_lmhead_fwd(_p(Hh), _p(W), C.c_int(M), C.c_int(V), C.c_int(K), _p(out))
     return out
+
+
+def attn_fwd(qkv, B, H, S):
+    """Causal attention in arithmetic version 2 (see v2.c).  qkv: uint16 [B*S, 3*H*128] (q | k | v column blocks).
+    Returns out bf16 [B*S, H*128] and lse f32 [B,H,S]."""
+    qkv = np.ascontiguousarray(qkv, dtype=np.uint16)
+    ld = qkv.shape[1]
+    assert qkv.shape[0] == B * S and ld == 3 * H * 128
+    out = np.empty((B * S, H * 128), np.uint16)
+    lse = np.empty((B, H, S), np.float32)
+    flat = qkv.reshape(-1)
+    q, k, v = flat[0:], flat[H * 128:], flat[2 * H * 128:]
+    lib().orc2_attn_fwd(_p(q), C.c_void_p(q.ctypes.data + 2 * H * 128), C.c_void_p(q.ctypes.data + 4 * H * 128), C.c_int(ld),
+                        C.c_int(B), C.c_int(H), C.c_int(S), _p(out), C.c_int(H * 128), _p(lse))
+    return out, lse
 
 
 def _f2bf(x):

@@ -157,3 +157,87 @@ def test_backward_is_the_contraction_on_transposed_operands_and_close_to_float64
     for (v, k) in ((0, 0), (11, 3), (39, 31)):
         want = _brute(np.ascontiguousarray(v2._f2bf(dl)[:, v]), np.ascontiguousarray(Hh[:, k]))
         assert dW[v, k].view(np.uint32) == F(want).view(np.uint32)
+
+
+# ---------------------------------------------------------------- attention in version 2
+def _qkv(S, H=1):
+    return np.zeros((S, 3 * H * 128), np.uint16)
+
+
+def test_attention_v2_uniform_weights_are_exact():
+    """q = 0: every logit is 0, every weight exactly 1, l_i = i + 1 exactly, and u is the exact integer sum of small
+    integer values (nothing is truncated: all within 2^-6 of the column's largest), so the output is
+    bf16(fmul(sum_{j<=i} v_jc, fdiv(1, i + 1))) and lse_i = log(i + 1) by the oracle's own log."""
+    import oracle
+    S = 70
+    rng = np.random.default_rng(3)
+    qkv = _qkv(S)
+    vals = rng.integers(-3, 4, (S, 128)).astype(F)
+    vals[0] = 3.0                                            # every column's largest magnitude is 3: exponent 128
+    qkv[:, 128:256] = synth.to_bf16(rng.standard_normal((S, 128)).astype(F))     # keys do not matter when q = 0
+    qkv[:, 256:] = synth.to_bf16(vals)
+    out, lse = v2.attn_fwd(qkv, 1, 1, S)
+    csum = np.cumsum(vals.astype(np.int64), 0)
+    for i in (0, 1, 2, 31, 63, 69):
+        il = F(F(1.0) / F(i + 1))
+        want = synth.to_bf16((csum[i].astype(F) * il).astype(F))
+        assert np.array_equal(out[i], want), i
+        assert lse[0, 0, i] == F(F(0.0) + oracle.prim("log", np.array([F(i + 1)], F))[0])
+
+
+def test_attention_v2_logits_are_the_v2_contraction():
+    """One query against itself and one earlier key (S = 2): lse_0 is the logit s_00 itself, and the pair of rows goes
+    through the brute-force restatement of the contraction (exact rational arithmetic from the values)."""
+    rng = np.random.default_rng(5)
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    for t in range(4):
+        qkv = _qkv(1)
+        qkv[0, :128] = synth.to_bf16((rng.standard_normal(128) * np.exp2(rng.integers(-8, 3, 128))).astype(F))
+        qkv[0, 128:256] = synth.to_bf16((rng.standard_normal(128) * np.exp2(rng.integers(-8, 3, 128))).astype(F))
+        qkv[0, 256:] = synth.to_bf16(rng.standard_normal(128).astype(F))
+        out, lse = v2.attn_fwd(qkv, 1, 1, 1)
+        want = F(_brute(qkv[0, :128], qkv[0, 128:256]) * scale)
+        assert lse[0, 0, 0] == want
+        # a single key: weight 1, u = the value aligned to its own exponent (exact), l = 1
+        assert np.array_equal(out[0], qkv[0, 256:])
+
+
+def test_attention_v2_is_causal_and_close_to_float64():
+    import math
+    B, H, S = 1, 2, 200
+    qkv = synth.normal_bf16((B * S, 3 * H * 128), 1.0, seed=0, tid=60)
+    out, lse = v2.attn_fwd(qkv, B, H, S)
+    x = synth.from_bf16(qkv).astype(np.float64).reshape(B, S, 3, H, 128)
+    q, k, v = (x[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+    s = q @ k.transpose(0, 1, 3, 2) / math.sqrt(128)
+    s = np.where(np.tril(np.ones((S, S), bool)), s, -np.inf)
+    l64 = np.log(np.exp(s - s.max(-1, keepdims=True)).sum(-1)) + s.max(-1)
+    o64 = (np.exp(s - l64[..., None]) @ v).transpose(0, 2, 1, 3).reshape(B * S, H * 128)
+    # truncation of the aligned values costs at most 2^-13 of the largest product per term; bf16 rounding of the weights and
+    # of the output dominates
+    assert np.abs(synth.from_bf16(out) - o64).max() < 0.02 and np.allclose(lse, l64, rtol=2e-4, atol=2e-4)
+    # causality: later keys and values leave earlier rows bit-identical -- EXCEPT through the exponent of a value column,
+    # which is taken over all keys of the sequence: keep the columns' largest magnitudes where they are
+    qkv2 = qkv.copy()
+    tail = synth.normal_bf16((S - 150, 2 * H * 128), 0.25, seed=1, tid=61)
+    qkv2[150:, H * 128:] = tail
+    e_before = ((qkv[:, 2 * H * 128:] >> 7) & 0xFF).max(0)
+    e_after = ((qkv2[:, 2 * H * 128:] >> 7) & 0xFF).max(0)
+    assert np.array_equal(e_before, e_after)                 # the recipe above keeps every column exponent
+    out2, lse2 = v2.attn_fwd(qkv2, B, H, S)
+    assert np.array_equal(out2[:150], out[:150]) and np.array_equal(lse2[:, :, :150], lse[:, :, :150])
+
+
+def test_attention_v2_does_not_depend_on_the_order_of_the_head_dimensions():
+    """The contraction over the 128 dimensions is order-free: permuting the dimensions of q and k together leaves every
+    logit, hence lse and the output, bit-identical (version 1's ordered dot does not have this property)."""
+    B, H, S = 1, 1, 96
+    rng = np.random.default_rng(11)
+    qkv = synth.to_bf16((rng.standard_normal((S, 384)) * np.exp2(rng.integers(-6, 3, (S, 384)))).astype(F))
+    out, lse = v2.attn_fwd(qkv, B, H, S)
+    perm = rng.permutation(128)
+    qkv2 = qkv.copy()
+    qkv2[:, :128] = qkv[:, :128][:, perm]
+    qkv2[:, 128:256] = qkv[:, 128:256][:, perm]
+    out2, lse2 = v2.attn_fwd(qkv2, B, H, S)
+    assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
