@@ -267,6 +267,21 @@ size_t det_lmhead_bwd_v2_ws_bytes(int M, int V, int K);
 int det_lmhead_bwd_v2(const float* dlogits, const det_bf16* H, const det_bf16* W, int M, int V, int K, det_bf16* dH, float* dW,
                       void* ws, size_t ws_bytes, void* stream, int* status_dev);
 
+/* Causal attention in arithmetic version 2 (optional mode; head dimension 128, one key/value head per query head, no
+ * window): the two contractions of the forward pass become the order-free contraction of det_lmhead_fwd_v2 (Sec. 3.2:
+ * exact integer products and a wide exact total "for bitwise reproducibility"), the softmax keeps the binary32
+ * arithmetic of det_attn_fwd.  With no order to respect there are no key tiles and no rescaling:
+ *   s_ij = fmul(C(q_i, k_j), 1/sqrt(128) in binary32), C over the 128 dimensions with the exponents of the two rows;
+ *   m_i = max_j s_ij, p_ij = det_exp(s_ij - m_i), l_i = det_sum(p_i0 .. p_ii), lse_i = m_i + det_log(l_i);
+ *   u_ic = C(bf16(p_i.), v_.c) over the keys 0 .. i, the exponent of a row of weights over its keys and the exponent of a
+ *   column of v over ALL keys of its sequence; out_ic = bf16(fmul(u_ic, fdiv(1, l_i))).
+ * q, k, v, out, lse laid out as for det_attn_fwd.  S % 128 == 0, S <= 8192, ld % 8 == 0.  ws: det_attn_fwd_v2_ws_bytes
+ * (slices, exponents, the f32 logits [B*H, S, S] and the sliced weights: about 6 B H S^2 bytes).  status_dev (device
+ * int, may be NULL) receives DET_DEV_TIMEOUT if a bounded wait of the tensor-core kernels expires. */
+size_t det_attn_fwd_v2_ws_bytes(int B, int H, int S);
+int det_attn_fwd_v2(const det_bf16* q, const det_bf16* k, const det_bf16* v, int ld, int B, int H, int S, det_bf16* out,
+                    int ld_out, float* lse, void* ws, size_t ws_bytes, void* stream, int* status_dev);
+
 /* ---- gradient accumulation = single-device replay of the data-parallel reduction
  *      (Sec. 6, Algorithm 1; Appendix A, Algorithm 2 "TreeFold"; A.3 reciprocal-multiply averages) -------
  * The state is a caller-owned POD; bufs holds det_grad_accum_nbufs(dp_replicate) * n floats on the device. */

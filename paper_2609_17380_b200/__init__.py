@@ -53,7 +53,8 @@ def load():
         for name in ("det_sum_ws_bytes", "det_grad_norm_ws_bytes", "det_lsq_weight_scale_ws_bytes",
                      "det_lsq_act_scale_init_ws_bytes", "det_lsq_quantize_weight_ws_bytes", "det_linear_bwd_ws_bytes",
                      "det_rmsnorm_bwd_ws_bytes", "det_xent_ws_bytes", "det_attn_bwd_ws_bytes", "det_attn_bwd_fixq_ws_bytes",
-                     "det_tensor_hash_ws_bytes", "det_lmhead_fwd_v2_ws_bytes", "det_lmhead_bwd_v2_ws_bytes"):
+                     "det_tensor_hash_ws_bytes", "det_lmhead_fwd_v2_ws_bytes", "det_lmhead_bwd_v2_ws_bytes",
+                     "det_attn_fwd_v2_ws_bytes"):
             getattr(_lib, name).restype = C.c_size_t
         _lib.det_launch_count.restype = C.c_ulonglong
     return _lib
@@ -328,6 +329,15 @@ def det_lmhead_bwd_v2_ws_bytes(M, V, K):
 def det_lmhead_bwd_v2(dlogits, H, W, M, V, K, dH, dW, ws, status_dev=None):
     _check("det_lmhead_bwd_v2", load().det_lmhead_bwd_v2(_ptr(dlogits), _ptr(H), _ptr(W), C.c_int(M), C.c_int(V), C.c_int(K),
                                                          _ptr(dH), _ptr(dW), *_ws(ws), _stream(), _ptr(status_dev)))
+
+
+def det_attn_fwd_v2_ws_bytes(B, H, S):
+    return load().det_attn_fwd_v2_ws_bytes(C.c_int(B), C.c_int(H), C.c_int(S))
+
+
+def det_attn_fwd_v2(q, k, v, ld, B, H, S, out, ld_out, lse, ws, status_dev=None):
+    _check("det_attn_fwd_v2", load().det_attn_fwd_v2(_ptr(q), _ptr(k), _ptr(v), C.c_int(ld), C.c_int(B), C.c_int(H), C.c_int(S),
+                                                     _ptr(out), C.c_int(ld_out), _ptr(lse), *_ws(ws), _stream(), _ptr(status_dev)))
 
 
 def det_lmhead_bwd(dlogits, H, W, M, V, K, dH, dW, first_chunk):

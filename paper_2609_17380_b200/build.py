@@ -10,8 +10,8 @@ from concurrent.futures import ThreadPoolExecutor
 _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
 OUT = os.path.join(_DIR, "libdet.so")
-SOURCES = ["reduce.cu", "norm_loss.cu", "glue_optim.cu", "igemm.cu", "lsq.cu", "ogemm.cu", "attn.cu", "attn_pv8.cu", "headops.cu", "sum_static.cu", "lmhead_v2.cu"]
-HEADERS = ["common.cuh", "internal.h", "ogemm_core.cuh", "tc05.cuh", os.path.join("..", "..", "include", "det.h"),
+SOURCES = ["reduce.cu", "norm_loss.cu", "glue_optim.cu", "igemm.cu", "lsq.cu", "ogemm.cu", "attn.cu", "attn_pv8.cu", "headops.cu", "sum_static.cu", "lmhead_v2.cu", "attn_v2.cu"]
+HEADERS = ["common.cuh", "internal.h", "ogemm_core.cuh", "tc05.cuh", "v2_slice.cuh", os.path.join("..", "..", "include", "det.h"),
            os.path.join("..", "..", "include", "det_test.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",
               "-ftz=true", "-prec-div=true", "-prec-sqrt=true", "-Xcompiler", "-fPIC"]

@@ -60,4 +60,22 @@ int dev_sm_count();                                                 // SMs of th
 // force_one_cta != 0 keeps the one-CTA kernel even where the two-CTA tiles would apply (the results are identical)
 int igemm_launch(int epi, const int8_t* A, const int8_t* B, int I, int J, int K, const EpiParams& ep, int* status,
                  cudaStream_t st, int force_one_cta = 0);
+
+// Sliced (arithmetic version 2) contractions: out = round(I 2^(Ea + Eb - 280)) from the int8 slices of both operands,
+// Z problems per launch (lmhead_v2.cu).
+enum { SL_F32 = 0, SL_BF16 = 1, SL_BF16_ROWSCALE = 2 };
+struct SlArgs {
+  const int32_t* Ea;       // [Z*I] row exponents of A (bit 30: non-finite row)
+  const int32_t* Eb;       // [Z*J]
+  void* out;               // f32 or bf16, element (z, i, j) at (z / hdiv) * o_b + (z % hdiv) * o_h + i * ldo + j
+  const float* rowscale;   // [Z*I], SL_BF16_ROWSCALE only
+  int I, J, K, Z, hdiv;
+  long long o_b, o_h;
+  int ldo;
+  int causal_tiles;        // only tiles with j0 <= i0
+  int krange;              // 0 all steps, 1 steps <= the row tile's, 2 steps >= the row tile's
+  int epi;
+};
+int sliced_gemm_launch(const int8_t* Ah, const int8_t* Al, const int8_t* Bh, const int8_t* Bl, const SlArgs& p, int* status,
+                       cudaStream_t st);
 }  // namespace det

@@ -15,22 +15,11 @@
 // Every mbarrier wait is bounded (DET_DEV_TIMEOUT), as in igemm.cu.
 #include "tc05.cuh"
 #include "internal.h"
+#include "v2_slice.cuh"
 
 namespace det {
 
-// ---- slicing ----------------------------------------------------------------------------------------------------------
-// bf16 bit pattern of a binary32 value (subnormal inputs flushed first), as the gradient of the logits is rounded
-__device__ __forceinline__ uint32_t bf_bits(float x) {
-  if (!(__float_as_uint(x) & 0x7f800000u)) x = __uint_as_float(__float_as_uint(x) & 0x80000000u);
-  return (uint32_t)f2bf(x);
-}
-// signed 14-bit aligned value of one bf16 pattern against the exponent e of its row, as two int8 slices
-__device__ __forceinline__ void slice1(uint32_t b, int e, int& h, int& l) {
-  const int ek = (b >> 7) & 0xFF, d = e - ek;
-  const int t = (ek == 0 || d >= 14) ? 0 : (int)(((128u + (b & 0x7Fu)) << 6) >> d);
-  h = t >> 7; l = t & 127;
-  if (b & 0x8000u) { h = -h; l = -l; }
-}
+// ---- slicing (bf_bits, slice1: v2_slice.cuh) ------------------------------------------------------------------------------
 // eight values of a row as four words of packed bf16 patterns: bf16 source as stored, f32 source rounded to bf16
 template <bool F32>
 __device__ __forceinline__ void load8_bits(const void* X, size_t idx, uint32_t (&w)[4]) {
@@ -151,11 +140,17 @@ __device__ __forceinline__ float round_scaled(long long I, int e) {
   return r;
 }
 
-template <bool OUT_BF16>
+// One launch covers Z independent problems of the same shape (the operands of problem z are rows z*I.. of A and z*J.. of
+// B; the result goes to out + (z / hdiv) * o_b + (z % hdiv) * o_h + i * ldo + j).  causal_tiles: only the tiles with
+// j0 <= i0 exist.  krange: 0 the whole contraction; 1 only the steps up to and including the row tile's own (a causal
+// product whose contracted index is the key); 2 only the steps from the row tile's own on (contracted index = query).
+// epi: SL_F32 | SL_BF16 | SL_BF16_ROWSCALE (the rounded result times rowscale[z*I + i] in binary32, then bf16).
 __global__ void __launch_bounds__(SL_THREADS, 1)
     k_igemm_sl(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
-               const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const int32_t* __restrict__ Ea,
-               const int32_t* __restrict__ Eb, void* __restrict__ out, int I, int J, int K, int* status) {
+               const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const SlArgs p, int* status) {
+  const int32_t* __restrict__ Ea = p.Ea;
+  const int32_t* __restrict__ Eb = p.Eb;
+  const int I = p.I, J = p.J, K = p.K;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ __align__(8) uint64_t bar_full[SL_STAGES], bar_empty[SL_STAGES], bar_tfull, bar_tempty;
@@ -179,7 +174,17 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  const int tiles_i = I / SL_T, tiles_j = J / SL_T, num_tiles = tiles_i * tiles_j, kblocks = K / SL_BK;
+  const int tiles_i = I / SL_T, tiles_j = J / SL_T, per_z = tiles_i * tiles_j, num_tiles = p.Z * per_z, kblocks = K / SL_BK;
+  // tile t -> problem z, row tile it, column tile jt (the rows run fastest: the CTAs resident at one time share a tile of
+  // B and stream A through L2); false when the tile does not exist; [k_lo, k_hi) = its steps along the contraction
+  auto tile_of = [&](int t, int& z, int& i0, int& j0, int& k_lo, int& k_hi) {
+    z = t / per_z;
+    const int r = t - z * per_z, it = r % tiles_i, jt = r / tiles_i;
+    i0 = it * SL_T; j0 = jt * SL_T;
+    k_lo = (p.krange == 2) ? it : 0;
+    k_hi = (p.krange == 1) ? min(kblocks, it + 1) : kblocks;
+    return !(p.causal_tiles && jt > it);
+  };
 
   if (warp == 0) {
     if (lane == 0) {
@@ -187,16 +192,16 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        // the rows of H run fastest: the CTAs resident at one time share a tile of W and stream H through L2
-        const int i0 = (tile % tiles_i) * SL_T, j0 = (tile / tiles_i) * SL_T;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        int z, i0, j0, k_lo, k_hi;
+        if (!tile_of(tile, z, i0, j0, k_lo, k_hi)) continue;
+        for (int kb = k_lo; kb < k_hi; ++kb) {
           if (!mbar_wait(&bar_empty[stage], phase ^ 1u, abort_flag, status)) { ok = false; break; }
           mbar_expect_tx(&bar_full[stage], SL_STAGE_BYTES);
           uint8_t* sa = smem + stage * SL_STAGE_BYTES;
-          tma_load_2d(sa, &tmAh, kb * SL_BK, i0, &bar_full[stage]);
-          tma_load_2d(sa + SL_TILE, &tmAl, kb * SL_BK, i0, &bar_full[stage]);
-          tma_load_2d(sa + 2 * SL_TILE, &tmBh, kb * SL_BK, j0, &bar_full[stage]);
-          tma_load_2d(sa + 3 * SL_TILE, &tmBl, kb * SL_BK, j0, &bar_full[stage]);
+          tma_load_2d(sa, &tmAh, kb * SL_BK, z * I + i0, &bar_full[stage]);
+          tma_load_2d(sa + SL_TILE, &tmAl, kb * SL_BK, z * I + i0, &bar_full[stage]);
+          tma_load_2d(sa + 2 * SL_TILE, &tmBh, kb * SL_BK, z * J + j0, &bar_full[stage]);
+          tma_load_2d(sa + 3 * SL_TILE, &tmBl, kb * SL_BK, z * J + j0, &bar_full[stage]);
           if (++stage == SL_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -208,10 +213,13 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       int stage = 0, it = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int z, i0, j0, k_lo, k_hi;
+        if (!tile_of(tile, z, i0, j0, k_lo, k_hi)) continue;
         if (!mbar_wait(&bar_tempty, ((uint32_t)it & 1u) ^ 1u, abort_flag, status)) { ok = false; break; }   // accumulators drained
+        ++it;
         tc_fence_after();
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = k_lo; kb < k_hi; ++kb) {
           if (!mbar_wait(&bar_full[stage], phase, abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * SL_STAGE_BYTES);
@@ -220,7 +228,7 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
 #pragma unroll
           for (int k4 = 0; k4 < SL_BK / 32; ++k4) {
             const uint64_t o = (uint64_t)(k4 * 2);
-            const uint32_t first = (kb | k4) ? 1u : 0u;
+            const uint32_t first = (kb != k_lo || k4) ? 1u : 0u;
             umma_i8(tmem_base, ah + o, bh + o, idesc, first);              // hh
             umma_i8(tmem_base + 128u, ah + o, bl + o, idesc, first);       // hl starts the cross accumulator ...
             umma_i8(tmem_base + 128u, al + o, bh + o, idesc, 1u);          // ... lh adds to it
@@ -236,15 +244,20 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-      const int i0 = (tile % tiles_i) * SL_T, j0 = (tile / tiles_i) * SL_T;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      int z, i0, j0, k_lo, k_hi;
+      if (!tile_of(tile, z, i0, j0, k_lo, k_hi)) continue;
       if (!mbar_wait(&bar_tfull, (uint32_t)it & 1u, abort_flag, status)) { ok = false; break; }
+      ++it;
       tc_fence_after();
       const int row = i0 + q * 32 + lane;
-      const int ea = Ea[row];
+      const int ea = Ea[(size_t)z * I + row];
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-      float* orow = reinterpret_cast<float*>(out) + (size_t)row * J + j0;
-      uint16_t* brow = reinterpret_cast<uint16_t*>(out) + (size_t)row * J + j0;
+      const size_t obase = (size_t)(z / p.hdiv) * p.o_b + (size_t)(z % p.hdiv) * p.o_h + (size_t)row * p.ldo + j0;
+      float* orow = reinterpret_cast<float*>(p.out) + obase;
+      uint16_t* brow = reinterpret_cast<uint16_t*>(p.out) + obase;
+      const float rsc = (p.epi == SL_BF16_ROWSCALE) ? p.rowscale[(size_t)z * I + row] : 1.0f;
+      const int32_t* Ebz = Eb + (size_t)z * J;
 #pragma unroll 1
       for (int c0 = 0; c0 < SL_T; c0 += 32) {
         uint32_t hh[32], cr[32], ll[32];
@@ -257,11 +270,15 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
             const int c = 4 * v + x;
-            const int eb = __ldg(Eb + j0 + c0 + c);
+            const int eb = __ldg(Ebz + j0 + c0 + c);
             const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
             f[x] = ((ea | eb) >> 30) ? __int_as_float(0x7FC00000) : round_scaled(Iv, (ea & 0xFF) + (eb & 0xFF) - 280);
           }
-          if (OUT_BF16) *reinterpret_cast<uint2*>(brow + c0 + 4 * v) = make_uint2(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]));
+          if (p.epi == SL_BF16_ROWSCALE) {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) f[x] = fmul(f[x], rsc);
+          }
+          if (p.epi != SL_F32) *reinterpret_cast<uint2*>(brow + c0 + 4 * v) = make_uint2(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]));
           else *reinterpret_cast<float4*>(orow + c0 + 4 * v) = make_float4(f[0], f[1], f[2], f[3]);
         }
       }
@@ -282,6 +299,25 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
   }
 }
 
+// host: Z sliced contractions in one launch (see k_igemm_sl); the slices of problem z are rows z*I.. / z*J.. of A / B
+int sliced_gemm_launch(const int8_t* Ah, const int8_t* Al, const int8_t* Bh, const int8_t* Bl, const SlArgs& p, int* status,
+                       cudaStream_t st) {
+  if (p.I % SL_T || p.J % SL_T || p.K % SL_BK || p.Z <= 0 || p.hdiv <= 0) return DET_ERR_SHAPE;
+  if (p.K >= (1 << 16)) return DET_ERR_RANGE;   // the cross accumulator holds two products: 2 K 127^2 must stay below 2^31
+  CUtensorMap tAh, tAl, tBh, tBl;
+  if (!make_map(&tAh, Ah, p.Z * p.I, p.K, SL_T) || !make_map(&tAl, Al, p.Z * p.I, p.K, SL_T) ||
+      !make_map(&tBh, Bh, p.Z * p.J, p.K, SL_T) || !make_map(&tBl, Bl, p.Z * p.J, p.K, SL_T))
+    return DET_ERR_CUDA;
+  static DevOnce once = {};
+  if (dev_ensure_smem(once, (const void*)k_igemm_sl, SL_SMEM) != DET_OK) return DET_ERR_CUDA;
+  const int sms = dev_sm_count();
+  if (sms <= 0) return DET_ERR_CUDA;
+  const long long tiles = (long long)p.Z * (p.I / SL_T) * (p.J / SL_T);
+  k_igemm_sl<<<DET_L((unsigned)(tiles < sms ? tiles : sms)), SL_THREADS, SL_SMEM, st>>>(tAh, tAl, tBh, tBl, p, status);
+  if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
+  return DET_OK;
+}
+
 }  // namespace det
 
 using namespace det;
@@ -290,18 +326,11 @@ using namespace det;
 template <bool OUT_BF16>
 static int sliced_gemm(const int8_t* Ah, const int8_t* Al, const int8_t* Bh, const int8_t* Bl, const int32_t* Ea, const int32_t* Eb,
                        void* out, int I, int J, int K, int* status, cudaStream_t st) {
-  CUtensorMap tAh, tAl, tBh, tBl;
-  if (!make_map(&tAh, Ah, I, K, SL_T) || !make_map(&tAl, Al, I, K, SL_T) || !make_map(&tBh, Bh, J, K, SL_T) ||
-      !make_map(&tBl, Bl, J, K, SL_T))
-    return DET_ERR_CUDA;
-  static DevOnce once = {};
-  if (dev_ensure_smem(once, (const void*)k_igemm_sl<OUT_BF16>, SL_SMEM) != DET_OK) return DET_ERR_CUDA;
-  const int sms = dev_sm_count();
-  if (sms <= 0) return DET_ERR_CUDA;
-  const int tiles = (I / SL_T) * (J / SL_T);
-  k_igemm_sl<OUT_BF16><<<DET_L(tiles < sms ? tiles : sms), SL_THREADS, SL_SMEM, st>>>(tAh, tAl, tBh, tBl, Ea, Eb, out, I, J, K, status);
-  if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DET_ERR_CUDA; }
-  return DET_OK;
+  SlArgs p = {};
+  p.Ea = Ea; p.Eb = Eb; p.out = out; p.rowscale = nullptr;
+  p.I = I; p.J = J; p.K = K; p.Z = 1; p.hdiv = 1; p.o_b = 0; p.o_h = 0; p.ldo = J;
+  p.causal_tiles = 0; p.krange = 0; p.epi = OUT_BF16 ? SL_BF16 : SL_F32;
+  return sliced_gemm_launch(Ah, Al, Bh, Bl, p, status, st);
 }
 
 static size_t v2_layout(int M, int V, int K, size_t* oAh, size_t* oAl, size_t* oBh, size_t* oBl, size_t* oEa, size_t* oEb) {

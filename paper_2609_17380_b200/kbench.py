@@ -156,6 +156,19 @@ def case_attn(small, bwd, int8pv=False, fixq=False):
                            dp + 4 * HD, 3 * HD, w)), 5 * unit, "flop"
 
 
+def case_attn_v2(small):
+    """Attention forward in arithmetic version 2 (not the benchmark's arithmetic): same workload as attn_fwd."""
+    B, H, S = (1 if small else 4), 16, 2048
+    T, dm = B * S, H * 128
+    qkv = randn_bf16(T * 3 * dm)
+    q, k, v = qkv, qkv[dm:], qkv[2 * dm:]
+    out, lse = torch.empty(T * dm, dtype=I16, device="cuda"), torch.empty(B * H * S, device="cuda")
+    w = ws(det.det_attn_fwd_v2_ws_bytes(B, H, S))
+    status = torch.zeros(1, dtype=I32, device="cuda")
+    flops = 2 * 2.0 * B * H * (S * (S + 1) / 2) * 128
+    return (lambda: det.det_attn_fwd_v2(q, k, v, 3 * dm, B, H, S, out, dm, lse, w, status)), flops, "flop"
+
+
 def case_lmhead(small, bwd):
     M, V, K = (1024 if small else 8192), 50304, 2048
     Hh, W = randn_bf16(M * K), randn_bf16(V * K, 0.02)
@@ -219,7 +232,7 @@ def build_cases():
     c = {"sumsq": case_sumsq, "grad_norm": case_grad_norm, "rmsnorm_fwd": lambda s: case_rmsnorm(s, False), "rmsnorm_bwd": lambda s: case_rmsnorm(s, True),
          "xent_fwd": lambda s: case_xent(s, False), "xent_bwd": lambda s: case_xent(s, True),
          "attn_fwd": lambda s: case_attn(s, False), "attn_bwd": lambda s: case_attn(s, True),
-         "attn_fwd_int8pv": lambda s: case_attn(s, False, True),
+         "attn_fwd_int8pv": lambda s: case_attn(s, False, True), "attn_fwd_v2": case_attn_v2,
          "attn_bwd_fixq": lambda s: case_attn(s, True, False, True),
          "lmhead_fwd": lambda s: case_lmhead(s, False), "lmhead_fwd_v2": case_lmhead_v2, "lmhead_bwd_v2": case_lmhead_bwd_v2, "lmhead_bwd": lambda s: case_lmhead(s, True),
          "accum": case_accum, "adamw": case_adamw, "hash": case_hash}

@@ -441,6 +441,34 @@ def test_lmhead_backward_version_2(det, M, V, K):
     assert_same_bits(gW[~nanW], wW[~nanW], "version-2 dW")
 
 
+@pytest.mark.parametrize("B,H,S", [(1, 1, 128), (1, 2, 384), (2, 3, 640)])
+def test_attention_forward_version_2(det, B, H, S):
+    """Causal attention in arithmetic version 2 (logits and P.V as order-free contractions on the int8 tensor cores, the
+    softmax in binary32) against its oracle, bit for bit: output and logsumexp; operands over a range of exponents so that
+    slices are truncated, a zero query row, a zero value column, subnormal inputs."""
+    import torch
+    from oracle import v2
+    rng = np.random.default_rng(B * 1000 + H * 100 + S)
+    x = rng.standard_normal((B * S, 3 * H * 128)) * np.exp2(rng.integers(-5, 2, (B * S, 3 * H * 128)))
+    x[:, :H * 128] *= 1.5                                       # sharper softmax rows
+    qkv = synth.to_bf16(x.astype(F))
+    qkv[5, :128] = 0                                            # a zero query row: uniform weights
+    qkv[:, 2 * H * 128 + 7] = 0                                 # a zero value column
+    qkv[9, H * 128:H * 128 + 128:5] = 0x0001                    # subnormal keys (count as zero)
+    ld = 3 * H * 128
+    d_qkv = dev(qkv)
+    flat = d_qkv.view(-1)
+    out, lse = empty((B * S, H * 128), np.uint16), empty((B, H, S), F)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    det.det_attn_fwd_v2(flat, flat[H * 128:], flat[2 * H * 128:], ld, B, H, S, out, H * 128, lse,
+                        ws(det.det_attn_fwd_v2_ws_bytes(B, H, S)), status)
+    _sync()
+    assert int(status.item()) == 0
+    w_out, w_lse = v2.attn_fwd(qkv, B, H, S)
+    assert_same_bits(host(lse), w_lse, "version-2 lse")
+    assert_same_bits(host(out, np.uint16), w_out, "version-2 attention output")
+
+
 def test_embedding(det):
     V, D, T = 1000, 512, 700
     E = synth.normal_bf16((V, D), 0.02, seed=7, tid=1)
