@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(128) k_slice_cols_heads(const uint16_t* __rest
 // One CTA (8 warps) per row (head z, query i) of the logits: a warp owns the leaves w, w + 8, ... of 256 keys, a lane 8
 // adjacent keys of a leaf, as in every fixed tree of this library; at most four leaves per warp (S <= 8192).
 constexpr int SM2_LPW = 4;
+template <int LPW>
 __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sraw, int S, float* __restrict__ lse,
                                                     float* __restrict__ inv_l, int8_t* __restrict__ Ph, int8_t* __restrict__ Pl,
                                                     int32_t* __restrict__ Ep) {
@@ -124,10 +125,10 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* s = Sraw + (size_t)row * S;
   const float NEG_INF = __int_as_float(0xff800000);
-  float pv[SM2_LPW][8];
+  float pv[LPW][8];
   float m = NEG_INF;
 #pragma unroll
-  for (int t = 0; t < SM2_LPW; ++t) {
+  for (int t = 0; t < LPW; ++t) {
     const int e0 = (warp + 8 * t) * 256 + lane * 8;
     if (e0 < n) {                                 // e0 + 7 < kend: inside the tiles that were computed
       const float4 a = *reinterpret_cast<const float4*>(s + e0), b = *reinterpret_cast<const float4*>(s + e0 + 4);
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
   const int nl = (n + 255) >> 8;
   int e = 0, bad = 0;
 #pragma unroll
-  for (int t = 0; t < SM2_LPW; ++t) {
+  for (int t = 0; t < LPW; ++t) {
     const int leaf = warp + 8 * t, e0 = leaf * 256 + lane * 8;
     if (leaf < nl) {                               // whole warp
 #pragma unroll
@@ -181,16 +182,17 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
   int key = 0;
 #pragma unroll
   for (int w = 0; w < 8; ++w) key |= redi[w] & (1 << 30), e = max(e, redi[w] & 0xFF);
-  smem_tree(leafs, nl);
-  if (threadIdx.x == 0) {
-    const float l = leafs[0];
-    lse[row] = fadd(m, det_log(l));
-    inv_l[row] = fdiv(1.0f, l);
-    Ep[row] = e | key;
+  if (warp == 0) {   // the tree over the leaf sums (at most 32 nodes of 256 keys) by one warp: no further barrier
+    const float l = warp_tree(lane < nl ? leafs[lane] : 0.0f, 0, 256, n);
+    if (lane == 0) {
+      lse[row] = fadd(m, det_log(l));
+      inv_l[row] = fdiv(1.0f, l);
+      Ep[row] = e | key;
+    }
   }
   // slices of bf16(p) for the keys below kend (zeros from i + 1 on)
 #pragma unroll
-  for (int t = 0; t < SM2_LPW; ++t) {
+  for (int t = 0; t < LPW; ++t) {
     const int e0 = (warp + 8 * t) * 256 + lane * 8;
     if (e0 < kend) {
       uint32_t h8[2] = {0u, 0u}, l8[2] = {0u, 0u};
@@ -261,7 +263,8 @@ extern "C" int det_attn_fwd_v2(const det_bf16* q, const det_bf16* k, const det_b
   a.causal_tiles = 1; a.krange = 0; a.epi = SL_F32;
   int rc = sliced_gemm_launch(Qh, Ql, Kh, Kl, a, status_dev, st);
   if (rc != DET_OK) return rc;
-  k_softmax_v2<<<DET_L(rows), 256, 0, st>>>(Sraw, S, lse, invl, Ph, Pl, Ep);
+  if (S <= 2048) k_softmax_v2<1><<<DET_L(rows), 256, 0, st>>>(Sraw, S, lse, invl, Ph, Pl, Ep);
+  else k_softmax_v2<SM2_LPW><<<DET_L(rows), 256, 0, st>>>(Sraw, S, lse, invl, Ph, Pl, Ep);
   DET_CHECK_LAUNCH();
   SlArgs u = {};
   u.Ea = Ep; u.Eb = Ev; u.out = out; u.rowscale = invl;

@@ -52,27 +52,6 @@ __device__ __forceinline__ void epi_scalars(const EpiParams& ep, float& cscale, 
     }
 }
 
-// A warp's 32 rows x 32 columns of output, held one row per lane (`w`: NW sixteen-byte words), go through a 32 x NW*16
-// byte staging tile in shared memory (sixteen-byte pieces XOR-swizzled, conflict-free both ways) so that every store
-// instruction writes whole 64- or 128-byte row segments instead of 16 bytes in each of 32 rows.
-template <int NW>
-__device__ __forceinline__ void store_rows32(uint8_t* stage, uint8_t* gbase, size_t row_pitch_bytes, const uint4 (&w)[NW]) {
-  const int lane = threadIdx.x & 31;
-  constexpr int SH = (NW == 4) ? 1 : 0;  // NW = 4: two rows share a 128-byte bank window, so the swizzle uses row >> 1
-  __syncwarp();                          // the previous chunk's reads are done
-#pragma unroll
-  for (int v = 0; v < NW; ++v)
-    *reinterpret_cast<uint4*>(stage + lane * (NW * 16) + ((v ^ ((lane >> SH) & (NW - 1))) << 4)) = w[v];
-  __syncwarp();
-  constexpr int RPI = 32 / NW;           // rows per store instruction
-#pragma unroll
-  for (int i = 0; i < NW; ++i) {
-    const int r = i * RPI + lane / NW, piece = lane % NW;
-    const uint4 x = *reinterpret_cast<const uint4*>(stage + r * (NW * 16) + ((piece ^ ((r >> SH) & (NW - 1))) << 4));
-    *reinterpret_cast<uint4*>(gbase + (size_t)r * row_pitch_bytes + piece * 16) = x;
-  }
-}
-
 // The reverse for the bf16 reference operand of the gradient epilogues: `pre` holds sixteen-byte pieces fetched with whole
 // 64-byte row segments per quad of lanes (fetch_rows32); rows32_to_lanes hands every lane the four words of its own row.
 __device__ __forceinline__ void fetch_rows32(const uint8_t* gbase, size_t row_pitch_bytes, uint4 (&pre)[4]) {

@@ -129,11 +129,19 @@ constexpr int SL_BK = 128;                    // bytes (= int8 elements) per ste
 constexpr int SL_STAGES = 3;
 constexpr int SL_TILE = SL_T * SL_BK;         // one operand tile: 16 KiB
 constexpr int SL_STAGE_BYTES = 4 * SL_TILE;   // H hi | H lo | W hi | W lo
-constexpr int SL_THREADS = 192;
-constexpr size_t SL_SMEM = (size_t)SL_STAGES * SL_STAGE_BYTES + 1024;
+constexpr int SL_EPI_WARPS = 8;               // warp & 3 = TMEM lane quarter, two warps per quarter take 64 columns each
+constexpr int SL_THREADS = 64 + 32 * SL_EPI_WARPS;
+constexpr size_t SL_SMEM = (size_t)SL_STAGES * SL_STAGE_BYTES + SL_EPI_WARPS * 4096 + 1024;   // ring + a staging tile per epilogue warp
 
-// the one rounding of the definition: I 2^e as binary32, nearest even; results below 2^-126 after the rounding are zeros
+// the one rounding of the definition: I 2^e as binary32, nearest even; results below 2^-126 after the rounding are zeros.
+// The conversion of the integer rounds once (nearest even) and a scaling by 2^e is exact while the result stays a
+// normal number, so the exponent is simply added; near the ends of the range the rounding is done in binary64 instead
+// (exact product, one conversion), where the subnormal grid decides what reaches 2^-126.
 __device__ __forceinline__ float round_scaled(long long I, int e) {
+  if (I == 0) return 0.0f;
+  const float f = __ll2float_rn(I);
+  const int ef = (int)((__float_as_uint(f) >> 23) & 0xFFu) + e;
+  if ((unsigned)(ef - 2) <= 252u) return __uint_as_float(__float_as_uint(f) + ((uint32_t)e << 23));
   const double v = (double)I * __longlong_as_double((long long)(e + 1023) << 52);   // exact: |I| < 2^53, e + 1023 in [745, 1253]
   float r = __double2float_rn(v);
   if (fabsf(r) < 0x1p-126f) r = copysignf(0.0f, r);
@@ -161,7 +169,7 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < SL_STAGES; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
     mbar_init(&bar_tfull, 1);
-    mbar_init(&bar_tempty, 4);
+    mbar_init(&bar_tempty, SL_EPI_WARPS);
     abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -241,7 +249,8 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       }
     }
   } else {
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int q = warp & 3, half = (warp - 2) >> 2;  // TMEM lane quarter this warp may read; its 64 of the 128 columns
+    uint8_t* stage = smem + SL_STAGES * SL_STAGE_BYTES + (warp - 2) * 4096;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -253,33 +262,51 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       const int row = i0 + q * 32 + lane;
       const int ea = Ea[(size_t)z * I + row];
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-      const size_t obase = (size_t)(z / p.hdiv) * p.o_b + (size_t)(z % p.hdiv) * p.o_h + (size_t)row * p.ldo + j0;
-      float* orow = reinterpret_cast<float*>(p.out) + obase;
-      uint16_t* brow = reinterpret_cast<uint16_t*>(p.out) + obase;
+      // the warp's first row: whole row segments leave through the staging tile (tc05.cuh: store_rows32)
+      const size_t wbase = (size_t)(z / p.hdiv) * p.o_b + (size_t)(z % p.hdiv) * p.o_h + (size_t)(row - lane) * p.ldo + j0;
       const float rsc = (p.epi == SL_BF16_ROWSCALE) ? p.rowscale[(size_t)z * I + row] : 1.0f;
-      const int32_t* Ebz = Eb + (size_t)z * J;
+      // the exponents of the warp's 64 columns, one load per tile: lane l keeps those of columns l and 32 + l, and a
+      // shuffle hands column c's to every row
+      const int ebv0 = Eb[(size_t)z * J + j0 + half * 64 + lane], ebv1 = Eb[(size_t)z * J + j0 + half * 64 + 32 + lane];
+      const int any_bad = __any_sync(0xffffffffu, ((ea | ebv0 | ebv1) >> 30) != 0);
+      const int ea280 = (ea & 0xFF) - 280;
 #pragma unroll 1
-      for (int c0 = 0; c0 < SL_T; c0 += 32) {
+      for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
         uint32_t hh[32], cr[32], ll[32];
-        tmem_ld32(taddr + (uint32_t)c0, hh);
-        tmem_ld32(taddr + 128u + (uint32_t)c0, cr);
-        tmem_ld32(taddr + 256u + (uint32_t)c0, ll);
+        tmem_ld32_nowait(taddr + (uint32_t)c0, hh);
+        tmem_ld32_nowait(taddr + 128u + (uint32_t)c0, cr);
+        tmem_ld32_nowait(taddr + 256u + (uint32_t)c0, ll);
+        tmem_wait_ld();
+        const int ebv = (c0 == half * 64) ? ebv0 : ebv1;
+        float f[32];
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
-          float f[4];
+        for (int c = 0; c < 32; ++c) {
+          const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
+          f[c] = round_scaled(Iv, ea280 + (__shfl_sync(0xffffffffu, ebv, c) & 0xFF));
+        }
+        if (any_bad) {   // a row or a column of the tile holds an infinity or a NaN: its results are NaN
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const int c = 4 * v + x;
-            const int eb = __ldg(Ebz + j0 + c0 + c);
-            const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
-            f[x] = ((ea | eb) >> 30) ? __int_as_float(0x7FC00000) : round_scaled(Iv, (ea & 0xFF) + (eb & 0xFF) - 280);
-          }
-          if (p.epi == SL_BF16_ROWSCALE) {
+          for (int c = 0; c < 32; ++c)
+            if ((ea | __shfl_sync(0xffffffffu, ebv, c)) >> 30) f[c] = __int_as_float(0x7FC00000);
+        }
+        if (p.epi == SL_BF16_ROWSCALE) {
 #pragma unroll
-            for (int x = 0; x < 4; ++x) f[x] = fmul(f[x], rsc);
-          }
-          if (p.epi != SL_F32) *reinterpret_cast<uint2*>(brow + c0 + 4 * v) = make_uint2(pack_bf2(f[0], f[1]), pack_bf2(f[2], f[3]));
-          else *reinterpret_cast<float4*>(orow + c0 + 4 * v) = make_float4(f[0], f[1], f[2], f[3]);
+          for (int c = 0; c < 32; ++c) f[c] = fmul(f[c], rsc);
+        }
+        if (p.epi != SL_F32) {
+          uint4 o[4];
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            o[v] = make_uint4(pack_bf2(f[8 * v], f[8 * v + 1]), pack_bf2(f[8 * v + 2], f[8 * v + 3]),
+                              pack_bf2(f[8 * v + 4], f[8 * v + 5]), pack_bf2(f[8 * v + 6], f[8 * v + 7]));
+          store_rows32<4>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(p.out) + wbase + c0), (size_t)p.ldo * 2, o);
+        } else {
+          uint4 o[8];
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            o[v] = make_uint4(__float_as_uint(f[4 * v]), __float_as_uint(f[4 * v + 1]), __float_as_uint(f[4 * v + 2]),
+                              __float_as_uint(f[4 * v + 3]));
+          store_rows32<8>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<float*>(p.out) + wbase + c0), (size_t)p.ldo * 4, o);
         }
       }
       tc_fence_before();

@@ -93,8 +93,42 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// the same load without the wait, so that several loads travel together; tmem_wait_ld() before the registers are read
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // host: tensor map of a row-major int8 matrix [rows, K] with boxes of box_rows x 128 bytes, 128-byte swizzle (igemm.cu)
 bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows);
+
+// A warp's 32 rows x 32 columns of output, held one row per lane (`w`: NW sixteen-byte words), go through a 32 x NW*16
+// byte staging tile in shared memory (sixteen-byte pieces XOR-swizzled, conflict-free both ways) so that every store
+// instruction writes whole 64- or 128-byte row segments instead of 16 bytes in each of 32 rows.
+template <int NW>
+__device__ __forceinline__ void store_rows32(uint8_t* stage, uint8_t* gbase, size_t row_pitch_bytes, const uint4 (&w)[NW]) {
+  const int lane = threadIdx.x & 31;
+  constexpr int SH = (NW == 4) ? 1 : 0;  // NW = 4: two rows share a 128-byte bank window, so the swizzle uses row >> 1
+  __syncwarp();                          // the previous chunk's reads are done
+#pragma unroll
+  for (int v = 0; v < NW; ++v)
+    *reinterpret_cast<uint4*>(stage + lane * (NW * 16) + ((v ^ ((lane >> SH) & (NW - 1))) << 4)) = w[v];
+  __syncwarp();
+  constexpr int RPI = 32 / NW;           // rows per store instruction
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    const int r = i * RPI + lane / NW, piece = lane % NW;
+    const uint4 x = *reinterpret_cast<const uint4*>(stage + r * (NW * 16) + ((piece ^ ((r >> SH) & (NW - 1))) << 4));
+    *reinterpret_cast<uint4*>(gbase + (size_t)r * row_pitch_bytes + piece * 16) = x;
+  }
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
