@@ -110,9 +110,15 @@ __global__ void __launch_bounds__(128) k_slice_cols_heads(const uint16_t* __rest
   }
 }
 
-// One CTA (8 warps) per row (head z, query i) of the logits: a warp owns the leaves w, w + 8, ... of 256 keys, a lane 8
-// adjacent keys of a leaf, as in every fixed tree of this library; at most four leaves per warp (S <= 8192).
+// One CTA per row (head z, query i) of the logits: a warp owns the leaves w, w + 8, ... of 256 keys, a lane 8 adjacent keys
+// of a leaf, as in every fixed tree of this library; at most LPW leaves per warp (S <= 2048 LPW).  Only the warps that
+// own a leaf of the row take part: the others leave at once and the barriers count the rest.
+//   * every weight is at most 1 and the maximum's own weight is exactly 1 (det_exp(0)), so the largest exponent among
+//     the bf16 weights equals the largest binary32 exponent field among the unrounded ones (rounding can lift a weight to
+//     1.0 but not beyond), and a NaN shows as 255 in both
+//   * the weights are not negative, so their slices carry no sign
 constexpr int SM2_LPW = 4;
+__device__ __forceinline__ void a2_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 template <int LPW>
 __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sraw, int S, float* __restrict__ lse,
                                                     float* __restrict__ inv_l, int8_t* __restrict__ Ph, int8_t* __restrict__ Pl,
@@ -123,6 +129,9 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
   const int row = blockIdx.x, i = row % S, n = i + 1;
   const int kend = ((i >> 7) + 1) << 7;           // the keys the row tile's contraction runs over
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nl = (n + 255) >> 8;                  // leaves of the row
+  const int nw = nl < 8 ? nl : 8;                 // warps that own one
+  if (warp >= nw) return;
   const float* s = Sraw + (size_t)row * S;
   const float NEG_INF = __int_as_float(0xff800000);
   float pv[LPW][8];
@@ -133,10 +142,12 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
     if (e0 < n) {                                 // e0 + 7 < kend: inside the tiles that were computed
       const float4 a = *reinterpret_cast<const float4*>(s + e0), b = *reinterpret_cast<const float4*>(s + e0 + 4);
       const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      if (e0 + 8 <= n) {
 #pragma unroll
-      for (int x = 0; x < 8; ++x) {
-        pv[t][x] = (e0 + x < n) ? fmul(v[x], ATT2_SCALE) : NEG_INF;
-        m = fmaxf(m, pv[t][x]);
+        for (int x = 0; x < 8; ++x) { pv[t][x] = fmul(v[x], ATT2_SCALE); m = fmaxf(m, pv[t][x]); }
+      } else {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) { pv[t][x] = (e0 + x < n) ? fmul(v[x], ATT2_SCALE) : NEG_INF; m = fmaxf(m, pv[t][x]); }
       }
     } else {
 #pragma unroll
@@ -145,52 +156,49 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
   }
 #pragma unroll
   for (int w = 16; w; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
-  if (lane == 0) redf[warp] = m;
-  __syncthreads();
-  m = redf[0];
-#pragma unroll
-  for (int w = 1; w < 8; ++w) m = fmaxf(m, redf[w]);
-  // exponentials (arguments <= 0), leaf sums of the fixed tree over the keys 0 .. i, exponent of the row of bf16 weights
-  const int nl = (n + 255) >> 8;
-  int e = 0, bad = 0;
+  if (nw > 1) {
+    if (lane == 0) redf[warp] = m;
+    a2_bar(nw * 32);
+    m = redf[0];
+    for (int w = 1; w < nw; ++w) m = fmaxf(m, redf[w]);
+  }
+  // exponentials (arguments <= 0; an invisible key has -inf and gives +0), leaf sums of the fixed tree over the keys 0 .. i
+  int e = 0;
 #pragma unroll
   for (int t = 0; t < LPW; ++t) {
     const int leaf = warp + 8 * t, e0 = leaf * 256 + lane * 8;
     if (leaf < nl) {                               // whole warp
 #pragma unroll
-      for (int x = 0; x < 8; ++x) pv[t][x] = (e0 + x < n) ? det_exp_le0(fsub(pv[t][x], m)) : 0.0f;
-      const float sum = warp_tree(tree8(pv[t], e0, n), (long long)leaf * 256, 8, n);
+      for (int x = 0; x < 8; ++x) pv[t][x] = det_exp_le0(fsub(pv[t][x], m));
+      const bool whole = leaf * 256 + 256 <= n;    // no existence tests inside a complete leaf
+      const float sum = whole ? warp_tree_full(tree8_full(pv[t])) : warp_tree(tree8(pv[t], e0, n), (long long)leaf * 256, 8, n);
       if (lane == 0) leafs[leaf] = sum;
 #pragma unroll
-      for (int x = 0; x < 8; ++x) {
-        const int ex = (int)((bf_bits(pv[t][x]) >> 7) & 0xFF);
-        bad |= (ex == 255);
-        e = max(e, ex);
-      }
+      for (int x = 0; x < 8; ++x) e = max(e, (int)((__float_as_uint(pv[t][x]) >> 23) & 0xFFu));
     } else {
 #pragma unroll
       for (int x = 0; x < 8; ++x) pv[t][x] = 0.0f;
     }
   }
 #pragma unroll
-  for (int w = 16; w; w >>= 1) {
-    e = max(e, __shfl_xor_sync(0xffffffffu, e, w));
-    bad |= __shfl_xor_sync(0xffffffffu, bad, w);
+  for (int w = 16; w; w >>= 1) e = max(e, __shfl_xor_sync(0xffffffffu, e, w));
+  if (nw > 1) {
+    if (lane == 0) redi[warp] = e;
+    a2_bar(nw * 32);                               // leaf sums and exponents are published
+    for (int w = 0; w < nw; ++w) e = max(e, redi[w]);
+  } else {
+    __syncwarp();
   }
-  if (lane == 0) redi[warp] = e | (bad << 30);
-  __syncthreads();                                 // leaf sums and exponents are published
-  int key = 0;
-#pragma unroll
-  for (int w = 0; w < 8; ++w) key |= redi[w] & (1 << 30), e = max(e, redi[w] & 0xFF);
   if (warp == 0) {   // the tree over the leaf sums (at most 32 nodes of 256 keys) by one warp: no further barrier
     const float l = warp_tree(lane < nl ? leafs[lane] : 0.0f, 0, 256, n);
     if (lane == 0) {
       lse[row] = fadd(m, det_log(l));
       inv_l[row] = fdiv(1.0f, l);
-      Ep[row] = e | key;
+      Ep[row] = (e == 255) ? (255 | (1 << 30)) : e;
     }
   }
   // slices of bf16(p) for the keys below kend (zeros from i + 1 on)
+  const int ee = e == 255 ? 255 : e;
 #pragma unroll
   for (int t = 0; t < LPW; ++t) {
     const int e0 = (warp + 8 * t) * 256 + lane * 8;
@@ -198,10 +206,11 @@ __global__ void __launch_bounds__(256) k_softmax_v2(const float* __restrict__ Sr
       uint32_t h8[2] = {0u, 0u}, l8[2] = {0u, 0u};
 #pragma unroll
       for (int x = 0; x < 8; ++x) {
-        int h, l;
-        slice1(bf_bits(pv[t][x]), e, h, l);
-        h8[x >> 2] |= (uint32_t)(uint8_t)(int8_t)h << (8 * (x & 3));
-        l8[x >> 2] |= (uint32_t)(uint8_t)(int8_t)l << (8 * (x & 3));
+        const uint32_t b = bf_bits(pv[t][x]);
+        const int ek = (int)(b >> 7) & 0xFF, d = ee - ek;
+        const uint32_t tt = (ek == 0 || d >= 14) ? 0u : (((128u + (b & 0x7Fu)) << 6) >> d);
+        h8[x >> 2] |= (tt >> 7) << (8 * (x & 3));
+        l8[x >> 2] |= (tt & 127u) << (8 * (x & 3));
       }
       *reinterpret_cast<uint2*>(Ph + (size_t)row * S + e0) = make_uint2(h8[0], h8[1]);
       *reinterpret_cast<uint2*>(Pl + (size_t)row * S + e0) = make_uint2(l8[0], l8[1]);

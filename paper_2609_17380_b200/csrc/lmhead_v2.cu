@@ -129,9 +129,9 @@ constexpr int SL_BK = 128;                    // bytes (= int8 elements) per ste
 constexpr int SL_STAGES = 3;
 constexpr int SL_TILE = SL_T * SL_BK;         // one operand tile: 16 KiB
 constexpr int SL_STAGE_BYTES = 4 * SL_TILE;   // H hi | H lo | W hi | W lo
-constexpr int SL_EPI_WARPS = 8;               // warp & 3 = TMEM lane quarter, two warps per quarter take 64 columns each
+constexpr int SL_EPI_WARPS = 16;              // warp & 3 = TMEM lane quarter, four warps per quarter take 32 columns each
 constexpr int SL_THREADS = 64 + 32 * SL_EPI_WARPS;
-constexpr size_t SL_SMEM = (size_t)SL_STAGES * SL_STAGE_BYTES + SL_EPI_WARPS * 4096 + 1024;   // ring + a staging tile per epilogue warp
+constexpr size_t SL_SMEM = (size_t)SL_STAGES * SL_STAGE_BYTES + SL_EPI_WARPS * 2048 + 1024;   // ring + a staging tile per epilogue warp
 
 // the one rounding of the definition: I 2^e as binary32, nearest even; results below 2^-126 after the rounding are zeros.
 // The conversion of the integer rounds once (nearest even) and a scaling by 2^e is exact while the result stays a
@@ -249,8 +249,8 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       }
     }
   } else {
-    const int q = warp & 3, half = (warp - 2) >> 2;  // TMEM lane quarter this warp may read; its 64 of the 128 columns
-    uint8_t* stage = smem + SL_STAGES * SL_STAGE_BYTES + (warp - 2) * 4096;
+    const int q = warp & 3, part = (warp - 2) >> 2;  // TMEM lane quarter this warp may read; its 32 of the 128 columns
+    uint8_t* stage = smem + SL_STAGES * SL_STAGE_BYTES + (warp - 2) * 2048;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -265,48 +265,48 @@ __global__ void __launch_bounds__(SL_THREADS, 1)
       // the warp's first row: whole row segments leave through the staging tile (tc05.cuh: store_rows32)
       const size_t wbase = (size_t)(z / p.hdiv) * p.o_b + (size_t)(z % p.hdiv) * p.o_h + (size_t)(row - lane) * p.ldo + j0;
       const float rsc = (p.epi == SL_BF16_ROWSCALE) ? p.rowscale[(size_t)z * I + row] : 1.0f;
-      // the exponents of the warp's 64 columns, one load per tile: lane l keeps those of columns l and 32 + l, and a
-      // shuffle hands column c's to every row
-      const int ebv0 = Eb[(size_t)z * J + j0 + half * 64 + lane], ebv1 = Eb[(size_t)z * J + j0 + half * 64 + 32 + lane];
-      const int any_bad = __any_sync(0xffffffffu, ((ea | ebv0 | ebv1) >> 30) != 0);
+      // the exponents of the warp's 32 columns, one load per tile: lane l keeps column l's, a shuffle hands column c's to
+      // every row
+      const int ebv = Eb[(size_t)z * J + j0 + part * 32 + lane];
+      const int any_bad = __any_sync(0xffffffffu, ((ea | ebv) >> 30) != 0);
       const int ea280 = (ea & 0xFF) - 280;
 #pragma unroll 1
-      for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
-        uint32_t hh[32], cr[32], ll[32];
-        tmem_ld32_nowait(taddr + (uint32_t)c0, hh);
-        tmem_ld32_nowait(taddr + 128u + (uint32_t)c0, cr);
-        tmem_ld32_nowait(taddr + 256u + (uint32_t)c0, ll);
+      for (int sub = 0; sub < 2; ++sub) {
+        const int c0 = part * 32 + sub * 16;
+        uint32_t hh[16], cr[16], ll[16];
+        tmem_ld16_nowait(taddr + (uint32_t)c0, hh);
+        tmem_ld16_nowait(taddr + 128u + (uint32_t)c0, cr);
+        tmem_ld16_nowait(taddr + 256u + (uint32_t)c0, ll);
         tmem_wait_ld();
-        const int ebv = (c0 == half * 64) ? ebv0 : ebv1;
-        float f[32];
+        float f[16];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
+        for (int c = 0; c < 16; ++c) {
           const long long Iv = ((long long)(int)hh[c] << 14) + ((long long)(int)cr[c] << 7) + (long long)(int)ll[c];
-          f[c] = round_scaled(Iv, ea280 + (__shfl_sync(0xffffffffu, ebv, c) & 0xFF));
+          f[c] = round_scaled(Iv, ea280 + (__shfl_sync(0xffffffffu, ebv, sub * 16 + c) & 0xFF));
         }
         if (any_bad) {   // a row or a column of the tile holds an infinity or a NaN: its results are NaN
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if ((ea | __shfl_sync(0xffffffffu, ebv, c)) >> 30) f[c] = __int_as_float(0x7FC00000);
+          for (int c = 0; c < 16; ++c)
+            if ((ea | __shfl_sync(0xffffffffu, ebv, sub * 16 + c)) >> 30) f[c] = __int_as_float(0x7FC00000);
         }
         if (p.epi == SL_BF16_ROWSCALE) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) f[c] = fmul(f[c], rsc);
+          for (int c = 0; c < 16; ++c) f[c] = fmul(f[c], rsc);
         }
         if (p.epi != SL_F32) {
+          uint4 o[2];
+#pragma unroll
+          for (int v = 0; v < 2; ++v)
+            o[v] = make_uint4(pack_bf2(f[8 * v], f[8 * v + 1]), pack_bf2(f[8 * v + 2], f[8 * v + 3]),
+                              pack_bf2(f[8 * v + 4], f[8 * v + 5]), pack_bf2(f[8 * v + 6], f[8 * v + 7]));
+          store_rows32<2>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(p.out) + wbase + c0), (size_t)p.ldo * 2, o);
+        } else {
           uint4 o[4];
 #pragma unroll
           for (int v = 0; v < 4; ++v)
-            o[v] = make_uint4(pack_bf2(f[8 * v], f[8 * v + 1]), pack_bf2(f[8 * v + 2], f[8 * v + 3]),
-                              pack_bf2(f[8 * v + 4], f[8 * v + 5]), pack_bf2(f[8 * v + 6], f[8 * v + 7]));
-          store_rows32<4>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(p.out) + wbase + c0), (size_t)p.ldo * 2, o);
-        } else {
-          uint4 o[8];
-#pragma unroll
-          for (int v = 0; v < 8; ++v)
             o[v] = make_uint4(__float_as_uint(f[4 * v]), __float_as_uint(f[4 * v + 1]), __float_as_uint(f[4 * v + 2]),
                               __float_as_uint(f[4 * v + 3]));
-          store_rows32<8>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<float*>(p.out) + wbase + c0), (size_t)p.ldo * 4, o);
+          store_rows32<4>(stage, reinterpret_cast<uint8_t*>(reinterpret_cast<float*>(p.out) + wbase + c0), (size_t)p.ldo * 4, o);
         }
       }
       tc_fence_before();

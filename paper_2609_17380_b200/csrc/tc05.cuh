@@ -105,6 +105,14 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // host: tensor map of a row-major int8 matrix [rows, K] with boxes of box_rows x 128 bytes, 128-byte swizzle (igemm.cu)
 bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows);
@@ -115,7 +123,7 @@ bool make_map(CUtensorMap* tm, const int8_t* base, int rows, int K, int box_rows
 template <int NW>
 __device__ __forceinline__ void store_rows32(uint8_t* stage, uint8_t* gbase, size_t row_pitch_bytes, const uint4 (&w)[NW]) {
   const int lane = threadIdx.x & 31;
-  constexpr int SH = (NW == 4) ? 1 : 0;  // NW = 4: two rows share a 128-byte bank window, so the swizzle uses row >> 1
+  constexpr int SH = (NW == 8) ? 0 : (NW == 4 ? 1 : 2);  // 128 / (16 NW) rows share a 128-byte bank window: swizzle by row >> SH
   __syncwarp();                          // the previous chunk's reads are done
 #pragma unroll
   for (int v = 0; v < NW; ++v)
