@@ -441,7 +441,7 @@ def test_lmhead_backward_version_2(det, M, V, K):
     assert_same_bits(gW[~nanW], wW[~nanW], "version-2 dW")
 
 
-@pytest.mark.parametrize("B,H,S", [(1, 1, 128), (1, 2, 384), (2, 3, 640)])
+@pytest.mark.parametrize("B,H,S", [(1, 1, 128), (1, 2, 384), (2, 3, 640), (1, 1, 2176)])   # 2176 > 2048: several leaves per warp
 def test_attention_forward_version_2(det, B, H, S):
     """Causal attention in arithmetic version 2 (logits and P.V as order-free contractions on the int8 tensor cores, the
     softmax in binary32) against its oracle, bit for bit: output and logsumexp; operands over a range of exponents so that
