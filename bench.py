@@ -179,6 +179,24 @@ def component_rates_configs_2_3(peaks, iters=5):
     return out
 
 
+def optional_arithmetic_v2_rates(iters=5):
+    """The optional arithmetic version 2 (NOT the benchmark's arithmetic; the default step does not use it): the LM head
+    and the attention forward as order-free contractions on the int8 tensor cores, each beside the default-arithmetic
+    kernel on the same workload (8192 x 50304 x 2048; 4 x 16 heads x 2048)."""
+    import torch
+    from paper_2609_17380_b200 import kbench
+    out = {}
+    for name, fn in (("lmhead_fwd", lambda: kbench.case_lmhead(False, False)), ("lmhead_fwd_v2", lambda: kbench.case_lmhead_v2(False)),
+                     ("lmhead_bwd", lambda: kbench.case_lmhead(False, True)), ("lmhead_bwd_v2", lambda: kbench.case_lmhead_bwd_v2(False)),
+                     ("attn_fwd", lambda: kbench.case_attn(False, False)), ("attn_fwd_v2", lambda: kbench.case_attn_v2(False))):
+        call, _, _ = fn()
+        torch.cuda.synchronize()
+        out[name + "_ms"] = round(kbench.timeit(call, iters), 4)
+        del call
+        torch.cuda.empty_cache()
+    return out
+
+
 def spawn_ranks(args):
     """`python bench.py --gpus N` without a launcher: start N local ranks, one GPU each, NCCL over 127.0.0.1."""
     import socket
@@ -505,6 +523,10 @@ def run_ours(args):
             line["component_rates"].update(component_rates_configs_2_3(peaks))
         except Exception as ex:
             line["component_rates"]["configs_2_3_error"] = repr(ex)
+        try:
+            line["optional_arithmetic_v2"] = optional_arithmetic_v2_rates()
+        except Exception as ex:
+            line["optional_arithmetic_v2"] = {"error": repr(ex)}
         line["state_hash"] = hash_keep
     if world == 1 and not args.no_cpu_baseline:
         try:
