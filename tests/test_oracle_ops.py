@@ -165,6 +165,27 @@ def test_hadamard_modes_agree_when_quantisation_is_exact():
     assert bf(a0[0])[5, 9] == F(0.25 * 0.5) and a0[1][17, 9] == F(0.25 * 2.0)
 
 
+def test_step_size_gradient_by_hand():
+    """ds_x = det_sum(gx * phi) / sqrt(M K 127) (the LSQ step-size gradient, Sec. 3.1) on two hand-made elements whose
+    quantisation is exact.  Element (5, 9): x / s = 4.5 rounds to the code 4 (ties to even), phi = 4 - 4.5 = -0.5, the
+    gradient reaching it is 0.25 * 0.5 = 0.125.  Element (6, 10): x / s = 200 lies above the range, so phi = 127, the
+    gradient of x is masked to 0 and the same 0.125 enters the step-size gradient.  The sum of the two terms,
+    0.125 * (127 - 0.5) = 15.8125, is exact; with or without the rotation."""
+    M = N = K = 128
+    X = np.zeros((M, K), F); W = np.zeros((N, K), F); dY = np.zeros((M, N), F)
+    X[5, 9], X[6, 10] = 2.25, 100.0
+    W[17, 9] = W[18, 10] = 0.5
+    dY[5, 17] = dY[6, 18] = 0.25
+    s_x = np.array([0.5], F); s_w = np.full(N, 0.5 / 64, F)
+    gs = F(1.0 / math.sqrt(M * K * 127.0))
+    for hb in (0, 128):
+        dX, dW, ds = oracle.linear_bwd(synth.to_bf16(dY), synth.to_bf16(X), synth.to_bf16(W), s_x, s_w, hb=hb)
+        assert bf(dX)[5, 9] == F(0.125) and bf(dX)[6, 10] == 0.0                  # in range: passed on; out of range: masked
+        assert ds[0] == F(gs * F(15.8125))
+        assert abs(float(ds[0]) - 15.8125 / math.sqrt(M * K * 127.0)) < 1e-9
+        assert dW[17, 9] == F(0.25 * 4 * 0.5) and abs(dW[18, 10] - 0.25 * 127 * 0.5) < 2e-6   # x^ = code * s_x: 2.0 and 63.5
+
+
 def test_hadamard_reduces_weight_gradient_error_on_heavy_tails():
     # Sec. 3.2: rotation flattens gradient outliers (paper: ~5% -> ~1% at its shapes; a sanity check)
     M, N, K = 1024, 128, 128
