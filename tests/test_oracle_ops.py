@@ -403,6 +403,72 @@ def test_attention_value_gradient_sums_queries_in_ascending_order():
     assert np.all(bf(d[1:, 256:]) == 0.0)                             # no weight on the other keys
 
 
+def test_attention_query_gradient_sums_keys_in_ascending_order():
+    """q = 0 makes the weights of row 63 uniform, values alternating +1, -1 in one column make O = 0 exactly (so Delta = 0)
+    and dP = +d, -d; dS_63,j is then +g, -g with ONE magnitude g.  Keys that carry the same alternating sign times
+    (2^25, 1, ..., 1, -2^25) in column 3 give dQ_63,3 = g 2^25 + g + ... + g - g 2^25: in ascending (or descending) order
+    every g is lost and the result is 0, in a tree the small terms meet first and survive.  Column 4 carries
+    (1, ..., 1, 2^25, -2^25): ascending, the 62 small terms are summed exactly and then rounded against the large one;
+    descending they would be added to an exact 0."""
+    S = 64
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    sign = np.where(np.arange(S) % 2 == 0, 1.0, -1.0).astype(F)
+    t1 = np.ones(S, F); t1[0] = 2.0 ** 25; t1[-1] = -2.0 ** 25
+    t2 = np.ones(S, F); t2[-2] = 2.0 ** 25; t2[-1] = -2.0 ** 25
+    qkv = _qkv_rows(S)
+    kk = np.zeros((S, 128), F); kk[:, 3] = sign * t1; kk[:, 4] = sign * t2
+    vv = np.zeros((S, 128), F); vv[:, 7] = sign
+    qkv[:, 128:256] = synth.to_bf16(kk)
+    qkv[:, 256:] = synth.to_bf16(vv)
+    out, lse = oracle.attn_fwd(qkv, 1, 1, S)
+    assert np.all(bf(out)[S - 1] == 0.0)
+    dO = np.zeros((S, 128), F); dO[S - 1, 7] = 1.0
+    d = oracle.attn_bwd(synth.to_bf16(dO), qkv, out, lse, 1, 1, S)
+    P = oracle.prim("exp", np.array([F(F(0.0) - lse[0, 0, S - 1])], F))[0]
+    g = bf(synth.to_bf16(np.array([F(F(P * F(1.0)) * scale)], F)))[0]
+    assert g > 0 and abs(g - 2.0 ** -3.5 / S) < 1e-4
+    dq = bf(d[S - 1, :128])
+    assert dq[3] == 0.0
+    acc = F(0.0)
+    for j in range(S):
+        acc = F(acc + F(g * t2[j]))
+    want = bf(synth.to_bf16(np.array([acc], F)))[0]
+    assert dq[4] == want and want != bf(synth.to_bf16(np.array([F(62 * g)], F)))[0]    # 62 g is what a descending sum gives
+    assert np.all(np.delete(dq, [3, 4]) == 0.0)
+
+
+def test_attention_key_gradient_sums_queries_in_ascending_order():
+    """Only keys 0 and 1 carry weight (logit 0; every other key far below), with values +1 and -1 in one column: every row
+    i >= 1 has the same two weights, O = 0 exactly, Delta = 0 and dS_i0 = +g, ONE value for all rows.  The queries carry
+    (2^25, 1, ..., 1, -2^25) in column 3 and (1, ..., 1, 2^25, -2^25) in column 4 (columns in which every key is 0, so the
+    logits do not see them): dK_0 is 0 in column 3 for a sequential sum, and in column 4 the ascending value, which differs
+    from the descending one (61 g) and from a tree's."""
+    S = 64
+    scale = F(float.fromhex("0x1.6a09e6p-4"))
+    t1 = np.ones(S, F); t1[1] = 2.0 ** 25; t1[-1] = -2.0 ** 25; t1[0] = 0.0
+    t2 = np.ones(S, F); t2[-2] = 2.0 ** 25; t2[-1] = -2.0 ** 25; t2[0] = 0.0
+    qq = np.zeros((S, 128), F); qq[:, 0] = 1.0; qq[:, 3] = t1; qq[:, 4] = t2
+    kk = np.zeros((S, 128), F); kk[2:, 0] = -30000.0
+    vv = np.zeros((S, 128), F); vv[0, 7] = 1.0; vv[1, 7] = -1.0
+    qkv = _qkv_rows(S)
+    qkv[:, :128] = synth.to_bf16(qq); qkv[:, 128:256] = synth.to_bf16(kk); qkv[:, 256:] = synth.to_bf16(vv)
+    out, lse = oracle.attn_fwd(qkv, 1, 1, S)
+    assert np.all(bf(out)[1:] == 0.0) and np.all(lse[0, 0, 1:] == lse[0, 0, 1])
+    dO = np.zeros((S, 128), F); dO[1:, 7] = 1.0
+    d = oracle.attn_bwd(synth.to_bf16(dO), qkv, out, lse, 1, 1, S)
+    P = oracle.prim("exp", np.array([F(F(0.0) - lse[0, 0, 1])], F))[0]
+    g = bf(synth.to_bf16(np.array([F(F(P * F(1.0)) * scale)], F)))[0]
+    assert abs(g - 2.0 ** -3.5 / 2) < 1e-3
+    dk0 = bf(d[0, 128:256])
+    assert dk0[3] == 0.0
+    acc = F(0.0)
+    for i in range(1, S):
+        acc = F(acc + F(g * t2[i]))
+    want = bf(synth.to_bf16(np.array([acc], F)))[0]
+    assert dk0[4] == want and want != bf(synth.to_bf16(np.array([F(61 * g)], F)))[0]
+    assert np.array_equal(bf(d[1, 128:256])[3:5], -dk0[3:5])                # key 1: the same sums with -g
+
+
 def test_attention_backward_recomputes_the_weights_from_lse():
     """Two keys, dO_0 = 0, dO_1 = e_c: dV_0 = bf16(P_10) in column c, with P_10 = exp(s_0 - lse_1) recomputed from the
     stored logsumexp (not the forward's p / l) and rounded to bf16 once more by the output."""
