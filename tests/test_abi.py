@@ -46,3 +46,14 @@ def test_host_side_argument_checks():
     assert lib.det_attn_fwd(a16, a16, a16, 512, 1, 4, 3, 128, 0, a16, 512, a16, None) == -2         # H % Hkv
     assert lib.det_attn_fwd(a16, a16, a16, 128, 1, 1, 1, 128, 100, a16, 128, a16, None) == -2       # window % 128
     assert lib.det_xent_fwd(a16, a16, 4, 8, ctypes.c_float(0), a16, a16, a16, a16, a16, ctypes.c_size_t(8), None, None) == -4
+    # the attention forward of arithmetic version 2: shape limits, alignment, workspace size
+    lib.det_attn_fwd_v2_ws_bytes.restype = ctypes.c_size_t
+    need = lib.det_attn_fwd_v2_ws_bytes(1, 2, 256)
+    assert need >= 2 * 256 * 256 * 6 and lib.det_attn_fwd_v2_ws_bytes(0, 2, 256) == 0
+    big = ctypes.c_size_t(1 << 40)
+    assert lib.det_attn_fwd_v2(a16, a16, a16, 768, 1, 2, 100, a16, 256, a16, a16, big, None, None) == -2      # S % 128
+    assert lib.det_attn_fwd_v2(a16, a16, a16, 768, 1, 2, 16384, a16, 256, a16, a16, big, None, None) == -2    # S > 8192
+    assert lib.det_attn_fwd_v2(a16, a16, a16, 128, 1, 2, 256, a16, 256, a16, a16, big, None, None) == -2      # ld < H * 128
+    assert lib.det_attn_fwd_v2(a1, a16, a16, 768, 1, 2, 256, a16, 256, a16, a16, big, None, None) == -3       # alignment
+    assert lib.det_attn_fwd_v2(a16, a16, a16, 768, 1, 2, 256, a16, 256, a16, a16, ctypes.c_size_t(need - 1), None, None) == -4
+    assert lib.det_attn_fwd_v2(None, a16, a16, 768, 1, 2, 256, a16, 256, a16, a16, big, None, None) == -1     # null operand
