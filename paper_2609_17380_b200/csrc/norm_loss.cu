@@ -93,108 +93,95 @@ __global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x
   }
 }
 
-// Backward for rows of at most 2048 elements.  A CTA takes a block of 8 adjacent rows in passes of RP rows (RP * 4
-// warps: warp quarter hw of a row owns its leaves 2 hw, 2 hw + 1, i.e. 16 values of dy and of x per lane), so that
-// two CTAs share an SM and one loads or stores while the other stands at a barrier (one CTA of 8 x 4 warps per SM
-// ran 20 % slower; without the gain gradient this kernel moves its bytes at 0.9 of the copy bandwidth).  With DG the
-// CTA also leaves the column-wise tree over its 8 rows of dy*xhat in partial8[block][D] (the first three levels of
-// the row-direction tree).
-#ifndef RMS_RP
-#define RMS_RP 4
-#endif
-template <bool BF, bool DG, int RP>
-__global__ void __launch_bounds__(RP * 128, 8 / RP) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
-                                                                const void* __restrict__ gamma,
-                                                                const float* __restrict__ rstd, int rows, int D, float invD,
-                                                                void* __restrict__ dx, float* __restrict__ partial8,
-                                                                int* __restrict__ tickets) {
-  constexpr int NT = RP * 128, NPASS = 8 / RP;
-  extern __shared__ __align__(16) float srow[];  // DG: [8][D]
-  __shared__ float half_sum[2][RP][4];
+// Backward for rows of at most 2048 elements.  A CTA of 8 warps takes a block of 8 adjacent rows in four passes of two
+// rows; warp j holds columns 256 j .. 256 j + 255 (one leaf of the fixed tree) of both rows, 8 adjacent columns per lane;
+// three CTAs per SM, so that one loads or stores while another stands at its barrier (one CTA of 8 rows x 4 warps per SM
+// ran 20 % slower).  A lane sees the same 8 columns of all 8 rows of the block, one pair of rows after the other, so with
+// DG the column tree over the 8 rows of dy*xhat (the first three levels of the gain gradient's row-direction tree,
+// written to partial8[block][D]) runs in its registers: no shared-memory copy of the products and no barrier of its own
+// (0.080 ms with the products staged through shared memory by warps that each owned a quarter row, 0.070 ms now;
+// 0.065-0.070 ms without the gain gradient, i.e. 0.9 of the copy bandwidth).  The row sums go through shared memory: one
+// value per leaf and row, one barrier per pass.
+template <bool BF, bool DG>
+__global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
+                                                        const void* __restrict__ gamma, const float* __restrict__ rstd,
+                                                        int rows, int D, float invD, void* __restrict__ dx,
+                                                        float* __restrict__ partial8, int* __restrict__ tickets) {
+  __shared__ float leaf_sum[2][2][8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int hw = warp & 3;
+  const int e0 = warp * 256 + lane * 8;
+  const bool have = e0 < D;                       // this lane's 8 columns exist (D is a multiple of 8)
   const bool full = (D & 255) == 0;
   const long long r0 = (long long)blockIdx.x * 8;
   if (DG && blockIdx.x == 0 && (int)threadIdx.x < ((D + 255) >> 8)) tickets[threadIdx.x] = 0;   // for the kernel that follows
-#pragma unroll 1
-  for (int pass = 0; pass < NPASS; ++pass) {
-    const int rl = pass * RP + (warp >> 2);       // row of the block, 0 .. 7
-    float (*hs)[4] = half_sum[pass & 1];
-    const int row = blockIdx.x * 8 + rl;
-    const bool live = row < rows;
-    const size_t rb = (size_t)row * D;
-    float w[2][8], xh[2][8];
+  float pair0[8], node[8];                        // column tree: a pair of rows waiting for the next pair; rows 0 .. 3
 #pragma unroll
-    for (int jj = 0; jj < 2; ++jj) {
-      const int e0 = (hw * 2 + jj) * 256 + lane * 8;
-      if (live && e0 < D) {
-        load8<BF>(dy, rb + e0, w[jj]);
-        load8<BF>(x, rb + e0, xh[jj]);
+  for (int t = 0; t < 8; ++t) { pair0[t] = 0.0f; node[t] = 0.0f; }
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const long long first = r0 + 2 * pass;
+    float w[2][8], xh[2][8], rs[2];
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      const long long row = first + a;
+      if (row < rows && have) {
+        load8<BF>(dy, (size_t)row * D + e0, w[a]);
+        load8<BF>(x, (size_t)row * D + e0, xh[a]);
       } else {
 #pragma unroll
-        for (int t = 0; t < 8; ++t) { w[jj][t] = 0.0f; xh[jj][t] = 0.0f; }
+        for (int t = 0; t < 8; ++t) { w[a][t] = 0.0f; xh[a][t] = 0.0f; }
+      }
+      rs[a] = row < rows ? rstd[row] : 0.0f;
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { xh[0][t] = fmul(xh[0][t], rs[0]); xh[1][t] = fmul(xh[1][t], rs[1]); }
+    if (DG) {   // rows 2 pass, 2 pass + 1 -> pair; pairs 0, 1 and 2, 3 -> nodes of four rows; those two -> the node of eight
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const float d0 = fmul(w[0][t], xh[0][t]), d1 = fmul(w[1][t], xh[1][t]);
+        const float pr2 = (first + 1 < rows) ? fadd(d0, d1) : d0;
+        if ((pass & 1) == 0) pair0[t] = pr2;
+        else {
+          const float four = (first < rows) ? fadd(pair0[t], pr2) : pair0[t];   // the right pair exists iff its first row does
+          node[t] = (pass == 1) ? four : ((r0 + 4 < rows) ? fadd(node[t], four) : node[t]);
+        }
       }
     }
-    const float rs = live ? rstd[row] : 0.0f;
-    float mine = 0.0f;
+    if (gamma && have) {
+      float g[8];
+      load8<BF>(gamma, e0, g);
 #pragma unroll
-    for (int jj = 0; jj < 2; ++jj) {
-      const int j = hw * 2 + jj;
-      const int e0 = j * 256 + lane * 8;
+      for (int t = 0; t < 8; ++t) { w[0][t] = fmul(w[0][t], g[t]); w[1][t] = fmul(w[1][t], g[t]); }
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
       float pr[8];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) xh[jj][t] = fmul(xh[jj][t], rs);
-      if (DG && e0 < D) {
-        float dgt[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) dgt[t] = fmul(w[jj][t], xh[jj][t]);
-        *reinterpret_cast<float4*>(&srow[rl * D + e0]) = make_float4(dgt[0], dgt[1], dgt[2], dgt[3]);
-        *reinterpret_cast<float4*>(&srow[rl * D + e0 + 4]) = make_float4(dgt[4], dgt[5], dgt[6], dgt[7]);
-      }
-      if (gamma && e0 < D) {
-        float g[8];
-        load8<BF>(gamma, e0, g);
-#pragma unroll
-        for (int t = 0; t < 8; ++t) w[jj][t] = fmul(w[jj][t], g[t]);
-      }
-#pragma unroll
-      for (int t = 0; t < 8; ++t) pr[t] = fmul(w[jj][t], xh[jj][t]);
+      for (int t = 0; t < 8; ++t) pr[t] = fmul(w[a][t], xh[a][t]);
       const float t8 = tree8_full(pr);
-      const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
-      if (lane == jj) mine = leaf;
+      const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)warp * 256, 8, D);
+      if (lane == 0) leaf_sum[pass & 1][a][warp] = leaf;
     }
-    // tree over this warp's two leaf sums (lanes 0, 1), then over the four quarters of the row (a node whose first
-    // element lies beyond D does not exist and its left neighbour is carried up unchanged)
-    {
-      const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
-      const bool right_valid = (long long)(hw * 2 + 1) * 256 < D;
-      mine = right_valid ? fadd(mine, o) : ((lane & 1) ? o : mine);
-    }
-    if (lane == 0) hs[warp >> 2][hw] = mine;
     __syncthreads();
-    const float h01 = (D > 512) ? fadd(hs[warp >> 2][0], hs[warp >> 2][1]) : hs[warp >> 2][0];
-    const float h23 = (D > 1536) ? fadd(hs[warp >> 2][2], hs[warp >> 2][3]) : hs[warp >> 2][2];
-    const float tot = (D > 1024) ? fadd(h01, h23) : h01;
-    const float c = fmul(tot, invD);
-    if (live) {
 #pragma unroll
-      for (int jj = 0; jj < 2; ++jj) {
-        const int e0 = (hw * 2 + jj) * 256 + lane * 8;
-        if (e0 >= D) continue;
+    for (int a = 0; a < 2; ++a) {
+      const long long row = first + a;
+      float L[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) L[j] = leaf_sum[pass & 1][a][j];
+      const float c = fmul(reg_tree<8>(L, 0, 256, D), invD);   // the row's tree over its leaves (a leaf beyond D does not exist)
+      if (row < rows && have) {
         float o[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) o[t] = fmul(rs, fsub(w[jj][t], fmul(xh[jj][t], c)));
-        store8<BF>(dx, rb + e0, o);
+        for (int t = 0; t < 8; ++t) o[t] = fmul(rs[a], fsub(w[a][t], fmul(xh[a][t], c)));
+        store8<BF>(dx, (size_t)row * D + e0, o);
       }
     }
   }
-  if (DG) {   // the last pass's barrier has published all eight rows of products
-    for (int col = threadIdx.x; col < D; col += NT) {
-      float v[8];
-#pragma unroll
-      for (int r = 0; r < 8; ++r) v[r] = srow[r * D + col];
-      partial8[(size_t)blockIdx.x * D + col] = reg_tree<8>(v, r0, 1, rows);
-    }
+  if (DG && have) {
+    float* dst = partial8 + (size_t)blockIdx.x * D + e0;
+    *reinterpret_cast<float4*>(dst) = make_float4(node[0], node[1], node[2], node[3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(node[4], node[5], node[6], node[7]);
   }
 }
 // partial8 [nb8][D] (node = 8 rows) -> partial256 [nb256][D]: tree over 32 adjacent 8-row nodes per column; the CTA
@@ -581,18 +568,15 @@ extern "C" size_t det_rmsnorm_bwd_ws_bytes(int rows, int D) {
 template <bool BF>
 static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma, const float* rstd, int rows, int D,
                                float invD, void* dx, float* dgamma, float* ws, cudaStream_t st) {
-  constexpr int RP = RMS_RP;
   const int nb8 = (rows + 7) / 8, nb256 = (rows + 255) / 256;
   if (!dgamma) {
-    k_rmsnorm_bwd8<BF, false, RP><<<DET_L(nb8), RP * 128, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr, nullptr);
+    k_rmsnorm_bwd8<BF, false><<<DET_L(nb8), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, nullptr, nullptr);
     return DET_OK;
   }
-  static DevOnce once = {};
-  if (dev_ensure_smem(once, (const void*)k_rmsnorm_bwd8<BF, true, RP>, 8 * 2048 * 4) != DET_OK) return DET_ERR_CUDA;
   float* partial8 = ws;
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);
   int* tickets = reinterpret_cast<int*>(partial256 + align_up((size_t)nb256 * D, 64));   // one per block of 256 columns (<= 8)
-  k_rmsnorm_bwd8<BF, true, RP><<<DET_L(nb8), RP * 128, (size_t)8 * D * sizeof(float), st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8, tickets);
+  k_rmsnorm_bwd8<BF, true><<<DET_L(nb8), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8, tickets);
   dim3 g2((D + 255) / 256, nb256);
   k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256, nb256, tickets, dgamma);
   return DET_OK;
