@@ -114,6 +114,7 @@ __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict_
   const bool full = (D & 255) == 0;
   const long long r0 = (long long)blockIdx.x * 8;
   if (DG && blockIdx.x == 0 && (int)threadIdx.x < ((D + 255) >> 8)) tickets[threadIdx.x] = 0;   // for the kernel that follows
+  if (DG) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // its blocks may start coming in; they wait for this grid
   float pair0[8], node[8];                        // column tree: a pair of rows waiting for the next pair; rows 0 .. 3
 #pragma unroll
   for (int t = 0; t < 8; ++t) { pair0[t] = 0.0f; node[t] = 0.0f; }
@@ -194,6 +195,9 @@ __global__ void __launch_bounds__(256) k_colsum32(const float* __restrict__ part
   __shared__ int last_s;
   const int col = blockIdx.x * 256 + threadIdx.x;
   const int g = blockIdx.y;
+  // launched as a programmatic dependent of the kernel that writes partial8: its blocks may be resident before that
+  // kernel has drained; nothing of its results is read before this wait returns
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (col < D) {
     float s[32];
 #pragma unroll
@@ -577,8 +581,23 @@ static int rmsnorm_bwd8_launch(const void* dy, const void* x, const void* gamma,
   float* partial256 = ws + align_up((size_t)nb8 * D, 64);
   int* tickets = reinterpret_cast<int*>(partial256 + align_up((size_t)nb256 * D, 64));   // one per block of 256 columns (<= 8)
   k_rmsnorm_bwd8<BF, true><<<DET_L(nb8), 256, 0, st>>>(dy, x, gamma, rstd, rows, D, invD, dx, partial8, tickets);
-  dim3 g2((D + 255) / 256, nb256);
-  k_colsum32<<<DET_L(g2), 256, 0, st>>>(partial8, nb8, rows, D, partial256, nb256, tickets, dgamma);
+  // the second launch overlaps its start-up with the first kernel's tail (programmatic dependent launch); the kernel
+  // itself waits for the first grid to complete before it reads anything
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((D + 255) / 256, nb256);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  note_launch();
+  if (cudaLaunchKernelEx(&cfg, k_colsum32, (const float*)partial8, nb8, rows, D, partial256, nb256, tickets, dgamma) != cudaSuccess) {
+    cudaGetLastError();
+    return DET_ERR_CUDA;
+  }
   return DET_OK;
 }
 
