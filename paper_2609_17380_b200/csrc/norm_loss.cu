@@ -32,63 +32,73 @@ __device__ __forceinline__ void store8(void* p, size_t idx, const float v[8]) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// RMSNorm.  One warp per row.  Rows of at most 2048 elements (8 leaves) are loaded completely into
-// registers first (16 independent 128-bit loads per lane), reduced, normalised and stored; longer rows
-// use the two-pass variant that reads the row again.
+// RMSNorm.  Rows of at most 2048 elements (8 leaves) are held in registers between the sum of squares and
+// the output (k_rmsnorm_fwd8); longer rows use the two-pass variant that reads the row again.
 // ------------------------------------------------------------------------------------------------
+// A warp per LEAF (256 columns, 8 adjacent columns per lane), a CTA of 8 warps per block of 8 rows in two passes of four
+// rows: 16 values and 8 loads in flight per lane, four CTAs per SM; the leaf sums of a row meet in shared memory (one
+// barrier per pass) and every thread forms the row's tree over its leaves itself.
 template <bool BF>
-__global__ void __launch_bounds__(256) k_rmsnorm_fwd8(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
-                                                      int D, float eps, float invD, void* __restrict__ y,
-                                                      float* __restrict__ rstd, const float* __restrict__ s_q = nullptr,
-                                                      int8_t* __restrict__ qy = nullptr) {
+__global__ void __launch_bounds__(256, 4) k_rmsnorm_fwd8(const void* __restrict__ x, const void* __restrict__ gamma, int rows,
+                                                         int D, float eps, float invD, void* __restrict__ y,
+                                                         float* __restrict__ rstd, const float* __restrict__ s_q = nullptr,
+                                                         int8_t* __restrict__ qy = nullptr) {
+  __shared__ float leaf_sum[2][4][8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.x * 8 + warp;
-  if (row >= rows) return;
-  const size_t rb = (size_t)row * D;
-  const float inv_q = (BF && qy) ? fdiv(1.0f, s_q[0]) : 0.0f;
-  float xr[8][8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int e0 = j * 256 + lane * 8;
-    if (e0 < D) load8<BF>(x, rb + e0, xr[j]);
-    else {
-#pragma unroll
-      for (int t = 0; t < 8; ++t) xr[j][t] = 0.0f;
-    }
-  }
-  float mine = 0.0f;
+  const int e0 = warp * 256 + lane * 8;
+  const bool have = e0 < D;
   const bool full = (D & 255) == 0;
+  const long long r0 = (long long)blockIdx.x * 8;
+  const float inv_q = (BF && qy) ? fdiv(1.0f, s_q[0]) : 0.0f;
+#pragma unroll 1
+  for (int pass = 0; pass < 2; ++pass) {
+    float xr[4][8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    float sq[8];
+    for (int a = 0; a < 4; ++a) {
+      const long long row = r0 + 4 * pass + a;
+      if (row < rows && have) load8<BF>(x, (size_t)row * D + e0, xr[a]);
+      else {
 #pragma unroll
-    for (int t = 0; t < 8; ++t) sq[t] = fmul(xr[j][t], xr[j][t]);
-    const float t8 = tree8_full(sq);
-    const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)j * 256, 8, D);
-    if (lane == j) mine = leaf;
-  }
-  const float ss = warp_tree(mine, 0, 256, D);
-  const float rs = fdiv(1.0f, fsqrt(fadd(fmul(ss, invD), eps)));
-  if (lane == 0) rstd[row] = rs;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int e0 = j * 256 + lane * 8;
-    if (e0 >= D) continue;
-    float o[8];
-    if (gamma) {
-      float g[8];
-      load8<BF>(gamma, e0, g);
-#pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = fmul(fmul(xr[j][t], rs), g[t]);
-    } else {
-#pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = fmul(xr[j][t], rs);
+        for (int t = 0; t < 8; ++t) xr[a][t] = 0.0f;
+      }
     }
-    store8<BF>(y, rb + e0, o);
-    if (BF && qy) {   // the next linear's quantiser, applied to the bf16 values just stored
 #pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = bf2f(f2bf(o[t]));
-      *reinterpret_cast<uint2*>(qy + rb + e0) = quant8(o, inv_q);
+    for (int a = 0; a < 4; ++a) {
+      float sq[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) sq[t] = fmul(xr[a][t], xr[a][t]);
+      const float t8 = tree8_full(sq);
+      const float leaf = full ? warp_tree_full(t8) : warp_tree(t8, (long long)warp * 256, 8, D);
+      if (lane == 0) leaf_sum[pass][a][warp] = leaf;
+    }
+    __syncthreads();
+    float g[8];
+    if (gamma && have) load8<BF>(gamma, e0, g);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const long long row = r0 + 4 * pass + a;
+      float L[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) L[j] = leaf_sum[pass][a][j];
+      const float ss = reg_tree<8>(L, 0, 256, D);          // a leaf beyond D does not exist
+      const float rs = fdiv(1.0f, fsqrt(fadd(fmul(ss, invD), eps)));
+      if (row >= rows) continue;
+      if (threadIdx.x == a) rstd[row] = rs;
+      if (!have) continue;
+      float o[8];
+      if (gamma) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) o[t] = fmul(fmul(xr[a][t], rs), g[t]);
+      } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) o[t] = fmul(xr[a][t], rs);
+      }
+      store8<BF>(y, (size_t)row * D + e0, o);
+      if (BF && qy) {   // the next linear's quantiser, applied to the bf16 values just stored
+#pragma unroll
+        for (int t = 0; t < 8; ++t) o[t] = bf2f(f2bf(o[t]));
+        *reinterpret_cast<uint2*>(qy + (size_t)row * D + e0) = quant8(o, inv_q);
+      }
     }
   }
 }
