@@ -514,27 +514,45 @@ __global__ void k_xent_finish(const float* ce_sum, const float* z_sum, float inv
   loss_mean[0] = (z_weight != 0.0f) ? fadd(ce, fmul(z_weight, zm)) : ce;
 }
 
+// Each thread takes two groups of four adjacent logits of a row, 1024 columns apart (every access of a warp covers whole
+// lines).  The argument z - lse is at most 0 whenever lse is the row's own logsumexp, and then the exponential without the
+// overflow range applies (same bits); lse is an input, though, so a thread that sees a positive argument takes the
+// general form for its eight values.
 __global__ void __launch_bounds__(256) k_xent_bwd(float* __restrict__ logits, const int32_t* __restrict__ target,
                                                   const float* __restrict__ lse, int rows, int V, float z_weight, float scale) {
-  const int i = (blockIdx.x * 256 + threadIdx.x) * 4;
-  if (i >= V) return;
+  const int i0 = blockIdx.x * 2048 + threadIdx.x * 4;
+  if (i0 >= V) return;
+  const bool two = i0 + 1024 < V;
   for (int row = blockIdx.y; row < rows; row += gridDim.y) {
-  float* z = logits + (size_t)row * V;
-  const int t = target[row];
-  const bool ok = t >= 0 && t < V;
-  const float l = lse[row];
-  const float zc = fmul(fmul(2.0f, z_weight), l);
-  float4 a = *reinterpret_cast<float4*>(z + i);
-  float v[4] = {a.x, a.y, a.z, a.w};
+    float* z = logits + (size_t)row * V;
+    const int t = target[row];
+    const bool ok = t >= 0 && t < V;
+    const float l = lse[row];
+    const float zc = fmul(fmul(2.0f, z_weight), l);
+    const float4 a = *reinterpret_cast<float4*>(z + i0);
+    const float4 b = two ? *reinterpret_cast<float4*>(z + i0 + 1024) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float x[8] = {fsub(a.x, l), fsub(a.y, l), fsub(a.z, l), fsub(a.w, l), fsub(b.x, l), fsub(b.y, l), fsub(b.z, l), fsub(b.w, l)};
+    bool pos = false;
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    if (!ok) { v[k] = 0.0f; continue; }
-    float p = det_exp(fsub(v[k], l));
-    float d = fsub(p, (i + k == t) ? 1.0f : 0.0f);
-    if (z_weight != 0.0f) d = fadd(d, fmul(zc, p));
-    v[k] = fmul(d, scale);
-  }
-  *reinterpret_cast<float4*>(z + i) = make_float4(v[0], v[1], v[2], v[3]);
+    for (int k = 0; k < 8; ++k) pos |= x[k] > 0.0f;
+    float p[8];
+    if (!pos) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) p[k] = det_exp_le0(x[k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) p[k] = det_exp(x[k]);
+    }
+    float v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int col = i0 + (k >> 2) * 1024 + (k & 3);
+      float d = fsub(p[k], (col == t) ? 1.0f : 0.0f);
+      if (z_weight != 0.0f) d = fadd(d, fmul(zc, p[k]));
+      v[k] = ok ? fmul(d, scale) : 0.0f;
+    }
+    *reinterpret_cast<float4*>(z + i0) = make_float4(v[0], v[1], v[2], v[3]);
+    if (two) *reinterpret_cast<float4*>(z + i0 + 1024) = make_float4(v[4], v[5], v[6], v[7]);
   }
 }
 
@@ -676,7 +694,7 @@ extern "C" int det_xent_bwd(float* logits_inout, const int32_t* target, const fl
   if (!logits_inout || !target || !lse || rows <= 0 || V <= 0) return DET_ERR_ARG;
   if (V % 4) return DET_ERR_SHAPE;
   if (!aligned16(logits_inout)) return DET_ERR_ALIGN;
-  dim3 grid((V / 4 + 255) / 256, rows < 65535 ? rows : 65535);
+  dim3 grid((V + 2047) / 2048, rows < 65535 ? rows : 65535);
   k_xent_bwd<<<DET_L(grid), 256, 0, (cudaStream_t)stream>>>(logits_inout, target, lse, rows, V, z_weight, scale);
   DET_CHECK_LAUNCH();
   return DET_OK;

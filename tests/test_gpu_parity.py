@@ -293,6 +293,30 @@ def test_xent(det, rows, V, zw):
     assert_same_bits(host(dz), oracle.xent_bwd(z, t, olse, zw, 1.0 / 64), "dlogits")
 
 
+def test_xent_backward_with_a_foreign_logsumexp(det):
+    """det_xent_bwd takes lse as an input: with values below a row's own logsumexp some arguments z - lse are positive
+    (up to the overflow of exp), and the kernel must leave its shortcut for non-positive arguments; with values far above,
+    every probability underflows.  Both against the oracle, bit for bit, on a width with a ragged last block."""
+    rows, V = 24, 6 * 2048 + 1024 + 36
+    z = synth.normal_f32((rows, V), 2.0, seed=3, tid=70)
+    t = synth.randint(rows, V, seed=3, tid=71)
+    _, olse, _, _, _ = oracle.xent_fwd(z, t, 0.0)
+    lse = olse.copy()
+    lse[0::4] -= 3.0                       # some positive arguments
+    lse[1::4] -= 95.0                      # arguments up to the edge of the overflow range
+    lse[3::4] -= 110.0                     # exp overflows for the largest logits
+    lse[2::4] += 100.0                     # every probability flushes to 0
+    for zw in (0.0, 1e-4):
+        dz = dev(z)
+        det.det_xent_bwd(dz, dev(t), dev(lse), rows, V, zw, 0.5)
+        _sync()
+        got, want = host(dz), oracle.xent_bwd(z, t, lse, zw, 0.5)
+        assert np.array_equal(np.isnan(got), np.isnan(want))
+        fin = ~np.isnan(want)
+        assert_same_bits(got[fin], want[fin], "dlogits with a foreign lse")
+        assert np.all(want[2][np.arange(V) != t[2]] == 0) and not np.all(np.isfinite(want[3]))
+
+
 def test_xent_closed_forms_and_bad_target(det):
     import torch
     V = 50304
