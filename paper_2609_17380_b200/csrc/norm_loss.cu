@@ -112,12 +112,14 @@ __global__ void __launch_bounds__(256, 4) k_rmsnorm_fwd8(const void* __restrict_
 // (0.080 ms with the products staged through shared memory by warps that each owned a quarter row, 0.070 ms now;
 // 0.065-0.070 ms without the gain gradient, i.e. 0.9 of the copy bandwidth).  The row sums go through shared memory: one
 // value per leaf and row, one barrier per pass.
+// RPP rows per pass: 2 for f32 rows, 4 for bf16 rows (16 values and 64 bytes of loads in flight per lane and tensor either way).
 template <bool BF, bool DG>
 __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict__ dy, const void* __restrict__ x,
                                                         const void* __restrict__ gamma, const float* __restrict__ rstd,
                                                         int rows, int D, float invD, void* __restrict__ dx,
                                                         float* __restrict__ partial8, int* __restrict__ tickets) {
-  __shared__ float leaf_sum[2][2][8];
+  constexpr int RPP = BF ? 4 : 2, NPASS = 8 / RPP;
+  __shared__ float leaf_sum[2][RPP][8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int e0 = warp * 256 + lane * 8;
   const bool have = e0 < D;                       // this lane's 8 columns exist (D is a multiple of 8)
@@ -129,11 +131,11 @@ __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict_
 #pragma unroll
   for (int t = 0; t < 8; ++t) { pair0[t] = 0.0f; node[t] = 0.0f; }
 #pragma unroll 1
-  for (int pass = 0; pass < 4; ++pass) {
-    const long long first = r0 + 2 * pass;
-    float w[2][8], xh[2][8], rs[2];
+  for (int pass = 0; pass < NPASS; ++pass) {
+    const long long first = r0 + RPP * pass;
+    float w[RPP][8], xh[RPP][8], rs[RPP];
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < RPP; ++a) {
       const long long row = first + a;
       if (row < rows && have) {
         load8<BF>(dy, (size_t)row * D + e0, w[a]);
@@ -145,15 +147,24 @@ __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict_
       rs[a] = row < rows ? rstd[row] : 0.0f;
     }
 #pragma unroll
-    for (int t = 0; t < 8; ++t) { xh[0][t] = fmul(xh[0][t], rs[0]); xh[1][t] = fmul(xh[1][t], rs[1]); }
-    if (DG) {   // rows 2 pass, 2 pass + 1 -> pair; pairs 0, 1 and 2, 3 -> nodes of four rows; those two -> the node of eight
+    for (int a = 0; a < RPP; ++a)
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xh[a][t] = fmul(xh[a][t], rs[a]);
+    if (DG) {   // rows in pairs; pairs 0, 1 and 2, 3 -> nodes of four rows; those two -> the node of eight (a right node exists
+                // iff its first row does, else the left one is carried up unchanged)
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
         const float d0 = fmul(w[0][t], xh[0][t]), d1 = fmul(w[1][t], xh[1][t]);
-        const float pr2 = (first + 1 < rows) ? fadd(d0, d1) : d0;
-        if ((pass & 1) == 0) pair0[t] = pr2;
-        else {
-          const float four = (first < rows) ? fadd(pair0[t], pr2) : pair0[t];   // the right pair exists iff its first row does
+        const float pa = (first + 1 < rows) ? fadd(d0, d1) : d0;
+        if (RPP == 4) {
+          const float d2 = fmul(w[RPP - 2][t], xh[RPP - 2][t]), d3 = fmul(w[RPP - 1][t], xh[RPP - 1][t]);
+          const float pb = (first + 3 < rows) ? fadd(d2, d3) : d2;
+          const float four = (first + 2 < rows) ? fadd(pa, pb) : pa;
+          node[t] = (pass == 0) ? four : ((r0 + 4 < rows) ? fadd(node[t], four) : node[t]);
+        } else if ((pass & 1) == 0) {
+          pair0[t] = pa;
+        } else {
+          const float four = (first < rows) ? fadd(pair0[t], pa) : pair0[t];
           node[t] = (pass == 1) ? four : ((r0 + 4 < rows) ? fadd(node[t], four) : node[t]);
         }
       }
@@ -162,10 +173,12 @@ __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict_
       float g[8];
       load8<BF>(gamma, e0, g);
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { w[0][t] = fmul(w[0][t], g[t]); w[1][t] = fmul(w[1][t], g[t]); }
+      for (int a = 0; a < RPP; ++a)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) w[a][t] = fmul(w[a][t], g[t]);
     }
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < RPP; ++a) {
       float pr[8];
 #pragma unroll
       for (int t = 0; t < 8; ++t) pr[t] = fmul(w[a][t], xh[a][t]);
@@ -175,7 +188,7 @@ __global__ void __launch_bounds__(256, 3) k_rmsnorm_bwd8(const void* __restrict_
     }
     __syncthreads();
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < RPP; ++a) {
       const long long row = first + a;
       float L[8];
 #pragma unroll
